@@ -1,0 +1,169 @@
+/*
+ * less.h -- C ABI of the B200 (sm_100a) LESS hot path.
+ *
+ * LESS ("Get More with LESS", arxiv 2402.09398) pairs an eviction-based sparse
+ * KV cache (here H2O: heavy hitters + recent window) with a constant-size
+ * low-rank state (H, z) that absorbs every evicted key/value pair, so that
+ * evicted tokens still contribute to later attention outputs.
+ *
+ * One "instance" is one (batch, layer, head); instances are independent.
+ * Flat instance index: inst = (b * layers + layer) * heads + head, the order of
+ * every [B, L, H, ...] buffer below.
+ *
+ * Conventions
+ *   - Every function returns 0 (LESS_OK) or a negative LESS_ERR_* code; nothing
+ *     throws or aborts across this boundary.
+ *   - Pointers named in a signature as "device" are CUDA device pointers of the
+ *     current device, 16-byte aligned; "host" are ordinary host pointers.
+ *   - The library allocates no device memory: the caller provides one arena
+ *     (less_arena_bytes) that the context carves up and owns until destroy.
+ *   - Weight buffers and the arena are BORROWED for the context's lifetime.
+ *   - less_prefill / less_decode_step are asynchronous on the given stream;
+ *     their inputs must stay valid until the stream reaches the call.
+ *   - A context is not thread-safe.
+ *   - 16-bit inputs are IEEE fp16; accumulation, scores, H, z and outputs fp32.
+ */
+#ifndef LESS_B200_H
+#define LESS_B200_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct less_ctx less_ctx; /* opaque */
+
+enum {
+  LESS_OK = 0,
+  LESS_ERR_INVALID_CONFIG = -1,
+  LESS_ERR_NULL_POINTER = -2,
+  LESS_ERR_MISALIGNED = -3,
+  LESS_ERR_ARENA_TOO_SMALL = -4,
+  LESS_ERR_PROMPT_TOO_LONG = -5,
+  LESS_ERR_BAD_LAYER_RANGE = -6,
+  LESS_ERR_DEVICE_TIMEOUT = -7,
+  LESS_ERR_DEVICE_BOUNDS = -8,
+  LESS_ERR_CUDA = -9,
+  LESS_ERR_BAD_STATE = -10,
+  LESS_ERR_BUFFER_TOO_SMALL = -11
+};
+
+/* flags */
+enum {
+  /* H2O accumulates e^{s_i} / (sparse-only denominator) instead of Eq. 3's
+   * full denominator (the paper only says "accumulates attention
+   * probabilities", Section 2.1). */
+  LESS_SCORE_NORM_SPARSE = 1u,
+  /* Sparse policy alone (the paper's Baseline / Baseline+, Section 4):
+   * evicted pairs are dropped, H and z stay zero. */
+  LESS_NO_STATE = 2u
+};
+
+typedef struct less_config {
+  int32_t batch, layers, heads;
+  int32_t head_dim;           /* D, must be 128 */
+  int32_t rank;               /* R: 8 or 16 (Section 4: R = 8 by default) */
+  int32_t hidden;             /* R' = 512 (Section 3.2) */
+  int32_t heavy, recent;      /* slots per instance: heavy >= 0, recent >= 1 */
+  int32_t max_prompt;         /* longest prompt less_prefill will be given (>= 0) */
+  int32_t max_prefill_layers; /* layers scored together in less_prefill (>= 1): sizes the workspace */
+  uint32_t flags;
+} less_config;
+
+/* Per-head feature-map weights (Eq. 1, Eq. 2), device, fp16, row-major, no biases:
+ *   phi(q) = | gelu( gelu(q W_phi1) W_phi2 ) |
+ *   psi(k) = | c2 * gelu( c1 * gelu(k W_psi1) W_psi2 ) W_psi3 |                     */
+typedef struct less_weights {
+  const void* w_phi1;     /* [L, H, D, R'] */
+  const void* w_phi2;     /* [L, H, R', R] */
+  const void* w_psi1;     /* [L, H, D, R'] */
+  const void* w_psi2;     /* [L, H, R', R] */
+  const void* w_psi3;     /* [L, H, R, R]  */
+  const float* psi_scale; /* optional device [L, H, 2] = (c1, c2), the learnable
+                             scalars of Section 3.2; NULL means 1 */
+} less_weights;
+
+/* Bytes of device memory a context of this shape needs (0 if the config is
+ * invalid).  The arena must be 256-byte aligned. */
+size_t less_arena_bytes(const less_config* cfg);
+
+/* Validates the config, carves the arena, zeroes H, z (H_0 = 0, z_0 = 0,
+ * Section 2.2) and the slot counts.  Synchronous; runs on the legacy default
+ * stream.  *out is set only on success. */
+int less_create(const less_config* cfg, const less_weights* weights, void* arena_device,
+                size_t arena_bytes, less_ctx** out);
+
+/* Prompt phase for layers [layer_begin, layer_begin + layer_count) (Section 3.1:
+ * regular attention since H_0 = 0; the policy and the state act afterwards):
+ *   1. causal softmax rows of Q K^T / sqrt(D);
+ *   2. H2O accumulated scores acc_j = sum_{i >= j} P_ij (diagonal included);
+ *   3. keep the `recent` last positions plus the `heavy` others with the
+ *      largest (acc, position) keys; if prompt_len <= heavy + recent keep all;
+ *   4. kept rows go to slots in ascending position; every other row is
+ *      absorbed: H = sum psi(k_j)^T v_j, z = sum psi(k_j) (Eq. 4, Eq. 5 over D_1).
+ * Q, K, V: device fp16 [B, layer_count, H, prompt_len, D] contiguous.
+ * attn_out: device fp32, same shape, or NULL when the caller does not need the
+ * prompt's attention output.
+ * Every call of one generation must pass the same prompt_len; the first decode
+ * token then has absolute position prompt_len.  A layer that was never
+ * prefilled starts empty and fills without eviction until its slots are full.
+ * Calling it again for a layer resets that layer.  prompt_len == 0 only resets. */
+int less_prefill(less_ctx* ctx, int32_t layer_begin, int32_t layer_count, int32_t prompt_len,
+                 const void* Q, const void* K, const void* V, void* attn_out, void* cuda_stream);
+
+/* One generation step for every instance (Algorithm 1), at position t = tokens seen:
+ *   phi(q_t), psi(k_t) (Eq. 1, 2); scores over the live slots plus the new pair;
+ *   out = (phi(q) H + sum e^{s_i} v_i) / (phi(q) z^T + sum e^{s_i})        (Eq. 3)
+ *   acc_i += p_i, acc_new = p_new  with p = e^{s} / denominator            (H2O)
+ *   if the slots overflow: victim = argmin (acc, position) over entries with
+ *   position <= t - recent;  H += psi(k_vic)^T v_vic,  z += psi(k_vic)  (Eq. 4, 5);
+ *   the new pair overwrites the victim's slot in place (Section 3.2), else
+ *   it takes the next free slot.
+ * q, k, v: device fp16 [B, L, H, D].  out: device fp32 [B, L, H, D].
+ * evicted_pos: device int32 [B, L, H] or NULL; receives the evicted position
+ * or -1.  Advances the context's position by one. */
+int less_decode_step(less_ctx* ctx, const void* q, const void* k, const void* v, void* out,
+                     int32_t* evicted_pos, void* cuda_stream);
+
+/* Tokens seen so far (= absolute position of the next decode token). */
+int64_t less_position(const less_ctx* ctx);
+
+/* Bytes of one exported instance record:
+ *   int32 count, int32 position, int32 reserved[2],
+ *   int32 pos[N], float acc[N], fp16 K[N][D], fp16 V[N][D], float psi[N][R],
+ *   float H[R][D], float z[R]        with N = heavy + recent.
+ * Slots [count, N) are unspecified. */
+size_t less_state_record_bytes(const less_config* cfg);
+
+/* Copies the records of the listed instances (host int32 list) to / from a
+ * host buffer of n * less_state_record_bytes bytes.  Synchronises the stream
+ * before returning.  Algorithm 1's "save K, V, H, z"; also what teacher-forced
+ * tests use.  Import sets the context's position from record 0. */
+int less_export_state(less_ctx* ctx, const int32_t* inst_host, int32_t n, void* host_buf,
+                      size_t bytes, void* cuda_stream);
+int less_import_state(less_ctx* ctx, const int32_t* inst_host, int32_t n, const void* host_buf,
+                      size_t bytes, void* cuda_stream);
+
+/* phi(q_t) and psi(k_t) of the last decode step, all instances: host float
+ * [B*L*H, R] each (either may be NULL).  Synchronises the stream. */
+int less_read_feature_maps(less_ctx* ctx, float* phi_host, float* psi_host, void* cuda_stream);
+
+/* Reads the device status word (synchronises the stream): 0, or
+ * LESS_ERR_DEVICE_TIMEOUT / LESS_ERR_DEVICE_BOUNDS if a kernel gave up on a
+ * bounded wait or refused an out-of-range index. */
+int less_poll_status(less_ctx* ctx, void* cuda_stream);
+
+/* Kernels of this library launched through this context so far. */
+int64_t less_launch_count(const less_ctx* ctx);
+
+const char* less_strerror(int code);
+
+/* Releases the context; frees nothing the caller owns. */
+int less_destroy(less_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LESS_B200_H */

@@ -1,0 +1,340 @@
+// Decode-step kernels (Algorithm 1):
+//   feature_map_kernel  phi(q_t), psi(k_t)                         (Eq. 1, Eq. 2)
+//   decode_kernel       scores over the live slots, Eq. 3, H2O score update,
+//                       argmin eviction, Eq. 4 / Eq. 5, in-place slot overwrite
+#include "feature_mlp.cuh"
+
+namespace less {
+
+// --------------------------------------------------------------------------- //
+// Feature maps.  One CTA = one (layer, head), one map (phi or psi), up to FM_BR
+// batch rows.  The hidden activations never leave shared memory.
+// --------------------------------------------------------------------------- //
+struct FmParams {
+  const __half* x[2];     // q, k                       [B, L, Hd, D]
+  const __half* w1[2];    // W_phi1, W_psi1             [L, Hd, D, Rp]
+  const __half* w2[2];    // W_phi2, W_psi2             [L, Hd, Rp, R]
+  const __half* w3;       // W_psi3                     [L, Hd, R, R]
+  const float* psi_scale; // [L, Hd, 2] or null
+  float* out[2];          // phi_q, psi_k               [I, R]
+  int B, L, Hd, Rp;
+};
+
+template <int R>
+__global__ void __launch_bounds__(FM_THREADS) feature_map_kernel(FmParams p) {
+  extern __shared__ float fm_smem[];
+  float* xs = fm_smem;                         // [FM_BR][128]
+  float* hs = xs + FM_BR * kHeadDim;           // [FM_BR][Rp]
+  float* part = hs + FM_BR * p.Rp;             // [ndg][FM_BR][Rp]
+  const int lh = blockIdx.x;                   // layer * Hd + head
+  const int which = blockIdx.y;                // 0 phi(q), 1 psi(k)
+  const int b0 = blockIdx.z * FM_BR;
+  const int nb = min(FM_BR, p.B - b0);
+  const int tid = threadIdx.x;
+  const int layer = lh / p.Hd, head = lh % p.Hd;
+  for (int e = tid; e < FM_BR * kHeadDim; e += FM_THREADS) {
+    const int b = e / kHeadDim, d = e % kHeadDim;
+    float v = 0.f;
+    if (b < nb)
+      v = __half2float(p.x[which][(((size_t)(b0 + b) * p.L + layer) * p.Hd + head) * kHeadDim + d]);
+    xs[e] = v;
+  }
+  __syncthreads();
+  float c1 = 1.f, c2 = 1.f;
+  if (which == 1 && p.psi_scale) {
+    c1 = p.psi_scale[lh * 2];
+    c2 = p.psi_scale[lh * 2 + 1];
+  }
+  const float r = mlp_rows<R>(xs, part, hs, nb, p.w1[which] + (size_t)lh * kHeadDim * p.Rp,
+                              p.w2[which] + (size_t)lh * p.Rp * R, p.w3 + (size_t)lh * R * R, c1,
+                              c2, p.Rp, which == 1);
+  const int warp = tid >> 5, lane = tid & 31;
+  if (warp < nb && lane < R) {
+    const size_t inst = ((size_t)(b0 + warp) * p.L + layer) * p.Hd + head;
+    p.out[which][inst * R + lane] = r;
+  }
+}
+
+int launch_feature_maps(less_ctx* c, const void* q, const void* k, cudaStream_t s) {
+  const Dims& d = c->d;
+  FmParams p;
+  p.x[0] = (const __half*)q;
+  p.x[1] = (const __half*)k;
+  p.w1[0] = (const __half*)c->w.w_phi1;
+  p.w1[1] = (const __half*)c->w.w_psi1;
+  p.w2[0] = (const __half*)c->w.w_phi2;
+  p.w2[1] = (const __half*)c->w.w_psi2;
+  p.w3 = (const __half*)c->w.w_psi3;
+  p.psi_scale = c->w.psi_scale;
+  p.out[0] = c->a.phi_q;
+  p.out[1] = c->a.psi_k;
+  p.B = d.B; p.L = d.L; p.Hd = d.Hd; p.Rp = d.Rp;
+  const int ndg = FM_THREADS / (d.Rp / 8);
+  const size_t smem = (size_t)(FM_BR * kHeadDim + FM_BR * d.Rp + ndg * FM_BR * d.Rp) * 4;
+  dim3 grid(d.L * d.Hd, (d.flags & LESS_NO_STATE) ? 1 : 2, (d.B + FM_BR - 1) / FM_BR);
+  if (d.flags & LESS_NO_STATE) return LESS_OK;   // neither phi nor psi is used
+  if (d.R == 8) {
+    cudaFuncSetAttribute(feature_map_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    feature_map_kernel<8><<<grid, FM_THREADS, smem, s>>>(p);
+  } else {
+    cudaFuncSetAttribute(feature_map_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    feature_map_kernel<16><<<grid, FM_THREADS, smem, s>>>(p);
+  }
+  c->launches += 1;
+  return cudaGetLastError() == cudaSuccess ? LESS_OK : LESS_ERR_CUDA;
+}
+
+// --------------------------------------------------------------------------- //
+// Fused decode step: one CTA per instance.
+// --------------------------------------------------------------------------- //
+constexpr int DEC_THREADS = 128;
+constexpr int DEC_RG = DEC_THREADS / 16;   // row groups: 16 lanes x 16 B cover one 256-B row
+
+struct DecParams {
+  const __half* q; const __half* k; const __half* v;   // [I, D]
+  float* out;                                           // [I, D]
+  int32_t* evicted_pos;                                 // [I] or null
+  Arena a;
+  int N, Np, recent, t;
+  uint32_t flags;
+};
+
+__device__ __forceinline__ float block_max(float v, float* red) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  if (lane == 0) red[warp] = v;
+  __syncthreads();
+  float r = red[0];
+#pragma unroll
+  for (int w = 1; w < DEC_THREADS / 32; ++w) r = fmaxf(r, red[w]);
+  __syncthreads();
+  return r;
+}
+
+__device__ __forceinline__ float block_sum(float v, float* red) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  if (lane == 0) red[warp] = v;
+  __syncthreads();
+  float r = red[0];
+#pragma unroll
+  for (int w = 1; w < DEC_THREADS / 32; ++w) r += red[w];   // fixed order
+  __syncthreads();
+  return r;
+}
+
+template <int R>
+__global__ void __launch_bounds__(DEC_THREADS) decode_kernel(DecParams p) {
+  extern __shared__ float dsm[];
+  float* s_sc = dsm;                               // [Np + 4] scores, then e^{s - m}
+  float* s_red = s_sc + p.Np + 4;                  // [DEC_RG][128] partial numerators
+  __shared__ float s_small[DEC_THREADS / 32];
+  __shared__ unsigned long long s_key[DEC_THREADS / 32];
+  __shared__ int s_vic;
+
+  const int tid = threadIdx.x;
+  const size_t inst = blockIdx.x;
+  const int l16 = tid & 15, rg = tid >> 4;
+  const int N = p.N;
+  int n = p.a.count[inst];
+  if (n < 0 || n > N) {                            // refuse a corrupt count, touch nothing
+    if (tid == 0) set_status(p.a.status, kStatusBounds, 1);
+    return;
+  }
+  const bool use_state = !(p.flags & LESS_NO_STATE);
+  const float scale = 0.08838834764831845f;        // 1 / sqrt(128)
+
+  const __half* Kb = p.a.kslots + inst * (size_t)N * kHeadDim;
+  const __half* Vb = p.a.vslots + inst * (size_t)N * kHeadDim;
+
+  float qf[8];
+  half8_to_float(*reinterpret_cast<const uint4*>(p.q + inst * kHeadDim + l16 * 8), qf);
+
+  // ---- scores s_i = q . k_i / sqrt(D) over live slots, and the new pair ----
+#pragma unroll 4
+  for (int r0 = 0; r0 < n; r0 += DEC_RG) {         // r0 is block-uniform: shuffles stay converged
+    const int r = r0 + rg;
+    float dot = 0.f;
+    if (r < n) {
+      float kf[8];
+      half8_to_float(ldg_stream(Kb + (size_t)r * kHeadDim + l16 * 8), kf);
+#pragma unroll
+      for (int c = 0; c < 8; ++c) dot = fmaf(qf[c], kf[c], dot);
+    }
+#pragma unroll
+    for (int o = 8; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+    if (l16 == 0 && r < n) s_sc[r] = dot * scale;
+  }
+  const uint4 knew = *reinterpret_cast<const uint4*>(p.k + inst * kHeadDim + l16 * 8);
+  const uint4 vnew = *reinterpret_cast<const uint4*>(p.v + inst * kHeadDim + l16 * 8);
+  if (tid < 32) {                                  // whole warp 0 (both halves compute the same)
+    float kf[8];
+    half8_to_float(knew, kf);
+    float dot = 0.f;
+#pragma unroll
+    for (int c = 0; c < 8; ++c) dot = fmaf(qf[c], kf[c], dot);
+#pragma unroll
+    for (int o = 8; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+    if (tid == 0) s_sc[n] = dot * scale;
+  }
+  __syncthreads();
+
+  // ---- m = max, e_i = exp(s_i - m), l = sum e_i  (entries 0..n, n = new pair) ----
+  float m = -INFINITY;
+  for (int i = tid; i <= n; i += DEC_THREADS) m = fmaxf(m, s_sc[i]);
+  m = block_max(m, s_small);
+  m = fmaxf(m, -80.f);                             // keeps e^{-m} finite for the low-rank terms
+  float lsum = 0.f;
+  for (int i = tid; i <= n; i += DEC_THREADS) {
+    const float e = __expf(s_sc[i] - m);
+    s_sc[i] = e;
+    lsum += e;
+  }
+  lsum = block_sum(lsum, s_small);                 // also orders the s_sc writes
+
+  // ---- u = sum e_i v_i ----
+  float u[8];
+#pragma unroll
+  for (int c = 0; c < 8; ++c) u[c] = 0.f;
+#pragma unroll 4
+  for (int r = rg; r < n; r += DEC_RG) {
+    float vf[8];
+    half8_to_float(ldg_stream(Vb + (size_t)r * kHeadDim + l16 * 8), vf);
+    const float e = s_sc[r];
+#pragma unroll
+    for (int c = 0; c < 8; ++c) u[c] = fmaf(e, vf[c], u[c]);
+  }
+  if (rg == 0) {
+    float vf[8];
+    half8_to_float(vnew, vf);
+    const float e = s_sc[n];
+#pragma unroll
+    for (int c = 0; c < 8; ++c) u[c] = fmaf(e, vf[c], u[c]);
+  }
+#pragma unroll
+  for (int c = 0; c < 8; ++c) s_red[rg * kHeadDim + l16 * 8 + c] = u[c];
+  __syncthreads();
+
+  // ---- low-rank correction and the single normalisation (Eq. 3) ----
+  const int d = tid;                               // DEC_THREADS == D: one column per thread
+  float num = 0.f;
+#pragma unroll
+  for (int g = 0; g < DEC_RG; ++g) num += s_red[g * kHeadDim + d];
+  float den = lsum;
+  float phi[R];
+  float* Hb = p.a.H + inst * (size_t)R * kHeadDim;
+  float* zb = p.a.z + inst * R;
+  float hcol[R];
+  if (use_state) {
+    const float em = __expf(-m);
+    float lr = 0.f, lz = 0.f;
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+      phi[r] = p.a.phi_q[inst * R + r];
+      hcol[r] = Hb[r * kHeadDim + d];
+      lr = fmaf(phi[r], hcol[r], lr);
+      lz = fmaf(phi[r], zb[r], lz);
+    }
+    num = fmaf(em, lr, num);
+    den = fmaf(em, lz, den);
+  }
+  p.out[inst * kHeadDim + d] = num / den;
+
+  // ---- H2O: acc_i += p_i; candidates pos <= t - recent; argmin (acc, pos) ----
+  const float inv = 1.0f / ((p.flags & LESS_SCORE_NORM_SPARSE) ? lsum : den);
+  int32_t* posb = p.a.pos + inst * (size_t)p.Np;
+  float* accb = p.a.acc + inst * (size_t)p.Np;
+  const bool full = (n == N);
+  unsigned long long best = ~0ull;
+  for (int i = tid; i < n; i += DEC_THREADS) {
+    const float a = accb[i] + s_sc[i] * inv;
+    accb[i] = a;
+    if (full) {
+      const int ps = posb[i];
+      if (ps <= p.t - p.recent) {
+        const unsigned long long key =
+            ((unsigned long long)__float_as_uint(a) << 32) | (unsigned int)ps;
+        best = key < best ? key : best;
+      }
+    }
+  }
+  const float p_new = s_sc[n] * inv;
+  int slot = n;                                    // next free slot
+  if (full) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const unsigned long long other = __shfl_xor_sync(0xffffffffu, best, o);
+      best = other < best ? other : best;
+    }
+    if ((tid & 31) == 0) s_key[tid >> 5] = best;
+    if (tid == 0) s_vic = -1;
+    __syncthreads();
+    best = s_key[0];
+#pragma unroll
+    for (int w = 1; w < DEC_THREADS / 32; ++w) best = s_key[w] < best ? s_key[w] : best;
+    const int vpos = (int)(unsigned int)(best & 0xffffffffull);
+    for (int i = tid; i < n; i += DEC_THREADS)
+      if (posb[i] == vpos && best != ~0ull) s_vic = i;     // positions are unique
+    __syncthreads();
+    slot = s_vic;
+    if (slot < 0) {                                // cannot happen with recent >= 1; refuse
+      if (tid == 0) {
+        set_status(p.a.status, kStatusBounds, 2);
+        if (p.evicted_pos) p.evicted_pos[inst] = -1;
+      }
+      return;
+    }
+    if (tid == 0 && p.evicted_pos) p.evicted_pos[inst] = vpos;
+    // ---- Eq. 4 / Eq. 5: absorb the victim ----
+    if (use_state) {
+      const float vv = __half2float(Vb[(size_t)slot * kHeadDim + d]);
+      const float* psv = p.a.psic + (inst * (size_t)N + slot) * R;
+#pragma unroll
+      for (int r = 0; r < R; ++r) Hb[r * kHeadDim + d] = fmaf(psv[r], vv, hcol[r]);
+      if (tid < R) zb[tid] += psv[tid];
+    }
+    __syncthreads();                               // victim row fully read before overwrite
+  } else {
+    if (tid == 0) {
+      p.a.count[inst] = n + 1;
+      if (p.evicted_pos) p.evicted_pos[inst] = -1;
+    }
+  }
+  // ---- the new pair takes the slot in place ----
+  __half* Kw = p.a.kslots + (inst * (size_t)N + slot) * kHeadDim;
+  __half* Vw = p.a.vslots + (inst * (size_t)N + slot) * kHeadDim;
+  if (rg == 0) *reinterpret_cast<uint4*>(Kw + l16 * 8) = knew;
+  if (rg == 1) *reinterpret_cast<uint4*>(Vw + l16 * 8) = vnew;
+  if (tid == 32) { posb[slot] = p.t; accb[slot] = p_new; }
+  if (tid >= 64 && tid < 64 + R)
+    p.a.psic[(inst * (size_t)N + slot) * R + (tid - 64)] =
+        use_state ? p.a.psi_k[inst * R + (tid - 64)] : 0.f;
+}
+
+int launch_decode(less_ctx* c, const void* q, const void* k, const void* v, void* out,
+                  int32_t* evicted_pos, cudaStream_t s) {
+  const Dims& d = c->d;
+  DecParams p;
+  p.q = (const __half*)q; p.k = (const __half*)k; p.v = (const __half*)v;
+  p.out = (float*)out;
+  p.evicted_pos = evicted_pos;
+  p.a = c->a;
+  p.N = d.N; p.Np = d.Np; p.recent = d.recent; p.t = (int)c->t;
+  p.flags = d.flags;
+  const size_t smem = (size_t)(d.Np + 4 + DEC_RG * kHeadDim) * 4;
+  if (d.R == 8) {
+    if (smem > 48 * 1024)
+      cudaFuncSetAttribute(decode_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    decode_kernel<8><<<d.I, DEC_THREADS, smem, s>>>(p);
+  } else {
+    if (smem > 48 * 1024)
+      cudaFuncSetAttribute(decode_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    decode_kernel<16><<<d.I, DEC_THREADS, smem, s>>>(p);
+  }
+  c->launches += 1;
+  return cudaGetLastError() == cudaSuccess ? LESS_OK : LESS_ERR_CUDA;
+}
+
+}  // namespace less

@@ -1,0 +1,301 @@
+// Host side of the C ABI: config validation, arena carving, state export /
+// import, status polling.  No device memory is allocated here.
+#include <new>
+#include <string.h>
+
+#include "less_internal.cuh"
+
+using namespace less;
+
+namespace {
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+bool valid_config(const less_config* c) {
+  if (!c) return false;
+  if (c->batch < 1 || c->layers < 1 || c->heads < 1) return false;
+  if (c->head_dim != kHeadDim) return false;
+  if (c->rank != 8 && c->rank != 16) return false;
+  if (c->hidden < 64 || c->hidden > 1024 || (c->hidden & (c->hidden - 1))) return false;
+  if (c->heavy < 0 || c->recent < 1) return false;
+  if ((int64_t)c->heavy + c->recent > 65536) return false;
+  if (c->max_prompt < 0 || c->max_prompt > (1 << 20)) return false;
+  if (c->max_prefill_layers < 1 || c->max_prefill_layers > c->layers) return false;
+  if (c->flags & ~(uint32_t)(LESS_SCORE_NORM_SPARSE | LESS_NO_STATE)) return false;
+  int64_t inst = (int64_t)c->batch * c->layers * c->heads;
+  if (inst > (1 << 24)) return false;
+  return true;
+}
+
+Dims make_dims(const less_config* c) {
+  Dims d;
+  d.B = c->batch;
+  d.L = c->layers;
+  d.Hd = c->heads;
+  d.D = c->head_dim;
+  d.R = c->rank;
+  d.Rp = c->hidden;
+  d.heavy = c->heavy;
+  d.recent = c->recent;
+  d.N = c->heavy + c->recent;
+  d.Np = (d.N + 3) & ~3;
+  d.I = c->batch * c->layers * c->heads;
+  d.Sp = (c->max_prompt + 3) & ~3;
+  d.Lw = c->max_prefill_layers;
+  d.flags = c->flags;
+  return d;
+}
+
+// Walks the arena layout; with base == nullptr only the total size is computed.
+size_t carve(const Dims& d, char* base, Arena* a) {
+  size_t off = 0;
+  auto take = [&](size_t bytes) {
+    char* p = base ? base + off : nullptr;
+    off = align_up(off + bytes, 256);
+    return p;
+  };
+  const size_t I = d.I, N = d.N, Np = d.Np, D = d.D, R = d.R;
+  const size_t Iw = (size_t)d.B * d.Hd * d.Lw, Sp = d.Sp;
+  Arena t;
+  t.kslots = (__half*)take(I * N * D * sizeof(__half));
+  t.vslots = (__half*)take(I * N * D * sizeof(__half));
+  t.pos = (int32_t*)take(I * Np * 4);
+  t.acc = (float*)take(I * Np * 4);
+  t.psic = (float*)take(I * N * R * 4);
+  t.H = (float*)take(I * R * D * 4);
+  t.z = (float*)take(I * R * 4);
+  t.count = (int32_t*)take(I * 4);
+  t.phi_q = (float*)take(I * R * 4);
+  t.psi_k = (float*)take(I * R * 4);
+  t.status = (int32_t*)take(4 * 4);
+  t.ws_m = (float*)take(Iw * Sp * 4);
+  t.ws_invl = (float*)take(Iw * Sp * 4);
+  t.ws_acc = (float*)take(Iw * Sp * 4);
+  t.ws_slot = (int32_t*)take(Iw * Sp * 4);
+  t.ws_hpart = (float*)take(Iw * kMaxSplit * (R * D + R) * 4);
+  if (a) *a = t;
+  return off;
+}
+
+inline bool misaligned(const void* p) { return ((uintptr_t)p & 15) != 0; }
+
+struct RecordLayout {
+  size_t pos, acc, K, V, psi, H, z, total;
+};
+
+RecordLayout record_layout(const Dims& d) {
+  RecordLayout r;
+  size_t off = 16;
+  r.pos = off; off += (size_t)d.N * 4;
+  r.acc = off; off += (size_t)d.N * 4;
+  r.K = off; off += (size_t)d.N * d.D * 2;
+  r.V = off; off += (size_t)d.N * d.D * 2;
+  r.psi = off; off += (size_t)d.N * d.R * 4;
+  r.H = off; off += (size_t)d.R * d.D * 4;
+  r.z = off; off += (size_t)d.R * 4;
+  r.total = off;
+  return r;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t less_arena_bytes(const less_config* cfg) {
+  if (!valid_config(cfg)) return 0;
+  Dims d = make_dims(cfg);
+  return carve(d, nullptr, nullptr);
+}
+
+size_t less_state_record_bytes(const less_config* cfg) {
+  if (!valid_config(cfg)) return 0;
+  return record_layout(make_dims(cfg)).total;
+}
+
+int less_create(const less_config* cfg, const less_weights* w, void* arena, size_t arena_bytes,
+                less_ctx** out) {
+  if (!cfg || !w || !arena || !out) return LESS_ERR_NULL_POINTER;
+  if (!valid_config(cfg)) return LESS_ERR_INVALID_CONFIG;
+  if (!w->w_phi1 || !w->w_phi2 || !w->w_psi1 || !w->w_psi2 || !w->w_psi3)
+    return LESS_ERR_NULL_POINTER;
+  if (misaligned(w->w_phi1) || misaligned(w->w_phi2) || misaligned(w->w_psi1) ||
+      misaligned(w->w_psi2) || misaligned(w->w_psi3) || ((uintptr_t)arena & 255))
+    return LESS_ERR_MISALIGNED;
+  Dims d = make_dims(cfg);
+  size_t need = carve(d, nullptr, nullptr);
+  if (arena_bytes < need) return LESS_ERR_ARENA_TOO_SMALL;
+  less_ctx* c = new (std::nothrow) less_ctx;
+  if (!c) return LESS_ERR_CUDA;
+  c->cfg = *cfg;
+  c->w = *w;
+  c->d = d;
+  carve(d, (char*)arena, &c->a);
+  c->arena_base = arena;
+  c->arena_bytes = need;
+  c->t = 0;
+  c->launches = 0;
+  if (cudaGetDevice(&c->device) != cudaSuccess) { delete c; return LESS_ERR_CUDA; }
+  // H_0 = 0, z_0 = 0, no live slots, clean status
+  cudaError_t e = cudaMemset(c->a.H, 0, (size_t)d.I * d.R * d.D * 4);
+  if (e == cudaSuccess) e = cudaMemset(c->a.z, 0, (size_t)d.I * d.R * 4);
+  if (e == cudaSuccess) e = cudaMemset(c->a.count, 0, (size_t)d.I * 4);
+  if (e == cudaSuccess) e = cudaMemset(c->a.status, 0, 16);
+  if (e == cudaSuccess) e = cudaMemset(c->a.phi_q, 0, (size_t)d.I * d.R * 4);
+  if (e == cudaSuccess) e = cudaMemset(c->a.psi_k, 0, (size_t)d.I * d.R * 4);
+  if (e == cudaSuccess) e = cudaDeviceSynchronize();
+  if (e != cudaSuccess) { delete c; return LESS_ERR_CUDA; }
+  *out = c;
+  return LESS_OK;
+}
+
+int less_destroy(less_ctx* ctx) {
+  if (!ctx) return LESS_ERR_NULL_POINTER;
+  delete ctx;
+  return LESS_OK;
+}
+
+int64_t less_position(const less_ctx* ctx) { return ctx ? ctx->t : -1; }
+int64_t less_launch_count(const less_ctx* ctx) { return ctx ? ctx->launches : -1; }
+
+int less_prefill(less_ctx* c, int32_t layer_begin, int32_t layer_count, int32_t prompt_len,
+                 const void* Q, const void* K, const void* V, void* attn_out, void* stream) {
+  if (!c) return LESS_ERR_NULL_POINTER;
+  if (layer_begin < 0 || layer_count < 1 || layer_begin + layer_count > c->d.L)
+    return LESS_ERR_BAD_LAYER_RANGE;
+  if (prompt_len < 0) return LESS_ERR_INVALID_CONFIG;
+  if (prompt_len > c->cfg.max_prompt) return LESS_ERR_PROMPT_TOO_LONG;
+  if (prompt_len > 0) {
+    if (!Q || !K || !V) return LESS_ERR_NULL_POINTER;
+    if (misaligned(Q) || misaligned(K) || misaligned(V) || misaligned(attn_out))
+      return LESS_ERR_MISALIGNED;
+  }
+  cudaStream_t s = (cudaStream_t)stream;
+  for (int lj0 = 0; lj0 < layer_count; lj0 += c->d.Lw) {
+    int nl = layer_count - lj0 < c->d.Lw ? layer_count - lj0 : c->d.Lw;
+    int rc = launch_prefill_group(c, layer_begin + lj0, nl, lj0, layer_count, prompt_len, Q, K, V,
+                                  attn_out, s);
+    if (rc != LESS_OK) return rc;
+  }
+  c->t = prompt_len;
+  return LESS_OK;
+}
+
+int less_decode_step(less_ctx* c, const void* q, const void* k, const void* v, void* out,
+                     int32_t* evicted_pos, void* stream) {
+  if (!c || !q || !k || !v || !out) return LESS_ERR_NULL_POINTER;
+  if (misaligned(q) || misaligned(k) || misaligned(v) || misaligned(out))
+    return LESS_ERR_MISALIGNED;
+  if (c->t >= 0x7fffff00) return LESS_ERR_BAD_STATE;
+  cudaStream_t s = (cudaStream_t)stream;
+  int rc = launch_feature_maps(c, q, k, s);
+  if (rc != LESS_OK) return rc;
+  rc = launch_decode(c, q, k, v, out, evicted_pos, s);
+  if (rc != LESS_OK) return rc;
+  c->t += 1;
+  return LESS_OK;
+}
+
+static int copy_state(less_ctx* c, const int32_t* inst, int32_t n, void* host, size_t bytes,
+                      cudaStream_t s, bool to_host) {
+  if (!c || !inst || !host) return LESS_ERR_NULL_POINTER;
+  if (n < 0) return LESS_ERR_INVALID_CONFIG;
+  const Dims& d = c->d;
+  RecordLayout r = record_layout(d);
+  if (bytes < r.total * (size_t)n) return LESS_ERR_BUFFER_TOO_SMALL;
+  cudaMemcpyKind kind = to_host ? cudaMemcpyDeviceToHost : cudaMemcpyHostToDevice;
+  cudaError_t e = cudaSuccess;
+  auto cp = [&](void* hostp, void* devp, size_t nbytes) {
+    if (e != cudaSuccess || nbytes == 0) return;
+    e = to_host ? cudaMemcpyAsync(hostp, devp, nbytes, kind, s)
+                : cudaMemcpyAsync(devp, hostp, nbytes, kind, s);
+  };
+  for (int i = 0; i < n; ++i) {
+    int32_t ii = inst[i];
+    if (ii < 0 || ii >= d.I) return LESS_ERR_INVALID_CONFIG;
+    char* rec = (char*)host + r.total * (size_t)i;
+    size_t I = ii;
+    cp(rec, c->a.count + I, 4);
+    cp(rec + r.pos, c->a.pos + I * d.Np, (size_t)d.N * 4);
+    cp(rec + r.acc, c->a.acc + I * d.Np, (size_t)d.N * 4);
+    cp(rec + r.K, c->a.kslots + I * d.N * d.D, (size_t)d.N * d.D * 2);
+    cp(rec + r.V, c->a.vslots + I * d.N * d.D, (size_t)d.N * d.D * 2);
+    cp(rec + r.psi, c->a.psic + I * d.N * d.R, (size_t)d.N * d.R * 4);
+    cp(rec + r.H, c->a.H + I * d.R * d.D, (size_t)d.R * d.D * 4);
+    cp(rec + r.z, c->a.z + I * d.R, (size_t)d.R * 4);
+  }
+  if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+  if (e != cudaSuccess) return LESS_ERR_CUDA;
+  if (to_host) {
+    for (int i = 0; i < n; ++i) {
+      int32_t* hdr = (int32_t*)((char*)host + r.total * (size_t)i);
+      hdr[1] = (int32_t)c->t;
+      hdr[2] = hdr[3] = 0;
+    }
+  } else if (n > 0) {
+    c->t = ((const int32_t*)host)[1];
+  }
+  return LESS_OK;
+}
+
+int less_export_state(less_ctx* c, const int32_t* inst, int32_t n, void* host, size_t bytes,
+                      void* stream) {
+  return copy_state(c, inst, n, host, bytes, (cudaStream_t)stream, true);
+}
+
+int less_import_state(less_ctx* c, const int32_t* inst, int32_t n, const void* host, size_t bytes,
+                      void* stream) {
+  if (c && host) {
+    // the count field must be sane before it reaches a kernel
+    RecordLayout r = record_layout(c->d);
+    if (bytes < r.total * (size_t)(n < 0 ? 0 : n)) return LESS_ERR_BUFFER_TOO_SMALL;
+    for (int i = 0; i < n; ++i) {
+      int32_t cnt = *(const int32_t*)((const char*)host + r.total * (size_t)i);
+      if (cnt < 0 || cnt > c->d.N) return LESS_ERR_BAD_STATE;
+    }
+  }
+  return copy_state(c, inst, n, const_cast<void*>(host), bytes, (cudaStream_t)stream, false);
+}
+
+int less_read_feature_maps(less_ctx* c, float* phi_host, float* psi_host, void* stream) {
+  if (!c) return LESS_ERR_NULL_POINTER;
+  cudaStream_t s = (cudaStream_t)stream;
+  size_t bytes = (size_t)c->d.I * c->d.R * 4;
+  cudaError_t e = cudaSuccess;
+  if (phi_host) e = cudaMemcpyAsync(phi_host, c->a.phi_q, bytes, cudaMemcpyDeviceToHost, s);
+  if (e == cudaSuccess && psi_host)
+    e = cudaMemcpyAsync(psi_host, c->a.psi_k, bytes, cudaMemcpyDeviceToHost, s);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+  return e == cudaSuccess ? LESS_OK : LESS_ERR_CUDA;
+}
+
+int less_poll_status(less_ctx* c, void* stream) {
+  if (!c) return LESS_ERR_NULL_POINTER;
+  int32_t st[4] = {0, 0, 0, 0};
+  cudaStream_t s = (cudaStream_t)stream;
+  cudaError_t e = cudaMemcpyAsync(st, c->a.status, 16, cudaMemcpyDeviceToHost, s);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+  if (e != cudaSuccess) return LESS_ERR_CUDA;
+  if (st[0] == kStatusTimeout) return LESS_ERR_DEVICE_TIMEOUT;
+  if (st[0] == kStatusBounds) return LESS_ERR_DEVICE_BOUNDS;
+  return LESS_OK;
+}
+
+const char* less_strerror(int code) {
+  switch (code) {
+    case LESS_OK: return "ok";
+    case LESS_ERR_INVALID_CONFIG: return "invalid configuration or argument";
+    case LESS_ERR_NULL_POINTER: return "null pointer";
+    case LESS_ERR_MISALIGNED: return "pointer not 16-byte aligned (arena: 256)";
+    case LESS_ERR_ARENA_TOO_SMALL: return "arena too small";
+    case LESS_ERR_PROMPT_TOO_LONG: return "prompt longer than max_prompt";
+    case LESS_ERR_BAD_LAYER_RANGE: return "layer range outside the model";
+    case LESS_ERR_DEVICE_TIMEOUT: return "a device-side wait ran out";
+    case LESS_ERR_DEVICE_BOUNDS: return "a device-side index check failed";
+    case LESS_ERR_CUDA: return "CUDA runtime error";
+    case LESS_ERR_BAD_STATE: return "state record or context state not usable";
+    case LESS_ERR_BUFFER_TOO_SMALL: return "host buffer too small";
+    default: return "unknown error";
+  }
+}
+
+}  // extern "C"

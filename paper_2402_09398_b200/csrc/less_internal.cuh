@@ -1,0 +1,105 @@
+// Internal definitions shared by the translation units of the LESS library:
+// the context, the arena layout and small device helpers.
+#pragma once
+
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "less.h"
+
+namespace less {
+
+constexpr int kHeadDim = 128;       // D
+constexpr int kMaxSplit = 32;       // token splits of the prompt state build
+constexpr int kSplitTokens = 256;   // tokens per split (lower bound)
+
+// Device views of the arena.  All arrays are instance-major.
+struct Arena {
+  __half* kslots;    // [I][N][D]
+  __half* vslots;    // [I][N][D]
+  int32_t* pos;      // [I][Np]     absolute position of the token in a slot
+  float* acc;        // [I][Np]     H2O accumulated attention probability
+  float* psic;       // [I][N][R]   psi(k) of the token in a slot (evaluated at insertion)
+  float* H;          // [I][R][D]   Eq. 4
+  float* z;          // [I][R]      Eq. 5
+  int32_t* count;    // [I]         live slots
+  float* phi_q;      // [I][R]      phi(q_t) of the current step
+  float* psi_k;      // [I][R]      psi(k_t) of the current step
+  int32_t* status;   // [4]         device status word(s)
+  // prompt-phase workspace, for Iw = B * H * max_prefill_layers instances
+  float* ws_m;       // [Iw][Sp]    row max of causal scores
+  float* ws_invl;    // [Iw][Sp]    1 / row sum
+  float* ws_acc;     // [Iw][Sp]    column sums
+  int32_t* ws_slot;  // [Iw][Sp]    slot of a prompt token, -1 = evicted
+  float* ws_hpart;   // [Iw][kMaxSplit][R*D + R]  partial H, z per token split
+};
+
+struct Dims {
+  int32_t B, L, Hd, D, R, Rp;   // batch, layers, heads, head_dim, rank, hidden
+  int32_t heavy, recent, N, Np; // slots; Np = N rounded up to a multiple of 4
+  int32_t I;                    // instances
+  int32_t Sp;                   // max_prompt rounded up to a multiple of 4
+  int32_t Lw;                   // max_prefill_layers
+  uint32_t flags;
+};
+
+}  // namespace less
+
+struct less_ctx {
+  less_config cfg;
+  less_weights w;
+  less::Dims d;
+  less::Arena a;
+  void* arena_base;
+  size_t arena_bytes;
+  int64_t t;           // tokens seen
+  int64_t launches;    // kernels launched
+  int device;
+};
+
+namespace less {
+
+// status word values written by kernels (first writer wins)
+constexpr int kStatusOk = 0;
+constexpr int kStatusTimeout = 1;
+constexpr int kStatusBounds = 2;
+
+__device__ __forceinline__ void set_status(int32_t* status, int code, int where) {
+  if (atomicCAS(status, 0, code) == 0) status[1] = where;
+}
+
+__device__ __forceinline__ float gelu_erf(float x) {
+  // exact-form GELU, x * Phi(x)
+  return 0.5f * x * (1.0f + erff(x * 0.70710678118654752440f));
+}
+
+__device__ __forceinline__ void half8_to_float(const uint4& u, float* f) {
+  const __half2* h = reinterpret_cast<const __half2*>(&u);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    float2 p = __half22float2(h[i]);
+    f[2 * i] = p.x;
+    f[2 * i + 1] = p.y;
+  }
+}
+
+__device__ __forceinline__ uint4 ldg_stream(const void* p) {
+  // 128-bit streaming load: K/V slots are read once per step
+  return __ldcs(reinterpret_cast<const uint4*>(p));
+}
+
+__device__ __forceinline__ uint4 ldg_readonly(const void* p) {
+  // 128-bit load through the read-only path (weights: never written by a kernel)
+  return __ldg(reinterpret_cast<const uint4*>(p));
+}
+
+// launchers (host), defined in the kernel translation units
+int launch_feature_maps(less_ctx* c, const void* q, const void* k, cudaStream_t s);
+int launch_decode(less_ctx* c, const void* q, const void* k, const void* v, void* out,
+                  int32_t* evicted_pos, cudaStream_t s);
+int launch_prefill_group(less_ctx* c, int layer0, int nlayers, int lj0, int layer_count, int S,
+                         const void* Q, const void* K, const void* V, void* attn_out,
+                         cudaStream_t s);
+
+}  // namespace less

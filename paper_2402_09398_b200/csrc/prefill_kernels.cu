@@ -1,0 +1,475 @@
+// Prompt-phase kernels (Section 3.1: regular attention, then the policy once):
+//   rowstat_kernel   m_i, 1/l_i of causal row i of Q K^T / sqrt(D)
+//   colsum_kernel    acc_j = sum_{i >= j} exp(s_ij - m_i) / l_i      (H2O scores)
+//   attn_out_kernel  optional prompt attention output
+//   select_kernel    recent window + `heavy` largest (acc, pos) -> slot of every token
+//   build_kernel     psi(k_j) for every token; kept rows -> slots, evicted rows ->
+//                    partial H, z (Eq. 4, Eq. 5 summed over D_1)
+//   finalize_kernel  fixed-order sum of the partials
+#include "feature_mlp.cuh"
+
+namespace less {
+
+struct PfParams {
+  const __half* Q; const __half* K; const __half* V;   // [B, layer_count, Hd, S, D]
+  float* attn_out;                                      // same shape or null
+  Arena a;
+  const __half* w_psi1; const __half* w_psi2; const __half* w_psi3;
+  const float* psi_scale;
+  int S, Sp;                 // prompt length, workspace row stride
+  int layer0, nl;            // first model layer of this group, layers in the group
+  int lj0, layer_count;      // first input layer of this group, layers in the input
+  int B, L, Hd, N, Np, heavy, recent, Rp;
+  int nsplit, split_tokens;
+  uint32_t flags;
+};
+
+struct InstMap {
+  size_t in_row0;   // first row (of S) of this instance in Q/K/V, in rows of D
+  size_t inst;      // global instance
+  int lh;           // layer * Hd + head
+};
+
+__device__ __forceinline__ InstMap map_instance(const PfParams& p, int g) {
+  const int h = g % p.Hd;
+  const int lj = (g / p.Hd) % p.nl;
+  const int b = g / (p.Hd * p.nl);
+  InstMap m;
+  m.in_row0 = (((size_t)b * p.layer_count + p.lj0 + lj) * p.Hd + h) * (size_t)p.S;
+  m.inst = ((size_t)b * p.L + p.layer0 + lj) * p.Hd + h;
+  m.lh = (p.layer0 + lj) * p.Hd + h;
+  return m;
+}
+
+constexpr int PF_TILE = 128;   // rows (or columns) per CTA, one per thread
+constexpr int PF_KT = 32;      // rows of the other operand staged per iteration
+constexpr float kScale = 0.08838834764831845f;   // 1 / sqrt(128)
+
+__device__ __forceinline__ float dot128(const float* x, const __half* row) {
+  float s = 0.f;
+#pragma unroll
+  for (int c8 = 0; c8 < 16; ++c8) {
+    float f[8];
+    half8_to_float(*reinterpret_cast<const uint4*>(row + c8 * 8), f);
+#pragma unroll
+    for (int c = 0; c < 8; ++c) s = fmaf(x[c8 * 8 + c], f[c], s);
+  }
+  return s;
+}
+
+__device__ __forceinline__ void load_row128(float* x, const __half* row) {
+#pragma unroll
+  for (int c8 = 0; c8 < 16; ++c8)
+    half8_to_float(__ldg(reinterpret_cast<const uint4*>(row + c8 * 8)), x + c8 * 8);
+}
+
+// ---- P1: row statistics -------------------------------------------------- //
+__global__ void __launch_bounds__(PF_TILE) rowstat_kernel(PfParams p) {
+  __shared__ __align__(16) __half ks[PF_KT][kHeadDim];
+  const int g = blockIdx.y, i0 = blockIdx.x * PF_TILE, tid = threadIdx.x;
+  const InstMap im = map_instance(p, g);
+  const int i = i0 + tid;
+  const bool live = i < p.S;
+  float q[kHeadDim];
+  if (live) load_row128(q, p.Q + (im.in_row0 + i) * kHeadDim);
+  else {
+#pragma unroll
+    for (int c = 0; c < kHeadDim; ++c) q[c] = 0.f;
+  }
+  float m = -INFINITY, l = 0.f;
+  const int jend = min(p.S, i0 + PF_TILE);
+  for (int j0 = 0; j0 < jend; j0 += PF_KT) {
+    for (int e = tid; e < PF_KT * 16; e += PF_TILE) {
+      const int r = e >> 4, c = e & 15;
+      uint4 v = make_uint4(0, 0, 0, 0);
+      if (j0 + r < p.S) v = __ldg(reinterpret_cast<const uint4*>(p.K + (im.in_row0 + j0 + r) * kHeadDim) + c);
+      reinterpret_cast<uint4*>(&ks[r][0])[c] = v;
+    }
+    __syncthreads();
+    if (live) {
+      const int jmax = min(PF_KT, i - j0 + 1);
+      for (int jj = 0; jj < jmax; ++jj) {
+        const float s = dot128(q, &ks[jj][0]) * kScale;
+        if (s > m) { l = l * __expf(m - s) + 1.f; m = s; }
+        else l += __expf(s - m);
+      }
+    }
+    __syncthreads();
+  }
+  if (live) {
+    p.a.ws_m[(size_t)g * p.Sp + i] = m;
+    p.a.ws_invl[(size_t)g * p.Sp + i] = 1.0f / l;
+  }
+}
+
+// ---- P2: column sums ------------------------------------------------------ //
+__global__ void __launch_bounds__(PF_TILE) colsum_kernel(PfParams p) {
+  __shared__ __align__(16) __half qs[PF_KT][kHeadDim];
+  __shared__ float ms[PF_KT], ls[PF_KT];
+  const int g = blockIdx.y, j0 = blockIdx.x * PF_TILE, tid = threadIdx.x;
+  const InstMap im = map_instance(p, g);
+  const int j = j0 + tid;
+  const bool live = j < p.S;
+  float k[kHeadDim];
+  if (live) load_row128(k, p.K + (im.in_row0 + j) * kHeadDim);
+  else {
+#pragma unroll
+    for (int c = 0; c < kHeadDim; ++c) k[c] = 0.f;
+  }
+  float acc = 0.f;
+  for (int i0 = j0; i0 < p.S; i0 += PF_KT) {       // j0 is a multiple of PF_KT
+    for (int e = tid; e < PF_KT * 16; e += PF_TILE) {
+      const int r = e >> 4, c = e & 15;
+      uint4 v = make_uint4(0, 0, 0, 0);
+      if (i0 + r < p.S) v = __ldg(reinterpret_cast<const uint4*>(p.Q + (im.in_row0 + i0 + r) * kHeadDim) + c);
+      reinterpret_cast<uint4*>(&qs[r][0])[c] = v;
+    }
+    if (tid < PF_KT) {
+      const bool ok = i0 + tid < p.S;
+      ms[tid] = ok ? p.a.ws_m[(size_t)g * p.Sp + i0 + tid] : 0.f;
+      ls[tid] = ok ? p.a.ws_invl[(size_t)g * p.Sp + i0 + tid] : 0.f;
+    }
+    __syncthreads();
+    if (live) {
+      const int iimax = min(PF_KT, p.S - i0);
+      for (int ii = max(0, j - i0); ii < iimax; ++ii) {
+        const float s = dot128(k, &qs[ii][0]) * kScale;
+        acc += __expf(s - ms[ii]) * ls[ii];
+      }
+    }
+    __syncthreads();
+  }
+  if (live) p.a.ws_acc[(size_t)g * p.Sp + j] = acc;
+}
+
+// ---- optional prompt attention output ------------------------------------- //
+constexpr int AO_ROWS = 8;
+__global__ void __launch_bounds__(PF_TILE) attn_out_kernel(PfParams p) {
+  __shared__ float qs[AO_ROWS][kHeadDim];
+  __shared__ __align__(16) __half ks[PF_KT][kHeadDim];
+  __shared__ __align__(16) __half vs[PF_KT][kHeadDim];
+  __shared__ float ps[AO_ROWS][PF_KT];
+  const int g = blockIdx.y, i0 = blockIdx.x * AO_ROWS, tid = threadIdx.x;
+  const InstMap im = map_instance(p, g);
+  for (int e = tid; e < AO_ROWS * kHeadDim; e += PF_TILE) {
+    const int r = e / kHeadDim, c = e % kHeadDim;
+    qs[r][c] = (i0 + r < p.S) ? __half2float(p.Q[(im.in_row0 + i0 + r) * kHeadDim + c]) : 0.f;
+  }
+  float o[AO_ROWS];
+#pragma unroll
+  for (int r = 0; r < AO_ROWS; ++r) o[r] = 0.f;
+  const int jend = min(p.S, i0 + AO_ROWS);
+  for (int j0 = 0; j0 < jend; j0 += PF_KT) {
+    __syncthreads();
+    for (int e = tid; e < PF_KT * 16; e += PF_TILE) {
+      const int r = e >> 4, c = e & 15;
+      uint4 kv = make_uint4(0, 0, 0, 0), vv = kv;
+      if (j0 + r < p.S) {
+        kv = __ldg(reinterpret_cast<const uint4*>(p.K + (im.in_row0 + j0 + r) * kHeadDim) + c);
+        vv = __ldg(reinterpret_cast<const uint4*>(p.V + (im.in_row0 + j0 + r) * kHeadDim) + c);
+      }
+      reinterpret_cast<uint4*>(&ks[r][0])[c] = kv;
+      reinterpret_cast<uint4*>(&vs[r][0])[c] = vv;
+    }
+    __syncthreads();
+    for (int e = tid; e < AO_ROWS * PF_KT; e += PF_TILE) {
+      const int r = e / PF_KT, jj = e % PF_KT;
+      const int i = i0 + r, j = j0 + jj;
+      float pr = 0.f;
+      if (i < p.S && j <= i) {
+        const float s = dot128(&qs[r][0], &ks[jj][0]) * kScale;
+        pr = __expf(s - p.a.ws_m[(size_t)g * p.Sp + i]) * p.a.ws_invl[(size_t)g * p.Sp + i];
+      }
+      ps[r][jj] = pr;
+    }
+    __syncthreads();
+    for (int jj = 0; jj < PF_KT; ++jj) {
+      const float vv = __half2float(vs[jj][tid]);
+#pragma unroll
+      for (int r = 0; r < AO_ROWS; ++r) o[r] = fmaf(ps[r][jj], vv, o[r]);
+    }
+  }
+#pragma unroll
+  for (int r = 0; r < AO_ROWS; ++r)
+    if (i0 + r < p.S) p.attn_out[(im.in_row0 + i0 + r) * kHeadDim + tid] = o[r];
+}
+
+// ---- P3: selection --------------------------------------------------------- //
+constexpr int SEL_THREADS = 1024;
+
+// exclusive block scan of one int per thread; returns the exclusive prefix and the total
+__device__ __forceinline__ int block_exscan(int v, int* warp_sums, int* total) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  int inc = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int t = __shfl_up_sync(0xffffffffu, inc, o);
+    if (lane >= o) inc += t;
+  }
+  if (lane == 31) warp_sums[warp] = inc;
+  __syncthreads();
+  if (warp == 0) {
+    int w = warp_sums[lane];
+    int winc = w;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int t = __shfl_up_sync(0xffffffffu, winc, o);
+      if (lane >= o) winc += t;
+    }
+    warp_sums[lane] = winc - w;            // exclusive
+    if (lane == 31) warp_sums[32] = winc;  // total
+  }
+  __syncthreads();
+  const int ex = inc - v + warp_sums[warp];
+  *total = warp_sums[32];
+  __syncthreads();
+  return ex;
+}
+
+__global__ void __launch_bounds__(SEL_THREADS) select_kernel(PfParams p) {
+  __shared__ int hist[256];
+  __shared__ int wsum[33];
+  __shared__ unsigned int s_prefix;
+  __shared__ int s_need;
+  const int g = blockIdx.x, tid = threadIdx.x;
+  const InstMap im = map_instance(p, g);
+  const float* acc = p.a.ws_acc + (size_t)g * p.Sp;
+  int32_t* slot_of = p.a.ws_slot + (size_t)g * p.Sp;
+  const int S = p.S, N = p.N;
+  if (tid == 0) p.a.count[im.inst] = min(S, N);
+  if (S <= N) {
+    for (int j = tid; j < S; j += SEL_THREADS) slot_of[j] = j;
+    return;
+  }
+  const int C = S - p.recent;                    // candidates: positions [0, C)
+  unsigned int thr = 0xffffffffu;                // threshold bit pattern (acc >= 0: monotone)
+  int need = 0;                                  // how many of the == threshold to keep
+  if (p.heavy > 0) {
+    // radix select: the heavy-th largest accumulated score among the candidates
+    if (tid == 0) { s_prefix = 0; s_need = p.heavy; }
+    for (int pass = 0; pass < 4; ++pass) {
+      const int shift = 24 - 8 * pass;
+      if (tid < 256) hist[tid] = 0;
+      __syncthreads();
+      const unsigned int prefix = s_prefix;
+      const unsigned int himask = pass == 0 ? 0u : (0xffffffffu << (shift + 8));
+      for (int j = tid; j < C; j += SEL_THREADS) {
+        const unsigned int b = __float_as_uint(acc[j]);
+        if ((b & himask) == prefix) atomicAdd(&hist[(b >> shift) & 255], 1);
+      }
+      __syncthreads();
+      if (tid == 0) {
+        int k = s_need, bin = 255;
+        for (; bin > 0; --bin) {
+          if (hist[bin] >= k) break;
+          k -= hist[bin];
+        }
+        s_prefix = prefix | ((unsigned int)bin << shift);
+        s_need = k;
+      }
+      __syncthreads();
+    }
+    thr = s_prefix;
+    need = s_need;
+  }
+  // ties at the threshold: the lowest positions go first (key (acc, pos) ascending),
+  // so the `need` HIGHEST positions among the equals stay.
+  const int per = (S + SEL_THREADS - 1) / SEL_THREADS;
+  const int jb = tid * per, je = min(S, jb + per);
+  int eq = 0;
+  for (int j = jb; j < je; ++j) eq += (j < C && __float_as_uint(acc[j]) == thr) ? 1 : 0;
+  int eq_total;
+  int eq_before = block_exscan(eq, wsum, &eq_total);
+  const int drop_eq = eq_total - need;           // equals with fewer than this many below them are evicted
+  int kept = 0;
+  for (int j = jb; j < je; ++j) {
+    bool k;
+    if (j >= C) k = true;
+    else {
+      const unsigned int b = __float_as_uint(acc[j]);
+      if (b == thr) { k = eq_before >= drop_eq; ++eq_before; }
+      else k = p.heavy > 0 && b > thr;
+    }
+    kept += k ? 1 : 0;
+  }
+  int kept_total;
+  int slot = block_exscan(kept, wsum, &kept_total);
+  // second walk assigns slots in ascending position
+  eq_before = 0;
+  {
+    // recompute this thread's exclusive count of equals (block_exscan result was consumed)
+    int dummy;
+    eq_before = block_exscan(eq, wsum, &dummy);
+  }
+  for (int j = jb; j < je; ++j) {
+    bool k;
+    if (j >= C) k = true;
+    else {
+      const unsigned int b = __float_as_uint(acc[j]);
+      if (b == thr) { k = eq_before >= drop_eq; ++eq_before; }
+      else k = p.heavy > 0 && b > thr;
+    }
+    slot_of[j] = k ? slot++ : -1;
+  }
+  if (tid == 0 && kept_total != N) set_status(p.a.status, kStatusBounds, 3);
+}
+
+// ---- P4-P6: gather kept rows, psi for every row, partial H and z ----------- //
+template <int R>
+__global__ void __launch_bounds__(FM_THREADS) build_kernel(PfParams p) {
+  extern __shared__ float bsm[];
+  float* xs = bsm;                              // [FM_BR][128]
+  float* hs = xs + FM_BR * kHeadDim;
+  float* part = hs + FM_BR * p.Rp;
+  __shared__ float psis[FM_BR][R];
+  const int split = blockIdx.x, g = blockIdx.y, tid = threadIdx.x;
+  const InstMap im = map_instance(p, g);
+  const bool use_state = !(p.flags & LESS_NO_STATE);
+  const int jbeg = split * p.split_tokens, jend = min(p.S, jbeg + p.split_tokens);
+  const int32_t* slot_of = p.a.ws_slot + (size_t)g * p.Sp;
+  const float* acc = p.a.ws_acc + (size_t)g * p.Sp;
+  float c1 = 1.f, c2 = 1.f;
+  if (p.psi_scale) { c1 = p.psi_scale[im.lh * 2]; c2 = p.psi_scale[im.lh * 2 + 1]; }
+  const __half* w1 = p.w_psi1 + (size_t)im.lh * kHeadDim * p.Rp;
+  const __half* w2 = p.w_psi2 + (size_t)im.lh * p.Rp * R;
+  const __half* w3 = p.w_psi3 + (size_t)im.lh * R * R;
+  float hacc[R];
+#pragma unroll
+  for (int r = 0; r < R; ++r) hacc[r] = 0.f;
+  float zacc = 0.f;
+  for (int j0 = jbeg; j0 < jend; j0 += FM_BR) {
+    const int nb = min(FM_BR, jend - j0);
+    if (use_state) {
+      for (int e = tid; e < FM_BR * kHeadDim; e += FM_THREADS) {
+        const int b = e / kHeadDim, d = e % kHeadDim;
+        xs[e] = b < nb ? __half2float(p.K[(im.in_row0 + j0 + b) * kHeadDim + d]) : 0.f;
+      }
+      __syncthreads();
+      const float r = mlp_rows<R>(xs, part, hs, nb, w1, w2, w3, c1, c2, p.Rp, true);
+      const int warp = tid >> 5, lane = tid & 31;
+      if (warp < FM_BR && lane < R) psis[warp][lane] = warp < nb ? r : 0.f;
+      __syncthreads();
+    }
+    for (int b = 0; b < nb; ++b) {
+      const int j = j0 + b;
+      const int sl = slot_of[j];
+      if (sl >= 0) {
+        if (sl >= p.N) {
+          if (tid == 0) set_status(p.a.status, kStatusBounds, 4);
+          continue;
+        }
+        const size_t dst = (im.inst * (size_t)p.N + sl) * kHeadDim;
+        if (tid < 16)
+          reinterpret_cast<uint4*>(p.a.kslots + dst)[tid] =
+              __ldg(reinterpret_cast<const uint4*>(p.K + (im.in_row0 + j) * kHeadDim) + tid);
+        else if (tid < 32)
+          reinterpret_cast<uint4*>(p.a.vslots + dst)[tid - 16] =
+              __ldg(reinterpret_cast<const uint4*>(p.V + (im.in_row0 + j) * kHeadDim) + (tid - 16));
+        else if (tid == 32) {
+          p.a.pos[im.inst * (size_t)p.Np + sl] = j;
+          p.a.acc[im.inst * (size_t)p.Np + sl] = acc[j];
+        } else if (tid >= 64 && tid < 64 + R)
+          p.a.psic[(im.inst * (size_t)p.N + sl) * R + (tid - 64)] = use_state ? psis[b][tid - 64] : 0.f;
+      } else if (use_state) {
+        if (tid < kHeadDim) {
+          const float vv = __half2float(p.V[(im.in_row0 + j) * kHeadDim + tid]);
+#pragma unroll
+          for (int r = 0; r < R; ++r) hacc[r] = fmaf(psis[b][r], vv, hacc[r]);
+        } else if (tid < kHeadDim + R) {
+          zacc += psis[b][tid - kHeadDim];
+        }
+      }
+    }
+    __syncthreads();
+  }
+  float* hp = p.a.ws_hpart + ((size_t)g * kMaxSplit + split) * (R * kHeadDim + R);
+  if (tid < kHeadDim) {
+#pragma unroll
+    for (int r = 0; r < R; ++r) hp[r * kHeadDim + tid] = hacc[r];
+  } else if (tid < kHeadDim + R) {
+    hp[R * kHeadDim + (tid - kHeadDim)] = zacc;
+  }
+}
+
+template <int R>
+__global__ void __launch_bounds__(kHeadDim) finalize_kernel(PfParams p) {
+  const int g = blockIdx.x, tid = threadIdx.x;
+  const InstMap im = map_instance(p, g);
+  const bool use_state = !(p.flags & LESS_NO_STATE);
+  const float* hp = p.a.ws_hpart + (size_t)g * kMaxSplit * (R * kHeadDim + R);
+  const int ns = use_state ? p.nsplit : 0;
+#pragma unroll
+  for (int r = 0; r < R; ++r) {
+    float s = 0.f;
+    for (int sp = 0; sp < ns; ++sp) s += hp[(size_t)sp * (R * kHeadDim + R) + r * kHeadDim + tid];
+    p.a.H[(im.inst * R + r) * kHeadDim + tid] = s;
+  }
+  if (tid < R) {
+    float s = 0.f;
+    for (int sp = 0; sp < ns; ++sp) s += hp[(size_t)sp * (R * kHeadDim + R) + R * kHeadDim + tid];
+    p.a.z[im.inst * R + tid] = s;
+  }
+}
+
+int launch_prefill_group(less_ctx* c, int layer0, int nl, int lj0, int layer_count, int S,
+                         const void* Q, const void* K, const void* V, void* attn_out,
+                         cudaStream_t s) {
+  const Dims& d = c->d;
+  PfParams p;
+  p.Q = (const __half*)Q; p.K = (const __half*)K; p.V = (const __half*)V;
+  p.attn_out = (float*)attn_out;
+  p.a = c->a;
+  p.w_psi1 = (const __half*)c->w.w_psi1;
+  p.w_psi2 = (const __half*)c->w.w_psi2;
+  p.w_psi3 = (const __half*)c->w.w_psi3;
+  p.psi_scale = c->w.psi_scale;
+  p.S = S; p.Sp = d.Sp;
+  p.layer0 = layer0; p.nl = nl; p.lj0 = lj0; p.layer_count = layer_count;
+  p.B = d.B; p.L = d.L; p.Hd = d.Hd; p.N = d.N; p.Np = d.Np;
+  p.heavy = d.heavy; p.recent = d.recent; p.Rp = d.Rp;
+  p.flags = d.flags;
+  int nsplit = 0, split_tokens = kSplitTokens;
+  if (S > 0) {
+    nsplit = (S + kSplitTokens - 1) / kSplitTokens;
+    if (nsplit > kMaxSplit) {
+      nsplit = kMaxSplit;
+      split_tokens = (S + kMaxSplit - 1) / kMaxSplit;
+      split_tokens = (split_tokens + FM_BR - 1) / FM_BR * FM_BR;
+      nsplit = (S + split_tokens - 1) / split_tokens;
+    }
+  }
+  p.nsplit = nsplit; p.split_tokens = split_tokens;
+  const int G = d.B * nl * d.Hd;
+  if (S > 0) {
+    const int tiles = (S + PF_TILE - 1) / PF_TILE;
+    rowstat_kernel<<<dim3(tiles, G), PF_TILE, 0, s>>>(p);
+    colsum_kernel<<<dim3(tiles, G), PF_TILE, 0, s>>>(p);
+    c->launches += 2;
+    if (attn_out) {
+      attn_out_kernel<<<dim3((S + AO_ROWS - 1) / AO_ROWS, G), PF_TILE, 0, s>>>(p);
+      c->launches += 1;
+    }
+  }
+  select_kernel<<<G, SEL_THREADS, 0, s>>>(p);
+  c->launches += 1;
+  const size_t smem = (size_t)(FM_BR * kHeadDim + mlp_smem_floats(d.Rp)) * 4;
+  if (d.R == 8) {
+    if (nsplit > 0) {
+      cudaFuncSetAttribute(build_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+      build_kernel<8><<<dim3(nsplit, G), FM_THREADS, smem, s>>>(p);
+      c->launches += 1;
+    }
+    finalize_kernel<8><<<G, kHeadDim, 0, s>>>(p);
+  } else {
+    if (nsplit > 0) {
+      cudaFuncSetAttribute(build_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+      build_kernel<16><<<dim3(nsplit, G), FM_THREADS, smem, s>>>(p);
+      c->launches += 1;
+    }
+    finalize_kernel<16><<<G, kHeadDim, 0, s>>>(p);
+  }
+  c->launches += 1;
+  return cudaGetLastError() == cudaSuccess ? LESS_OK : LESS_ERR_CUDA;
+}
+
+}  // namespace less

@@ -1,0 +1,233 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the fp64 oracle
+on the same seeded inputs."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2402_09398_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+DEV = "cuda"
+
+
+def _setup(w, flags=0, psi_scale=None, max_prefill_layers=None, heavy=None, recent=None,
+           max_prompt=None):
+    from paper_2402_09398_b200 import binding
+    W = wl.make_weights(w, DEV)
+    ctx = binding.from_workload(w, W, DEV, max_prefill_layers=max_prefill_layers or w.layers,
+                                flags=flags, psi_scale=psi_scale, heavy=heavy, recent=recent,
+                                max_prompt=max_prompt)
+    return ctx, {k: v.cpu() for k, v in W.items()}
+
+
+def small(cfg_id=71, **kw):
+    base = dict(batch=2, layers=2, heads=3, head_dim=128, prompt=300, steps=12, heavy=20, recent=20,
+                rank=8, hidden=512, heavy_rule="bernoulli", heavy_param=0.05, weight_std=0.02)
+    base.update(kw)
+    return wl.Workload(cfg_id, **base)
+
+
+def _prefill_all(ctx, w, with_out=True, prompt=None):
+    Q, K, V = wl.make_prompt(w, 0, w.layers, DEV, prompt=prompt)
+    out = torch.empty(Q.shape, dtype=torch.float32, device=DEV) if with_out else None
+    ctx.prefill(Q, K, V, 0, attn_out=out)
+    torch.cuda.synchronize()
+    return Q, K, V, out
+
+
+@pytest.mark.parametrize("variant", ["base", "rank16", "boosted", "ragged", "sparse_norm", "no_state",
+                                     "scaled", "heavy0", "recent1", "hidden256"])
+def test_prefill_and_teacher_forced_decode(variant):
+    import harness
+    flags, psi_scale = 0, None
+    w = small()
+    if variant == "rank16":
+        w = small(72, rank=16, prompt=257)
+    elif variant == "boosted":
+        w = small(73, weight_std=0.2)           # low-rank mass is a large share of the denominator
+    elif variant == "ragged":
+        w = small(74, prompt=131, heavy=7, recent=9, batch=3, heads=2)
+    elif variant == "sparse_norm":
+        w, flags = small(75, weight_std=0.2), 1
+    elif variant == "no_state":
+        w, flags = small(76), 2
+    elif variant == "scaled":
+        w = small(77, weight_std=0.1)
+        g = torch.Generator().manual_seed(5)
+        psi_scale = 0.5 + 2.0 * torch.rand(w.layers, w.heads, 2, generator=g)
+    elif variant == "heavy0":
+        w = small(78, heavy=0, recent=24)
+    elif variant == "recent1":
+        w = small(79, heavy=30, recent=1)
+    elif variant == "hidden256":
+        w = small(80, hidden=256, weight_std=0.05)
+    ctx, W = _setup(w, flags, psi_scale)
+    Q, K, V, out = _prefill_all(ctx, w)
+    inst = list(range(w.instances))
+    summary = harness.check_prefill(ctx, w, W, Q, K, V, inst, out, flags, psi_scale)
+    assert ctx.poll_status() == 0
+    tf = harness.TeacherForced(ctx, w, W, inst, flags, psi_scale)
+    for s in range(w.steps):
+        q, k, v = wl.make_decode_inputs(w, s, DEV)
+        tf.step(q, k, v)
+    assert ctx.poll_status() == 0
+    assert tf.evictions == w.steps * w.instances
+    assert tf.exempt <= 0.02 * tf.evictions + 1
+    if variant in ("boosted", "scaled"):
+        assert tf.worst["lr_den"] > 0     # the low-rank path was really exercised and compared
+    print(variant, summary, tf.worst, "exempt", tf.exempt)
+    ctx.close()
+
+
+def test_short_prompt_fills_without_eviction_then_evicts():
+    """prompt_len <= slots: everything is kept; decode appends until full."""
+    import harness
+    w = small(81, prompt=30, steps=25, heavy=20, recent=20)
+    ctx, W = _setup(w)
+    Q, K, V, out = _prefill_all(ctx, w)
+    inst = list(range(w.instances))
+    harness.check_prefill(ctx, w, W, Q, K, V, inst, out)
+    tf = harness.TeacherForced(ctx, w, W, inst)
+    for s in range(w.steps):
+        tf.step(*wl.make_decode_inputs(w, s, DEV))
+    # 30 prompt + 25 steps = 55 tokens, 40 slots -> 15 evictions per instance
+    assert tf.evictions == 15 * w.instances
+    assert ctx.poll_status() == 0
+    ctx.close()
+
+
+def test_decode_from_empty_context_and_reset():
+    """No prefill at all: the cache fills from empty; the first output is v itself."""
+    import harness
+    w = small(82, prompt=0, steps=10, heavy=3, recent=3)
+    ctx, W = _setup(w, max_prompt=16)
+    inst = list(range(w.instances))
+    tf = harness.TeacherForced(ctx, w, W, inst)
+    q, k, v = wl.make_decode_inputs(w, 0, DEV)
+    out = tf.step(q, k, v)
+    assert torch.allclose(out, v.float(), atol=1e-6)      # softmax over one entry
+    for s in range(1, w.steps):
+        tf.step(*wl.make_decode_inputs(w, s, DEV))
+    assert tf.evictions == (w.steps - 6) * w.instances
+    ctx.reset()
+    assert ctx.position == 0
+    rec = ctx.export_state(inst[:2])
+    assert rec[0]["count"] == 0 and not rec[0]["H"].any() and not rec[0]["z"].any()
+    ctx.close()
+
+
+def test_layer_groups_and_per_layer_prefill_agree():
+    """Prefilling layer by layer, in groups, or all at once gives identical state."""
+    w = small(83, layers=3, batch=1, heads=2, prompt=200)
+    states = []
+    for mode in ("all", "one", "two"):
+        ctx, W = _setup(w, max_prefill_layers={"all": 3, "one": 1, "two": 2}[mode])
+        if mode == "one":
+            for layer in range(w.layers):
+                Q, K, V = wl.make_prompt(w, layer, 1, DEV)
+                ctx.prefill(Q, K, V, layer)
+        else:
+            Q, K, V = wl.make_prompt(w, 0, w.layers, DEV)
+            ctx.prefill(Q, K, V, 0)
+        states.append(ctx.export_state(list(range(w.instances))))
+        ctx.close()
+    for other in states[1:]:
+        for a, b in zip(states[0], other):
+            for key in ("pos", "acc", "K", "V", "psi", "H", "z"):
+                assert np.array_equal(a[key], b[key]), key
+
+
+def test_bit_identical_reruns():
+    """Same inputs twice -> bit-identical outputs and state (no atomics, no races)."""
+    w = small(84, steps=6)
+    results = []
+    for _ in range(2):
+        ctx, W = _setup(w)
+        _prefill_all(ctx, w, with_out=False)
+        outs = [ctx.decode_step(*wl.make_decode_inputs(w, s, DEV)).cpu() for s in range(w.steps)]
+        results.append((outs, ctx.export_state(list(range(w.instances)))))
+        ctx.close()
+    for a, b in zip(results[0][0], results[1][0]):
+        assert torch.equal(a, b)
+    for a, b in zip(results[0][1], results[1][1]):
+        for key in ("pos", "acc", "K", "V", "psi", "H", "z"):
+            assert np.array_equal(a[key], b[key]), key
+
+
+def test_free_running_state_equals_sum_over_evicted_log():
+    """End state after a free run: H, z against the plain sum over the positions the
+    library itself evicted (prompt-phase evictions = positions not kept)."""
+    import harness
+    w = small(85, steps=40, weight_std=0.1)
+    ctx, W = _setup(w)
+    Q, K, V, _ = _prefill_all(ctx, w, with_out=False)
+    inst = list(range(w.instances))
+    pre = ctx.export_state(inst)
+    evlog = {i: sorted(set(range(w.prompt)) - set(r["pos"].tolist())) for i, r in zip(inst, pre)}
+    Kd, Vd = [], []
+    ev = torch.empty(w.instances, dtype=torch.int32, device=DEV)
+    for s in range(w.steps):
+        q, k, v = wl.make_decode_inputs(w, s, DEV)
+        ctx.decode_step(q, k, v, evicted_pos=ev)
+        Kd.append(k.reshape(-1, w.head_dim).cpu())
+        Vd.append(v.reshape(-1, w.head_dim).cpu())
+        for i, p in enumerate(ev.cpu().tolist()):
+            assert p >= 0
+            evlog[i].append(p)
+    post = ctx.export_state(inst)
+    for i, r in zip(inst, post):
+        b, layer, head = wl.instance_coords(w, i)
+        Kh = torch.cat([K[b, layer, head].cpu()] + [kd[i][None] for kd in Kd]).double().numpy()
+        Vh = torch.cat([V[b, layer, head].cpu()] + [vd[i][None] for vd in Vd]).double().numpy()
+        assert len(set(evlog[i])) == len(evlog[i]) == w.prompt + w.steps - w.slots
+        H, z = harness.brute_force_state(w, W, i, Kh, Vh, evlog[i])
+        assert harness.rel_err(r["H"], H) <= 1e-3 and harness.rel_err(r["z"], z) <= 1e-3
+        assert not (set(r["pos"].tolist()) & set(evlog[i]))
+    ctx.close()
+
+
+def test_crafted_tie_evicts_lowest_position():
+    """Equal accumulated scores: the lowest position goes (imported state)."""
+    w = small(86, batch=1, layers=1, heads=1, prompt=0, heavy=2, recent=2)
+    ctx, W = _setup(w, max_prompt=8)
+    D, R = w.head_dim, w.rank
+    rec = {"count": 4, "t": 10, "pos": np.array([7, 3, 5, 9], dtype=np.int32),
+           "acc": np.array([0.5, 0.5, 0.5, 0.1], dtype=np.float32),
+           "K": np.zeros((4, D), dtype=np.float16),
+           "V": np.arange(4 * D, dtype=np.float16).reshape(4, D) / 64,
+           "psi": np.ones((4, R), dtype=np.float32), "H": np.zeros((R, D), dtype=np.float32),
+           "z": np.zeros(R, dtype=np.float32)}
+    ctx.import_state([0], [rec])
+    assert ctx.position == 10
+    z = torch.zeros(1, 1, 1, D, dtype=torch.float16, device=DEV)
+    ev = torch.empty(1, dtype=torch.int32, device=DEV)
+    ctx.decode_step(z, z, z + 1, evicted_pos=ev)
+    assert int(ev.item()) == 3        # candidates pos <= 8: {7,3,5}, all tied -> lowest position
+    post = ctx.export_state([0])[0]
+    assert sorted(post["pos"].tolist()) == [5, 7, 9, 10]
+    assert np.allclose(post["H"], np.outer(np.ones(R), rec["V"][1].astype(np.float32)))
+    assert np.allclose(post["z"], 1.0)
+    ctx.close()
+
+
+def test_host_side_errors_on_gpu_box():
+    from paper_2402_09398_b200 import binding as B
+    w = small(87)
+    ctx, W = _setup(w)
+    Q, K, V = wl.make_prompt(w, 0, w.layers, DEV, prompt=w.prompt + 8)
+    with pytest.raises(B.LessError) as e:
+        ctx.prefill(Q, K, V, 0)
+    assert e.value.code == -5                                  # prompt too long
+    Q, K, V = wl.make_prompt(w, 0, w.layers, DEV)
+    with pytest.raises(B.LessError) as e:
+        ctx.prefill(Q, K, V, 1)
+    assert e.value.code == -6                                  # layer range
+    q, k, v = wl.make_decode_inputs(w, 0, DEV)
+    rc = B.less_decode_step(ctx.ctx, q.data_ptr() + 2, k.data_ptr(), v.data_ptr(),
+                            torch.empty(q.shape, device=DEV).data_ptr(), None, 0)
+    assert rc == -3                                            # misaligned
+    rc = B.less_decode_step(ctx.ctx, None, k.data_ptr(), v.data_ptr(), q.data_ptr(), None, 0)
+    assert rc == -2
+    assert ctx.poll_status() == 0
+    ctx.close()
