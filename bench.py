@@ -1,0 +1,393 @@
+#!/usr/bin/env python
+"""Benchmark of the LESS decode hot path on B200.
+
+A step = one generation step (Algorithm 1) of every (batch, layer, head)
+instance of the workload: feature maps, attention over the kept slots with the
+low-rank correction, score update, eviction, state update.  The cache is first
+built by the library's own prompt phase from seeded synthetic Q/K/V, then
+`--warmup` untimed and `--steps` timed decode steps run.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config 2] [--impl reference]
+
+Prints ONE JSON line (rank 0).  With --impl reference the fp64 CPU oracle is
+timed instead, on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "decode attention head-tokens/s (B x layers x heads per step)"
+UNIT = "head-tokens/s"
+FALLBACK_HBM_GBS = 6650.0
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures
+# summarised under profiles/ (None until a capture of that kernel/workload exists)
+NCU_TRAFFIC_BYTES = {}
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=64)
+    ap.add_argument("--warmup", type=int, default=8)
+    ap.add_argument("--config", type=int, default=2, help="workload id (1-4)")
+    ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
+    ap.add_argument("--cpu-seconds", type=float, default=12.0, help="budget of the CPU-baseline leg")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--full-cache", action="store_true",
+                    help="context run: slots >= prompt + steps, so nothing is ever evicted")
+    ap.add_argument("--no-state", action="store_true", help="context run: sparse policy alone (Baseline+)")
+    return ap.parse_args()
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return float(d["hbm_gbs"]), "measured"
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+# --------------------------------------------------------------------------- #
+# algorithmic bytes per launch (the figures the design doc derives)
+# --------------------------------------------------------------------------- #
+def feature_map_bytes(w, no_state=False):
+    if no_state:
+        return 0
+    D, Rp, R = w.head_dim, w.hidden, w.rank
+    weights = w.layers * w.heads * (2 * (D * Rp + Rp * R) + R * R) * 2
+    io = w.instances * (2 * D * 2 + 2 * R * 4)
+    return weights + io
+
+
+def decode_bytes(w, n_live, evicting=True, no_state=False):
+    D, R = w.head_dim, w.rank
+    per = n_live * (2 * D * 2)              # K and V rows
+    per += n_live * (4 + 4)                 # accumulated score read + write
+    per += n_live * 4 if evicting else 0    # positions (only read when a victim is needed)
+    per += 3 * D * 2 + D * 4                # q, k, v in; out
+    per += 2 * D * 2 + 8                    # new pair into its slot, pos, acc
+    per += 4                                # slot count
+    if not no_state:
+        per += R * D * 4 + R * 4            # H, z read
+        per += 2 * R * 4                    # phi(q), psi(k) read
+        per += R * 4                        # psi into the slot's cache
+        if evicting:
+            per += R * D * 4 + R * 4 + R * 4 + D * 2   # H, z write; victim psi; victim v row
+    return w.instances * per
+
+
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.lines, self.proc = [], None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={index}", f"--query-gpu={self.FIELDS}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._pump, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append((time.time(), line.strip()))
+
+    def stop(self, t0, t1):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        sm, mx, reasons = [], None, set()
+        rows = [l for (t, l) in self.lines if t0 - 0.05 <= t <= t1 + 0.15] or [l for _, l in self.lines]
+        for l in rows:
+            f = [x.strip() for x in l.split(",")]
+            try:
+                sm.append(float(f[0]))
+                mx = float(f[1])
+            except (ValueError, IndexError):
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown",
+                                  "sw_power_cap"), f[4:8]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": mx,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# --------------------------------------------------------------------------- #
+# CPU oracle timing (cpu_baseline leg and --impl reference)
+# --------------------------------------------------------------------------- #
+def oracle_rate(w, seconds, records=None, instances=None, W=None, max_instances=16):
+    """Times oracle decode steps on a bounded sample of instances.  With
+    `records` (states exported from the GPU) the oracle starts from them, else it
+    runs its own prompt phase first (untimed).  Returns (head-tokens/s, cores, text)."""
+    import numpy as np
+    from threadpoolctl import threadpool_limits
+    from oracle import less_oracle as lo
+    from paper_2402_09398_b200 import workloads as wl
+    if W is None:
+        W = wl.make_weights(w, "cpu")
+    with threadpool_limits(limits=1):
+        if instances is None:
+            instances = list(range(0, w.instances, max(1, w.instances // max_instances)))[:max_instances]
+        orcs = []
+        prompt_cache = {}
+        for n, inst in enumerate(instances):
+            b, layer, head = wl.instance_coords(w, inst)
+            wts = [W[k][layer, head].double().cpu().numpy() for k in
+                   ("w_phi1", "w_phi2", "w_psi1", "w_psi2", "w_psi3")]
+            o = lo.LessInstance(w.head_dim, w.rank, w.heavy, w.recent, *lo.make_mlp_maps(*wts))
+            if records is not None:
+                r = records[n]
+                o.import_state(r["pos"], r["K"], r["V"], r["acc"], r["H"], r["z"], r["t"])
+            else:
+                if layer not in prompt_cache:
+                    prompt_cache = {layer: wl.make_prompt(w, layer, 1, "cpu")}
+                Q, K, V = prompt_cache[layer]
+                o.prefill(*(t[b, 0, head].double().numpy() for t in (Q, K, V)))
+            orcs.append(o)
+        units, t_used, step = 0, 0.0, 0
+        while t_used < seconds and step < max(w.steps, 1):
+            q, k, v = wl.make_decode_inputs(w, step, "cpu")
+            q, k, v = (t.reshape(-1, w.head_dim).double().numpy() for t in (q, k, v))
+            t0 = time.perf_counter()
+            for inst, o in zip(instances, orcs):
+                o.decode(q[inst], k[inst], v[inst])
+            t_used += time.perf_counter() - t0
+            units += len(instances)
+            step += 1
+    sample = (f"{len(instances)} of {w.instances} instances x {step} decode steps "
+              f"({'GPU-exported' if records is not None else 'oracle-prefilled'} state), fp64 numpy, 1 thread")
+    return units / t_used, 1, sample, step, t_used
+
+
+def run_reference(args):
+    from paper_2402_09398_b200 import workloads as wl
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    w = wl.CONFIGS[args.config]
+    # each "step" = one oracle decode step over the sampled instances
+    per_step_budget = 120.0 / max(1, args.steps + args.warmup)
+    n_inst = 8
+    w_run = w.with_(steps=args.steps + args.warmup)
+    rate, cores, sample, steps_done, t_used = oracle_rate(
+        w_run, seconds=per_step_budget * (args.steps + args.warmup), max_instances=n_inst)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": rate, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t_used / max(1, steps_done),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic", "config": workload_config(w, args),
+        "cpu_baseline": {"value": rate, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": rate, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def workload_config(w, args):
+    name = {1: "cfg1 smallest (B=1, 1 layer x 8 heads, prompt 256, 32+32 slots, R=8)",
+            2: "cfg2 Llama-2-7B shape (B=1, 32 layers x 32 heads, prompt 2048, 102+102 slots, R=8)",
+            3: "cfg3 batched serving (B=64, 32 layers x 32 heads, prompt 1024, 102+102 slots, R=8)",
+            4: "cfg4 long context (B=4, 40 layers x 40 heads, prompt 16384, 327+327 slots, R=16)"}[w.cfg_id]
+    c = {"workload": name, "instances": w.instances, "slots": w.slots, "rank": w.rank,
+         "prompt": w.prompt, "l2": "bytes touched per step exceed the 126 MB L2"
+         if w.cfg_id != 1 else "L2 flushed by a 256 MB write between steps is NOT done: cfg1 is launch-bound"}
+    if getattr(args, "full_cache", False):
+        c["variant"] = "full cache (no eviction)"
+    if getattr(args, "no_state", False):
+        c["variant"] = "sparse policy alone (Baseline+)"
+    return c
+
+
+# --------------------------------------------------------------------------- #
+def run_b200(args):
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+    from paper_2402_09398_b200 import binding, build, workloads as wl
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the LESS path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = f"cuda:{local}"
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+    build.build()
+    binding.lib()
+
+    w = wl.CONFIGS[args.config]
+    K_steps, W_steps = args.steps, args.warmup
+    total_steps = K_steps * 3 + W_steps + 2
+    heavy, recent, flags = w.heavy, w.recent, 0
+    if args.full_cache:
+        heavy = w.prompt + total_steps
+    if args.no_state:
+        flags |= binding.LESS_NO_STATE
+        heavy += 2 if w.rank == 8 else 4      # Baseline+: slots matching H's storage (Section 4)
+        recent += 2 if w.rank == 8 else 4
+    w_run = w.with_(heavy=heavy, recent=recent)
+
+    # replicas: every rank runs the whole workload on its own GPU, no collective in the path
+    Wt = wl.make_weights(w, dev)
+    layers_per_call = max(1, min(w.layers, (1 << 30) // max(1, w.batch * w.heads * w.prompt * w.head_dim * 2)))
+    ctx = binding.from_workload(w_run, Wt, dev, max_prefill_layers=layers_per_call, flags=flags)
+    t_pre0 = time.perf_counter()
+    for l0 in range(0, w.layers, layers_per_call):
+        n = min(layers_per_call, w.layers - l0)
+        Q, Kp, V = wl.make_prompt(w, l0, n, dev)
+        ctx.prefill(Q, Kp, V, l0)
+        del Q, Kp, V
+    torch.cuda.synchronize()
+    t_prefill = time.perf_counter() - t_pre0
+
+    # decode inputs for every step, resident in HBM before the timed region
+    inputs = [wl.make_decode_inputs(w, s % max(1, w.steps), dev) if s < 8 else None for s in range(total_steps)]
+    base = [i for i in inputs if i is not None]
+    inputs = [base[s % len(base)] for s in range(total_steps)]
+    out = torch.empty(w.batch, w.layers, w.heads, w.head_dim, dtype=torch.float32, device=dev)
+    stream = torch.cuda.current_stream()
+    step_no = [0]
+
+    def one_step():
+        q, k, v = inputs[step_no[0] % total_steps]
+        ctx.decode_step(q, k, v, out=out)
+        step_no[0] += 1
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(W_steps, 3)):
+        one_step()
+    barrier()
+
+    # ---- timed region: K steps, device-resident inputs ----
+    sampler = ClockSampler(local) if rank == 0 else None
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    launches0 = ctx.launches
+    barrier()
+    t0 = time.time()
+    e0.record(stream)
+    for _ in range(K_steps):
+        one_step()
+    e1.record(stream)
+    barrier()
+    t1 = time.time()
+    launches = ctx.launches - launches0
+    ms = e0.elapsed_time(e1)
+    clocks = sampler.stop(t0, t1) if sampler else None
+
+    # ---- same K steps with an event pair around every kernel: per-kernel durations ----
+    ctx.profile(True)
+    for _ in range(K_steps):
+        one_step()
+    torch.cuda.synchronize()
+    prof = ctx.profile_read()
+    ctx.profile(False)
+
+    # ---- end to end through the host-buffer entry point ----
+    hq, hk, hv = (torch.empty(inputs[0][0].shape, dtype=torch.float16).pin_memory() for _ in range(3))
+    hq.copy_(inputs[0][0]); hk.copy_(inputs[0][1]); hv.copy_(inputs[0][2])
+    hout = torch.empty(out.shape, dtype=torch.float32).pin_memory()
+    for _ in range(3):
+        ctx.decode_step_host(hq, hk, hv, hout)
+    barrier()
+    e2, e3 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e2.record(stream)
+    tw0 = time.perf_counter()
+    for _ in range(K_steps):
+        ctx.decode_step_host(hq, hk, hv, hout)
+    e3.record(stream)
+    torch.cuda.synchronize()
+    ms_e2e = max(e2.elapsed_time(e3), 1e3 * (time.perf_counter() - tw0))
+    status = ctx.poll_status()
+    if status != 0:
+        raise RuntimeError(f"device status {status}")
+
+    if world > 1:
+        t = torch.tensor([ms, ms_e2e], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms, ms_e2e = float(t[0]), float(t[1])
+
+    if rank == 0:
+        units = w.instances * world
+        value = units * K_steps / (ms * 1e-3)
+        e2e_value = units * K_steps / (ms_e2e * 1e-3)
+        peak, peak_kind = peaks()
+        n_live = min(w_run.slots, w.prompt + W_steps)
+        evicting = not args.full_cache
+        kb = {"feature_map": feature_map_bytes(w, args.no_state),
+              "decode": decode_bytes(w, n_live, evicting, args.no_state)}
+        kt = {k: (prof[k][0] / prof[k][1] if prof[k][1] else 0.0) for k in ("feature_map", "decode")}
+        dominant = max(kt, key=lambda k: kt[k])
+        ach = kb[dominant] / (kt[dominant] * 1e-3) / 1e9 if kt[dominant] > 0 else 0.0
+        step_bytes = kb["feature_map"] + kb["decode"]
+        kv_state_bytes = w.instances * (n_live * (4 * w.head_dim + 8) + (0 if args.no_state else 2 * w.rank * w.head_dim * 4))
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K_steps,
+            "warmup": max(W_steps, 3), "ms_per_step": ms / K_steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": workload_config(w, args),
+            "clocks": clocks,
+            "e2e": {"value": e2e_value, "unit": UNIT,
+                    "h2d_bytes_per_step": 3 * w.instances * w.head_dim * 2,
+                    "d2h_bytes_per_step": w.instances * w.head_dim * 4},
+            "gpu_launches": int(launches),
+            "roofline": {"bound": "hbm", "kernel": dominant + "_kernel", "achieved": ach, "peak": peak,
+                         "unit": "GB/s", "frac": ach / peak, "peak_kind": f"of {peak_kind}",
+                         "frac_of_nominal_8TBs": ach / 8000.0,
+                         "traffic": NCU_TRAFFIC_BYTES.get((w.cfg_id, dominant)),
+                         "algorithmic_bytes_per_launch": kb[dominant],
+                         "kernel_us": {k: 1e3 * v for k, v in kt.items()},
+                         "kernel_GBs": {k: (kb[k] / (kt[k] * 1e-3) / 1e9 if kt[k] > 0 else 0.0) for k in kt},
+                         "step_algorithmic_bytes": step_bytes,
+                         "step_GBs": step_bytes / (ms / K_steps * 1e-3) / 1e9,
+                         "step_frac": step_bytes / (ms / K_steps * 1e-3) / 1e9 / peak,
+                         "kv_state_scores_GBs": kv_state_bytes / (ms / K_steps * 1e-3) / 1e9},
+            "prefill_s": t_prefill,
+        }
+        if not args.no_cpu_baseline and world == 1:
+            instances = list(range(0, w.instances, max(1, w.instances // 16)))[:16]
+            recs = ctx.export_state(instances)
+            Wc = {k: v.cpu() for k, v in Wt.items()}
+            rate, cores, sample, _, _ = oracle_rate(w.with_(steps=max(w.steps, 64)), args.cpu_seconds, recs, instances, Wc)
+            line["cpu_baseline"] = {"value": rate, "unit": UNIT, "cores": cores, "kind": "oracle",
+                                    "sample": sample}
+        print(json.dumps(line))
+    ctx.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_b200(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -127,6 +127,33 @@ int less_prefill(less_ctx* ctx, int32_t layer_begin, int32_t layer_count, int32_
 int less_decode_step(less_ctx* ctx, const void* q, const void* k, const void* v, void* out,
                      int32_t* evicted_pos, void* cuda_stream);
 
+/* The same step for callers whose tensors live in host memory (Algorithm 1's
+ * inputs and return value): copies q, k, v (host fp16 [B, L, H, D], ideally
+ * pinned) to staging buffers inside the arena, runs less_decode_step, copies
+ * out (host fp32 [B, L, H, D]) back, all on the given stream, and synchronises
+ * it before returning. */
+int less_decode_step_host(less_ctx* ctx, const void* q_host, const void* k_host, const void* v_host,
+                          void* out_host, void* cuda_stream);
+
+/* Per-kernel device timing.  less_profile(ctx, 1) makes every later kernel
+ * launch of this context record a CUDA event pair on its stream;
+ * less_profile(ctx, 0) stops and discards.  less_profile_read synchronises the
+ * recorded events and adds up, per kernel id, the elapsed milliseconds and the
+ * launch count since profiling was enabled (arrays of LESS_KERNEL_COUNT). */
+enum {
+  LESS_KERNEL_FEATURE_MAP = 0,
+  LESS_KERNEL_DECODE = 1,
+  LESS_KERNEL_ROWSTAT = 2,
+  LESS_KERNEL_COLSUM = 3,
+  LESS_KERNEL_ATTN_OUT = 4,
+  LESS_KERNEL_SELECT = 5,
+  LESS_KERNEL_BUILD = 6,
+  LESS_KERNEL_FINALIZE = 7,
+  LESS_KERNEL_COUNT = 8
+};
+int less_profile(less_ctx* ctx, int enable);
+int less_profile_read(less_ctx* ctx, float* ms_total_host, int64_t* launches_host);
+
 /* Tokens seen so far (= absolute position of the next decode token). */
 int64_t less_position(const less_ctx* ctx);
 

@@ -24,8 +24,10 @@ EXPORTED = [
     "less_arena_bytes", "less_create", "less_prefill", "less_decode_step", "less_position",
     "less_state_record_bytes", "less_export_state", "less_import_state",
     "less_read_feature_maps", "less_poll_status", "less_launch_count", "less_strerror",
-    "less_destroy",
+    "less_destroy", "less_decode_step_host", "less_profile", "less_profile_read",
 ]
+
+KERNEL_NAMES = ["feature_map", "decode", "rowstat", "colsum", "attn_out", "select", "build", "finalize"]
 
 
 class less_config(C.Structure):
@@ -71,6 +73,12 @@ def lib() -> C.CDLL:
     L.less_prefill.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp]
     L.less_decode_step.restype = C.c_int
     L.less_decode_step.argtypes = [vp, vp, vp, vp, vp, vp, vp]
+    L.less_decode_step_host.restype = C.c_int
+    L.less_decode_step_host.argtypes = [vp, vp, vp, vp, vp, vp]
+    L.less_profile.restype = C.c_int
+    L.less_profile.argtypes = [vp, C.c_int]
+    L.less_profile_read.restype = C.c_int
+    L.less_profile_read.argtypes = [vp, vp, vp]
     L.less_position.restype = i64
     L.less_position.argtypes = [vp]
     L.less_launch_count.restype = i64
@@ -118,6 +126,18 @@ def less_prefill(ctx, layer_begin, layer_count, prompt_len, Q, K, V, attn_out, s
 
 def less_decode_step(ctx, q, k, v, out, evicted_pos, stream) -> int:
     return lib().less_decode_step(ctx, q, k, v, out, evicted_pos, stream)
+
+
+def less_decode_step_host(ctx, q_host, k_host, v_host, out_host, stream) -> int:
+    return lib().less_decode_step_host(ctx, q_host, k_host, v_host, out_host, stream)
+
+
+def less_profile(ctx, enable: int) -> int:
+    return lib().less_profile(ctx, int(enable))
+
+
+def less_profile_read(ctx, ms_ptr, launches_ptr) -> int:
+    return lib().less_profile_read(ctx, ms_ptr, launches_ptr)
 
 
 def less_position(ctx) -> int:
@@ -213,6 +233,21 @@ class LessContext:
         _check(less_decode_step(self.ctx, _ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(evicted_pos),
                                 _stream_ptr(stream)), "less_decode_step")
         return out
+
+    def decode_step_host(self, q, k, v, out, stream=None):
+        """q, k, v, out: host tensors (pinned for speed); synchronous."""
+        _check(less_decode_step_host(self.ctx, _ptr(q), _ptr(k), _ptr(v), _ptr(out),
+                                     _stream_ptr(stream)), "less_decode_step_host")
+        return out
+
+    def profile(self, enable: bool):
+        _check(less_profile(self.ctx, 1 if enable else 0), "less_profile")
+
+    def profile_read(self):
+        ms = np.zeros(len(KERNEL_NAMES), dtype=np.float32)
+        n = np.zeros(len(KERNEL_NAMES), dtype=np.int64)
+        _check(less_profile_read(self.ctx, ms.ctypes.data, n.ctypes.data), "less_profile_read")
+        return {k: (float(a), int(b)) for k, a, b in zip(KERNEL_NAMES, ms, n)}
 
     # -- state ------------------------------------------------------------- #
     @property

@@ -73,6 +73,7 @@ int launch_feature_maps(less_ctx* c, const void* q, const void* k, cudaStream_t 
   const size_t smem = (size_t)(FM_BR * kHeadDim + FM_BR * d.Rp + ndg * FM_BR * d.Rp) * 4;
   dim3 grid(d.L * d.Hd, (d.flags & LESS_NO_STATE) ? 1 : 2, (d.B + FM_BR - 1) / FM_BR);
   if (d.flags & LESS_NO_STATE) return LESS_OK;   // neither phi nor psi is used
+  LaunchScope scope(c, LESS_KERNEL_FEATURE_MAP, s);
   if (d.R == 8) {
     cudaFuncSetAttribute(feature_map_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     feature_map_kernel<8><<<grid, FM_THREADS, smem, s>>>(p);
@@ -80,7 +81,6 @@ int launch_feature_maps(less_ctx* c, const void* q, const void* k, cudaStream_t 
     cudaFuncSetAttribute(feature_map_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     feature_map_kernel<16><<<grid, FM_THREADS, smem, s>>>(p);
   }
-  c->launches += 1;
   return cudaGetLastError() == cudaSuccess ? LESS_OK : LESS_ERR_CUDA;
 }
 
@@ -324,6 +324,7 @@ int launch_decode(less_ctx* c, const void* q, const void* k, const void* v, void
   p.N = d.N; p.Np = d.Np; p.recent = d.recent; p.t = (int)c->t;
   p.flags = d.flags;
   const size_t smem = (size_t)(d.Np + 4 + DEC_RG * kHeadDim) * 4;
+  LaunchScope scope(c, LESS_KERNEL_DECODE, s);
   if (d.R == 8) {
     if (smem > 48 * 1024)
       cudaFuncSetAttribute(decode_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -333,7 +334,6 @@ int launch_decode(less_ctx* c, const void* q, const void* k, const void* v, void
       cudaFuncSetAttribute(decode_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     decode_kernel<16><<<d.I, DEC_THREADS, smem, s>>>(p);
   }
-  c->launches += 1;
   return cudaGetLastError() == cudaSuccess ? LESS_OK : LESS_ERR_CUDA;
 }
 

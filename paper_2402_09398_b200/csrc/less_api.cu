@@ -68,6 +68,10 @@ size_t carve(const Dims& d, char* base, Arena* a) {
   t.phi_q = (float*)take(I * R * 4);
   t.psi_k = (float*)take(I * R * 4);
   t.status = (int32_t*)take(4 * 4);
+  t.stage_q = (__half*)take(I * D * 2);
+  t.stage_k = (__half*)take(I * D * 2);
+  t.stage_v = (__half*)take(I * D * 2);
+  t.stage_out = (float*)take(I * D * 4);
   t.ws_m = (float*)take(Iw * Sp * 4);
   t.ws_invl = (float*)take(Iw * Sp * 4);
   t.ws_acc = (float*)take(Iw * Sp * 4);
@@ -134,6 +138,7 @@ int less_create(const less_config* cfg, const less_weights* w, void* arena, size
   c->arena_bytes = need;
   c->t = 0;
   c->launches = 0;
+  c->profile = false;
   if (cudaGetDevice(&c->device) != cudaSuccess) { delete c; return LESS_ERR_CUDA; }
   // H_0 = 0, z_0 = 0, no live slots, clean status
   cudaError_t e = cudaMemset(c->a.H, 0, (size_t)d.I * d.R * d.D * 4);
@@ -150,6 +155,8 @@ int less_create(const less_config* cfg, const less_weights* w, void* arena, size
 
 int less_destroy(less_ctx* ctx) {
   if (!ctx) return LESS_ERR_NULL_POINTER;
+  for (cudaEvent_t e : ctx->prof_events) cudaEventDestroy(e);
+  for (cudaEvent_t e : ctx->prof_pool) cudaEventDestroy(e);
   delete ctx;
   return LESS_OK;
 }
@@ -192,6 +199,45 @@ int less_decode_step(less_ctx* c, const void* q, const void* k, const void* v, v
   rc = launch_decode(c, q, k, v, out, evicted_pos, s);
   if (rc != LESS_OK) return rc;
   c->t += 1;
+  return LESS_OK;
+}
+
+int less_decode_step_host(less_ctx* c, const void* qh, const void* kh, const void* vh, void* outh,
+                          void* stream) {
+  if (!c || !qh || !kh || !vh || !outh) return LESS_ERR_NULL_POINTER;
+  cudaStream_t s = (cudaStream_t)stream;
+  const size_t nin = (size_t)c->d.I * c->d.D * 2, nout = (size_t)c->d.I * c->d.D * 4;
+  cudaError_t e = cudaMemcpyAsync(c->a.stage_q, qh, nin, cudaMemcpyHostToDevice, s);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(c->a.stage_k, kh, nin, cudaMemcpyHostToDevice, s);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(c->a.stage_v, vh, nin, cudaMemcpyHostToDevice, s);
+  if (e != cudaSuccess) return LESS_ERR_CUDA;
+  int rc = less_decode_step(c, c->a.stage_q, c->a.stage_k, c->a.stage_v, c->a.stage_out, nullptr, s);
+  if (rc != LESS_OK) return rc;
+  e = cudaMemcpyAsync(outh, c->a.stage_out, nout, cudaMemcpyDeviceToHost, s);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+  return e == cudaSuccess ? LESS_OK : LESS_ERR_CUDA;
+}
+
+int less_profile(less_ctx* c, int enable) {
+  if (!c) return LESS_ERR_NULL_POINTER;
+  for (cudaEvent_t e : c->prof_events) c->prof_pool.push_back(e);
+  c->prof_events.clear();
+  c->prof_kernel.clear();
+  c->profile = enable != 0;
+  return LESS_OK;
+}
+
+int less_profile_read(less_ctx* c, float* ms_total, int64_t* launches) {
+  if (!c || !ms_total || !launches) return LESS_ERR_NULL_POINTER;
+  for (int i = 0; i < LESS_KERNEL_COUNT; ++i) { ms_total[i] = 0.f; launches[i] = 0; }
+  for (size_t i = 0; i < c->prof_kernel.size(); ++i) {
+    cudaEvent_t a = c->prof_events[2 * i], b = c->prof_events[2 * i + 1];
+    if (cudaEventSynchronize(b) != cudaSuccess) return LESS_ERR_CUDA;
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, a, b) != cudaSuccess) return LESS_ERR_CUDA;
+    const int k = c->prof_kernel[i];
+    if (k >= 0 && k < LESS_KERNEL_COUNT) { ms_total[k] += ms; launches[k] += 1; }
+  }
   return LESS_OK;
 }
 

@@ -6,6 +6,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <vector>
+
 #include "less.h"
 
 namespace less {
@@ -27,6 +29,10 @@ struct Arena {
   float* phi_q;      // [I][R]      phi(q_t) of the current step
   float* psi_k;      // [I][R]      psi(k_t) of the current step
   int32_t* status;   // [4]         device status word(s)
+  __half* stage_q;   // [I][D]      staging of host inputs (less_decode_step_host)
+  __half* stage_k;   // [I][D]
+  __half* stage_v;   // [I][D]
+  float* stage_out;  // [I][D]
   // prompt-phase workspace, for Iw = B * H * max_prefill_layers instances
   float* ws_m;       // [Iw][Sp]    row max of causal scores
   float* ws_invl;    // [Iw][Sp]    1 / row sum
@@ -56,6 +62,10 @@ struct less_ctx {
   int64_t t;           // tokens seen
   int64_t launches;    // kernels launched
   int device;
+  bool profile;                         // record an event pair around every launch
+  std::vector<cudaEvent_t> prof_events; // start, stop, start, stop, ...
+  std::vector<int> prof_kernel;         // kernel id of each pair
+  std::vector<cudaEvent_t> prof_pool;   // events ready for reuse
 };
 
 namespace less {
@@ -93,6 +103,35 @@ __device__ __forceinline__ uint4 ldg_readonly(const void* p) {
   // 128-bit load through the read-only path (weights: never written by a kernel)
   return __ldg(reinterpret_cast<const uint4*>(p));
 }
+
+// Brackets one kernel launch with an event pair when profiling is on, and counts it.
+struct LaunchScope {
+  less_ctx* c;
+  cudaStream_t s;
+  bool on;
+  LaunchScope(less_ctx* ctx, int kernel_id, cudaStream_t stream) : c(ctx), s(stream), on(ctx->profile) {
+    c->launches += 1;
+    if (!on) return;
+    cudaEvent_t a = take(), b = take();
+    c->prof_events.push_back(a);
+    c->prof_events.push_back(b);
+    c->prof_kernel.push_back(kernel_id);
+    cudaEventRecord(a, s);
+  }
+  ~LaunchScope() {
+    if (on) cudaEventRecord(c->prof_events.back(), s);
+  }
+  cudaEvent_t take() {
+    cudaEvent_t e;
+    if (!c->prof_pool.empty()) {
+      e = c->prof_pool.back();
+      c->prof_pool.pop_back();
+    } else {
+      cudaEventCreate(&e);
+    }
+    return e;
+  }
+};
 
 // launchers (host), defined in the kernel translation units
 int launch_feature_maps(less_ctx* c, const void* q, const void* k, cudaStream_t s);

@@ -442,33 +442,39 @@ int launch_prefill_group(less_ctx* c, int layer0, int nl, int lj0, int layer_cou
   const int G = d.B * nl * d.Hd;
   if (S > 0) {
     const int tiles = (S + PF_TILE - 1) / PF_TILE;
-    rowstat_kernel<<<dim3(tiles, G), PF_TILE, 0, s>>>(p);
-    colsum_kernel<<<dim3(tiles, G), PF_TILE, 0, s>>>(p);
-    c->launches += 2;
+    {
+      LaunchScope scope(c, LESS_KERNEL_ROWSTAT, s);
+      rowstat_kernel<<<dim3(tiles, G), PF_TILE, 0, s>>>(p);
+    }
+    {
+      LaunchScope scope(c, LESS_KERNEL_COLSUM, s);
+      colsum_kernel<<<dim3(tiles, G), PF_TILE, 0, s>>>(p);
+    }
     if (attn_out) {
+      LaunchScope scope(c, LESS_KERNEL_ATTN_OUT, s);
       attn_out_kernel<<<dim3((S + AO_ROWS - 1) / AO_ROWS, G), PF_TILE, 0, s>>>(p);
-      c->launches += 1;
     }
   }
-  select_kernel<<<G, SEL_THREADS, 0, s>>>(p);
-  c->launches += 1;
+  {
+    LaunchScope scope(c, LESS_KERNEL_SELECT, s);
+    select_kernel<<<G, SEL_THREADS, 0, s>>>(p);
+  }
   const size_t smem = (size_t)(FM_BR * kHeadDim + mlp_smem_floats(d.Rp)) * 4;
-  if (d.R == 8) {
-    if (nsplit > 0) {
+  if (nsplit > 0) {
+    LaunchScope scope(c, LESS_KERNEL_BUILD, s);
+    if (d.R == 8) {
       cudaFuncSetAttribute(build_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
       build_kernel<8><<<dim3(nsplit, G), FM_THREADS, smem, s>>>(p);
-      c->launches += 1;
-    }
-    finalize_kernel<8><<<G, kHeadDim, 0, s>>>(p);
-  } else {
-    if (nsplit > 0) {
+    } else {
       cudaFuncSetAttribute(build_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
       build_kernel<16><<<dim3(nsplit, G), FM_THREADS, smem, s>>>(p);
-      c->launches += 1;
     }
-    finalize_kernel<16><<<G, kHeadDim, 0, s>>>(p);
   }
-  c->launches += 1;
+  {
+    LaunchScope scope(c, LESS_KERNEL_FINALIZE, s);
+    if (d.R == 8) finalize_kernel<8><<<G, kHeadDim, 0, s>>>(p);
+    else finalize_kernel<16><<<G, kHeadDim, 0, s>>>(p);
+  }
   return cudaGetLastError() == cudaSuccess ? LESS_OK : LESS_ERR_CUDA;
 }
 
