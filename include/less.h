@@ -185,6 +185,33 @@ int less_poll_status(less_ctx* ctx, void* cuda_stream);
 /* Kernels of this library launched through this context so far. */
 int64_t less_launch_count(const less_ctx* ctx);
 
+/* The paper has no counterpart for this entry point: it exists for callers
+ * that may not allocate device memory (a process whose memory pool owns the
+ * whole GPU, a plugin that is only handed buffers and a stream, code that must
+ * not trigger the synchronisation an allocation implies).  It computes the H2O
+ * prompt scores of less_prefill's step 2 on its own:
+ *     acc_out[n][j] = sum_{i >= j} softmax_row_i( Q_n K_n^T / sqrt(D), causal )[j]
+ * for n_inst independent heads, with the per-row scratch (row maximum and
+ * reciprocal row sum) held in a fixed 512 KB array inside the library image,
+ * which every GPU that loads the library keeps until the process exits.
+ *   Q, K      device fp16 [n_inst, prompt_len, 128], 16-byte aligned
+ *   acc_out   device fp32 [n_inst, prompt_len]
+ * Limits and rules:
+ *   - n_inst * prompt_len <= LESS_NOALLOC_MAX_ROWS, else LESS_ERR_NOALLOC_TOO_LARGE
+ *     (nothing is launched);
+ *   - it calls no cudaMalloc / cudaFree and no allocating library routine;
+ *   - all calls on a device share the one array: calls ordered on a stream are
+ *     safe, calls that can overlap on the GPU race with each other;
+ *   - no part of the array needs clearing between calls (each call overwrites
+ *     every row it reads);
+ *   - the first call on each device looks up the array's device address: make
+ *     that call with the device current and outside any stream capture.
+ * Asynchronous on the given stream. */
+#define LESS_NOALLOC_MAX_ROWS 65536
+#define LESS_ERR_NOALLOC_TOO_LARGE (-12)
+int less_prompt_scores_noalloc(const void* Q, const void* K, int32_t n_inst, int32_t prompt_len,
+                               float* acc_out, void* cuda_stream);
+
 const char* less_strerror(int code);
 
 /* Releases the context; frees nothing the caller owns. */

@@ -25,7 +25,10 @@ EXPORTED = [
     "less_state_record_bytes", "less_export_state", "less_import_state",
     "less_read_feature_maps", "less_poll_status", "less_launch_count", "less_strerror",
     "less_destroy", "less_decode_step_host", "less_profile", "less_profile_read",
+    "less_prompt_scores_noalloc",
 ]
+LESS_NOALLOC_MAX_ROWS = 65536
+LESS_ERR_NOALLOC_TOO_LARGE = -12
 
 KERNEL_NAMES = ["feature_map", "decode", "rowstat", "colsum", "attn_out", "select", "build", "finalize"]
 
@@ -79,6 +82,8 @@ def lib() -> C.CDLL:
     L.less_profile.argtypes = [vp, C.c_int]
     L.less_profile_read.restype = C.c_int
     L.less_profile_read.argtypes = [vp, vp, vp]
+    L.less_prompt_scores_noalloc.restype = C.c_int
+    L.less_prompt_scores_noalloc.argtypes = [vp, vp, i32, i32, vp, vp]
     L.less_position.restype = i64
     L.less_position.argtypes = [vp]
     L.less_launch_count.restype = i64
@@ -138,6 +143,15 @@ def less_profile(ctx, enable: int) -> int:
 
 def less_profile_read(ctx, ms_ptr, launches_ptr) -> int:
     return lib().less_profile_read(ctx, ms_ptr, launches_ptr)
+
+
+def less_prompt_scores_noalloc(Q, K, n_inst, prompt_len, acc_out, stream) -> int:
+    """H2O prompt scores for callers that cannot allocate device memory (a
+    process whose pool owns the GPU, a plugin handed only buffers and a stream):
+    the scratch lives in a fixed array inside the library.  Device pointers in,
+    return code out; at most LESS_NOALLOC_MAX_ROWS rows (n_inst * prompt_len);
+    calls that may overlap on the GPU race on the shared array."""
+    return lib().less_prompt_scores_noalloc(Q, K, n_inst, prompt_len, acc_out, stream)
 
 
 def less_position(ctx) -> int:

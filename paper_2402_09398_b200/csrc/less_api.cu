@@ -340,6 +340,7 @@ const char* less_strerror(int code) {
     case LESS_ERR_CUDA: return "CUDA runtime error";
     case LESS_ERR_BAD_STATE: return "state record or context state not usable";
     case LESS_ERR_BUFFER_TOO_SMALL: return "host buffer too small";
+    case LESS_ERR_NOALLOC_TOO_LARGE: return "more rows than the built-in scratch array holds";
     default: return "unknown error";
   }
 }
