@@ -2,24 +2,16 @@
 //   feature_map_kernel  phi(q_t), psi(k_t)                         (Eq. 1, Eq. 2)
 //   decode_kernel       scores over the live slots, Eq. 3, H2O score update,
 //                       argmin eviction, Eq. 4 / Eq. 5, in-place slot overwrite
+#include "feature_gemv.cuh"
 #include "feature_mlp.cuh"
 
 namespace less {
 
 // --------------------------------------------------------------------------- //
-// Feature maps.  One CTA = one (layer, head), one map (phi or psi), up to FM_BR
-// batch rows.  The hidden activations never leave shared memory.
+// Feature maps, plain version (hidden widths the streaming kernel does not take).
+// One CTA = one (layer, head), one map (phi or psi), up to FM_BR batch rows.
+// The hidden activations never leave shared memory.
 // --------------------------------------------------------------------------- //
-struct FmParams {
-  const __half* x[2];     // q, k                       [B, L, Hd, D]
-  const __half* w1[2];    // W_phi1, W_psi1             [L, Hd, D, Rp]
-  const __half* w2[2];    // W_phi2, W_psi2             [L, Hd, Rp, R]
-  const __half* w3;       // W_psi3                     [L, Hd, R, R]
-  const float* psi_scale; // [L, Hd, 2] or null
-  float* out[2];          // phi_q, psi_k               [I, R]
-  int B, L, Hd, Rp;
-};
-
 template <int R>
 __global__ void __launch_bounds__(FM_THREADS) feature_map_kernel(FmParams p) {
   extern __shared__ float fm_smem[];
@@ -73,6 +65,7 @@ int launch_feature_maps(less_ctx* c, const void* q, const void* k, cudaStream_t 
   const size_t smem = (size_t)(FM_BR * kHeadDim + FM_BR * d.Rp + ndg * FM_BR * d.Rp) * 4;
   dim3 grid(d.L * d.Hd, (d.flags & LESS_NO_STATE) ? 1 : 2, (d.B + FM_BR - 1) / FM_BR);
   if (d.flags & LESS_NO_STATE) return LESS_OK;   // neither phi nor psi is used
+  if (feature_gemv_supported(d)) return launch_feature_gemv(c, p, s);
   LaunchScope scope(c, LESS_KERNEL_FEATURE_MAP, s);
   if (d.R == 8) {
     cudaFuncSetAttribute(feature_map_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);

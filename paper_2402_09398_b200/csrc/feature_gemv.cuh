@@ -1,0 +1,21 @@
+// Parameters and launcher of the streaming feature-map kernel.
+#pragma once
+
+#include "less_internal.cuh"
+
+namespace less {
+
+struct FmParams {
+  const __half* x[2];     // q, k                       [B, L, Hd, D]
+  const __half* w1[2];    // W_phi1, W_psi1             [L, Hd, D, Rp]
+  const __half* w2[2];    // W_phi2, W_psi2             [L, Hd, Rp, R]
+  const __half* w3;       // W_psi3                     [L, Hd, R, R]
+  const float* psi_scale; // [L, Hd, 2] or null
+  float* out[2];          // phi_q, psi_k               [I, R]
+  int B, L, Hd, Rp;
+};
+
+bool feature_gemv_supported(const Dims& d);
+int launch_feature_gemv(less_ctx* c, const FmParams& p, cudaStream_t s);
+
+}  // namespace less
