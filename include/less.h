@@ -149,7 +149,9 @@ enum {
   LESS_KERNEL_SELECT = 5,
   LESS_KERNEL_BUILD = 6,
   LESS_KERNEL_FINALIZE = 7,
-  LESS_KERNEL_COUNT = 8
+  LESS_KERNEL_PSI = 8,
+  LESS_KERNEL_GATHER = 9,
+  LESS_KERNEL_COUNT = 10
 };
 int less_profile(less_ctx* ctx, int enable);
 int less_profile_read(less_ctx* ctx, float* ms_total_host, int64_t* launches_host);

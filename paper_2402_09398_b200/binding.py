@@ -30,7 +30,8 @@ EXPORTED = [
 LESS_NOALLOC_MAX_ROWS = 65536
 LESS_ERR_NOALLOC_TOO_LARGE = -12
 
-KERNEL_NAMES = ["feature_map", "decode", "rowstat", "colsum", "attn_out", "select", "build", "finalize"]
+KERNEL_NAMES = ["feature_map", "decode", "rowstat", "colsum", "attn_out", "select", "build", "finalize",
+                "psi", "gather"]
 
 
 class less_config(C.Structure):

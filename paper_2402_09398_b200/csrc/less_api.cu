@@ -21,6 +21,7 @@ bool valid_config(const less_config* c) {
   if ((int64_t)c->heavy + c->recent > 65536) return false;
   if (c->max_prompt < 0 || c->max_prompt > (1 << 20)) return false;
   if (c->max_prefill_layers < 1 || c->max_prefill_layers > c->layers) return false;
+  if ((int64_t)c->batch * c->heads * c->max_prefill_layers > 65535) return false;   // grid.y of the prompt kernels
   if (c->flags & ~(uint32_t)(LESS_SCORE_NORM_SPARSE | LESS_NO_STATE)) return false;
   int64_t inst = (int64_t)c->batch * c->layers * c->heads;
   if (inst > (1 << 24)) return false;
@@ -77,6 +78,7 @@ size_t carve(const Dims& d, char* base, Arena* a) {
   t.ws_acc = (float*)take(Iw * Sp * 4);
   t.ws_slot = (int32_t*)take(Iw * Sp * 4);
   t.ws_hpart = (float*)take(Iw * kMaxSplit * (R * D + R) * 4);
+  t.ws_psi = (float*)take(Iw * Sp * R * 4);
   if (a) *a = t;
   return off;
 }

@@ -39,6 +39,7 @@ struct Arena {
   float* ws_acc;     // [Iw][Sp]    column sums
   int32_t* ws_slot;  // [Iw][Sp]    slot of a prompt token, -1 = evicted
   float* ws_hpart;   // [Iw][kMaxSplit][R*D + R]  partial H, z per token split
+  float* ws_psi;     // [Iw][Sp][R]  psi(k_j) of every prompt token
 };
 
 struct Dims {

@@ -1,0 +1,42 @@
+// Parameters shared by the prompt-phase kernels and their launchers.
+#pragma once
+
+#include "less_internal.cuh"
+
+namespace less {
+
+struct PfParams {
+  const __half* Q; const __half* K; const __half* V;   // [B, layer_count, Hd, S, D]
+  float* attn_out;                                      // same shape or null
+  Arena a;
+  const __half* w_psi1; const __half* w_psi2; const __half* w_psi3;
+  const float* psi_scale;
+  int S, Sp;                 // prompt length, workspace row stride
+  int layer0, nl;            // first model layer of this group, layers in the group
+  int lj0, layer_count;      // first input layer of this group, layers in the input
+  int B, L, Hd, N, Np, heavy, recent, Rp;
+  int nsplit, split_tokens;
+  uint32_t flags;
+};
+
+struct InstMap {
+  size_t in_row0;   // first row (of S) of this instance in Q/K/V, in rows of D
+  size_t inst;      // global instance
+  int lh;           // layer * Hd + head
+};
+
+__device__ __forceinline__ InstMap map_instance(const PfParams& p, int g) {
+  const int h = g % p.Hd;
+  const int lj = (g / p.Hd) % p.nl;
+  const int b = g / (p.Hd * p.nl);
+  InstMap m;
+  m.in_row0 = (((size_t)b * p.layer_count + p.lj0 + lj) * p.Hd + h) * (size_t)p.S;
+  m.inst = ((size_t)b * p.L + p.layer0 + lj) * p.Hd + h;
+  m.lh = (p.layer0 + lj) * p.Hd + h;
+  return m;
+}
+
+// launcher of the tensor-core state build (state_tc.cu)
+int launch_state_tc(less_ctx* c, const PfParams& p, int G, cudaStream_t s);
+
+}  // namespace less

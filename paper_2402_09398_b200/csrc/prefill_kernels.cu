@@ -7,39 +7,9 @@
 //                    partial H, z (Eq. 4, Eq. 5 summed over D_1)
 //   finalize_kernel  fixed-order sum of the partials
 #include "feature_mlp.cuh"
+#include "prefill.cuh"
 
 namespace less {
-
-struct PfParams {
-  const __half* Q; const __half* K; const __half* V;   // [B, layer_count, Hd, S, D]
-  float* attn_out;                                      // same shape or null
-  Arena a;
-  const __half* w_psi1; const __half* w_psi2; const __half* w_psi3;
-  const float* psi_scale;
-  int S, Sp;                 // prompt length, workspace row stride
-  int layer0, nl;            // first model layer of this group, layers in the group
-  int lj0, layer_count;      // first input layer of this group, layers in the input
-  int B, L, Hd, N, Np, heavy, recent, Rp;
-  int nsplit, split_tokens;
-  uint32_t flags;
-};
-
-struct InstMap {
-  size_t in_row0;   // first row (of S) of this instance in Q/K/V, in rows of D
-  size_t inst;      // global instance
-  int lh;           // layer * Hd + head
-};
-
-__device__ __forceinline__ InstMap map_instance(const PfParams& p, int g) {
-  const int h = g % p.Hd;
-  const int lj = (g / p.Hd) % p.nl;
-  const int b = g / (p.Hd * p.nl);
-  InstMap m;
-  m.in_row0 = (((size_t)b * p.layer_count + p.lj0 + lj) * p.Hd + h) * (size_t)p.S;
-  m.inst = ((size_t)b * p.L + p.layer0 + lj) * p.Hd + h;
-  m.lh = (p.layer0 + lj) * p.Hd + h;
-  return m;
-}
 
 constexpr int PF_TILE = 128;   // rows (or columns) per CTA, one per thread
 constexpr int PF_KT = 32;      // rows of the other operand staged per iteration
@@ -314,80 +284,66 @@ __global__ void __launch_bounds__(SEL_THREADS) select_kernel(PfParams p) {
   if (tid == 0 && kept_total != N) set_status(p.a.status, kStatusBounds, 3);
 }
 
-// ---- P4-P6: gather kept rows, psi for every row, partial H and z ----------- //
+// ---- P5: psi(k_j) of every prompt token (CUDA-core MLP) -------------------- //
 template <int R>
-__global__ void __launch_bounds__(FM_THREADS) build_kernel(PfParams p) {
+__global__ void __launch_bounds__(FM_THREADS) psi_kernel(PfParams p) {
   extern __shared__ float bsm[];
   float* xs = bsm;                              // [FM_BR][128]
   float* hs = xs + FM_BR * kHeadDim;
   float* part = hs + FM_BR * p.Rp;
-  __shared__ float psis[FM_BR][R];
   const int split = blockIdx.x, g = blockIdx.y, tid = threadIdx.x;
   const InstMap im = map_instance(p, g);
-  const bool use_state = !(p.flags & LESS_NO_STATE);
   const int jbeg = split * p.split_tokens, jend = min(p.S, jbeg + p.split_tokens);
-  const int32_t* slot_of = p.a.ws_slot + (size_t)g * p.Sp;
-  const float* acc = p.a.ws_acc + (size_t)g * p.Sp;
   float c1 = 1.f, c2 = 1.f;
   if (p.psi_scale) { c1 = p.psi_scale[im.lh * 2]; c2 = p.psi_scale[im.lh * 2 + 1]; }
   const __half* w1 = p.w_psi1 + (size_t)im.lh * kHeadDim * p.Rp;
   const __half* w2 = p.w_psi2 + (size_t)im.lh * p.Rp * R;
   const __half* w3 = p.w_psi3 + (size_t)im.lh * R * R;
-  float hacc[R];
-#pragma unroll
-  for (int r = 0; r < R; ++r) hacc[r] = 0.f;
-  float zacc = 0.f;
+  float* psi = p.a.ws_psi + (size_t)g * p.Sp * R;
   for (int j0 = jbeg; j0 < jend; j0 += FM_BR) {
     const int nb = min(FM_BR, jend - j0);
-    if (use_state) {
-      for (int e = tid; e < FM_BR * kHeadDim; e += FM_THREADS) {
-        const int b = e / kHeadDim, d = e % kHeadDim;
-        xs[e] = b < nb ? __half2float(p.K[(im.in_row0 + j0 + b) * kHeadDim + d]) : 0.f;
-      }
-      __syncthreads();
-      const float r = mlp_rows<R>(xs, part, hs, nb, w1, w2, w3, c1, c2, p.Rp, true);
-      const int warp = tid >> 5, lane = tid & 31;
-      if (warp < FM_BR && lane < R) psis[warp][lane] = warp < nb ? r : 0.f;
-      __syncthreads();
-    }
-    for (int b = 0; b < nb; ++b) {
-      const int j = j0 + b;
-      const int sl = slot_of[j];
-      if (sl >= 0) {
-        if (sl >= p.N) {
-          if (tid == 0) set_status(p.a.status, kStatusBounds, 4);
-          continue;
-        }
-        const size_t dst = (im.inst * (size_t)p.N + sl) * kHeadDim;
-        if (tid < 16)
-          reinterpret_cast<uint4*>(p.a.kslots + dst)[tid] =
-              __ldg(reinterpret_cast<const uint4*>(p.K + (im.in_row0 + j) * kHeadDim) + tid);
-        else if (tid < 32)
-          reinterpret_cast<uint4*>(p.a.vslots + dst)[tid - 16] =
-              __ldg(reinterpret_cast<const uint4*>(p.V + (im.in_row0 + j) * kHeadDim) + (tid - 16));
-        else if (tid == 32) {
-          p.a.pos[im.inst * (size_t)p.Np + sl] = j;
-          p.a.acc[im.inst * (size_t)p.Np + sl] = acc[j];
-        } else if (tid >= 64 && tid < 64 + R)
-          p.a.psic[(im.inst * (size_t)p.N + sl) * R + (tid - 64)] = use_state ? psis[b][tid - 64] : 0.f;
-      } else if (use_state) {
-        if (tid < kHeadDim) {
-          const float vv = __half2float(p.V[(im.in_row0 + j) * kHeadDim + tid]);
-#pragma unroll
-          for (int r = 0; r < R; ++r) hacc[r] = fmaf(psis[b][r], vv, hacc[r]);
-        } else if (tid < kHeadDim + R) {
-          zacc += psis[b][tid - kHeadDim];
-        }
-      }
+    for (int e = tid; e < FM_BR * kHeadDim; e += FM_THREADS) {
+      const int b = e / kHeadDim, d = e % kHeadDim;
+      xs[e] = b < nb ? __half2float(p.K[(im.in_row0 + j0 + b) * kHeadDim + d]) : 0.f;
     }
     __syncthreads();
+    const float r = mlp_rows<R>(xs, part, hs, nb, w1, w2, w3, c1, c2, p.Rp, true);
+    const int warp = tid >> 5, lane = tid & 31;
+    if (warp < nb && lane < R) psi[(size_t)(j0 + warp) * R + lane] = r;
   }
-  float* hp = p.a.ws_hpart + ((size_t)g * kMaxSplit + split) * (R * kHeadDim + R);
-  if (tid < kHeadDim) {
-#pragma unroll
-    for (int r = 0; r < R; ++r) hp[r * kHeadDim + tid] = hacc[r];
-  } else if (tid < kHeadDim + R) {
-    hp[R * kHeadDim + (tid - kHeadDim)] = zacc;
+}
+
+// ---- P4: kept rows go to their slots (K, V, position, score, psi) ----------- //
+constexpr int GA_THREADS = 256;
+template <int R>
+__global__ void __launch_bounds__(GA_THREADS) gather_kernel(PfParams p) {
+  const int g = blockIdx.y, tid = threadIdx.x;
+  const InstMap im = map_instance(p, g);
+  const bool use_state = !(p.flags & LESS_NO_STATE);
+  const int32_t* slot_of = p.a.ws_slot + (size_t)g * p.Sp;
+  const float* acc = p.a.ws_acc + (size_t)g * p.Sp;
+  const float* psi = p.a.ws_psi + (size_t)g * p.Sp * R;
+  // 32 threads per token: 16 move the K row, 16 the V row
+  const int sub = tid & 31;
+  for (int j = blockIdx.x * (GA_THREADS / 32) + (tid >> 5); j < p.S; j += gridDim.x * (GA_THREADS / 32)) {
+    const int sl = slot_of[j];
+    if (sl < 0) continue;
+    if (sl >= p.N) {
+      if (sub == 0) set_status(p.a.status, kStatusBounds, 4);
+      continue;
+    }
+    const size_t dst = (im.inst * (size_t)p.N + sl) * kHeadDim;
+    const size_t src = (im.in_row0 + j) * kHeadDim;
+    if (sub < 16)
+      reinterpret_cast<uint4*>(p.a.kslots + dst)[sub] = __ldg(reinterpret_cast<const uint4*>(p.K + src) + sub);
+    else
+      reinterpret_cast<uint4*>(p.a.vslots + dst)[sub - 16] =
+          __ldg(reinterpret_cast<const uint4*>(p.V + src) + (sub - 16));
+    if (sub == 0) {
+      p.a.pos[im.inst * (size_t)p.Np + sl] = j;
+      p.a.acc[im.inst * (size_t)p.Np + sl] = acc[j];
+    }
+    if (sub < R) p.a.psic[(im.inst * (size_t)p.N + sl) * R + sub] = use_state ? psi[(size_t)j * R + sub] : 0.f;
   }
 }
 
@@ -460,15 +416,26 @@ int launch_prefill_group(less_ctx* c, int layer0, int nl, int lj0, int layer_cou
     select_kernel<<<G, SEL_THREADS, 0, s>>>(p);
   }
   const size_t smem = (size_t)(FM_BR * kHeadDim + mlp_smem_floats(d.Rp)) * 4;
-  if (nsplit > 0) {
-    LaunchScope scope(c, LESS_KERNEL_BUILD, s);
+  const bool use_state = !(d.flags & LESS_NO_STATE);
+  if (nsplit > 0 && use_state) {
+    LaunchScope scope(c, LESS_KERNEL_PSI, s);
     if (d.R == 8) {
-      cudaFuncSetAttribute(build_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-      build_kernel<8><<<dim3(nsplit, G), FM_THREADS, smem, s>>>(p);
+      cudaFuncSetAttribute(psi_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+      psi_kernel<8><<<dim3(nsplit, G), FM_THREADS, smem, s>>>(p);
     } else {
-      cudaFuncSetAttribute(build_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-      build_kernel<16><<<dim3(nsplit, G), FM_THREADS, smem, s>>>(p);
+      cudaFuncSetAttribute(psi_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+      psi_kernel<16><<<dim3(nsplit, G), FM_THREADS, smem, s>>>(p);
     }
+  }
+  if (S > 0) {
+    LaunchScope scope(c, LESS_KERNEL_GATHER, s);
+    const int gx = (min(S, d.N) + 63) / 64 > 0 ? (min(S, d.N) + 63) / 64 : 1;
+    if (d.R == 8) gather_kernel<8><<<dim3(gx, G), GA_THREADS, 0, s>>>(p);
+    else gather_kernel<16><<<dim3(gx, G), GA_THREADS, 0, s>>>(p);
+  }
+  if (nsplit > 0 && use_state) {
+    const int rc = launch_state_tc(c, p, G, s);
+    if (rc != LESS_OK) return rc;
   }
   {
     LaunchScope scope(c, LESS_KERNEL_FINALIZE, s);
