@@ -36,7 +36,9 @@ __device__ __forceinline__ InstMap map_instance(const PfParams& p, int g) {
   return m;
 }
 
-// launcher of the tensor-core state build (state_tc.cu)
+// launchers of the tensor-core kernels (state_tc.cu, psi_tc.cu)
 int launch_state_tc(less_ctx* c, const PfParams& p, int G, cudaStream_t s);
+bool psi_tc_supported(const Dims& d);
+int launch_psi_tc(less_ctx* c, const PfParams& p, int G, cudaStream_t s);
 
 }  // namespace less

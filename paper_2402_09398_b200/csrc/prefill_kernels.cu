@@ -384,18 +384,17 @@ int launch_prefill_group(less_ctx* c, int layer0, int nl, int lj0, int layer_cou
   p.B = d.B; p.L = d.L; p.Hd = d.Hd; p.N = d.N; p.Np = d.Np;
   p.heavy = d.heavy; p.recent = d.recent; p.Rp = d.Rp;
   p.flags = d.flags;
-  int nsplit = 0, split_tokens = kSplitTokens;
+  // Token splits of the state build: whole 128-token tiles, long enough that the head's W1
+  // (128 KB, reloaded per split) is amortised, short enough that the grid fills the GPU.
+  const int G = d.B * nl * d.Hd;
+  int nsplit = 0, split_tokens = 1024;
   if (S > 0) {
-    nsplit = (S + kSplitTokens - 1) / kSplitTokens;
-    if (nsplit > kMaxSplit) {
-      nsplit = kMaxSplit;
-      split_tokens = (S + kMaxSplit - 1) / kMaxSplit;
-      split_tokens = (split_tokens + FM_BR - 1) / FM_BR * FM_BR;
-      nsplit = (S + split_tokens - 1) / split_tokens;
-    }
+    while (split_tokens > 128 && (long long)G * ((S + split_tokens - 1) / split_tokens) < 148) split_tokens >>= 1;
+    if ((S + split_tokens - 1) / split_tokens > kMaxSplit)
+      split_tokens = ((S + kMaxSplit - 1) / kMaxSplit + 127) / 128 * 128;
+    nsplit = (S + split_tokens - 1) / split_tokens;
   }
   p.nsplit = nsplit; p.split_tokens = split_tokens;
-  const int G = d.B * nl * d.Hd;
   if (S > 0) {
     const int tiles = (S + PF_TILE - 1) / PF_TILE;
     {
@@ -417,7 +416,10 @@ int launch_prefill_group(less_ctx* c, int layer0, int nl, int lj0, int layer_cou
   }
   const size_t smem = (size_t)(FM_BR * kHeadDim + mlp_smem_floats(d.Rp)) * 4;
   const bool use_state = !(d.flags & LESS_NO_STATE);
-  if (nsplit > 0 && use_state) {
+  if (nsplit > 0 && use_state && psi_tc_supported(d)) {
+    const int rc = launch_psi_tc(c, p, G, s);
+    if (rc != LESS_OK) return rc;
+  } else if (nsplit > 0 && use_state) {
     LaunchScope scope(c, LESS_KERNEL_PSI, s);
     if (d.R == 8) {
       cudaFuncSetAttribute(psi_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);

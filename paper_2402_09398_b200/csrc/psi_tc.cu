@@ -1,0 +1,259 @@
+// psi(k_j) of every prompt token on the tensor cores (Eq. 2):
+//     psi(k) = | c2 * gelu( c1 * gelu(k W1) W2 ) W3 |
+//
+// One CTA = one token split of one instance; W1 of the instance's head (128 KB)
+// stays in shared memory for all of the split's tiles.  Per 128-token tile:
+//   GEMM1  D1[128 x 64] = Ktile[128 x 128] * W1[:, chunk]       8 chunks of 64 hidden units,
+//                                                               D1 double-buffered in tensor memory
+//   epilogue warps: tcgen05.ld D1 -> c1 * gelu -> fp16 hi + lo -> shared memory (A operands of GEMM2;
+//                   a single fp16 rounding of the hidden layer costs ~2e-3 on individual psi vectors)
+//   GEMM2  G2[128 x 16] += (hidden_hi + hidden_lo)[128 x 64] * W2[chunk rows, :]
+//   after 8 chunks: tcgen05.ld G2 -> c2 * gelu -> W3 on CUDA cores -> abs -> psi[token][R]
+// Roles: warps 0-3 epilogue (thread = token row = tensor-memory lane), warp 4 TMA
+// producer, warp 5 MMA issuer.  Operands come in by TMA tiled loads with the 128-byte
+// swizzle (no multicast).  Every wait is bounded.
+#include "prefill.cuh"
+#include "tc_common.cuh"
+
+namespace less {
+
+constexpr int PT_WORKERS = 128;
+constexpr int PT_THREADS = PT_WORKERS + 64;
+constexpr int PT_TILE = 128;                       // tokens per tile
+constexpr int PT_CHUNK = 64;                       // hidden units per GEMM1 chunk
+constexpr int PT_KBYTES = PT_TILE * kHeadDim * 2;  // one K tile
+constexpr int PT_W2N = 16;                         // GEMM2 N (R padded to 16)
+
+struct PtShared {
+  uint64_t w1_full;
+  uint64_t k_full, k_empty;
+  uint64_t d1_full[2], d1_free[2];
+  uint64_t hid_full, hid_free;
+  uint64_t g2_full, g2_free;
+  uint32_t tmem_base;
+  int abort;
+  float w3[16 * 16];
+  float c1, c2;
+};
+
+__device__ __forceinline__ void pt_wait(uint64_t* bar, uint32_t parity, volatile int* abort, int32_t* status,
+                                        int where) {
+  if (*abort) return;
+  if (!mbar_wait(bar, parity)) {
+    *abort = 1;
+    set_status(status, kStatusTimeout, where);
+  }
+}
+
+template <int R>
+__global__ void __launch_bounds__(PT_THREADS) psi_tc_kernel(const __grid_constant__ CUtensorMap tmap_k,
+                                                            const __grid_constant__ CUtensorMap tmap_w1,
+                                                            PfParams p) {
+  extern __shared__ __align__(1024) unsigned char pt_smem[];
+  const int Rp = p.Rp;
+  const int nchunk = Rp / PT_CHUNK;
+  unsigned char* w1s = pt_smem;                                  // [nchunk][128 k][64 n]  (16 KB each)
+  unsigned char* kbuf = w1s + (size_t)nchunk * 16384;            // [2 kblocks][128 tok][64]
+  unsigned char* hid = kbuf + PT_KBYTES;                         // hi, lo: [128 tok][64 hidden] fp16, swizzled
+  unsigned char* w2s = hid + 2 * 16384;                          // [Rp/8][2 nblocks][8 k][8 n] fp16
+  PtShared* sh = reinterpret_cast<PtShared*>(w2s + (size_t)Rp * PT_W2N * 2);
+
+  const int tid = threadIdx.x, warp = tid >> 5;
+  const int split = blockIdx.x, g = blockIdx.y;
+  const InstMap im = map_instance(p, g);
+  const int jbeg = split * p.split_tokens, jend = min(p.S, jbeg + p.split_tokens);
+  const int ntiles = (jend - jbeg + PT_TILE - 1) / PT_TILE;
+
+  if (tid == 0) {
+    mbar_init(&sh->w1_full, 1);
+    mbar_init(&sh->k_full, 1);
+    mbar_init(&sh->k_empty, 1);
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(&sh->d1_full[s], 1);
+      mbar_init(&sh->d1_free[s], PT_WORKERS);
+    }
+    mbar_init(&sh->hid_full, PT_WORKERS);
+    mbar_init(&sh->hid_free, 1);
+    mbar_init(&sh->g2_full, 1);
+    mbar_init(&sh->g2_free, PT_WORKERS);
+    sh->abort = 0;
+    sh->c1 = p.psi_scale ? p.psi_scale[im.lh * 2] : 1.f;
+    sh->c2 = p.psi_scale ? p.psi_scale[im.lh * 2 + 1] : 1.f;
+    mbar_fence_init();
+  }
+  // W2 as the GEMM2 B operand (N padded to 16 with zeros), W3 as fp32
+  {
+    const __half* w2 = p.w_psi2 + (size_t)im.lh * Rp * R;
+    for (int e = tid; e < Rp * 2; e += PT_THREADS) {             // e = (k, nblock)
+      const int k = e >> 1, nb = e & 1;
+      uint4 v = make_uint4(0, 0, 0, 0);
+      if (nb * 8 < R) v = __ldg(reinterpret_cast<const uint4*>(w2 + (size_t)k * R + nb * 8));
+      *reinterpret_cast<uint4*>(w2s + (k >> 3) * 256 + nb * 128 + (k & 7) * 16) = v;
+    }
+    const __half* w3 = p.w_psi3 + (size_t)im.lh * R * R;
+    for (int e = tid; e < R * R; e += PT_THREADS) sh->w3[e] = __half2float(w3[e]);
+  }
+  if (warp == 5) tmem_alloc(&sh->tmem_base, 256);
+  fence_proxy_async_smem();
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem = sh->tmem_base;
+  volatile int* abortp = &sh->abort;
+  int32_t* status = p.a.status;
+
+  if (warp == 4) {
+    // ---------------- TMA producer ----------------
+    if (tid == PT_WORKERS) {
+      mbar_expect_tx(&sh->w1_full, (uint32_t)nchunk * 16384);
+      for (int c = 0; c < nchunk; ++c)
+        tma_load_2d(w1s + (size_t)c * 16384, &tmap_w1, c * 64, im.lh * kHeadDim, &sh->w1_full);
+      for (int i = 0; i < ntiles; ++i) {
+        pt_wait(&sh->k_empty, (i & 1) ^ 1, abortp, status, 30);
+        mbar_expect_tx(&sh->k_full, PT_KBYTES);
+        const int row = (int)(im.in_row0 + jbeg + (size_t)i * PT_TILE);
+        tma_load_2d(kbuf, &tmap_k, 0, row, &sh->k_full);
+        tma_load_2d(kbuf + PT_KBYTES / 2, &tmap_k, 64, row, &sh->k_full);
+      }
+    }
+  } else if (warp == 5) {
+    // ---------------- MMA issuer ----------------
+    if (tid == PT_WORKERS + 32) {
+      constexpr uint32_t idesc1 = idesc_f16(128, PT_CHUNK, 0, 1);   // A = K tile (K-major), B = W1 (N-major)
+      constexpr uint32_t idesc2 = idesc_f16(128, PT_W2N, 0, 1);     // A = hidden (K-major), B = W2 (N-major)
+      const uint32_t w1a = smem_u32(w1s), w2a = smem_u32(w2s), hida = smem_u32(hid);
+      pt_wait(&sh->w1_full, 0, abortp, status, 31);
+      uint32_t q = 0;                                               // chunk counter over all tiles
+      auto issue_gemm1 = [&](uint32_t ka, int c, uint32_t qq) {
+        const int b = qq & 1;
+        pt_wait(&sh->d1_free[b], ((qq >> 1) & 1) ^ 1, abortp, status, 32);
+        tc_fence_after_sync();
+#pragma unroll
+        for (int ks = 0; ks < kHeadDim / 16; ++ks) {
+          const uint64_t ad = smem_desc(ka + (ks >> 2) * (PT_KBYTES / 2) + (ks & 3) * 32, 16, 1024, kLayoutSw128);
+          const uint64_t bd = smem_desc(w1a + c * 16384 + ks * 2048, 16384, 1024, kLayoutSw128);
+          mma_f16_ss(tmem + b * PT_CHUNK, ad, bd, idesc1, ks ? 1u : 0u);
+        }
+        mma_commit(&sh->d1_full[b]);
+      };
+      for (int i = 0; i < ntiles; ++i) {
+        pt_wait(&sh->k_full, i & 1, abortp, status, 33);
+        const uint32_t ka = smem_u32(kbuf);
+        issue_gemm1(ka, 0, q);
+        for (int c = 0; c < nchunk; ++c, ++q) {
+          if (c + 1 < nchunk) issue_gemm1(ka, c + 1, q + 1);
+          else mma_commit(&sh->k_empty);                            // all GEMM1s of this tile are issued
+          if (c == 0) pt_wait(&sh->g2_free, (i & 1) ^ 1, abortp, status, 34);
+          pt_wait(&sh->hid_full, q & 1, abortp, status, 35);
+          tc_fence_after_sync();
+#pragma unroll
+          for (int ks = 0; ks < PT_CHUNK / 16; ++ks) {
+            const uint64_t bd = smem_desc(w2a + (c * (PT_CHUNK / 8) + ks * 2) * 256, 256, 128, kLayoutNone);
+            const uint64_t ah = smem_desc(hida + ks * 32, 16, 1024, kLayoutSw128);
+            const uint64_t al = smem_desc(hida + 16384 + ks * 32, 16, 1024, kLayoutSw128);
+            mma_f16_ss(tmem + 128, ah, bd, idesc2, (c | ks) ? 1u : 0u);
+            mma_f16_ss(tmem + 128, al, bd, idesc2, 1u);
+          }
+          mma_commit(&sh->hid_free);
+        }
+        mma_commit(&sh->g2_full);
+      }
+    }
+  } else {
+    // ---------------- epilogue workers: thread = token row ----------------
+    const float c1 = sh->c1, c2 = sh->c2;
+    const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
+    float* psi = p.a.ws_psi + (size_t)g * p.Sp * R;
+    unsigned char* hrow = hid + tid * 128;
+    uint32_t q = 0;
+    for (int i = 0; i < ntiles; ++i) {
+      for (int c = 0; c < nchunk; ++c, ++q) {
+        const int b = q & 1;
+        pt_wait(&sh->d1_full[b], (q >> 1) & 1, abortp, status, 36);
+        tc_fence_after_sync();
+        uint32_t acc[PT_CHUNK];
+#pragma unroll
+        for (int cc = 0; cc < PT_CHUNK / 16; ++cc) tmem_ld16(lane_addr + b * PT_CHUNK + cc * 16, acc + cc * 16);
+        tmem_ld_wait();
+        tc_fence_before_sync();
+        mbar_arrive(&sh->d1_free[b]);
+        uint32_t phi_[PT_CHUNK / 2], plo_[PT_CHUNK / 2];
+#pragma unroll
+        for (int e = 0; e < PT_CHUNK / 2; ++e) {
+          const float h0 = c1 * gelu_erf(__uint_as_float(acc[2 * e]));
+          const float h1 = c1 * gelu_erf(__uint_as_float(acc[2 * e + 1]));
+          const __half2 hh = __floats2half2_rn(h0, h1);
+          const float2 hf = __half22float2(hh);
+          const __half2 ll = __floats2half2_rn(h0 - hf.x, h1 - hf.y);
+          phi_[e] = *reinterpret_cast<const uint32_t*>(&hh);
+          plo_[e] = *reinterpret_cast<const uint32_t*>(&ll);
+        }
+        pt_wait(&sh->hid_free, (q & 1) ^ 1, abortp, status, 37);
+#pragma unroll
+        for (int ch = 0; ch < 8; ++ch) {               // 16-byte chunk ch of this row, 128-byte swizzle
+          const int off = (ch ^ (tid & 7)) << 4;
+          *reinterpret_cast<uint4*>(hrow + off) =
+              make_uint4(phi_[ch * 4], phi_[ch * 4 + 1], phi_[ch * 4 + 2], phi_[ch * 4 + 3]);
+          *reinterpret_cast<uint4*>(hrow + 16384 + off) =
+              make_uint4(plo_[ch * 4], plo_[ch * 4 + 1], plo_[ch * 4 + 2], plo_[ch * 4 + 3]);
+        }
+        fence_proxy_async_smem();
+        mbar_arrive(&sh->hid_full);
+      }
+      pt_wait(&sh->g2_full, i & 1, abortp, status, 38);
+      tc_fence_after_sync();
+      uint32_t g2[PT_W2N];
+      tmem_ld16(lane_addr + 128, g2);
+      tmem_ld_wait();
+      tc_fence_before_sync();
+      mbar_arrive(&sh->g2_free);
+      float gv[R];
+#pragma unroll
+      for (int r = 0; r < R; ++r) gv[r] = c2 * gelu_erf(__uint_as_float(g2[r]));
+      const int j = jbeg + i * PT_TILE + tid;
+      if (j < jend) {
+        float out[R];
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+          float s = 0.f;
+#pragma unroll
+          for (int rr = 0; rr < R; ++rr) s = fmaf(gv[rr], sh->w3[rr * R + r], s);
+          out[r] = fabsf(s);
+        }
+#pragma unroll
+        for (int r4 = 0; r4 < R / 4; ++r4)
+          reinterpret_cast<float4*>(psi + (size_t)j * R)[r4] =
+              make_float4(out[r4 * 4], out[r4 * 4 + 1], out[r4 * 4 + 2], out[r4 * 4 + 3]);
+      }
+    }
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 5) tmem_dealloc(tmem, 256);
+}
+
+bool psi_tc_supported(const Dims& d) { return d.Rp == 512 || d.Rp == 256 || d.Rp == 128 || d.Rp == 64; }
+
+int launch_psi_tc(less_ctx* c, const PfParams& p, int G, cudaStream_t s) {
+  const Dims& d = c->d;
+  CUtensorMap tmap_k, tmap_w1;
+  const uint64_t rows = (uint64_t)d.B * p.layer_count * d.Hd * p.S;
+  if (!make_tmap_f16_2d(&tmap_k, p.K, rows, kHeadDim, kHeadDim * 2, PT_TILE)) return LESS_ERR_CUDA;
+  if (!make_tmap_f16_2d(&tmap_w1, p.w_psi1, (uint64_t)d.L * d.Hd * kHeadDim, d.Rp, (uint64_t)d.Rp * 2, kHeadDim))
+    return LESS_ERR_CUDA;
+  const size_t smem = (size_t)(d.Rp / PT_CHUNK) * 16384 + PT_KBYTES + 2 * 16384 + (size_t)d.Rp * PT_W2N * 2 +
+                      sizeof(PtShared) + 64;
+  LaunchScope scope(c, LESS_KERNEL_PSI, s);
+  if (d.R == 8) {
+    if (cudaFuncSetAttribute(psi_tc_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+      return LESS_ERR_CUDA;
+    psi_tc_kernel<8><<<dim3(p.nsplit, G), PT_THREADS, smem, s>>>(tmap_k, tmap_w1, p);
+  } else {
+    if (cudaFuncSetAttribute(psi_tc_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+      return LESS_ERR_CUDA;
+    psi_tc_kernel<16><<<dim3(p.nsplit, G), PT_THREADS, smem, s>>>(tmap_k, tmap_w1, p);
+  }
+  return cudaGetLastError() == cudaSuccess ? LESS_OK : LESS_ERR_CUDA;
+}
+
+}  // namespace less
