@@ -67,7 +67,8 @@ __global__ void __launch_bounds__(GV_THREADS) feature_gemv_kernel(FmParams p, in
       mbar_init(&sh->aux_full[s], 1);
       mbar_init(&sh->aux_empty[s], GV_CONSUMERS / 32);
     }
-    sh->abort = 0;
+    // a CTA that starts after another one has given up skips every wait: the grid drains at once
+    sh->abort = *reinterpret_cast<volatile int32_t*>(status) != 0;
     mbar_fence_init();
   }
   __syncthreads();

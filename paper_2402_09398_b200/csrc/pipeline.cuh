@@ -52,6 +52,13 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
   return false;
 }
 
+// Error path only: a CTA that gave up on a wait lets its bulk copies and MMAs in flight land
+// (a bounded pause, ~0.25 ms) before it releases shared and tensor memory.
+__device__ __forceinline__ void drain_after_abort(volatile int* abort) {
+  if (*abort)
+    for (int i = 0; i < 64; ++i) __nanosleep(4000);
+}
+
 // 1-D bulk copy global -> shared; completes `bytes` on the barrier.
 // dst, src 16-byte aligned; bytes a multiple of 16.
 __device__ __forceinline__ void bulk_g2s(void* dst_smem, const void* src_gmem, uint32_t bytes,

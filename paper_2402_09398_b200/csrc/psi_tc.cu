@@ -76,7 +76,8 @@ __global__ void __launch_bounds__(PT_THREADS) psi_tc_kernel(const __grid_constan
     mbar_init(&sh->hid_free, 1);
     mbar_init(&sh->g2_full, 1);
     mbar_init(&sh->g2_free, PT_WORKERS);
-    sh->abort = 0;
+    // a CTA that starts after another one has given up skips every wait: the grid drains at once
+    sh->abort = *reinterpret_cast<volatile int32_t*>(p.a.status) != 0;
     sh->c1 = p.psi_scale ? p.psi_scale[im.lh * 2] : 1.f;
     sh->c2 = p.psi_scale ? p.psi_scale[im.lh * 2 + 1] : 1.f;
     mbar_fence_init();
@@ -110,6 +111,7 @@ __global__ void __launch_bounds__(PT_THREADS) psi_tc_kernel(const __grid_constan
         tma_load_2d(w1s + (size_t)c * 16384, &tmap_w1, c * 64, im.lh * kHeadDim, &sh->w1_full);
       for (int i = 0; i < ntiles; ++i) {
         pt_wait(&sh->k_empty, (i & 1) ^ 1, abortp, status, 30);
+        if (*abortp) break;                      // issue nothing more once the CTA has given up
         mbar_expect_tx(&sh->k_full, PT_KBYTES);
         const int row = (int)(im.in_row0 + jbeg + (size_t)i * PT_TILE);
         tma_load_2d(kbuf, &tmap_k, 0, row, &sh->k_full);
@@ -136,7 +138,7 @@ __global__ void __launch_bounds__(PT_THREADS) psi_tc_kernel(const __grid_constan
         }
         mma_commit(&sh->d1_full[b]);
       };
-      for (int i = 0; i < ntiles; ++i) {
+      for (int i = 0; i < ntiles && !*abortp; ++i) {
         pt_wait(&sh->k_full, i & 1, abortp, status, 33);
         const uint32_t ka = smem_u32(kbuf);
         issue_gemm1(ka, 0, q);
@@ -145,6 +147,7 @@ __global__ void __launch_bounds__(PT_THREADS) psi_tc_kernel(const __grid_constan
           else mma_commit(&sh->k_empty);                            // all GEMM1s of this tile are issued
           if (c == 0) pt_wait(&sh->g2_free, (i & 1) ^ 1, abortp, status, 34);
           pt_wait(&sh->hid_full, q & 1, abortp, status, 35);
+          if (*abortp) break;
           tc_fence_after_sync();
 #pragma unroll
           for (int ks = 0; ks < PT_CHUNK / 16; ++ks) {
@@ -166,8 +169,8 @@ __global__ void __launch_bounds__(PT_THREADS) psi_tc_kernel(const __grid_constan
     float* psi = p.a.ws_psi + (size_t)g * p.Sp * R;
     unsigned char* hrow = hid + tid * 128;
     uint32_t q = 0;
-    for (int i = 0; i < ntiles; ++i) {
-      for (int c = 0; c < nchunk; ++c, ++q) {
+    for (int i = 0; i < ntiles && !*abortp; ++i) {
+      for (int c = 0; c < nchunk && !*abortp; ++c, ++q) {
         const int b = q & 1;
         pt_wait(&sh->d1_full[b], (q >> 1) & 1, abortp, status, 36);
         tc_fence_after_sync();
@@ -227,6 +230,7 @@ __global__ void __launch_bounds__(PT_THREADS) psi_tc_kernel(const __grid_constan
       }
     }
   }
+  drain_after_abort(abortp);
   tc_fence_before_sync();
   __syncthreads();
   if (warp == 5) tmem_dealloc(tmem, 256);

@@ -68,7 +68,8 @@ __global__ void __launch_bounds__(ST_THREADS) state_tc_kernel(const __grid_const
       mbar_init(&sh->empty[s], 1);
     }
     mbar_init(&sh->done, 1);
-    sh->abort = 0;
+    // a CTA that starts after another one has given up skips every wait: the grid drains at once
+    sh->abort = *reinterpret_cast<volatile int32_t*>(p.a.status) != 0;
     mbar_fence_init();
   }
   for (int e = tid; e < 2048; e += ST_THREADS) ones[e] = __float2half(1.0f);
@@ -86,6 +87,7 @@ __global__ void __launch_bounds__(ST_THREADS) state_tc_kernel(const __grid_const
       for (int i = 0; i < ntiles; ++i) {
         const int s = i % ST_STAGES;
         st_wait(&sh->empty[s], ((i / ST_STAGES) & 1) ^ 1, abortp, p.a.status, 20);
+        if (*abortp) break;                      // issue nothing more once the CTA has given up
         mbar_expect_tx(&sh->full_v[s], ST_VBYTES);
         const int row = (int)(im.in_row0 + jbeg + (size_t)i * ST_TILE);
         tma_load_2d(vbuf + s * ST_VBYTES, &tmap_v, 0, row, &sh->full_v[s]);
@@ -103,6 +105,7 @@ __global__ void __launch_bounds__(ST_THREADS) state_tc_kernel(const __grid_const
         const uint32_t par = (i / ST_STAGES) & 1;
         st_wait(&sh->full_v[s], par, abortp, p.a.status, 21);
         st_wait(&sh->full_b[s], par, abortp, p.a.status, 22);
+        if (*abortp) break;
         tc_fence_after_sync();
         const uint32_t va = smem_u32(vbuf + s * ST_VBYTES), ba = smem_u32(bbuf + s * BBYTES);
 #pragma unroll
@@ -144,6 +147,7 @@ __global__ void __launch_bounds__(ST_THREADS) state_tc_kernel(const __grid_const
         lo[r] = __float2half_rn(x - __half2float(hi[r]));
       }
       st_wait(&sh->empty[s], ((i / ST_STAGES) & 1) ^ 1, abortp, p.a.status, 23);
+      if (*abortp) break;
       unsigned char* brow = bbuf + s * BBYTES + (tid >> 3) * B_LBO + (tid & 7) * 16;
 #pragma unroll
       for (int nb = 0; nb < R / 8; ++nb) {
@@ -176,6 +180,7 @@ __global__ void __launch_bounds__(ST_THREADS) state_tc_kernel(const __grid_const
       }
     }
   }
+  drain_after_abort(abortp);
   tc_fence_before_sync();
   __syncthreads();
   if (warp == 5) tmem_dealloc(tmem, 64);
