@@ -65,7 +65,8 @@ int launch_feature_maps(less_ctx* c, const void* q, const void* k, cudaStream_t 
   const size_t smem = (size_t)(FM_BR * kHeadDim + FM_BR * d.Rp + ndg * FM_BR * d.Rp) * 4;
   dim3 grid(d.L * d.Hd, (d.flags & LESS_NO_STATE) ? 1 : 2, (d.B + FM_BR - 1) / FM_BR);
   if (d.flags & LESS_NO_STATE) return LESS_OK;   // neither phi nor psi is used
-  if (feature_gemv_supported(d)) return launch_feature_gemv(c, p, s);
+  if (c->feature_path == 2 && feature_tc_supported(d)) return launch_feature_tc(c, p, s);
+  if (c->feature_path >= 1 && feature_gemv_supported(d)) return launch_feature_gemv(c, p, s);
   LaunchScope scope(c, LESS_KERNEL_FEATURE_MAP, s);
   if (d.R == 8) {
     cudaFuncSetAttribute(feature_map_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);

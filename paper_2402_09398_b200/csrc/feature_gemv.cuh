@@ -18,4 +18,8 @@ struct FmParams {
 bool feature_gemv_supported(const Dims& d);
 int launch_feature_gemv(less_ctx* c, const FmParams& p, cudaStream_t s);
 
+// tensor-core weight-streaming kernel (feature_tc.cu)
+bool feature_tc_supported(const Dims& d);
+int launch_feature_tc(less_ctx* c, const FmParams& p, cudaStream_t s);
+
 }  // namespace less

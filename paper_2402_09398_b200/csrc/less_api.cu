@@ -1,6 +1,7 @@
 // Host side of the C ABI: config validation, arena carving, state export /
 // import, status polling.  No device memory is allocated here.
 #include <new>
+#include <stdlib.h>
 #include <string.h>
 
 #include "less_internal.cuh"
@@ -141,6 +142,11 @@ int less_create(const less_config* cfg, const less_weights* w, void* arena, size
   c->t = 0;
   c->launches = 0;
   c->profile = false;
+  c->feature_path = 2;
+  if (const char* e = getenv("LESS_FEATURE_KERNEL")) {
+    if (!strcmp(e, "gemv")) c->feature_path = 1;
+    else if (!strcmp(e, "plain")) c->feature_path = 0;
+  }
   if (cudaGetDevice(&c->device) != cudaSuccess) { delete c; return LESS_ERR_CUDA; }
   // H_0 = 0, z_0 = 0, no live slots, clean status
   cudaError_t e = cudaMemset(c->a.H, 0, (size_t)d.I * d.R * d.D * 4);

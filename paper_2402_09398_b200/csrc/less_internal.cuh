@@ -63,6 +63,7 @@ struct less_ctx {
   int64_t t;           // tokens seen
   int64_t launches;    // kernels launched
   int device;
+  int feature_path;    // feature-map kernel: 2 tensor cores, 1 streaming GEMV, 0 plain (LESS_FEATURE_KERNEL)
   bool profile;                         // record an event pair around every launch
   std::vector<cudaEvent_t> prof_events; // start, stop, start, stop, ...
   std::vector<int> prof_kernel;         // kernel id of each pair

@@ -32,19 +32,26 @@ inline EncodeTiledFn encode_tiled_fn() {
   return fn;
 }
 
-// 2-D fp16 tensor [rows][cols] with row pitch `pitch_bytes`; box = box_rows x 64 columns
-// (128 bytes, the 128-byte swizzle span).  Out-of-range elements read as zero.
-inline bool make_tmap_f16_2d(CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols,
-                             uint64_t pitch_bytes, uint32_t box_rows) {
+// 2-D fp16 tensor [rows][cols] with row pitch `pitch_bytes`; box = box_rows x box_cols.
+// swizzle128: box_cols must be 64 (128 bytes, the 128-byte swizzle span); otherwise the box
+// lands in shared memory as plain rows of box_cols elements.  Out-of-range elements read as zero.
+inline bool make_tmap_f16_2d_box(CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols,
+                                 uint64_t pitch_bytes, uint32_t box_rows, uint32_t box_cols, bool swizzle128) {
   EncodeTiledFn fn = encode_tiled_fn();
   if (!fn) return false;
   cuuint64_t dims[2] = {cols, rows};
   cuuint64_t strides[1] = {pitch_bytes};
-  cuuint32_t box[2] = {64, box_rows};
+  cuuint32_t box[2] = {box_cols, box_rows};
   cuuint32_t estr[2] = {1, 1};
   return fn(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+            CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
+            CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// box = box_rows x 64 columns with the 128-byte swizzle
+inline bool make_tmap_f16_2d(CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols,
+                             uint64_t pitch_bytes, uint32_t box_rows) {
+  return make_tmap_f16_2d_box(m, base, rows, cols, pitch_bytes, box_rows, 64, true);
 }
 
 // ---------------------------------------------------------------------------

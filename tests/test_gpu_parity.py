@@ -231,3 +231,42 @@ def test_host_side_errors_on_gpu_box():
     assert rc == -2
     assert ctx.poll_status() == 0
     ctx.close()
+
+
+@pytest.mark.parametrize("batch,rank,hidden", [(1, 8, 512), (5, 16, 512), (17, 8, 256), (40, 16, 128),
+                                               (64, 8, 512), (130, 16, 512)])
+def test_feature_maps_over_batch_sizes(batch, rank, hidden):
+    """phi(q_t), psi(k_t) and the step built on them for token tiles of every padded
+    width (16, 32, 64, 128 tokens, and more than one tile)."""
+    import harness
+    w = small(88 + batch, batch=batch, layers=1, heads=2, prompt=40, steps=3, heavy=8, recent=8,
+              rank=rank, hidden=hidden, weight_std=0.1)
+    g = torch.Generator().manual_seed(batch)
+    psi_scale = 0.5 + torch.rand(w.layers, w.heads, 2, generator=g)
+    ctx, W = _setup(w, 0, psi_scale)
+    Q, K, V, _ = _prefill_all(ctx, w, with_out=False)
+    inst = list(range(w.instances))
+    harness.check_prefill(ctx, w, W, Q, K, V, inst, None, 0, psi_scale)
+    tf = harness.TeacherForced(ctx, w, W, inst, 0, psi_scale)
+    for s in range(w.steps):
+        tf.step(*wl.make_decode_inputs(w, s, DEV))
+    assert ctx.poll_status() == 0
+    assert tf.worst["lr_den"] > 0
+    print(batch, rank, hidden, tf.worst)
+    ctx.close()
+
+
+@pytest.mark.parametrize("path", ["gemv", "plain"])
+def test_cuda_core_feature_map_kernels(path, monkeypatch):
+    """The streaming GEMV and the plain feature-map kernels (hidden widths the tensor-core
+    kernel does not take fall back to them) against the oracle."""
+    import harness
+    monkeypatch.setenv("LESS_FEATURE_KERNEL", path)
+    w = small(97, batch=3, layers=2, heads=2, prompt=60, steps=3, heavy=8, recent=8, weight_std=0.1)
+    ctx, W = _setup(w)
+    _prefill_all(ctx, w, with_out=False)
+    tf = harness.TeacherForced(ctx, w, W, list(range(w.instances)))
+    for s in range(w.steps):
+        tf.step(*wl.make_decode_inputs(w, s, DEV))
+    assert ctx.poll_status() == 0
+    ctx.close()
