@@ -75,7 +75,7 @@ int launch_feature_maps(less_ctx* c, const void* q, const void* k, cudaStream_t 
     cudaFuncSetAttribute(feature_map_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     feature_map_kernel<16><<<grid, FM_THREADS, smem, s>>>(p);
   }
-  return cudaGetLastError() == cudaSuccess ? LESS_OK : LESS_ERR_CUDA;
+  return check_launch("feature_map_kernel");
 }
 
 // --------------------------------------------------------------------------- //
@@ -328,7 +328,7 @@ int launch_decode(less_ctx* c, const void* q, const void* k, const void* v, void
       cudaFuncSetAttribute(decode_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     decode_kernel<16><<<d.I, DEC_THREADS, smem, s>>>(p);
   }
-  return cudaGetLastError() == cudaSuccess ? LESS_OK : LESS_ERR_CUDA;
+  return check_launch("decode_kernel");
 }
 
 }  // namespace less

@@ -244,7 +244,7 @@ static int launch_one(less_ctx* c, const FmParams& p, cudaStream_t s) {
                       (size_t)(BR * d.Rp + ndg * BR * d.Rp + 8 * BR * R) * 4 + sizeof(GvShared) + 16;
   auto kern = feature_gemv_kernel<R, BR, NS>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-    return LESS_ERR_CUDA;
+    return fail_cuda("tensor map or shared memory opt-in");
   int sms = 148;
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, c->device);
   int per_sm = 1;
@@ -253,7 +253,7 @@ static int launch_one(less_ctx* c, const FmParams& p, cudaStream_t s) {
   const int grid = items < sms * per_sm ? items : sms * per_sm;
   LaunchScope scope(c, LESS_KERNEL_FEATURE_MAP, s);
   kern<<<grid, GV_THREADS, smem, s>>>(p, nchunk_b, items, c->a.status);
-  return cudaGetLastError() == cudaSuccess ? LESS_OK : LESS_ERR_CUDA;
+  return check_launch("feature_gemv_kernel");
 }
 
 bool feature_gemv_supported(const Dims& d) { return d.Rp <= 512 && d.Rp >= 64; }

@@ -177,7 +177,10 @@ __global__ void __launch_bounds__(FT_THREADS) feature_tc_kernel(
         tc_fence_after_sync();
 #pragma unroll
         for (int ks = 0; ks < FT_CHUNK / 16; ++ks) {
-          const uint64_t bd = smem_desc(w2_a + a * w2bytes + (c * FT_CHUNK + ks * 16) * 16, 128, (uint32_t)Rp * 16, kLayoutNone);
+          // R = 8 fills one 8-column block; the second block of the N = 16 tile then only has to
+          // lie inside this CTA's shared memory (its columns of D2 are never read)
+          const uint64_t bd = smem_desc(w2_a + a * w2bytes + (c * FT_CHUNK + ks * 16) * 16, 128,
+                                        R == 16 ? (uint32_t)Rp * 16 : 128u, kLayoutNone);
           const uint64_t ah = smem_desc(h_a + ks * 256, 128, 2048, kLayoutNone);
           const uint64_t al = smem_desc(h_a + hbytes + ks * 256, 128, 2048, kLayoutNone);
           mma_f16_ss(tmem + d2col, ah, bd, idesc2, (c | ks) ? 1u : 0u);
@@ -323,14 +326,16 @@ int launch_feature_tc(less_ctx* c, const FmParams& p, cudaStream_t s) {
   CUtensorMap tq, tk, tw1a, tw1b, tw2a, tw2b;
   const uint64_t lh = (uint64_t)d.L * d.Hd;
   // q, k: [B rows][L*Hd*128 columns]; a box is npad batch rows x 64 columns of one head
-  bool ok = make_tmap_f16_2d(&tq, p.x[0], d.B, lh * kHeadDim, lh * kHeadDim * 2, gm.npad) &&
-            make_tmap_f16_2d(&tk, p.x[1], d.B, lh * kHeadDim, lh * kHeadDim * 2, gm.npad) &&
-            make_tmap_f16_2d(&tw1a, p.w1[0], lh * kHeadDim, d.Rp, (uint64_t)d.Rp * 2, kHeadDim) &&
-            make_tmap_f16_2d(&tw1b, p.w1[1], lh * kHeadDim, d.Rp, (uint64_t)d.Rp * 2, kHeadDim);
+  if (!make_tmap_f16_2d(&tq, p.x[0], d.B, lh * kHeadDim, lh * kHeadDim * 2, gm.npad) ||
+      !make_tmap_f16_2d(&tk, p.x[1], d.B, lh * kHeadDim, lh * kHeadDim * 2, gm.npad))
+    return fail_cuda("tensor map of q / k");
+  if (!make_tmap_f16_2d(&tw1a, p.w1[0], lh * kHeadDim, d.Rp, (uint64_t)d.Rp * 2, kHeadDim) ||
+      !make_tmap_f16_2d(&tw1b, p.w1[1], lh * kHeadDim, d.Rp, (uint64_t)d.Rp * 2, kHeadDim))
+    return fail_cuda("tensor map of W1");
   const uint32_t wrows = d.Rp < 256 ? d.Rp : 256;
-  ok = ok && make_tmap_f16_2d_box(&tw2a, p.w2[0], lh * d.Rp, d.R, (uint64_t)d.R * 2, wrows, 8, false) &&
-       make_tmap_f16_2d_box(&tw2b, p.w2[1], lh * d.Rp, d.R, (uint64_t)d.R * 2, wrows, 8, false);
-  if (!ok) return LESS_ERR_CUDA;
+  if (!make_tmap_f16_2d_box(&tw2a, p.w2[0], lh * d.Rp, d.R, (uint64_t)d.R * 2, wrows, 8, false) ||
+      !make_tmap_f16_2d_box(&tw2b, p.w2[1], lh * d.Rp, d.R, (uint64_t)d.R * 2, wrows, 8, false))
+    return fail_cuda("tensor map of W2");
 
   int sms = 148;
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, c->device);
@@ -338,14 +343,14 @@ int launch_feature_tc(less_ctx* c, const FmParams& p, cudaStream_t s) {
   LaunchScope scope(c, LESS_KERNEL_FEATURE_MAP, s);
   if (d.R == 8) {
     if (cudaFuncSetAttribute(feature_tc_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-      return LESS_ERR_CUDA;
+      return fail_cuda("shared memory opt-in of feature_tc_kernel");
     feature_tc_kernel<8><<<grid, FT_THREADS, smem, s>>>(tq, tk, tw1a, tw1b, tw2a, tw2b, p, gm, c->a.status);
   } else {
     if (cudaFuncSetAttribute(feature_tc_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-      return LESS_ERR_CUDA;
+      return fail_cuda("shared memory opt-in of feature_tc_kernel");
     feature_tc_kernel<16><<<grid, FT_THREADS, smem, s>>>(tq, tk, tw1a, tw1b, tw2a, tw2b, p, gm, c->a.status);
   }
-  return cudaGetLastError() == cudaSuccess ? LESS_OK : LESS_ERR_CUDA;
+  return check_launch("feature_tc_kernel");
 }
 
 }  // namespace less

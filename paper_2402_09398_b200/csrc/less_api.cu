@@ -1,6 +1,7 @@
 // Host side of the C ABI: config validation, arena carving, state export /
 // import, status polling.  No device memory is allocated here.
 #include <new>
+#include <stdio.h>
 #include <stdlib.h>
 #include <string.h>
 
@@ -105,6 +106,16 @@ RecordLayout record_layout(const Dims& d) {
 }
 
 }  // namespace
+
+namespace less {
+int fail_cuda(const char* what, cudaError_t e) {
+  if (getenv("LESS_LOG")) {
+    if (e == cudaSuccess) e = cudaPeekAtLastError();
+    fprintf(stderr, "[less] %s failed: %s\n", what, e == cudaSuccess ? "(no CUDA error recorded)" : cudaGetErrorString(e));
+  }
+  return LESS_ERR_CUDA;
+}
+}  // namespace less
 
 extern "C" {
 

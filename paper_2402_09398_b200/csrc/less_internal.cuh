@@ -135,6 +135,15 @@ struct LaunchScope {
   }
 };
 
+// Host-side failure report: with LESS_LOG set in the environment, says on stderr which call
+// failed and why; always returns LESS_ERR_CUDA.
+int fail_cuda(const char* what, cudaError_t e = cudaSuccess);
+// after a kernel launch: LESS_OK, or the report above for the launch error
+inline int check_launch(const char* kernel) {
+  const cudaError_t e = cudaGetLastError();
+  return e == cudaSuccess ? LESS_OK : fail_cuda(kernel, e);
+}
+
 // launchers (host), defined in the kernel translation units
 int launch_feature_maps(less_ctx* c, const void* q, const void* k, cudaStream_t s);
 int launch_decode(less_ctx* c, const void* q, const void* k, const void* v, void* out,

@@ -444,7 +444,7 @@ int launch_prefill_group(less_ctx* c, int layer0, int nl, int lj0, int layer_cou
     if (d.R == 8) finalize_kernel<8><<<G, kHeadDim, 0, s>>>(p);
     else finalize_kernel<16><<<G, kHeadDim, 0, s>>>(p);
   }
-  return cudaGetLastError() == cudaSuccess ? LESS_OK : LESS_ERR_CUDA;
+  return check_launch("the prompt-phase kernels");
 }
 
 }  // namespace less

@@ -242,22 +242,22 @@ int launch_psi_tc(less_ctx* c, const PfParams& p, int G, cudaStream_t s) {
   const Dims& d = c->d;
   CUtensorMap tmap_k, tmap_w1;
   const uint64_t rows = (uint64_t)d.B * p.layer_count * d.Hd * p.S;
-  if (!make_tmap_f16_2d(&tmap_k, p.K, rows, kHeadDim, kHeadDim * 2, PT_TILE)) return LESS_ERR_CUDA;
+  if (!make_tmap_f16_2d(&tmap_k, p.K, rows, kHeadDim, kHeadDim * 2, PT_TILE)) return fail_cuda("tensor map of K");
   if (!make_tmap_f16_2d(&tmap_w1, p.w_psi1, (uint64_t)d.L * d.Hd * kHeadDim, d.Rp, (uint64_t)d.Rp * 2, kHeadDim))
-    return LESS_ERR_CUDA;
+    return fail_cuda("tensor map or shared memory opt-in");
   const size_t smem = (size_t)(d.Rp / PT_CHUNK) * 16384 + PT_KBYTES + 2 * 16384 + (size_t)d.Rp * PT_W2N * 2 +
                       sizeof(PtShared) + 64;
   LaunchScope scope(c, LESS_KERNEL_PSI, s);
   if (d.R == 8) {
     if (cudaFuncSetAttribute(psi_tc_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-      return LESS_ERR_CUDA;
+      return fail_cuda("tensor map or shared memory opt-in");
     psi_tc_kernel<8><<<dim3(p.nsplit, G), PT_THREADS, smem, s>>>(tmap_k, tmap_w1, p);
   } else {
     if (cudaFuncSetAttribute(psi_tc_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-      return LESS_ERR_CUDA;
+      return fail_cuda("tensor map or shared memory opt-in");
     psi_tc_kernel<16><<<dim3(p.nsplit, G), PT_THREADS, smem, s>>>(tmap_k, tmap_w1, p);
   }
-  return cudaGetLastError() == cudaSuccess ? LESS_OK : LESS_ERR_CUDA;
+  return check_launch("psi_tc_kernel");
 }
 
 }  // namespace less

@@ -190,7 +190,7 @@ int launch_state_tc(less_ctx* c, const PfParams& p, int G, cudaStream_t s) {
   const Dims& d = c->d;
   CUtensorMap tmap_v;
   const uint64_t rows = (uint64_t)d.B * p.layer_count * d.Hd * p.S;
-  if (!make_tmap_f16_2d(&tmap_v, p.V, rows, kHeadDim, kHeadDim * 2, ST_TILE)) return LESS_ERR_CUDA;
+  if (!make_tmap_f16_2d(&tmap_v, p.V, rows, kHeadDim, kHeadDim * 2, ST_TILE)) return fail_cuda("tensor map of V");
   const int NB = 2 * d.R;
   const size_t smem = (size_t)ST_STAGES * (ST_VBYTES + ST_TILE * NB * 2) + 4096 + sizeof(StShared) + 1024;
   LaunchScope scope(c, LESS_KERNEL_BUILD, s);
@@ -201,7 +201,7 @@ int launch_state_tc(less_ctx* c, const PfParams& p, int G, cudaStream_t s) {
     cudaFuncSetAttribute(state_tc_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     state_tc_kernel<16><<<dim3(p.nsplit, G), ST_THREADS, smem, s>>>(tmap_v, p);
   }
-  return cudaGetLastError() == cudaSuccess ? LESS_OK : LESS_ERR_CUDA;
+  return check_launch("state_tc_kernel");
 }
 
 }  // namespace less

@@ -270,3 +270,20 @@ def test_cuda_core_feature_map_kernels(path, monkeypatch):
         tf.step(*wl.make_decode_inputs(w, s, DEV))
     assert ctx.poll_status() == 0
     ctx.close()
+
+
+@pytest.mark.parametrize("batch,rank", [(1, 8), (3, 16)])
+def test_feature_maps_many_heads_per_cta(batch, rank):
+    """More (layer, head, map) items than SMs: every persistent CTA of the feature-map kernel
+    walks several items, so its rings and double buffers wrap."""
+    import harness
+    w = small(120 + rank, batch=batch, layers=5, heads=40, prompt=24, steps=2, heavy=6, recent=6,
+              rank=rank, weight_std=0.1)
+    ctx, W = _setup(w)
+    _prefill_all(ctx, w, with_out=False)
+    inst = list(range(0, w.instances, 3))
+    tf = harness.TeacherForced(ctx, w, W, inst)
+    for s in range(w.steps):
+        tf.step(*wl.make_decode_inputs(w, s, DEV))
+    assert ctx.poll_status() == 0
+    ctx.close()
