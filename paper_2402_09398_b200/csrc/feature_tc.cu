@@ -46,28 +46,66 @@ struct FtShared {
   __align__(16) __half w3[2][16 * 16];
 };
 
-__device__ __forceinline__ void ft_wait(uint64_t* bar, uint32_t parity, volatile int* abort, int32_t* status,
-                                        int where) {
-  if (*abort) return;
-  if (!mbar_wait(bar, parity)) {
-    *abort = 1;
-    set_status(status, kStatusTimeout, where);
-  }
-}
-
 struct FtGeom {
-  int npad;        // tokens per tile (GEMM1 N): 16, 32, 64 or 128
+  int npad;        // tokens per tile (GEMM1 N): 16, 32 or 64
   int ntile;       // token tiles per (layer-head, map)
   int items;       // work items
   int nstage;      // ring stages
   uint32_t tmem_cols;
 };
 
+
+// Work item -> (token tile, map, layer-head)
+struct FtItem { int tile, which, lh; };
+__device__ __forceinline__ FtItem ft_item(int it, int ntile) {
+  FtItem r;
+  r.tile = it % ntile;
+  r.which = (it / ntile) & 1;
+  r.lh = it / (2 * ntile);
+  return r;
+}
+
+// The producer thread of both kernels: per item the input rows, W2 and W3 into the item's aux
+// buffers, then W1 in 32-KB chunks through the ring.  Ring positions advance by counting, not by
+// dividing: this thread's instruction latency is on the critical path of the whole stream.
+template <int R>
+__device__ __forceinline__ void ft_produce(const CUtensorMap* tm_q, const CUtensorMap* tm_k, const CUtensorMap* tm_w1phi,
+                                           const CUtensorMap* tm_w1psi, const FmParams& p, const FtGeom& gm, int my_items,
+                                           int nchunk, unsigned char* xbuf, uint32_t xbytes, unsigned char* w2dst,
+                                           uint32_t w2bytes, __half* w3buf /* [2][256] */, unsigned char* ring,
+                                           uint64_t* full, uint64_t* empty, uint64_t* aux_full, uint64_t* aux_empty,
+                                           volatile int* abortp, int32_t* status) {
+  uint32_t s = 0, sph = 0;
+  for (int n = 0; n < my_items; ++n) {
+    const FtItem im = ft_item(blockIdx.x + n * gridDim.x, gm.ntile);
+    const int a = n & 1;
+    wait_or_give_up(&aux_empty[a], ((n >> 1) & 1) ^ 1, abortp, status, 40);
+    if (*abortp) return;                                 // issue nothing more once the CTA has given up
+    const CUtensorMap* tx = im.which ? tm_k : tm_q;
+    const CUtensorMap* tw1 = im.which ? tm_w1psi : tm_w1phi;
+    mbar_expect_tx(&aux_full[a], xbytes + w2bytes + (im.which ? R * R * 2 : 0));
+    unsigned char* xa = xbuf + a * xbytes;
+    tma_load_2d(xa, tx, im.lh * kHeadDim, im.tile * gm.npad, &aux_full[a]);
+    tma_load_2d(xa + xbytes / 2, tx, im.lh * kHeadDim + 64, im.tile * gm.npad, &aux_full[a]);
+    // W2 comes as one contiguous copy (a tiled load of 16-byte rows is far slower)
+    bulk_g2s(w2dst + a * w2bytes, p.w2[im.which] + (size_t)im.lh * p.Rp * R, w2bytes, &aux_full[a]);
+    if (im.which) bulk_g2s(w3buf + a * 256, p.w3 + (size_t)im.lh * R * R, R * R * 2, &aux_full[a]);
+    for (int c = 0; c < nchunk; ++c) {
+      wait_or_give_up(&empty[s], sph ^ 1, abortp, status, 41);
+      if (*abortp) return;
+      mbar_expect_tx(&full[s], FT_STAGE_BYTES);
+      unsigned char* st = ring + (size_t)s * FT_STAGE_BYTES;
+      tma_load_2d(st, tw1, c * FT_CHUNK, im.lh * kHeadDim, &full[s]);
+      tma_load_2d(st + FT_STAGE_BYTES / 2, tw1, c * FT_CHUNK + 64, im.lh * kHeadDim, &full[s]);
+      if (++s == (uint32_t)gm.nstage) { s = 0; sph ^= 1; }
+    }
+  }
+}
+
 template <int R>
 __global__ void __launch_bounds__(FT_THREADS) feature_tc_kernel(
     const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-    const __grid_constant__ CUtensorMap tm_w1phi, const __grid_constant__ CUtensorMap tm_w1psi,
-    const __grid_constant__ CUtensorMap tm_w2phi, const __grid_constant__ CUtensorMap tm_w2psi, FmParams p,
+    const __grid_constant__ CUtensorMap tm_w1phi, const __grid_constant__ CUtensorMap tm_w1psi, FmParams p,
     FtGeom gm, int32_t* status) {
   extern __shared__ __align__(1024) unsigned char ft_smem[];
   const int Rp = p.Rp, nchunk = Rp / FT_CHUNK, npad = gm.npad, nstage = gm.nstage;
@@ -78,7 +116,8 @@ __global__ void __launch_bounds__(FT_THREADS) feature_tc_kernel(
   unsigned char* xbuf = hbuf + 2 * hbytes;           // [2][xbytes]
   unsigned char* ring = xbuf + 2 * xbytes;           // [nstage][32 KB]
   unsigned char* w2buf = ring + (size_t)nstage * FT_STAGE_BYTES;   // [2][R/8 column blocks][Rp rows][16 B]
-  FtShared* sh = reinterpret_cast<FtShared*>(w2buf + 2 * w2bytes);
+  unsigned char* w2raw = w2buf + 2 * w2bytes;        // R = 16 only: [2][Rp rows][32 B] as it lies in HBM
+  FtShared* sh = reinterpret_cast<FtShared*>(w2raw + (R == 16 ? 2 * w2bytes : 0));
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   if (tid == 0) {
@@ -90,12 +129,12 @@ __global__ void __launch_bounds__(FT_THREADS) feature_tc_kernel(
       mbar_init(&sh->aux_full[s], 1);
       mbar_init(&sh->aux_empty[s], 1 + FT_EPI_WARPS);
       mbar_init(&sh->d1_full[s], 1);
-      mbar_init(&sh->d1_free[s], FT_EPI_THREADS);
+      mbar_init(&sh->d1_free[s], FT_EPI_WARPS);
     }
-    mbar_init(&sh->hid_full, FT_EPI_THREADS);
+    mbar_init(&sh->hid_full, FT_EPI_WARPS);
     mbar_init(&sh->hid_free, 1);
     mbar_init(&sh->d2_full, 1);
-    mbar_init(&sh->d2_free, FT_EPI_THREADS);
+    mbar_init(&sh->d2_free, FT_EPI_WARPS);
     // a CTA that starts after another one has given up skips every wait: the grid drains at once
     sh->abort = *reinterpret_cast<volatile int32_t*>(status) != 0;
     mbar_fence_init();
@@ -111,86 +150,71 @@ __global__ void __launch_bounds__(FT_THREADS) feature_tc_kernel(
 
   if (warp == 0) {
     // ---------------- TMA producer ----------------
-    if (lane == 0) {
-      uint32_t g = 0;
-      for (int n = 0; n < my_items; ++n) {
-        const int it = blockIdx.x + n * gridDim.x;
-        const int tile = it % gm.ntile, which = (it / gm.ntile) & 1, lh = it / (2 * gm.ntile);
-        const int a = n & 1;
-        ft_wait(&sh->aux_empty[a], ((n >> 1) & 1) ^ 1, abortp, status, 40);
-        if (*abortp) break;
-        const CUtensorMap* tx = which ? &tm_k : &tm_q;
-        const CUtensorMap* tw1 = which ? &tm_w1psi : &tm_w1phi;
-        const CUtensorMap* tw2 = which ? &tm_w2psi : &tm_w2phi;
-        mbar_expect_tx(&sh->aux_full[a], xbytes + w2bytes + (which ? R * R * 2 : 0));
-        unsigned char* xa = xbuf + a * xbytes;
-        tma_load_2d(xa, tx, lh * kHeadDim, tile * npad, &sh->aux_full[a]);
-        tma_load_2d(xa + xbytes / 2, tx, lh * kHeadDim + 64, tile * npad, &sh->aux_full[a]);
-        const int wrows = Rp < 256 ? Rp : 256;           // rows per W2 box
-        for (int nb = 0; nb < R / 8; ++nb)
-          for (int r0 = 0; r0 < Rp; r0 += wrows)
-            tma_load_2d(w2buf + a * w2bytes + ((size_t)nb * Rp + r0) * 16, tw2, nb * 8, lh * Rp + r0,
-                        &sh->aux_full[a]);
-        if (which) bulk_g2s(&sh->w3[a][0], p.w3 + (size_t)lh * R * R, R * R * 2, &sh->aux_full[a]);
-        for (int c = 0; c < nchunk; ++c, ++g) {
-          const int s = g % nstage;
-          ft_wait(&sh->empty[s], ((g / nstage) & 1) ^ 1, abortp, status, 41);
-          if (*abortp) break;
-          mbar_expect_tx(&sh->full[s], FT_STAGE_BYTES);
-          unsigned char* st = ring + (size_t)s * FT_STAGE_BYTES;
-          tma_load_2d(st, tw1, c * FT_CHUNK, lh * kHeadDim, &sh->full[s]);
-          tma_load_2d(st + FT_STAGE_BYTES / 2, tw1, c * FT_CHUNK + 64, lh * kHeadDim, &sh->full[s]);
-        }
-      }
-    }
+    if (lane == 0)
+      ft_produce<R>(&tm_q, &tm_k, &tm_w1phi, &tm_w1psi, p, gm, my_items, nchunk, xbuf, xbytes,
+                    R == 16 ? w2raw : w2buf, w2bytes, &sh->w3[0][0], ring, sh->full, sh->empty, sh->aux_full,
+                    sh->aux_empty, abortp, status);
   } else if (warp == 1) {
     // ---------------- MMA issuer ----------------
     if (lane == 0 && my_items > 0) {
       const uint32_t idesc1 = idesc_f16(128, npad, 1, 0);   // A = W1 chunk (M-major), B = x rows (K-major)
       constexpr uint32_t idesc2 = idesc_f16(128, 16, 1, 1); // A = hidden (M-major), B = W2 (N-major)
-      const uint32_t ring_a = smem_u32(ring), x_a = smem_u32(xbuf), h_a = smem_u32(hbuf), w2_a = smem_u32(w2buf);
-      const uint32_t Q = (uint32_t)my_items * nchunk;
-      auto issue_gemm1 = [&](uint32_t qq) {
-        const uint32_t n = qq / nchunk, c = qq % nchunk, a = n & 1, s = qq % nstage, b = qq & 1;
-        if (c == 0) ft_wait(&sh->aux_full[a], (n >> 1) & 1, abortp, status, 42);
-        ft_wait(&sh->full[s], (qq / nstage) & 1, abortp, status, 43);
-        ft_wait(&sh->d1_free[b], ((qq >> 1) & 1) ^ 1, abortp, status, 44);
+      // Descriptors are built once; afterwards only the start address (bits [0, 14), in 16-byte
+      // units) moves.  Every index below advances by counting: a division on this thread would
+      // sit on the critical path of the stream.
+      const uint64_t ad_ring = smem_desc(smem_u32(ring), FT_STAGE_BYTES / 2, 1024, kLayoutSw128);
+      const uint64_t bd_x = smem_desc(smem_u32(xbuf), 16, 1024, kLayoutSw128);
+      // R = 8 fills one 8-column block; the second block of the N = 16 tile then only has to
+      // lie inside this CTA's shared memory (its columns of D2 are never read)
+      const uint64_t bd_w2 = smem_desc(smem_u32(w2buf), 128, R == 16 ? (uint32_t)Rp * 16 : 128u, kLayoutNone);
+      const uint64_t ad_hi = smem_desc(smem_u32(hbuf), 128, 2048, kLayoutNone);
+      const uint64_t ad_lo = ad_hi + (uint64_t)(hbytes >> 4);
+      const uint32_t total = (uint32_t)my_items * nchunk;
+      // GEMM1 runs one chunk ahead of GEMM2
+      uint32_t s = 0, sph = 0, b1 = 0, b1ph = 0, c1 = 0, n1 = 0, issued = 0;
+      auto issue_gemm1 = [&]() {
+        const uint32_t a = n1 & 1;
+        if (c1 == 0) wait_or_give_up(&sh->aux_full[a], (n1 >> 1) & 1, abortp, status, 42);
+        wait_or_give_up(&sh->full[s], sph, abortp, status, 43);
+        wait_or_give_up(&sh->d1_free[b1], b1ph ^ 1, abortp, status, 44);
         if (*abortp) return;
         tc_fence_after_sync();
+        const uint64_t ad0 = ad_ring + (uint64_t)(s * (FT_STAGE_BYTES >> 4));
+        const uint64_t bd0 = bd_x + (uint64_t)(a * (xbytes >> 4));
+        const uint64_t bd1 = bd0 + (uint64_t)(xbytes >> 5);
 #pragma unroll
-        for (int ks = 0; ks < kHeadDim / 16; ++ks) {
-          const uint64_t ad = smem_desc(ring_a + s * FT_STAGE_BYTES + ks * 2048, FT_STAGE_BYTES / 2, 1024, kLayoutSw128);
-          const uint64_t bd =
-              smem_desc(x_a + a * xbytes + (ks >> 2) * (xbytes / 2) + (ks & 3) * 32, 16, 1024, kLayoutSw128);
-          mma_f16_ss(tmem + b * npad, ad, bd, idesc1, ks ? 1u : 0u);
-        }
+        for (int ks = 0; ks < kHeadDim / 16; ++ks)
+          mma_f16_ss(tmem + b1 * npad, ad0 + (uint64_t)(ks * (2048 >> 4)), (ks < 4 ? bd0 : bd1) + (uint64_t)((ks & 3) * 2),
+                     idesc1, ks ? 1u : 0u);
         mma_commit(&sh->empty[s]);
-        mma_commit(&sh->d1_full[b]);
+        mma_commit(&sh->d1_full[b1]);
+        if (++s == (uint32_t)nstage) { s = 0; sph ^= 1; }
+        if (b1 ^= 1, b1 == 0) b1ph ^= 1;
+        if (++c1 == (uint32_t)nchunk) { c1 = 0; ++n1; }
+        ++issued;
       };
-      issue_gemm1(0);
-      for (uint32_t q = 0; q < Q && !*abortp; ++q) {
-        if (q + 1 < Q) issue_gemm1(q + 1);
-        const uint32_t n = q / nchunk, c = q % nchunk, a = n & 1;
-        if (c == 0) ft_wait(&sh->d2_free, (n & 1) ^ 1, abortp, status, 45);
-        ft_wait(&sh->hid_full, q & 1, abortp, status, 46);
-        if (*abortp) break;
-        tc_fence_after_sync();
+      issue_gemm1();
+      uint32_t hph = 0;
+      for (uint32_t n = 0; n < (uint32_t)my_items && !*abortp; ++n) {
+        const uint32_t a = n & 1;
+        for (uint32_t c = 0; c < (uint32_t)nchunk; ++c) {
+          if (issued < total) issue_gemm1();
+          if (c == 0) wait_or_give_up(&sh->d2_free, (n & 1) ^ 1, abortp, status, 45);
+          wait_or_give_up(&sh->hid_full, hph, abortp, status, 46);
+          if (*abortp) break;
+          hph ^= 1;
+          tc_fence_after_sync();
+          const uint64_t bd0 = bd_w2 + (uint64_t)(a * (w2bytes >> 4) + c * (FT_CHUNK * 16 >> 4));
 #pragma unroll
-        for (int ks = 0; ks < FT_CHUNK / 16; ++ks) {
-          // R = 8 fills one 8-column block; the second block of the N = 16 tile then only has to
-          // lie inside this CTA's shared memory (its columns of D2 are never read)
-          const uint64_t bd = smem_desc(w2_a + a * w2bytes + (c * FT_CHUNK + ks * 16) * 16, 128,
-                                        R == 16 ? (uint32_t)Rp * 16 : 128u, kLayoutNone);
-          const uint64_t ah = smem_desc(h_a + ks * 256, 128, 2048, kLayoutNone);
-          const uint64_t al = smem_desc(h_a + hbytes + ks * 256, 128, 2048, kLayoutNone);
-          mma_f16_ss(tmem + d2col, ah, bd, idesc2, (c | ks) ? 1u : 0u);
-          mma_f16_ss(tmem + d2col, al, bd, idesc2, 1u);
+          for (int ks = 0; ks < FT_CHUNK / 16; ++ks) {
+            mma_f16_ss(tmem + d2col, ad_hi + (uint64_t)(ks * 16), bd0 + (uint64_t)(ks * 16), idesc2, (c | ks) ? 1u : 0u);
+            mma_f16_ss(tmem + d2col, ad_lo + (uint64_t)(ks * 16), bd0 + (uint64_t)(ks * 16), idesc2, 1u);
+          }
+          mma_commit(&sh->hid_free);
         }
-        mma_commit(&sh->hid_free);
-        if (c == (uint32_t)nchunk - 1) {
-          mma_commit(&sh->d2_full);
-          mma_commit(&sh->aux_empty[a]);
-        }
+        if (*abortp) break;
+        mma_commit(&sh->d2_full);
+        mma_commit(&sh->aux_empty[a]);
       }
     }
   } else {
@@ -209,9 +233,18 @@ __global__ void __launch_bounds__(FT_THREADS) feature_tc_kernel(
       const int b0 = tile * npad, nb = min(npad, p.B - b0), nblk = (nb + 7) >> 3;
       float c1 = 1.f, c2 = 1.f;
       if (which && p.psi_scale) { c1 = __ldg(p.psi_scale + lh * 2); c2 = __ldg(p.psi_scale + lh * 2 + 1); }
+      wait_or_give_up(&sh->aux_full[a], (n >> 1) & 1, abortp, status, 50);
+      if (R == 16) {
+        // 32-byte rows -> two blocks of 16-byte rows; the GEMM2s that read this buffer two items
+        // ago are complete (their D2 was read), and the first hid_full arrival below publishes it
+        const uint4* src = reinterpret_cast<const uint4*>(w2raw + a * w2bytes);
+        unsigned char* dst = w2buf + a * w2bytes;
+        for (int u = tid - 64; u < Rp * 2; u += FT_EPI_THREADS)
+          *reinterpret_cast<uint4*>(dst + ((size_t)(u & 1) * Rp + (u >> 1)) * 16) = src[u];
+      }
       for (int c = 0; c < nchunk && !*abortp; ++c, ++q) {
         const int b = q & 1;
-        ft_wait(&sh->d1_full[b], (q >> 1) & 1, abortp, status, 47);
+        wait_or_give_up(&sh->d1_full[b], (q >> 1) & 1, abortp, status, 47);
         tc_fence_after_sync();
         // this warp's token blocks: hf, hf + 2, ...   (at most 8 of the 16 blocks of a 128-token tile)
         uint32_t acc[8][8];
@@ -222,7 +255,7 @@ __global__ void __launch_bounds__(FT_THREADS) feature_tc_kernel(
         }
         tmem_ld_wait();
         tc_fence_before_sync();
-        mbar_arrive(&sh->d1_free[b]);
+        mbar_arrive_warp(&sh->d1_free[b]);
         uint4 hi[8], lo[8];
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
@@ -231,8 +264,9 @@ __global__ void __launch_bounds__(FT_THREADS) feature_tc_kernel(
             uint32_t ph[4], pl[4];
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
-              const float h0 = c1 * gelu_erf(__uint_as_float(acc[i][2 * e]));
-              const float h1 = c1 * gelu_erf(__uint_as_float(acc[i][2 * e + 1]));
+              // columns past the last token hold products with zero-filled rows: no GELU spent on them
+              const float h0 = blk * 8 + 2 * e < nb ? c1 * gelu_erf(__uint_as_float(acc[i][2 * e])) : 0.f;
+              const float h1 = blk * 8 + 2 * e + 1 < nb ? c1 * gelu_erf(__uint_as_float(acc[i][2 * e + 1])) : 0.f;
               const __half2 hh = __floats2half2_rn(h0, h1);
               const float2 hf2 = __half22float2(hh);
               const __half2 ll = __floats2half2_rn(h0 - hf2.x, h1 - hf2.y);
@@ -243,7 +277,7 @@ __global__ void __launch_bounds__(FT_THREADS) feature_tc_kernel(
             lo[i] = make_uint4(pl[0], pl[1], pl[2], pl[3]);
           }
         }
-        ft_wait(&sh->hid_free, (q & 1) ^ 1, abortp, status, 48);
+        wait_or_give_up(&sh->hid_free, (q & 1) ^ 1, abortp, status, 48);
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
           const int blk = hf + 2 * i;
@@ -253,11 +287,11 @@ __global__ void __launch_bounds__(FT_THREADS) feature_tc_kernel(
           }
         }
         fence_proxy_async_smem();
-        mbar_arrive(&sh->hid_full);
+        mbar_arrive_warp(&sh->hid_full);
       }
       if (*abortp) break;
       // ---- layer 2 result: token = accumulator lane ----
-      ft_wait(&sh->d2_full, n & 1, abortp, status, 49);
+      wait_or_give_up(&sh->d2_full, n & 1, abortp, status, 49);
       tc_fence_after_sync();
       const bool mine = hf == 0 && quad * 32 < nb;         // warp-uniform
       uint32_t g2[16];
@@ -267,7 +301,7 @@ __global__ void __launch_bounds__(FT_THREADS) feature_tc_kernel(
         tmem_ld_wait();
       }
       tc_fence_before_sync();
-      mbar_arrive(&sh->d2_free);
+      mbar_arrive_warp(&sh->d2_free);
       if (mine && j < nb) {
         float gv[R], out[R];
 #pragma unroll
@@ -300,19 +334,239 @@ __global__ void __launch_bounds__(FT_THREADS) feature_tc_kernel(
   if (warp == 1) tmem_dealloc(tmem, gm.tmem_cols);
 }
 
+// --------------------------------------------------------------------------- //
+// Small batches (at most 8 tokens per head): the same weight stream and the same
+// transposed GEMM1, but layer 2 stays on CUDA cores.  A tensor-core instruction
+// with a 128-row operand costs about a hundred cycles however narrow it is, and
+// GEMM2 needs 64 of them per item (hi and lo halves of 512 hidden units); with a
+// handful of tokens the epilogue thread that owns hidden unit j multiplies its
+// activations with row j of W2 in fp32 registers instead, and one shuffle
+// reduction per item replaces the second GEMM.
+// --------------------------------------------------------------------------- //
+constexpr int FS_BUFS = 4;        // D1^T buffers in tensor memory (16 columns each)
+constexpr int FS_NPAD = 16;
+constexpr int FS_XBYTES = FS_NPAD * 256;
+
+struct FsShared {
+  uint64_t full[FT_MAX_STAGES], empty[FT_MAX_STAGES];
+  uint64_t aux_full[2], aux_empty[2];
+  uint64_t d1_full[FS_BUFS], d1_free[FS_BUFS];
+  uint32_t tmem_base;
+  int abort;
+  __align__(16) __half w3[2][16 * 16];
+  float red[2][FT_EPI_WARPS][8 * 16];   // per item parity, per warp: partial layer-2 sums [token][r]
+  float g[2][8 * 16];                   // c2 * gelu(layer-2 sums)
+};
+
+__device__ __forceinline__ void epi_sync() { asm volatile("bar.sync 1, %0;" ::"n"(FT_EPI_THREADS) : "memory"); }
+
+// Sum over the 32 lanes of V values per lane, V a power of two: every exchange halves the
+// values a lane keeps, so it costs about V shuffles instead of 5 V.  Afterwards v[0 .. count)
+// are complete sums of the indices base .. base + count, and lanes with `owner` false hold copies.
+template <int V>
+__device__ __forceinline__ void lane_reduce_scatter(float (&v)[V], int lane, int& base, int& count, bool& owner) {
+  int n = V;
+  base = 0;
+  owner = true;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const bool up = (lane & o) != 0;
+    if (n > 1) {
+      n >>= 1;
+#pragma unroll
+      for (int i = 0; i < V / 2; ++i) {
+        if (i < n) {
+          const float keep = up ? v[i + n] : v[i];
+          const float send = up ? v[i] : v[i + n];
+          v[i] = keep + __shfl_xor_sync(0xffffffffu, send, o);
+        }
+      }
+      if (up) base += n;
+    } else {
+      v[0] += __shfl_xor_sync(0xffffffffu, v[0], o);
+      if (up) owner = false;
+    }
+  }
+  count = n;
+}
+
+template <int R, int NT>
+__global__ void __launch_bounds__(FT_THREADS) feature_tc_small_kernel(
+    const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+    const __grid_constant__ CUtensorMap tm_w1phi, const __grid_constant__ CUtensorMap tm_w1psi, FmParams p,
+    FtGeom gm, int32_t* status) {
+  extern __shared__ __align__(1024) unsigned char ft_smem[];
+  constexpr int V = NT * R;
+  const int Rp = p.Rp, nchunk = Rp / FT_CHUNK, nstage = gm.nstage;
+  const uint32_t w2bytes = (uint32_t)Rp * R * 2;
+  unsigned char* xbuf = ft_smem;                                   // [2][16 rows x 2 halves x 128 B]
+  unsigned char* ring = xbuf + 2 * FS_XBYTES;                      // [nstage][32 KB]
+  unsigned char* w2raw = ring + (size_t)nstage * FT_STAGE_BYTES;   // [2][Rp rows][R] as it lies in HBM
+  FsShared* sh = reinterpret_cast<FsShared*>(w2raw + 2 * w2bytes);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  if (tid == 0) {
+    for (int s = 0; s < nstage; ++s) {
+      mbar_init(&sh->full[s], 1);
+      mbar_init(&sh->empty[s], 1);
+    }
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(&sh->aux_full[s], 1);
+      mbar_init(&sh->aux_empty[s], 1 + FT_EPI_WARPS);
+    }
+    for (int s = 0; s < FS_BUFS; ++s) {
+      mbar_init(&sh->d1_full[s], 1);
+      mbar_init(&sh->d1_free[s], FT_EPI_WARPS / 2);
+    }
+    sh->abort = *reinterpret_cast<volatile int32_t*>(status) != 0;
+    mbar_fence_init();
+  }
+  if (warp == 1) tmem_alloc(&sh->tmem_base, FS_BUFS * FS_NPAD);
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem = sh->tmem_base;
+  volatile int* abortp = &sh->abort;
+  const int my_items = blockIdx.x < gm.items ? (gm.items - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
+
+  if (warp == 0) {
+    // ---------------- TMA producer ----------------
+    if (lane == 0)
+      ft_produce<R>(&tm_q, &tm_k, &tm_w1phi, &tm_w1psi, p, gm, my_items, nchunk, xbuf, FS_XBYTES, w2raw, w2bytes,
+                    &sh->w3[0][0], ring, sh->full, sh->empty, sh->aux_full, sh->aux_empty, abortp, status);
+  } else if (warp == 1) {
+    // ---------------- MMA issuer: GEMM1 only ----------------
+    if (lane == 0) {
+      constexpr uint32_t idesc1 = idesc_f16(128, FS_NPAD, 1, 0);
+      const uint64_t ad_ring = smem_desc(smem_u32(ring), FT_STAGE_BYTES / 2, 1024, kLayoutSw128);
+      const uint64_t bd_x = smem_desc(smem_u32(xbuf), 16, 1024, kLayoutSw128);
+      uint32_t s = 0, sph = 0, b = 0, bph = 0;      // ring stage / D1 buffer and their phases: counted, never divided
+      for (int n = 0; n < my_items; ++n) {
+        const uint32_t a = n & 1;
+        wait_or_give_up(&sh->aux_full[a], (n >> 1) & 1, abortp, status, 62);
+        const uint64_t bd0 = bd_x + (uint64_t)(a * (FS_XBYTES >> 4));
+        const uint64_t bd1 = bd0 + (uint64_t)(FS_XBYTES >> 5);
+        for (int c = 0; c < nchunk; ++c) {
+          wait_or_give_up(&sh->full[s], sph, abortp, status, 63);
+          wait_or_give_up(&sh->d1_free[b], bph ^ 1, abortp, status, 64);
+          if (*abortp) break;
+          tc_fence_after_sync();
+          const uint64_t ad0 = ad_ring + (uint64_t)(s * (FT_STAGE_BYTES >> 4));
+#pragma unroll
+          for (int ks = 0; ks < kHeadDim / 16; ++ks)
+            mma_f16_ss(tmem + b * FS_NPAD, ad0 + (uint64_t)(ks * (2048 >> 4)),
+                       (ks < 4 ? bd0 : bd1) + (uint64_t)((ks & 3) * 2), idesc1, ks ? 1u : 0u);
+          mma_commit(&sh->empty[s]);
+          mma_commit(&sh->d1_full[b]);
+          if (++s == (uint32_t)nstage) { s = 0; sph ^= 1; }
+          if (++b == FS_BUFS) { b = 0; bph ^= 1; }
+        }
+        if (*abortp) break;
+        mma_commit(&sh->aux_empty[a]);
+      }
+    }
+  } else {
+    // ---------------- epilogue warps ----------------
+    // No early exit here: the warps meet at named barriers, so after a timed-out wait they keep
+    // walking their items (every later wait returns at once) and the CTA ends normally.
+    const int ew = warp - 2, quad = warp & 3, hf = ew >> 2;
+    const int j = quad * 32 + lane;            // hidden unit inside a chunk = accumulator lane
+    const int et = tid - 64;                   // 0..255
+    const uint32_t lane_addr = tmem + ((uint32_t)(quad * 32) << 16);
+    for (int n = 0; n < my_items; ++n) {
+      const int it = blockIdx.x + n * gridDim.x;
+      const int tile = it % gm.ntile, which = (it / gm.ntile) & 1, lh = it / (2 * gm.ntile);
+      const int a = n & 1;
+      const int b0 = tile * FS_NPAD, nb = min(NT, p.B - b0);
+      float c1 = 1.f, c2 = 1.f;
+      if (which && p.psi_scale) { c1 = __ldg(p.psi_scale + lh * 2); c2 = __ldg(p.psi_scale + lh * 2 + 1); }
+      wait_or_give_up(&sh->aux_full[a], (n >> 1) & 1, abortp, status, 65);
+      float part[V];
+#pragma unroll
+      for (int e = 0; e < V; ++e) part[e] = 0.f;
+      // the two warps of a lane quadrant take alternate chunks
+      for (int c = hf; c < nchunk; c += 2) {
+        const uint32_t q = (uint32_t)n * nchunk + c, b = q % FS_BUFS;
+        wait_or_give_up(&sh->d1_full[b], (q / FS_BUFS) & 1, abortp, status, 66);
+        tc_fence_after_sync();
+        uint32_t acc[8];
+        tmem_ld8(lane_addr + b * FS_NPAD, acc);
+        tmem_ld_wait();
+        tc_fence_before_sync();
+        mbar_arrive_warp(&sh->d1_free[b]);
+        float w[R];
+        const uint4* wr = reinterpret_cast<const uint4*>(w2raw + a * w2bytes + (size_t)(c * FT_CHUNK + j) * R * 2);
+#pragma unroll
+        for (int r8 = 0; r8 < R / 8; ++r8) half8_to_float(wr[r8], w + r8 * 8);
+#pragma unroll
+        for (int t = 0; t < NT; ++t) {
+          const float h = t < nb ? c1 * gelu_erf(__uint_as_float(acc[t])) : 0.f;
+#pragma unroll
+          for (int r = 0; r < R; ++r) part[t * R + r] = fmaf(h, w[r], part[t * R + r]);
+        }
+      }
+      int base, count;
+      bool owner;
+      lane_reduce_scatter<V>(part, lane, base, count, owner);
+      float* red = &sh->red[n & 1][ew][0];
+      if (owner) {
+#pragma unroll
+        for (int i = 0; i < (V >= 32 ? V / 32 : 1); ++i) red[base + i] = part[i];
+      }
+      epi_sync();
+      float gv = 0.f;
+      if (et < V) {
+        float sum = 0.f;
+#pragma unroll
+        for (int wq = 0; wq < FT_EPI_WARPS; ++wq) sum += sh->red[n & 1][wq][et];   // fixed order
+        gv = c2 * gelu_erf(sum);
+      }
+      const int t = et / R, r = et % R;
+      if (which) {
+        if (et < V) sh->g[n & 1][et] = gv;
+        epi_sync();
+        if (et < V) {
+          const __half* w3 = &sh->w3[a][0];
+          float sacc = 0.f;
+#pragma unroll
+          for (int rr = 0; rr < R; ++rr) sacc = fmaf(sh->g[n & 1][t * R + rr], __half2float(w3[rr * R + r]), sacc);
+          gv = sacc;
+        }
+      }
+      if (et < V && t < nb) p.out[which][((size_t)(b0 + t) * p.L * p.Hd + lh) * R + r] = fabsf(gv);
+      // this warp is done with the item's W2 and W3
+      mbar_arrive_warp(&sh->aux_empty[a]);
+    }
+  }
+  drain_after_abort(abortp);
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 1) tmem_dealloc(tmem, FS_BUFS * FS_NPAD);
+}
+
+template <int R, int NT>
+static int launch_small(less_ctx* c, const FmParams& p, const FtGeom& gm, const CUtensorMap& tq, const CUtensorMap& tk,
+                        const CUtensorMap& tw1a, const CUtensorMap& tw1b, size_t smem, int grid, cudaStream_t s) {
+  auto kern = feature_tc_small_kernel<R, NT>;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+    return fail_cuda("shared memory opt-in of feature_tc_small_kernel");
+  kern<<<grid, FT_THREADS, smem, s>>>(tq, tk, tw1a, tw1b, p, gm, c->a.status);
+  return check_launch("feature_tc_small_kernel");
+}
+
 bool feature_tc_supported(const Dims& d) {
   return (d.Rp == 128 || d.Rp == 256 || d.Rp == 512) && encode_tiled_fn() != nullptr;
 }
 
 static size_t ft_fixed_smem(const Dims& d, int npad) {
-  return (size_t)4 * npad * 256 + (size_t)2 * d.Rp * d.R * 2 + sizeof(FtShared) + 1024;
+  return (size_t)4 * npad * 256 + (size_t)(d.R == 16 ? 4 : 2) * d.Rp * d.R * 2 + sizeof(FtShared) + 1024;
 }
 
 int launch_feature_tc(less_ctx* c, const FmParams& p, cudaStream_t s) {
   const Dims& d = c->d;
   FtGeom gm;
-  const int bt = d.B < 128 ? d.B : 128;
-  gm.npad = bt <= 16 ? 16 : bt <= 32 ? 32 : bt <= 64 ? 64 : 128;
+  // token tiles of at most 64: larger tiles leave too little shared memory for the weight ring
+  gm.npad = d.B <= 16 ? 16 : d.B <= 32 ? 32 : 64;
   gm.ntile = (d.B + gm.npad - 1) / gm.npad;
   gm.items = d.L * d.Hd * 2 * gm.ntile;
   const size_t fixed = ft_fixed_smem(d, gm.npad);
@@ -323,7 +577,7 @@ int launch_feature_tc(less_ctx* c, const FmParams& p, cudaStream_t s) {
   gm.tmem_cols = need <= 64 ? 64 : need <= 128 ? 128 : need <= 256 ? 256 : 512;
   const size_t smem = fixed + (size_t)gm.nstage * FT_STAGE_BYTES;
 
-  CUtensorMap tq, tk, tw1a, tw1b, tw2a, tw2b;
+  CUtensorMap tq, tk, tw1a, tw1b;
   const uint64_t lh = (uint64_t)d.L * d.Hd;
   // q, k: [B rows][L*Hd*128 columns]; a box is npad batch rows x 64 columns of one head
   if (!make_tmap_f16_2d(&tq, p.x[0], d.B, lh * kHeadDim, lh * kHeadDim * 2, gm.npad) ||
@@ -332,23 +586,35 @@ int launch_feature_tc(less_ctx* c, const FmParams& p, cudaStream_t s) {
   if (!make_tmap_f16_2d(&tw1a, p.w1[0], lh * kHeadDim, d.Rp, (uint64_t)d.Rp * 2, kHeadDim) ||
       !make_tmap_f16_2d(&tw1b, p.w1[1], lh * kHeadDim, d.Rp, (uint64_t)d.Rp * 2, kHeadDim))
     return fail_cuda("tensor map of W1");
-  const uint32_t wrows = d.Rp < 256 ? d.Rp : 256;
-  if (!make_tmap_f16_2d_box(&tw2a, p.w2[0], lh * d.Rp, d.R, (uint64_t)d.R * 2, wrows, 8, false) ||
-      !make_tmap_f16_2d_box(&tw2b, p.w2[1], lh * d.Rp, d.R, (uint64_t)d.R * 2, wrows, 8, false))
-    return fail_cuda("tensor map of W2");
-
   int sms = 148;
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, c->device);
   const int grid = gm.items < sms ? gm.items : sms;
   LaunchScope scope(c, LESS_KERNEL_FEATURE_MAP, s);
+  if (d.B <= 8) {
+    const size_t fx = (size_t)2 * FS_XBYTES + (size_t)2 * d.Rp * d.R * 2 + sizeof(FsShared) + 256;
+    const int nsm = (int)((FT_SMEM_LIMIT - fx) / FT_STAGE_BYTES);
+    gm.nstage = nsm > FT_MAX_STAGES ? FT_MAX_STAGES : nsm;
+    const size_t sm = fx + (size_t)gm.nstage * FT_STAGE_BYTES;
+    const int nt = d.B <= 1 ? 1 : d.B <= 2 ? 2 : d.B <= 4 ? 4 : 8;
+    if (d.R == 8) {
+      if (nt == 1) return launch_small<8, 1>(c, p, gm, tq, tk, tw1a, tw1b, sm, grid, s);
+      if (nt == 2) return launch_small<8, 2>(c, p, gm, tq, tk, tw1a, tw1b, sm, grid, s);
+      if (nt == 4) return launch_small<8, 4>(c, p, gm, tq, tk, tw1a, tw1b, sm, grid, s);
+      return launch_small<8, 8>(c, p, gm, tq, tk, tw1a, tw1b, sm, grid, s);
+    }
+    if (nt == 1) return launch_small<16, 1>(c, p, gm, tq, tk, tw1a, tw1b, sm, grid, s);
+    if (nt == 2) return launch_small<16, 2>(c, p, gm, tq, tk, tw1a, tw1b, sm, grid, s);
+    if (nt == 4) return launch_small<16, 4>(c, p, gm, tq, tk, tw1a, tw1b, sm, grid, s);
+    return launch_small<16, 8>(c, p, gm, tq, tk, tw1a, tw1b, sm, grid, s);
+  }
   if (d.R == 8) {
     if (cudaFuncSetAttribute(feature_tc_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
       return fail_cuda("shared memory opt-in of feature_tc_kernel");
-    feature_tc_kernel<8><<<grid, FT_THREADS, smem, s>>>(tq, tk, tw1a, tw1b, tw2a, tw2b, p, gm, c->a.status);
+    feature_tc_kernel<8><<<grid, FT_THREADS, smem, s>>>(tq, tk, tw1a, tw1b, p, gm, c->a.status);
   } else {
     if (cudaFuncSetAttribute(feature_tc_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
       return fail_cuda("shared memory opt-in of feature_tc_kernel");
-    feature_tc_kernel<16><<<grid, FT_THREADS, smem, s>>>(tq, tk, tw1a, tw1b, tw2a, tw2b, p, gm, c->a.status);
+    feature_tc_kernel<16><<<grid, FT_THREADS, smem, s>>>(tq, tk, tw1a, tw1b, p, gm, c->a.status);
   }
   return check_launch("feature_tc_kernel");
 }

@@ -33,6 +33,14 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 
+// One arrival for a whole warp: every lane has finished (and fenced) its own accesses, the
+// warp converges, lane 0 arrives.  Barriers counted in warps avoid hundreds of serialised
+// arrivals on one shared-memory word.
+__device__ __forceinline__ void mbar_arrive_warp(uint64_t* bar) {
+  __syncwarp();
+  if ((threadIdx.x & 31) == 0) mbar_arrive(bar);
+}
+
 __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
@@ -50,6 +58,19 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
   for (uint32_t i = 0; i < kSpinLimit; ++i)
     if (mbar_try_wait(bar, parity)) return true;
   return false;
+}
+
+// The wait every pipeline role uses.  Fast path: the phase is already complete.  Otherwise the
+// waiter leaves at once if its CTA has given up; a wait that runs out makes the CTA give up and
+// records where in the device status word (first writer wins), so that nothing can hang.
+__device__ __forceinline__ void wait_or_give_up(uint64_t* bar, uint32_t parity, volatile int* abort, int32_t* status,
+                                                int where) {
+  if (mbar_try_wait(bar, parity)) return;
+  if (*abort) return;
+  if (!mbar_wait(bar, parity)) {
+    *abort = 1;
+    if (atomicCAS(status, 0, 1 /* timeout */) == 0) status[1] = where;
+  }
 }
 
 // Error path only: a CTA that gave up on a wait lets its bulk copies and MMAs in flight land

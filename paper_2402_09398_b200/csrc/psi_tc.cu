@@ -70,12 +70,12 @@ __global__ void __launch_bounds__(PT_THREADS) psi_tc_kernel(const __grid_constan
     mbar_init(&sh->k_empty, 1);
     for (int s = 0; s < 2; ++s) {
       mbar_init(&sh->d1_full[s], 1);
-      mbar_init(&sh->d1_free[s], PT_WORKERS);
+      mbar_init(&sh->d1_free[s], PT_WORKERS / 32);
     }
-    mbar_init(&sh->hid_full, PT_WORKERS);
+    mbar_init(&sh->hid_full, PT_WORKERS / 32);
     mbar_init(&sh->hid_free, 1);
     mbar_init(&sh->g2_full, 1);
-    mbar_init(&sh->g2_free, PT_WORKERS);
+    mbar_init(&sh->g2_free, PT_WORKERS / 32);
     // a CTA that starts after another one has given up skips every wait: the grid drains at once
     sh->abort = *reinterpret_cast<volatile int32_t*>(p.a.status) != 0;
     sh->c1 = p.psi_scale ? p.psi_scale[im.lh * 2] : 1.f;
@@ -179,7 +179,7 @@ __global__ void __launch_bounds__(PT_THREADS) psi_tc_kernel(const __grid_constan
         for (int cc = 0; cc < PT_CHUNK / 16; ++cc) tmem_ld16(lane_addr + b * PT_CHUNK + cc * 16, acc + cc * 16);
         tmem_ld_wait();
         tc_fence_before_sync();
-        mbar_arrive(&sh->d1_free[b]);
+        mbar_arrive_warp(&sh->d1_free[b]);
         uint32_t phi_[PT_CHUNK / 2], plo_[PT_CHUNK / 2];
 #pragma unroll
         for (int e = 0; e < PT_CHUNK / 2; ++e) {
@@ -201,7 +201,7 @@ __global__ void __launch_bounds__(PT_THREADS) psi_tc_kernel(const __grid_constan
               make_uint4(plo_[ch * 4], plo_[ch * 4 + 1], plo_[ch * 4 + 2], plo_[ch * 4 + 3]);
         }
         fence_proxy_async_smem();
-        mbar_arrive(&sh->hid_full);
+        mbar_arrive_warp(&sh->hid_full);
       }
       pt_wait(&sh->g2_full, i & 1, abortp, status, 38);
       tc_fence_after_sync();
@@ -209,7 +209,7 @@ __global__ void __launch_bounds__(PT_THREADS) psi_tc_kernel(const __grid_constan
       tmem_ld16(lane_addr + 128, g2);
       tmem_ld_wait();
       tc_fence_before_sync();
-      mbar_arrive(&sh->g2_free);
+      mbar_arrive_warp(&sh->g2_free);
       float gv[R];
 #pragma unroll
       for (int r = 0; r < R; ++r) gv[r] = c2 * gelu_erf(__uint_as_float(g2[r]));

@@ -64,7 +64,7 @@ __global__ void __launch_bounds__(ST_THREADS) state_tc_kernel(const __grid_const
   if (tid == 0) {
     for (int s = 0; s < ST_STAGES; ++s) {
       mbar_init(&sh->full_v[s], 1);
-      mbar_init(&sh->full_b[s], ST_WORKERS);
+      mbar_init(&sh->full_b[s], ST_WORKERS / 32);
       mbar_init(&sh->empty[s], 1);
     }
     mbar_init(&sh->done, 1);
@@ -155,7 +155,7 @@ __global__ void __launch_bounds__(ST_THREADS) state_tc_kernel(const __grid_const
         *reinterpret_cast<uint4*>(brow + (R / 8 + nb) * B_SBO) = *reinterpret_cast<const uint4*>(&lo[nb * 8]);
       }
       fence_proxy_async_smem();
-      mbar_arrive(&sh->full_b[s]);
+      mbar_arrive_warp(&sh->full_b[s]);
     }
     st_wait(&sh->done, 0, abortp, p.a.status, 24);
     tc_fence_after_sync();
