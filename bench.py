@@ -31,7 +31,10 @@ FALLBACK_HBM_GBS = 6650.0
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures
 # summarised under profiles/ (None until a capture of that kernel/workload exists)
-NCU_TRAFFIC_BYTES = {}
+NCU_TRAFFIC_BYTES = {
+    (2, "feature_map"): 285.92e6 + 8.43e6,   # profiles/decode_step_cfg2.md
+    (2, "decode"): 113.87e6 + 3.58e6,
+}
 
 
 def parse_args():

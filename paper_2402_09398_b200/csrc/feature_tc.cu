@@ -74,12 +74,11 @@ __device__ __forceinline__ void ft_produce(const CUtensorMap* tm_q, const CUtens
                                            int nchunk, unsigned char* xbuf, uint32_t xbytes, unsigned char* w2dst,
                                            uint32_t w2bytes, __half* w3buf /* [2][256] */, unsigned char* ring,
                                            uint64_t* full, uint64_t* empty, uint64_t* aux_full, uint64_t* aux_empty,
-                                           volatile int* abortp, int32_t* status) {
-  uint32_t s = 0, sph = 0;
-  for (int n = 0; n < my_items; ++n) {
+                                           int naux, volatile int* abortp, int32_t* status) {
+  uint32_t s = 0, sph = 0, a = 0, aph = 0;
+  for (int n = 0; n < my_items; ++n, (++a == (uint32_t)naux ? (a = 0, aph ^= 1) : 0u)) {
     const FtItem im = ft_item(blockIdx.x + n * gridDim.x, gm.ntile);
-    const int a = n & 1;
-    wait_or_give_up(&aux_empty[a], ((n >> 1) & 1) ^ 1, abortp, status, 40);
+    wait_or_give_up(&aux_empty[a], aph ^ 1, abortp, status, 40);
     if (*abortp) return;                                 // issue nothing more once the CTA has given up
     const CUtensorMap* tx = im.which ? tm_k : tm_q;
     const CUtensorMap* tw1 = im.which ? tm_w1psi : tm_w1phi;
@@ -153,7 +152,7 @@ __global__ void __launch_bounds__(FT_THREADS) feature_tc_kernel(
     if (lane == 0)
       ft_produce<R>(&tm_q, &tm_k, &tm_w1phi, &tm_w1psi, p, gm, my_items, nchunk, xbuf, xbytes,
                     R == 16 ? w2raw : w2buf, w2bytes, &sh->w3[0][0], ring, sh->full, sh->empty, sh->aux_full,
-                    sh->aux_empty, abortp, status);
+                    sh->aux_empty, 2, abortp, status);
   } else if (warp == 1) {
     // ---------------- MMA issuer ----------------
     if (lane == 0 && my_items > 0) {
@@ -344,18 +343,21 @@ __global__ void __launch_bounds__(FT_THREADS) feature_tc_kernel(
 // reduction per item replaces the second GEMM.
 // --------------------------------------------------------------------------- //
 constexpr int FS_BUFS = 4;        // D1^T buffers in tensor memory (16 columns each)
-constexpr int FS_NPAD = 16;
-constexpr int FS_XBYTES = FS_NPAD * 256;
+constexpr int FS_NPAD = 16;       // GEMM1 N (the narrowest a 128-row MMA takes)
+constexpr int FS_XROWS = 8;       // input rows really loaded: the other 8 columns of D1^T are never read
+constexpr int FS_XBYTES = FS_XROWS * 256;
+constexpr int FS_AUX = 3;         // items whose inputs, W2 and W3 may be in flight
 
+template <int V>
 struct FsShared {
   uint64_t full[FT_MAX_STAGES], empty[FT_MAX_STAGES];
-  uint64_t aux_full[2], aux_empty[2];
+  uint64_t aux_full[FS_AUX], aux_empty[FS_AUX];
   uint64_t d1_full[FS_BUFS], d1_free[FS_BUFS];
   uint32_t tmem_base;
   int abort;
-  __align__(16) __half w3[2][16 * 16];
-  float red[2][FT_EPI_WARPS][8 * 16];   // per item parity, per warp: partial layer-2 sums [token][r]
-  float g[2][8 * 16];                   // c2 * gelu(layer-2 sums)
+  __align__(16) __half w3[FS_AUX][16 * 16];
+  float red[2][FT_EPI_WARPS][V];        // per item parity, per warp: partial layer-2 sums [token][r]
+  float g[2][V];                        // c2 * gelu(layer-2 sums)
 };
 
 __device__ __forceinline__ void epi_sync() { asm volatile("bar.sync 1, %0;" ::"n"(FT_EPI_THREADS) : "memory"); }
@@ -399,10 +401,13 @@ __global__ void __launch_bounds__(FT_THREADS) feature_tc_small_kernel(
   constexpr int V = NT * R;
   const int Rp = p.Rp, nchunk = Rp / FT_CHUNK, nstage = gm.nstage;
   const uint32_t w2bytes = (uint32_t)Rp * R * 2;
-  unsigned char* xbuf = ft_smem;                                   // [2][16 rows x 2 halves x 128 B]
-  unsigned char* ring = xbuf + 2 * FS_XBYTES;                      // [nstage][32 KB]
-  unsigned char* w2raw = ring + (size_t)nstage * FT_STAGE_BYTES;   // [2][Rp rows][R] as it lies in HBM
-  FsShared* sh = reinterpret_cast<FsShared*>(w2raw + 2 * w2bytes);
+  // x: [FS_AUX][2 halves][8 rows x 128 B], padded to 8 KB.  GEMM1 reads 16 rows per half; rows 8..15
+  // are whatever follows in shared memory (the other half, the next buffer, the pad) and only feed
+  // D1^T columns that no one reads.
+  unsigned char* xbuf = ft_smem;
+  unsigned char* ring = xbuf + 8192;                               // [nstage][32 KB]
+  unsigned char* w2raw = ring + (size_t)nstage * FT_STAGE_BYTES;   // [FS_AUX][Rp rows][R] as it lies in HBM
+  FsShared<V>* sh = reinterpret_cast<FsShared<V>*>(w2raw + FS_AUX * w2bytes);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   if (tid == 0) {
@@ -410,7 +415,7 @@ __global__ void __launch_bounds__(FT_THREADS) feature_tc_small_kernel(
       mbar_init(&sh->full[s], 1);
       mbar_init(&sh->empty[s], 1);
     }
-    for (int s = 0; s < 2; ++s) {
+    for (int s = 0; s < FS_AUX; ++s) {
       mbar_init(&sh->aux_full[s], 1);
       mbar_init(&sh->aux_empty[s], 1 + FT_EPI_WARPS);
     }
@@ -433,7 +438,7 @@ __global__ void __launch_bounds__(FT_THREADS) feature_tc_small_kernel(
     // ---------------- TMA producer ----------------
     if (lane == 0)
       ft_produce<R>(&tm_q, &tm_k, &tm_w1phi, &tm_w1psi, p, gm, my_items, nchunk, xbuf, FS_XBYTES, w2raw, w2bytes,
-                    &sh->w3[0][0], ring, sh->full, sh->empty, sh->aux_full, sh->aux_empty, abortp, status);
+                    &sh->w3[0][0], ring, sh->full, sh->empty, sh->aux_full, sh->aux_empty, FS_AUX, abortp, status);
   } else if (warp == 1) {
     // ---------------- MMA issuer: GEMM1 only ----------------
     if (lane == 0) {
@@ -441,9 +446,9 @@ __global__ void __launch_bounds__(FT_THREADS) feature_tc_small_kernel(
       const uint64_t ad_ring = smem_desc(smem_u32(ring), FT_STAGE_BYTES / 2, 1024, kLayoutSw128);
       const uint64_t bd_x = smem_desc(smem_u32(xbuf), 16, 1024, kLayoutSw128);
       uint32_t s = 0, sph = 0, b = 0, bph = 0;      // ring stage / D1 buffer and their phases: counted, never divided
-      for (int n = 0; n < my_items; ++n) {
-        const uint32_t a = n & 1;
-        wait_or_give_up(&sh->aux_full[a], (n >> 1) & 1, abortp, status, 62);
+      uint32_t a = 0, aph = 0;
+      for (int n = 0; n < my_items; ++n, (++a == FS_AUX ? (a = 0, aph ^= 1) : 0u)) {
+        wait_or_give_up(&sh->aux_full[a], aph, abortp, status, 62);
         const uint64_t bd0 = bd_x + (uint64_t)(a * (FS_XBYTES >> 4));
         const uint64_t bd1 = bd0 + (uint64_t)(FS_XBYTES >> 5);
         for (int c = 0; c < nchunk; ++c) {
@@ -473,14 +478,14 @@ __global__ void __launch_bounds__(FT_THREADS) feature_tc_small_kernel(
     const int j = quad * 32 + lane;            // hidden unit inside a chunk = accumulator lane
     const int et = tid - 64;                   // 0..255
     const uint32_t lane_addr = tmem + ((uint32_t)(quad * 32) << 16);
-    for (int n = 0; n < my_items; ++n) {
+    uint32_t a = 0, aph = 0;
+    for (int n = 0; n < my_items; ++n, (++a == FS_AUX ? (a = 0, aph ^= 1) : 0u)) {
       const int it = blockIdx.x + n * gridDim.x;
       const int tile = it % gm.ntile, which = (it / gm.ntile) & 1, lh = it / (2 * gm.ntile);
-      const int a = n & 1;
       const int b0 = tile * FS_NPAD, nb = min(NT, p.B - b0);
       float c1 = 1.f, c2 = 1.f;
       if (which && p.psi_scale) { c1 = __ldg(p.psi_scale + lh * 2); c2 = __ldg(p.psi_scale + lh * 2 + 1); }
-      wait_or_give_up(&sh->aux_full[a], (n >> 1) & 1, abortp, status, 65);
+      wait_or_give_up(&sh->aux_full[a], aph, abortp, status, 65);
       float part[V];
 #pragma unroll
       for (int e = 0; e < V; ++e) part[e] = 0.f;
@@ -591,11 +596,17 @@ int launch_feature_tc(less_ctx* c, const FmParams& p, cudaStream_t s) {
   const int grid = gm.items < sms ? gm.items : sms;
   LaunchScope scope(c, LESS_KERNEL_FEATURE_MAP, s);
   if (d.B <= 8) {
-    const size_t fx = (size_t)2 * FS_XBYTES + (size_t)2 * d.Rp * d.R * 2 + sizeof(FsShared) + 256;
+    const int nt = d.B <= 1 ? 1 : d.B <= 2 ? 2 : d.B <= 4 ? 4 : 8;
+    const size_t shared_struct = sizeof(FsShared<1>) + (size_t)(2 * FT_EPI_WARPS + 2) * (nt * d.R - 1) * 4;
+    const size_t fx = 8192 + (size_t)FS_AUX * d.Rp * d.R * 2 + shared_struct + 256;
     const int nsm = (int)((FT_SMEM_LIMIT - fx) / FT_STAGE_BYTES);
     gm.nstage = nsm > FT_MAX_STAGES ? FT_MAX_STAGES : nsm;
+    if (gm.nstage < 2) return LESS_ERR_INVALID_CONFIG;
     const size_t sm = fx + (size_t)gm.nstage * FT_STAGE_BYTES;
-    const int nt = d.B <= 1 ? 1 : d.B <= 2 ? 2 : d.B <= 4 ? 4 : 8;
+    // the small kernel loads 8 input rows per half tile
+    if (!make_tmap_f16_2d(&tq, p.x[0], d.B, lh * kHeadDim, lh * kHeadDim * 2, FS_XROWS) ||
+        !make_tmap_f16_2d(&tk, p.x[1], d.B, lh * kHeadDim, lh * kHeadDim * 2, FS_XROWS))
+      return fail_cuda("tensor map of q / k");
     if (d.R == 8) {
       if (nt == 1) return launch_small<8, 1>(c, p, gm, tq, tk, tw1a, tw1b, sm, grid, s);
       if (nt == 2) return launch_small<8, 2>(c, p, gm, tq, tk, tw1a, tw1b, sm, grid, s);
