@@ -18,6 +18,7 @@ __global__ void __launch_bounds__(FM_THREADS) feature_map_kernel(FmParams p) {
   float* xs = fm_smem;                         // [FM_BR][128]
   float* hs = xs + FM_BR * kHeadDim;           // [FM_BR][Rp]
   float* part = hs + FM_BR * p.Rp;             // [ndg][FM_BR][Rp]
+  pdl_launch_dependents();
   const int lh = blockIdx.x;                   // layer * Hd + head
   const int which = blockIdx.y;                // 0 phi(q), 1 psi(k)
   const int b0 = blockIdx.z * FM_BR;
@@ -222,6 +223,7 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_kernel(DecParams p) {
   float* zb = p.a.z + inst * R;
   float hcol[R];
   if (use_state) {
+    pdl_wait_primary();                            // phi(q_t), psi(k_t) of this step are complete from here on
     const float em = __expf(-m);
     float lr = 0.f, lz = 0.f;
 #pragma unroll
@@ -319,15 +321,25 @@ int launch_decode(less_ctx* c, const void* q, const void* k, const void* v, void
   p.flags = d.flags;
   const size_t smem = (size_t)(d.Np + 4 + DEC_RG * kHeadDim) * 4;
   LaunchScope scope(c, LESS_KERNEL_DECODE, s);
-  if (d.R == 8) {
-    if (smem > 48 * 1024)
-      cudaFuncSetAttribute(decode_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    decode_kernel<8><<<d.I, DEC_THREADS, smem, s>>>(p);
-  } else {
-    if (smem > 48 * 1024)
-      cudaFuncSetAttribute(decode_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    decode_kernel<16><<<d.I, DEC_THREADS, smem, s>>>(p);
-  }
+  auto kern = d.R == 8 ? decode_kernel<8> : decode_kernel<16>;
+  if (smem > 48 * 1024 &&
+      cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+    return fail_cuda("shared memory opt-in of decode_kernel");
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(d.I);
+  cfg.blockDim = dim3(DEC_THREADS);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  // Directly behind this step's feature-map kernel the decode kernel may start early and overlap
+  // its K / V reads with the weight stream (it waits for the feature maps on the device).  With
+  // per-kernel timing on, or without feature maps, it is an ordinary launch.
+  const bool overlap = overlap_decode(c);
+  cfg.attrs = attr;
+  cfg.numAttrs = overlap ? 1 : 0;
+  if (cudaLaunchKernelEx(&cfg, kern, p) != cudaSuccess) return fail_cuda("launch of decode_kernel");
   return check_launch("decode_kernel");
 }
 

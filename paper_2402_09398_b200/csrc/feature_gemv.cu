@@ -72,6 +72,7 @@ __global__ void __launch_bounds__(GV_THREADS) feature_gemv_kernel(FmParams p, in
     mbar_fence_init();
   }
   __syncthreads();
+  pdl_launch_dependents();
   volatile int* abortp = &sh->abort;
 
   if (tid >= GV_CONSUMERS) {

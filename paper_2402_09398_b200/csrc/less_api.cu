@@ -154,11 +154,16 @@ int less_create(const less_config* cfg, const less_weights* w, void* arena, size
   c->launches = 0;
   c->profile = false;
   c->feature_path = 2;
+  c->pdl = getenv("LESS_NO_OVERLAP") == nullptr;
+  c->feature_stages = 0;
+  if (const char* e = getenv("LESS_FEATURE_STAGES")) c->feature_stages = atoi(e);
   if (const char* e = getenv("LESS_FEATURE_KERNEL")) {
     if (!strcmp(e, "gemv")) c->feature_path = 1;
     else if (!strcmp(e, "plain")) c->feature_path = 0;
   }
   if (cudaGetDevice(&c->device) != cudaSuccess) { delete c; return LESS_ERR_CUDA; }
+  c->sms = 148;
+  cudaDeviceGetAttribute(&c->sms, cudaDevAttrMultiProcessorCount, c->device);
   // H_0 = 0, z_0 = 0, no live slots, clean status
   cudaError_t e = cudaMemset(c->a.H, 0, (size_t)d.I * d.R * d.D * 4);
   if (e == cudaSuccess) e = cudaMemset(c->a.z, 0, (size_t)d.I * d.R * 4);

@@ -287,3 +287,21 @@ def test_feature_maps_many_heads_per_cta(batch, rank):
         tf.step(*wl.make_decode_inputs(w, s, DEV))
     assert ctx.poll_status() == 0
     ctx.close()
+
+
+@pytest.mark.parametrize("overlap", [True, False])
+def test_decode_many_instances_and_ragged_slots(overlap, monkeypatch):
+    """More instances than one wave of CTAs and a slot count that is not a multiple of a row
+    group, with the decode kernel launched as a programmatic dependent of the feature-map
+    kernel (it overlaps the weight stream and waits for phi, psi on the device) and without."""
+    import harness
+    if not overlap:
+        monkeypatch.setenv("LESS_NO_OVERLAP", "1")
+    w = small(99, batch=4, layers=4, heads=25, prompt=150, steps=3, heavy=37, recent=40, weight_std=0.1)
+    ctx, W = _setup(w)
+    _prefill_all(ctx, w, with_out=False)
+    tf = harness.TeacherForced(ctx, w, W, list(range(0, w.instances, 7)))
+    for s in range(w.steps):
+        tf.step(*wl.make_decode_inputs(w, s, DEV))
+    assert ctx.poll_status() == 0
+    ctx.close()
