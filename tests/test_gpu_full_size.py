@@ -1,0 +1,158 @@
+"""GPU parity at the full benchmark sizes, in the launch configurations bench.py times.
+
+The contexts have the workloads' real shapes (all instances, all slots), so every
+kernel runs with the grid, shared memory and tiling of the timed runs; the oracle
+checks sampled (batch, layer, head) instances one by one: the prompt phase
+(kept set, accumulated scores, cached psi, H, z) and teacher-forced decode steps
+(output, feature maps, low-rank terms, eviction decision, score and state updates).
+The long-prompt workloads prefill only the layers that hold sampled instances (the
+prompt kernels' configuration depends on the layer group, not on how many groups
+run); their other layers start empty, which does not change any launch.
+"""
+import numpy as np
+import pytest
+import torch
+
+from paper_2402_09398_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def _ctx(w, layers_per_call):
+    from paper_2402_09398_b200 import binding
+    W = wl.make_weights(w, DEV)
+    ctx = binding.from_workload(w, W, DEV, max_prefill_layers=layers_per_call)
+    return ctx, W
+
+
+def _sample(w, n):
+    """n instances spread over batch, layer and head, first and last included."""
+    idx = sorted({int(round(i * (w.instances - 1) / (n - 1))) for i in range(n)}) if n > 1 else [0]
+    return idx
+
+
+def _check_prompt(ctx, w, W, instances):
+    import harness
+    worst = {}
+    for inst in instances:
+        b, layer, head = wl.instance_coords(w, inst)
+        Q, K, V = wl.make_prompt(w, layer, 1, DEV)
+        r = harness.check_prefill(ctx, w, _HeadView(W), Q, K, V, [inst], None, 0, None, layer_begin=layer)
+        for k, v in r.items():
+            worst[k] = max(worst.get(k, 0), v)
+        del Q, K, V
+    return worst
+
+
+class _HeadView(dict):
+    """Weights kept on the device; a head's matrices are copied out when asked for."""
+
+    def __init__(self, W):
+        super().__init__(W)
+
+    def __getitem__(self, name):
+        return _Lazy(dict.__getitem__(self, name))
+
+
+class _Lazy:
+    def __init__(self, t):
+        self.t = t
+
+    def __getitem__(self, idx):
+        return self.t[idx].cpu()
+
+
+def _decode_steps(ctx, w, W, instances, steps):
+    import harness
+    tf = harness.TeacherForced(ctx, w, _HeadView(W), instances)
+    for s in range(steps):
+        tf.step(*wl.make_decode_inputs(w, s, DEV))
+    assert ctx.poll_status() == 0
+    assert tf.exempt <= 0.02 * len(instances) * steps + 1
+    return tf
+
+
+def test_cfg1_smallest_every_instance_every_step():
+    w = wl.CONFIGS[1]
+    ctx, W = _ctx(w, w.layers)
+    Q, K, V = wl.make_prompt(w, 0, w.layers, DEV)
+    ctx.prefill(Q, K, V, 0)
+    inst = list(range(w.instances))
+    print("cfg1 prompt", _check_prompt(ctx, w, W, inst))
+    tf = _decode_steps(ctx, w, W, inst, w.steps)
+    assert tf.evictions == w.steps * w.instances
+    print("cfg1 decode", tf.worst, "exempt", tf.exempt)
+    ctx.close()
+
+
+def test_cfg2_llama7b_shape_sampled_instances():
+    w = wl.CONFIGS[2]
+    ctx, W = _ctx(w, w.layers)
+    Q, K, V = wl.make_prompt(w, 0, w.layers, DEV)
+    ctx.prefill(Q, K, V, 0)
+    del Q, K, V
+    inst = _sample(w, 6)
+    print("cfg2 prompt", _check_prompt(ctx, w, W, inst))
+    tf = _decode_steps(ctx, w, W, inst, 12)
+    assert tf.evictions == 12 * len(inst)
+    print("cfg2 decode", tf.worst, "exempt", tf.exempt)
+    ctx.close()
+
+
+def test_cfg3_batched_serving_sampled_instances():
+    w = wl.CONFIGS[3]
+    per_call = 2
+    ctx, W = _ctx(w, per_call)
+    for l0 in range(0, w.layers, per_call):
+        Q, K, V = wl.make_prompt(w, l0, per_call, DEV)
+        ctx.prefill(Q, K, V, l0)
+        del Q, K, V
+    inst = _sample(w, 6)
+    print("cfg3 prompt", _check_prompt(ctx, w, W, inst))
+    tf = _decode_steps(ctx, w, W, inst, 4)
+    assert tf.evictions == 4 * len(inst)
+    print("cfg3 decode", tf.worst, "exempt", tf.exempt)
+    ctx.close()
+    torch.cuda.empty_cache()
+
+
+def test_cfg4_long_context_sampled_instances():
+    w = wl.CONFIGS[4]
+    ctx, W = _ctx(w, 1)
+    inst = [wl.instance_index(w, 0, 0, 0), wl.instance_index(w, w.batch - 1, w.layers - 1, w.heads - 1)]
+    for layer in (0, w.layers - 1):
+        Q, K, V = wl.make_prompt(w, layer, 1, DEV)
+        ctx.prefill(Q, K, V, layer)
+        del Q, K, V
+    print("cfg4 prompt", _check_prompt(ctx, w, W, inst))
+    tf = _decode_steps(ctx, w, W, inst, 4)
+    assert tf.evictions == 4 * len(inst)
+    print("cfg4 decode", tf.worst, "exempt", tf.exempt)
+    ctx.close()
+    torch.cuda.empty_cache()
+
+
+def test_cfg5_prefill_compression_one_layer_sampled_instance():
+    """Prompt of 32 768 tokens: one whole layer (256 instances) goes through the prompt kernels;
+    one instance is checked against the oracle (kept set, scores, cached psi, H, z)."""
+    w = wl.CONFIGS[5]
+    ctx, W = _ctx(w, 1)
+    layer = 3
+    Q, K, V = wl.make_prompt(w, layer, 1, DEV)
+    ctx.prefill(Q, K, V, layer)
+    torch.cuda.synchronize()
+    assert ctx.poll_status() == 0
+    del Q, K, V
+    inst = [wl.instance_index(w, w.batch - 1, layer, 5)]
+    r = _check_prompt(ctx, w, W, inst)
+    print("cfg5 prompt", r)
+    # bookkeeping of every instance of the layer: all slots filled, positions ascending, recent window kept
+    some = [wl.instance_index(w, b, layer, h) for b in (0, 3, 7) for h in (0, 17, 31)]
+    for rec in ctx.export_state(some):
+        assert rec["count"] == w.slots
+        pos = rec["pos"].astype(np.int64)
+        assert np.all(np.diff(pos) > 0) and np.array_equal(pos[-w.recent:], np.arange(w.prompt - w.recent, w.prompt))
+        assert np.isfinite(rec["H"]).all() and rec["z"].min() >= 0
+    ctx.close()
+    torch.cuda.empty_cache()
