@@ -76,6 +76,7 @@ __device__ __forceinline__ void ft_produce(const CUtensorMap* tm_q, const CUtens
                                            uint64_t* full, uint64_t* empty, uint64_t* aux_full, uint64_t* aux_empty,
                                            int naux, volatile int* abortp, int32_t* status) {
   uint32_t s = 0, sph = 0, a = 0, aph = 0;
+  const uint64_t stream_policy = l2_evict_first_policy();
   for (int n = 0; n < my_items; ++n, (++a == (uint32_t)naux ? (a = 0, aph ^= 1) : 0u)) {
     const FtItem im = ft_item(blockIdx.x + n * gridDim.x, gm.ntile);
     wait_or_give_up(&aux_empty[a], aph ^ 1, abortp, status, 40);
@@ -94,8 +95,8 @@ __device__ __forceinline__ void ft_produce(const CUtensorMap* tm_q, const CUtens
       if (*abortp) return;
       mbar_expect_tx(&full[s], FT_STAGE_BYTES);
       unsigned char* st = ring + (size_t)s * FT_STAGE_BYTES;
-      tma_load_2d(st, tw1, c * FT_CHUNK, im.lh * kHeadDim, &full[s]);
-      tma_load_2d(st + FT_STAGE_BYTES / 2, tw1, c * FT_CHUNK + 64, im.lh * kHeadDim, &full[s]);
+      tma_load_2d_hint(st, tw1, c * FT_CHUNK, im.lh * kHeadDim, &full[s], stream_policy);
+      tma_load_2d_hint(st + FT_STAGE_BYTES / 2, tw1, c * FT_CHUNK + 64, im.lh * kHeadDim, &full[s], stream_policy);
       if (++s == (uint32_t)gm.nstage) { s = 0; sph ^= 1; }
     }
   }

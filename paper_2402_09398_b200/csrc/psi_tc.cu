@@ -106,6 +106,7 @@ __global__ void __launch_bounds__(PT_THREADS) psi_tc_kernel(const __grid_constan
   if (warp == 4) {
     // ---------------- TMA producer ----------------
     if (tid == PT_WORKERS) {
+      const uint64_t stream_policy = l2_evict_first_policy();
       mbar_expect_tx(&sh->w1_full, (uint32_t)nchunk * 16384);
       for (int c = 0; c < nchunk; ++c)
         tma_load_2d(w1s + (size_t)c * 16384, &tmap_w1, c * 64, im.lh * kHeadDim, &sh->w1_full);
@@ -114,8 +115,8 @@ __global__ void __launch_bounds__(PT_THREADS) psi_tc_kernel(const __grid_constan
         if (*abortp) break;                      // issue nothing more once the CTA has given up
         mbar_expect_tx(&sh->k_full, PT_KBYTES);
         const int row = (int)(im.in_row0 + jbeg + (size_t)i * PT_TILE);
-        tma_load_2d(kbuf, &tmap_k, 0, row, &sh->k_full);
-        tma_load_2d(kbuf + PT_KBYTES / 2, &tmap_k, 64, row, &sh->k_full);
+        tma_load_2d_hint(kbuf, &tmap_k, 0, row, &sh->k_full, stream_policy);
+        tma_load_2d_hint(kbuf + PT_KBYTES / 2, &tmap_k, 64, row, &sh->k_full, stream_policy);
       }
     }
   } else if (warp == 5) {

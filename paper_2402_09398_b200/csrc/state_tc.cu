@@ -84,14 +84,15 @@ __global__ void __launch_bounds__(ST_THREADS) state_tc_kernel(const __grid_const
   if (warp == 4) {
     // ---------------- TMA producer ----------------
     if (tid == ST_WORKERS) {
+      const uint64_t stream_policy = l2_evict_first_policy();
       for (int i = 0; i < ntiles; ++i) {
         const int s = i % ST_STAGES;
         st_wait(&sh->empty[s], ((i / ST_STAGES) & 1) ^ 1, abortp, p.a.status, 20);
         if (*abortp) break;                      // issue nothing more once the CTA has given up
         mbar_expect_tx(&sh->full_v[s], ST_VBYTES);
         const int row = (int)(im.in_row0 + jbeg + (size_t)i * ST_TILE);
-        tma_load_2d(vbuf + s * ST_VBYTES, &tmap_v, 0, row, &sh->full_v[s]);
-        tma_load_2d(vbuf + s * ST_VBYTES + ST_VBYTES / 2, &tmap_v, 64, row, &sh->full_v[s]);
+        tma_load_2d_hint(vbuf + s * ST_VBYTES, &tmap_v, 0, row, &sh->full_v[s], stream_policy);
+        tma_load_2d_hint(vbuf + s * ST_VBYTES + ST_VBYTES / 2, &tmap_v, 64, row, &sh->full_v[s], stream_policy);
       }
     }
   } else if (warp == 5) {
