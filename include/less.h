@@ -22,6 +22,10 @@
  *     their inputs must stay valid until the stream reaches the call.
  *   - A context is not thread-safe.
  *   - 16-bit inputs are IEEE fp16; accumulation, scores, H, z and outputs fp32.
+ *   - Environment, read by less_create: LESS_LOG (explain host-side failures on
+ *     stderr), LESS_FEATURE_KERNEL=gemv|plain (CUDA-core feature-map kernels),
+ *     LESS_NO_OVERLAP (no programmatic dependent launch of the decode kernel),
+ *     LESS_FEATURE_STAGES=n (cap on the feature kernels' weight ring).
  */
 #ifndef LESS_B200_H
 #define LESS_B200_H
