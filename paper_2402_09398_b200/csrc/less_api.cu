@@ -155,6 +155,9 @@ int less_create(const less_config* cfg, const less_weights* w, void* arena, size
   c->profile = false;
   c->feature_path = 2;
   c->pdl = getenv("LESS_NO_OVERLAP") == nullptr;
+  c->score_path = 1;
+  if (const char* e = getenv("LESS_SCORE_KERNEL"))
+    if (!strcmp(e, "plain")) c->score_path = 0;
   c->feature_stages = 0;
   if (const char* e = getenv("LESS_FEATURE_STAGES")) c->feature_stages = atoi(e);
   if (const char* e = getenv("LESS_FEATURE_KERNEL")) {

@@ -66,6 +66,7 @@ struct less_ctx {
   int sms;             // multiprocessors of the device
   bool pdl;            // decode kernel overlaps the feature-map kernel (off with LESS_NO_OVERLAP)
   int feature_stages;  // cap on the feature kernels' ring stages (LESS_FEATURE_STAGES), 0 = default
+  int score_path;      // prompt scoring: 1 tensor cores, 0 CUDA cores (LESS_SCORE_KERNEL=plain)
   int feature_path;    // feature-map kernel: 2 tensor cores, 1 streaming GEMV, 0 plain (LESS_FEATURE_KERNEL)
   bool profile;                         // record an event pair around every launch
   std::vector<cudaEvent_t> prof_events; // start, stop, start, stop, ...

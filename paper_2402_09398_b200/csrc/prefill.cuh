@@ -36,7 +36,9 @@ __device__ __forceinline__ InstMap map_instance(const PfParams& p, int g) {
   return m;
 }
 
-// launchers of the tensor-core kernels (state_tc.cu, psi_tc.cu)
+// launchers of the tensor-core kernels (score_tc.cu, state_tc.cu, psi_tc.cu)
+bool score_tc_supported();
+int launch_score_tc(less_ctx* c, const PfParams& p, int G, cudaStream_t s);
 int launch_state_tc(less_ctx* c, const PfParams& p, int G, cudaStream_t s);
 bool psi_tc_supported(const Dims& d);
 int launch_psi_tc(less_ctx* c, const PfParams& p, int G, cudaStream_t s);

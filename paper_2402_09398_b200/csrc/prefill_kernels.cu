@@ -397,13 +397,18 @@ int launch_prefill_group(less_ctx* c, int layer0, int nl, int lj0, int layer_cou
   p.nsplit = nsplit; p.split_tokens = split_tokens;
   if (S > 0) {
     const int tiles = (S + PF_TILE - 1) / PF_TILE;
-    {
-      LaunchScope scope(c, LESS_KERNEL_ROWSTAT, s);
-      rowstat_kernel<<<dim3(tiles, G), PF_TILE, 0, s>>>(p);
-    }
-    {
-      LaunchScope scope(c, LESS_KERNEL_COLSUM, s);
-      colsum_kernel<<<dim3(tiles, G), PF_TILE, 0, s>>>(p);
+    if (c->score_path == 1 && score_tc_supported()) {
+      const int rc = launch_score_tc(c, p, G, s);
+      if (rc != LESS_OK) return rc;
+    } else {
+      {
+        LaunchScope scope(c, LESS_KERNEL_ROWSTAT, s);
+        rowstat_kernel<<<dim3(tiles, G), PF_TILE, 0, s>>>(p);
+      }
+      {
+        LaunchScope scope(c, LESS_KERNEL_COLSUM, s);
+        colsum_kernel<<<dim3(tiles, G), PF_TILE, 0, s>>>(p);
+      }
     }
     if (attn_out) {
       LaunchScope scope(c, LESS_KERNEL_ATTN_OUT, s);

@@ -37,8 +37,9 @@ def _prefill_all(ctx, w, with_out=True, prompt=None):
 
 
 @pytest.mark.parametrize("variant", ["base", "rank16", "boosted", "ragged", "sparse_norm", "no_state",
-                                     "scaled", "heavy0", "recent1", "hidden256"])
-def test_prefill_and_teacher_forced_decode(variant):
+                                     "scaled", "heavy0", "recent1", "hidden256", "long_prompt",
+                                     "cuda_core_scoring"])
+def test_prefill_and_teacher_forced_decode(variant, monkeypatch):
     import harness
     flags, psi_scale = 0, None
     w = small()
@@ -62,6 +63,11 @@ def test_prefill_and_teacher_forced_decode(variant):
         w = small(79, heavy=30, recent=1)
     elif variant == "hidden256":
         w = small(80, hidden=256, weight_std=0.05)
+    elif variant == "long_prompt":          # several streamed 256-row tiles per scoring CTA, rings wrap
+        w = small(60, prompt=1100, batch=1, heads=2, steps=4, heavy=50, recent=30)
+    elif variant == "cuda_core_scoring":    # the prompt scoring kernels used when no tensor map can be made
+        monkeypatch.setenv("LESS_SCORE_KERNEL", "plain")
+        w = small(59, prompt=420)
     ctx, W = _setup(w, flags, psi_scale)
     Q, K, V, out = _prefill_all(ctx, w)
     inst = list(range(w.instances))
