@@ -44,6 +44,7 @@ Dims make_dims(const less_config* c) {
   d.Np = (d.N + 3) & ~3;
   d.I = c->batch * c->layers * c->heads;
   d.Sp = (c->max_prompt + 3) & ~3;
+  d.Sbx = ((c->max_prompt + 255) & ~255) + 256;
   d.Lw = c->max_prefill_layers;
   d.flags = c->flags;
   return d;
@@ -81,6 +82,7 @@ size_t carve(const Dims& d, char* base, Arena* a) {
   t.ws_slot = (int32_t*)take(Iw * Sp * 4);
   t.ws_hpart = (float*)take(Iw * kMaxSplit * (R * D + R) * 4);
   t.ws_psi = (float*)take(Iw * Sp * R * 4);
+  t.ws_bx = (uint4*)take(Iw * (size_t)d.Sbx * 16);
   if (a) *a = t;
   return off;
 }

@@ -40,6 +40,7 @@ struct Arena {
   int32_t* ws_slot;  // [Iw][Sp]    slot of a prompt token, -1 = evicted
   float* ws_hpart;   // [Iw][kMaxSplit][R*D + R]  partial H, z per token split
   float* ws_psi;     // [Iw][Sp][R]  psi(k_j) of every prompt token
+  uint4* ws_bx;      // [Iw][Sbx]    per prompt row: -(m_i sqrt(D) - log2(1/l_i) / c) as three fp16 parts (column sums)
 };
 
 struct Dims {
@@ -47,6 +48,7 @@ struct Dims {
   int32_t heavy, recent, N, Np; // slots; Np = N rounded up to a multiple of 4
   int32_t I;                    // instances
   int32_t Sp;                   // max_prompt rounded up to a multiple of 4
+  int32_t Sbx;                  // max_prompt rounded up to a multiple of 256 (+256)
   int32_t Lw;                   // max_prefill_layers
   uint32_t flags;
 };

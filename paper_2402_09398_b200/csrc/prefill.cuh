@@ -11,7 +11,7 @@ struct PfParams {
   Arena a;
   const __half* w_psi1; const __half* w_psi2; const __half* w_psi3;
   const float* psi_scale;
-  int S, Sp;                 // prompt length, workspace row stride
+  int S, Sp, Sbx;            // prompt length, workspace row strides
   int layer0, nl;            // first model layer of this group, layers in the group
   int lj0, layer_count;      // first input layer of this group, layers in the input
   int B, L, Hd, N, Np, heavy, recent, Rp;

@@ -379,7 +379,7 @@ int launch_prefill_group(less_ctx* c, int layer0, int nl, int lj0, int layer_cou
   p.w_psi2 = (const __half*)c->w.w_psi2;
   p.w_psi3 = (const __half*)c->w.w_psi3;
   p.psi_scale = c->w.psi_scale;
-  p.S = S; p.Sp = d.Sp;
+  p.S = S; p.Sp = d.Sp; p.Sbx = d.Sbx;
   p.layer0 = layer0; p.nl = nl; p.lj0 = lj0; p.layer_count = layer_count;
   p.B = d.B; p.L = d.L; p.Hd = d.Hd; p.N = d.N; p.Np = d.Np;
   p.heavy = d.heavy; p.recent = d.recent; p.Rp = d.Rp;

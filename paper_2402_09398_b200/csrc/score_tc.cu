@@ -15,8 +15,10 @@
 // exp2 and one add per element:
 //     p_ij = exp2( c (q_i . k_j - b_i) ),   c = log2(e) / sqrt(D),   b_i = m_i sqrt(D) - log2(1 / l_i) / c
 // A ninth k-step multiplies a column of ones on the key side with (-b_i), split into three
-// fp16 parts, on the query side; rows past the prompt get b = +60000, which turns them into
-// exact zeros.  Only the tile on the diagonal needs a per-element causal test.
+// fp16 parts, on the query side; the row-statistics kernel leaves those parts in the workspace
+// in operand layout (16 bytes per row), so they arrive with one bulk copy per tile.  Rows past
+// the prompt get b = +60000, which turns them into exact zeros.  Only the tile on the diagonal
+// needs a per-element causal test.
 // Every wait is bounded (pipeline.cuh).
 #include "prefill.cuh"
 #include "tc_common.cuh"
@@ -36,7 +38,6 @@ constexpr float kExpScale = 0.12751743074602468f;             // log2(e) / sqrt(
 struct ScShared {
   uint64_t res_full;
   uint64_t full[SC_STAGES], empty[SC_STAGES];
-  uint64_t bx_full[SC_STAGES], bx_empty[SC_STAGES];
   uint64_t d_full[2], d_free[2];
   uint32_t tmem_base;
   int abort;
@@ -44,6 +45,16 @@ struct ScShared {
 };
 
 __device__ __forceinline__ void sc_epi_sync() { asm volatile("bar.sync 1, %0;" ::"n"(SC_EPI_THREADS) : "memory"); }
+
+// -b as three fp16 parts (k = 0, 1, 2 of the ninth k-step), the row's other 5 halves zero
+__device__ __forceinline__ uint4 pack_neg_b(float nb) {
+  const __half h0 = __float2half_rn(nb);
+  const float r1 = nb - __half2float(h0);
+  const __half h1 = __float2half_rn(r1);
+  const __half h2 = __float2half_rn(r1 - __half2float(h1));
+  return make_uint4((uint32_t)__half_as_ushort(h0) | ((uint32_t)__half_as_ushort(h1) << 16),
+                    (uint32_t)__half_as_ushort(h2), 0u, 0u);
+}
 
 __device__ __forceinline__ float ex2_approx(float x) {
   float y;
@@ -189,9 +200,15 @@ __global__ void __launch_bounds__(RS_THREADS) rowstat_tc_kernel(const __grid_con
       float lt = 0.f;
       if (m > -INFINITY) lt += l * ex2_approx((m - mm) * kExpScale);
       if (m2 > -INFINITY) lt += l2 * ex2_approx((m2 - mm) * kExpScale);
+      const float il = 1.0f / lt;
       p.a.ws_m[(size_t)g * p.Sp + i] = mm * kRawScale;
-      p.a.ws_invl[(size_t)g * p.Sp + i] = 1.0f / lt;
+      p.a.ws_invl[(size_t)g * p.Sp + i] = il;
+      p.a.ws_bx[(size_t)g * p.Sbx + i] = pack_neg_b(-(mm - log2f(il) * (1.0f / kExpScale)));
     }
+    // rows between the prompt's end and the end of its last 256-row tile: exact zeros in the column sums
+    if (half == 0 && tile == tiles - 1 && !*abortp)
+      for (int x = p.S + r; x < ((p.S + SC_TILE_N - 1) & ~(SC_TILE_N - 1)); x += SC_TILE_M)
+        p.a.ws_bx[(size_t)g * p.Sbx + x] = pack_neg_b(-60000.f);
   }
   drain_after_abort(abortp);
   tc_fence_before_sync();
@@ -200,19 +217,20 @@ __global__ void __launch_bounds__(RS_THREADS) rowstat_tc_kernel(const __grid_con
 }
 
 // ------------------------------------------------------------------------------------------- //
-// P2: column sums.  warp 0 TMA, warp 1 MMA, warps 2..9 epilogue, warp 10 builds the (-b_i) operand.
+// P2: column sums.  warp 0 TMA, warp 1 MMA, warps 2..9 epilogue.
 // ------------------------------------------------------------------------------------------- //
-constexpr int CS_THREADS = 64 + SC_EPI_THREADS + 32;
-constexpr int SC_BX_BYTES = SC_TILE_N * 32;        // [32 row groups][2 k halves][8 rows][16 B]
-constexpr int SC_ONES_BYTES = SC_TILE_M * 32;
+constexpr int CS_THREADS = 64 + SC_EPI_THREADS;
+constexpr int SC_BX_BYTES = SC_TILE_N * 16;        // one stage: [32 row groups][8 rows][16 B], k = 0..7 of the ninth k-step
+constexpr int SC_BXZ_BYTES = SC_STAGES * SC_BX_BYTES;   // zeros: k = 8..15, at the same offset behind every stage
+constexpr int SC_ONES_BYTES = SC_TILE_M * 32;      // [16 row groups][2 k halves][8 rows][16 B]
 
 __global__ void __launch_bounds__(CS_THREADS) colsum_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
                                                                const __grid_constant__ CUtensorMap tm_k, PfParams p) {
   extern __shared__ __align__(1024) unsigned char sc_smem[];
   unsigned char* kres = sc_smem;                                 // resident K tile
   unsigned char* ring = kres + SC_RES_BYTES;                     // streamed Q tiles
-  unsigned char* bx = ring + SC_STAGES * SC_STAGE_BYTES;         // [stages] (-b_i) columns of the Q tiles
-  unsigned char* ones = bx + SC_STAGES * SC_BX_BYTES;            // ones columns of the K tile
+  unsigned char* bx = ring + SC_STAGES * SC_STAGE_BYTES;         // [stages] (-b_i) columns of the Q tiles, then zeros
+  unsigned char* ones = bx + SC_STAGES * SC_BX_BYTES + SC_BXZ_BYTES;   // ones columns of the K tile
   ScShared* sh = reinterpret_cast<ScShared*>(ones + SC_ONES_BYTES);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -228,8 +246,6 @@ __global__ void __launch_bounds__(CS_THREADS) colsum_tc_kernel(const __grid_cons
     for (int s = 0; s < SC_STAGES; ++s) {
       mbar_init(&sh->full[s], 1);
       mbar_init(&sh->empty[s], 1);
-      mbar_init(&sh->bx_full[s], 1);
-      mbar_init(&sh->bx_empty[s], 1);
     }
     for (int s = 0; s < 2; ++s) {
       mbar_init(&sh->d_full[s], 1);
@@ -238,16 +254,13 @@ __global__ void __launch_bounds__(CS_THREADS) colsum_tc_kernel(const __grid_cons
     sh->abort = *reinterpret_cast<volatile int32_t*>(status) != 0;
     mbar_fence_init();
   }
-  // constant parts of the ninth k-step: ones (1, 1, 1, 0 ...) on the key side, zeros in the
-  // second k half of both sides
-  for (int e = tid; e < (SC_ONES_BYTES + SC_STAGES * SC_BX_BYTES) / 16; e += CS_THREADS) {
-    unsigned char* dst = (e < SC_STAGES * SC_BX_BYTES / 16) ? bx + e * 16 : ones + (e - SC_STAGES * SC_BX_BYTES / 16) * 16;
-    const bool key_side = e >= SC_STAGES * SC_BX_BYTES / 16;
-    const int unit = key_side ? e - SC_STAGES * SC_BX_BYTES / 16 : e;
-    const bool first_half = ((unit >> 3) & 1) == 0;              // 128-byte blocks alternate k halves
+  // constant parts of the ninth k-step: zeros for k = 8..15 of the query side; on the key side
+  // ones (1, 1, 1, 0 ...) for k = 0..7 and zeros for k = 8..15
+  for (int e = tid; e < (SC_BXZ_BYTES + SC_ONES_BYTES) / 16; e += CS_THREADS) {
     uint4 v = make_uint4(0, 0, 0, 0);
-    if (key_side && first_half) v = make_uint4(0x3c003c00u, 0x00003c00u, 0, 0);   // fp16 1, 1, 1, 0, 0, 0, 0, 0
-    *reinterpret_cast<uint4*>(dst) = v;
+    const int unit = e - SC_BXZ_BYTES / 16;                      // 16-byte unit inside the ones block
+    if (unit >= 0 && ((unit >> 3) & 1) == 0) v = make_uint4(0x3c003c00u, 0x00003c00u, 0, 0);   // fp16 1, 1, 1, 0 ...
+    *reinterpret_cast<uint4*>(bx + SC_STAGES * SC_BX_BYTES + e * 16) = v;
   }
   if (warp == 1) tmem_alloc(&sh->tmem_base, 512);
   fence_proxy_async_smem();
@@ -269,9 +282,11 @@ __global__ void __launch_bounds__(CS_THREADS) colsum_tc_kernel(const __grid_cons
         if (*abortp) break;
         const int qrow = (int)(im.in_row0 + (size_t)(t0 + t) * SC_TILE_N);
         unsigned char* st = ring + s * SC_STAGE_BYTES;
-        mbar_expect_tx(&sh->full[s], SC_STAGE_BYTES);
+        mbar_expect_tx(&sh->full[s], SC_STAGE_BYTES + SC_BX_BYTES);
         tma_load_2d(st, &tm_q, 0, qrow, &sh->full[s]);
         tma_load_2d(st + SC_STAGE_BYTES / 2, &tm_q, 64, qrow, &sh->full[s]);
+        bulk_g2s(bx + s * SC_BX_BYTES, p.a.ws_bx + (size_t)g * p.Sbx + (size_t)(t0 + t) * SC_TILE_N, SC_BX_BYTES,
+                 &sh->full[s]);
         if (++s == SC_STAGES) { s = 0; ph ^= 1; }
       }
     }
@@ -281,12 +296,11 @@ __global__ void __launch_bounds__(CS_THREADS) colsum_tc_kernel(const __grid_cons
       const uint64_t ad0 = smem_desc(smem_u32(kres), 16, 1024, kLayoutSw128);
       const uint64_t bd_ring = smem_desc(smem_u32(ring), 16, 1024, kLayoutSw128);
       const uint64_t ad_ones = smem_desc(smem_u32(ones), 128, 256, kLayoutNone);
-      const uint64_t bd_bx = smem_desc(smem_u32(bx), 128, 256, kLayoutNone);
+      const uint64_t bd_bx = smem_desc(smem_u32(bx), SC_STAGES * SC_BX_BYTES, 128, kLayoutNone);
       wait_or_give_up(&sh->res_full, 0, abortp, status, 86);
       uint32_t s = 0, ph = 0, b = 0, bph = 0;
       for (int t = 0; t < ntile; ++t) {
         wait_or_give_up(&sh->full[s], ph, abortp, status, 87);
-        wait_or_give_up(&sh->bx_full[s], ph, abortp, status, 88);
         wait_or_give_up(&sh->d_free[b], bph ^ 1, abortp, status, 89);
         if (*abortp) break;
         tc_fence_after_sync();
@@ -297,40 +311,10 @@ __global__ void __launch_bounds__(CS_THREADS) colsum_tc_kernel(const __grid_cons
                      bd0 + (uint64_t)((ks >> 2) * (SC_STAGE_BYTES >> 5) + (ks & 3) * 2), idesc, ks ? 1u : 0u);
         mma_f16_ss(tmem + b * SC_TILE_N, ad_ones, bd_bx + (uint64_t)(s * (SC_BX_BYTES >> 4)), idesc, 1u);
         mma_commit(&sh->empty[s]);
-        mma_commit(&sh->bx_empty[s]);
         mma_commit(&sh->d_full[b]);
         if (++s == SC_STAGES) { s = 0; ph ^= 1; }
         if (b ^= 1, b == 0) bph ^= 1;
       }
-    }
-  } else if (warp == 10) {
-    // ---- (-b_i) of the streamed rows: three fp16 parts in k = 0, 1, 2 of the ninth k-step ----
-    uint32_t s = 0, ph = 0;
-    for (int t = 0; t < ntile; ++t) {
-      wait_or_give_up(&sh->bx_empty[s], ph ^ 1, abortp, status, 90);
-      if (*abortp) break;
-      unsigned char* dst = bx + s * SC_BX_BYTES;
-#pragma unroll
-      for (int rr = 0; rr < SC_TILE_N / 32; ++rr) {
-        const int n = rr * 32 + lane;                              // row inside the tile
-        const int i = (t0 + t) * SC_TILE_N + n;
-        float nb = -60000.f;                                       // rows past the prompt: p = exp2(c (qk - 60000)) = 0
-        if (i < p.S) {
-          const float mi = p.a.ws_m[(size_t)g * p.Sp + i], il = p.a.ws_invl[(size_t)g * p.Sp + i];
-          nb = -(mi * 11.313708498984761f - log2f(il) * (1.0f / kExpScale));
-        }
-        const __half h0 = __float2half_rn(nb);
-        const float r1 = nb - __half2float(h0);
-        const __half h1 = __float2half_rn(r1);
-        const __half h2 = __float2half_rn(r1 - __half2float(h1));
-        const uint32_t w0 = (uint32_t)__half_as_ushort(h0) | ((uint32_t)__half_as_ushort(h1) << 16);
-        const uint32_t w1 = (uint32_t)__half_as_ushort(h2);
-        *reinterpret_cast<uint4*>(dst + (n >> 3) * 256 + (n & 7) * 16) = make_uint4(w0, w1, 0, 0);
-      }
-      fence_proxy_async_smem();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&sh->bx_full[s]);
-      if (++s == SC_STAGES) { s = 0; ph ^= 1; }
     }
   } else {
     // ---- epilogue: lane = key of the K tile; the two warps of a lane quadrant split the rows i ----
@@ -391,7 +375,7 @@ int launch_score_tc(less_ctx* c, const PfParams& p, int G, cudaStream_t s) {
     return fail_cuda("tensor maps of Q / K");
   const int tiles = (p.S + SC_TILE_M - 1) / SC_TILE_M;
   const size_t smem1 = SC_RES_BYTES + SC_STAGES * SC_STAGE_BYTES + sizeof(ScShared) + 1024;
-  const size_t smem2 = smem1 + SC_STAGES * SC_BX_BYTES + SC_ONES_BYTES;
+  const size_t smem2 = smem1 + SC_STAGES * SC_BX_BYTES + SC_BXZ_BYTES + SC_ONES_BYTES;
   if (cudaFuncSetAttribute(rowstat_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem1) != cudaSuccess ||
       cudaFuncSetAttribute(colsum_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem2) != cudaSuccess)
     return fail_cuda("shared memory opt-in of the scoring kernels");
