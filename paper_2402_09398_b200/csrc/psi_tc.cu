@@ -9,15 +9,15 @@
 //                   a single fp16 rounding of the hidden layer costs ~2e-3 on individual psi vectors)
 //   GEMM2  G2[128 x 16] += (hidden_hi + hidden_lo)[128 x 64] * W2[chunk rows, :]
 //   after 8 chunks: tcgen05.ld G2 -> c2 * gelu -> W3 on CUDA cores -> abs -> psi[token][R]
-// Roles: warps 0-3 epilogue (thread = token row = tensor-memory lane), warp 4 TMA
-// producer, warp 5 MMA issuer.  Operands come in by TMA tiled loads with the 128-byte
+// Roles: warps 0-7 epilogue (lane quadrant = warp & 3, token row = tensor-memory lane; the two
+// warps of a quadrant split a chunk's 64 columns), warp 8 TMA producer, warp 9 MMA issuer.  Operands come in by TMA tiled loads with the 128-byte
 // swizzle (no multicast).  Every wait is bounded.
 #include "prefill.cuh"
 #include "tc_common.cuh"
 
 namespace less {
 
-constexpr int PT_WORKERS = 128;
+constexpr int PT_WORKERS = 256;                    // 8 epilogue warps: two per tensor-memory lane quadrant
 constexpr int PT_THREADS = PT_WORKERS + 64;
 constexpr int PT_TILE = 128;                       // tokens per tile
 constexpr int PT_CHUNK = 64;                       // hidden units per GEMM1 chunk
@@ -94,7 +94,7 @@ __global__ void __launch_bounds__(PT_THREADS) psi_tc_kernel(const __grid_constan
     const __half* w3 = p.w_psi3 + (size_t)im.lh * R * R;
     for (int e = tid; e < R * R; e += PT_THREADS) sh->w3[e] = __half2float(w3[e]);
   }
-  if (warp == 5) tmem_alloc(&sh->tmem_base, 256);
+  if (warp == PT_WORKERS / 32 + 1) tmem_alloc(&sh->tmem_base, 256);
   fence_proxy_async_smem();
   tc_fence_before_sync();
   __syncthreads();
@@ -103,7 +103,7 @@ __global__ void __launch_bounds__(PT_THREADS) psi_tc_kernel(const __grid_constan
   volatile int* abortp = &sh->abort;
   int32_t* status = p.a.status;
 
-  if (warp == 4) {
+  if (warp == PT_WORKERS / 32) {
     // ---------------- TMA producer ----------------
     if (tid == PT_WORKERS) {
       const uint64_t stream_policy = l2_evict_first_policy();
@@ -119,7 +119,7 @@ __global__ void __launch_bounds__(PT_THREADS) psi_tc_kernel(const __grid_constan
         tma_load_2d_hint(kbuf + PT_KBYTES / 2, &tmap_k, 64, row, &sh->k_full, stream_policy);
       }
     }
-  } else if (warp == 5) {
+  } else if (warp == PT_WORKERS / 32 + 1) {
     // ---------------- MMA issuer ----------------
     if (tid == PT_WORKERS + 32) {
       constexpr uint32_t idesc1 = idesc_f16(128, PT_CHUNK, 0, 1);   // A = K tile (K-major), B = W1 (N-major)
@@ -164,26 +164,29 @@ __global__ void __launch_bounds__(PT_THREADS) psi_tc_kernel(const __grid_constan
       }
     }
   } else {
-    // ---------------- epilogue workers: thread = token row ----------------
+    // ---------------- epilogue workers ----------------
     const float c1 = sh->c1, c2 = sh->c2;
-    const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
+    const int quad = warp & 3, half = warp >> 2;
+    const int row = quad * 32 + (tid & 31);                         // token row of the tile = tensor-memory lane
+    const uint32_t lane_addr = tmem + ((uint32_t)(quad * 32) << 16);
     float* psi = p.a.ws_psi + (size_t)g * p.Sp * R;
-    unsigned char* hrow = hid + tid * 128;
+    unsigned char* hrow = hid + row * 128;
     uint32_t q = 0;
     for (int i = 0; i < ntiles && !*abortp; ++i) {
       for (int c = 0; c < nchunk && !*abortp; ++c, ++q) {
         const int b = q & 1;
         pt_wait(&sh->d1_full[b], (q >> 1) & 1, abortp, status, 36);
         tc_fence_after_sync();
-        uint32_t acc[PT_CHUNK];
+        uint32_t acc[PT_CHUNK / 2];                                  // this warp's 32 of the chunk's 64 columns
 #pragma unroll
-        for (int cc = 0; cc < PT_CHUNK / 16; ++cc) tmem_ld16(lane_addr + b * PT_CHUNK + cc * 16, acc + cc * 16);
+        for (int cc = 0; cc < PT_CHUNK / 32; ++cc)
+          tmem_ld16(lane_addr + b * PT_CHUNK + half * (PT_CHUNK / 2) + cc * 16, acc + cc * 16);
         tmem_ld_wait();
         tc_fence_before_sync();
         mbar_arrive_warp(&sh->d1_free[b]);
-        uint32_t phi_[PT_CHUNK / 2], plo_[PT_CHUNK / 2];
+        uint32_t phi_[PT_CHUNK / 4], plo_[PT_CHUNK / 4];
 #pragma unroll
-        for (int e = 0; e < PT_CHUNK / 2; ++e) {
+        for (int e = 0; e < PT_CHUNK / 4; ++e) {
           const float h0 = c1 * gelu_erf(__uint_as_float(acc[2 * e]));
           const float h1 = c1 * gelu_erf(__uint_as_float(acc[2 * e + 1]));
           const __half2 hh = __floats2half2_rn(h0, h1);
@@ -194,12 +197,12 @@ __global__ void __launch_bounds__(PT_THREADS) psi_tc_kernel(const __grid_constan
         }
         pt_wait(&sh->hid_free, (q & 1) ^ 1, abortp, status, 37);
 #pragma unroll
-        for (int ch = 0; ch < 8; ++ch) {               // 16-byte chunk ch of this row, 128-byte swizzle
-          const int off = (ch ^ (tid & 7)) << 4;
+        for (int cq = 0; cq < 4; ++cq) {               // 16-byte chunk half * 4 + cq of this row, 128-byte swizzle
+          const int off = ((half * 4 + cq) ^ (row & 7)) << 4;
           *reinterpret_cast<uint4*>(hrow + off) =
-              make_uint4(phi_[ch * 4], phi_[ch * 4 + 1], phi_[ch * 4 + 2], phi_[ch * 4 + 3]);
+              make_uint4(phi_[cq * 4], phi_[cq * 4 + 1], phi_[cq * 4 + 2], phi_[cq * 4 + 3]);
           *reinterpret_cast<uint4*>(hrow + 16384 + off) =
-              make_uint4(plo_[ch * 4], plo_[ch * 4 + 1], plo_[ch * 4 + 2], plo_[ch * 4 + 3]);
+              make_uint4(plo_[cq * 4], plo_[cq * 4 + 1], plo_[cq * 4 + 2], plo_[cq * 4 + 3]);
         }
         fence_proxy_async_smem();
         mbar_arrive_warp(&sh->hid_full);
@@ -207,16 +210,17 @@ __global__ void __launch_bounds__(PT_THREADS) psi_tc_kernel(const __grid_constan
       pt_wait(&sh->g2_full, i & 1, abortp, status, 38);
       tc_fence_after_sync();
       uint32_t g2[PT_W2N];
-      tmem_ld16(lane_addr + 128, g2);
-      tmem_ld_wait();
+      if (half == 0) {                                 // warp-uniform: one warp per quadrant finishes the rows
+        tmem_ld16(lane_addr + 128, g2);
+        tmem_ld_wait();
+      }
       tc_fence_before_sync();
       mbar_arrive_warp(&sh->g2_free);
-      float gv[R];
+      const int j = jbeg + i * PT_TILE + row;
+      if (half == 0 && j < jend) {
+        float gv[R], out[R];
 #pragma unroll
-      for (int r = 0; r < R; ++r) gv[r] = c2 * gelu_erf(__uint_as_float(g2[r]));
-      const int j = jbeg + i * PT_TILE + tid;
-      if (j < jend) {
-        float out[R];
+        for (int r = 0; r < R; ++r) gv[r] = c2 * gelu_erf(__uint_as_float(g2[r]));
 #pragma unroll
         for (int r = 0; r < R; ++r) {
           float s = 0.f;
@@ -234,7 +238,7 @@ __global__ void __launch_bounds__(PT_THREADS) psi_tc_kernel(const __grid_constan
   drain_after_abort(abortp);
   tc_fence_before_sync();
   __syncthreads();
-  if (warp == 5) tmem_dealloc(tmem, 256);
+  if (warp == PT_WORKERS / 32 + 1) tmem_dealloc(tmem, 256);
 }
 
 bool psi_tc_supported(const Dims& d) { return d.Rp == 512 || d.Rp == 256 || d.Rp == 128 || d.Rp == 64; }
