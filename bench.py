@@ -49,6 +49,8 @@ def parse_args():
     ap.add_argument("--full-cache", action="store_true",
                     help="context run: slots >= prompt + steps, so nothing is ever evicted")
     ap.add_argument("--no-state", action="store_true", help="context run: sparse policy alone (Baseline+)")
+    ap.add_argument("--batch", type=int, default=0,
+                    help="override the workload's batch (smaller captures for ncu; named in config.workload)")
     return ap.parse_args()
 
 
@@ -419,6 +421,8 @@ def run_prefill(args):
         dist.init_process_group("nccl", device_id=torch.device(dev))
     build.build()
     w = wl.CONFIGS[args.config]
+    if args.batch:
+        w = w.with_(batch=args.batch)
     K_steps, W_steps = args.steps, max(args.warmup, 3)
     Wt = wl.make_weights(w, dev)
     ctx = binding.from_workload(w, Wt, dev, max_prefill_layers=1)
@@ -492,8 +496,10 @@ def run_prefill(args):
                 "value": tokens * K_steps / (ms * 1e-3), "unit": "head-tokens/s", "n_gpus": world, "steps": K_steps,
                 "warmup": W_steps, "ms_per_step": ms / K_steps, "higher_is_better": True, "scaling": "weak",
                 "vs_baseline": None, "dtype": "f16 inputs, f32 accumulate", "data": "synthetic",
-                "config": {"workload": "cfg5 prefill compression (B=8, 32 heads, one layer per step, prompt 32768, "
-                                       "1638+1638 slots, R=16)", "instances_per_step": w.batch * w.heads,
+                "config": {"workload": f"cfg5 prefill compression (B={w.batch}, 32 heads, one layer per step, "
+                                       "prompt 32768, 1638+1638 slots, R=16)"
+                                       + (" [batch reduced for profiling]" if args.batch else ""),
+                           "instances_per_step": w.batch * w.heads,
                            "l2": "6.3 GB of Q, K, V per step exceed the 126 MB L2"},
                 "clocks": clocks,
                 "e2e": {"value": tokens / (ms_e2e * 1e-3), "unit": "head-tokens/s",

@@ -25,6 +25,7 @@
  *   - Environment, read by less_create: LESS_LOG (explain host-side failures on
  *     stderr), LESS_FEATURE_KERNEL=gemv|plain (CUDA-core feature-map kernels),
  *     LESS_NO_OVERLAP (no programmatic dependent launch of the decode kernel),
+ *     LESS_SCORE_KERNEL=plain (CUDA-core prompt scoring),
  *     LESS_FEATURE_STAGES=n (cap on the feature kernels' weight ring).
  */
 #ifndef LESS_B200_H
