@@ -30,6 +30,11 @@ namespace less {
 constexpr int FT_EPI_WARPS = 8;
 constexpr int FT_EPI_THREADS = FT_EPI_WARPS * 32;
 constexpr int FT_THREADS = 64 + FT_EPI_THREADS;   // warp 0 TMA, warp 1 MMA, warps 2..9 epilogue
+// The larger-batch kernel runs four epilogue warps per lane quadrant: its GELU chains are long and
+// dependent, and with two warps per scheduler the issue slots sat idle (4700 cycles per chunk
+// measured for 32 GELUs per thread).
+constexpr int FL_EPI_WARPS = 16;
+constexpr int FL_THREADS = 64 + FL_EPI_WARPS * 32;
 constexpr int FT_CHUNK = 128;                     // hidden units per GEMM1
 constexpr int FT_STAGE_BYTES = FT_CHUNK * kHeadDim * 2;
 constexpr int FT_MAX_STAGES = 6;
@@ -103,7 +108,7 @@ __device__ __forceinline__ void ft_produce(const CUtensorMap* tm_q, const CUtens
 }
 
 template <int R>
-__global__ void __launch_bounds__(FT_THREADS) feature_tc_kernel(
+__global__ void __launch_bounds__(FL_THREADS) feature_tc_kernel(
     const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
     const __grid_constant__ CUtensorMap tm_w1phi, const __grid_constant__ CUtensorMap tm_w1psi, FmParams p,
     FtGeom gm, int32_t* status) {
@@ -127,14 +132,14 @@ __global__ void __launch_bounds__(FT_THREADS) feature_tc_kernel(
     }
     for (int s = 0; s < 2; ++s) {
       mbar_init(&sh->aux_full[s], 1);
-      mbar_init(&sh->aux_empty[s], 1 + FT_EPI_WARPS);
+      mbar_init(&sh->aux_empty[s], 1 + FL_EPI_WARPS);
       mbar_init(&sh->d1_full[s], 1);
-      mbar_init(&sh->d1_free[s], FT_EPI_WARPS);
+      mbar_init(&sh->d1_free[s], FL_EPI_WARPS);
     }
-    mbar_init(&sh->hid_full, FT_EPI_WARPS);
+    mbar_init(&sh->hid_full, FL_EPI_WARPS);
     mbar_init(&sh->hid_free, 1);
     mbar_init(&sh->d2_full, 1);
-    mbar_init(&sh->d2_free, FT_EPI_WARPS);
+    mbar_init(&sh->d2_free, FL_EPI_WARPS);
     // a CTA that starts after another one has given up skips every wait: the grid drains at once
     sh->abort = *reinterpret_cast<volatile int32_t*>(status) != 0;
     mbar_fence_init();
@@ -220,9 +225,9 @@ __global__ void __launch_bounds__(FT_THREADS) feature_tc_kernel(
     }
   } else {
     // ---------------- epilogue warps ----------------
-    const int ew = warp - 2;                   // 0..7
+    const int ew = warp - 2;                   // 0..15
     const int quad = warp & 3;                 // tensor-memory lane quadrant this warp may read
-    const int hf = ew >> 2;                    // which half of the token blocks
+    const int hf = ew >> 2;                    // which quarter of the token blocks (0..3)
     const int j = quad * 32 + lane;            // hidden unit inside the chunk = accumulator lane
     const uint32_t lane_addr = tmem + ((uint32_t)(quad * 32) << 16);
     unsigned char* hrow = hbuf + (j >> 3) * 128 + (j & 7) * 16;
@@ -240,27 +245,27 @@ __global__ void __launch_bounds__(FT_THREADS) feature_tc_kernel(
         // ago are complete (their D2 was read), and the first hid_full arrival below publishes it
         const uint4* src = reinterpret_cast<const uint4*>(w2raw + a * w2bytes);
         unsigned char* dst = w2buf + a * w2bytes;
-        for (int u = tid - 64; u < Rp * 2; u += FT_EPI_THREADS)
+        for (int u = tid - 64; u < Rp * 2; u += FL_EPI_WARPS * 32)
           *reinterpret_cast<uint4*>(dst + ((size_t)(u & 1) * Rp + (u >> 1)) * 16) = src[u];
       }
       for (int c = 0; c < nchunk && !*abortp; ++c, ++q) {
         const int b = q & 1;
         wait_or_give_up(&sh->d1_full[b], (q >> 1) & 1, abortp, status, 47);
         tc_fence_after_sync();
-        // this warp's token blocks: hf, hf + 2, ...   (at most 8 of the 16 blocks of a 128-token tile)
-        uint32_t acc[8][8];
+        // this warp's token blocks: hf, hf + 4  (a tile has at most 8 blocks of 8 tokens)
+        uint32_t acc[2][8];
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          const int blk = hf + 2 * i;
+        for (int i = 0; i < 2; ++i) {
+          const int blk = hf + 4 * i;
           if (blk < nblk) tmem_ld8(lane_addr + b * npad + blk * 8, acc[i]);
         }
         tmem_ld_wait();
         tc_fence_before_sync();
         mbar_arrive_warp(&sh->d1_free[b]);
-        uint4 hi[8], lo[8];
+        uint4 hi[2], lo[2];
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          const int blk = hf + 2 * i;
+        for (int i = 0; i < 2; ++i) {
+          const int blk = hf + 4 * i;
           if (blk < nblk) {
             uint32_t ph[4], pl[4];
 #pragma unroll
@@ -280,8 +285,8 @@ __global__ void __launch_bounds__(FT_THREADS) feature_tc_kernel(
         }
         wait_or_give_up(&sh->hid_free, (q & 1) ^ 1, abortp, status, 48);
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          const int blk = hf + 2 * i;
+        for (int i = 0; i < 2; ++i) {
+          const int blk = hf + 4 * i;
           if (blk < nblk) {
             *reinterpret_cast<uint4*>(hrow + blk * 2048) = hi[i];
             *reinterpret_cast<uint4*>(hrow + hbytes + blk * 2048) = lo[i];
@@ -629,11 +634,11 @@ int launch_feature_tc(less_ctx* c, const FmParams& p, cudaStream_t s) {
   if (d.R == 8) {
     if (cudaFuncSetAttribute(feature_tc_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
       return fail_cuda("shared memory opt-in of feature_tc_kernel");
-    feature_tc_kernel<8><<<grid, FT_THREADS, smem, s>>>(tq, tk, tw1a, tw1b, p, gm, c->a.status);
+    feature_tc_kernel<8><<<grid, FL_THREADS, smem, s>>>(tq, tk, tw1a, tw1b, p, gm, c->a.status);
   } else {
     if (cudaFuncSetAttribute(feature_tc_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
       return fail_cuda("shared memory opt-in of feature_tc_kernel");
-    feature_tc_kernel<16><<<grid, FT_THREADS, smem, s>>>(tq, tk, tw1a, tw1b, p, gm, c->a.status);
+    feature_tc_kernel<16><<<grid, FL_THREADS, smem, s>>>(tq, tk, tw1a, tw1b, p, gm, c->a.status);
   }
   return check_launch("feature_tc_kernel");
 }
