@@ -91,6 +91,23 @@ def decode_bytes(w, n_live, evicting=True, no_state=False):
     return w.instances * per
 
 
+def max_over_ranks(values, device, world):
+    """Replicas only: every rank runs the whole workload on its own GPU and the job's time is the
+    slowest rank's.  Element-wise maximum of `values` over the ranks (identity for one rank)."""
+    if world <= 1:
+        return [float(v) for v in values]
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([float(v) for v in values], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t]
+
+
+def job_throughput(units_per_rank, steps, ms, world):
+    """Whole-job units per second: all ranks' units over the slowest rank's time."""
+    return units_per_rank * world * steps / (ms * 1e-3)
+
+
 class ClockSampler:
     """Samples SM clock and clock-event reasons through NVML (read-only) every
     10 ms on a thread while the timed region runs."""
@@ -338,15 +355,11 @@ def run_b200(args):
     if status != 0:
         raise RuntimeError(f"device status {status}")
 
-    if world > 1:
-        t = torch.tensor([ms, ms_e2e], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms, ms_e2e = float(t[0]), float(t[1])
+    ms, ms_e2e = max_over_ranks([ms, ms_e2e], dev, world)
 
     if rank == 0:
-        units = w.instances * world
-        value = units * K_steps / (ms * 1e-3)
-        e2e_value = units * K_steps / (ms_e2e * 1e-3)
+        value = job_throughput(w.instances, K_steps, ms, world)
+        e2e_value = job_throughput(w.instances, K_steps, ms_e2e, world)
         peak, peak_kind = peaks()
         n_live = min(w_run.slots, w.prompt + W_steps)
         evicting = not args.full_cache
@@ -478,10 +491,7 @@ def run_prefill(args):
     ms_e2e = 1e3 * (time.perf_counter() - tw0) / n_e2e
     if ctx.poll_status() != 0:
         raise RuntimeError("device status")
-    if world > 1:
-        t = torch.tensor([ms, ms_e2e], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms, ms_e2e = float(t[0]), float(t[1])
+    ms, ms_e2e = max_over_ranks([ms, ms_e2e], dev, world)
     if rank == 0:
         tokens = w.batch * w.heads * w.prompt * world
         fl = prefill_flops(w)
