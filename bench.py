@@ -32,8 +32,8 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures
 # summarised under profiles/ (None until a capture of that kernel/workload exists)
 NCU_TRAFFIC_BYTES = {
-    (2, "feature_map"): 285.92e6 + 8.43e6,   # profiles/decode_step_cfg2.md
-    (2, "decode"): 113.87e6 + 3.58e6,
+    (2, "feature_map"): 285.93e6 + 5.82e6,   # profiles/decode_step_cfg2.md
+    (2, "decode"): 113.87e6 + 3.10e6,
 }
 
 
@@ -236,6 +236,8 @@ def workload_config(w, args):
             2: "cfg2 Llama-2-7B shape (B=1, 32 layers x 32 heads, prompt 2048, 102+102 slots, R=8)",
             3: "cfg3 batched serving (B=64, 32 layers x 32 heads, prompt 1024, 102+102 slots, R=8)",
             4: "cfg4 long context (B=4, 40 layers x 40 heads, prompt 16384, 327+327 slots, R=16)"}[w.cfg_id]
+    if getattr(args, "batch", 0):
+        name += f" [batch set to {w.batch} for profiling]"
     c = {"workload": name, "instances": w.instances, "slots": w.slots, "rank": w.rank,
          "prompt": w.prompt, "l2": "bytes touched per step exceed the 126 MB L2"
          if w.cfg_id != 1 else "L2 flushed by a 256 MB write between steps is NOT done: cfg1 is launch-bound"}
@@ -266,6 +268,8 @@ def run_b200(args):
     binding.lib()
 
     w = wl.CONFIGS[args.config]
+    if args.batch:
+        w = w.with_(batch=args.batch)
     K_steps, W_steps = args.steps, args.warmup
     total_steps = K_steps * 3 + W_steps + 2
     heavy, recent, flags = w.heavy, w.recent, 0
