@@ -18,6 +18,7 @@ Paper passages followed:
   * Section 2.1 / Section 4  H2O policy: accumulated attention probabilities,
                     equal heavy/recent split, even-floored token counts (Table 1)
   * Section 3.1     the prompt phase is regular attention (H_0 = 0, z_0 = 0)
+  * Section 4       Lambda-masking as the sparse policy: the first tokens plus the most recent ones
 
 Readings where the paper is silent (none of them is fixed by a printed number,
 so they are "parity unpinned" by the paper and fixed by this build's design
@@ -93,9 +94,15 @@ class LessInstance:
     def __init__(self, head_dim: int, rank: int, heavy: int, recent: int,
                  phi_fn: Callable[[np.ndarray], np.ndarray],
                  psi_fn: Callable[[np.ndarray], np.ndarray],
-                 score_norm: str = "less", use_state: bool = True):
+                 score_norm: str = "less", use_state: bool = True, policy: str = "h2o"):
         if recent < 1 or heavy < 0:
             raise ValueError("need recent >= 1 and heavy >= 0")
+        if policy not in ("h2o", "lambda"):
+            raise ValueError("policy is 'h2o' or 'lambda'")
+        # 'lambda' = Lambda-masking (Section 4: "the cache consists of the first 4 and most recent
+        # tokens"): `heavy` counts the first tokens that are always kept, `recent` the window;
+        # accumulated scores play no role in it.
+        self.policy = policy
         if score_norm not in ("less", "sparse"):
             raise ValueError("score_norm is 'less' or 'sparse'")
         self.D, self.R = int(head_dim), int(rank)
@@ -157,13 +164,18 @@ class LessInstance:
             acc[:r1] += P.sum(axis=0)                         # H2O: column sums, diagonal included
         self.t = S
         pos = np.arange(S, dtype=np.int64)
+        if self.policy == "lambda":
+            acc = np.zeros(S)                                 # the policy keeps no scores
         if S <= self.N:
             keep = pos
             evict = pos[:0]
         else:
-            cand = pos[: S - self.recent]                     # recent window is protected
-            order = np.lexsort((cand, acc[cand]))             # key (acc, pos) ascending
-            evict = np.sort(cand[order[: S - self.N]])
+            if self.policy == "lambda":
+                evict = pos[self.heavy: S - self.recent]      # everything between the first tokens and the window
+            else:
+                cand = pos[: S - self.recent]                 # recent window is protected
+                order = np.lexsort((cand, acc[cand]))         # key (acc, pos) ascending
+                evict = np.sort(cand[order[: S - self.N]])
             keep_mask = np.ones(S, dtype=bool)
             keep_mask[evict] = False
             keep = pos[keep_mask]
@@ -201,10 +213,14 @@ class LessInstance:
         pos = np.concatenate([self.pos, np.array([t], dtype=np.int64)])
         evicted_pos, gap, dH, dz = -1, None, None, None
         if pos.size > self.N:
-            cand = np.nonzero(pos <= t - self.recent)[0]
-            order = np.lexsort((pos[cand], acc[cand]))        # (acc, pos) ascending
+            if self.policy == "lambda":
+                cand = np.nonzero(pos >= self.heavy)[0]       # never one of the first tokens
+                order = np.argsort(pos[cand])                 # the oldest of the others leaves the window
+            else:
+                cand = np.nonzero(pos <= t - self.recent)[0]
+                order = np.lexsort((pos[cand], acc[cand]))    # (acc, pos) ascending
             vic = int(cand[order[0]])
-            if cand.size > 1:
+            if cand.size > 1 and self.policy == "h2o":
                 a0, a1 = acc[cand[order[0]]], acc[cand[order[1]]]
                 gap = abs(a1 - a0) / max(abs(a0), abs(a1), 1e-300)
             evicted_pos = int(pos[vic])

@@ -44,7 +44,7 @@ def torch_phi(q, w1, w2):
     return g(g(q @ w1) @ w2).abs()
 
 
-def run_instance(w, head=0, score_norm="less", use_state=True, heavy=None, recent=None):
+def run_instance(w, head=0, score_norm="less", use_state=True, heavy=None, recent=None, policy="h2o"):
     """Oracle free run of one head of workload w; returns instance + history."""
     W = wl.make_weights(w)
     Q, K, V = wl.make_prompt(w, 0, 1)
@@ -52,7 +52,7 @@ def run_instance(w, head=0, score_norm="less", use_state=True, heavy=None, recen
     phi_fn, psi_fn = lo.make_mlp_maps(*wts)
     inst = lo.LessInstance(w.head_dim, w.rank, w.heavy if heavy is None else heavy,
                            w.recent if recent is None else recent, phi_fn, psi_fn,
-                           score_norm=score_norm, use_state=use_state)
+                           score_norm=score_norm, use_state=use_state, policy=policy)
     q_all = [Q[0, 0, head].double().numpy()]
     k_all = [K[0, 0, head].double().numpy()]
     v_all = [V[0, 0, head].double().numpy()]
@@ -447,3 +447,50 @@ def test_planted_mistakes_are_caught(kind):
         if r["evicted_pos"] != victims[s] or not np.allclose(r["out"], outs[s], rtol=1e-10, atol=1e-13):
             bad = True
     assert bad, f"mutant {kind} slipped through the replay pin"
+
+
+# --------------------------------------------------------------------------- #
+# Lambda-masking as the sparse policy (Section 4: the first tokens plus the most recent ones)
+# --------------------------------------------------------------------------- #
+@pytest.mark.parametrize("use_state", [True, False])
+def test_lambda_masking_closed_forms(use_state):
+    """The kept set has a closed form at every step; with the state off the output is the
+    softmax over exactly that set (the streaming pattern), with it on H and z are the plain sums
+    over every other position (Eq. 6) and the step obeys Eq. 3 with those sums."""
+    sinks, window = 4, 7
+    w = tiny(cfg_id=96, S=33, T=14, heavy=sinks, recent=window, D=16, R=4)
+    inst, _, steps, (_, Kh, Vh), wts = run_instance(w, use_state=use_state, policy="lambda")
+    Kt, Vt = torch.tensor(Kh), torch.tensor(Vh)
+    for i, r in enumerate(steps):
+        t = w.prompt + i                                             # position of the new token
+        kept = list(range(sinks)) + list(range(t - window, t))      # sinks + the `window` latest cached tokens
+        assert list(r["kept_before"]) == kept
+        assert r["evicted_pos"] == t - window                        # the oldest token of the window leaves
+        idx = kept + [t]
+        e = torch.exp(Kt[idx] @ torch.tensor(r["q"]) / math.sqrt(w.head_dim))
+        if not use_state:
+            p = e / e.sum()
+            assert np.allclose(r["out"], (p @ Vt[idx]).numpy(), rtol=1e-12, atol=1e-14)
+        else:
+            gone = [j for j in range(t) if j not in kept]
+            psi = torch_psi(Kh[gone], *wts[2:])
+            phi = torch_phi(r["q"][None], *wts[:2])[0]
+            num = phi @ (psi.T @ Vt[gone]) + e @ Vt[idx]
+            den = phi @ psi.sum(0) + e.sum()
+            assert np.allclose(r["out"], (num / den).numpy(), rtol=1e-10, atol=1e-13)
+    t_end = w.prompt + w.steps
+    assert list(inst.pos) == list(range(sinks)) + list(range(t_end - window, t_end))
+    assert sorted(inst.evicted) == list(range(sinks, t_end - window))
+    if not use_state:
+        assert (inst.H == 0).all() and (inst.z == 0).all()
+
+
+def test_lambda_masking_short_context_and_budget_that_holds_everything():
+    w = tiny(cfg_id=97, S=6, T=9, heavy=2, recent=5, D=16, R=4)    # 7 slots, prompt of 6: fills, then slides
+    inst, _, steps, _, _ = run_instance(w, policy="lambda")
+    assert [r["evicted_pos"] for r in steps] == [-1] + list(range(2, 10))
+    w = tiny(cfg_id=98, S=12, T=5, D=16)
+    a, _, sa, _, _ = run_instance(w, heavy=4, recent=30, policy="lambda")
+    b, _, sb, _, _ = run_instance(w, heavy=30, recent=30, policy="h2o")
+    for x, y in zip(sa, sb):                                         # nothing evicted: the policy cannot matter
+        assert np.array_equal(x["out"], y["out"]) and x["evicted_pos"] == -1
