@@ -49,6 +49,8 @@ def parse_args():
     ap.add_argument("--full-cache", action="store_true",
                     help="context run: slots >= prompt + steps, so nothing is ever evicted")
     ap.add_argument("--no-state", action="store_true", help="context run: sparse policy alone (Baseline+)")
+    ap.add_argument("--lambda-masking", action="store_true",
+                    help="context run: Lambda-masking as the sparse policy (first 4 tokens + window, same slot count)")
     ap.add_argument("--batch", type=int, default=0,
                     help="override the workload's batch (smaller captures for ncu; named in config.workload)")
     return ap.parse_args()
@@ -243,6 +245,8 @@ def workload_config(w, args):
          if w.cfg_id != 1 else "L2 flushed by a 256 MB write between steps is NOT done: cfg1 is launch-bound"}
     if getattr(args, "full_cache", False):
         c["variant"] = "full cache (no eviction)"
+    if getattr(args, "lambda_masking", False):
+        c["variant"] = "Lambda-masking policy (first 4 tokens + recent window)"
     if getattr(args, "no_state", False):
         c["variant"] = "sparse policy alone (Baseline+)"
     return c
@@ -279,6 +283,9 @@ def run_b200(args):
         flags |= binding.LESS_NO_STATE
         heavy += 2 if w.rank == 8 else 4      # Baseline+: slots matching H's storage (Section 4)
         recent += 2 if w.rank == 8 else 4
+    if args.lambda_masking:
+        flags |= binding.LESS_POLICY_LAMBDA
+        heavy, recent = 4, heavy + recent - 4
     w_run = w.with_(heavy=heavy, recent=recent)
 
     # replicas: every rank runs the whole workload on its own GPU, no collective in the path

@@ -63,7 +63,14 @@ enum {
   LESS_SCORE_NORM_SPARSE = 1u,
   /* Sparse policy alone (the paper's Baseline / Baseline+, Section 4):
    * evicted pairs are dropped, H and z stay zero. */
-  LESS_NO_STATE = 2u
+  LESS_NO_STATE = 2u,
+  /* Lambda-masking as the sparse policy (Section 4: "the cache consists of the
+   * first 4 and most recent tokens") instead of H2O: `heavy` counts the first
+   * positions, which are never evicted, `recent` the sliding window; the prompt
+   * keeps positions [0, heavy) and the last `recent`, a decode step evicts the
+   * lowest position >= heavy.  Accumulated scores are not used (prompt scoring
+   * is skipped unless attn_out is asked for); evicted pairs go to H, z as usual. */
+  LESS_POLICY_LAMBDA = 4u
 };
 
 typedef struct less_config {

@@ -90,7 +90,7 @@ struct DecParams {
   float* out;                                           // [I, D]
   int32_t* evicted_pos;                                 // [I] or null
   Arena a;
-  int N, Np, recent, t;
+  int N, Np, heavy, recent, t;
   uint32_t flags;
 };
 
@@ -243,13 +243,16 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_kernel(DecParams p) {
   int32_t* posb = p.a.pos + inst * (size_t)p.Np;
   float* accb = p.a.acc + inst * (size_t)p.Np;
   const bool full = (n == N);
+  const bool lambda_policy = (p.flags & LESS_POLICY_LAMBDA) != 0;
   unsigned long long best = ~0ull;
   for (int i = tid; i < n; i += DEC_THREADS) {
     const float a = accb[i] + s_sc[i] * inv;
     accb[i] = a;
     if (full) {
       const int ps = posb[i];
-      if (ps <= p.t - p.recent) {
+      if (lambda_policy) {                           // Lambda-masking: the oldest position past the first tokens
+        if (ps >= p.heavy) best = (unsigned long long)(unsigned int)ps < best ? (unsigned int)ps : best;
+      } else if (ps <= p.t - p.recent) {             // H2O: lowest (accumulated score, position) outside the window
         const unsigned long long key =
             ((unsigned long long)__float_as_uint(a) << 32) | (unsigned int)ps;
         best = key < best ? key : best;
@@ -317,7 +320,7 @@ int launch_decode(less_ctx* c, const void* q, const void* k, const void* v, void
   p.out = (float*)out;
   p.evicted_pos = evicted_pos;
   p.a = c->a;
-  p.N = d.N; p.Np = d.Np; p.recent = d.recent; p.t = (int)c->t;
+  p.N = d.N; p.Np = d.Np; p.heavy = d.heavy; p.recent = d.recent; p.t = (int)c->t;
   p.flags = d.flags;
   const size_t smem = (size_t)(d.Np + 4 + DEC_RG * kHeadDim) * 4;
   LaunchScope scope(c, LESS_KERNEL_DECODE, s);

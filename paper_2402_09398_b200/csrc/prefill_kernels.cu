@@ -211,6 +211,12 @@ __global__ void __launch_bounds__(SEL_THREADS) select_kernel(PfParams p) {
     for (int j = tid; j < S; j += SEL_THREADS) slot_of[j] = j;
     return;
   }
+  if (p.flags & LESS_POLICY_LAMBDA) {
+    // Lambda-masking (Section 4): the first `heavy` positions and the last `recent` stay
+    for (int j = tid; j < S; j += SEL_THREADS)
+      slot_of[j] = j < p.heavy ? j : (j >= S - p.recent ? p.heavy + j - (S - p.recent) : -1);
+    return;
+  }
   const int C = S - p.recent;                    // candidates: positions [0, C)
   unsigned int thr = 0xffffffffu;                // threshold bit pattern (acc >= 0: monotone)
   int need = 0;                                  // how many of the == threshold to keep
@@ -341,7 +347,7 @@ __global__ void __launch_bounds__(GA_THREADS) gather_kernel(PfParams p) {
           __ldg(reinterpret_cast<const uint4*>(p.V + src) + (sub - 16));
     if (sub == 0) {
       p.a.pos[im.inst * (size_t)p.Np + sl] = j;
-      p.a.acc[im.inst * (size_t)p.Np + sl] = acc[j];
+      p.a.acc[im.inst * (size_t)p.Np + sl] = (p.flags & LESS_POLICY_LAMBDA) ? 0.f : acc[j];   // no scores under Lambda-masking
     }
     if (sub < R) p.a.psic[(im.inst * (size_t)p.N + sl) * R + sub] = use_state ? psi[(size_t)j * R + sub] : 0.f;
   }
@@ -395,7 +401,9 @@ int launch_prefill_group(less_ctx* c, int layer0, int nl, int lj0, int layer_cou
     nsplit = (S + split_tokens - 1) / split_tokens;
   }
   p.nsplit = nsplit; p.split_tokens = split_tokens;
-  if (S > 0) {
+  // Lambda-masking needs no scores; the row statistics are still needed for the prompt's attention output
+  const bool need_scores = !(d.flags & LESS_POLICY_LAMBDA) || attn_out != nullptr;
+  if (S > 0 && need_scores) {
     const int tiles = (S + PF_TILE - 1) / PF_TILE;
     if (c->score_path == 1 && score_tc_supported()) {
       const int rc = launch_score_tc(c, p, G, s);

@@ -38,7 +38,7 @@ def _prefill_all(ctx, w, with_out=True, prompt=None):
 
 @pytest.mark.parametrize("variant", ["base", "rank16", "boosted", "ragged", "sparse_norm", "no_state",
                                      "scaled", "heavy0", "recent1", "hidden256", "long_prompt",
-                                     "cuda_core_scoring"])
+                                     "cuda_core_scoring", "lambda_masking", "lambda_no_state"])
 def test_prefill_and_teacher_forced_decode(variant, monkeypatch):
     import harness
     flags, psi_scale = 0, None
@@ -63,6 +63,10 @@ def test_prefill_and_teacher_forced_decode(variant, monkeypatch):
         w = small(79, heavy=30, recent=1)
     elif variant == "hidden256":
         w = small(80, hidden=256, weight_std=0.05)
+    elif variant == "lambda_masking":       # first 4 tokens + sliding window, evicted pairs into H, z
+        w, flags = small(58, heavy=4, recent=36, weight_std=0.1), 4
+    elif variant == "lambda_no_state":
+        w, flags = small(57, heavy=4, recent=21, prompt=211), 4 | 2
     elif variant == "long_prompt":          # several streamed 256-row tiles per scoring CTA, rings wrap
         w = small(60, prompt=1100, batch=1, heads=2, steps=4, heavy=50, recent=30)
     elif variant == "cuda_core_scoring":    # the prompt scoring kernels used when no tensor map can be made
