@@ -14,12 +14,12 @@
 // so the GELU work of the epilogue grows with the number of tokens, not with the
 // 128-row tile, and a batch of one costs one GELU per thread and chunk.
 // Epilogue warps (two per lane quadrant) read D1^T from tensor memory, apply
-// c1 * gelu, split the result into fp16 hi + lo (one fp16 rounding of the hidden
+// gelu, split the result into fp16 hi + lo (one fp16 rounding of the hidden
 // layer would cost ~2e-3 on psi) and store it, tokens contiguous, as the M-major
 // A operand of
 //     D2[tokens x 16] += H[tokens x 128 hidden] * W2[chunk rows, :]       (GEMM2)
 // whose accumulator lives in tensor memory across the chunks.  After the last
-// chunk: c2 * gelu, W3 (psi only) and the absolute value on CUDA cores.
+// chunk: c2 * gelu(c1 * .), W3 (psi only) and the absolute value on CUDA cores.
 // The hidden activations never leave the SM (the paper's "absorbed activation",
 // Section 3.2, taken to the whole MLP).  No multicast; every wait is bounded.
 #include "feature_gemv.cuh"
@@ -271,8 +271,10 @@ __global__ void __launch_bounds__(FL_THREADS) feature_tc_kernel(
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
               // columns past the last token hold products with zero-filled rows: no GELU spent on them
-              const float h0 = blk * 8 + 2 * e < nb ? c1 * gelu_erf(__uint_as_float(acc[i][2 * e])) : 0.f;
-              const float h1 = blk * 8 + 2 * e + 1 < nb ? c1 * gelu_erf(__uint_as_float(acc[i][2 * e + 1])) : 0.f;
+              // (c1 multiplies the layer-2 sums instead: the fp16 operand must not depend on how
+              // small that learnable scalar is)
+              const float h0 = blk * 8 + 2 * e < nb ? gelu_erf(__uint_as_float(acc[i][2 * e])) : 0.f;
+              const float h1 = blk * 8 + 2 * e + 1 < nb ? gelu_erf(__uint_as_float(acc[i][2 * e + 1])) : 0.f;
               const __half2 hh = __floats2half2_rn(h0, h1);
               const float2 hf2 = __half22float2(hh);
               const __half2 ll = __floats2half2_rn(h0 - hf2.x, h1 - hf2.y);
@@ -311,7 +313,7 @@ __global__ void __launch_bounds__(FL_THREADS) feature_tc_kernel(
       if (mine && j < nb) {
         float gv[R], out[R];
 #pragma unroll
-        for (int r = 0; r < R; ++r) gv[r] = c2 * gelu_erf(__uint_as_float(g2[r]));
+        for (int r = 0; r < R; ++r) gv[r] = c2 * gelu_erf(c1 * __uint_as_float(g2[r]));
         if (which) {
           const __half* w3 = &sh->w3[a][0];
 #pragma unroll

@@ -83,6 +83,7 @@ size_t carve(const Dims& d, char* base, Arena* a) {
   t.ws_hpart = (float*)take(Iw * kMaxSplit * (R * D + R) * 4);
   t.ws_psi = (float*)take(Iw * Sp * R * 4);
   t.ws_bx = (uint4*)take(Iw * (size_t)d.Sbx * 16);
+  t.ws_pmax = (int32_t*)take(Iw * 4);
   if (a) *a = t;
   return off;
 }

@@ -40,6 +40,7 @@ struct Arena {
   int32_t* ws_slot;  // [Iw][Sp]    slot of a prompt token, -1 = evicted
   float* ws_hpart;   // [Iw][kMaxSplit][R*D + R]  partial H, z per token split
   float* ws_psi;     // [Iw][Sp][R]  psi(k_j) of every prompt token
+  int32_t* ws_pmax;  // [Iw]        bit pattern of max psi over the instance's prompt tokens (scales the state build's fp16 operand)
   uint4* ws_bx;      // [Iw][Sbx]    per prompt row: -(m_i sqrt(D) - log2(1/l_i) / c) as three fp16 parts (column sums)
 };
 

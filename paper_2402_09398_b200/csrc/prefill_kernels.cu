@@ -206,7 +206,10 @@ __global__ void __launch_bounds__(SEL_THREADS) select_kernel(PfParams p) {
   const float* acc = p.a.ws_acc + (size_t)g * p.Sp;
   int32_t* slot_of = p.a.ws_slot + (size_t)g * p.Sp;
   const int S = p.S, N = p.N;
-  if (tid == 0) p.a.count[im.inst] = min(S, N);
+  if (tid == 0) {
+    p.a.count[im.inst] = min(S, N);
+    p.a.ws_pmax[g] = 0;                          // the psi kernels that follow take the maximum into it
+  }
   if (S <= N) {
     for (int j = tid; j < S; j += SEL_THREADS) slot_of[j] = j;
     return;
@@ -306,6 +309,7 @@ __global__ void __launch_bounds__(FM_THREADS) psi_kernel(PfParams p) {
   const __half* w2 = p.w_psi2 + (size_t)im.lh * p.Rp * R;
   const __half* w3 = p.w_psi3 + (size_t)im.lh * R * R;
   float* psi = p.a.ws_psi + (size_t)g * p.Sp * R;
+  float pmax = 0.f;
   for (int j0 = jbeg; j0 < jend; j0 += FM_BR) {
     const int nb = min(FM_BR, jend - j0);
     for (int e = tid; e < FM_BR * kHeadDim; e += FM_THREADS) {
@@ -315,8 +319,13 @@ __global__ void __launch_bounds__(FM_THREADS) psi_kernel(PfParams p) {
     __syncthreads();
     const float r = mlp_rows<R>(xs, part, hs, nb, w1, w2, w3, c1, c2, p.Rp, true);
     const int warp = tid >> 5, lane = tid & 31;
-    if (warp < nb && lane < R) psi[(size_t)(j0 + warp) * R + lane] = r;
+    if (warp < nb && lane < R) {
+      psi[(size_t)(j0 + warp) * R + lane] = r;
+      pmax = fmaxf(pmax, r);
+    }
   }
+  // psi >= 0: its bit pattern orders like an integer, and a maximum does not depend on the order
+  if (pmax > 0.f && pmax < INFINITY) atomicMax(p.a.ws_pmax + g, __float_as_int(pmax));
 }
 
 // ---- P4: kept rows go to their slots (K, V, position, score, psi) ----------- //

@@ -5,10 +5,10 @@
 // stays in shared memory for all of the split's tiles.  Per 128-token tile:
 //   GEMM1  D1[128 x 64] = Ktile[128 x 128] * W1[:, chunk]       8 chunks of 64 hidden units,
 //                                                               D1 double-buffered in tensor memory
-//   epilogue warps: tcgen05.ld D1 -> c1 * gelu -> fp16 hi + lo -> shared memory (A operands of GEMM2;
+//   epilogue warps: tcgen05.ld D1 -> gelu -> fp16 hi + lo -> shared memory (A operands of GEMM2;
 //                   a single fp16 rounding of the hidden layer costs ~2e-3 on individual psi vectors)
 //   GEMM2  G2[128 x 16] += (hidden_hi + hidden_lo)[128 x 64] * W2[chunk rows, :]
-//   after 8 chunks: tcgen05.ld G2 -> c2 * gelu -> W3 on CUDA cores -> abs -> psi[token][R]
+//   after 8 chunks: tcgen05.ld G2 -> c2 * gelu(c1 * .) -> W3 on CUDA cores -> abs -> psi[token][R]
 // Roles: warps 0-7 epilogue (lane quadrant = warp & 3, token row = tensor-memory lane; the two
 // warps of a quadrant split a chunk's 64 columns), warp 8 TMA producer, warp 9 MMA issuer.  Operands come in by TMA tiled loads with the 128-byte
 // swizzle (no multicast).  Every wait is bounded.
@@ -172,6 +172,7 @@ __global__ void __launch_bounds__(PT_THREADS) psi_tc_kernel(const __grid_constan
     float* psi = p.a.ws_psi + (size_t)g * p.Sp * R;
     unsigned char* hrow = hid + row * 128;
     uint32_t q = 0;
+    float pmax = 0.f;                                               // largest psi this thread has produced
     for (int i = 0; i < ntiles && !*abortp; ++i) {
       for (int c = 0; c < nchunk && !*abortp; ++c, ++q) {
         const int b = q & 1;
@@ -187,8 +188,10 @@ __global__ void __launch_bounds__(PT_THREADS) psi_tc_kernel(const __grid_constan
         uint32_t phi_[PT_CHUNK / 4], plo_[PT_CHUNK / 4];
 #pragma unroll
         for (int e = 0; e < PT_CHUNK / 4; ++e) {
-          const float h0 = c1 * gelu_erf(__uint_as_float(acc[2 * e]));
-          const float h1 = c1 * gelu_erf(__uint_as_float(acc[2 * e + 1]));
+          // c1 multiplies the layer-2 sums instead (same value): the fp16 hi + lo operand then never
+          // depends on how small the learnable scalar is (the paper initialises it to 1e-4)
+          const float h0 = gelu_erf(__uint_as_float(acc[2 * e]));
+          const float h1 = gelu_erf(__uint_as_float(acc[2 * e + 1]));
           const __half2 hh = __floats2half2_rn(h0, h1);
           const float2 hf = __half22float2(hh);
           const __half2 ll = __floats2half2_rn(h0 - hf.x, h1 - hf.y);
@@ -220,13 +223,14 @@ __global__ void __launch_bounds__(PT_THREADS) psi_tc_kernel(const __grid_constan
       if (half == 0 && j < jend) {
         float gv[R], out[R];
 #pragma unroll
-        for (int r = 0; r < R; ++r) gv[r] = c2 * gelu_erf(__uint_as_float(g2[r]));
+        for (int r = 0; r < R; ++r) gv[r] = c2 * gelu_erf(c1 * __uint_as_float(g2[r]));
 #pragma unroll
         for (int r = 0; r < R; ++r) {
           float s = 0.f;
 #pragma unroll
           for (int rr = 0; rr < R; ++rr) s = fmaf(gv[rr], sh->w3[rr * R + r], s);
           out[r] = fabsf(s);
+          pmax = fmaxf(pmax, out[r]);
         }
 #pragma unroll
         for (int r4 = 0; r4 < R / 4; ++r4)
@@ -234,6 +238,11 @@ __global__ void __launch_bounds__(PT_THREADS) psi_tc_kernel(const __grid_constan
               make_float4(out[r4 * 4], out[r4 * 4 + 1], out[r4 * 4 + 2], out[r4 * 4 + 3]);
       }
     }
+    // maximum over the split, into the instance's cell: psi >= 0, so its bit pattern orders like an
+    // integer, and a maximum does not depend on the order of the atomics
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) pmax = fmaxf(pmax, __shfl_xor_sync(0xffffffffu, pmax, o));
+    if ((tid & 31) == 0 && pmax > 0.f && pmax < INFINITY) atomicMax(p.a.ws_pmax + g, __float_as_int(pmax));
   }
   drain_after_abort(abortp);
   tc_fence_before_sync();

@@ -5,8 +5,8 @@
 //   * TMA brings the V tile [128 tokens x 128] into shared memory (128-byte swizzle);
 //     as the A operand it is "M-major": M = head dimension, K = tokens;
 //   * four worker warps read psi of their token, zero it for kept / out-of-range
-//     tokens, split it into fp16 hi + lo (so the fp16 tensor-core product keeps
-//     fp32 accuracy) and lay it out as the B operand [K = tokens, N = 2R];
+//     tokens, scale it by a per-instance power of two, split it into fp16 hi + lo (so the
+//     fp16 tensor-core product keeps fp32 accuracy) and lay it out as the B operand [K = tokens, N = 2R];
 //   * one thread issues tcgen05.mma: 8 k-steps into the H accumulator and 8 more
 //     with an all-ones A operand into the z accumulator, both in tensor memory.
 // After the last tile the workers read the accumulators back (tcgen05.ld), add
@@ -22,7 +22,6 @@ constexpr int ST_THREADS = ST_WORKERS + 64;      // + TMA warp + MMA warp
 constexpr int ST_STAGES = 2;
 constexpr int ST_TILE = 128;                     // tokens per tile
 constexpr int ST_VBYTES = ST_TILE * kHeadDim * 2;
-constexpr float kPsiScale = 256.f;               // keeps the lo parts in fp16's normal range
 
 struct StShared {
   uint64_t full_v[ST_STAGES];
@@ -123,6 +122,12 @@ __global__ void __launch_bounds__(ST_THREADS) state_tc_kernel(const __grid_const
     }
   } else {
     // ---------------- workers: B operand, then epilogue ----------------
+    // psi is scaled by a power of two so that the instance's largest value lands near 8192: the hi
+    // parts stay far from fp16's overflow and the lo parts as far from its underflow as they can be,
+    // whatever the magnitude of the trained maps (the paper initialises psi's scalars to 1e-4)
+    const float pmax = __int_as_float(p.a.ws_pmax[g]);
+    float scale = 1.f;
+    if (pmax > 0.f && pmax < INFINITY) scale = exp2f(fminf(fmaxf(floorf(log2f(8192.f / pmax)), -100.f), 100.f));
     const float* psi = p.a.ws_psi + (size_t)g * p.Sp * R;
     const int32_t* slot_of = p.a.ws_slot + (size_t)g * p.Sp;
     for (int i = 0; i < ntiles; ++i) {
@@ -143,7 +148,7 @@ __global__ void __launch_bounds__(ST_THREADS) state_tc_kernel(const __grid_const
       __align__(16) __half hi[R], lo[R];
 #pragma unroll
       for (int r = 0; r < R; ++r) {
-        const float x = v[r] * kPsiScale;
+        const float x = v[r] * scale;
         hi[r] = __float2half_rn(x);
         lo[r] = __float2half_rn(x - __half2float(hi[r]));
       }
@@ -166,7 +171,7 @@ __global__ void __launch_bounds__(ST_THREADS) state_tc_kernel(const __grid_const
     for (int c = 0; c < NB / 8; ++c) tmem_ld8(lane_addr + c * 8, acc + c * 8);
     tmem_ld_wait();
     float* hp = p.a.ws_hpart + ((size_t)g * kMaxSplit + split) * (R * kHeadDim + R);
-    const float inv = 1.0f / kPsiScale;
+    const float inv = 1.0f / scale;                    // exact: a power of two
 #pragma unroll
     for (int r = 0; r < R; ++r)
       hp[r * kHeadDim + tid] = (__uint_as_float(acc[r]) + __uint_as_float(acc[R + r])) * inv;

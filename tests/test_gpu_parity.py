@@ -38,7 +38,8 @@ def _prefill_all(ctx, w, with_out=True, prompt=None):
 
 @pytest.mark.parametrize("variant", ["base", "rank16", "boosted", "ragged", "sparse_norm", "no_state",
                                      "scaled", "heavy0", "recent1", "hidden256", "long_prompt",
-                                     "cuda_core_scoring", "lambda_masking", "lambda_no_state"])
+                                     "cuda_core_scoring", "lambda_masking", "lambda_no_state",
+                                     "tiny_scalars", "huge_psi"])
 def test_prefill_and_teacher_forced_decode(variant, monkeypatch):
     import harness
     flags, psi_scale = 0, None
@@ -67,6 +68,12 @@ def test_prefill_and_teacher_forced_decode(variant, monkeypatch):
         w, flags = small(58, heavy=4, recent=36, weight_std=0.1), 4
     elif variant == "lambda_no_state":
         w, flags = small(57, heavy=4, recent=21, prompt=211), 4 | 2
+    elif variant == "tiny_scalars":         # the paper initialises psi's learnable scalars to 1e-4
+        w = small(56, weight_std=0.1)
+        psi_scale = torch.full((w.layers, w.heads, 2), 1e-4)
+    elif variant == "huge_psi":             # psi of the order of 1e4: the fp16 operands must be rescaled
+        w = small(55, weight_std=0.2)
+        psi_scale = torch.full((w.layers, w.heads, 2), 40.0)
     elif variant == "long_prompt":          # several streamed 256-row tiles per scoring CTA, rings wrap
         w = small(60, prompt=1100, batch=1, heads=2, steps=4, heavy=50, recent=30)
     elif variant == "cuda_core_scoring":    # the prompt scoring kernels used when no tensor map can be made
