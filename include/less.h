@@ -140,10 +140,11 @@ int less_decode_step(less_ctx* ctx, const void* q, const void* k, const void* v,
                      int32_t* evicted_pos, void* cuda_stream);
 
 /* The same step for callers whose tensors live in host memory (Algorithm 1's
- * inputs and return value): copies q, k, v (host fp16 [B, L, H, D], ideally
- * pinned) to staging buffers inside the arena, runs less_decode_step, copies
- * out (host fp32 [B, L, H, D]) back, all on the given stream, and synchronises
- * it before returning. */
+ * inputs and return value): q, k, v are host fp16 [B, L, H, D], out host fp32
+ * [B, L, H, D].  q and k are copied to staging buffers inside the arena; v and
+ * out are read / written in place by the decode kernel when they lie in pinned
+ * (page-locked, device-mapped) memory, else they are staged and copied too.
+ * Everything runs on the given stream, which is synchronised before returning. */
 int less_decode_step_host(less_ctx* ctx, const void* q_host, const void* k_host, const void* v_host,
                           void* out_host, void* cuda_stream);
 

@@ -232,18 +232,36 @@ int less_decode_step(less_ctx* c, const void* q, const void* k, const void* v, v
   return LESS_OK;
 }
 
+// Device-visible alias of a host buffer: pinned (page-locked, mapped) memory can be read and
+// written by kernels directly over PCIe; pageable memory cannot (nullptr).
+static void* device_alias(const void* host) {
+  cudaPointerAttributes at;
+  if (cudaPointerGetAttributes(&at, host) != cudaSuccess) {
+    cudaGetLastError();                       // not a CUDA-known pointer: clear the error, use the staging path
+    return nullptr;
+  }
+  return at.type == cudaMemoryTypeHost ? at.devicePointer : nullptr;
+}
+
 int less_decode_step_host(less_ctx* c, const void* qh, const void* kh, const void* vh, void* outh,
                           void* stream) {
   if (!c || !qh || !kh || !vh || !outh) return LESS_ERR_NULL_POINTER;
   cudaStream_t s = (cudaStream_t)stream;
   const size_t nin = (size_t)c->d.I * c->d.D * 2, nout = (size_t)c->d.I * c->d.D * 4;
+  // q and k feed the feature-map kernel's TMA loads and are staged in the arena.  v and the output
+  // are touched once per instance by the decode kernel: from pinned host memory it reads / writes
+  // them in place, which saves two copy launches per step.
+  const void* v_dev = device_alias(vh);
+  void* out_dev = device_alias(outh);
+  if (((uintptr_t)v_dev & 15) || ((uintptr_t)out_dev & 15)) { v_dev = nullptr; out_dev = nullptr; }
   cudaError_t e = cudaMemcpyAsync(c->a.stage_q, qh, nin, cudaMemcpyHostToDevice, s);
   if (e == cudaSuccess) e = cudaMemcpyAsync(c->a.stage_k, kh, nin, cudaMemcpyHostToDevice, s);
-  if (e == cudaSuccess) e = cudaMemcpyAsync(c->a.stage_v, vh, nin, cudaMemcpyHostToDevice, s);
+  if (e == cudaSuccess && !v_dev) e = cudaMemcpyAsync(c->a.stage_v, vh, nin, cudaMemcpyHostToDevice, s);
   if (e != cudaSuccess) return LESS_ERR_CUDA;
-  int rc = less_decode_step(c, c->a.stage_q, c->a.stage_k, c->a.stage_v, c->a.stage_out, nullptr, s);
+  int rc = less_decode_step(c, c->a.stage_q, c->a.stage_k, v_dev ? v_dev : c->a.stage_v,
+                            out_dev ? out_dev : c->a.stage_out, nullptr, s);
   if (rc != LESS_OK) return rc;
-  e = cudaMemcpyAsync(outh, c->a.stage_out, nout, cudaMemcpyDeviceToHost, s);
+  if (!out_dev) e = cudaMemcpyAsync(outh, c->a.stage_out, nout, cudaMemcpyDeviceToHost, s);
   if (e == cudaSuccess) e = cudaStreamSynchronize(s);
   return e == cudaSuccess ? LESS_OK : LESS_ERR_CUDA;
 }

@@ -322,3 +322,29 @@ def test_decode_many_instances_and_ragged_slots(overlap, monkeypatch):
         tf.step(*wl.make_decode_inputs(w, s, DEV))
     assert ctx.poll_status() == 0
     ctx.close()
+
+
+@pytest.mark.parametrize("pinned", [True, False])
+def test_host_buffer_entry_matches_device_entry(pinned):
+    """less_decode_step_host with pinned (read / written in place by the kernel) and pageable
+    (staged and copied) host tensors gives bit-identical outputs and state to less_decode_step."""
+    w = small(54, steps=5, weight_std=0.1)
+    ctx_d, W = _setup(w)
+    ctx_h, _ = _setup(w)
+    for ctx in (ctx_d, ctx_h):
+        _prefill_all(ctx, w, with_out=False)
+    for s in range(w.steps):
+        q, k, v = wl.make_decode_inputs(w, s, DEV)
+        ref = ctx_d.decode_step(q, k, v).cpu()
+        hq, hk, hv = (t.cpu() for t in (q, k, v))
+        hout = torch.full(ref.shape, float("nan"), dtype=torch.float32)
+        if pinned:
+            hq, hk, hv, hout = (t.pin_memory() for t in (hq, hk, hv, hout))
+        ctx_h.decode_step_host(hq, hk, hv, hout)
+        assert torch.equal(hout, ref)
+    inst = list(range(w.instances))
+    for a, b in zip(ctx_d.export_state(inst), ctx_h.export_state(inst)):
+        for key in ("pos", "acc", "K", "V", "psi", "H", "z"):
+            assert np.array_equal(a[key], b[key]), key
+    assert ctx_h.poll_status() == 0
+    ctx_d.close(); ctx_h.close()
