@@ -30,7 +30,7 @@ UNIT = "head-tokens/s"
 FALLBACK_HBM_GBS = 6650.0
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures
-# summarised under profiles/ (None until a capture of that kernel/workload exists)
+# summarised under profiles/ (None where no capture of that kernel and workload exists)
 NCU_TRAFFIC_BYTES = {
     (2, "feature_map"): 285.93e6 + 5.82e6,   # profiles/decode_step_cfg2.md
     (2, "decode"): 113.87e6 + 3.10e6,
@@ -65,7 +65,7 @@ def peaks():
 
 
 # --------------------------------------------------------------------------- #
-# algorithmic bytes per launch (the figures the design doc derives)
+# algorithmic bytes per launch
 # --------------------------------------------------------------------------- #
 def feature_map_bytes(w, no_state=False):
     if no_state:

@@ -73,12 +73,14 @@ enum {
   LESS_POLICY_LAMBDA = 4u
 };
 
+#define LESS_MAX_SLOTS 32768
+
 typedef struct less_config {
   int32_t batch, layers, heads;
   int32_t head_dim;           /* D, must be 128 */
   int32_t rank;               /* R: 8 or 16 (Section 4: R = 8 by default) */
   int32_t hidden;             /* R' = 512 (Section 3.2) */
-  int32_t heavy, recent;      /* slots per instance: heavy >= 0, recent >= 1 */
+  int32_t heavy, recent;      /* slots per instance: heavy >= 0, recent >= 1, heavy + recent <= LESS_MAX_SLOTS */
   int32_t max_prompt;         /* longest prompt less_prefill will be given (>= 0) */
   int32_t max_prefill_layers; /* layers scored together in less_prefill (>= 1): sizes the workspace */
   uint32_t flags;
@@ -115,7 +117,8 @@ int less_create(const less_config* cfg, const less_weights* weights, void* arena
  *      largest (acc, position) keys; if prompt_len <= heavy + recent keep all;
  *   4. kept rows go to slots in ascending position; every other row is
  *      absorbed: H = sum psi(k_j)^T v_j, z = sum psi(k_j) (Eq. 4, Eq. 5 over D_1).
- * Q, K, V: device fp16 [B, layer_count, H, prompt_len, D] contiguous.
+ * Q, K, V: device fp16 [B, layer_count, H, prompt_len, D] contiguous, fewer than
+ * 2^31 rows (B * layer_count * H * prompt_len) per call, else LESS_ERR_PROMPT_TOO_LONG.
  * attn_out: device fp32, same shape, or NULL when the caller does not need the
  * prompt's attention output.
  * Every call of one generation must pass the same prompt_len; the first decode

@@ -21,8 +21,8 @@ Paper passages followed:
   * Section 4       Lambda-masking as the sparse policy: the first tokens plus the most recent ones
 
 Readings where the paper is silent (none of them is fixed by a printed number,
-so they are "parity unpinned" by the paper and fixed by this build's design
-notes): exact erf GELU without biases; the learnable psi scalars sit after each
+so they are "parity unpinned" by the paper and fixed by the design notes that
+come with this code): exact erf GELU without biases; the learnable psi scalars sit after each
 GELU of psi; the accumulated probabilities use Eq. 3's full denominator (flag
 for the sparse-only one); the new token's own probability seeds its score and
 the diagonal counts in the prompt column sums; "recent" = the `recent` highest

@@ -20,7 +20,7 @@ bool valid_config(const less_config* c) {
   if (c->rank != 8 && c->rank != 16) return false;
   if (c->hidden < 64 || c->hidden > 1024 || (c->hidden & (c->hidden - 1))) return false;
   if (c->heavy < 0 || c->recent < 1) return false;
-  if ((int64_t)c->heavy + c->recent > 65536) return false;
+  if ((int64_t)c->heavy + c->recent > LESS_MAX_SLOTS) return false;   // the decode kernel keeps one score per slot in shared memory
   if (c->max_prompt < 0 || c->max_prompt > (1 << 20)) return false;
   if (c->max_prefill_layers < 1 || c->max_prefill_layers > c->layers) return false;
   if ((int64_t)c->batch * c->heads * c->max_prefill_layers > 65535) return false;   // grid.y of the prompt kernels
@@ -202,6 +202,8 @@ int less_prefill(less_ctx* c, int32_t layer_begin, int32_t layer_count, int32_t 
   if (prompt_len < 0) return LESS_ERR_INVALID_CONFIG;
   if (prompt_len > c->cfg.max_prompt) return LESS_ERR_PROMPT_TOO_LONG;
   if (prompt_len > 0) {
+    // the tiled loads address prompt rows with 32-bit coordinates
+    if ((int64_t)c->d.B * layer_count * c->d.Hd * prompt_len > 0x7fffffffLL) return LESS_ERR_PROMPT_TOO_LONG;
     if (!Q || !K || !V) return LESS_ERR_NULL_POINTER;
     if (misaligned(Q) || misaligned(K) || misaligned(V) || misaligned(attn_out))
       return LESS_ERR_MISALIGNED;

@@ -43,8 +43,10 @@ def test_config_validation(B):
     assert good > 0 and good % 256 == 0
     assert B.less_state_record_bytes(cfg()) == 16 + 16 * 8 + 2 * 16 * 128 * 2 + 16 * 8 * 4 + 8 * 128 * 4 + 8 * 4
     for bad in (dict(head_dim=64), dict(rank=4), dict(recent=0), dict(heavy=-1), dict(hidden=500),
-                dict(batch=0), dict(max_prefill_layers=3), dict(flags=64), dict(max_prompt=-1)):
+                dict(batch=0), dict(max_prefill_layers=3), dict(flags=64), dict(max_prompt=-1),
+                dict(heavy=32000, recent=769)):        # more than LESS_MAX_SLOTS = 32768
         assert B.less_arena_bytes(cfg(**bad)) == 0, bad
+    assert B.less_arena_bytes(cfg(heavy=32000, recent=768)) > good
     # arena grows with slots and with the prefill workspace
     assert B.less_arena_bytes(cfg(heavy=80)) > good
     assert B.less_arena_bytes(cfg(max_prompt=4096)) > good

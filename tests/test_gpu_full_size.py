@@ -156,3 +156,20 @@ def test_cfg5_prefill_compression_one_layer_sampled_instance():
         assert np.isfinite(rec["H"]).all() and rec["z"].min() >= 0
     ctx.close()
     torch.cuda.empty_cache()
+
+
+def test_maximum_slot_count_one_instance():
+    """LESS_MAX_SLOTS = 32 768 slots in one instance: the decode kernel's largest shared-memory
+    footprint and longest slot loops, with a prompt just longer than the cache so that the
+    prompt selection and every decode step evict."""
+    w = wl.Workload(50, 1, 1, 2, 128, 33000, 3, 16384, 16384, 8, heavy_rule="bernoulli", heavy_param=0.01)
+    ctx, W = _ctx(w, 1)
+    Q, K, V = wl.make_prompt(w, 0, 1, DEV)
+    ctx.prefill(Q, K, V, 0)
+    inst = [1]
+    print("max slots prompt", _check_prompt(ctx, w, W, inst))
+    tf = _decode_steps(ctx, w, W, inst, w.steps)
+    assert tf.evictions == w.steps
+    print("max slots decode", tf.worst)
+    ctx.close()
+    torch.cuda.empty_cache()
