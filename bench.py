@@ -34,6 +34,9 @@ FALLBACK_HBM_GBS = 6650.0
 NCU_TRAFFIC_BYTES = {
     (2, "feature_map"): 285.93e6 + 5.82e6,   # profiles/decode_step_cfg2.md
     (2, "decode"): 113.87e6 + 3.10e6,
+    # cfg3 captured at batch 16 (a quarter of the instances; both kernels' traffic is per instance or
+    # per head, so the decode kernel's scales by 4 and the feature maps' weights do not)
+    (3, "decode"): 4 * (1.824e9 + 50.2e6),
 }
 
 

@@ -10,10 +10,10 @@
 // GEMM1 is computed transposed, hidden units on the accumulator's 128 lanes and
 // tokens on its columns:
 //     D1^T[128 hidden x n tokens] = W1[:, chunk]^T (A, M-major, as it lies in HBM)
-//                                   * X^T           (B, K-major, n = tokens padded to 16..128)
+//                                   * X^T           (B, K-major, n = tokens padded to 16, 32 or 64)
 // so the GELU work of the epilogue grows with the number of tokens, not with the
 // 128-row tile, and a batch of one costs one GELU per thread and chunk.
-// Epilogue warps (two per lane quadrant) read D1^T from tensor memory, apply
+// Epilogue warps (four per lane quadrant) read D1^T from tensor memory, apply
 // gelu, split the result into fp16 hi + lo (one fp16 rounding of the hidden
 // layer would cost ~2e-3 on psi) and store it, tokens contiguous, as the M-major
 // A operand of
@@ -29,7 +29,7 @@ namespace less {
 
 constexpr int FT_EPI_WARPS = 8;
 constexpr int FT_EPI_THREADS = FT_EPI_WARPS * 32;
-constexpr int FT_THREADS = 64 + FT_EPI_THREADS;   // warp 0 TMA, warp 1 MMA, warps 2..9 epilogue
+constexpr int FT_THREADS = 64 + FT_EPI_THREADS;   // small-batch kernel: warp 0 TMA, warp 1 MMA, warps 2..9 epilogue
 // The larger-batch kernel runs four epilogue warps per lane quadrant: its GELU chains are long and
 // dependent, and with two warps per scheduler the issue slots sat idle (4700 cycles per chunk
 // measured for 32 GELUs per thread).
