@@ -54,6 +54,8 @@ def parse_args():
     ap.add_argument("--no-state", action="store_true", help="context run: sparse policy alone (Baseline+)")
     ap.add_argument("--lambda-masking", action="store_true",
                     help="context run: Lambda-masking as the sparse policy (first 4 tokens + window, same slot count)")
+    ap.add_argument("--attn-out", action="store_true",
+                    help="prompt compression: also produce the prompt's attention output (optional in less_prefill)")
     ap.add_argument("--batch", type=int, default=0,
                     help="override the workload's batch (smaller captures for ncu; named in config.workload)")
     return ap.parse_args()
@@ -429,7 +431,7 @@ def prefill_flops(w):
     inst = w.batch * w.heads
     S, D, Rp, R = w.prompt, w.head_dim, w.hidden, w.rank
     causal = S * (S + 1) // 2
-    return {"rowstat": inst * causal * 2 * D, "colsum": inst * causal * 2 * D,
+    return {"rowstat": inst * causal * 2 * D, "colsum": inst * causal * 2 * D, "attn_out": inst * causal * 4 * D,
             "psi": inst * S * 2 * (D * Rp + Rp * R + R * R), "build": inst * S * 2 * R * D}
 
 
@@ -454,11 +456,12 @@ def run_prefill(args):
     Wt = wl.make_weights(w, dev)
     ctx = binding.from_workload(w, Wt, dev, max_prefill_layers=1)
     Q, Kp, V = wl.make_prompt(w, 0, 1, dev)          # one layer of inputs, reused for every layer index
+    attn = torch.empty(Q.shape, dtype=torch.float32, device=dev) if args.attn_out else None
     stream = torch.cuda.current_stream()
     step_no = [0]
 
     def one_step():
-        ctx.prefill(Q, Kp, V, step_no[0] % w.layers)
+        ctx.prefill(Q, Kp, V, step_no[0] % w.layers, attn_out=attn)
         step_no[0] += 1
 
     def barrier():

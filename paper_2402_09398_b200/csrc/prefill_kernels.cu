@@ -427,7 +427,10 @@ int launch_prefill_group(less_ctx* c, int layer0, int nl, int lj0, int layer_cou
         colsum_kernel<<<dim3(tiles, G), PF_TILE, 0, s>>>(p);
       }
     }
-    if (attn_out) {
+    if (attn_out && c->score_path == 1 && score_tc_supported()) {
+      const int rc = launch_attn_out_tc(c, p, G, s);
+      if (rc != LESS_OK) return rc;
+    } else if (attn_out) {
       LaunchScope scope(c, LESS_KERNEL_ATTN_OUT, s);
       attn_out_kernel<<<dim3((S + AO_ROWS - 1) / AO_ROWS, G), PF_TILE, 0, s>>>(p);
     }
