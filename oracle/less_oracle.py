@@ -18,7 +18,8 @@ Paper passages followed:
   * Section 2.1 / Section 4  H2O policy: accumulated attention probabilities,
                     equal heavy/recent split, even-floored token counts (Table 1)
   * Section 3.1     the prompt phase is regular attention (H_0 = 0, z_0 = 0)
-  * Section 4       Lambda-masking as the sparse policy: the first tokens plus the most recent ones
+  * Section 4       Lambda-masking as the sparse policy: the first tokens plus the most recent ones;
+                    TOVA is named there without a definition (the rule of the cited work is used)
 
 Readings where the paper is silent (none of them is fixed by a printed number,
 so they are "parity unpinned" by the paper and fixed by the design notes that
@@ -97,11 +98,16 @@ class LessInstance:
                  score_norm: str = "less", use_state: bool = True, policy: str = "h2o"):
         if recent < 1 or heavy < 0:
             raise ValueError("need recent >= 1 and heavy >= 0")
-        if policy not in ("h2o", "lambda"):
-            raise ValueError("policy is 'h2o' or 'lambda'")
+        if policy not in ("h2o", "lambda", "tova"):
+            raise ValueError("policy is 'h2o', 'lambda' or 'tova'")
         # 'lambda' = Lambda-masking (Section 4: "the cache consists of the first 4 and most recent
         # tokens"): `heavy` counts the first tokens that are always kept, `recent` the window;
         # accumulated scores play no role in it.
+        # 'tova' = the third policy Section 4 names.  The paper gives no definition of it; this is
+        # the published rule of the work it cites, per head: whenever the cache overflows, the
+        # entry with the lowest attention probability OF THE CURRENT QUERY leaves, the newest one
+        # included and no window protected; `heavy + recent` only sets the slot count.  Under the
+        # one-shot reading of the prompt phase the current query at its end is the last prompt token.
         self.policy = policy
         if score_norm not in ("less", "sparse"):
             raise ValueError("score_norm is 'less' or 'sparse'")
@@ -162,16 +168,23 @@ class LessInstance:
             P = e / e.sum(axis=1, keepdims=True)              # softmax rows
             out[r0:r1] = P @ V[:r1]
             acc[:r1] += P.sum(axis=0)                         # H2O: column sums, diagonal included
+            if r1 == S:
+                last_row = P[-1].copy()                       # TOVA: the last query's probabilities
         self.t = S
         pos = np.arange(S, dtype=np.int64)
         if self.policy == "lambda":
             acc = np.zeros(S)                                 # the policy keeps no scores
+        elif self.policy == "tova":
+            acc = last_row                                    # attention of the last prompt query
         if S <= self.N:
             keep = pos
             evict = pos[:0]
         else:
             if self.policy == "lambda":
                 evict = pos[self.heavy: S - self.recent]      # everything between the first tokens and the window
+            elif self.policy == "tova":
+                order = np.lexsort((pos, acc))                # key (p, pos) ascending, nothing protected
+                evict = np.sort(pos[order[: S - self.N]])
             else:
                 cand = pos[: S - self.recent]                 # recent window is protected
                 order = np.lexsort((cand, acc[cand]))         # key (acc, pos) ascending
@@ -209,18 +222,24 @@ class LessInstance:
         out = num / den
         # H2O: accumulate this step's attention probabilities
         p = e / (den if self.score_norm == "less" else den_sparse)
-        acc = np.concatenate([self.acc + p[:-1], p[-1:]])
+        if self.policy == "tova":
+            acc = p.copy()                                     # TOVA scores = this query's probabilities
+        else:
+            acc = np.concatenate([self.acc + p[:-1], p[-1:]])
         pos = np.concatenate([self.pos, np.array([t], dtype=np.int64)])
         evicted_pos, gap, dH, dz = -1, None, None, None
         if pos.size > self.N:
             if self.policy == "lambda":
                 cand = np.nonzero(pos >= self.heavy)[0]       # never one of the first tokens
                 order = np.argsort(pos[cand])                 # the oldest of the others leaves the window
+            elif self.policy == "tova":
+                cand = np.arange(pos.size)                    # every entry, the new pair included
+                order = np.lexsort((pos, acc))
             else:
                 cand = np.nonzero(pos <= t - self.recent)[0]
                 order = np.lexsort((pos[cand], acc[cand]))    # (acc, pos) ascending
             vic = int(cand[order[0]])
-            if cand.size > 1 and self.policy == "h2o":
+            if cand.size > 1 and self.policy != "lambda":
                 a0, a1 = acc[cand[order[0]]], acc[cand[order[1]]]
                 gap = abs(a1 - a0) / max(abs(a0), abs(a1), 1e-300)
             evicted_pos = int(pos[vic])

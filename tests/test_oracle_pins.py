@@ -494,3 +494,64 @@ def test_lambda_masking_short_context_and_budget_that_holds_everything():
     b, _, sb, _, _ = run_instance(w, heavy=30, recent=30, policy="h2o")
     for x, y in zip(sa, sb):                                         # nothing evicted: the policy cannot matter
         assert np.array_equal(x["out"], y["out"]) and x["evicted_pos"] == -1
+
+
+# --------------------------------------------------------------------------- #
+# TOVA as the sparse policy (named in Section 4; the rule is the cited work's: the entry with the
+# lowest attention probability of the current query leaves, the newest included)
+# --------------------------------------------------------------------------- #
+@pytest.mark.parametrize("use_state", [True, False])
+def test_tova_against_an_independent_replay(use_state):
+    """A replay kept as a plain python set of positions, with torch softmax for the probabilities,
+    must choose the same victims; the outputs obey Eq. 3 with torch-computed Eq. 6 sums."""
+    w = tiny(cfg_id=99, S=26, T=16, heavy=3, recent=4, D=16, R=4)
+    N = w.heavy + w.recent
+    inst, _, steps, (Qp, Kh, Vh), wts = run_instance(w, use_state=use_state, policy="tova")
+    Kt, Vt = torch.tensor(Kh), torch.tensor(Vh)
+    # prompt: the last prompt query's causal softmax row ranks the prompt tokens
+    p_last = torch.softmax(Kt[: w.prompt] @ torch.tensor(Qp[-1]) / math.sqrt(w.head_dim), dim=0).numpy()
+    order = sorted(range(w.prompt), key=lambda j: (p_last[j], j))
+    kept = set(range(w.prompt)) - set(order[: w.prompt - N])
+    gone = set(order[: w.prompt - N])
+    new_token_evicted = 0
+    for i, r in enumerate(steps):
+        t = w.prompt + i
+        assert sorted(kept) == list(r["kept_before"])
+        idx = sorted(kept) + [t]
+        e = torch.exp(Kt[idx] @ torch.tensor(r["q"]) / math.sqrt(w.head_dim))
+        if use_state and gone:
+            g = sorted(gone)
+            psi = torch_psi(Kh[g], *wts[2:])
+            phi = torch_phi(r["q"][None], *wts[:2])[0]
+            num, den = phi @ (psi.T @ Vt[g]) + e @ Vt[idx], phi @ psi.sum(0) + e.sum()
+        else:
+            num, den = e @ Vt[idx], e.sum()
+        assert np.allclose(r["out"], (num / den).numpy(), rtol=1e-10, atol=1e-13)
+        prob = (e / den).numpy()
+        victim = min(zip(prob, idx))[1]                     # lowest probability, then lowest position
+        assert r["evicted_pos"] == victim
+        new_token_evicted += victim == t
+        kept = (kept | {t}) - {victim}
+        gone.add(victim)
+    assert sorted(kept) == list(inst.pos) and sorted(gone) == sorted(inst.evicted)
+    assert len(kept) == N
+    if not use_state:
+        assert (inst.H == 0).all() and (inst.z == 0).all()
+
+
+def test_tova_can_evict_the_new_token_itself():
+    """A new key that the query points away from gets the lowest probability of its own step:
+    it never enters the cache and is absorbed into H, z at once."""
+    D, R = 8, 2
+    phi = lambda x: np.abs(x[:, :R])
+    psi = lambda x: np.abs(x[:, :R]) + 1.0
+    inst = lo.LessInstance(D, R, 2, 2, phi, psi, policy="tova")
+    K = np.eye(D)[:4] * 3.0
+    V = np.arange(4 * D, dtype=np.float64).reshape(4, D)
+    inst.prefill(np.ones((4, D)), K, V)
+    assert list(inst.pos) == [0, 1, 2, 3]
+    q = np.ones(D)
+    k_new, v_new = -5.0 * np.ones(D), np.full(D, 7.0)
+    r = inst.decode(q, k_new, v_new)
+    assert r["evicted_pos"] == 4 and list(inst.pos) == [0, 1, 2, 3]
+    assert np.allclose(inst.H, np.outer(psi(k_new[None])[0], v_new)) and np.allclose(inst.z, psi(k_new[None])[0])
