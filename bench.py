@@ -54,6 +54,8 @@ def parse_args():
     ap.add_argument("--no-state", action="store_true", help="context run: sparse policy alone (Baseline+)")
     ap.add_argument("--lambda-masking", action="store_true",
                     help="context run: Lambda-masking as the sparse policy (first 4 tokens + window, same slot count)")
+    ap.add_argument("--tova", action="store_true",
+                    help="context run: TOVA as the sparse policy (same slot count)")
     ap.add_argument("--attn-out", action="store_true",
                     help="prompt compression: also produce the prompt's attention output (optional in less_prefill)")
     ap.add_argument("--batch", type=int, default=0,
@@ -250,6 +252,8 @@ def workload_config(w, args):
          if w.cfg_id != 1 else "L2 flushed by a 256 MB write between steps is NOT done: cfg1 is launch-bound"}
     if getattr(args, "full_cache", False):
         c["variant"] = "full cache (no eviction)"
+    if getattr(args, "tova", False):
+        c["variant"] = "TOVA policy (lowest probability of the current query leaves)"
     if getattr(args, "lambda_masking", False):
         c["variant"] = "Lambda-masking policy (first 4 tokens + recent window)"
     if getattr(args, "no_state", False):
@@ -291,6 +295,8 @@ def run_b200(args):
     if args.lambda_masking:
         flags |= binding.LESS_POLICY_LAMBDA
         heavy, recent = 4, heavy + recent - 4
+    if args.tova:
+        flags |= binding.LESS_POLICY_TOVA
     w_run = w.with_(heavy=heavy, recent=recent)
 
     # replicas: every rank runs the whole workload on its own GPU, no collective in the path

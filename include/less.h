@@ -70,7 +70,16 @@ enum {
    * keeps positions [0, heavy) and the last `recent`, a decode step evicts the
    * lowest position >= heavy.  Accumulated scores are not used (prompt scoring
    * is skipped unless attn_out is asked for); evicted pairs go to H, z as usual. */
-  LESS_POLICY_LAMBDA = 4u
+  LESS_POLICY_LAMBDA = 4u,
+  /* TOVA as the sparse policy (named in Section 4; the paper does not define
+   * it, the rule is the cited work's, applied per head): when the slots
+   * overflow, the entry with the lowest attention probability of the CURRENT
+   * query is evicted, ties to the lowest position; the new pair competes too
+   * (if it loses it is absorbed into H, z and never cached) and no window is
+   * protected.  `heavy + recent` only sets the slot count.  The prompt is
+   * ranked once, by its last query's attention row.  Not together with
+   * LESS_POLICY_LAMBDA. */
+  LESS_POLICY_TOVA = 8u
 };
 
 #define LESS_MAX_SLOTS 32768

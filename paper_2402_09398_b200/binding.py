@@ -20,6 +20,7 @@ LESS_OK = 0
 LESS_SCORE_NORM_SPARSE = 1
 LESS_NO_STATE = 2
 LESS_POLICY_LAMBDA = 4
+LESS_POLICY_TOVA = 8
 
 EXPORTED = [
     "less_arena_bytes", "less_create", "less_prefill", "less_decode_step", "less_position",

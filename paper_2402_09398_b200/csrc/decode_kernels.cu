@@ -244,13 +244,19 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_kernel(DecParams p) {
   float* accb = p.a.acc + inst * (size_t)p.Np;
   const bool full = (n == N);
   const bool lambda_policy = (p.flags & LESS_POLICY_LAMBDA) != 0;
+  const bool tova_policy = (p.flags & LESS_POLICY_TOVA) != 0;
   unsigned long long best = ~0ull;
   for (int i = tid; i < n; i += DEC_THREADS) {
-    const float a = accb[i] + s_sc[i] * inv;
+    // TOVA scores an entry by this query's probability alone; H2O accumulates
+    const float a = tova_policy ? s_sc[i] * inv : accb[i] + s_sc[i] * inv;
     accb[i] = a;
     if (full) {
       const int ps = posb[i];
-      if (lambda_policy) {                           // Lambda-masking: the oldest position past the first tokens
+      if (tova_policy) {                             // TOVA: every entry competes, nothing is protected
+        const unsigned long long key =
+            ((unsigned long long)__float_as_uint(a) << 32) | (unsigned int)ps;
+        best = key < best ? key : best;
+      } else if (lambda_policy) {                           // Lambda-masking: the oldest position past the first tokens
         if (ps >= p.heavy) best = (unsigned long long)(unsigned int)ps < best ? (unsigned int)ps : best;
       } else if (ps <= p.t - p.recent) {             // H2O: lowest (accumulated score, position) outside the window
         const unsigned long long key =
@@ -273,6 +279,23 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_kernel(DecParams p) {
     best = s_key[0];
 #pragma unroll
     for (int w = 1; w < DEC_THREADS / 32; ++w) best = s_key[w] < best ? s_key[w] : best;
+    if (tova_policy) {
+      // the new pair competes too; if its own probability is the lowest it never enters the
+      // cache: it is absorbed into H, z at once and every slot stays as it is
+      const unsigned long long key_new =
+          ((unsigned long long)__float_as_uint(p_new) << 32) | (unsigned int)p.t;
+      if (key_new < best) {                          // uniform over the CTA
+        if (tid == 0 && p.evicted_pos) p.evicted_pos[inst] = p.t;
+        if (use_state) {
+          const float vv = __half2float(p.v[inst * kHeadDim + d]);
+          const float* psn = p.a.psi_k + inst * R;
+#pragma unroll
+          for (int r = 0; r < R; ++r) Hb[r * kHeadDim + d] = fmaf(psn[r], vv, hcol[r]);
+          if (tid < R) zb[tid] += psn[tid];
+        }
+        return;
+      }
+    }
     const int vpos = (int)(unsigned int)(best & 0xffffffffull);
     for (int i = tid; i < n; i += DEC_THREADS)
       if (posb[i] == vpos && best != ~0ull) s_vic = i;     // positions are unique

@@ -24,7 +24,8 @@ bool valid_config(const less_config* c) {
   if (c->max_prompt < 0 || c->max_prompt > (1 << 20)) return false;
   if (c->max_prefill_layers < 1 || c->max_prefill_layers > c->layers) return false;
   if ((int64_t)c->batch * c->heads * c->max_prefill_layers > 65535) return false;   // grid.y of the prompt kernels
-  if (c->flags & ~(uint32_t)(LESS_SCORE_NORM_SPARSE | LESS_NO_STATE | LESS_POLICY_LAMBDA)) return false;
+  if (c->flags & ~(uint32_t)(LESS_SCORE_NORM_SPARSE | LESS_NO_STATE | LESS_POLICY_LAMBDA | LESS_POLICY_TOVA)) return false;
+  if ((c->flags & LESS_POLICY_LAMBDA) && (c->flags & LESS_POLICY_TOVA)) return false;
   int64_t inst = (int64_t)c->batch * c->layers * c->heads;
   if (inst > (1 << 24)) return false;
   return true;

@@ -164,6 +164,47 @@ __global__ void __launch_bounds__(PF_TILE) attn_out_kernel(PfParams p) {
     if (i0 + r < p.S) p.attn_out[(im.in_row0 + i0 + r) * kHeadDim + tid] = o[r];
 }
 
+// ---- TOVA: the last prompt query's attention probabilities ------------------- //
+// p_j = softmax_j( q_{S-1} . k_j / sqrt(D) ) over the whole prompt, into ws_acc.  One CTA per
+// instance: scores, block maximum, exponentials and their block sum, normalisation in place.
+constexpr int LR_THREADS = 1024;
+__global__ void __launch_bounds__(LR_THREADS) lastrow_kernel(PfParams p) {
+  __shared__ float qs[kHeadDim];
+  __shared__ float red[LR_THREADS / 32];
+  const int g = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const InstMap im = map_instance(p, g);
+  float* pr = p.a.ws_acc + (size_t)g * p.Sp;
+  if (tid < kHeadDim) qs[tid] = __half2float(p.Q[(im.in_row0 + p.S - 1) * kHeadDim + tid]);
+  __syncthreads();
+  float m = -INFINITY;
+  for (int j = tid; j < p.S; j += LR_THREADS) {
+    const float s = dot128(qs, p.K + (im.in_row0 + j) * kHeadDim) * kScale;
+    pr[j] = s;
+    m = fmaxf(m, s);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+  if (lane == 0) red[warp] = m;
+  __syncthreads();
+  m = red[0];
+  for (int w = 1; w < LR_THREADS / 32; ++w) m = fmaxf(m, red[w]);
+  __syncthreads();
+  float l = 0.f;
+  for (int j = tid; j < p.S; j += LR_THREADS) {
+    const float e = __expf(pr[j] - m);
+    pr[j] = e;
+    l += e;
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
+  if (lane == 0) red[warp] = l;
+  __syncthreads();
+  l = 0.f;
+  for (int w = 0; w < LR_THREADS / 32; ++w) l += red[w];      // fixed order
+  const float inv = 1.0f / l;
+  for (int j = tid; j < p.S; j += LR_THREADS) pr[j] *= inv;
+}
+
 // ---- P3: selection --------------------------------------------------------- //
 constexpr int SEL_THREADS = 1024;
 
@@ -220,12 +261,15 @@ __global__ void __launch_bounds__(SEL_THREADS) select_kernel(PfParams p) {
       slot_of[j] = j < p.heavy ? j : (j >= S - p.recent ? p.heavy + j - (S - p.recent) : -1);
     return;
   }
-  const int C = S - p.recent;                    // candidates: positions [0, C)
+  // TOVA protects no window and ranks every position by the last query's probabilities
+  const bool tova = (p.flags & LESS_POLICY_TOVA) != 0;
+  const int heavy = tova ? N : p.heavy;
+  const int C = tova ? S : S - p.recent;         // candidates: positions [0, C)
   unsigned int thr = 0xffffffffu;                // threshold bit pattern (acc >= 0: monotone)
   int need = 0;                                  // how many of the == threshold to keep
-  if (p.heavy > 0) {
+  if (heavy > 0) {
     // radix select: the heavy-th largest accumulated score among the candidates
-    if (tid == 0) { s_prefix = 0; s_need = p.heavy; }
+    if (tid == 0) { s_prefix = 0; s_need = heavy; }
     for (int pass = 0; pass < 4; ++pass) {
       const int shift = 24 - 8 * pass;
       if (tid < 256) hist[tid] = 0;
@@ -267,7 +311,7 @@ __global__ void __launch_bounds__(SEL_THREADS) select_kernel(PfParams p) {
     else {
       const unsigned int b = __float_as_uint(acc[j]);
       if (b == thr) { k = eq_before >= drop_eq; ++eq_before; }
-      else k = p.heavy > 0 && b > thr;
+      else k = heavy > 0 && b > thr;
     }
     kept += k ? 1 : 0;
   }
@@ -286,7 +330,7 @@ __global__ void __launch_bounds__(SEL_THREADS) select_kernel(PfParams p) {
     else {
       const unsigned int b = __float_as_uint(acc[j]);
       if (b == thr) { k = eq_before >= drop_eq; ++eq_before; }
-      else k = p.heavy > 0 && b > thr;
+      else k = heavy > 0 && b > thr;
     }
     slot_of[j] = k ? slot++ : -1;
   }
@@ -410,8 +454,10 @@ int launch_prefill_group(less_ctx* c, int layer0, int nl, int lj0, int layer_cou
     nsplit = (S + split_tokens - 1) / split_tokens;
   }
   p.nsplit = nsplit; p.split_tokens = split_tokens;
-  // Lambda-masking needs no scores; the row statistics are still needed for the prompt's attention output
-  const bool need_scores = !(d.flags & LESS_POLICY_LAMBDA) || attn_out != nullptr;
+  // Lambda-masking needs no scores and TOVA only the last query's row; the row statistics are still
+  // needed for the prompt's attention output
+  const bool h2o = !(d.flags & (LESS_POLICY_LAMBDA | LESS_POLICY_TOVA));
+  const bool need_scores = h2o || attn_out != nullptr;
   if (S > 0 && need_scores) {
     const int tiles = (S + PF_TILE - 1) / PF_TILE;
     if (c->score_path == 1 && score_tc_supported()) {
@@ -434,6 +480,10 @@ int launch_prefill_group(less_ctx* c, int layer0, int nl, int lj0, int layer_cou
       LaunchScope scope(c, LESS_KERNEL_ATTN_OUT, s);
       attn_out_kernel<<<dim3((S + AO_ROWS - 1) / AO_ROWS, G), PF_TILE, 0, s>>>(p);
     }
+  }
+  if (S > 0 && (d.flags & LESS_POLICY_TOVA)) {   // after the column sums, if any ran: both write ws_acc
+    LaunchScope scope(c, LESS_KERNEL_COLSUM, s);
+    lastrow_kernel<<<G, LR_THREADS, 0, s>>>(p);
   }
   {
     LaunchScope scope(c, LESS_KERNEL_SELECT, s);

@@ -44,7 +44,7 @@ def make_oracle(w, W, inst, flags=0, psi_scale=None, heavy=None, recent=None):
     return lo.LessInstance(w.head_dim, w.rank, w.heavy if heavy is None else heavy,
                            w.recent if recent is None else recent, phi_fn, psi_fn,
                            score_norm="sparse" if flags & 1 else "less",
-                           use_state=not (flags & 2), policy="lambda" if flags & 4 else "h2o")
+                           use_state=not (flags & 2), policy="lambda" if flags & 4 else ("tova" if flags & 8 else "h2o"))
 
 
 def check_prefill(ctx, w, W, Q, K, V, instances, attn_out=None, flags=0, psi_scale=None,

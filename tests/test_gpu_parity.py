@@ -39,7 +39,7 @@ def _prefill_all(ctx, w, with_out=True, prompt=None):
 @pytest.mark.parametrize("variant", ["base", "rank16", "boosted", "ragged", "sparse_norm", "no_state",
                                      "scaled", "heavy0", "recent1", "hidden256", "long_prompt",
                                      "cuda_core_scoring", "lambda_masking", "lambda_no_state",
-                                     "tiny_scalars", "huge_psi"])
+                                     "tiny_scalars", "huge_psi", "tova", "tova_no_state"])
 def test_prefill_and_teacher_forced_decode(variant, monkeypatch):
     import harness
     flags, psi_scale = 0, None
@@ -68,6 +68,10 @@ def test_prefill_and_teacher_forced_decode(variant, monkeypatch):
         w, flags = small(58, heavy=4, recent=36, weight_std=0.1), 4
     elif variant == "lambda_no_state":
         w, flags = small(57, heavy=4, recent=21, prompt=211), 4 | 2
+    elif variant == "tova":                 # lowest probability of the current query leaves, the new pair included
+        w, flags = small(53, weight_std=0.1, steps=16), 8
+    elif variant == "tova_no_state":
+        w, flags = small(52, prompt=190, heavy=9, recent=8), 8 | 2
     elif variant == "tiny_scalars":         # the paper initialises psi's learnable scalars to 1e-4
         w = small(56, weight_std=0.1)
         psi_scale = torch.full((w.layers, w.heads, 2), 1e-4)
