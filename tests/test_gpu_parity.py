@@ -352,3 +352,32 @@ def test_host_buffer_entry_matches_device_entry(pinned):
             assert np.array_equal(a[key], b[key]), key
     assert ctx_h.poll_status() == 0
     ctx_d.close(); ctx_h.close()
+
+
+def test_tova_new_token_can_evict_itself():
+    """TOVA: a new key the query points away from has the lowest probability of its own step;
+    it is absorbed into H, z at once and no slot changes (imported state)."""
+    w = small(51, batch=1, layers=1, heads=1, prompt=0, heavy=2, recent=2, weight_std=0.1)
+    ctx, W = _setup(w, flags=8, max_prompt=8)
+    D, R = w.head_dim, w.rank
+    K = np.zeros((4, D), dtype=np.float16)
+    K[np.arange(4), np.arange(4)] = 3.0
+    rec = {"count": 4, "t": 10, "pos": np.array([2, 5, 7, 9], dtype=np.int32),
+           "acc": np.full(4, 0.25, dtype=np.float32), "K": K,
+           "V": np.arange(4 * D, dtype=np.float16).reshape(4, D) / 64,
+           "psi": np.ones((4, R), dtype=np.float32), "H": np.zeros((R, D), dtype=np.float32),
+           "z": np.zeros(R, dtype=np.float32)}
+    ctx.import_state([0], [rec])
+    q = torch.ones(1, 1, 1, D, dtype=torch.float16, device=DEV)
+    k = torch.full((1, 1, 1, D), -5.0, dtype=torch.float16, device=DEV)
+    v = torch.full((1, 1, 1, D), 7.0, dtype=torch.float16, device=DEV)
+    ev = torch.empty(1, dtype=torch.int32, device=DEV)
+    ctx.decode_step(q, k, v, evicted_pos=ev)
+    assert int(ev.item()) == 10                        # the new token's own position
+    post = ctx.export_state([0])[0]
+    assert post["pos"].tolist() == [2, 5, 7, 9] and post["count"] == 4
+    assert np.array_equal(post["K"], K)
+    _, psi_k = ctx.read_feature_maps()
+    assert np.allclose(post["H"], np.outer(psi_k[0], np.full(D, 7.0)), rtol=1e-6)
+    assert np.allclose(post["z"], psi_k[0], rtol=1e-6)
+    ctx.close()
