@@ -21,7 +21,7 @@ namespace less {
 
 constexpr int AO_EPI_WARPS = 8;
 constexpr int AO_EPI_THREADS = AO_EPI_WARPS * 32;
-constexpr int AO_THREADS = 64 + AO_EPI_THREADS;     // warp 0 TMA, warp 1 MMA, warps 2..9 epilogue
+constexpr int AO_THREADS = 64 + AO_EPI_THREADS + 32;   // warp 0 TMA (Q, K), warp 1 MMA, warps 2..9 epilogue, warp 10 TMA (V)
 constexpr int AO_TILE = 128;                        // query rows per CTA and keys per streamed tile
 constexpr int AO_TILE_BYTES = AO_TILE * kHeadDim * 2;
 constexpr int AO_STAGES = 2;
@@ -32,7 +32,10 @@ constexpr float kAoExpScale = 0.12751743074602468f; // log2(e) / sqrt(128)
 
 struct AoShared {
   uint64_t res_full;
-  uint64_t kv_full[AO_STAGES], kv_empty[AO_STAGES];
+  // K and V tiles have rings of their own: a K stage is free again as soon as its scores are
+  // computed, a V stage only after P V, and the next scores must not wait for the latter
+  uint64_t k_full[AO_STAGES], k_empty[AO_STAGES];
+  uint64_t v_full[AO_STAGES], v_empty[AO_STAGES];
   uint64_t s_full[2], s_free[2];
   uint64_t p_full, p_free;
   uint64_t o_full;
@@ -69,8 +72,10 @@ __global__ void __launch_bounds__(AO_THREADS) attn_out_tc_kernel(const __grid_co
   if (tid == 0) {
     mbar_init(&sh->res_full, 1);
     for (int s = 0; s < AO_STAGES; ++s) {
-      mbar_init(&sh->kv_full[s], 1);
-      mbar_init(&sh->kv_empty[s], 1);
+      mbar_init(&sh->k_full[s], 1);
+      mbar_init(&sh->k_empty[s], 1);
+      mbar_init(&sh->v_full[s], 1);
+      mbar_init(&sh->v_empty[s], 1);
     }
     for (int s = 0; s < 2; ++s) {
       mbar_init(&sh->s_full[s], 1);
@@ -109,15 +114,28 @@ __global__ void __launch_bounds__(AO_THREADS) attn_out_tc_kernel(const __grid_co
       bulk_g2s(qx, p.a.ws_bx + (size_t)g * p.Sbx + i0, AO_QX_BYTES, &sh->res_full);
       uint32_t s = 0, ph = 0;
       for (int t = 0; t < ntile; ++t) {
-        wait_or_give_up(&sh->kv_empty[s], ph ^ 1, abortp, status, 100);
+        wait_or_give_up(&sh->k_empty[s], ph ^ 1, abortp, status, 100);
         if (*abortp) break;
         const int krow = (int)(im.in_row0 + (size_t)t * AO_TILE);
         unsigned char* st = ring + s * AO_STAGE_BYTES;
-        mbar_expect_tx(&sh->kv_full[s], AO_STAGE_BYTES);
-        tma_load_2d(st, &tm_k, 0, krow, &sh->kv_full[s]);
-        tma_load_2d(st + AO_TILE_BYTES / 2, &tm_k, 64, krow, &sh->kv_full[s]);
-        tma_load_2d(st + AO_TILE_BYTES, &tm_v, 0, krow, &sh->kv_full[s]);
-        tma_load_2d(st + AO_TILE_BYTES + AO_TILE_BYTES / 2, &tm_v, 64, krow, &sh->kv_full[s]);
+        mbar_expect_tx(&sh->k_full[s], AO_TILE_BYTES);
+        tma_load_2d(st, &tm_k, 0, krow, &sh->k_full[s]);
+        tma_load_2d(st + AO_TILE_BYTES / 2, &tm_k, 64, krow, &sh->k_full[s]);
+        if (++s == AO_STAGES) { s = 0; ph ^= 1; }
+      }
+    }
+  } else if (warp == 10) {
+    // ---------------- TMA producer of the V tiles ----------------
+    if (lane == 0) {
+      uint32_t s = 0, ph = 0;
+      for (int t = 0; t < ntile; ++t) {
+        wait_or_give_up(&sh->v_empty[s], ph ^ 1, abortp, status, 108);
+        if (*abortp) break;
+        const int krow = (int)(im.in_row0 + (size_t)t * AO_TILE);
+        unsigned char* st = ring + s * AO_STAGE_BYTES + AO_TILE_BYTES;
+        mbar_expect_tx(&sh->v_full[s], AO_TILE_BYTES);
+        tma_load_2d(st, &tm_v, 0, krow, &sh->v_full[s]);
+        tma_load_2d(st + AO_TILE_BYTES / 2, &tm_v, 64, krow, &sh->v_full[s]);
         if (++s == AO_STAGES) { s = 0; ph ^= 1; }
       }
     }
@@ -136,7 +154,7 @@ __global__ void __launch_bounds__(AO_THREADS) attn_out_tc_kernel(const __grid_co
       uint32_t s1 = 0, ph1 = 0, b1 = 0, bph1 = 0;      // S stream: stage, S buffer and their phases
       int issued = 0;
       auto issue_s = [&]() {
-        wait_or_give_up(&sh->kv_full[s1], ph1, abortp, status, 102);
+        wait_or_give_up(&sh->k_full[s1], ph1, abortp, status, 102);
         wait_or_give_up(&sh->s_free[b1], bph1 ^ 1, abortp, status, 103);
         if (*abortp) return;
         tc_fence_after_sync();
@@ -146,15 +164,17 @@ __global__ void __launch_bounds__(AO_THREADS) attn_out_tc_kernel(const __grid_co
           mma_f16_ss(tmem + b1 * AO_TILE, ad_q + (uint64_t)((ks >> 2) * (AO_TILE_BYTES >> 5) + (ks & 3) * 2),
                      bd0 + (uint64_t)((ks >> 2) * (AO_TILE_BYTES >> 5) + (ks & 3) * 2), idesc_s, ks ? 1u : 0u);
         mma_f16_ss(tmem + b1 * AO_TILE, ad_qx, bd_ones, idesc_s, 1u);
+        mma_commit(&sh->k_empty[s1]);
         mma_commit(&sh->s_full[b1]);
         if (++s1 == AO_STAGES) { s1 = 0; ph1 ^= 1; }
         if (b1 ^= 1, b1 == 0) bph1 ^= 1;
         ++issued;
       };
       issue_s();
-      uint32_t s2 = 0, pph = 0;
+      uint32_t s2 = 0, vph = 0, pph = 0;
       for (int t = 0; t < ntile && !*abortp; ++t) {
         if (issued < ntile) issue_s();                 // the next tile's scores run ahead of this tile's P V
+        wait_or_give_up(&sh->v_full[s2], vph, abortp, status, 109);
         wait_or_give_up(&sh->p_full, pph, abortp, status, 104);
         if (*abortp) break;
         pph ^= 1;
@@ -165,8 +185,8 @@ __global__ void __launch_bounds__(AO_THREADS) attn_out_tc_kernel(const __grid_co
           mma_f16_ss(tmem + ocol, ad_p + (uint64_t)((ks >> 2) * (AO_TILE_BYTES >> 5) + (ks & 3) * 2),
                      bv0 + (uint64_t)(ks * (2048 >> 4)), idesc_o, (t | ks) ? 1u : 0u);
         mma_commit(&sh->p_free);
-        mma_commit(&sh->kv_empty[s2]);
-        if (++s2 == AO_STAGES) s2 = 0;
+        mma_commit(&sh->v_empty[s2]);
+        if (++s2 == AO_STAGES) { s2 = 0; vph ^= 1; }
       }
       mma_commit(&sh->o_full);
     }
