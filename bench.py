@@ -389,6 +389,10 @@ def run_b200(args):
               "decode": decode_bytes(w, n_live, evicting, args.no_state)}
         kt = {k: (prof[k][0] / prof[k][1] if prof[k][1] else 0.0) for k in ("feature_map", "decode")}
         dominant = max(kt, key=lambda k: kt[k])
+        kernel_names = {"feature_map": ("feature_tc_small_kernel" if w.batch <= 8 else "feature_tc_kernel")
+                        + f"<{w.rank}" + (f", {1 if w.batch <= 1 else 2 if w.batch <= 2 else 4 if w.batch <= 4 else 8}>"
+                                          if w.batch <= 8 else ">"),
+                        "decode": f"decode_kernel<{w.rank}>"}
         ach = kb[dominant] / (kt[dominant] * 1e-3) / 1e9 if kt[dominant] > 0 else 0.0
         step_bytes = kb["feature_map"] + kb["decode"]
         kv_state_bytes = w.instances * (n_live * (4 * w.head_dim + 8) + (0 if args.no_state else 2 * w.rank * w.head_dim * 4))
@@ -402,7 +406,7 @@ def run_b200(args):
                     "h2d_bytes_per_step": 3 * w.instances * w.head_dim * 2,
                     "d2h_bytes_per_step": w.instances * w.head_dim * 4},
             "gpu_launches": int(launches),
-            "roofline": {"bound": "hbm", "kernel": dominant + "_kernel", "achieved": ach, "peak": peak,
+            "roofline": {"bound": "hbm", "kernel": kernel_names[dominant], "achieved": ach, "peak": peak,
                          "unit": "GB/s", "frac": ach / peak, "peak_kind": f"of {peak_kind}",
                          "frac_of_nominal_8TBs": ach / 8000.0,
                          "traffic": NCU_TRAFFIC_BYTES.get((w.cfg_id, dominant)),
@@ -538,7 +542,7 @@ def run_prefill(args):
                 "e2e": {"value": tokens / (ms_e2e * 1e-3), "unit": "head-tokens/s",
                         "h2d_bytes_per_step": 3 * Q.numel() * 2, "d2h_bytes_per_step": rec_bytes},
                 "gpu_launches": int(launches),
-                "roofline": {"bound": "tensor", "kernel": dominant + "_tc_kernel", "achieved": ach, "peak": peak,
+                "roofline": {"bound": "tensor", "kernel": {"build": "state_tc_kernel"}.get(dominant, dominant + "_tc_kernel"), "achieved": ach, "peak": peak,
                              "unit": "TFLOP/s", "frac": ach / peak, "peak_kind": kind, "traffic": None,
                              "algorithmic_flops_per_launch": fl[dominant],
                              "kernel_ms": {k: v for k, v in kt.items() if v},
