@@ -38,7 +38,7 @@ __device__ __forceinline__ InstMap map_instance(const PfParams& p, int g) {
 
 // launchers of the tensor-core kernels (score_tc.cu, state_tc.cu, psi_tc.cu)
 bool score_tc_supported();
-int launch_score_tc(less_ctx* c, const PfParams& p, int G, cudaStream_t s);
+int launch_score_tc(less_ctx* c, const PfParams& p, int G, cudaStream_t s, bool with_column_sums);
 // prompt attention output from the row statistics launch_score_tc leaves behind (attn_out_tc.cu)
 int launch_attn_out_tc(less_ctx* c, const PfParams& p, int G, cudaStream_t s);
 int launch_state_tc(less_ctx* c, const PfParams& p, int G, cudaStream_t s);

@@ -1,11 +1,12 @@
-// Prompt-phase kernels (Section 3.1: regular attention, then the policy once):
-//   rowstat_kernel   m_i, 1/l_i of causal row i of Q K^T / sqrt(D)
-//   colsum_kernel    acc_j = sum_{i >= j} exp(s_ij - m_i) / l_i      (H2O scores)
-//   attn_out_kernel  optional prompt attention output
-//   select_kernel    recent window + `heavy` largest (acc, pos) -> slot of every token
-//   build_kernel     psi(k_j) for every token; kept rows -> slots, evicted rows ->
-//                    partial H, z (Eq. 4, Eq. 5 summed over D_1)
-//   finalize_kernel  fixed-order sum of the partials
+// Prompt-phase kernels that run on CUDA cores, and the launcher of the whole prompt phase
+// (Section 3.1: regular attention, then the policy once):
+//   select_kernel    recent window + `heavy` largest (acc, pos) -> slot of every token (H2O);
+//                    first tokens + window (Lambda-masking); N largest of the last row (TOVA)
+//   lastrow_kernel   TOVA: the last prompt query's attention probabilities
+//   gather_kernel    kept rows -> slots (K, V, position, score, cached psi)
+//   finalize_kernel  fixed-order sum of the state build's partial H, z
+//   rowstat_kernel, colsum_kernel, attn_out_kernel, psi_kernel
+//                    fallbacks of the tensor-core kernels (score_tc.cu, attn_out_tc.cu, psi_tc.cu)
 #include "feature_mlp.cuh"
 #include "prefill.cuh"
 
@@ -461,14 +462,14 @@ int launch_prefill_group(less_ctx* c, int layer0, int nl, int lj0, int layer_cou
   if (S > 0 && need_scores) {
     const int tiles = (S + PF_TILE - 1) / PF_TILE;
     if (c->score_path == 1 && score_tc_supported()) {
-      const int rc = launch_score_tc(c, p, G, s);
+      const int rc = launch_score_tc(c, p, G, s, h2o);   // column sums only where H2O ranks by them
       if (rc != LESS_OK) return rc;
     } else {
       {
         LaunchScope scope(c, LESS_KERNEL_ROWSTAT, s);
         rowstat_kernel<<<dim3(tiles, G), PF_TILE, 0, s>>>(p);
       }
-      {
+      if (h2o) {
         LaunchScope scope(c, LESS_KERNEL_COLSUM, s);
         colsum_kernel<<<dim3(tiles, G), PF_TILE, 0, s>>>(p);
       }
@@ -481,7 +482,7 @@ int launch_prefill_group(less_ctx* c, int layer0, int nl, int lj0, int layer_cou
       attn_out_kernel<<<dim3((S + AO_ROWS - 1) / AO_ROWS, G), PF_TILE, 0, s>>>(p);
     }
   }
-  if (S > 0 && (d.flags & LESS_POLICY_TOVA)) {   // after the column sums, if any ran: both write ws_acc
+  if (S > 0 && (d.flags & LESS_POLICY_TOVA)) {
     LaunchScope scope(c, LESS_KERNEL_COLSUM, s);
     lastrow_kernel<<<G, LR_THREADS, 0, s>>>(p);
   }

@@ -369,7 +369,7 @@ __global__ void __launch_bounds__(CS_THREADS) colsum_tc_kernel(const __grid_cons
 
 bool score_tc_supported() { return encode_tiled_fn() != nullptr; }
 
-int launch_score_tc(less_ctx* c, const PfParams& p, int G, cudaStream_t s) {
+int launch_score_tc(less_ctx* c, const PfParams& p, int G, cudaStream_t s, bool with_column_sums) {
   const Dims& d = c->d;
   CUtensorMap tq, tk;
   const uint64_t rows = (uint64_t)d.B * p.layer_count * d.Hd * p.S;
@@ -390,7 +390,7 @@ int launch_score_tc(less_ctx* c, const PfParams& p, int G, cudaStream_t s) {
     LaunchScope scope(c, LESS_KERNEL_ROWSTAT, s);
     rowstat_tc_kernel<<<dim3(tiles, G), RS_THREADS, smem1, s>>>(tq_res, tk, p);
   }
-  {
+  if (with_column_sums) {
     LaunchScope scope(c, LESS_KERNEL_COLSUM, s);
     colsum_tc_kernel<<<dim3(tiles, G), CS_THREADS, smem2, s>>>(tq, tk_res, p);
   }
