@@ -147,7 +147,12 @@ int less_prefill(less_ctx* ctx, int32_t layer_begin, int32_t layer_count, int32_
  *   it takes the next free slot.
  * q, k, v: device fp16 [B, L, H, D].  out: device fp32 [B, L, H, D].
  * evicted_pos: device int32 [B, L, H] or NULL; receives the evicted position
- * or -1.  Advances the context's position by one. */
+ * or -1.  Advances the context's position by one.  A step captured in a CUDA
+ * graph (fixed q, k, v, out buffers; make one direct call first) reads the
+ * position from device memory and advances it there, so every replay is the
+ * next step; after replays, call less_poll_status (or less_export_state)
+ * before the next direct call so that the host's copy of the position catches
+ * up. */
 int less_decode_step(less_ctx* ctx, const void* q, const void* k, const void* v, void* out,
                      int32_t* evicted_pos, void* cuda_stream);
 
@@ -181,7 +186,9 @@ enum {
 int less_profile(less_ctx* ctx, int enable);
 int less_profile_read(less_ctx* ctx, float* ms_total_host, int64_t* launches_host);
 
-/* Tokens seen so far (= absolute position of the next decode token). */
+/* Tokens seen so far (= absolute position of the next decode token), as the
+ * host last knew it: direct calls keep it current; after graph replays
+ * less_poll_status or less_export_state refresh it from the device. */
 int64_t less_position(const less_ctx* ctx);
 
 /* Bytes of one exported instance record:

@@ -90,7 +90,8 @@ struct DecParams {
   float* out;                                           // [I, D]
   int32_t* evicted_pos;                                 // [I] or null
   Arena a;
-  int N, Np, heavy, recent, t;
+  int N, Np, heavy, recent;
+  int t;             // position of this step's token (direct calls)
   uint32_t flags;
 };
 
@@ -120,7 +121,23 @@ __device__ __forceinline__ float block_sum(float v, float* red) {
   return r;
 }
 
-template <int R>
+// The position of the step's token.  A direct call passes it as a kernel argument and CTA 0
+// leaves position + 1 in device memory.  A step that is being captured in a CUDA graph cannot bake
+// the position in: it reads it from device memory, and the CTAs count themselves out so that the
+// last one advances it for the next replay (one contended atomic per CTA: the price of replaying
+// without the host, paid only by captured steps).
+template <bool kCaptured>
+__device__ __forceinline__ void step_done(int32_t* tpos, int t) {
+  if (threadIdx.x != 0) return;
+  if (!kCaptured) {
+    if (blockIdx.x == 0) tpos[0] = t + 1;
+  } else if (atomicAdd(tpos + 1, 1) == (int)gridDim.x - 1) {   // every thread read the position barriers ago
+    tpos[1] = 0;
+    atomicAdd(tpos, 1);
+  }
+}
+
+template <int R, bool kCaptured>
 __global__ void __launch_bounds__(DEC_THREADS) decode_kernel(DecParams p) {
   extern __shared__ float dsm[];
   float* s_sc = dsm;                               // [Np + 4] scores, then e^{s - m}
@@ -133,9 +150,11 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_kernel(DecParams p) {
   const size_t inst = blockIdx.x;
   const int l16 = tid & 15, rg = tid >> 4;
   const int N = p.N;
+  const int t_now = kCaptured ? __ldcg(p.a.tpos) : p.t;   // tokens seen = this token's position
   int n = p.a.count[inst];
   if (n < 0 || n > N) {                            // refuse a corrupt count, touch nothing
     if (tid == 0) set_status(p.a.status, kStatusBounds, 1);
+    step_done<kCaptured>(p.a.tpos, p.t);
     return;
   }
   const bool use_state = !(p.flags & LESS_NO_STATE);
@@ -258,7 +277,7 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_kernel(DecParams p) {
         best = key < best ? key : best;
       } else if (lambda_policy) {                           // Lambda-masking: the oldest position past the first tokens
         if (ps >= p.heavy) best = (unsigned long long)(unsigned int)ps < best ? (unsigned int)ps : best;
-      } else if (ps <= p.t - p.recent) {             // H2O: lowest (accumulated score, position) outside the window
+      } else if (ps <= t_now - p.recent) {             // H2O: lowest (accumulated score, position) outside the window
         const unsigned long long key =
             ((unsigned long long)__float_as_uint(a) << 32) | (unsigned int)ps;
         best = key < best ? key : best;
@@ -283,9 +302,9 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_kernel(DecParams p) {
       // the new pair competes too; if its own probability is the lowest it never enters the
       // cache: it is absorbed into H, z at once and every slot stays as it is
       const unsigned long long key_new =
-          ((unsigned long long)__float_as_uint(p_new) << 32) | (unsigned int)p.t;
+          ((unsigned long long)__float_as_uint(p_new) << 32) | (unsigned int)t_now;
       if (key_new < best) {                          // uniform over the CTA
-        if (tid == 0 && p.evicted_pos) p.evicted_pos[inst] = p.t;
+        if (tid == 0 && p.evicted_pos) p.evicted_pos[inst] = t_now;
         if (use_state) {
           const float vv = __half2float(p.v[inst * kHeadDim + d]);
           const float* psn = p.a.psi_k + inst * R;
@@ -293,6 +312,7 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_kernel(DecParams p) {
           for (int r = 0; r < R; ++r) Hb[r * kHeadDim + d] = fmaf(psn[r], vv, hcol[r]);
           if (tid < R) zb[tid] += psn[tid];
         }
+        step_done<kCaptured>(p.a.tpos, p.t);
         return;
       }
     }
@@ -306,6 +326,7 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_kernel(DecParams p) {
         set_status(p.a.status, kStatusBounds, 2);
         if (p.evicted_pos) p.evicted_pos[inst] = -1;
       }
+      step_done<kCaptured>(p.a.tpos, p.t);
       return;
     }
     if (tid == 0 && p.evicted_pos) p.evicted_pos[inst] = vpos;
@@ -329,10 +350,11 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_kernel(DecParams p) {
   __half* Vw = p.a.vslots + (inst * (size_t)N + slot) * kHeadDim;
   if (rg == 0) *reinterpret_cast<uint4*>(Kw + l16 * 8) = knew;
   if (rg == 1) *reinterpret_cast<uint4*>(Vw + l16 * 8) = vnew;
-  if (tid == 32) { posb[slot] = p.t; accb[slot] = p_new; }
+  if (tid == 32) { posb[slot] = t_now; accb[slot] = p_new; }
   if (tid >= 64 && tid < 64 + R)
     p.a.psic[(inst * (size_t)N + slot) * R + (tid - 64)] =
         use_state ? p.a.psi_k[inst * R + (tid - 64)] : 0.f;
+  step_done<kCaptured>(p.a.tpos, p.t);
 }
 
 int launch_decode(less_ctx* c, const void* q, const void* k, const void* v, void* out,
@@ -343,11 +365,16 @@ int launch_decode(less_ctx* c, const void* q, const void* k, const void* v, void
   p.out = (float*)out;
   p.evicted_pos = evicted_pos;
   p.a = c->a;
-  p.N = d.N; p.Np = d.Np; p.heavy = d.heavy; p.recent = d.recent; p.t = (int)c->t;
+  p.N = d.N; p.Np = d.Np; p.heavy = d.heavy; p.recent = d.recent;
+  p.t = (int)c->t;
+  cudaStreamCaptureStatus capturing = cudaStreamCaptureStatusNone;
+  cudaStreamIsCapturing(s, &capturing);
+  const bool captured = capturing == cudaStreamCaptureStatusActive;   // then the position is read from, and advanced in, device memory
   p.flags = d.flags;
   const size_t smem = (size_t)(d.Np + 4 + DEC_RG * kHeadDim) * 4;
   LaunchScope scope(c, LESS_KERNEL_DECODE, s);
-  auto kern = d.R == 8 ? decode_kernel<8> : decode_kernel<16>;
+  auto kern = d.R == 8 ? (captured ? decode_kernel<8, true> : decode_kernel<8, false>)
+                       : (captured ? decode_kernel<16, true> : decode_kernel<16, false>);
   if (smem > 48 * 1024 &&
       cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
     return fail_cuda("shared memory opt-in of decode_kernel");

@@ -73,6 +73,7 @@ size_t carve(const Dims& d, char* base, Arena* a) {
   t.phi_q = (float*)take(I * R * 4);
   t.psi_k = (float*)take(I * R * 4);
   t.status = (int32_t*)take(4 * 4);
+  t.tpos = (int32_t*)take(4 * 4);
   t.stage_q = (__half*)take(I * D * 2);
   t.stage_k = (__half*)take(I * D * 2);
   t.stage_v = (__half*)take(I * D * 2);
@@ -176,6 +177,7 @@ int less_create(const less_config* cfg, const less_weights* w, void* arena, size
   if (e == cudaSuccess) e = cudaMemset(c->a.z, 0, (size_t)d.I * d.R * 4);
   if (e == cudaSuccess) e = cudaMemset(c->a.count, 0, (size_t)d.I * 4);
   if (e == cudaSuccess) e = cudaMemset(c->a.status, 0, 16);
+  if (e == cudaSuccess) e = cudaMemset(c->a.tpos, 0, 16);
   if (e == cudaSuccess) e = cudaMemset(c->a.phi_q, 0, (size_t)d.I * d.R * 4);
   if (e == cudaSuccess) e = cudaMemset(c->a.psi_k, 0, (size_t)d.I * d.R * 4);
   if (e == cudaSuccess) e = cudaDeviceSynchronize();
@@ -320,16 +322,26 @@ static int copy_state(less_ctx* c, const int32_t* inst, int32_t n, void* host, s
     cp(rec + r.H, c->a.H + I * d.R * d.D, (size_t)d.R * d.D * 4);
     cp(rec + r.z, c->a.z + I * d.R, (size_t)d.R * 4);
   }
+  // the position lives on the device (a captured step advances it without the host); the host
+  // keeps a copy for less_position
+  int32_t tdev = 0;
+  if (to_host) {
+    if (e == cudaSuccess) e = cudaMemcpyAsync(&tdev, c->a.tpos, 4, cudaMemcpyDeviceToHost, s);
+  } else if (n > 0) {
+    tdev = ((const int32_t*)host)[1];
+    if (e == cudaSuccess) e = cudaMemcpyAsync(c->a.tpos, &tdev, 4, cudaMemcpyHostToDevice, s);
+  }
   if (e == cudaSuccess) e = cudaStreamSynchronize(s);
   if (e != cudaSuccess) return LESS_ERR_CUDA;
   if (to_host) {
+    c->t = tdev;
     for (int i = 0; i < n; ++i) {
       int32_t* hdr = (int32_t*)((char*)host + r.total * (size_t)i);
-      hdr[1] = (int32_t)c->t;
+      hdr[1] = tdev;
       hdr[2] = hdr[3] = 0;
     }
   } else if (n > 0) {
-    c->t = ((const int32_t*)host)[1];
+    c->t = tdev;
   }
   return LESS_OK;
 }
@@ -369,9 +381,12 @@ int less_poll_status(less_ctx* c, void* stream) {
   if (!c) return LESS_ERR_NULL_POINTER;
   int32_t st[4] = {0, 0, 0, 0};
   cudaStream_t s = (cudaStream_t)stream;
+  int32_t tdev = 0;
   cudaError_t e = cudaMemcpyAsync(st, c->a.status, 16, cudaMemcpyDeviceToHost, s);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(&tdev, c->a.tpos, 4, cudaMemcpyDeviceToHost, s);
   if (e == cudaSuccess) e = cudaStreamSynchronize(s);
   if (e != cudaSuccess) return LESS_ERR_CUDA;
+  c->t = tdev;                                   // replays of a captured step advance only the device's count
   if (st[0] == kStatusTimeout) return LESS_ERR_DEVICE_TIMEOUT;
   if (st[0] == kStatusBounds) return LESS_ERR_DEVICE_BOUNDS;
   return LESS_OK;

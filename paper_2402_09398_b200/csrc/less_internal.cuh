@@ -29,6 +29,7 @@ struct Arena {
   float* phi_q;      // [I][R]      phi(q_t) of the current step
   float* psi_k;      // [I][R]      psi(k_t) of the current step
   int32_t* status;   // [4]         device status word(s)
+  int32_t* tpos;     // [4]         [0] tokens seen = position of the next decode token, [1] decode CTAs finished this step
   __half* stage_q;   // [I][D]      staging of host inputs (less_decode_step_host)
   __half* stage_k;   // [I][D]
   __half* stage_v;   // [I][D]

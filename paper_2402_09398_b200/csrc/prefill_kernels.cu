@@ -251,6 +251,7 @@ __global__ void __launch_bounds__(SEL_THREADS) select_kernel(PfParams p) {
   if (tid == 0) {
     p.a.count[im.inst] = min(S, N);
     p.a.ws_pmax[g] = 0;                          // the psi kernels that follow take the maximum into it
+    if (g == 0) { p.a.tpos[0] = S; p.a.tpos[1] = 0; }   // the first decode token has position S
   }
   if (S <= N) {
     for (int j = tid; j < S; j += SEL_THREADS) slot_of[j] = j;

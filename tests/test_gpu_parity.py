@@ -381,3 +381,39 @@ def test_tova_new_token_can_evict_itself():
     assert np.allclose(post["H"], np.outer(psi_k[0], np.full(D, 7.0)), rtol=1e-6)
     assert np.allclose(post["z"], psi_k[0], rtol=1e-6)
     ctx.close()
+
+
+@pytest.mark.parametrize("batch", [1, 12])
+def test_captured_step_replays_like_direct_calls(batch):
+    """One decode step captured in a CUDA graph (fixed input / output buffers) and replayed: the
+    position advances on the device, so every replay is the next step.  Outputs and state must be
+    bit-identical to direct calls on a second context."""
+    w = small(49, batch=batch, layers=2, heads=2, steps=7, weight_std=0.1)
+    ctx_d, _ = _setup(w)
+    ctx_g, _ = _setup(w)
+    for ctx in (ctx_d, ctx_g):
+        _prefill_all(ctx, w, with_out=False)
+    q0, k0, v0 = wl.make_decode_inputs(w, 0, DEV)
+    qb, kb, vb = q0.clone(), k0.clone(), v0.clone()
+    ob = torch.empty(q0.shape, dtype=torch.float32, device=DEV)
+    evb = torch.empty(w.instances, dtype=torch.int32, device=DEV)
+    ref0 = ctx_d.decode_step(q0, k0, v0)
+    assert torch.equal(ctx_g.decode_step(qb, kb, vb, out=ob, evicted_pos=evb), ref0)   # also the warm-up launch
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        ctx_g.decode_step(qb, kb, vb, out=ob, evicted_pos=evb)
+    evd = torch.empty_like(evb)
+    for s in range(1, w.steps):
+        q, k, v = wl.make_decode_inputs(w, s, DEV)
+        qb.copy_(q); kb.copy_(k); vb.copy_(v)
+        graph.replay()
+        ref = ctx_d.decode_step(q, k, v, evicted_pos=evd)
+        assert torch.equal(ob, ref) and torch.equal(evb, evd), s
+    assert ctx_g.poll_status() == 0 and ctx_d.poll_status() == 0
+    assert ctx_g.position == ctx_d.position == w.prompt + w.steps
+    inst = list(range(w.instances))
+    for a, b in zip(ctx_d.export_state(inst), ctx_g.export_state(inst)):
+        assert a["t"] == b["t"]
+        for key in ("pos", "acc", "K", "V", "psi", "H", "z"):
+            assert np.array_equal(a[key], b[key]), key
+    ctx_d.close(); ctx_g.close()
