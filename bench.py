@@ -32,11 +32,8 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures
 # summarised under profiles/ (None where no capture of that kernel and workload exists)
 NCU_TRAFFIC_BYTES = {
-    (2, "feature_map"): 285.93e6 + 5.82e6,   # profiles/decode_step_cfg2.md
-    (2, "decode"): 113.87e6 + 3.10e6,
-    # cfg3 captured at batch 16 (a quarter of the instances; both kernels' traffic is per instance or
-    # per head, so the decode kernel's scales by 4 and the feature maps' weights do not)
-    (3, "decode"): 4 * (1.824e9 + 50.2e6),
+    (2, "feature_map"): 285.91e6 + 5.46e6,   # profiles/decode_step_cfg2.md
+    (2, "decode"): 113.87e6 + 3.32e6,
 }
 
 
@@ -417,7 +414,7 @@ def run_b200(args):
         kernel_names = {"feature_map": ("feature_tc_small_kernel" if w.batch <= 8 else "feature_tc_kernel")
                         + f"<{w.rank}" + (f", {1 if w.batch <= 1 else 2 if w.batch <= 2 else 4 if w.batch <= 4 else 8}>"
                                           if w.batch <= 8 else ">"),
-                        "decode": f"decode_kernel<{w.rank}>"}
+                        "decode": f"decode_kernel<{w.rank}, {1 if args.graph else 0}>"}
         ach = kb[dominant] / (kt[dominant] * 1e-3) / 1e9 if kt[dominant] > 0 else 0.0
         step_bytes = kb["feature_map"] + kb["decode"]
         kv_state_bytes = w.instances * (n_live * (4 * w.head_dim + 8) + (0 if args.no_state else 2 * w.rank * w.head_dim * 4))
