@@ -260,6 +260,125 @@ class LessInstance:
                 "dH": dH, "dz": dz}
 
 
+class LessGroup:
+    """One KV head shared by G query heads (multi-query / grouped-query attention).
+
+    Section 3.2: "For multi-query attention, we extend H2O to aggregate attention scores across
+    all query attention heads to determine KV pairs to evict."  Reading taken here: the cache
+    (kept K, V), the accumulated scores and the low-rank state H, z belong to the KV head (psi
+    acts on keys, so H = sum psi(k)^T v does not depend on the query head); every query head g has
+    its own phi_g and its own Eq. 3 over the shared cache and state; the H2O score of an entry
+    grows by the sum over g of the probabilities p_{g,i}; one entry is evicted per step for all G
+    heads.  Policies: 'h2o' and 'lambda' (TOVA is left per head).  With G = 1 this is LessInstance.
+    """
+
+    def __init__(self, head_dim, rank, heavy, recent, phi_fns, psi_fn, score_norm="less",
+                 use_state=True, policy="h2o"):
+        if policy not in ("h2o", "lambda"):
+            raise ValueError("grouped heads support the 'h2o' and 'lambda' policies")
+        self.G = len(phi_fns)
+        self.phi_fns = list(phi_fns)
+        # bookkeeping (slots, scores, state, eviction) is that of a single instance
+        self.core = LessInstance(head_dim, rank, heavy, recent, phi_fns[0], psi_fn, score_norm, use_state, policy)
+
+    # the shared state, as LessInstance exposes it
+    def __getattr__(self, name):
+        if name in ("pos", "K", "V", "acc", "H", "z", "t", "evicted", "N", "heavy", "recent", "prompt_acc",
+                    "psi_fn", "import_state"):
+            return getattr(self.core, name)
+        raise AttributeError(name)
+
+    def prefill(self, Q, K, V, row_block=512):
+        """Q [G, S, D]; K, V [S, D].  Returns the G causal attention outputs [G, S, D]."""
+        c = self.core
+        Q = np.asarray(Q, dtype=np.float64)
+        K = np.asarray(K, dtype=np.float64)
+        V = np.asarray(V, dtype=np.float64)
+        G, S, D = Q.shape
+        c.reset()
+        out = np.zeros((G, S, D))
+        acc = np.zeros(S)
+        for g in range(G):
+            for r0 in range(0, S, row_block):
+                r1 = min(S, r0 + row_block)
+                s = (Q[g, r0:r1] @ K[:r1].T) / math.sqrt(D)
+                s = np.where(np.arange(r1)[None, :] <= np.arange(r0, r1)[:, None], s, -np.inf)
+                e = np.exp(s - s.max(axis=1, keepdims=True))
+                P = e / e.sum(axis=1, keepdims=True)
+                out[g, r0:r1] = P @ V[:r1]
+                acc[:r1] += P.sum(axis=0)                     # summed over rows and over the G heads
+        c.t = S
+        pos = np.arange(S, dtype=np.int64)
+        if c.policy == "lambda":
+            acc = np.zeros(S)
+        if S <= c.N:
+            keep, evict = pos, pos[:0]
+        else:
+            if c.policy == "lambda":
+                evict = pos[c.heavy: S - c.recent]
+            else:
+                cand = pos[: S - c.recent]
+                order = np.lexsort((cand, acc[cand]))
+                evict = np.sort(cand[order[: S - c.N]])
+            mask = np.ones(S, dtype=bool)
+            mask[evict] = False
+            keep = pos[mask]
+        c.pos, c.K, c.V, c.acc = keep.copy(), K[keep].copy(), V[keep].copy(), acc[keep].copy()
+        if evict.size and c.use_state:
+            psi = c.psi_fn(K[evict])
+            c.H, c.z = psi.T @ V[evict], psi.sum(axis=0)
+        c.evicted = [int(p) for p in evict]
+        c.prompt_acc = acc
+        return out
+
+    def decode(self, q, k, v):
+        """q [G, D]; k, v [D].  One step for the G query heads of this KV head."""
+        c = self.core
+        q = np.asarray(q, dtype=np.float64)
+        k = np.asarray(k, dtype=np.float64)
+        v = np.asarray(v, dtype=np.float64)
+        t = c.t
+        Kp, Vp = np.vstack([c.K, k[None]]), np.vstack([c.V, v[None]])
+        outs, p_sum, lr_nums, lr_dens = [], np.zeros(Kp.shape[0]), [], []
+        for g in range(self.G):
+            e = np.exp((Kp @ q[g]) / math.sqrt(c.D))                 # Eq. 3 for head g
+            phi = self.phi_fns[g](q[g][None])[0]
+            lr_num, lr_den = phi @ c.H, float(phi @ c.z)
+            den_sparse = float(e.sum())
+            den = lr_den + den_sparse
+            outs.append((lr_num + e @ Vp) / den)
+            p_sum += e / (den if c.score_norm == "less" else den_sparse)
+            lr_nums.append(lr_num)
+            lr_dens.append(lr_den)
+        acc = np.concatenate([c.acc + p_sum[:-1], p_sum[-1:]])       # aggregated over the heads
+        pos = np.concatenate([c.pos, np.array([t], dtype=np.int64)])
+        evicted_pos, gap, dH, dz = -1, None, None, None
+        if pos.size > c.N:
+            if c.policy == "lambda":
+                cand = np.nonzero(pos >= c.heavy)[0]
+                order = np.argsort(pos[cand])
+            else:
+                cand = np.nonzero(pos <= t - c.recent)[0]
+                order = np.lexsort((pos[cand], acc[cand]))
+            vic = int(cand[order[0]])
+            if cand.size > 1 and c.policy == "h2o":
+                a0, a1 = acc[cand[order[0]]], acc[cand[order[1]]]
+                gap = abs(a1 - a0) / max(abs(a0), abs(a1), 1e-300)
+            evicted_pos = int(pos[vic])
+            if c.use_state:
+                psi = c.psi_fn(Kp[vic][None])[0]
+                dH, dz = np.outer(psi, Vp[vic]), psi
+                c.H, c.z = c.H + dH, c.z + dz
+            c.evicted.append(evicted_pos)
+            keep = np.ones(pos.size, dtype=bool)
+            keep[vic] = False
+            pos, acc, Kp, Vp = pos[keep], acc[keep], Kp[keep], Vp[keep]
+        c.pos, c.acc, c.K, c.V = pos, acc, Kp, Vp
+        c.t = t + 1
+        return {"out": np.stack(outs), "evicted_pos": evicted_pos, "tie_gap": gap, "p": p_sum,
+                "lr_num": np.stack(lr_nums), "lr_den": np.array(lr_dens), "dH": dH, "dz": dz}
+
+
 def make_mlp_maps(w_phi1, w_phi2, w_psi1, w_psi2, w_psi3, psi_scale=None):
     """phi/psi callables of one head from its weight matrices."""
     def phi_fn(x):

@@ -555,3 +555,79 @@ def test_tova_can_evict_the_new_token_itself():
     r = inst.decode(q, k_new, v_new)
     assert r["evicted_pos"] == 4 and list(inst.pos) == [0, 1, 2, 3]
     assert np.allclose(inst.H, np.outer(psi(k_new[None])[0], v_new)) and np.allclose(inst.z, psi(k_new[None])[0])
+
+
+# --------------------------------------------------------------------------- #
+# Grouped query heads (Section 3.2: H2O scores aggregated across the query heads of a KV head)
+# --------------------------------------------------------------------------- #
+def _group_case(G, cfg_id=100, S=28, T=12, heavy=3, recent=4, D=16, R=4, policy="h2o", use_state=True):
+    w = tiny(cfg_id=cfg_id, S=S, T=T, heavy=heavy, recent=recent, D=D, R=R, heads=G + 1)
+    W = wl.make_weights(w)
+    Q, K, V = wl.make_prompt(w, 0, 1)
+    phis = [lo.make_mlp_maps(*head_weights(W, 0, g))[0] for g in range(G)]      # phi of query head g
+    psi_w = head_weights(W, 0, G)                                               # psi of the KV head
+    psi_fn = lo.make_mlp_maps(*psi_w)[1]
+    grp = lo.LessGroup(D, R, heavy, recent, phis, psi_fn, use_state=use_state, policy=policy)
+    Qg = np.stack([Q[0, 0, g].double().numpy() for g in range(G)])
+    Kk, Vv = K[0, 0, G].double().numpy(), V[0, 0, G].double().numpy()
+    return w, W, grp, Qg, Kk, Vv, psi_w
+
+
+def test_group_of_one_is_the_single_head_instance():
+    w, W, grp, Qg, Kk, Vv, psi_w = _group_case(1)
+    one = lo.LessInstance(16, 4, 3, 4, grp.phi_fns[0], grp.psi_fn)
+    assert np.array_equal(grp.prefill(Qg, Kk, Vv)[0], one.prefill(Qg[0], Kk, Vv))
+    for s in range(w.steps):
+        q, k, v = (a[0, 0].double().numpy() for a in wl.make_decode_inputs(w, s))
+        a, b = grp.decode(q[:1], k[1], v[1]), one.decode(q[0], k[1], v[1])
+        assert np.array_equal(a["out"][0], b["out"]) and a["evicted_pos"] == b["evicted_pos"]
+    assert np.array_equal(grp.H, one.H) and list(grp.pos) == list(one.pos)
+
+
+@pytest.mark.parametrize("G", [2, 4])
+def test_group_scores_are_summed_over_heads_and_state_is_shared(G):
+    """Independent check with torch: every head's output is Eq. 3 over the shared kept set and the
+    shared Eq. 6 sums; the victim is the minimum of the head-summed accumulated probabilities, kept
+    here in a dict by position and rebuilt from scratch every step."""
+    w, W, grp, Qg, Kk, Vv, psi_w = _group_case(G, cfg_id=101)
+    heavy, recent, N = 3, 4, 7
+    grp.prefill(Qg, Kk, Vv)
+    Kt, Vt = [torch.tensor(Kk)], [torch.tensor(Vv)]
+    S = w.prompt
+    # prompt scores: sum over heads of the causal softmax column sums
+    score = np.zeros(S)
+    for g in range(G):
+        s = torch.tensor(Qg[g]) @ Kt[0].T / math.sqrt(16)
+        s = s.masked_fill(torch.triu(torch.ones_like(s), 1).bool(), float("-inf"))
+        score += torch.softmax(s, dim=-1).sum(0).numpy()
+    cand = sorted(range(S - recent), key=lambda j: (score[j], j))
+    kept = set(range(S)) - set(cand[: S - N])
+    hist = {j: score[j] for j in kept}
+    gone = set(cand[: S - N])
+    assert sorted(kept) == list(grp.pos)
+    phi_w = [head_weights(W, 0, g)[:2] for g in range(G)]
+    for i in range(w.steps):
+        q, k, v = (a[0, 0].double().numpy() for a in wl.make_decode_inputs(w, i))
+        t = S + i
+        Kt.append(torch.tensor(k[G])[None]); Vt.append(torch.tensor(v[G])[None])
+        Kall, Vall = torch.cat(Kt), torch.cat(Vt)
+        r = grp.decode(q[:G], k[G], v[G])
+        idx = sorted(kept) + [t]
+        g_idx = sorted(gone)
+        psi = torch_psi(Kall[g_idx].numpy(), *psi_w[2:])
+        Hs, zs = psi.T @ Vall[g_idx], psi.sum(0)
+        psum = np.zeros(len(idx))
+        for g in range(G):
+            e = torch.exp(Kall[idx] @ torch.tensor(q[g]) / math.sqrt(16))
+            phi = torch_phi(q[g][None], *phi_w[g])[0]
+            den = phi @ zs + e.sum()
+            assert np.allclose(r["out"][g], ((phi @ Hs + e @ Vall[idx]) / den).numpy(), rtol=1e-10, atol=1e-13)
+            psum += (e / den).numpy()
+        for j, pj in zip(idx, psum):
+            hist[j] = hist.get(j, 0.0) + pj
+        victim = min((hist[j], j) for j in idx if j <= t - recent)[1]
+        assert r["evicted_pos"] == victim
+        kept = (kept | {t}) - {victim}
+        gone.add(victim)
+        del hist[victim]
+    assert sorted(kept) == list(grp.pos)
