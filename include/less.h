@@ -85,7 +85,7 @@ enum {
 #define LESS_MAX_SLOTS 32768
 
 typedef struct less_config {
-  int32_t batch, layers, heads;
+  int32_t batch, layers, heads; /* heads = KV heads: one cache, one H, z and one eviction per (batch, layer, head) */
   int32_t head_dim;           /* D, must be 128 */
   int32_t rank;               /* R: 8 or 16 (Section 4: R = 8 by default) */
   int32_t hidden;             /* R' = 512 (Section 3.2) */
@@ -93,14 +93,15 @@ typedef struct less_config {
   int32_t max_prompt;         /* longest prompt less_prefill will be given (>= 0) */
   int32_t max_prefill_layers; /* layers scored together in less_prefill (>= 1): sizes the workspace */
   uint32_t flags;
+  int32_t group;              /* query heads per KV head (grouped- / multi-query attention); 0 or 1 = one */
 } less_config;
 
 /* Per-head feature-map weights (Eq. 1, Eq. 2), device, fp16, row-major, no biases:
  *   phi(q) = | gelu( gelu(q W_phi1) W_phi2 ) |
  *   psi(k) = | c2 * gelu( c1 * gelu(k W_psi1) W_psi2 ) W_psi3 |                     */
 typedef struct less_weights {
-  const void* w_phi1;     /* [L, H, D, R'] */
-  const void* w_phi2;     /* [L, H, R', R] */
+  const void* w_phi1;     /* [L, H * group, D, R']   (phi belongs to the query head) */
+  const void* w_phi2;     /* [L, H * group, R', R] */
   const void* w_psi1;     /* [L, H, D, R'] */
   const void* w_psi2;     /* [L, H, R', R] */
   const void* w_psi3;     /* [L, H, R, R]  */
@@ -126,9 +127,10 @@ int less_create(const less_config* cfg, const less_weights* weights, void* arena
  *      largest (acc, position) keys; if prompt_len <= heavy + recent keep all;
  *   4. kept rows go to slots in ascending position; every other row is
  *      absorbed: H = sum psi(k_j)^T v_j, z = sum psi(k_j) (Eq. 4, Eq. 5 over D_1).
- * Q, K, V: device fp16 [B, layer_count, H, prompt_len, D] contiguous, fewer than
+ * Q: device fp16 [B, layer_count, H * group, prompt_len, D]; K, V: device fp16
+ * [B, layer_count, H, prompt_len, D]; all contiguous, fewer than
  * 2^31 rows (B * layer_count * H * prompt_len) per call, else LESS_ERR_PROMPT_TOO_LONG.
- * attn_out: device fp32, same shape, or NULL when the caller does not need the
+ * attn_out: device fp32, same shape as Q, or NULL when the caller does not need the
  * prompt's attention output.
  * Every call of one generation must pass the same prompt_len; the first decode
  * token then has absolute position prompt_len.  A layer that was never
@@ -145,7 +147,11 @@ int less_prefill(less_ctx* ctx, int32_t layer_begin, int32_t layer_count, int32_
  *   position <= t - recent;  H += psi(k_vic)^T v_vic,  z += psi(k_vic)  (Eq. 4, 5);
  *   the new pair overwrites the victim's slot in place (Section 3.2), else
  *   it takes the next free slot.
- * q, k, v: device fp16 [B, L, H, D].  out: device fp32 [B, L, H, D].
+ * q: device fp16 [B, L, H * group, D]; k, v: device fp16 [B, L, H, D]; out: device fp32
+ * [B, L, H * group, D] (query head h * group + g belongs to KV head h).  With group > 1
+ * (Section 3.2: multi-query attention) every query head has its own phi and its own Eq. 3 over
+ * the KV head's cache and state, and the H2O score of an entry grows by the sum of the query
+ * heads' probabilities; policies: H2O and Lambda-masking.
  * evicted_pos: device int32 [B, L, H] or NULL; receives the evicted position
  * or -1.  Advances the context's position by one.  A step captured in a CUDA
  * graph (fixed q, k, v, out buffers; make one direct call first) reads the
@@ -207,8 +213,8 @@ int less_export_state(less_ctx* ctx, const int32_t* inst_host, int32_t n, void* 
 int less_import_state(less_ctx* ctx, const int32_t* inst_host, int32_t n, const void* host_buf,
                       size_t bytes, void* cuda_stream);
 
-/* phi(q_t) and psi(k_t) of the last decode step, all instances: host float
- * [B*L*H, R] each (either may be NULL).  Synchronises the stream. */
+/* phi(q_t) and psi(k_t) of the last decode step: host float [B*L*H*group, R]
+ * and [B*L*H, R] (either may be NULL).  Synchronises the stream. */
 int less_read_feature_maps(less_ctx* ctx, float* phi_host, float* psi_host, void* cuda_stream);
 
 /* Reads the device status word (synchronises the stream): 0, or

@@ -40,7 +40,7 @@ class less_config(C.Structure):
     _fields_ = [("batch", C.c_int32), ("layers", C.c_int32), ("heads", C.c_int32),
                 ("head_dim", C.c_int32), ("rank", C.c_int32), ("hidden", C.c_int32),
                 ("heavy", C.c_int32), ("recent", C.c_int32), ("max_prompt", C.c_int32),
-                ("max_prefill_layers", C.c_int32), ("flags", C.c_uint32)]
+                ("max_prefill_layers", C.c_int32), ("flags", C.c_uint32), ("group", C.c_int32)]
 
 
 class less_weights(C.Structure):
@@ -207,13 +207,13 @@ class LessContext:
 
     def __init__(self, batch, layers, heads, head_dim, rank, hidden, heavy, recent, max_prompt,
                  weights: Dict[str, torch.Tensor], max_prefill_layers: int = 1, flags: int = 0,
-                 psi_scale: Optional[torch.Tensor] = None, device="cuda"):
+                 psi_scale: Optional[torch.Tensor] = None, device="cuda", group: int = 1):
         if not torch.cuda.is_available():
             raise RuntimeError("the LESS library needs a CUDA device (there is no CPU path)")
         lib()
         self.device = torch.device(device)
         self.cfg = less_config(batch, layers, heads, head_dim, rank, hidden, heavy, recent,
-                               max_prompt, max_prefill_layers, flags)
+                               max_prompt, max_prefill_layers, flags, group)
         nbytes = less_arena_bytes(self.cfg)
         if nbytes == 0:
             raise LessError(-1, "less_arena_bytes")
@@ -227,6 +227,7 @@ class LessContext:
         _check(rc, "less_create")
         self.ctx = ctx
         self.instances = batch * layers * heads
+        self.group = max(1, group)
         self.N = heavy + recent
         self.record_bytes = less_state_record_bytes(self.cfg)
 
@@ -321,7 +322,7 @@ class LessContext:
 
     def read_feature_maps(self, stream=None):
         R = self.cfg.rank
-        phi = np.zeros((self.instances, R), dtype=np.float32)
+        phi = np.zeros((self.instances * self.group, R), dtype=np.float32)
         psi = np.zeros((self.instances, R), dtype=np.float32)
         _check(less_read_feature_maps(self.ctx, phi.ctypes.data, psi.ctypes.data, _stream_ptr(stream)),
                "less_read_feature_maps")
@@ -352,4 +353,4 @@ def from_workload(w, weights=None, device="cuda", max_prefill_layers=1, flags=0,
                        w.heavy if heavy is None else heavy, w.recent if recent is None else recent,
                        w.prompt if max_prompt is None else max_prompt, weights,
                        max_prefill_layers=max_prefill_layers, flags=flags, psi_scale=psi_scale,
-                       device=device)
+                       device=device, group=getattr(w, "group", 1))

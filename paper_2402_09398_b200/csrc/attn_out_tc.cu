@@ -63,8 +63,8 @@ __global__ void __launch_bounds__(AO_THREADS) attn_out_tc_kernel(const __grid_co
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int tiles = (p.S + AO_TILE - 1) / AO_TILE;
   const int tile = tiles - 1 - (int)blockIdx.x;                    // long rows first
-  const int g = blockIdx.y;
-  const InstMap im = map_instance(p, g);
+  const int g = blockIdx.y;                                        // query head (KV instance * grp + head of the group)
+  const QueryMap qm = map_query(p, g);
   const int i0 = tile * AO_TILE;
   const int ntile = tile + 1;                                      // key tiles 0 .. tile (the last holds the diagonal)
   int32_t* status = p.a.status;
@@ -107,7 +107,7 @@ __global__ void __launch_bounds__(AO_THREADS) attn_out_tc_kernel(const __grid_co
   if (warp == 0) {
     // ---------------- TMA producer ----------------
     if (lane == 0) {
-      const int row0 = (int)(im.in_row0 + i0);
+      const int row0 = (int)(qm.q_row0 + i0);
       mbar_expect_tx(&sh->res_full, AO_TILE_BYTES + AO_QX_BYTES);
       tma_load_2d(qres, &tm_q, 0, row0, &sh->res_full);
       tma_load_2d(qres + AO_TILE_BYTES / 2, &tm_q, 64, row0, &sh->res_full);
@@ -116,7 +116,7 @@ __global__ void __launch_bounds__(AO_THREADS) attn_out_tc_kernel(const __grid_co
       for (int t = 0; t < ntile; ++t) {
         wait_or_give_up(&sh->k_empty[s], ph ^ 1, abortp, status, 100);
         if (*abortp) break;
-        const int krow = (int)(im.in_row0 + (size_t)t * AO_TILE);
+        const int krow = (int)(qm.kv_row0 + (size_t)t * AO_TILE);
         unsigned char* st = ring + s * AO_STAGE_BYTES;
         mbar_expect_tx(&sh->k_full[s], AO_TILE_BYTES);
         tma_load_2d(st, &tm_k, 0, krow, &sh->k_full[s]);
@@ -131,7 +131,7 @@ __global__ void __launch_bounds__(AO_THREADS) attn_out_tc_kernel(const __grid_co
       for (int t = 0; t < ntile; ++t) {
         wait_or_give_up(&sh->v_empty[s], ph ^ 1, abortp, status, 108);
         if (*abortp) break;
-        const int krow = (int)(im.in_row0 + (size_t)t * AO_TILE);
+        const int krow = (int)(qm.kv_row0 + (size_t)t * AO_TILE);
         unsigned char* st = ring + s * AO_STAGE_BYTES + AO_TILE_BYTES;
         mbar_expect_tx(&sh->v_full[s], AO_TILE_BYTES);
         tma_load_2d(st, &tm_v, 0, krow, &sh->v_full[s]);
@@ -236,7 +236,7 @@ __global__ void __launch_bounds__(AO_THREADS) attn_out_tc_kernel(const __grid_co
     // ---- the finished rows: O[row][64 columns of this warp] ----
     wait_or_give_up(&sh->o_full, 0, abortp, status, 107);
     tc_fence_after_sync();
-    float* orow = p.attn_out + (im.in_row0 + i) * kHeadDim + half * 64;
+    float* orow = p.attn_out + (qm.q_row0 + i) * kHeadDim + half * 64;
 #pragma unroll 1
     for (int cg = 0; cg < 2; ++cg) {
       uint32_t o[32];
@@ -261,7 +261,7 @@ int launch_attn_out_tc(less_ctx* c, const PfParams& p, int G, cudaStream_t s) {
   const Dims& d = c->d;
   CUtensorMap tq, tk, tv;
   const uint64_t rows = (uint64_t)d.B * p.layer_count * d.Hd * p.S;
-  if (!make_tmap_f16_2d(&tq, p.Q, rows, kHeadDim, kHeadDim * 2, AO_TILE) ||
+  if (!make_tmap_f16_2d(&tq, p.Q, rows * p.grp, kHeadDim, kHeadDim * 2, AO_TILE) ||
       !make_tmap_f16_2d(&tk, p.K, rows, kHeadDim, kHeadDim * 2, AO_TILE) ||
       !make_tmap_f16_2d(&tv, p.V, rows, kHeadDim, kHeadDim * 2, AO_TILE))
     return fail_cuda("tensor maps of Q / K / V");
@@ -271,7 +271,7 @@ int launch_attn_out_tc(less_ctx* c, const PfParams& p, int G, cudaStream_t s) {
     return fail_cuda("shared memory opt-in of attn_out_tc_kernel");
   const int tiles = (p.S + AO_TILE - 1) / AO_TILE;
   LaunchScope scope(c, LESS_KERNEL_ATTN_OUT, s);
-  attn_out_tc_kernel<<<dim3(tiles, G), AO_THREADS, smem, s>>>(tq, tk, tv, p);
+  attn_out_tc_kernel<<<dim3(tiles, G * p.grp), AO_THREADS, smem, s>>>(tq, tk, tv, p);
   return check_launch("attn_out_tc_kernel");
 }
 

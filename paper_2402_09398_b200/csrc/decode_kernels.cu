@@ -62,11 +62,13 @@ int launch_feature_maps(less_ctx* c, const void* q, const void* k, cudaStream_t 
   p.out[0] = c->a.phi_q;
   p.out[1] = c->a.psi_k;
   p.B = d.B; p.L = d.L; p.Hd = d.Hd; p.Rp = d.Rp;
+  p.Hh[0] = d.Hd * d.G; p.Hh[1] = d.Hd;
   const int ndg = FM_THREADS / (d.Rp / 8);
   const size_t smem = (size_t)(FM_BR * kHeadDim + FM_BR * d.Rp + ndg * FM_BR * d.Rp) * 4;
   dim3 grid(d.L * d.Hd, (d.flags & LESS_NO_STATE) ? 1 : 2, (d.B + FM_BR - 1) / FM_BR);
   if (d.flags & LESS_NO_STATE) return LESS_OK;   // neither phi nor psi is used
-  if (c->feature_path == 2 && feature_tc_supported(d)) return launch_feature_tc(c, p, s);
+  if ((c->feature_path == 2 || d.G > 1) && feature_tc_supported(d)) return launch_feature_tc(c, p, s);
+  if (d.G > 1) return LESS_ERR_INVALID_CONFIG;    // the CUDA-core kernels know one query head per KV head
   if (c->feature_path >= 1 && feature_gemv_supported(d)) return launch_feature_gemv(c, p, s);
   LaunchScope scope(c, LESS_KERNEL_FEATURE_MAP, s);
   if (d.R == 8) {
@@ -357,6 +359,264 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_kernel(DecParams p) {
   step_done<kCaptured>(p.a.tpos, p.t);
 }
 
+// --------------------------------------------------------------------------- //
+// Grouped query heads (Section 3.2, multi-query attention): G query heads share one KV head.
+// One CTA per KV head reads its K and V slots once and serves the G queries from registers;
+// every query head has its own Eq. 3 (own phi, own normaliser) over the shared cache and
+// the shared H, z; an entry's H2O score grows by the sum of the G heads' probabilities and
+// one entry is evicted for all of them.
+// --------------------------------------------------------------------------- //
+template <int R, int G, bool kCaptured>
+__global__ void __launch_bounds__(DEC_THREADS) decode_group_kernel(DecParams p) {
+  extern __shared__ float dsm[];
+  const int Ns = p.Np + 4;
+  float* s_sc = dsm;                               // [G][Np + 4] scores, then e^{s - m_g}
+  float* s_red = s_sc + G * Ns;                    // [G][DEC_RG][128] partial numerators
+  __shared__ float s_small[DEC_THREADS / 32];
+  __shared__ unsigned long long s_key[DEC_THREADS / 32];
+  __shared__ int s_vic;
+  __shared__ float s_inv[G];
+
+  const int tid = threadIdx.x;
+  const size_t inst = blockIdx.x;
+  const int l16 = tid & 15, rg = tid >> 4;
+  const int N = p.N;
+  const int t_now = kCaptured ? __ldcg(p.a.tpos) : p.t;
+  int n = p.a.count[inst];
+  if (n < 0 || n > N) {
+    if (tid == 0) set_status(p.a.status, kStatusBounds, 1);
+    step_done<kCaptured>(p.a.tpos, p.t);
+    return;
+  }
+  const bool use_state = !(p.flags & LESS_NO_STATE);
+  const float scale = 0.08838834764831845f;        // 1 / sqrt(128)
+
+  const __half* Kb = p.a.kslots + inst * (size_t)N * kHeadDim;
+  const __half* Vb = p.a.vslots + inst * (size_t)N * kHeadDim;
+
+  float qf[G][8];
+#pragma unroll
+  for (int g = 0; g < G; ++g)
+    half8_to_float(*reinterpret_cast<const uint4*>(p.q + (inst * G + g) * kHeadDim + l16 * 8), qf[g]);
+
+  // ---- scores of the G heads against every live slot (each K row is read once) ----
+#pragma unroll 2
+  for (int r0 = 0; r0 < n; r0 += DEC_RG) {
+    const int r = r0 + rg;
+    float dot[G];
+#pragma unroll
+    for (int g = 0; g < G; ++g) dot[g] = 0.f;
+    if (r < n) {
+      float kf[8];
+      half8_to_float(ldg_stream(Kb + (size_t)r * kHeadDim + l16 * 8), kf);
+#pragma unroll
+      for (int g = 0; g < G; ++g)
+#pragma unroll
+        for (int c = 0; c < 8; ++c) dot[g] = fmaf(qf[g][c], kf[c], dot[g]);
+    }
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+#pragma unroll
+      for (int o = 8; o > 0; o >>= 1) dot[g] += __shfl_xor_sync(0xffffffffu, dot[g], o);
+      if (l16 == 0 && r < n) s_sc[g * Ns + r] = dot[g] * scale;
+    }
+  }
+  const uint4 knew = *reinterpret_cast<const uint4*>(p.k + inst * kHeadDim + l16 * 8);
+  const uint4 vnew = *reinterpret_cast<const uint4*>(p.v + inst * kHeadDim + l16 * 8);
+  if (tid < 32) {
+    float kf[8];
+    half8_to_float(knew, kf);
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+      float dot = 0.f;
+#pragma unroll
+      for (int c = 0; c < 8; ++c) dot = fmaf(qf[g][c], kf[c], dot);
+#pragma unroll
+      for (int o = 8; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+      if (tid == 0) s_sc[g * Ns + n] = dot * scale;
+    }
+  }
+  __syncthreads();
+
+  // ---- per head: m_g, e_i = exp(s_i - m_g), l_g ----
+  float mg[G], lg[G];
+#pragma unroll
+  for (int g = 0; g < G; ++g) {
+    float* sc = s_sc + g * Ns;
+    float m = -INFINITY;
+    for (int i = tid; i <= n; i += DEC_THREADS) m = fmaxf(m, sc[i]);
+    m = block_max(m, s_small);
+    m = fmaxf(m, -80.f);
+    float lsum = 0.f;
+    for (int i = tid; i <= n; i += DEC_THREADS) {
+      const float e = __expf(sc[i] - m);
+      sc[i] = e;
+      lsum += e;
+    }
+    mg[g] = m;
+    lg[g] = block_sum(lsum, s_small);
+  }
+
+  // ---- u_g = sum e_{g,i} v_i (each V row is read once) ----
+  float u[G][8];
+#pragma unroll
+  for (int g = 0; g < G; ++g)
+#pragma unroll
+    for (int c = 0; c < 8; ++c) u[g][c] = 0.f;
+#pragma unroll 2
+  for (int r = rg; r < n; r += DEC_RG) {
+    float vf[8];
+    half8_to_float(ldg_stream(Vb + (size_t)r * kHeadDim + l16 * 8), vf);
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+      const float e = s_sc[g * Ns + r];
+#pragma unroll
+      for (int c = 0; c < 8; ++c) u[g][c] = fmaf(e, vf[c], u[g][c]);
+    }
+  }
+  if (rg == 0) {
+    float vf[8];
+    half8_to_float(vnew, vf);
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+      const float e = s_sc[g * Ns + n];
+#pragma unroll
+      for (int c = 0; c < 8; ++c) u[g][c] = fmaf(e, vf[c], u[g][c]);
+    }
+  }
+#pragma unroll
+  for (int g = 0; g < G; ++g)
+#pragma unroll
+    for (int c = 0; c < 8; ++c) s_red[(g * DEC_RG + rg) * kHeadDim + l16 * 8 + c] = u[g][c];
+  __syncthreads();
+
+  // ---- Eq. 3 per head over the shared H, z ----
+  const int d = tid;
+  float* Hb = p.a.H + inst * (size_t)R * kHeadDim;
+  float* zb = p.a.z + inst * R;
+  float hcol[R], zr[R];
+  if (use_state) {
+    pdl_wait_primary();
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+      hcol[r] = Hb[r * kHeadDim + d];
+      zr[r] = zb[r];
+    }
+  }
+#pragma unroll
+  for (int g = 0; g < G; ++g) {
+    float num = 0.f;
+#pragma unroll
+    for (int j = 0; j < DEC_RG; ++j) num += s_red[(g * DEC_RG + j) * kHeadDim + d];
+    float den = lg[g];
+    if (use_state) {
+      const float em = __expf(-mg[g]);
+      const float* ph = p.a.phi_q + (inst * G + g) * R;
+      float lr = 0.f, lz = 0.f;
+#pragma unroll
+      for (int r = 0; r < R; ++r) {
+        const float f = ph[r];
+        lr = fmaf(f, hcol[r], lr);
+        lz = fmaf(f, zr[r], lz);
+      }
+      num = fmaf(em, lr, num);
+      den = fmaf(em, lz, den);
+    }
+    p.out[(inst * G + g) * kHeadDim + d] = num / den;
+    if (tid == 0) s_inv[g] = 1.0f / ((p.flags & LESS_SCORE_NORM_SPARSE) ? lg[g] : den);
+  }
+  __syncthreads();
+  float inv[G];
+#pragma unroll
+  for (int g = 0; g < G; ++g) inv[g] = s_inv[g];
+
+  // ---- H2O over the group: acc_i += sum_g p_{g,i}; one victim for all heads ----
+  int32_t* posb = p.a.pos + inst * (size_t)p.Np;
+  float* accb = p.a.acc + inst * (size_t)p.Np;
+  const bool full = (n == N);
+  const bool lambda_policy = (p.flags & LESS_POLICY_LAMBDA) != 0;
+  unsigned long long best = ~0ull;
+  for (int i = tid; i < n; i += DEC_THREADS) {
+    float ps_sum = 0.f;
+#pragma unroll
+    for (int g = 0; g < G; ++g) ps_sum = fmaf(s_sc[g * Ns + i], inv[g], ps_sum);
+    const float a = accb[i] + ps_sum;
+    accb[i] = a;
+    if (full) {
+      const int ps = posb[i];
+      if (lambda_policy) {
+        if (ps >= p.heavy) best = (unsigned long long)(unsigned int)ps < best ? (unsigned int)ps : best;
+      } else if (ps <= t_now - p.recent) {
+        const unsigned long long key =
+            ((unsigned long long)__float_as_uint(a) << 32) | (unsigned int)ps;
+        best = key < best ? key : best;
+      }
+    }
+  }
+  float p_new = 0.f;
+#pragma unroll
+  for (int g = 0; g < G; ++g) p_new = fmaf(s_sc[g * Ns + n], inv[g], p_new);
+  int slot = n;
+  if (full) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const unsigned long long other = __shfl_xor_sync(0xffffffffu, best, o);
+      best = other < best ? other : best;
+    }
+    if ((tid & 31) == 0) s_key[tid >> 5] = best;
+    if (tid == 0) s_vic = -1;
+    __syncthreads();
+    best = s_key[0];
+#pragma unroll
+    for (int w = 1; w < DEC_THREADS / 32; ++w) best = s_key[w] < best ? s_key[w] : best;
+    const int vpos = (int)(unsigned int)(best & 0xffffffffull);
+    for (int i = tid; i < n; i += DEC_THREADS)
+      if (posb[i] == vpos && best != ~0ull) s_vic = i;
+    __syncthreads();
+    slot = s_vic;
+    if (slot < 0) {
+      if (tid == 0) {
+        set_status(p.a.status, kStatusBounds, 2);
+        if (p.evicted_pos) p.evicted_pos[inst] = -1;
+      }
+      step_done<kCaptured>(p.a.tpos, p.t);
+      return;
+    }
+    if (tid == 0 && p.evicted_pos) p.evicted_pos[inst] = vpos;
+    if (use_state) {                               // Eq. 4 / Eq. 5: psi acts on the key, the state is the KV head's
+      const float vv = __half2float(Vb[(size_t)slot * kHeadDim + d]);
+      const float* psv = p.a.psic + (inst * (size_t)N + slot) * R;
+#pragma unroll
+      for (int r = 0; r < R; ++r) Hb[r * kHeadDim + d] = fmaf(psv[r], vv, hcol[r]);
+      if (tid < R) zb[tid] += psv[tid];
+    }
+    __syncthreads();
+  } else {
+    if (tid == 0) {
+      p.a.count[inst] = n + 1;
+      if (p.evicted_pos) p.evicted_pos[inst] = -1;
+    }
+  }
+  __half* Kw = p.a.kslots + (inst * (size_t)N + slot) * kHeadDim;
+  __half* Vw = p.a.vslots + (inst * (size_t)N + slot) * kHeadDim;
+  if (rg == 0) *reinterpret_cast<uint4*>(Kw + l16 * 8) = knew;
+  if (rg == 1) *reinterpret_cast<uint4*>(Vw + l16 * 8) = vnew;
+  if (tid == 32) { posb[slot] = t_now; accb[slot] = p_new; }
+  if (tid >= 64 && tid < 64 + R)
+    p.a.psic[(inst * (size_t)N + slot) * R + (tid - 64)] =
+        use_state ? p.a.psi_k[inst * R + (tid - 64)] : 0.f;
+  step_done<kCaptured>(p.a.tpos, p.t);
+}
+
+size_t decode_smem_bytes(const Dims& d) {
+  return (size_t)d.G * (d.Np + 4 + DEC_RG * kHeadDim) * 4;
+}
+
+template <int R, int G>
+static void* decode_group_entry(bool captured) {
+  return captured ? (void*)decode_group_kernel<R, G, true> : (void*)decode_group_kernel<R, G, false>;
+}
+
 int launch_decode(less_ctx* c, const void* q, const void* k, const void* v, void* out,
                   int32_t* evicted_pos, cudaStream_t s) {
   const Dims& d = c->d;
@@ -371,10 +631,13 @@ int launch_decode(less_ctx* c, const void* q, const void* k, const void* v, void
   cudaStreamIsCapturing(s, &capturing);
   const bool captured = capturing == cudaStreamCaptureStatusActive;   // then the position is read from, and advanced in, device memory
   p.flags = d.flags;
-  const size_t smem = (size_t)(d.Np + 4 + DEC_RG * kHeadDim) * 4;
+  const size_t smem = decode_smem_bytes(d);
   LaunchScope scope(c, LESS_KERNEL_DECODE, s);
-  auto kern = d.R == 8 ? (captured ? decode_kernel<8, true> : decode_kernel<8, false>)
-                       : (captured ? decode_kernel<16, true> : decode_kernel<16, false>);
+  void* kern = d.R == 8 ? (captured ? (void*)decode_kernel<8, true> : (void*)decode_kernel<8, false>)
+                        : (captured ? (void*)decode_kernel<16, true> : (void*)decode_kernel<16, false>);
+  if (d.G == 2) kern = d.R == 8 ? decode_group_entry<8, 2>(captured) : decode_group_entry<16, 2>(captured);
+  if (d.G == 4) kern = d.R == 8 ? decode_group_entry<8, 4>(captured) : decode_group_entry<16, 4>(captured);
+  if (d.G == 8) kern = d.R == 8 ? decode_group_entry<8, 8>(captured) : decode_group_entry<16, 8>(captured);
   if (smem > 48 * 1024 &&
       cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
     return fail_cuda("shared memory opt-in of decode_kernel");
@@ -392,7 +655,8 @@ int launch_decode(less_ctx* c, const void* q, const void* k, const void* v, void
   const bool overlap = overlap_decode(c);
   cfg.attrs = attr;
   cfg.numAttrs = overlap ? 1 : 0;
-  if (cudaLaunchKernelEx(&cfg, kern, p) != cudaSuccess) return fail_cuda("launch of decode_kernel");
+  void* args[] = {&p};
+  if (cudaLaunchKernelExC(&cfg, kern, args) != cudaSuccess) return fail_cuda("launch of decode_kernel");
   return check_launch("decode_kernel");
 }
 

@@ -6,13 +6,14 @@
 namespace less {
 
 struct FmParams {
-  const __half* x[2];     // q, k                       [B, L, Hd, D]
+  const __half* x[2];     // q [B, L, Hh[0], D], k [B, L, Hh[1], D]
   const __half* w1[2];    // W_phi1, W_psi1             [L, Hd, D, Rp]
   const __half* w2[2];    // W_phi2, W_psi2             [L, Hd, Rp, R]
   const __half* w3;       // W_psi3                     [L, Hd, R, R]
   const float* psi_scale; // [L, Hd, 2] or null
-  float* out[2];          // phi_q, psi_k               [I, R]
+  float* out[2];          // phi_q [B, L, Hh[0], R], psi_k [B, L, Hh[1], R]
   int B, L, Hd, Rp;
+  int Hh[2];              // heads of each map per layer: query heads for phi (Hd * group), KV heads for psi
 };
 
 bool feature_gemv_supported(const Dims& d);

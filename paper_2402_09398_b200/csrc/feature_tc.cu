@@ -55,18 +55,21 @@ struct FtGeom {
   int npad;        // tokens per tile (GEMM1 N): 16, 32 or 64
   int ntile;       // token tiles per (layer-head, map)
   int items;       // work items
+  int items_phi;   // of which phi items (L * query heads * ntile)
   int nstage;      // ring stages
   uint32_t tmem_cols;
 };
 
 
-// Work item -> (token tile, map, layer-head)
+// Work item -> (token tile, map, layer-head of that map).  The phi items (one per query head)
+// come first, then the psi items (one per KV head).
 struct FtItem { int tile, which, lh; };
-__device__ __forceinline__ FtItem ft_item(int it, int ntile) {
+__device__ __forceinline__ FtItem ft_item(int it, const FtGeom& gm) {
   FtItem r;
-  r.tile = it % ntile;
-  r.which = (it / ntile) & 1;
-  r.lh = it / (2 * ntile);
+  r.which = it >= gm.items_phi;
+  const int rest = r.which ? it - gm.items_phi : it;
+  r.tile = rest % gm.ntile;
+  r.lh = rest / gm.ntile;
   return r;
 }
 
@@ -83,7 +86,7 @@ __device__ __forceinline__ void ft_produce(const CUtensorMap* tm_q, const CUtens
   uint32_t s = 0, sph = 0, a = 0, aph = 0;
   const uint64_t stream_policy = l2_evict_first_policy();
   for (int n = 0; n < my_items; ++n, (++a == (uint32_t)naux ? (a = 0, aph ^= 1) : 0u)) {
-    const FtItem im = ft_item(blockIdx.x + n * gridDim.x, gm.ntile);
+    const FtItem im = ft_item(blockIdx.x + n * gridDim.x, gm);
     wait_or_give_up(&aux_empty[a], aph ^ 1, abortp, status, 40);
     if (*abortp) return;                                 // issue nothing more once the CTA has given up
     const CUtensorMap* tx = im.which ? tm_k : tm_q;
@@ -234,7 +237,8 @@ __global__ void __launch_bounds__(FL_THREADS) feature_tc_kernel(
     uint32_t q = 0;
     for (int n = 0; n < my_items && !*abortp; ++n) {
       const int it = blockIdx.x + n * gridDim.x;
-      const int tile = it % gm.ntile, which = (it / gm.ntile) & 1, lh = it / (2 * gm.ntile);
+      const FtItem im = ft_item(it, gm);
+      const int tile = im.tile, which = im.which, lh = im.lh;
       const int a = n & 1;
       const int b0 = tile * npad, nb = min(npad, p.B - b0), nblk = (nb + 7) >> 3;
       float c1 = 1.f, c2 = 1.f;
@@ -327,7 +331,7 @@ __global__ void __launch_bounds__(FL_THREADS) feature_tc_kernel(
 #pragma unroll
           for (int r = 0; r < R; ++r) out[r] = fabsf(gv[r]);
         }
-        float4* dst = reinterpret_cast<float4*>(p.out[which] + ((size_t)(b0 + j) * p.L * p.Hd + lh) * R);
+        float4* dst = reinterpret_cast<float4*>(p.out[which] + ((size_t)(b0 + j) * p.L * p.Hh[which] + lh) * R);
 #pragma unroll
         for (int r4 = 0; r4 < R / 4; ++r4) dst[r4] = make_float4(out[r4 * 4], out[r4 * 4 + 1], out[r4 * 4 + 2], out[r4 * 4 + 3]);
       }
@@ -491,7 +495,8 @@ __global__ void __launch_bounds__(FT_THREADS) feature_tc_small_kernel(
     uint32_t a = 0, aph = 0;
     for (int n = 0; n < my_items; ++n, (++a == FS_AUX ? (a = 0, aph ^= 1) : 0u)) {
       const int it = blockIdx.x + n * gridDim.x;
-      const int tile = it % gm.ntile, which = (it / gm.ntile) & 1, lh = it / (2 * gm.ntile);
+      const FtItem im = ft_item(it, gm);
+      const int tile = im.tile, which = im.which, lh = im.lh;
       const int b0 = tile * FS_NPAD, nb = min(NT, p.B - b0);
       float c1 = 1.f, c2 = 1.f;
       if (which && p.psi_scale) { c1 = __ldg(p.psi_scale + lh * 2); c2 = __ldg(p.psi_scale + lh * 2 + 1); }
@@ -548,7 +553,7 @@ __global__ void __launch_bounds__(FT_THREADS) feature_tc_small_kernel(
           gv = sacc;
         }
       }
-      if (et < V && t < nb) p.out[which][((size_t)(b0 + t) * p.L * p.Hd + lh) * R + r] = fabsf(gv);
+      if (et < V && t < nb) p.out[which][((size_t)(b0 + t) * p.L * p.Hh[which] + lh) * R + r] = fabsf(gv);
       // this warp is done with the item's W2 and W3
       mbar_arrive_warp(&sh->aux_empty[a]);
     }
@@ -583,7 +588,8 @@ int launch_feature_tc(less_ctx* c, const FmParams& p, cudaStream_t s) {
   // token tiles of at most 64: larger tiles leave too little shared memory for the weight ring
   gm.npad = d.B <= 16 ? 16 : d.B <= 32 ? 32 : 64;
   gm.ntile = (d.B + gm.npad - 1) / gm.npad;
-  gm.items = d.L * d.Hd * 2 * gm.ntile;
+  gm.items_phi = d.L * p.Hh[0] * gm.ntile;
+  gm.items = gm.items_phi + d.L * p.Hh[1] * gm.ntile;
   const size_t fixed = ft_fixed_smem(d, gm.npad);
   int ns = (int)((FT_SMEM_LIMIT - fixed) / FT_STAGE_BYTES);
   gm.nstage = ns > FT_MAX_STAGES ? FT_MAX_STAGES : ns;
@@ -593,13 +599,13 @@ int launch_feature_tc(less_ctx* c, const FmParams& p, cudaStream_t s) {
   const size_t smem = fixed + (size_t)gm.nstage * FT_STAGE_BYTES;
 
   CUtensorMap tq, tk, tw1a, tw1b;
-  const uint64_t lh = (uint64_t)d.L * d.Hd;
+  const uint64_t lhq = (uint64_t)d.L * p.Hh[0], lhk = (uint64_t)d.L * p.Hh[1];   // layer-heads of phi / psi
   // q, k: [B rows][L*Hd*128 columns]; a box is npad batch rows x 64 columns of one head
-  if (!make_tmap_f16_2d(&tq, p.x[0], d.B, lh * kHeadDim, lh * kHeadDim * 2, gm.npad) ||
-      !make_tmap_f16_2d(&tk, p.x[1], d.B, lh * kHeadDim, lh * kHeadDim * 2, gm.npad))
+  if (!make_tmap_f16_2d(&tq, p.x[0], d.B, lhq * kHeadDim, lhq * kHeadDim * 2, gm.npad) ||
+      !make_tmap_f16_2d(&tk, p.x[1], d.B, lhk * kHeadDim, lhk * kHeadDim * 2, gm.npad))
     return fail_cuda("tensor map of q / k");
-  if (!make_tmap_f16_2d(&tw1a, p.w1[0], lh * kHeadDim, d.Rp, (uint64_t)d.Rp * 2, kHeadDim) ||
-      !make_tmap_f16_2d(&tw1b, p.w1[1], lh * kHeadDim, d.Rp, (uint64_t)d.Rp * 2, kHeadDim))
+  if (!make_tmap_f16_2d(&tw1a, p.w1[0], lhq * kHeadDim, d.Rp, (uint64_t)d.Rp * 2, kHeadDim) ||
+      !make_tmap_f16_2d(&tw1b, p.w1[1], lhk * kHeadDim, d.Rp, (uint64_t)d.Rp * 2, kHeadDim))
     return fail_cuda("tensor map of W1");
   int sms = 148;
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, c->device);
@@ -619,8 +625,8 @@ int launch_feature_tc(less_ctx* c, const FmParams& p, cudaStream_t s) {
     if (gm.nstage < 2) return LESS_ERR_INVALID_CONFIG;
     const size_t sm = fx + (size_t)gm.nstage * FT_STAGE_BYTES;
     // the small kernel loads 8 input rows per half tile
-    if (!make_tmap_f16_2d(&tq, p.x[0], d.B, lh * kHeadDim, lh * kHeadDim * 2, FS_XROWS) ||
-        !make_tmap_f16_2d(&tk, p.x[1], d.B, lh * kHeadDim, lh * kHeadDim * 2, FS_XROWS))
+    if (!make_tmap_f16_2d(&tq, p.x[0], d.B, lhq * kHeadDim, lhq * kHeadDim * 2, FS_XROWS) ||
+        !make_tmap_f16_2d(&tk, p.x[1], d.B, lhk * kHeadDim, lhk * kHeadDim * 2, FS_XROWS))
       return fail_cuda("tensor map of q / k");
     if (d.R == 8) {
       if (nt == 1) return launch_small<8, 1>(c, p, gm, tq, tk, tw1a, tw1b, sm, grid, s);

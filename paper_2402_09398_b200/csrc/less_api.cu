@@ -23,9 +23,16 @@ bool valid_config(const less_config* c) {
   if ((int64_t)c->heavy + c->recent > LESS_MAX_SLOTS) return false;   // the decode kernel keeps one score per slot in shared memory
   if (c->max_prompt < 0 || c->max_prompt > (1 << 20)) return false;
   if (c->max_prefill_layers < 1 || c->max_prefill_layers > c->layers) return false;
-  if ((int64_t)c->batch * c->heads * c->max_prefill_layers > 65535) return false;   // grid.y of the prompt kernels
+  if ((int64_t)c->batch * c->heads * c->max_prefill_layers * (c->group > 1 ? c->group : 1) > 65535)
+    return false;                                                                   // grid.y of the prompt kernels
   if (c->flags & ~(uint32_t)(LESS_SCORE_NORM_SPARSE | LESS_NO_STATE | LESS_POLICY_LAMBDA | LESS_POLICY_TOVA)) return false;
   if ((c->flags & LESS_POLICY_LAMBDA) && (c->flags & LESS_POLICY_TOVA)) return false;
+  if (c->group < 0 || c->group > 8 || (c->group & (c->group - 1))) return false;          // 0, 1, 2, 4, 8
+  if (c->group > 1 && (c->flags & LESS_POLICY_TOVA)) return false;                         // TOVA stays per head
+  // the decode kernel keeps one score per slot and query head in shared memory (227 KB per CTA)
+  if (c->group > 1 && (int64_t)c->group * ((((int64_t)c->heavy + c->recent + 3) & ~3) + 4 + 1024) * 4 > 227 * 1024)
+    return false;
+  if (c->group > 1 && c->hidden != 128 && c->hidden != 256 && c->hidden != 512) return false;   // tensor-core feature maps only
   int64_t inst = (int64_t)c->batch * c->layers * c->heads;
   if (inst > (1 << 24)) return false;
   return true;
@@ -44,6 +51,7 @@ Dims make_dims(const less_config* c) {
   d.N = c->heavy + c->recent;
   d.Np = (d.N + 3) & ~3;
   d.I = c->batch * c->layers * c->heads;
+  d.G = c->group > 1 ? c->group : 1;
   d.Sp = (c->max_prompt + 3) & ~3;
   d.Sbx = ((c->max_prompt + 255) & ~255) + 256;
   d.Lw = c->max_prefill_layers;
@@ -60,7 +68,7 @@ size_t carve(const Dims& d, char* base, Arena* a) {
     return p;
   };
   const size_t I = d.I, N = d.N, Np = d.Np, D = d.D, R = d.R;
-  const size_t Iw = (size_t)d.B * d.Hd * d.Lw, Sp = d.Sp;
+  const size_t Iw = (size_t)d.B * d.Hd * d.Lw, Sp = d.Sp, G = d.G;
   Arena t;
   t.kslots = (__half*)take(I * N * D * sizeof(__half));
   t.vslots = (__half*)take(I * N * D * sizeof(__half));
@@ -70,21 +78,21 @@ size_t carve(const Dims& d, char* base, Arena* a) {
   t.H = (float*)take(I * R * D * 4);
   t.z = (float*)take(I * R * 4);
   t.count = (int32_t*)take(I * 4);
-  t.phi_q = (float*)take(I * R * 4);
+  t.phi_q = (float*)take(I * G * R * 4);
   t.psi_k = (float*)take(I * R * 4);
   t.status = (int32_t*)take(4 * 4);
   t.tpos = (int32_t*)take(4 * 4);
-  t.stage_q = (__half*)take(I * D * 2);
+  t.stage_q = (__half*)take(I * G * D * 2);
   t.stage_k = (__half*)take(I * D * 2);
   t.stage_v = (__half*)take(I * D * 2);
-  t.stage_out = (float*)take(I * D * 4);
-  t.ws_m = (float*)take(Iw * Sp * 4);
-  t.ws_invl = (float*)take(Iw * Sp * 4);
+  t.stage_out = (float*)take(I * G * D * 4);
+  t.ws_m = (float*)take(Iw * G * Sp * 4);
+  t.ws_invl = (float*)take(Iw * G * Sp * 4);
   t.ws_acc = (float*)take(Iw * Sp * 4);
   t.ws_slot = (int32_t*)take(Iw * Sp * 4);
   t.ws_hpart = (float*)take(Iw * kMaxSplit * (R * D + R) * 4);
   t.ws_psi = (float*)take(Iw * Sp * R * 4);
-  t.ws_bx = (uint4*)take(Iw * (size_t)d.Sbx * 16);
+  t.ws_bx = (uint4*)take(Iw * G * (size_t)d.Sbx * 16);
   t.ws_pmax = (int32_t*)take(Iw * 4);
   if (a) *a = t;
   return off;
@@ -178,7 +186,7 @@ int less_create(const less_config* cfg, const less_weights* w, void* arena, size
   if (e == cudaSuccess) e = cudaMemset(c->a.count, 0, (size_t)d.I * 4);
   if (e == cudaSuccess) e = cudaMemset(c->a.status, 0, 16);
   if (e == cudaSuccess) e = cudaMemset(c->a.tpos, 0, 16);
-  if (e == cudaSuccess) e = cudaMemset(c->a.phi_q, 0, (size_t)d.I * d.R * 4);
+  if (e == cudaSuccess) e = cudaMemset(c->a.phi_q, 0, (size_t)d.I * d.G * d.R * 4);
   if (e == cudaSuccess) e = cudaMemset(c->a.psi_k, 0, (size_t)d.I * d.R * 4);
   if (e == cudaSuccess) e = cudaDeviceSynchronize();
   if (e != cudaSuccess) { delete c; return LESS_ERR_CUDA; }
@@ -206,7 +214,7 @@ int less_prefill(less_ctx* c, int32_t layer_begin, int32_t layer_count, int32_t 
   if (prompt_len > c->cfg.max_prompt) return LESS_ERR_PROMPT_TOO_LONG;
   if (prompt_len > 0) {
     // the tiled loads address prompt rows with 32-bit coordinates
-    if ((int64_t)c->d.B * layer_count * c->d.Hd * prompt_len > 0x7fffffffLL) return LESS_ERR_PROMPT_TOO_LONG;
+    if ((int64_t)c->d.B * layer_count * c->d.Hd * c->d.G * prompt_len > 0x7fffffffLL) return LESS_ERR_PROMPT_TOO_LONG;
     if (!Q || !K || !V) return LESS_ERR_NULL_POINTER;
     if (misaligned(Q) || misaligned(K) || misaligned(V) || misaligned(attn_out))
       return LESS_ERR_MISALIGNED;
@@ -252,14 +260,14 @@ int less_decode_step_host(less_ctx* c, const void* qh, const void* kh, const voi
                           void* stream) {
   if (!c || !qh || !kh || !vh || !outh) return LESS_ERR_NULL_POINTER;
   cudaStream_t s = (cudaStream_t)stream;
-  const size_t nin = (size_t)c->d.I * c->d.D * 2, nout = (size_t)c->d.I * c->d.D * 4;
+  const size_t nin = (size_t)c->d.I * c->d.D * 2, nq = nin * c->d.G, nout = (size_t)c->d.I * c->d.G * c->d.D * 4;
   // q and k feed the feature-map kernel's TMA loads and are staged in the arena.  v and the output
   // are touched once per instance by the decode kernel: from pinned host memory it reads / writes
   // them in place, which saves two copy launches per step.
   const void* v_dev = device_alias(vh);
   void* out_dev = device_alias(outh);
   if (((uintptr_t)v_dev & 15) || ((uintptr_t)out_dev & 15)) { v_dev = nullptr; out_dev = nullptr; }
-  cudaError_t e = cudaMemcpyAsync(c->a.stage_q, qh, nin, cudaMemcpyHostToDevice, s);
+  cudaError_t e = cudaMemcpyAsync(c->a.stage_q, qh, nq, cudaMemcpyHostToDevice, s);
   if (e == cudaSuccess) e = cudaMemcpyAsync(c->a.stage_k, kh, nin, cudaMemcpyHostToDevice, s);
   if (e == cudaSuccess && !v_dev) e = cudaMemcpyAsync(c->a.stage_v, vh, nin, cudaMemcpyHostToDevice, s);
   if (e != cudaSuccess) return LESS_ERR_CUDA;
@@ -370,7 +378,7 @@ int less_read_feature_maps(less_ctx* c, float* phi_host, float* psi_host, void* 
   cudaStream_t s = (cudaStream_t)stream;
   size_t bytes = (size_t)c->d.I * c->d.R * 4;
   cudaError_t e = cudaSuccess;
-  if (phi_host) e = cudaMemcpyAsync(phi_host, c->a.phi_q, bytes, cudaMemcpyDeviceToHost, s);
+  if (phi_host) e = cudaMemcpyAsync(phi_host, c->a.phi_q, bytes * c->d.G, cudaMemcpyDeviceToHost, s);
   if (e == cudaSuccess && psi_host)
     e = cudaMemcpyAsync(psi_host, c->a.psi_k, bytes, cudaMemcpyDeviceToHost, s);
   if (e == cudaSuccess) e = cudaStreamSynchronize(s);

@@ -26,29 +26,30 @@ struct Arena {
   float* H;          // [I][R][D]   Eq. 4
   float* z;          // [I][R]      Eq. 5
   int32_t* count;    // [I]         live slots
-  float* phi_q;      // [I][R]      phi(q_t) of the current step
+  float* phi_q;      // [I*G][R]    phi(q_t) of the current step, per query head
   float* psi_k;      // [I][R]      psi(k_t) of the current step
   int32_t* status;   // [4]         device status word(s)
   int32_t* tpos;     // [4]         [0] tokens seen = position of the next decode token, [1] decode CTAs finished this step
-  __half* stage_q;   // [I][D]      staging of host inputs (less_decode_step_host)
+  __half* stage_q;   // [I*G][D]    staging of host inputs (less_decode_step_host)
   __half* stage_k;   // [I][D]
   __half* stage_v;   // [I][D]
-  float* stage_out;  // [I][D]
+  float* stage_out;  // [I*G][D]
   // prompt-phase workspace, for Iw = B * H * max_prefill_layers instances
-  float* ws_m;       // [Iw][Sp]    row max of causal scores
-  float* ws_invl;    // [Iw][Sp]    1 / row sum
+  float* ws_m;       // [Iw*G][Sp]  row max of causal scores, per query head
+  float* ws_invl;    // [Iw*G][Sp]  1 / row sum
   float* ws_acc;     // [Iw][Sp]    column sums
   int32_t* ws_slot;  // [Iw][Sp]    slot of a prompt token, -1 = evicted
   float* ws_hpart;   // [Iw][kMaxSplit][R*D + R]  partial H, z per token split
   float* ws_psi;     // [Iw][Sp][R]  psi(k_j) of every prompt token
   int32_t* ws_pmax;  // [Iw]        bit pattern of max psi over the instance's prompt tokens (scales the state build's fp16 operand)
-  uint4* ws_bx;      // [Iw][Sbx]    per prompt row: -(m_i sqrt(D) - log2(1/l_i) / c) as three fp16 parts (column sums)
+  uint4* ws_bx;      // [Iw*G][Sbx]  per prompt row: -(m_i sqrt(D) - log2(1/l_i) / c) as three fp16 parts (column sums)
 };
 
 struct Dims {
   int32_t B, L, Hd, D, R, Rp;   // batch, layers, heads, head_dim, rank, hidden
   int32_t heavy, recent, N, Np; // slots; Np = N rounded up to a multiple of 4
-  int32_t I;                    // instances
+  int32_t I;                    // instances (one per KV head)
+  int32_t G;                    // query heads per KV head
   int32_t Sp;                   // max_prompt rounded up to a multiple of 4
   int32_t Sbx;                  // max_prompt rounded up to a multiple of 256 (+256)
   int32_t Lw;                   // max_prefill_layers

@@ -6,8 +6,9 @@
 namespace less {
 
 struct PfParams {
-  const __half* Q; const __half* K; const __half* V;   // [B, layer_count, Hd, S, D]
-  float* attn_out;                                      // same shape or null
+  const __half* Q;                                      // [B, layer_count, Hd * grp, S, D]
+  const __half* K; const __half* V;                     // [B, layer_count, Hd, S, D]
+  float* attn_out;                                      // Q's shape or null
   Arena a;
   const __half* w_psi1; const __half* w_psi2; const __half* w_psi3;
   const float* psi_scale;
@@ -16,6 +17,7 @@ struct PfParams {
   int lj0, layer_count;      // first input layer of this group, layers in the input
   int B, L, Hd, N, Np, heavy, recent, Rp;
   int nsplit, split_tokens;
+  int grp;                   // query heads per KV head (Section 3.2, multi-query attention)
   uint32_t flags;
 };
 
@@ -33,6 +35,24 @@ __device__ __forceinline__ InstMap map_instance(const PfParams& p, int g) {
   m.in_row0 = (((size_t)b * p.layer_count + p.lj0 + lj) * p.Hd + h) * (size_t)p.S;
   m.inst = ((size_t)b * p.L + p.layer0 + lj) * p.Hd + h;
   m.lh = (p.layer0 + lj) * p.Hd + h;
+  return m;
+}
+
+// A query head of the group: gq = instance-in-group * grp + head-in-group.  Its Q rows (and
+// attention-output rows), and the K / V rows of the KV head it reads.
+struct QueryMap {
+  size_t q_row0, kv_row0;
+};
+
+__device__ __forceinline__ QueryMap map_query(const PfParams& p, int gq) {
+  const int g = gq / p.grp, qg = gq - g * p.grp;
+  const int h = g % p.Hd;
+  const int lj = (g / p.Hd) % p.nl;
+  const int b = g / (p.Hd * p.nl);
+  const size_t bl = (size_t)b * p.layer_count + p.lj0 + lj;
+  QueryMap m;
+  m.q_row0 = ((bl * p.Hd + h) * p.grp + qg) * (size_t)p.S;
+  m.kv_row0 = (bl * p.Hd + h) * (size_t)p.S;
   return m;
 }
 

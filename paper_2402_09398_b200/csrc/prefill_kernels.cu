@@ -445,6 +445,9 @@ int launch_prefill_group(less_ctx* c, int layer0, int nl, int lj0, int layer_cou
   p.B = d.B; p.L = d.L; p.Hd = d.Hd; p.N = d.N; p.Np = d.Np;
   p.heavy = d.heavy; p.recent = d.recent; p.Rp = d.Rp;
   p.flags = d.flags;
+  p.grp = d.G;
+  // grouped query heads run on the tensor-core scoring kernels only
+  if (d.G > 1 && S > 0 && !(c->score_path == 1 && score_tc_supported())) return LESS_ERR_INVALID_CONFIG;
   // Token splits of the state build: whole 128-token tiles, long enough that the head's W1
   // (128 KB, reloaded per split) is amortised, short enough that the grid fills the GPU.
   const int G = d.B * nl * d.Hd;

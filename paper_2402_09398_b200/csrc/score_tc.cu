@@ -84,8 +84,8 @@ __global__ void __launch_bounds__(RS_THREADS) rowstat_tc_kernel(const __grid_con
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int tiles = (p.S + SC_TILE_M - 1) / SC_TILE_M;
   const int tile = tiles - 1 - (int)blockIdx.x;                  // long rows first
-  const int g = blockIdx.y;
-  const InstMap im = map_instance(p, g);
+  const int g = blockIdx.y;                                      // query head (KV instance * grp + head of the group)
+  const QueryMap qm = map_query(p, g);
   const int i0 = tile * SC_TILE_M;
   const int ncol = min(p.S, i0 + SC_TILE_M);                     // causal: columns [0, ncol)
   const int ntile = (ncol + SC_TILE_N - 1) / SC_TILE_N;
@@ -113,7 +113,7 @@ __global__ void __launch_bounds__(RS_THREADS) rowstat_tc_kernel(const __grid_con
 
   if (warp == 0) {
     if (lane == 0) {
-      const int row0 = (int)(im.in_row0 + i0);
+      const int row0 = (int)(qm.q_row0 + i0);
       mbar_expect_tx(&sh->res_full, SC_RES_BYTES);
       tma_load_2d(qres, &tm_q, 0, row0, &sh->res_full);
       tma_load_2d(qres + SC_RES_BYTES / 2, &tm_q, 64, row0, &sh->res_full);
@@ -121,7 +121,7 @@ __global__ void __launch_bounds__(RS_THREADS) rowstat_tc_kernel(const __grid_con
       for (int t = 0; t < ntile; ++t) {
         wait_or_give_up(&sh->empty[s], ph ^ 1, abortp, status, 80);
         if (*abortp) break;
-        const int krow = (int)(im.in_row0 + (size_t)t * SC_TILE_N);
+        const int krow = (int)(qm.kv_row0 + (size_t)t * SC_TILE_N);
         unsigned char* st = ring + s * SC_STAGE_BYTES;
         mbar_expect_tx(&sh->full[s], SC_STAGE_BYTES);
         tma_load_2d(st, &tm_k, 0, krow, &sh->full[s]);
@@ -245,7 +245,8 @@ __global__ void __launch_bounds__(CS_THREADS) colsum_tc_kernel(const __grid_cons
   const InstMap im = map_instance(p, g);
   const int j0 = tile * SC_TILE_M;
   const int t0 = j0 / SC_TILE_N;                                 // first Q tile: the one that holds row j0
-  const int ntile = (p.S + SC_TILE_N - 1) / SC_TILE_N - t0;
+  const int ntile = (p.S + SC_TILE_N - 1) / SC_TILE_N - t0;      // Q tiles of one query head
+  const int nstream = ntile * p.grp;                             // the heads of the group one after the other
   int32_t* status = p.a.status;
 
   if (tid == 0) {
@@ -284,17 +285,22 @@ __global__ void __launch_bounds__(CS_THREADS) colsum_tc_kernel(const __grid_cons
       tma_load_2d(kres, &tm_k, 0, row0, &sh->res_full);
       tma_load_2d(kres + SC_RES_BYTES / 2, &tm_k, 64, row0, &sh->res_full);
       uint32_t s = 0, ph = 0;
-      for (int t = 0; t < ntile; ++t) {
-        wait_or_give_up(&sh->empty[s], ph ^ 1, abortp, status, 85);
+      for (int qg = 0; qg < p.grp; ++qg) {
+        const int gq = g * p.grp + qg;
+        const size_t q_row0 = map_query(p, gq).q_row0;
+        for (int t = 0; t < ntile; ++t) {
+          wait_or_give_up(&sh->empty[s], ph ^ 1, abortp, status, 85);
+          if (*abortp) break;
+          const int qrow = (int)(q_row0 + (size_t)(t0 + t) * SC_TILE_N);
+          unsigned char* st = ring + s * SC_STAGE_BYTES;
+          mbar_expect_tx(&sh->full[s], SC_STAGE_BYTES + SC_BX_BYTES);
+          tma_load_2d(st, &tm_q, 0, qrow, &sh->full[s]);
+          tma_load_2d(st + SC_STAGE_BYTES / 2, &tm_q, 64, qrow, &sh->full[s]);
+          bulk_g2s(bx + s * SC_BX_BYTES, p.a.ws_bx + (size_t)gq * p.Sbx + (size_t)(t0 + t) * SC_TILE_N, SC_BX_BYTES,
+                   &sh->full[s]);
+          if (++s == SC_STAGES) { s = 0; ph ^= 1; }
+        }
         if (*abortp) break;
-        const int qrow = (int)(im.in_row0 + (size_t)(t0 + t) * SC_TILE_N);
-        unsigned char* st = ring + s * SC_STAGE_BYTES;
-        mbar_expect_tx(&sh->full[s], SC_STAGE_BYTES + SC_BX_BYTES);
-        tma_load_2d(st, &tm_q, 0, qrow, &sh->full[s]);
-        tma_load_2d(st + SC_STAGE_BYTES / 2, &tm_q, 64, qrow, &sh->full[s]);
-        bulk_g2s(bx + s * SC_BX_BYTES, p.a.ws_bx + (size_t)g * p.Sbx + (size_t)(t0 + t) * SC_TILE_N, SC_BX_BYTES,
-                 &sh->full[s]);
-        if (++s == SC_STAGES) { s = 0; ph ^= 1; }
       }
     }
   } else if (warp == 1) {
@@ -306,7 +312,7 @@ __global__ void __launch_bounds__(CS_THREADS) colsum_tc_kernel(const __grid_cons
       const uint64_t bd_bx = smem_desc(smem_u32(bx), SC_STAGES * SC_BX_BYTES, 128, kLayoutNone);
       wait_or_give_up(&sh->res_full, 0, abortp, status, 86);
       uint32_t s = 0, ph = 0, b = 0, bph = 0;
-      for (int t = 0; t < ntile; ++t) {
+      for (int t = 0; t < nstream; ++t) {
         wait_or_give_up(&sh->full[s], ph, abortp, status, 87);
         wait_or_give_up(&sh->d_free[b], bph ^ 1, abortp, status, 89);
         if (*abortp) break;
@@ -330,7 +336,7 @@ __global__ void __launch_bounds__(CS_THREADS) colsum_tc_kernel(const __grid_cons
     const uint32_t lane_addr = tmem + ((uint32_t)(quad * 32) << 16) + half * (SC_TILE_N / 2);
     float acc = 0.f;
     uint32_t b = 0, bph = 0;
-    for (int t = 0; t < ntile; ++t) {
+    for (int ts = 0, t = 0; ts < nstream; ++ts, t = (t + 1 == ntile ? 0 : t + 1)) {   // t: tile within the head
       wait_or_give_up(&sh->d_full[b], bph, abortp, status, 91);
       tc_fence_after_sync();
       const int c0 = (t0 + t) * SC_TILE_N + half * (SC_TILE_N / 2);
@@ -372,12 +378,12 @@ bool score_tc_supported() { return encode_tiled_fn() != nullptr; }
 int launch_score_tc(less_ctx* c, const PfParams& p, int G, cudaStream_t s, bool with_column_sums) {
   const Dims& d = c->d;
   CUtensorMap tq, tk;
-  const uint64_t rows = (uint64_t)d.B * p.layer_count * d.Hd * p.S;
-  if (!make_tmap_f16_2d(&tq, p.Q, rows, kHeadDim, kHeadDim * 2, SC_TILE_N) ||
+  const uint64_t rows = (uint64_t)d.B * p.layer_count * d.Hd * p.S, qrows = rows * p.grp;
+  if (!make_tmap_f16_2d(&tq, p.Q, qrows, kHeadDim, kHeadDim * 2, SC_TILE_N) ||
       !make_tmap_f16_2d(&tk, p.K, rows, kHeadDim, kHeadDim * 2, SC_TILE_N))
     return fail_cuda("tensor maps of Q / K");
   CUtensorMap tq_res, tk_res;
-  if (!make_tmap_f16_2d(&tq_res, p.Q, rows, kHeadDim, kHeadDim * 2, SC_TILE_M) ||
+  if (!make_tmap_f16_2d(&tq_res, p.Q, qrows, kHeadDim, kHeadDim * 2, SC_TILE_M) ||
       !make_tmap_f16_2d(&tk_res, p.K, rows, kHeadDim, kHeadDim * 2, SC_TILE_M))
     return fail_cuda("tensor maps of Q / K");
   const int tiles = (p.S + SC_TILE_M - 1) / SC_TILE_M;
@@ -388,7 +394,7 @@ int launch_score_tc(less_ctx* c, const PfParams& p, int G, cudaStream_t s, bool 
     return fail_cuda("shared memory opt-in of the scoring kernels");
   {
     LaunchScope scope(c, LESS_KERNEL_ROWSTAT, s);
-    rowstat_tc_kernel<<<dim3(tiles, G), RS_THREADS, smem1, s>>>(tq_res, tk, p);
+    rowstat_tc_kernel<<<dim3(tiles, G * p.grp), RS_THREADS, smem1, s>>>(tq_res, tk, p);   // one row of CTAs per query head
   }
   if (with_column_sums) {
     LaunchScope scope(c, LESS_KERNEL_COLSUM, s);

@@ -37,6 +37,7 @@ class Workload:
     sink_prefix: int = 0          # first tokens whose keys are scaled too
     key_boost: float = 4.0
     weight_std: float = 0.02
+    group: int = 1                # query heads per KV head (`heads` counts KV heads)
 
     @property
     def instances(self) -> int:
@@ -82,9 +83,11 @@ def _randn_half(shape, g, device, std: float = 1.0) -> torch.Tensor:
 
 def make_weights(w: Workload, device="cpu") -> Dict[str, torch.Tensor]:
     """Per-head feature-map weights, fp16, row-major:
-    w_phi1/w_psi1 [L,H,D,R'], w_phi2/w_psi2 [L,H,R',R], w_psi3 [L,H,R,R]."""
+    w_phi1/w_psi1 [L,H,D,R'], w_phi2/w_psi2 [L,H,R',R], w_psi3 [L,H,R,R]; with grouped
+    query heads the phi weights have one set per query head: [L, H*group, ...]."""
     L, H, D, Rp, R = w.layers, w.heads, w.head_dim, w.hidden, w.rank
-    shapes = {"w_phi1": (L, H, D, Rp), "w_phi2": (L, H, Rp, R),
+    Hq = H * w.group
+    shapes = {"w_phi1": (L, Hq, D, Rp), "w_phi2": (L, Hq, Rp, R),
               "w_psi1": (L, H, D, Rp), "w_psi2": (L, H, Rp, R), "w_psi3": (L, H, R, R)}
     out = {}
     for i, (name, shape) in enumerate(shapes.items()):
@@ -112,16 +115,18 @@ def _boost_mask(w: Workload, shape_prefix: Tuple[int, ...], positions: torch.Ten
 def make_prompt(w: Workload, layer_begin: int, layer_count: int, device="cpu",
                 prompt: Optional[int] = None):
     """Prompt Q, K, V, fp16 [B, layer_count, H, S, D], generated layer by layer
-    so that a layer's bits do not depend on how the layers are grouped."""
+    so that a layer's bits do not depend on how the layers are grouped.  With grouped query
+    heads Q is [B, layer_count, H*group, S, D]."""
     S = w.prompt if prompt is None else prompt
     B, H, D = w.batch, w.heads, w.head_dim
-    Q = torch.empty((B, layer_count, H, S, D), dtype=torch.float16, device=device)
-    K = torch.empty_like(Q)
-    V = torch.empty_like(Q)
+    Hq = H * w.group
+    Q = torch.empty((B, layer_count, Hq, S, D), dtype=torch.float16, device=device)
+    K = torch.empty((B, layer_count, H, S, D), dtype=torch.float16, device=device)
+    V = torch.empty_like(K)
     positions = torch.arange(S, device=device)
     for j in range(layer_count):
         layer = layer_begin + j
-        Q[:, j] = _randn_half((B, H, S, D), _gen(device, w.cfg_id, _Q, layer), device)
+        Q[:, j] = _randn_half((B, Hq, S, D), _gen(device, w.cfg_id, _Q, layer), device)
         k = torch.randn((B, H, S, D), generator=_gen(device, w.cfg_id, _K, layer),
                         device=device, dtype=torch.float32)
         m = _boost_mask(w, (B, H), positions, _gen(device, w.cfg_id, _MASK, layer), device)
@@ -132,10 +137,12 @@ def make_prompt(w: Workload, layer_begin: int, layer_count: int, device="cpu",
 
 
 def make_decode_inputs(w: Workload, step: int, device="cpu", prompt: Optional[int] = None):
-    """q, k, v of decode step `step` (absolute position prompt+step), fp16 [B,L,H,D]."""
+    """q, k, v of decode step `step` (absolute position prompt+step), fp16 [B,L,H,D]
+    (q [B,L,H*group,D] with grouped query heads)."""
     S = w.prompt if prompt is None else prompt
     shape = (w.batch, w.layers, w.heads, w.head_dim)
-    q = _randn_half(shape, _gen(device, w.cfg_id, _DQ, step), device)
+    q = _randn_half((w.batch, w.layers, w.heads * w.group, w.head_dim),
+                    _gen(device, w.cfg_id, _DQ, step), device)
     k = torch.randn(shape, generator=_gen(device, w.cfg_id, _DK, step), device=device,
                     dtype=torch.float32)
     pos = torch.tensor([S + step], device=device)

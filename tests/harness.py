@@ -201,3 +201,140 @@ def brute_force_state(w, W, inst, K_hist, V_hist, evicted_positions, psi_scale=N
         return np.zeros((w.rank, w.head_dim)), np.zeros(w.rank)
     psi = orc.psi_fn(K_hist[ev])
     return psi.T @ V_hist[ev], psi.sum(axis=0)
+
+
+# --------------------------------------------------------------------------- #
+# grouped query heads over one KV head (Section 3.2, multi-query attention)
+# --------------------------------------------------------------------------- #
+def make_group_oracle(w, W, inst, flags=0, psi_scale=None):
+    b, layer, head = wl.instance_coords(w, inst)
+    G = w.group
+    sc = None if psi_scale is None else psi_scale[layer, head].double().cpu().numpy()
+    psi_w = [W[n][layer, head].double().cpu().numpy() for n in ("w_psi1", "w_psi2", "w_psi3")]
+    phi_fns = []
+    for g in range(G):
+        w1, w2 = (W[n][layer, head * G + g].double().cpu().numpy() for n in ("w_phi1", "w_phi2"))
+        phi_fns.append(lo.make_mlp_maps(w1, w2, *psi_w, sc)[0])
+    psi_fn = lo.make_mlp_maps(W["w_phi1"][layer, head * G].double().cpu().numpy(),
+                              W["w_phi2"][layer, head * G].double().cpu().numpy(), *psi_w, sc)[1]
+    return lo.LessGroup(w.head_dim, w.rank, w.heavy, w.recent, phi_fns, psi_fn,
+                        score_norm="sparse" if flags & 1 else "less", use_state=not (flags & 2),
+                        policy="lambda" if flags & 4 else "h2o")
+
+
+def check_prefill_group(ctx, w, W, Q, K, V, instances, attn_out=None, flags=0, psi_scale=None, layer_begin=0):
+    """Grouped version of check_prefill: Q [B, Lc, H*G, S, D], K, V [B, Lc, H, S, D];
+    attn_out [B, Lc, H*G, S, D]."""
+    recs = ctx.export_state(instances)
+    S, G = Q.shape[3], w.group
+    exempt = 0
+    worst = {"out": 0.0, "H": 0.0, "z": 0.0, "acc": 0.0}
+    for inst, rec in zip(instances, recs):
+        b, layer, head = wl.instance_coords(w, inst)
+        lj = layer - layer_begin
+        q = Q[b, lj, head * G:(head + 1) * G].double().cpu().numpy()
+        k, v = (t[b, lj, head].double().cpu().numpy() for t in (K, V))
+        orc = make_group_oracle(w, W, inst, flags, psi_scale)
+        out = orc.prefill(q, k, v)
+        assert rec["t"] == S and rec["count"] == min(S, orc.N), (inst, rec["count"])
+        if attn_out is not None and S:
+            err = float(np.max(np.abs(attn_out[b, lj, head * G:(head + 1) * G].double().cpu().numpy() - out)))
+            worst["out"] = max(worst["out"], err)
+            assert err <= OUT_TOL, f"inst {inst}: prompt attention max-abs {err}"
+        gpu_pos = rec["pos"].astype(np.int64)
+        assert np.all(np.diff(gpu_pos) > 0), "prefill slots must ascend in position"
+        kept_o, kept_g = set(orc.pos.tolist()), set(gpu_pos.tolist())
+        if kept_o != kept_g:
+            acc_o = orc.prompt_acc
+            cand = np.arange(S - orc.recent)
+            thr = np.sort(acc_o[cand])[::-1][orc.heavy - 1] if orc.heavy > 0 else np.inf
+            diff = kept_o ^ kept_g
+            for pz in diff:
+                assert pz < S - orc.recent, f"inst {inst}: recent token {pz} mis-kept"
+                assert abs(acc_o[pz] - thr) <= TIE_BAND * abs(thr), f"inst {inst}: pos {pz}"
+            exempt += len(diff)
+            assert len(kept_g) == len(kept_o)
+        Kh, Vh = K[b, lj, head].cpu().numpy(), V[b, lj, head].cpu().numpy()
+        assert np.array_equal(rec["K"], Kh[gpu_pos]) and np.array_equal(rec["V"], Vh[gpu_pos])
+        acc_ref = orc.prompt_acc[gpu_pos]
+        aerr = np.max(np.abs(rec["acc"] - acc_ref) / (np.abs(acc_ref) + 1e-30)) if len(gpu_pos) else 0.0
+        worst["acc"] = max(worst["acc"], float(aerr))
+        assert np.allclose(rec["acc"], acc_ref, rtol=1e-4, atol=1e-6), f"inst {inst}: acc rel {aerr}"
+        if kept_o == kept_g and not (flags & 2):
+            eH, ez = rel_err(rec["H"], orc.H), rel_err(rec["z"], orc.z)
+            worst["H"], worst["z"] = max(worst["H"], eH), max(worst["z"], ez)
+            assert eH <= REL_TOL and ez <= REL_TOL, f"inst {inst}: H rel {eH}, z rel {ez}"
+    return {"exempt": exempt, **worst}
+
+
+class GroupTeacherForced:
+    """TeacherForced for G query heads per KV head: every step of the library is checked
+    against one LessGroup step started from the library's own pre-step state."""
+
+    def __init__(self, ctx, w, W, instances, flags=0, psi_scale=None):
+        self.ctx, self.w, self.instances, self.flags = ctx, w, list(instances), flags
+        self.oracles = [make_group_oracle(w, W, i, flags, psi_scale) for i in instances]
+        self.exempt = 0
+        self.evictions = 0
+        self.worst = {"out": 0.0, "dH": 0.0, "dz": 0.0, "acc": 0.0, "phi": 0.0, "psi": 0.0}
+        self.evicted = torch.empty(ctx.instances, dtype=torch.int32, device=ctx.device)
+
+    def step(self, q, k, v):
+        ctx, w, G, D = self.ctx, self.w, self.w.group, self.w.head_dim
+        pre = ctx.export_state(self.instances)
+        out = ctx.decode_step(q, k, v, evicted_pos=self.evicted)
+        post = ctx.export_state(self.instances)
+        ev = self.evicted.cpu().numpy()
+        out_h = out.reshape(-1, G, D).cpu().numpy()
+        phi_g, psi_g = ctx.read_feature_maps()
+        phi_g = phi_g.reshape(-1, G, w.rank)
+        qh = q.reshape(-1, G, D).cpu().numpy().astype(np.float64)
+        kh = k.reshape(-1, D).cpu().numpy().astype(np.float64)
+        vh = v.reshape(-1, D).cpu().numpy().astype(np.float64)
+        use_state = not (self.flags & 2)
+        for inst, orc, a, b in zip(self.instances, self.oracles, pre, post):
+            orc.import_state(a["pos"], a["K"], a["V"], a["acc"], a["H"], a["z"], a["t"])
+            r = orc.decode(qh[inst], kh[inst], vh[inst])
+            err = float(np.max(np.abs(out_h[inst] - r["out"])))
+            self.worst["out"] = max(self.worst["out"], err)
+            assert err <= OUT_TOL, f"inst {inst} t={a['t']}: out max-abs {err}"
+            if use_state:
+                for g in range(G):
+                    e1 = rel_err(phi_g[inst, g], orc.phi_fns[g](qh[inst, g][None])[0])
+                    self.worst["phi"] = max(self.worst["phi"], e1)
+                    assert e1 <= REL_TOL, f"inst {inst} head {g}: phi rel {e1}"
+                e2 = rel_err(psi_g[inst], orc.psi_fn(kh[inst][None])[0])
+                self.worst["psi"] = max(self.worst["psi"], e2)
+                assert e2 <= REL_TOL, f"inst {inst}: psi rel {e2}"
+            gpu_vic = int(ev[inst])
+            exempt = False
+            if gpu_vic != r["evicted_pos"]:
+                assert r["tie_gap"] is not None and r["tie_gap"] < TIE_BAND, \
+                    f"inst {inst} t={a['t']}: evicted {gpu_vic}, oracle {r['evicted_pos']}, gap {r['tie_gap']}"
+                self.exempt += 1
+                exempt = True
+            if gpu_vic >= 0:
+                self.evictions += 1
+            assert b["t"] == a["t"] + 1
+            gpos = b["pos"].astype(np.int64)
+            assert len(set(gpos.tolist())) == len(gpos)
+            if not exempt:
+                assert set(gpos.tolist()) == set(orc.pos.tolist()), f"inst {inst}: kept sets differ"
+                order_g, order_o = np.argsort(gpos), np.argsort(orc.pos)
+                assert np.array_equal(b["K"][order_g].astype(np.float64), orc.K[order_o])
+                assert np.array_equal(b["V"][order_g].astype(np.float64), orc.V[order_o])
+                acc_g, acc_o = b["acc"][order_g], orc.acc[order_o]
+                aerr = float(np.max(np.abs(acc_g - acc_o) / (np.abs(acc_o) + 1e-30)))
+                self.worst["acc"] = max(self.worst["acc"], aerr)
+                assert np.allclose(acc_g, acc_o, rtol=ACC_RTOL, atol=ACC_ATOL), f"inst {inst}: acc rel {aerr}"
+                if use_state and r["dH"] is not None:
+                    dH_g = b["H"].astype(np.float64) - a["H"].astype(np.float64)
+                    dz_g = b["z"].astype(np.float64) - a["z"].astype(np.float64)
+                    slack_H = 2e-7 * np.linalg.norm(a["H"]) / max(np.linalg.norm(r["dH"]), 1e-300)
+                    slack_z = 2e-7 * np.linalg.norm(a["z"]) / max(np.linalg.norm(r["dz"]), 1e-300)
+                    eH, ez = rel_err(dH_g, r["dH"]), rel_err(dz_g, r["dz"])
+                    self.worst["dH"], self.worst["dz"] = max(self.worst["dH"], eH), max(self.worst["dz"], ez)
+                    assert eH <= REL_TOL + slack_H and ez <= REL_TOL + slack_z, f"inst {inst}: dH {eH} dz {ez}"
+                elif use_state:
+                    assert np.array_equal(a["H"], b["H"]) and np.array_equal(a["z"], b["z"])
+        return out

@@ -417,3 +417,25 @@ def test_captured_step_replays_like_direct_calls(batch):
         for key in ("pos", "acc", "K", "V", "psi", "H", "z"):
             assert np.array_equal(a[key], b[key]), key
     ctx_d.close(); ctx_g.close()
+
+
+@pytest.mark.parametrize("group,rank,flags", [(2, 8, 0), (4, 16, 0), (8, 8, 0), (4, 8, 4), (2, 16, 1), (4, 8, 2)])
+def test_grouped_query_heads_decode_from_empty(group, rank, flags):
+    """Section 3.2, multi-query attention: G query heads share one KV head's cache, scores and
+    state; every step is checked against the grouped oracle (outputs of all G heads, per-head phi,
+    aggregated H2O scores, the one eviction, Eq. 4 / Eq. 5)."""
+    import harness
+    w = small(60 + group, prompt=0, steps=30, heavy=9, recent=8, rank=rank, weight_std=0.1, group=group)
+    ctx, W = _setup(w, flags=flags, max_prompt=16)
+    inst = list(range(w.instances))
+    tf = harness.GroupTeacherForced(ctx, w, W, inst, flags)
+    for s in range(w.steps):
+        q, k, v = wl.make_decode_inputs(w, s, DEV)
+        assert q.shape[2] == w.heads * group
+        out = tf.step(q, k, v)
+        assert out.shape == q.shape
+    assert tf.evictions == (w.steps - w.slots) * w.instances
+    assert tf.exempt <= 2
+    assert ctx.poll_status() == 0
+    print("grouped decode", group, tf.worst)
+    ctx.close()
