@@ -61,6 +61,9 @@ def parse_args():
                     help="context run: TOVA as the sparse policy (same slot count)")
     ap.add_argument("--attn-out", action="store_true",
                     help="prompt compression: also produce the prompt's attention output (optional in less_prefill)")
+    ap.add_argument("--group", type=int, default=1, choices=[1, 2, 4, 8],
+                    help="context run: grouped query heads, G query heads per KV head (query heads unchanged, "
+                         "KV heads divided by G)")
     ap.add_argument("--batch", type=int, default=0,
                     help="override the workload's batch (smaller captures for ncu; named in config.workload)")
     return ap.parse_args()
@@ -80,23 +83,23 @@ def peaks():
 def feature_map_bytes(w, no_state=False):
     if no_state:
         return 0
-    D, Rp, R = w.head_dim, w.hidden, w.rank
-    weights = w.layers * w.heads * (2 * (D * Rp + Rp * R) + R * R) * 2
-    io = w.instances * (2 * D * 2 + 2 * R * 4)
+    D, Rp, R, G = w.head_dim, w.hidden, w.rank, w.group
+    weights = w.layers * w.heads * ((G + 1) * (D * Rp + Rp * R) + R * R) * 2    # phi per query head, psi per KV head
+    io = w.instances * ((G + 1) * D * 2 + (G + 1) * R * 4)
     return weights + io
 
 
 def decode_bytes(w, n_live, evicting=True, no_state=False):
-    D, R = w.head_dim, w.rank
+    D, R, G = w.head_dim, w.rank, w.group
     per = n_live * (2 * D * 2)              # K and V rows
     per += n_live * (4 + 4)                 # accumulated score read + write
     per += n_live * 4 if evicting else 0    # positions (only read when a victim is needed)
-    per += 3 * D * 2 + D * 4                # q, k, v in; out
+    per += (2 + G) * D * 2 + G * D * 4      # q, k, v in; out (G query heads per KV head)
     per += 2 * D * 2 + 8                    # new pair into its slot, pos, acc
     per += 4                                # slot count
     if not no_state:
         per += R * D * 4 + R * 4            # H, z read
-        per += 2 * R * 4                    # phi(q), psi(k) read
+        per += (G + 1) * R * 4              # phi(q) of the G heads, psi(k) read
         per += R * 4                        # psi into the slot's cache
         if evicting:
             per += R * D * 4 + R * 4 + R * 4 + D * 2   # H, z write; victim psi; victim v row
@@ -263,6 +266,9 @@ def workload_config(w, args):
         c["variant"] = "Lambda-masking policy (first 4 tokens + recent window)"
     if getattr(args, "no_state", False):
         c["variant"] = "sparse policy alone (Baseline+)"
+    if getattr(args, "group", 1) > 1:
+        c["variant"] = (f"grouped query heads: {w.heads} KV heads x {w.group} query heads per layer; "
+                        "the unit counts query heads")
     return c
 
 
@@ -288,6 +294,11 @@ def run_b200(args):
     w = wl.CONFIGS[args.config]
     if args.batch:
         w = w.with_(batch=args.batch)
+    if args.group > 1:
+        if args.tova or w.heads % args.group:
+            raise SystemExit("--group needs a head count it divides and is not defined for --tova")
+        w = w.with_(heads=w.heads // args.group, group=args.group)
+        args.no_cpu_baseline = True      # context run; the timed oracle leg covers the default workload
     K_steps, W_steps = args.steps, args.warmup
     total_steps = K_steps * 3 + W_steps + 2
     heavy, recent, flags = w.heavy, w.recent, 0
@@ -306,7 +317,7 @@ def run_b200(args):
 
     # replicas: every rank runs the whole workload on its own GPU, no collective in the path
     Wt = wl.make_weights(w, dev)
-    layers_per_call = max(1, min(w.layers, (1 << 30) // max(1, w.batch * w.heads * w.prompt * w.head_dim * 2)))
+    layers_per_call = max(1, min(w.layers, (1 << 30) // max(1, w.batch * w.heads * w.group * w.prompt * w.head_dim * 2)))
     ctx = binding.from_workload(w_run, Wt, dev, max_prefill_layers=layers_per_call, flags=flags)
     t_pre0 = time.perf_counter()
     for l0 in range(0, w.layers, layers_per_call):
@@ -321,7 +332,7 @@ def run_b200(args):
     inputs = [wl.make_decode_inputs(w, s % max(1, w.steps), dev) if s < 8 else None for s in range(total_steps)]
     base = [i for i in inputs if i is not None]
     inputs = [base[s % len(base)] for s in range(total_steps)]
-    out = torch.empty(w.batch, w.layers, w.heads, w.head_dim, dtype=torch.float32, device=dev)
+    out = torch.empty(w.batch, w.layers, w.heads * w.group, w.head_dim, dtype=torch.float32, device=dev)
     stream = torch.cuda.current_stream()
     step_no = [0]
 
@@ -384,7 +395,7 @@ def run_b200(args):
     ctx.profile(False)
 
     # ---- end to end through the host-buffer entry point ----
-    hq, hk, hv = (torch.empty(inputs[0][0].shape, dtype=torch.float16).pin_memory() for _ in range(3))
+    hq, hk, hv = (torch.empty(inputs[0][i].shape, dtype=torch.float16).pin_memory() for i in range(3))
     hq.copy_(inputs[0][0]); hk.copy_(inputs[0][1]); hv.copy_(inputs[0][2])
     hout = torch.empty(out.shape, dtype=torch.float32).pin_memory()
     for _ in range(3):
@@ -405,8 +416,8 @@ def run_b200(args):
     ms, ms_e2e = max_over_ranks([ms, ms_e2e], dev, world)
 
     if rank == 0:
-        value = job_throughput(w.instances, K_steps, ms, world)
-        e2e_value = job_throughput(w.instances, K_steps, ms_e2e, world)
+        value = job_throughput(w.instances * w.group, K_steps, ms, world)
+        e2e_value = job_throughput(w.instances * w.group, K_steps, ms_e2e, world)
         peak, peak_kind = peaks()
         n_live = min(w_run.slots, w.prompt + W_steps)
         evicting = not args.full_cache
@@ -417,7 +428,8 @@ def run_b200(args):
         kernel_names = {"feature_map": ("feature_tc_small_kernel" if w.batch <= 8 else "feature_tc_kernel")
                         + f"<{w.rank}" + (f", {1 if w.batch <= 1 else 2 if w.batch <= 2 else 4 if w.batch <= 4 else 8}>"
                                           if w.batch <= 8 else ">"),
-                        "decode": f"decode_kernel<{w.rank}, {1 if args.graph else 0}>"}
+                        "decode": (f"decode_kernel<{w.rank}, {1 if args.graph else 0}>" if w.group == 1 else
+                                   f"decode_group_kernel<{w.rank}, {w.group}, {1 if args.graph else 0}>")}
         ach = kb[dominant] / (kt[dominant] * 1e-3) / 1e9 if kt[dominant] > 0 else 0.0
         step_bytes = kb["feature_map"] + kb["decode"]
         kv_state_bytes = w.instances * (n_live * (4 * w.head_dim + 8) + (0 if args.no_state else 2 * w.rank * w.head_dim * 4))
@@ -428,8 +440,8 @@ def run_b200(args):
             "config": workload_config(w, args),
             "clocks": clocks,
             "e2e": {"value": e2e_value, "unit": UNIT,
-                    "h2d_bytes_per_step": 3 * w.instances * w.head_dim * 2,
-                    "d2h_bytes_per_step": w.instances * w.head_dim * 4},
+                    "h2d_bytes_per_step": (2 + w.group) * w.instances * w.head_dim * 2,
+                    "d2h_bytes_per_step": w.group * w.instances * w.head_dim * 4},
             "gpu_launches": int(launches),
             "roofline": {"bound": "hbm", "kernel": kernel_names[dominant], "achieved": ach, "peak": peak,
                          "unit": "GB/s", "frac": ach / peak, "peak_kind": f"of {peak_kind}",
@@ -466,7 +478,8 @@ def prefill_flops(w):
     inst = w.batch * w.heads
     S, D, Rp, R = w.prompt, w.head_dim, w.hidden, w.rank
     causal = S * (S + 1) // 2
-    return {"rowstat": inst * causal * 2 * D, "colsum": inst * causal * 2 * D, "attn_out": inst * causal * 4 * D,
+    qh = inst * w.group                    # the scoring kernels work per query head
+    return {"rowstat": qh * causal * 2 * D, "colsum": qh * causal * 2 * D, "attn_out": qh * causal * 4 * D,
             "psi": inst * S * 2 * (D * Rp + Rp * R + R * R), "build": inst * S * 2 * R * D}
 
 
@@ -487,6 +500,8 @@ def run_prefill(args):
     w = wl.CONFIGS[args.config]
     if args.batch:
         w = w.with_(batch=args.batch)
+    if args.group > 1:
+        w = w.with_(heads=w.heads // args.group, group=args.group)
     K_steps, W_steps = args.steps, max(args.warmup, 3)
     Wt = wl.make_weights(w, dev)
     ctx = binding.from_workload(w, Wt, dev, max_prefill_layers=1)
@@ -512,11 +527,12 @@ def run_prefill(args):
     launches0 = ctx.launches
     t0 = time.time()
     e0.record(stream)
-    run_steps(K_steps)
+    for _ in range(K_steps):
+        one_step()
     e1.record(stream)
     barrier()
     t1 = time.time()
-    launches = (ctx.launches - launches0) if not args.graph else 2 * K_steps
+    launches = ctx.launches - launches0
     ms = e0.elapsed_time(e1)
     clocks = sampler.stop(t0, t1) if sampler else None
     ctx.profile(True)
@@ -526,7 +542,7 @@ def run_prefill(args):
     prof = ctx.profile_read()
     ctx.profile(False)
     # end to end: the layer's Q, K, V come from pinned host memory, the kept positions go back
-    hq, hk, hv = (torch.empty(Q.shape, dtype=torch.float16).pin_memory() for _ in range(3))
+    hq, hk, hv = (torch.empty(t.shape, dtype=torch.float16).pin_memory() for t in (Q, Kp, V))
     hq.copy_(Q); hk.copy_(Kp); hv.copy_(V)
     dq, dk, dv = torch.empty_like(Q), torch.empty_like(Kp), torch.empty_like(V)
     inst0 = list(range(0, w.batch * w.layers * w.heads, w.layers * w.heads))[:w.batch]
@@ -544,7 +560,7 @@ def run_prefill(args):
         raise RuntimeError("device status")
     ms, ms_e2e = max_over_ranks([ms, ms_e2e], dev, world)
     if rank == 0:
-        tokens = w.batch * w.heads * w.prompt * world
+        tokens = w.batch * w.heads * w.group * w.prompt * world
         fl = prefill_flops(w)
         kt = {k: (prof[k][0] / prof[k][1] if prof[k][1] else 0.0) for k in prof}
         dominant = max(fl, key=lambda k: kt.get(k, 0.0))
@@ -559,12 +575,14 @@ def run_prefill(args):
                 "vs_baseline": None, "dtype": "f16 inputs, f32 accumulate", "data": "synthetic",
                 "config": {"workload": f"cfg5 prefill compression (B={w.batch}, 32 heads, one layer per step, "
                                        "prompt 32768, 1638+1638 slots, R=16)"
-                                       + (" [batch reduced for profiling]" if args.batch else ""),
+                                       + (" [batch reduced for profiling]" if args.batch else "")
+                                       + (f" [grouped query heads: {w.heads} KV heads x {w.group}; the unit counts query heads]"
+                                          if w.group > 1 else ""),
                            "instances_per_step": w.batch * w.heads,
                            "l2": "6.3 GB of Q, K, V per step exceed the 126 MB L2"},
                 "clocks": clocks,
                 "e2e": {"value": tokens / (ms_e2e * 1e-3), "unit": "head-tokens/s",
-                        "h2d_bytes_per_step": 3 * Q.numel() * 2, "d2h_bytes_per_step": rec_bytes},
+                        "h2d_bytes_per_step": (Q.numel() + Kp.numel() + V.numel()) * 2, "d2h_bytes_per_step": rec_bytes},
                 "gpu_launches": int(launches),
                 "roofline": {"bound": "tensor", "kernel": {"build": "state_tc_kernel"}.get(dominant, dominant + "_tc_kernel"), "achieved": ach, "peak": peak,
                              "unit": "TFLOP/s", "frac": ach / peak, "peak_kind": kind, "traffic": None,

@@ -26,7 +26,10 @@
  *     stderr), LESS_FEATURE_KERNEL=gemv|plain (CUDA-core feature-map kernels),
  *     LESS_NO_OVERLAP (no programmatic dependent launch of the decode kernel),
  *     LESS_SCORE_KERNEL=plain (CUDA-core prompt scoring),
- *     LESS_FEATURE_STAGES=n (cap on the feature kernels' weight ring).
+ *     LESS_FEATURE_STAGES=n (cap on the feature kernels' weight ring),
+ *     LESS_GROUP_KERNEL=teams|rows (grouped query heads: force the decode kernel with
+ *     one 128-thread team per query head, or the one with one 128-thread CTA per KV
+ *     head; by default the number of KV heads per multiprocessor decides).
  */
 #ifndef LESS_B200_H
 #define LESS_B200_H
@@ -93,7 +96,12 @@ typedef struct less_config {
   int32_t max_prompt;         /* longest prompt less_prefill will be given (>= 0) */
   int32_t max_prefill_layers; /* layers scored together in less_prefill (>= 1): sizes the workspace */
   uint32_t flags;
-  int32_t group;              /* query heads per KV head (grouped- / multi-query attention); 0 or 1 = one */
+  int32_t group;              /* query heads per KV head (Section 3.2, multi-query attention): 0 or 1 = one;
+                               * 2, 4 or 8 need hidden in {128, 256, 512}, a policy other than
+                               * LESS_POLICY_TOVA, the tensor-core prompt scoring, and
+                               * group * (heavy + recent + 1028) * 4 bytes <= 227 KB (the decode kernel
+                               * keeps one score per slot and query head in shared memory);
+                               * anything else is LESS_ERR_INVALID_CONFIG */
 } less_config;
 
 /* Per-head feature-map weights (Eq. 1, Eq. 2), device, fp16, row-major, no biases:
@@ -163,8 +171,8 @@ int less_decode_step(less_ctx* ctx, const void* q, const void* k, const void* v,
                      int32_t* evicted_pos, void* cuda_stream);
 
 /* The same step for callers whose tensors live in host memory (Algorithm 1's
- * inputs and return value): q, k, v are host fp16 [B, L, H, D], out host fp32
- * [B, L, H, D].  q and k are copied to staging buffers inside the arena; v and
+ * inputs and return value): q host fp16 [B, L, H * group, D], k, v host fp16
+ * [B, L, H, D], out host fp32 [B, L, H * group, D].  q and k are copied to staging buffers inside the arena; v and
  * out are read / written in place by the decode kernel when they lie in pinned
  * (page-locked, device-mapped) memory, else they are staged and copied too.
  * Everything runs on the given stream, which is synchronised before returning. */

@@ -361,13 +361,253 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_kernel(DecParams p) {
 
 // --------------------------------------------------------------------------- //
 // Grouped query heads (Section 3.2, multi-query attention): G query heads share one KV head.
-// One CTA per KV head reads its K and V slots once and serves the G queries from registers;
-// every query head has its own Eq. 3 (own phi, own normaliser) over the shared cache and
-// the shared H, z; an entry's H2O score grows by the sum of the G heads' probabilities and
-// one entry is evicted for all of them.
+// One CTA per KV head, 128 threads per query head: each 128-thread team runs Eq. 3 for its own
+// head (own phi, own normaliser) over the shared slots and the shared H, z, exactly as
+// decode_kernel does for a single head; the teams' reads of the same K / V rows meet in L1, so
+// the slots cross HBM once.  Then all threads add the G heads' probabilities into the entries'
+// H2O scores and pick the one entry that leaves for all heads.
 // --------------------------------------------------------------------------- //
+__device__ __forceinline__ void team_sync(int team) {
+  asm volatile("bar.sync %0, %1;" ::"r"(team + 1), "n"(DEC_THREADS) : "memory");
+}
+
+__device__ __forceinline__ float team_max(float v, float* red, int team) {
+  const int lane = threadIdx.x & 31, warp = (threadIdx.x >> 5) & 3;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  if (lane == 0) red[warp] = v;
+  team_sync(team);
+  const float r = fmaxf(fmaxf(red[0], red[1]), fmaxf(red[2], red[3]));
+  team_sync(team);
+  return r;
+}
+
+__device__ __forceinline__ float team_sum(float v, float* red, int team) {
+  const int lane = threadIdx.x & 31, warp = (threadIdx.x >> 5) & 3;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  if (lane == 0) red[warp] = v;
+  team_sync(team);
+  const float r = ((red[0] + red[1]) + red[2]) + red[3];   // fixed order
+  team_sync(team);
+  return r;
+}
+
 template <int R, int G, bool kCaptured>
-__global__ void __launch_bounds__(DEC_THREADS) decode_group_kernel(DecParams p) {
+__global__ void __launch_bounds__(DEC_THREADS * G) decode_group_kernel(DecParams p) {
+  extern __shared__ float dsm[];
+  const int Ns = p.Np + 4;
+  float* s_sc_all = dsm;                           // [G][Np + 4] scores, then e^{s - m_g}
+  float* s_red_all = s_sc_all + G * Ns;            // [G][DEC_RG][128] partial numerators
+  __shared__ float s_small[G][4];
+  __shared__ unsigned long long s_key[G * 4];
+  __shared__ int s_vic;
+  __shared__ float s_inv[G];
+
+  const int team = threadIdx.x / DEC_THREADS;      // query head of the group
+  const int tid = threadIdx.x % DEC_THREADS;       // thread within the team
+  const size_t inst = blockIdx.x;
+  const size_t qi = inst * G + team;               // query head among all query heads
+  const int l16 = tid & 15, rg = tid >> 4;
+  const int N = p.N;
+  const int t_now = kCaptured ? __ldcg(p.a.tpos) : p.t;
+  int n = p.a.count[inst];
+  if (n < 0 || n > N) {
+    if (threadIdx.x == 0) set_status(p.a.status, kStatusBounds, 1);
+    step_done<kCaptured>(p.a.tpos, p.t);
+    return;
+  }
+  const bool use_state = !(p.flags & LESS_NO_STATE);
+  const float scale = 0.08838834764831845f;        // 1 / sqrt(128)
+  float* s_sc = s_sc_all + team * Ns;
+  float* s_red = s_red_all + team * DEC_RG * kHeadDim;
+
+  const __half* Kb = p.a.kslots + inst * (size_t)N * kHeadDim;
+  const __half* Vb = p.a.vslots + inst * (size_t)N * kHeadDim;
+
+  float qf[8];
+  half8_to_float(*reinterpret_cast<const uint4*>(p.q + qi * kHeadDim + l16 * 8), qf);
+
+  // ---- this head's scores over the live slots and the new pair ----
+#pragma unroll 4
+  for (int r0 = 0; r0 < n; r0 += DEC_RG) {
+    const int r = r0 + rg;
+    float dot = 0.f;
+    if (r < n) {
+      float kf[8];
+      half8_to_float(*reinterpret_cast<const uint4*>(Kb + (size_t)r * kHeadDim + l16 * 8), kf);
+#pragma unroll
+      for (int c = 0; c < 8; ++c) dot = fmaf(qf[c], kf[c], dot);
+    }
+#pragma unroll
+    for (int o = 8; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+    if (l16 == 0 && r < n) s_sc[r] = dot * scale;
+  }
+  const uint4 knew = *reinterpret_cast<const uint4*>(p.k + inst * kHeadDim + l16 * 8);
+  const uint4 vnew = *reinterpret_cast<const uint4*>(p.v + inst * kHeadDim + l16 * 8);
+  if (tid < 32) {
+    float kf[8];
+    half8_to_float(knew, kf);
+    float dot = 0.f;
+#pragma unroll
+    for (int c = 0; c < 8; ++c) dot = fmaf(qf[c], kf[c], dot);
+#pragma unroll
+    for (int o = 8; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+    if (tid == 0) s_sc[n] = dot * scale;
+  }
+  team_sync(team);
+
+  float m = -INFINITY;
+  for (int i = tid; i <= n; i += DEC_THREADS) m = fmaxf(m, s_sc[i]);
+  m = team_max(m, s_small[team], team);
+  m = fmaxf(m, -80.f);
+  float lsum = 0.f;
+  for (int i = tid; i <= n; i += DEC_THREADS) {
+    const float e = __expf(s_sc[i] - m);
+    s_sc[i] = e;
+    lsum += e;
+  }
+  lsum = team_sum(lsum, s_small[team], team);
+
+  // ---- u = sum e_i v_i ----
+  float u[8];
+#pragma unroll
+  for (int c = 0; c < 8; ++c) u[c] = 0.f;
+#pragma unroll 4
+  for (int r = rg; r < n; r += DEC_RG) {
+    float vf[8];
+    half8_to_float(*reinterpret_cast<const uint4*>(Vb + (size_t)r * kHeadDim + l16 * 8), vf);
+    const float e = s_sc[r];
+#pragma unroll
+    for (int c = 0; c < 8; ++c) u[c] = fmaf(e, vf[c], u[c]);
+  }
+  if (rg == 0) {
+    float vf[8];
+    half8_to_float(vnew, vf);
+    const float e = s_sc[n];
+#pragma unroll
+    for (int c = 0; c < 8; ++c) u[c] = fmaf(e, vf[c], u[c]);
+  }
+#pragma unroll
+  for (int c = 0; c < 8; ++c) s_red[rg * kHeadDim + l16 * 8 + c] = u[c];
+  team_sync(team);
+
+  // ---- Eq. 3 of this head over the shared H, z ----
+  const int d = tid;
+  float num = 0.f;
+#pragma unroll
+  for (int j = 0; j < DEC_RG; ++j) num += s_red[j * kHeadDim + d];
+  float den = lsum;
+  float* Hb = p.a.H + inst * (size_t)R * kHeadDim;
+  float* zb = p.a.z + inst * R;
+  float hcol[R];
+  if (use_state) {
+    pdl_wait_primary();
+    const float em = __expf(-m);
+    const float* ph = p.a.phi_q + qi * R;
+    float lr = 0.f, lz = 0.f;
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+      const float f = ph[r];
+      hcol[r] = Hb[r * kHeadDim + d];
+      lr = fmaf(f, hcol[r], lr);
+      lz = fmaf(f, zb[r], lz);
+    }
+    num = fmaf(em, lr, num);
+    den = fmaf(em, lz, den);
+  }
+  p.out[qi * kHeadDim + d] = num / den;
+  if (tid == 0) s_inv[team] = 1.0f / ((p.flags & LESS_SCORE_NORM_SPARSE) ? lsum : den);
+  __syncthreads();                                 // every head's e_i and 1 / normaliser are in shared memory; H, z are read
+
+  // ---- H2O over the group: acc_i += sum_g p_{g,i}; one victim for all heads ----
+  float inv[G];
+#pragma unroll
+  for (int g = 0; g < G; ++g) inv[g] = s_inv[g];
+  int32_t* posb = p.a.pos + inst * (size_t)p.Np;
+  float* accb = p.a.acc + inst * (size_t)p.Np;
+  const bool full = (n == N);
+  const bool lambda_policy = (p.flags & LESS_POLICY_LAMBDA) != 0;
+  unsigned long long best = ~0ull;
+  for (int i = threadIdx.x; i < n; i += DEC_THREADS * G) {
+    float ps_sum = 0.f;
+#pragma unroll
+    for (int g = 0; g < G; ++g) ps_sum = fmaf(s_sc_all[g * Ns + i], inv[g], ps_sum);
+    const float a = accb[i] + ps_sum;
+    accb[i] = a;
+    if (full) {
+      const int ps = posb[i];
+      if (lambda_policy) {
+        if (ps >= p.heavy) best = (unsigned long long)(unsigned int)ps < best ? (unsigned int)ps : best;
+      } else if (ps <= t_now - p.recent) {
+        const unsigned long long key =
+            ((unsigned long long)__float_as_uint(a) << 32) | (unsigned int)ps;
+        best = key < best ? key : best;
+      }
+    }
+  }
+  float p_new = 0.f;
+#pragma unroll
+  for (int g = 0; g < G; ++g) p_new = fmaf(s_sc_all[g * Ns + n], inv[g], p_new);
+  int slot = n;
+  if (full) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const unsigned long long other = __shfl_xor_sync(0xffffffffu, best, o);
+      best = other < best ? other : best;
+    }
+    if ((threadIdx.x & 31) == 0) s_key[threadIdx.x >> 5] = best;
+    if (threadIdx.x == 0) s_vic = -1;
+    __syncthreads();
+    best = s_key[0];
+#pragma unroll
+    for (int w = 1; w < G * 4; ++w) best = s_key[w] < best ? s_key[w] : best;
+    const int vpos = (int)(unsigned int)(best & 0xffffffffull);
+    for (int i = threadIdx.x; i < n; i += DEC_THREADS * G)
+      if (posb[i] == vpos && best != ~0ull) s_vic = i;
+    __syncthreads();
+    slot = s_vic;
+    if (slot < 0) {
+      if (threadIdx.x == 0) {
+        set_status(p.a.status, kStatusBounds, 2);
+        if (p.evicted_pos) p.evicted_pos[inst] = -1;
+      }
+      step_done<kCaptured>(p.a.tpos, p.t);
+      return;
+    }
+    if (threadIdx.x == 0 && p.evicted_pos) p.evicted_pos[inst] = vpos;
+    if (use_state && team == 0) {                  // Eq. 4 / Eq. 5: psi acts on the key, the state is the KV head's
+      const float vv = __half2float(Vb[(size_t)slot * kHeadDim + d]);
+      const float* psv = p.a.psic + (inst * (size_t)N + slot) * R;
+#pragma unroll
+      for (int r = 0; r < R; ++r) Hb[r * kHeadDim + d] = fmaf(psv[r], vv, hcol[r]);
+      if (tid < R) zb[tid] += psv[tid];
+    }
+    __syncthreads();                               // victim row fully read before overwrite
+  } else {
+    if (threadIdx.x == 0) {
+      p.a.count[inst] = n + 1;
+      if (p.evicted_pos) p.evicted_pos[inst] = -1;
+    }
+  }
+  if (team == 0) {                                 // the new pair takes the slot in place
+    __half* Kw = p.a.kslots + (inst * (size_t)N + slot) * kHeadDim;
+    __half* Vw = p.a.vslots + (inst * (size_t)N + slot) * kHeadDim;
+    if (rg == 0) *reinterpret_cast<uint4*>(Kw + l16 * 8) = knew;
+    if (rg == 1) *reinterpret_cast<uint4*>(Vw + l16 * 8) = vnew;
+    if (tid == 32) { posb[slot] = t_now; accb[slot] = p_new; }
+    if (tid >= 64 && tid < 64 + R)
+      p.a.psic[(inst * (size_t)N + slot) * R + (tid - 64)] =
+          use_state ? p.a.psi_k[inst * R + (tid - 64)] : 0.f;
+  }
+  step_done<kCaptured>(p.a.tpos, p.t);
+}
+
+// The same step for many KV heads per SM (batched serving): 128 threads per KV head, so that
+// several CTAs share an SM; every K / V row is loaded and converted once and meets the G
+// queries in registers.
+template <int R, int G, bool kCaptured>
+__global__ void __launch_bounds__(DEC_THREADS) decode_group_rows_kernel(DecParams p) {
   extern __shared__ float dsm[];
   const int Ns = p.Np + 4;
   float* s_sc = dsm;                               // [G][Np + 4] scores, then e^{s - m_g}
@@ -612,9 +852,11 @@ size_t decode_smem_bytes(const Dims& d) {
   return (size_t)d.G * (d.Np + 4 + DEC_RG * kHeadDim) * 4;
 }
 
+// teams: one 128-thread team per query head (few KV heads, latency matters); else one 128-thread CTA per KV head
 template <int R, int G>
-static void* decode_group_entry(bool captured) {
-  return captured ? (void*)decode_group_kernel<R, G, true> : (void*)decode_group_kernel<R, G, false>;
+static void* decode_group_entry(bool captured, bool teams) {
+  if (teams) return captured ? (void*)decode_group_kernel<R, G, true> : (void*)decode_group_kernel<R, G, false>;
+  return captured ? (void*)decode_group_rows_kernel<R, G, true> : (void*)decode_group_rows_kernel<R, G, false>;
 }
 
 int launch_decode(less_ctx* c, const void* q, const void* k, const void* v, void* out,
@@ -635,15 +877,18 @@ int launch_decode(less_ctx* c, const void* q, const void* k, const void* v, void
   LaunchScope scope(c, LESS_KERNEL_DECODE, s);
   void* kern = d.R == 8 ? (captured ? (void*)decode_kernel<8, true> : (void*)decode_kernel<8, false>)
                         : (captured ? (void*)decode_kernel<16, true> : (void*)decode_kernel<16, false>);
-  if (d.G == 2) kern = d.R == 8 ? decode_group_entry<8, 2>(captured) : decode_group_entry<16, 2>(captured);
-  if (d.G == 4) kern = d.R == 8 ? decode_group_entry<8, 4>(captured) : decode_group_entry<16, 4>(captured);
-  if (d.G == 8) kern = d.R == 8 ? decode_group_entry<8, 8>(captured) : decode_group_entry<16, 8>(captured);
+  // grouped query heads: with fewer KV heads than two per SM a CTA's latency is the step's, and the
+  // heads of a group run side by side (128 threads each); with more, throughput per SM counts
+  const bool teams = d.G > 1 && (c->group_path == 1 || (c->group_path == 0 && d.I < 2 * c->sms));
+  if (d.G == 2) kern = d.R == 8 ? decode_group_entry<8, 2>(captured, teams) : decode_group_entry<16, 2>(captured, teams);
+  if (d.G == 4) kern = d.R == 8 ? decode_group_entry<8, 4>(captured, teams) : decode_group_entry<16, 4>(captured, teams);
+  if (d.G == 8) kern = d.R == 8 ? decode_group_entry<8, 8>(captured, teams) : decode_group_entry<16, 8>(captured, teams);
   if (smem > 48 * 1024 &&
       cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
     return fail_cuda("shared memory opt-in of decode_kernel");
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(d.I);
-  cfg.blockDim = dim3(DEC_THREADS);
+  cfg.blockDim = dim3(teams ? DEC_THREADS * d.G : DEC_THREADS);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = s;
   cudaLaunchAttribute attr[1];

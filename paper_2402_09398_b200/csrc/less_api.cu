@@ -178,6 +178,11 @@ int less_create(const less_config* cfg, const less_weights* w, void* arena, size
     else if (!strcmp(e, "plain")) c->feature_path = 0;
   }
   if (cudaGetDevice(&c->device) != cudaSuccess) { delete c; return LESS_ERR_CUDA; }
+  c->group_path = 0;
+  if (const char* e = getenv("LESS_GROUP_KERNEL")) {
+    if (!strcmp(e, "teams")) c->group_path = 1;
+    else if (!strcmp(e, "rows")) c->group_path = 2;
+  }
   c->sms = 148;
   cudaDeviceGetAttribute(&c->sms, cudaDevAttrMultiProcessorCount, c->device);
   // H_0 = 0, z_0 = 0, no live slots, clean status

@@ -173,3 +173,28 @@ def test_maximum_slot_count_one_instance():
     print("max slots decode", tf.worst)
     ctx.close()
     torch.cuda.empty_cache()
+
+
+def test_cfg2_grouped_query_heads_sampled_instances():
+    """The cfg2 shape with its 32 query heads per layer grouped over 4 KV heads (G = 8), in the
+    launch configuration of `bench.py --group 8`: prompt phase and teacher-forced decode steps of
+    sampled KV heads against the grouped oracle."""
+    import harness
+    w = wl.CONFIGS[2]
+    w = w.with_(heads=w.heads // 8, group=8)
+    ctx, W = _ctx(w, w.layers)
+    Q, K, V = wl.make_prompt(w, 0, w.layers, DEV)
+    ctx.prefill(Q, K, V, 0)
+    assert ctx.poll_status() == 0
+    inst = _sample(w, 4)
+    Wc = {k: v.cpu() for k, v in W.items()}
+    r = harness.check_prefill_group(ctx, w, Wc, Q.cpu(), K.cpu(), V.cpu(), inst)
+    print("cfg2 grouped prompt", r)
+    del Q, K, V
+    tf = harness.GroupTeacherForced(ctx, w, Wc, inst)
+    for s in range(8):
+        tf.step(*wl.make_decode_inputs(w, s, DEV))
+    assert ctx.poll_status() == 0 and tf.evictions == 8 * len(inst) and tf.exempt <= 1
+    print("cfg2 grouped decode", tf.worst)
+    ctx.close()
+    torch.cuda.empty_cache()

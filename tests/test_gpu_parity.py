@@ -328,11 +328,11 @@ def test_decode_many_instances_and_ragged_slots(overlap, monkeypatch):
     ctx.close()
 
 
-@pytest.mark.parametrize("pinned", [True, False])
-def test_host_buffer_entry_matches_device_entry(pinned):
+@pytest.mark.parametrize("pinned,group", [(True, 1), (False, 1), (True, 4), (False, 2)])
+def test_host_buffer_entry_matches_device_entry(pinned, group):
     """less_decode_step_host with pinned (read / written in place by the kernel) and pageable
     (staged and copied) host tensors gives bit-identical outputs and state to less_decode_step."""
-    w = small(54, steps=5, weight_std=0.1)
+    w = small(54, steps=5, weight_std=0.1, group=group)
     ctx_d, W = _setup(w)
     ctx_h, _ = _setup(w)
     for ctx in (ctx_d, ctx_h):
@@ -384,11 +384,11 @@ def test_tova_new_token_can_evict_itself():
 
 
 @pytest.mark.parametrize("batch", [1, 12])
-def test_captured_step_replays_like_direct_calls(batch):
+def test_captured_step_replays_like_direct_calls(batch, group=1):
     """One decode step captured in a CUDA graph (fixed input / output buffers) and replayed: the
     position advances on the device, so every replay is the next step.  Outputs and state must be
     bit-identical to direct calls on a second context."""
-    w = small(49, batch=batch, layers=2, heads=2, steps=7, weight_std=0.1)
+    w = small(49, batch=batch, layers=2, heads=2, steps=7, weight_std=0.1, group=group)
     ctx_d, _ = _setup(w)
     ctx_g, _ = _setup(w)
     for ctx in (ctx_d, ctx_g):
@@ -419,12 +419,18 @@ def test_captured_step_replays_like_direct_calls(batch):
     ctx_d.close(); ctx_g.close()
 
 
+def test_captured_step_replays_with_grouped_query_heads():
+    test_captured_step_replays_like_direct_calls(3, group=4)
+
+
+@pytest.mark.parametrize("kernel", ["teams", "rows"])
 @pytest.mark.parametrize("group,rank,flags", [(2, 8, 0), (4, 16, 0), (8, 8, 0), (4, 8, 4), (2, 16, 1), (4, 8, 2)])
-def test_grouped_query_heads_decode_from_empty(group, rank, flags):
+def test_grouped_query_heads_decode_from_empty(group, rank, flags, kernel, monkeypatch):
     """Section 3.2, multi-query attention: G query heads share one KV head's cache, scores and
     state; every step is checked against the grouped oracle (outputs of all G heads, per-head phi,
     aggregated H2O scores, the one eviction, Eq. 4 / Eq. 5)."""
     import harness
+    monkeypatch.setenv("LESS_GROUP_KERNEL", kernel)     # both decode kernels for grouped heads
     w = small(60 + group, prompt=0, steps=30, heavy=9, recent=8, rank=rank, weight_std=0.1, group=group)
     ctx, W = _setup(w, flags=flags, max_prompt=16)
     inst = list(range(w.instances))
@@ -438,4 +444,58 @@ def test_grouped_query_heads_decode_from_empty(group, rank, flags):
     assert tf.exempt <= 2
     assert ctx.poll_status() == 0
     print("grouped decode", group, tf.worst)
+    ctx.close()
+
+
+@pytest.mark.parametrize("group,rank,prompt,flags", [(2, 8, 300, 0), (4, 16, 513, 0), (8, 8, 131, 0),
+                                                     (4, 8, 300, 4), (2, 8, 700, 1), (2, 16, 260, 2)])
+def test_grouped_query_heads_prompt_and_decode(group, rank, prompt, flags):
+    """Prompt phase with grouped query heads: per-query-head causal attention output, column sums
+    aggregated over the group's heads (Section 3.2), one kept set and one H, z per KV head; then
+    teacher-forced decode steps on top of it."""
+    import harness
+    w = small(40 + group, prompt=prompt, steps=8, heavy=20, recent=20, rank=rank, weight_std=0.1, group=group)
+    if flags & 4:
+        w = w.with_(heavy=4, recent=36)
+    ctx, W = _setup(w, flags=flags)
+    Q, K, V, out = _prefill_all(ctx, w)
+    assert Q.shape[2] == w.heads * group and K.shape[2] == w.heads and out.shape == Q.shape
+    assert ctx.poll_status() == 0
+    inst = list(range(w.instances))
+    r = harness.check_prefill_group(ctx, w, W, Q, K, V, inst, out, flags)
+    assert r["exempt"] <= 2
+    tf = harness.GroupTeacherForced(ctx, w, W, inst, flags)
+    for s in range(w.steps):
+        tf.step(*wl.make_decode_inputs(w, s, DEV))
+    assert tf.evictions == w.steps * w.instances
+    assert ctx.poll_status() == 0
+    print("grouped prompt", group, r, tf.worst)
+    ctx.close()
+
+
+def test_grouped_query_heads_rejected_configurations(monkeypatch):
+    from paper_2402_09398_b200 import binding
+    w = small(39, group=3)
+    W = wl.make_weights(w.with_(group=4), DEV)
+    with pytest.raises(binding.LessError):
+        binding.from_workload(w, W, DEV)                       # not a power of two
+    with pytest.raises(binding.LessError):
+        binding.from_workload(small(39, group=2), W, DEV, flags=8)   # TOVA stays per head
+    with pytest.raises(binding.LessError):
+        binding.from_workload(small(39, group=8, heavy=4000, recent=4000), W, DEV)   # scores of 8 heads x 8000 slots exceed shared memory
+
+
+def test_grouped_query_heads_many_kv_heads_pick_the_row_sharing_kernel():
+    """More than two KV heads per multiprocessor: the default choice is the decode kernel with one
+    128-thread CTA per KV head (K / V rows loaded once, G queries in registers)."""
+    import harness
+    w = small(38, batch=11, layers=3, heads=10, prompt=150, steps=4, heavy=12, recent=12, weight_std=0.1, group=4)
+    assert w.instances > 2 * torch.cuda.get_device_properties(0).multi_processor_count
+    ctx, W = _setup(w)
+    _prefill_all(ctx, w, with_out=False)
+    inst = list(range(0, w.instances, 7))
+    tf = harness.GroupTeacherForced(ctx, w, W, inst)
+    for s in range(w.steps):
+        tf.step(*wl.make_decode_inputs(w, s, DEV))
+    assert tf.evictions == w.steps * len(inst) and ctx.poll_status() == 0
     ctx.close()
