@@ -20,6 +20,9 @@ Paper passages followed:
   * Section 3.1     the prompt phase is regular attention (H_0 = 0, z_0 = 0)
   * Section 4       Lambda-masking as the sparse policy: the first tokens plus the most recent ones;
                     TOVA is named there without a definition (the rule of the cited work is used)
+  * Section 3.2 (Inexpensive Training), Section 4.1   the parallel form used for training and for the
+                    language-modelling evaluation: the whole causal attention matrix at once, entries
+                    the sparse policy does not keep replaced by phi(q_i) psi(k_j)^T
 
 Readings where the paper is silent (none of them is fixed by a printed number,
 so they are "parity unpinned" by the paper and fixed by the design notes that
@@ -394,3 +397,43 @@ def hellinger(p: np.ndarray, q: np.ndarray) -> float:
     p = np.asarray(p, dtype=np.float64)
     q = np.asarray(q, dtype=np.float64)
     return float(np.linalg.norm(np.sqrt(p) - np.sqrt(q)) / _SQRT2)
+
+
+NEVER = np.iinfo(np.int32).max
+
+
+def masked_parallel_attention(Q, K, V, exact_until, phi_fn, psi_fn):
+    """The parallel form (Section 3.2, Inexpensive Training; Section 4.1): every row of the causal
+    attention matrix at once.  Entry (i, j), j <= i, is exp(q_i . k_j / sqrt(D)) while key j is still
+    in the sparse cache when query i attends, i.e. i < exact_until[j], and phi(q_i) psi(k_j)^T from
+    then on (the entry "found by the kernel functions"); each row is normalised once, as in Eq. 3:
+
+        out_i = sum_j A_ij v_j / sum_j A_ij.
+
+    The sparse policies here discard a pair once and for all, so one integer per key describes the
+    mask: exact_until[j] = 1 + (the step at whose end j was evicted), NEVER if it stays.
+    Q, K, V: [S, D]; returns (out [S, D], A / row sums [S, S])."""
+    Q = np.asarray(Q, dtype=np.float64)
+    K = np.asarray(K, dtype=np.float64)
+    V = np.asarray(V, dtype=np.float64)
+    eu = np.asarray(exact_until, dtype=np.int64)
+    S, D = Q.shape
+    i = np.arange(S)[:, None]
+    j = np.arange(S)[None, :]
+    causal = j <= i
+    exact = causal & (i < eu[None, :])
+    A_exact = np.exp((Q @ K.T) / math.sqrt(D))
+    A_low = phi_fn(Q) @ psi_fn(K).T
+    A = np.where(exact, A_exact, np.where(causal, A_low, 0.0))
+    P = A / A.sum(axis=1, keepdims=True)
+    return P @ V, P
+
+
+def eviction_schedule(evicted_positions, first_step, S):
+    """exact_until of a sequence of S tokens from the list of positions a sequential run evicted:
+    evicted_positions[n] is the position discarded at the end of step first_step + n (-1 = none)."""
+    eu = np.full(S, NEVER, dtype=np.int64)
+    for n, pos in enumerate(evicted_positions):
+        if pos >= 0:
+            eu[pos] = first_step + n + 1
+    return eu

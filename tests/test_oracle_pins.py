@@ -631,3 +631,76 @@ def test_group_scores_are_summed_over_heads_and_state_is_shared(G):
         gone.add(victim)
         del hist[victim]
     assert sorted(kept) == list(grp.pos)
+
+
+# --------------------------------------------------------------------------- #
+# The parallel form (Section 3.2, Inexpensive Training; Section 4.1): the whole causal attention
+# matrix at once, entries the sparse policy dropped replaced by phi(q_i) psi(k_j)^T
+# --------------------------------------------------------------------------- #
+def _sequence_case(cfg_id, S=40, heavy=3, recent=4, D=16, R=4, policy="h2o"):
+    w = tiny(cfg_id=cfg_id, S=S, T=0, heavy=heavy, recent=recent, D=D, R=R, heads=1, std=0.4)
+    W = wl.make_weights(w)
+    Q, K, V = (t[0, 0, 0].double().numpy() for t in wl.make_prompt(w, 0, 1))
+    phi_fn, psi_fn = lo.make_mlp_maps(*head_weights(W, 0, 0))
+    return w, Q, K, V, phi_fn, psi_fn
+
+
+@pytest.mark.parametrize("policy", ["h2o", "lambda", "tova"])
+def test_parallel_form_rows_are_the_sequential_steps(policy):
+    """Row i of the parallel form is Algorithm 1's output at step i when the mask is the schedule
+    the sequential run produced: the two share nothing but the feature maps (the sequential run
+    keeps H, z by Eq. 4 / Eq. 5 and a slot cache; the parallel form builds the S x S matrix)."""
+    w, Q, K, V, phi_fn, psi_fn = _sequence_case(110, policy=policy)
+    S = Q.shape[0]
+    inst = lo.LessInstance(w.head_dim, w.rank, w.heavy, w.recent, phi_fn, psi_fn, policy=policy)
+    outs, ev = [], []
+    for t in range(S):
+        r = inst.decode(Q[t], K[t], V[t])
+        outs.append(r["out"])
+        ev.append(r["evicted_pos"])
+    eu = lo.eviction_schedule(ev, 0, S)
+    assert (eu != lo.NEVER).sum() == S - inst.N and np.all(eu > np.arange(S))
+    out, P = lo.masked_parallel_attention(Q, K, V, eu, phi_fn, psi_fn)
+    assert np.allclose(P.sum(axis=1), 1.0) and np.all(np.triu(P, 1) == 0)
+    assert np.allclose(out, np.stack(outs), rtol=1e-10, atol=1e-12)
+
+
+def test_parallel_form_with_nothing_evicted_is_causal_softmax():
+    w, Q, K, V, phi_fn, psi_fn = _sequence_case(111)
+    S, D = Q.shape
+    out, P = lo.masked_parallel_attention(Q, K, V, np.full(S, lo.NEVER), phi_fn, psi_fn)
+    ref = torch.nn.functional.scaled_dot_product_attention(
+        *(torch.as_tensor(a)[None, None] for a in (Q, K, V)), is_causal=True)[0, 0].numpy()
+    assert np.allclose(out, ref, rtol=1e-10, atol=1e-12)
+
+
+def test_parallel_form_with_everything_evicted_at_once_is_linear_attention():
+    """exact_until[j] = j + 1: only the diagonal is exact, the rest of a row is the kernel
+    phi(q_i) psi(k_j)^T; closed form with prefix sums (Eq. 6 for every prefix)."""
+    w, Q, K, V, phi_fn, psi_fn = _sequence_case(112)
+    S, D = Q.shape
+    out, _ = lo.masked_parallel_attention(Q, K, V, np.arange(S) + 1, phi_fn, psi_fn)
+    tQ, tK, tV = (torch.as_tensor(a) for a in (Q, K, V))
+    phi, psi = torch.as_tensor(phi_fn(Q)), torch.as_tensor(psi_fn(K))
+    Hpre = torch.cumsum(psi[:, :, None] * tV[:, None, :], dim=0) - psi[:, :, None] * tV[:, None, :]   # sum over j < i
+    zpre = torch.cumsum(psi, dim=0) - psi
+    d = torch.exp((tQ * tK).sum(1) / math.sqrt(D))
+    num = d[:, None] * tV + torch.einsum("ir,ird->id", phi, Hpre)
+    den = d + (phi * zpre).sum(1)
+    assert np.allclose(out, (num / den[:, None]).numpy(), rtol=1e-10, atol=1e-12)
+
+
+def test_parallel_form_mask_boundary_is_strict():
+    """Key j is exact for query i = exact_until[j] - 1 and low-rank for i = exact_until[j]."""
+    w, Q, K, V, phi_fn, psi_fn = _sequence_case(113, S=12)
+    S, D = Q.shape
+    eu = np.full(S, lo.NEVER)
+    eu[2] = 7
+    _, P = lo.masked_parallel_attention(Q, K, V, eu, phi_fn, psi_fn)
+    e = np.exp(Q @ K.T / math.sqrt(D))
+    low = phi_fn(Q) @ psi_fn(K).T
+    for i, want in ((6, e[6, 2]), (7, low[7, 2])):
+        row = np.where(np.arange(S) <= i, e[i], 0.0)
+        if i >= 7:
+            row[2] = low[i, 2]
+        assert np.isclose(P[i, 2], want / row.sum(), rtol=1e-12)
