@@ -82,7 +82,9 @@ enum {
    * protected.  `heavy + recent` only sets the slot count.  The prompt is
    * ranked once, by its last query's attention row.  Not together with
    * LESS_POLICY_LAMBDA. */
-  LESS_POLICY_TOVA = 8u
+  LESS_POLICY_TOVA = 8u,
+  /* Reserve the workspace of less_masked_attention (the parallel form) in the arena. */
+  LESS_WITH_PARALLEL_FORM = 16u
 };
 
 #define LESS_MAX_SLOTS 32768
@@ -147,6 +149,23 @@ int less_create(const less_config* cfg, const less_weights* weights, void* arena
 int less_prefill(less_ctx* ctx, int32_t layer_begin, int32_t layer_count, int32_t prompt_len,
                  const void* Q, const void* K, const void* V, void* attn_out, void* cuda_stream);
 
+/* The parallel form (Section 3.2, Inexpensive Training; Section 4.1): all rows of the
+ * causal attention matrix of a sequence at once, for training-time / evaluation-time use of
+ * the feature maps.  Entry (i, j), j <= i, is exp(q_i . k_j / sqrt(D)) while key j is in the
+ * sparse cache when query i attends (i < exact_until[j]) and phi(q_i) psi(k_j)^T from then
+ * on; every row is normalised once (Eq. 3):  out_i = sum_j A_ij v_j / sum_j A_ij.
+ * exact_until: device int32 [B, layer_count, H, seq_len]: 1 + the step at whose end the
+ * policy discarded key j (so exact_until[j] > j when a token attends to itself), INT32_MAX
+ * for a key that is never discarded; the caller obtains it from the policy (e.g. the
+ * evicted_pos record of less_decode_step).
+ * Q, K, V as in less_prefill (seq_len <= max_prompt); out: device fp32 [B, layer_count, H,
+ * seq_len, D].  Reads the context's weights, touches no cache or state; needs
+ * LESS_WITH_PARALLEL_FORM at creation, group <= 1 and the tensor-core kernels
+ * (hidden in {64, 128, 256, 512}), else LESS_ERR_INVALID_CONFIG. */
+int less_masked_attention(less_ctx* ctx, int32_t layer_begin, int32_t layer_count, int32_t seq_len,
+                          const void* Q, const void* K, const void* V, const int32_t* exact_until,
+                          void* out, void* cuda_stream);
+
 /* One generation step for every instance (Algorithm 1), at position t = tokens seen:
  *   phi(q_t), psi(k_t) (Eq. 1, 2); scores over the live slots plus the new pair;
  *   out = (phi(q) H + sum e^{s_i} v_i) / (phi(q) z^T + sum e^{s_i})        (Eq. 3)
@@ -195,7 +214,9 @@ enum {
   LESS_KERNEL_FINALIZE = 7,
   LESS_KERNEL_PSI = 8,
   LESS_KERNEL_GATHER = 9,
-  LESS_KERNEL_COUNT = 10
+  LESS_KERNEL_MASKED_PACK = 10,
+  LESS_KERNEL_MASKED_OUT = 11,
+  LESS_KERNEL_COUNT = 12
 };
 int less_profile(less_ctx* ctx, int enable);
 int less_profile_read(less_ctx* ctx, float* ms_total_host, int64_t* launches_host);

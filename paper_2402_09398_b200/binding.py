@@ -21,19 +21,20 @@ LESS_SCORE_NORM_SPARSE = 1
 LESS_NO_STATE = 2
 LESS_POLICY_LAMBDA = 4
 LESS_POLICY_TOVA = 8
+LESS_WITH_PARALLEL_FORM = 16
 
 EXPORTED = [
     "less_arena_bytes", "less_create", "less_prefill", "less_decode_step", "less_position",
     "less_state_record_bytes", "less_export_state", "less_import_state",
     "less_read_feature_maps", "less_poll_status", "less_launch_count", "less_strerror",
     "less_destroy", "less_decode_step_host", "less_profile", "less_profile_read",
-    "less_prompt_scores_noalloc",
+    "less_prompt_scores_noalloc", "less_masked_attention",
 ]
 LESS_NOALLOC_MAX_ROWS = 65536
 LESS_ERR_NOALLOC_TOO_LARGE = -12
 
 KERNEL_NAMES = ["feature_map", "decode", "rowstat", "colsum", "attn_out", "select", "build", "finalize",
-                "psi", "gather"]
+                "psi", "gather", "masked_pack", "masked_out"]
 
 
 class less_config(C.Structure):
@@ -95,6 +96,8 @@ def lib() -> C.CDLL:
     L.less_export_state.argtypes = [vp, vp, i32, vp, sz, vp]
     L.less_import_state.restype = C.c_int
     L.less_import_state.argtypes = [vp, vp, i32, vp, sz, vp]
+    L.less_masked_attention.restype = C.c_int
+    L.less_masked_attention.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp, vp]
     L.less_read_feature_maps.restype = C.c_int
     L.less_read_feature_maps.argtypes = [vp, vp, vp, vp]
     L.less_poll_status.restype = C.c_int
@@ -173,6 +176,10 @@ def less_import_state(ctx, inst_ptr, n, host_ptr, nbytes, stream) -> int:
     return lib().less_import_state(ctx, inst_ptr, n, host_ptr, nbytes, stream)
 
 
+def less_masked_attention(ctx, layer_begin, layer_count, seq_len, Q, K, V, exact_until, out, stream) -> int:
+    return lib().less_masked_attention(ctx, layer_begin, layer_count, seq_len, Q, K, V, exact_until, out, stream)
+
+
 def less_read_feature_maps(ctx, phi_ptr, psi_ptr, stream) -> int:
     return lib().less_read_feature_maps(ctx, phi_ptr, psi_ptr, stream)
 
@@ -238,6 +245,17 @@ class LessContext:
         assert Q.is_contiguous() and K.is_contiguous() and V.is_contiguous()
         _check(less_prefill(self.ctx, layer_begin, Lc, S, _ptr(Q), _ptr(K), _ptr(V), _ptr(attn_out),
                             _stream_ptr(stream)), "less_prefill")
+
+    def masked_attention(self, Q, K, V, exact_until, layer_begin=0, out=None, stream=None):
+        """The parallel form: Q, K, V fp16 [B, Lc, H, S, D], exact_until int32 [B, Lc, H, S]."""
+        B, Lc, H, S, D = Q.shape
+        assert Q.dtype == K.dtype == V.dtype == torch.float16 and exact_until.dtype == torch.int32
+        assert Q.is_contiguous() and K.is_contiguous() and V.is_contiguous() and exact_until.is_contiguous()
+        if out is None:
+            out = torch.empty(Q.shape, dtype=torch.float32, device=Q.device)
+        _check(less_masked_attention(self.ctx, layer_begin, Lc, S, _ptr(Q), _ptr(K), _ptr(V), _ptr(exact_until),
+                                     _ptr(out), _stream_ptr(stream)), "less_masked_attention")
+        return out
 
     def reset(self, layer_begin=0, layer_count=None, stream=None):
         n = self.cfg.layers - layer_begin if layer_count is None else layer_count

@@ -25,7 +25,7 @@ bool valid_config(const less_config* c) {
   if (c->max_prefill_layers < 1 || c->max_prefill_layers > c->layers) return false;
   if ((int64_t)c->batch * c->heads * c->max_prefill_layers * (c->group > 1 ? c->group : 1) > 65535)
     return false;                                                                   // grid.y of the prompt kernels
-  if (c->flags & ~(uint32_t)(LESS_SCORE_NORM_SPARSE | LESS_NO_STATE | LESS_POLICY_LAMBDA | LESS_POLICY_TOVA)) return false;
+  if (c->flags & ~(uint32_t)(LESS_SCORE_NORM_SPARSE | LESS_NO_STATE | LESS_POLICY_LAMBDA | LESS_POLICY_TOVA | LESS_WITH_PARALLEL_FORM)) return false;
   if ((c->flags & LESS_POLICY_LAMBDA) && (c->flags & LESS_POLICY_TOVA)) return false;
   if (c->group < 0 || c->group > 8 || (c->group & (c->group - 1))) return false;          // 0, 1, 2, 4, 8
   if (c->group > 1 && (c->flags & LESS_POLICY_TOVA)) return false;                         // TOVA stays per head
@@ -54,6 +54,7 @@ Dims make_dims(const less_config* c) {
   d.G = c->group > 1 ? c->group : 1;
   d.Sp = (c->max_prompt + 3) & ~3;
   d.Sbx = ((c->max_prompt + 255) & ~255) + 256;
+  d.St = (c->max_prompt + 127) / 128;
   d.Lw = c->max_prefill_layers;
   d.flags = c->flags;
   return d;
@@ -94,6 +95,13 @@ size_t carve(const Dims& d, char* base, Arena* a) {
   t.ws_psi = (float*)take(Iw * Sp * R * 4);
   t.ws_bx = (uint4*)take(Iw * G * (size_t)d.Sbx * 16);
   t.ws_pmax = (int32_t*)take(Iw * 4);
+  const size_t St = (d.flags & LESS_WITH_PARALLEL_FORM) ? d.St : 0;
+  t.ws_phi = (float*)take(St ? Iw * Sp * R * 4 : 0);
+  t.ws_phiop = (unsigned char*)take(Iw * St * 8192);
+  t.ws_psiop = (unsigned char*)take(Iw * St * 8192);
+  t.ws_g = (float*)take(Iw * St * 128 * 4);
+  t.ws_nb = (float*)take(Iw * St * 128 * 4);
+  t.ws_eu = (int32_t*)take(Iw * St * 128 * 4);
   if (a) *a = t;
   return off;
 }
@@ -232,6 +240,29 @@ int less_prefill(less_ctx* c, int32_t layer_begin, int32_t layer_count, int32_t 
     if (rc != LESS_OK) return rc;
   }
   c->t = prompt_len;
+  return LESS_OK;
+}
+
+int less_masked_attention(less_ctx* c, int32_t layer_begin, int32_t layer_count, int32_t seq_len,
+                          const void* Q, const void* K, const void* V, const int32_t* exact_until,
+                          void* out, void* stream) {
+  if (!c) return LESS_ERR_NULL_POINTER;
+  if (!(c->d.flags & LESS_WITH_PARALLEL_FORM) || c->d.G > 1) return LESS_ERR_INVALID_CONFIG;
+  if (layer_begin < 0 || layer_count < 1 || layer_begin + layer_count > c->d.L)
+    return LESS_ERR_BAD_LAYER_RANGE;
+  if (seq_len < 0) return LESS_ERR_INVALID_CONFIG;
+  if (seq_len > c->cfg.max_prompt) return LESS_ERR_PROMPT_TOO_LONG;
+  if (seq_len == 0) return LESS_OK;
+  if ((int64_t)c->d.B * layer_count * c->d.Hd * seq_len > 0x7fffffffLL) return LESS_ERR_PROMPT_TOO_LONG;
+  if (!Q || !K || !V || !exact_until || !out) return LESS_ERR_NULL_POINTER;
+  if (misaligned(Q) || misaligned(K) || misaligned(V) || misaligned(out) || ((uintptr_t)exact_until & 3))
+    return LESS_ERR_MISALIGNED;
+  cudaStream_t s = (cudaStream_t)stream;
+  for (int lj0 = 0; lj0 < layer_count; lj0 += c->d.Lw) {
+    int nl = layer_count - lj0 < c->d.Lw ? layer_count - lj0 : c->d.Lw;
+    int rc = launch_masked_form(c, layer_begin + lj0, nl, lj0, layer_count, seq_len, Q, K, V, exact_until, out, s);
+    if (rc != LESS_OK) return rc;
+  }
   return LESS_OK;
 }
 

@@ -42,6 +42,13 @@ struct Arena {
   float* ws_hpart;   // [Iw][kMaxSplit][R*D + R]  partial H, z per token split
   float* ws_psi;     // [Iw][Sp][R]  psi(k_j) of every prompt token
   int32_t* ws_pmax;  // [Iw]        bit pattern of max psi over the instance's prompt tokens (scales the state build's fp16 operand)
+  // parallel form only (LESS_WITH_PARALLEL_FORM); St = 128-row tiles of max_prompt
+  float* ws_phi;     // [Iw][Sp][R]  phi(q_i) of every row
+  unsigned char* ws_phiop;  // [Iw][St][8 KB]  phi as fp16 hi / lo operand tiles
+  unsigned char* ws_psiop;  // [Iw][St][8 KB]  psi likewise
+  float* ws_g;       // [Iw][St*128]  per row: factor of the low-rank entries
+  float* ws_nb;      // [Iw][St*128]  per row: exponent offset of the exact entries
+  int32_t* ws_eu;    // [Iw][St*128]  exact_until, padded with zeros
   uint4* ws_bx;      // [Iw*G][Sbx]  per prompt row: -(m_i sqrt(D) - log2(1/l_i) / c) as three fp16 parts (column sums)
 };
 
@@ -52,6 +59,7 @@ struct Dims {
   int32_t G;                    // query heads per KV head
   int32_t Sp;                   // max_prompt rounded up to a multiple of 4
   int32_t Sbx;                  // max_prompt rounded up to a multiple of 256 (+256)
+  int32_t St;                   // 128-row tiles of max_prompt
   int32_t Lw;                   // max_prefill_layers
   uint32_t flags;
 };
@@ -192,5 +200,8 @@ int launch_decode(less_ctx* c, const void* q, const void* k, const void* v, void
 int launch_prefill_group(less_ctx* c, int layer0, int nlayers, int lj0, int layer_count, int S,
                          const void* Q, const void* K, const void* V, void* attn_out,
                          cudaStream_t s);
+// the parallel form of one layer group (masked_tc.cu)
+int launch_masked_form(less_ctx* c, int layer0, int nlayers, int lj0, int layer_count, int S, const void* Q,
+                       const void* K, const void* V, const int32_t* exact_until, void* out, cudaStream_t s);
 
 }  // namespace less

@@ -1,0 +1,505 @@
+// The parallel form on the tensor cores (Section 3.2, Inexpensive Training; Section 4.1): all rows
+// of a sequence's causal attention matrix at once, entries the sparse policy has discarded
+// replaced by phi(q_i) psi(k_j)^T, one normalisation per row (Eq. 3):
+//
+//     A_ij = exp(q_i . k_j / sqrt(D))     if i < exact_until[j]          (key j still cached)
+//            phi(q_i) psi(k_j)^T          otherwise                      (j <= i)
+//     out_i = sum_j A_ij v_j / sum_j A_ij
+//
+// Steps (launch_masked_form): the row statistics m_i, 1 / l_i of the plain causal softmax
+// (rowstat_tc_kernel) serve as each row's reference; psi(K) and phi(Q) come from the MLP kernel
+// (psi_tc.cu); masked_pack_kernel turns them into fp16 hi / lo operand tiles and computes the
+// per-row constants; masked_out_tc_kernel then works like the prompt-output kernel, with a second
+// accumulator:
+//   S = Q K^T                       tcgen05, fp32 in tensor memory (double-buffered)
+//   L = phi~ psi~^T                 tcgen05, hi hi + lo hi + hi lo of the scaled fp16 splits
+//   P_ij = i < exact_until[j] ? exp2(c S_ij + nb_i) : L_ij g_i       (epilogue warps, lane = row)
+//   O += P V                        tcgen05;   r_i += sum_j P_ij (fp32, before rounding P to fp16)
+//   out_i = O_i / r_i
+// The key tiles stream past the Q tile twice.  The first sweep only adds up each row's entries in
+// fp32: a row whose dominant key has been discarded keeps a tiny share of the plain softmax's
+// mass, and its entries would sink into fp16's subnormals if P were formed against the plain
+// normaliser.  The second sweep divides by that sum first, so P holds the row's true
+// probabilities when it is rounded to fp16 for P V.
+// nb_i = -m_i log2(e) + log2(1 / l_i) + log2(w_i) makes the exact entries the plain softmax
+// probabilities times w_i, and g_i carries the same factors plus the operands' power-of-two scales.
+// w_i <= 1 is a power of two chosen from the bound  L_ij <= max(psi) sum_r phi_ir  so that no
+// entry of P exceeds 1 before it is rounded to fp16; it cancels in O_i / r_i.
+// Every wait is bounded (pipeline.cuh).
+#include "prefill.cuh"
+#include "tc_common.cuh"
+
+namespace less {
+
+constexpr int MF_TILE = 128;
+constexpr int MF_TILE_BYTES = MF_TILE * kHeadDim * 2;
+constexpr int MF_OP_BYTES = 8192;                   // operand tile: [4 chunks of 8 k][16 row groups][8 rows][16 B]
+constexpr int MF_EU_BYTES = MF_TILE * 4;
+constexpr int MF_STAGES = 2;
+constexpr int MF_EU_SLOTS = 4;                      // exact_until tiles in flight: the epilogue frees them, later than the K stage
+constexpr int MF_STAGE_BYTES = 2 * MF_TILE_BYTES;   // K tile, then V tile
+constexpr int MF_EPI_WARPS = 8;
+constexpr int MF_EPI_THREADS = MF_EPI_WARPS * 32;
+constexpr int MF_THREADS = 64 + MF_EPI_THREADS + 32;   // warp 0 TMA (Q, K, operands), warp 1 MMA, warps 2..9 epilogue, warp 10 TMA (V)
+constexpr float kMfExpScale = 0.12751743074602468f; // log2(e) / sqrt(128)
+constexpr float kLog2e = 1.4426950408889634f;
+
+struct MfParams {
+  const int32_t* exact_until;   // [B, layer_count, Hd, S]
+  float* out;                   // [B, layer_count, Hd, S, D]
+  int St;                       // operand tiles per instance in the workspace
+};
+
+// ------------------------------------------------------------------------------------------- //
+// Operand tiles and row constants.  One CTA = one 128-row tile of one instance, one thread per row.
+// ------------------------------------------------------------------------------------------- //
+__device__ __forceinline__ float pow2_scale_exponent(float vmax) {
+  // exponent e with vmax * 2^e in [8192, 16384): hi parts far from fp16's overflow, lo parts far from its underflow
+  if (!(vmax > 0.f) || !(vmax < INFINITY)) return 0.f;
+  return fminf(fmaxf(floorf(log2f(8192.f / vmax)), -100.f), 100.f);
+}
+
+template <int R>
+__device__ __forceinline__ void split_row(const float* x, float scale, uint4* hi, uint4* lo) {
+  // x[R] * scale -> fp16 hi and lo parts, 8 values per 16-byte chunk
+  uint32_t h[R / 2], l[R / 2];
+#pragma unroll
+  for (int e = 0; e < R / 2; ++e) {
+    const float a = x[2 * e] * scale, b = x[2 * e + 1] * scale;
+    const __half2 hh = __floats2half2_rn(a, b);
+    const float2 hf = __half22float2(hh);
+    const __half2 ll = __floats2half2_rn(a - hf.x, b - hf.y);
+    h[e] = *reinterpret_cast<const uint32_t*>(&hh);
+    l[e] = *reinterpret_cast<const uint32_t*>(&ll);
+  }
+#pragma unroll
+  for (int c = 0; c < R / 8; ++c) {
+    hi[c] = make_uint4(h[c * 4], h[c * 4 + 1], h[c * 4 + 2], h[c * 4 + 3]);
+    lo[c] = make_uint4(l[c * 4], l[c * 4 + 1], l[c * 4 + 2], l[c * 4 + 3]);
+  }
+}
+
+template <int R>
+__global__ void __launch_bounds__(MF_TILE) masked_pack_kernel(PfParams p, MfParams mf) {
+  const int T = blockIdx.x, g = blockIdx.y, r = threadIdx.x;
+  const int i = T * MF_TILE + r;
+  const bool valid = i < p.S;
+  const InstMap im = map_instance(p, g);
+  const float pmax = __int_as_float(p.a.ws_pmax[g]);
+  const float epsi = pow2_scale_exponent(pmax);
+
+  float ph[R], ps[R];
+#pragma unroll
+  for (int e = 0; e < R; ++e) ph[e] = ps[e] = 0.f;
+  if (valid) {
+    const float4* a = reinterpret_cast<const float4*>(p.a.ws_phi + ((size_t)g * p.Sp + i) * R);
+    const float4* b = reinterpret_cast<const float4*>(p.a.ws_psi + ((size_t)g * p.Sp + i) * R);
+#pragma unroll
+    for (int e = 0; e < R / 4; ++e) {
+      const float4 x = a[e], y = b[e];
+      ph[4 * e] = x.x; ph[4 * e + 1] = x.y; ph[4 * e + 2] = x.z; ph[4 * e + 3] = x.w;
+      ps[4 * e] = y.x; ps[4 * e + 1] = y.y; ps[4 * e + 2] = y.z; ps[4 * e + 3] = y.w;
+    }
+  }
+  float phmax = 0.f, phsum = 0.f;
+#pragma unroll
+  for (int e = 0; e < R; ++e) {
+    phmax = fmaxf(phmax, ph[e]);
+    phsum += ph[e];
+  }
+  const float ephi = pow2_scale_exponent(phmax);
+
+  // operand tiles.  The k-steps the MMA issues pair the chunks as
+  //   R = 8 :  phi (hi, lo) x psi (hi, hi),   phi (hi, 0) x psi (lo, 0)
+  //   R = 16:  phi hi x psi hi,  phi lo x psi hi,  phi hi x psi lo          (each 16 wide = 2 chunks)
+  uint4 fh[R / 8], fl[R / 8], sh_[R / 8], sl[R / 8];
+  split_row<R>(ph, exp2f(ephi), fh, fl);
+  split_row<R>(ps, exp2f(epsi), sh_, sl);
+  const size_t tile = ((size_t)g * mf.St + T) * MF_OP_BYTES;
+  const int off = (r >> 3) * 128 + (r & 7) * 16;
+  uint4* fo = reinterpret_cast<uint4*>(p.a.ws_phiop + tile + off);
+  uint4* so = reinterpret_cast<uint4*>(p.a.ws_psiop + tile + off);
+  const uint4 zero = make_uint4(0, 0, 0, 0);
+  constexpr int CH = 2048 / 16;                        // chunk stride in uint4
+  if (R == 8) {
+    fo[0] = fh[0]; fo[CH] = fl[0]; fo[2 * CH] = fh[0]; fo[3 * CH] = zero;
+    so[0] = sh_[0]; so[CH] = sh_[0]; so[2 * CH] = sl[0]; so[3 * CH] = zero;
+  } else {
+    fo[0] = fh[0]; fo[CH] = fh[R / 8 - 1]; fo[2 * CH] = fl[0]; fo[3 * CH] = fl[R / 8 - 1];
+    so[0] = sh_[0]; so[CH] = sh_[R / 8 - 1]; so[2 * CH] = sl[0]; so[3 * CH] = sl[R / 8 - 1];
+  }
+
+  // row constants
+  float nb = -60000.f, gi = 0.f;
+  int eu = 0;
+  if (valid) {
+    const float m = p.a.ws_m[(size_t)g * p.Sp + i];
+    const float il = p.a.ws_invl[(size_t)g * p.Sp + i];
+    const float base = fmaf(-m, kLog2e, log2f(il));      // log2 of e^{-m} / l
+    float lw = 0.f;                                      // log2 w_i
+    const float bound = pmax * phsum;                    // >= every phi(q_i) psi(k_j)^T of the row
+    if (bound > 0.f && bound < INFINITY) {
+      const float lb = log2f(bound) + base;
+      if (lb > 0.f) lw = -ceilf(lb);
+    }
+    nb = base + lw;
+    gi = exp2f(fminf(nb - ephi - epsi, 120.f));
+    eu = mf.exact_until[im.in_row0 + i];
+  }
+  const size_t row = (size_t)g * mf.St * MF_TILE + i;
+  p.a.ws_nb[row] = nb;
+  p.a.ws_g[row] = gi;
+  p.a.ws_eu[row] = eu;
+}
+
+// ------------------------------------------------------------------------------------------- //
+// One CTA = one 128-row Q tile of one instance; key tiles 0 .. diagonal stream past it.
+// ------------------------------------------------------------------------------------------- //
+struct MfShared {
+  uint64_t res_full;
+  uint64_t k_full[MF_STAGES], k_empty[MF_STAGES];     // K tile + psi operand tile
+  uint64_t v_full[MF_STAGES], v_empty[MF_STAGES];
+  uint64_t eu_full[MF_EU_SLOTS], eu_empty[MF_EU_SLOTS];   // exact_until of the key tile
+  uint64_t s_full[2], s_free[2];                      // S buffer (and L) written / read
+  uint64_t l_free;                                    // the single L buffer has been read
+  uint64_t p_full, p_free;
+  uint64_t o_full;
+  uint32_t tmem_base;
+  int abort;
+  float rsum[2][MF_TILE];
+};
+
+__device__ __forceinline__ float mf_ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+__device__ __forceinline__ void mf_epi_sync() { asm volatile("bar.sync 1, %0;" ::"n"(MF_EPI_THREADS) : "memory"); }
+
+template <int R>
+__global__ void __launch_bounds__(MF_THREADS) masked_out_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
+                                                                   const __grid_constant__ CUtensorMap tm_k,
+                                                                   const __grid_constant__ CUtensorMap tm_v,
+                                                                   PfParams p, MfParams mf) {
+  extern __shared__ __align__(1024) unsigned char mf_smem[];
+  unsigned char* qres = mf_smem;                                   // Q tile: [2 halves][128 rows][128 B]
+  unsigned char* ring = qres + MF_TILE_BYTES;                      // [stages][K tile, V tile]
+  unsigned char* pbuf = ring + MF_STAGES * MF_STAGE_BYTES;         // P: [2 key halves][128 rows][128 B], swizzled
+  unsigned char* phires = pbuf + MF_TILE_BYTES;                    // phi operand tile of the rows
+  unsigned char* psiring = phires + MF_OP_BYTES;                   // [stages] psi operand tiles of the keys
+  unsigned char* euring = psiring + MF_STAGES * MF_OP_BYTES;       // [slots] exact_until of the keys
+  MfShared* sh = reinterpret_cast<MfShared*>(euring + MF_EU_SLOTS * MF_EU_BYTES);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int tiles = (p.S + MF_TILE - 1) / MF_TILE;
+  const int tile = tiles - 1 - (int)blockIdx.x;                    // long rows first
+  const int g = blockIdx.y;
+  const InstMap im = map_instance(p, g);
+  const int i0 = tile * MF_TILE;
+  const int ntile = tile + 1;                                      // key tiles 0 .. tile (the last holds the diagonal)
+  int32_t* status = p.a.status;
+  const size_t op0 = (size_t)g * mf.St * MF_OP_BYTES;              // this instance's operand tiles
+  const size_t rc0 = (size_t)g * mf.St * MF_TILE;                  // ... and row constants
+
+  if (tid == 0) {
+    mbar_init(&sh->res_full, 1);
+    for (int s = 0; s < MF_STAGES; ++s) {
+      mbar_init(&sh->k_full[s], 1);
+      mbar_init(&sh->k_empty[s], 1);
+      mbar_init(&sh->v_full[s], 1);
+      mbar_init(&sh->v_empty[s], 1);
+    }
+    for (int s = 0; s < MF_EU_SLOTS; ++s) {
+      mbar_init(&sh->eu_full[s], 1);
+      mbar_init(&sh->eu_empty[s], MF_EPI_WARPS);
+    }
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(&sh->s_full[s], 1);
+      mbar_init(&sh->s_free[s], MF_EPI_WARPS);
+    }
+    mbar_init(&sh->l_free, MF_EPI_WARPS);
+    mbar_init(&sh->p_full, MF_EPI_WARPS);
+    mbar_init(&sh->p_free, 1);
+    mbar_init(&sh->o_full, 1);
+    sh->abort = *reinterpret_cast<volatile int32_t*>(status) != 0;
+    mbar_fence_init();
+  }
+  if (warp == 1) tmem_alloc(&sh->tmem_base, 512);
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem = sh->tmem_base;
+  const uint32_t ocol = 2 * MF_TILE, lcol = 3 * MF_TILE;           // O and L behind the two S buffers
+  volatile int* abortp = &sh->abort;
+
+  if (warp == 0) {
+    // ---------------- producer: Q and its phi operand, then K + psi operand + exact_until per key tile ----------------
+    if (lane == 0) {
+      const int row0 = (int)(im.in_row0 + i0);
+      mbar_expect_tx(&sh->res_full, MF_TILE_BYTES + MF_OP_BYTES);
+      tma_load_2d(qres, &tm_q, 0, row0, &sh->res_full);
+      tma_load_2d(qres + MF_TILE_BYTES / 2, &tm_q, 64, row0, &sh->res_full);
+      bulk_g2s(phires, p.a.ws_phiop + op0 + (size_t)tile * MF_OP_BYTES, MF_OP_BYTES, &sh->res_full);
+      uint32_t s = 0, ph = 0;
+      for (int u = 0; u < 2 * ntile; ++u) {              // two sweeps over the key tiles
+        const int t = u < ntile ? u : u - ntile;
+        wait_or_give_up(&sh->k_empty[s], ph ^ 1, abortp, status, 110);
+        const int es = u % MF_EU_SLOTS;
+        wait_or_give_up(&sh->eu_empty[es], ((u / MF_EU_SLOTS) & 1) ^ 1, abortp, status, 111);
+        if (*abortp) break;
+        const int krow = (int)(im.in_row0 + (size_t)t * MF_TILE);
+        unsigned char* st = ring + s * MF_STAGE_BYTES;
+        mbar_expect_tx(&sh->k_full[s], MF_TILE_BYTES + MF_OP_BYTES);
+        tma_load_2d(st, &tm_k, 0, krow, &sh->k_full[s]);
+        tma_load_2d(st + MF_TILE_BYTES / 2, &tm_k, 64, krow, &sh->k_full[s]);
+        bulk_g2s(psiring + s * MF_OP_BYTES, p.a.ws_psiop + op0 + (size_t)t * MF_OP_BYTES, MF_OP_BYTES, &sh->k_full[s]);
+        mbar_expect_tx(&sh->eu_full[es], MF_EU_BYTES);
+        bulk_g2s(euring + es * MF_EU_BYTES, p.a.ws_eu + rc0 + (size_t)t * MF_TILE, MF_EU_BYTES, &sh->eu_full[es]);
+        if (++s == MF_STAGES) { s = 0; ph ^= 1; }
+      }
+    }
+  } else if (warp == 10) {
+    // ---------------- producer of the V tiles ----------------
+    if (lane == 0) {
+      uint32_t s = 0, ph = 0;
+      for (int t = 0; t < ntile; ++t) {
+        wait_or_give_up(&sh->v_empty[s], ph ^ 1, abortp, status, 112);
+        if (*abortp) break;
+        const int krow = (int)(im.in_row0 + (size_t)t * MF_TILE);
+        unsigned char* st = ring + s * MF_STAGE_BYTES + MF_TILE_BYTES;
+        mbar_expect_tx(&sh->v_full[s], MF_TILE_BYTES);
+        tma_load_2d(st, &tm_v, 0, krow, &sh->v_full[s]);
+        tma_load_2d(st + MF_TILE_BYTES / 2, &tm_v, 64, krow, &sh->v_full[s]);
+        if (++s == MF_STAGES) { s = 0; ph ^= 1; }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer ----------------
+    if (lane == 0) {
+      constexpr uint32_t idesc_s = idesc_f16(MF_TILE, MF_TILE, 0, 0);   // A = Q (K-major), B = K (K-major); also phi x psi
+      constexpr uint32_t idesc_o = idesc_f16(MF_TILE, kHeadDim, 0, 1);  // A = P (K-major), B = V (N-major)
+      const uint64_t ad_q = smem_desc(smem_u32(qres), 16, 1024, kLayoutSw128);
+      // operand tiles without swizzle: chunks of 8 k are 2048 bytes apart, 8-row groups 128 bytes
+      const uint64_t ad_phi = smem_desc(smem_u32(phires), 2048, 128, kLayoutNone);
+      const uint64_t bd_psi = smem_desc(smem_u32(psiring), 2048, 128, kLayoutNone);
+      const uint64_t ad_p = smem_desc(smem_u32(pbuf), 16, 1024, kLayoutSw128);
+      const uint64_t bd_ring = smem_desc(smem_u32(ring), 16, 1024, kLayoutSw128);
+      const uint64_t bd_vring = smem_desc(smem_u32(ring) + MF_TILE_BYTES, MF_TILE_BYTES / 2, 1024, kLayoutSw128);
+      constexpr uint64_t kPair = 4096 >> 4;                             // two chunks = one 16-wide k-step further
+      wait_or_give_up(&sh->res_full, 0, abortp, status, 113);
+      uint32_t s1 = 0, ph1 = 0, b1 = 0, bph1 = 0;
+      int issued = 0;
+      auto issue_s = [&]() {
+        wait_or_give_up(&sh->k_full[s1], ph1, abortp, status, 114);
+        wait_or_give_up(&sh->s_free[b1], bph1 ^ 1, abortp, status, 115);
+        wait_or_give_up(&sh->l_free, (issued & 1) ^ 1, abortp, status, 116);
+        if (*abortp) return;
+        tc_fence_after_sync();
+        const uint64_t bd0 = bd_ring + (uint64_t)(s1 * (MF_STAGE_BYTES >> 4));
+#pragma unroll
+        for (int ks = 0; ks < kHeadDim / 16; ++ks)
+          mma_f16_ss(tmem + b1 * MF_TILE, ad_q + (uint64_t)((ks >> 2) * (MF_TILE_BYTES >> 5) + (ks & 3) * 2),
+                     bd0 + (uint64_t)((ks >> 2) * (MF_TILE_BYTES >> 5) + (ks & 3) * 2), idesc_s, ks ? 1u : 0u);
+        const uint64_t bp = bd_psi + (uint64_t)(s1 * (MF_OP_BYTES >> 4));
+        if (R == 8) {
+          mma_f16_ss(tmem + lcol, ad_phi, bp, idesc_s, 0u);                   // (hi, lo) x (hi, hi)
+          mma_f16_ss(tmem + lcol, ad_phi + kPair, bp + kPair, idesc_s, 1u);   // (hi, 0) x (lo, 0)
+        } else {
+          mma_f16_ss(tmem + lcol, ad_phi, bp, idesc_s, 0u);                   // hi x hi
+          mma_f16_ss(tmem + lcol, ad_phi + kPair, bp, idesc_s, 1u);           // lo x hi
+          mma_f16_ss(tmem + lcol, ad_phi, bp + kPair, idesc_s, 1u);           // hi x lo
+        }
+        mma_commit(&sh->k_empty[s1]);
+        mma_commit(&sh->s_full[b1]);
+        if (++s1 == MF_STAGES) { s1 = 0; ph1 ^= 1; }
+        if (b1 ^= 1, b1 == 0) bph1 ^= 1;
+        ++issued;
+      };
+      for (int u = 0; u < ntile && !*abortp; ++u) issue_s();   // first sweep: scores and kernel values only
+      issue_s();
+      uint32_t s2 = 0, vph = 0, pph = 0;
+      for (int t = 0; t < ntile && !*abortp; ++t) {
+        if (issued < 2 * ntile) issue_s();             // the next tile's scores run ahead of this tile's P V
+        wait_or_give_up(&sh->v_full[s2], vph, abortp, status, 117);
+        wait_or_give_up(&sh->p_full, pph, abortp, status, 118);
+        if (*abortp) break;
+        pph ^= 1;
+        tc_fence_after_sync();
+        const uint64_t bv0 = bd_vring + (uint64_t)(s2 * (MF_STAGE_BYTES >> 4));
+#pragma unroll
+        for (int ks = 0; ks < MF_TILE / 16; ++ks)
+          mma_f16_ss(tmem + ocol, ad_p + (uint64_t)((ks >> 2) * (MF_TILE_BYTES >> 5) + (ks & 3) * 2),
+                     bv0 + (uint64_t)(ks * (2048 >> 4)), idesc_o, (t | ks) ? 1u : 0u);
+        mma_commit(&sh->p_free);
+        mma_commit(&sh->v_empty[s2]);
+        if (++s2 == MF_STAGES) { s2 = 0; vph ^= 1; }
+      }
+      mma_commit(&sh->o_full);
+    }
+  } else {
+    // ---------------- epilogue warps: lane = query row, the two warps of a quadrant split the keys ----------------
+    const int quad = warp & 3, half = (warp - 2) >> 2;
+    const int r = quad * 32 + lane, i = i0 + r;
+    const uint32_t lane_addr = tmem + ((uint32_t)(quad * 32) << 16);
+    unsigned char* prow = pbuf + half * (MF_TILE_BYTES / 2) + r * 128;   // this row's 64 keys of the half
+    float nb = p.a.ws_nb[rc0 + i], gi = p.a.ws_g[rc0 + i];
+    float rsum = 0.f;
+    uint32_t b = 0, bph = 0;
+    for (int u = 0; u < 2 * ntile; ++u) {
+      const bool second = u >= ntile;
+      const int t = second ? u - ntile : u;
+      if (u == ntile) {
+        // between the sweeps: the row's sum against the plain normaliser becomes its normaliser
+        sh->rsum[half][r] = rsum;
+        mf_epi_sync();
+        const float total = sh->rsum[0][r] + sh->rsum[1][r];
+        mf_epi_sync();                                   // rsum is used again at the end
+        if (total > 0.f && total < INFINITY) {
+          nb -= log2f(total);
+          gi /= total;
+        }
+        rsum = 0.f;
+      }
+      wait_or_give_up(&sh->s_full[b], bph, abortp, status, 119);
+      const int es = u % MF_EU_SLOTS;
+      wait_or_give_up(&sh->eu_full[es], (u / MF_EU_SLOTS) & 1, abortp, status, 120);
+      tc_fence_after_sync();
+      const int j0 = t * MF_TILE + half * 64;
+      const int2* eu2 = reinterpret_cast<const int2*>(euring + es * MF_EU_BYTES) + half * 32;
+      const bool diag = t == ntile - 1;
+      uint32_t pk[32];
+#pragma unroll
+      for (int hh = 0; hh < 2; ++hh) {
+        uint32_t v[32], w[32];
+        tmem_ld32(lane_addr + b * MF_TILE + half * 64 + hh * 32, v);
+        tmem_ld32(lane_addr + lcol + half * 64 + hh * 32, w);
+        tmem_ld_wait();
+        if (hh == 1) {                                   // both accumulators of this tile are in registers
+          tc_fence_before_sync();
+          mbar_arrive_warp(&sh->s_free[b]);
+          mbar_arrive_warp(&sh->l_free);
+        }
+#pragma unroll
+        for (int e = 0; e < 16; ++e) {
+          const int2 eu = eu2[hh * 16 + e];
+          const int j = j0 + hh * 32 + 2 * e;
+          float p0 = i < eu.x ? mf_ex2(fmaf(__uint_as_float(v[2 * e]), kMfExpScale, nb)) : __uint_as_float(w[2 * e]) * gi;
+          float p1 = i < eu.y ? mf_ex2(fmaf(__uint_as_float(v[2 * e + 1]), kMfExpScale, nb))
+                              : __uint_as_float(w[2 * e + 1]) * gi;
+          if (diag) {
+            p0 = j <= i ? p0 : 0.f;
+            p1 = j + 1 <= i ? p1 : 0.f;
+          }
+          rsum += p0 + p1;
+          const __half2 h = __floats2half2_rn(p0, p1);
+          pk[hh * 16 + e] = *reinterpret_cast<const uint32_t*>(&h);
+        }
+      }
+      mbar_arrive_warp(&sh->eu_empty[es]);
+      if (second) {
+        wait_or_give_up(&sh->p_free, (t & 1) ^ 1, abortp, status, 121);   // the previous tile's P V has read P
+#pragma unroll
+        for (int ch = 0; ch < 8; ++ch)                 // 16-byte chunk ch of the row, 128-byte swizzle
+          *reinterpret_cast<uint4*>(prow + ((ch ^ (r & 7)) << 4)) =
+              make_uint4(pk[ch * 4], pk[ch * 4 + 1], pk[ch * 4 + 2], pk[ch * 4 + 3]);
+        fence_proxy_async_smem();
+        mbar_arrive_warp(&sh->p_full);
+      }
+      if (b ^= 1, b == 0) bph ^= 1;
+    }
+    // ---- the row's normaliser: both halves' sums ----
+    sh->rsum[half][r] = rsum;
+    mf_epi_sync();
+    const float total = sh->rsum[0][r] + sh->rsum[1][r];
+    const float inv = total > 0.f ? 1.0f / total : 0.f;
+    // ---- the finished rows: O[row][64 columns of this warp] / r_i ----
+    wait_or_give_up(&sh->o_full, 0, abortp, status, 122);
+    tc_fence_after_sync();
+    float* orow = mf.out + (im.in_row0 + i) * kHeadDim + half * 64;
+#pragma unroll 1
+    for (int cg = 0; cg < 2; ++cg) {
+      uint32_t o[32];
+      tmem_ld32(lane_addr + ocol + half * 64 + cg * 32, o);
+      tmem_ld_wait();
+      if (i < p.S && !*abortp) {
+#pragma unroll
+        for (int e = 0; e < 32; e += 4)
+          *reinterpret_cast<float4*>(orow + cg * 32 + e) =
+              make_float4(__uint_as_float(o[e]) * inv, __uint_as_float(o[e + 1]) * inv,
+                          __uint_as_float(o[e + 2]) * inv, __uint_as_float(o[e + 3]) * inv);
+      }
+    }
+  }
+  drain_after_abort(abortp);
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 1) tmem_dealloc(tmem, 512);
+}
+
+int launch_masked_form(less_ctx* c, int layer0, int nl, int lj0, int layer_count, int S, const void* Q,
+                       const void* K, const void* V, const int32_t* exact_until, void* out, cudaStream_t s) {
+  const Dims& d = c->d;
+  if (!score_tc_supported() || !psi_tc_supported(d) || c->score_path != 1) return LESS_ERR_INVALID_CONFIG;
+  PfParams p;
+  p.Q = (const __half*)Q; p.K = (const __half*)K; p.V = (const __half*)V;
+  p.attn_out = nullptr;
+  p.a = c->a;
+  p.w_psi1 = (const __half*)c->w.w_psi1;
+  p.w_psi2 = (const __half*)c->w.w_psi2;
+  p.w_psi3 = (const __half*)c->w.w_psi3;
+  p.psi_scale = c->w.psi_scale;
+  p.S = S; p.Sp = d.Sp; p.Sbx = d.Sbx;
+  p.layer0 = layer0; p.nl = nl; p.lj0 = lj0; p.layer_count = layer_count;
+  p.B = d.B; p.L = d.L; p.Hd = d.Hd; p.N = d.N; p.Np = d.Np;
+  p.heavy = d.heavy; p.recent = d.recent; p.Rp = d.Rp;
+  p.flags = d.flags;
+  p.grp = 1;
+  const int G = d.B * nl * d.Hd;
+  // token splits of the MLP kernel, as in the prompt phase
+  int split_tokens = 1024;
+  while (split_tokens > 128 && (long long)G * ((S + split_tokens - 1) / split_tokens) < 148) split_tokens >>= 1;
+  if ((S + split_tokens - 1) / split_tokens > kMaxSplit)
+    split_tokens = ((S + kMaxSplit - 1) / kMaxSplit + 127) / 128 * 128;
+  p.nsplit = (S + split_tokens - 1) / split_tokens;
+  p.split_tokens = split_tokens;
+  MfParams mf;
+  mf.exact_until = exact_until;
+  mf.out = (float*)out;
+  mf.St = d.St;
+
+  int rc = launch_score_tc(c, p, G, s, false);           // m_i, 1 / l_i of the plain causal rows
+  if (rc != LESS_OK) return rc;
+  if (cudaMemsetAsync(c->a.ws_pmax, 0, (size_t)G * 4, s) != cudaSuccess) return fail_cuda("clearing the psi maxima");
+  rc = launch_psi_tc(c, p, G, s);
+  if (rc != LESS_OK) return rc;
+  rc = launch_phi_tc(c, p, G, s, c->a.ws_phi);
+  if (rc != LESS_OK) return rc;
+  const int tiles = (S + MF_TILE - 1) / MF_TILE;
+  {
+    LaunchScope scope(c, LESS_KERNEL_MASKED_PACK, s);
+    if (d.R == 8) masked_pack_kernel<8><<<dim3(tiles, G), MF_TILE, 0, s>>>(p, mf);
+    else masked_pack_kernel<16><<<dim3(tiles, G), MF_TILE, 0, s>>>(p, mf);
+  }
+  CUtensorMap tq, tk, tv;
+  const uint64_t rows = (uint64_t)d.B * layer_count * d.Hd * S;
+  if (!make_tmap_f16_2d(&tq, p.Q, rows, kHeadDim, kHeadDim * 2, MF_TILE) ||
+      !make_tmap_f16_2d(&tk, p.K, rows, kHeadDim, kHeadDim * 2, MF_TILE) ||
+      !make_tmap_f16_2d(&tv, p.V, rows, kHeadDim, kHeadDim * 2, MF_TILE))
+    return fail_cuda("tensor maps of Q / K / V");
+  const size_t smem = (size_t)MF_TILE_BYTES * 2 + MF_STAGES * MF_STAGE_BYTES + MF_OP_BYTES + MF_STAGES * MF_OP_BYTES +
+                      MF_EU_SLOTS * MF_EU_BYTES + sizeof(MfShared) + 1024;
+  LaunchScope scope(c, LESS_KERNEL_MASKED_OUT, s);
+  if (d.R == 8) {
+    if (cudaFuncSetAttribute(masked_out_tc_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+      return fail_cuda("shared memory opt-in of masked_out_tc_kernel");
+    masked_out_tc_kernel<8><<<dim3(tiles, G), MF_THREADS, smem, s>>>(tq, tk, tv, p, mf);
+  } else {
+    if (cudaFuncSetAttribute(masked_out_tc_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+      return fail_cuda("shared memory opt-in of masked_out_tc_kernel");
+    masked_out_tc_kernel<16><<<dim3(tiles, G), MF_THREADS, smem, s>>>(tq, tk, tv, p, mf);
+  }
+  return check_launch("the parallel-form kernels");
+}
+
+}  // namespace less

@@ -9,6 +9,8 @@
 //                   a single fp16 rounding of the hidden layer costs ~2e-3 on individual psi vectors)
 //   GEMM2  G2[128 x 16] += (hidden_hi + hidden_lo)[128 x 64] * W2[chunk rows, :]
 //   after 8 chunks: tcgen05.ld G2 -> c2 * gelu(c1 * .) -> W3 on CUDA cores -> abs -> psi[token][R]
+// The same kernel evaluates phi(q) = | gelu( gelu(q W1) W2 ) | (Eq. 1) over a sequence of queries for
+// the parallel form (PtMap::is_phi: no W3, no scalars, rows of Q).
 // Roles: warps 0-7 epilogue (lane quadrant = warp & 3, token row = tensor-memory lane; the two
 // warps of a quadrant split a chunk's 64 columns), warp 8 TMA producer, warp 9 MMA issuer.  Operands come in by TMA tiled loads with the 128-byte
 // swizzle (no multicast).  Every wait is bounded.
@@ -45,10 +47,19 @@ __device__ __forceinline__ void pt_wait(uint64_t* bar, uint32_t parity, volatile
   }
 }
 
+// which map: its layer-2 (and layer-3) weights, where the result goes
+struct PtMap {
+  const __half* w2;     // [L, Hd, Rp, R]
+  const __half* w3;     // [L, Hd, R, R], psi only
+  float* out;           // [Iw][Sp][R]
+  int32_t* pmax;        // [Iw] bit pattern of the largest value per instance, or null
+  int is_phi;
+};
+
 template <int R>
 __global__ void __launch_bounds__(PT_THREADS) psi_tc_kernel(const __grid_constant__ CUtensorMap tmap_k,
                                                             const __grid_constant__ CUtensorMap tmap_w1,
-                                                            PfParams p) {
+                                                            PfParams p, PtMap mp) {
   extern __shared__ __align__(1024) unsigned char pt_smem[];
   const int Rp = p.Rp;
   const int nchunk = Rp / PT_CHUNK;
@@ -78,21 +89,23 @@ __global__ void __launch_bounds__(PT_THREADS) psi_tc_kernel(const __grid_constan
     mbar_init(&sh->g2_free, PT_WORKERS / 32);
     // a CTA that starts after another one has given up skips every wait: the grid drains at once
     sh->abort = *reinterpret_cast<volatile int32_t*>(p.a.status) != 0;
-    sh->c1 = p.psi_scale ? p.psi_scale[im.lh * 2] : 1.f;
-    sh->c2 = p.psi_scale ? p.psi_scale[im.lh * 2 + 1] : 1.f;
+    sh->c1 = (p.psi_scale && !mp.is_phi) ? p.psi_scale[im.lh * 2] : 1.f;
+    sh->c2 = (p.psi_scale && !mp.is_phi) ? p.psi_scale[im.lh * 2 + 1] : 1.f;
     mbar_fence_init();
   }
   // W2 as the GEMM2 B operand (N padded to 16 with zeros), W3 as fp32
   {
-    const __half* w2 = p.w_psi2 + (size_t)im.lh * Rp * R;
+    const __half* w2 = mp.w2 + (size_t)im.lh * Rp * R;
     for (int e = tid; e < Rp * 2; e += PT_THREADS) {             // e = (k, nblock)
       const int k = e >> 1, nb = e & 1;
       uint4 v = make_uint4(0, 0, 0, 0);
       if (nb * 8 < R) v = __ldg(reinterpret_cast<const uint4*>(w2 + (size_t)k * R + nb * 8));
       *reinterpret_cast<uint4*>(w2s + (k >> 3) * 256 + nb * 128 + (k & 7) * 16) = v;
     }
-    const __half* w3 = p.w_psi3 + (size_t)im.lh * R * R;
-    for (int e = tid; e < R * R; e += PT_THREADS) sh->w3[e] = __half2float(w3[e]);
+    if (!mp.is_phi) {
+      const __half* w3 = mp.w3 + (size_t)im.lh * R * R;
+      for (int e = tid; e < R * R; e += PT_THREADS) sh->w3[e] = __half2float(w3[e]);
+    }
   }
   if (warp == PT_WORKERS / 32 + 1) tmem_alloc(&sh->tmem_base, 256);
   fence_proxy_async_smem();
@@ -169,7 +182,7 @@ __global__ void __launch_bounds__(PT_THREADS) psi_tc_kernel(const __grid_constan
     const int quad = warp & 3, half = warp >> 2;
     const int row = quad * 32 + (tid & 31);                         // token row of the tile = tensor-memory lane
     const uint32_t lane_addr = tmem + ((uint32_t)(quad * 32) << 16);
-    float* psi = p.a.ws_psi + (size_t)g * p.Sp * R;
+    float* psi = mp.out + (size_t)g * p.Sp * R;
     unsigned char* hrow = hid + row * 128;
     uint32_t q = 0;
     float pmax = 0.f;                                               // largest psi this thread has produced
@@ -226,9 +239,12 @@ __global__ void __launch_bounds__(PT_THREADS) psi_tc_kernel(const __grid_constan
         for (int r = 0; r < R; ++r) gv[r] = c2 * gelu_erf(c1 * __uint_as_float(g2[r]));
 #pragma unroll
         for (int r = 0; r < R; ++r) {
-          float s = 0.f;
+          float s = gv[r];                               // phi stops after the second layer (Eq. 1)
+          if (!mp.is_phi) {
+            s = 0.f;
 #pragma unroll
-          for (int rr = 0; rr < R; ++rr) s = fmaf(gv[rr], sh->w3[rr * R + r], s);
+            for (int rr = 0; rr < R; ++rr) s = fmaf(gv[rr], sh->w3[rr * R + r], s);
+          }
           out[r] = fabsf(s);
           pmax = fmaxf(pmax, out[r]);
         }
@@ -242,7 +258,7 @@ __global__ void __launch_bounds__(PT_THREADS) psi_tc_kernel(const __grid_constan
     // integer, and a maximum does not depend on the order of the atomics
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) pmax = fmaxf(pmax, __shfl_xor_sync(0xffffffffu, pmax, o));
-    if ((tid & 31) == 0 && pmax > 0.f && pmax < INFINITY) atomicMax(p.a.ws_pmax + g, __float_as_int(pmax));
+    if ((tid & 31) == 0 && mp.pmax && pmax > 0.f && pmax < INFINITY) atomicMax(mp.pmax + g, __float_as_int(pmax));
   }
   drain_after_abort(abortp);
   tc_fence_before_sync();
@@ -252,12 +268,14 @@ __global__ void __launch_bounds__(PT_THREADS) psi_tc_kernel(const __grid_constan
 
 bool psi_tc_supported(const Dims& d) { return d.Rp == 512 || d.Rp == 256 || d.Rp == 128 || d.Rp == 64; }
 
-int launch_psi_tc(less_ctx* c, const PfParams& p, int G, cudaStream_t s) {
+// x: the rows the map is applied to ([B, layer_count, Hd, S, D]); which = 0 phi (w_phi1, w_phi2 -> out), 1 psi
+static int launch_map_tc(less_ctx* c, const PfParams& p, int G, cudaStream_t s, const __half* x, const void* w1,
+                         const PtMap& mp) {
   const Dims& d = c->d;
   CUtensorMap tmap_k, tmap_w1;
   const uint64_t rows = (uint64_t)d.B * p.layer_count * d.Hd * p.S;
-  if (!make_tmap_f16_2d(&tmap_k, p.K, rows, kHeadDim, kHeadDim * 2, PT_TILE)) return fail_cuda("tensor map of K");
-  if (!make_tmap_f16_2d(&tmap_w1, p.w_psi1, (uint64_t)d.L * d.Hd * kHeadDim, d.Rp, (uint64_t)d.Rp * 2, kHeadDim))
+  if (!make_tmap_f16_2d(&tmap_k, x, rows, kHeadDim, kHeadDim * 2, PT_TILE)) return fail_cuda("tensor map of K");
+  if (!make_tmap_f16_2d(&tmap_w1, w1, (uint64_t)d.L * d.Hd * kHeadDim, d.Rp, (uint64_t)d.Rp * 2, kHeadDim))
     return fail_cuda("tensor map or shared memory opt-in");
   const size_t smem = (size_t)(d.Rp / PT_CHUNK) * 16384 + PT_KBYTES + 2 * 16384 + (size_t)d.Rp * PT_W2N * 2 +
                       sizeof(PtShared) + 64;
@@ -265,13 +283,26 @@ int launch_psi_tc(less_ctx* c, const PfParams& p, int G, cudaStream_t s) {
   if (d.R == 8) {
     if (cudaFuncSetAttribute(psi_tc_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
       return fail_cuda("tensor map or shared memory opt-in");
-    psi_tc_kernel<8><<<dim3(p.nsplit, G), PT_THREADS, smem, s>>>(tmap_k, tmap_w1, p);
+    psi_tc_kernel<8><<<dim3(p.nsplit, G), PT_THREADS, smem, s>>>(tmap_k, tmap_w1, p, mp);
   } else {
     if (cudaFuncSetAttribute(psi_tc_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
       return fail_cuda("tensor map or shared memory opt-in");
-    psi_tc_kernel<16><<<dim3(p.nsplit, G), PT_THREADS, smem, s>>>(tmap_k, tmap_w1, p);
+    psi_tc_kernel<16><<<dim3(p.nsplit, G), PT_THREADS, smem, s>>>(tmap_k, tmap_w1, p, mp);
   }
   return check_launch("psi_tc_kernel");
+}
+
+int launch_psi_tc(less_ctx* c, const PfParams& p, int G, cudaStream_t s) {
+  PtMap mp;
+  mp.w2 = p.w_psi2; mp.w3 = p.w_psi3; mp.out = p.a.ws_psi; mp.pmax = p.a.ws_pmax; mp.is_phi = 0;
+  return launch_map_tc(c, p, G, s, p.K, p.w_psi1, mp);
+}
+
+// phi(q_i) of every row of Q into `out` [Iw][Sp][R] (one query head per KV head)
+int launch_phi_tc(less_ctx* c, const PfParams& p, int G, cudaStream_t s, float* out) {
+  PtMap mp;
+  mp.w2 = (const __half*)c->w.w_phi2; mp.w3 = nullptr; mp.out = out; mp.pmax = nullptr; mp.is_phi = 1;
+  return launch_map_tc(c, p, G, s, p.Q, c->w.w_phi1, mp);
 }
 
 }  // namespace less

@@ -499,3 +499,103 @@ def test_grouped_query_heads_many_kv_heads_pick_the_row_sharing_kernel():
         tf.step(*wl.make_decode_inputs(w, s, DEV))
     assert tf.evictions == w.steps * len(inst) and ctx.poll_status() == 0
     ctx.close()
+
+
+# --------------------------------------------------------------------------- #
+# The parallel form (Section 3.2, Inexpensive Training; Section 4.1)
+# --------------------------------------------------------------------------- #
+def _schedule(w, kind, S, seed):
+    """exact_until [B, L, H, S] int32: 'random' = every key leaves a random number of steps after
+    its own (a tenth never leave), 'never', 'at_once' (only the diagonal stays exact)."""
+    g = torch.Generator().manual_seed(seed)
+    shape = (w.batch, w.layers, w.heads, S)
+    pos = torch.arange(S).expand(shape)
+    if kind == "never":
+        return torch.full(shape, 2**31 - 1, dtype=torch.int32)
+    if kind == "at_once":
+        return (pos + 1).to(torch.int32)
+    life = torch.randint(1, max(2, S // 3), shape, generator=g)
+    eu = pos + life
+    keep = torch.rand(shape, generator=g) < 0.1
+    return torch.where(keep, torch.full_like(eu, 2**31 - 1), eu).to(torch.int32)
+
+
+def _check_parallel_form(w, W, Q, K, V, eu, out, instances, psi_scale=None):
+    from oracle import less_oracle as lo
+    import harness
+    worst = 0.0
+    for inst in instances:
+        b, layer, head = wl.instance_coords(w, inst)
+        sc = None if psi_scale is None else psi_scale[layer, head].double().cpu().numpy()
+        phi_fn, psi_fn = lo.make_mlp_maps(*harness.head_weights(W, layer, head), sc)
+        ref, _ = lo.masked_parallel_attention(*(t[b, layer, head].double().cpu().numpy() for t in (Q, K, V)),
+                                              eu[b, layer, head].cpu().numpy(), phi_fn, psi_fn)
+        err = float(np.max(np.abs(out[b, layer, head].double().cpu().numpy() - ref)))
+        worst = max(worst, err)
+        assert err <= harness.OUT_TOL, f"inst {inst}: parallel form max-abs {err}"
+    return worst
+
+
+@pytest.mark.parametrize("kind,rank,S,std", [("random", 8, 300, 0.1), ("random", 16, 513, 0.2), ("never", 8, 131, 0.1),
+                                             ("at_once", 16, 257, 0.2), ("random", 8, 128, 0.3), ("random", 16, 40, 0.1)])
+def test_parallel_form_against_the_oracle(kind, rank, S, std):
+    from paper_2402_09398_b200 import binding
+    w = small(30 + rank, prompt=S, rank=rank, weight_std=std)
+    ctx, W = _setup(w, flags=binding.LESS_WITH_PARALLEL_FORM)
+    Q, K, V = wl.make_prompt(w, 0, w.layers, DEV)
+    eu = _schedule(w, kind, S, seed=S)
+    out = ctx.masked_attention(Q, K, V, eu.to(DEV))
+    torch.cuda.synchronize()
+    assert ctx.poll_status() == 0
+    worst = _check_parallel_form(w, W, Q, K, V, eu, out, list(range(w.instances)))
+    print("parallel form", kind, rank, S, worst)
+    ctx.close()
+
+
+def test_parallel_form_rows_equal_the_decode_steps():
+    """The library against itself through the paper's identity: with the schedule its own sequential
+    decode steps produced (evicted_pos), row i of the parallel form is the output of step i."""
+    from paper_2402_09398_b200 import binding
+    S = 150
+    w = small(29, prompt=0, steps=S, heavy=12, recent=12, weight_std=0.2)
+    ctx, W = _setup(w, flags=binding.LESS_WITH_PARALLEL_FORM, max_prompt=S)
+    qs, ks, vs, outs = [], [], [], []
+    eu = torch.full((w.batch, w.layers, w.heads, S), 2**31 - 1, dtype=torch.int32)
+    ev = torch.empty(w.instances, dtype=torch.int32, device=DEV)
+    for t in range(S):
+        q, k, v = wl.make_decode_inputs(w, t, DEV)
+        outs.append(ctx.decode_step(q, k, v, evicted_pos=ev).clone())
+        e = ev.cpu().reshape(w.batch, w.layers, w.heads)
+        idx = torch.nonzero(e >= 0, as_tuple=True)
+        eu[idx[0], idx[1], idx[2], e[idx].long()] = t + 1
+        qs.append(q); ks.append(k); vs.append(v)
+    Q, K, V = (torch.stack(x, dim=3).contiguous() for x in (qs, ks, vs))
+    seq = torch.stack(outs, dim=3)
+    par = ctx.masked_attention(Q, K, V, eu.to(DEV))
+    torch.cuda.synchronize()
+    assert ctx.poll_status() == 0
+    assert (eu != 2**31 - 1).sum() == (S - w.slots) * w.instances
+    err = float((par - seq).abs().max())
+    print("parallel vs sequential", err)
+    assert err <= 2e-3
+    ctx.close()
+
+
+def test_parallel_form_needs_its_flag_and_scaled_maps():
+    from paper_2402_09398_b200 import binding
+    w = small(28, prompt=200, weight_std=0.2)
+    ctx, W = _setup(w)
+    Q, K, V = wl.make_prompt(w, 0, w.layers, DEV)
+    eu = _schedule(w, "random", 200, 1).to(DEV)
+    with pytest.raises(binding.LessError):
+        ctx.masked_attention(Q, K, V, eu)                 # workspace not reserved
+    ctx.close()
+    # psi of the order of 1e4 and of 1e-4: the operands' power-of-two scales and the row factor w_i
+    for c in (40.0, 1e-4):
+        ps = torch.full((w.layers, w.heads, 2), c)
+        ctx, W = _setup(w, flags=binding.LESS_WITH_PARALLEL_FORM, psi_scale=ps)
+        out = ctx.masked_attention(Q, K, V, eu)
+        torch.cuda.synchronize()
+        assert ctx.poll_status() == 0
+        print("parallel form psi scale", c, _check_parallel_form(w, W, Q, K, V, eu.cpu(), out, [0, 5, w.instances - 1], ps))
+        ctx.close()
