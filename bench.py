@@ -61,6 +61,10 @@ def parse_args():
                     help="context run: TOVA as the sparse policy (same slot count)")
     ap.add_argument("--attn-out", action="store_true",
                     help="prompt compression: also produce the prompt's attention output (optional in less_prefill)")
+    ap.add_argument("--masked-form", action="store_true",
+                    help="context run: the parallel form (training / evaluation): sequences of --seq tokens, batch 2, "
+                         "32 heads, one layer per step")
+    ap.add_argument("--seq", type=int, default=4096, help="sequence length of --masked-form")
     ap.add_argument("--group", type=int, default=1, choices=[1, 2, 4, 8],
                     help="context run: grouped query heads, G query heads per KV head (query heads unchanged, "
                          "KV heads divided by G)")
@@ -594,10 +598,127 @@ def run_prefill(args):
     if world > 1:
         dist.destroy_process_group()
 
+def run_masked(args):
+    """The parallel form: a step = less_masked_attention over one layer (B x heads sequences)."""
+    import torch
+    import torch.distributed as dist
+    from paper_2402_09398_b200 import binding, build, workloads as wl
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the LESS path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = f"cuda:{local}"
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+    build.build()
+    S = args.seq
+    w = wl.CONFIGS[2].with_(batch=args.batch or 2, prompt=S, heavy=int(0.05 * S), recent=int(0.05 * S))
+    K_steps, W_steps = args.steps, max(args.warmup, 3)
+    Wt = wl.make_weights(w, dev)
+    ctx = binding.from_workload(w, Wt, dev, max_prefill_layers=1, flags=binding.LESS_WITH_PARALLEL_FORM)
+    Q, Kp, V = wl.make_prompt(w, 0, 1, dev)
+    # schedule: every key leaves between `recent` and `recent + 2 * slots` steps after its own
+    gen = torch.Generator(device=dev).manual_seed(1234)
+    pos = torch.arange(S, device=dev).expand(w.batch, 1, w.heads, S)
+    eu = (pos + w.recent + torch.randint(0, 2 * w.slots, pos.shape, generator=gen, device=dev)).to(torch.int32).contiguous()
+    out = torch.empty(Q.shape, dtype=torch.float32, device=dev)
+    stream = torch.cuda.current_stream()
+    step_no = [0]
+
+    def one_step():
+        ctx.masked_attention(Q, Kp, V, eu, layer_begin=step_no[0] % w.layers, out=out)
+        step_no[0] += 1
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(W_steps):
+        one_step()
+    barrier()
+    sampler = ClockSampler(local) if rank == 0 else None
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    launches0 = ctx.launches
+    t0 = time.time()
+    e0.record(stream)
+    for _ in range(K_steps):
+        one_step()
+    e1.record(stream)
+    barrier()
+    t1 = time.time()
+    launches = ctx.launches - launches0
+    ms = e0.elapsed_time(e1)
+    clocks = sampler.stop(t0, t1) if sampler else None
+    ctx.profile(True)
+    for _ in range(K_steps):
+        one_step()
+    torch.cuda.synchronize()
+    prof = ctx.profile_read()
+    ctx.profile(False)
+    # end to end: inputs from pinned host memory, the output read back
+    hq, hk, hv = (torch.empty(t.shape, dtype=torch.float16).pin_memory() for t in (Q, Kp, V))
+    heu = torch.empty(eu.shape, dtype=torch.int32).pin_memory()
+    hq.copy_(Q); hk.copy_(Kp); hv.copy_(V); heu.copy_(eu)
+    hout = torch.empty(out.shape, dtype=torch.float32).pin_memory()
+    dq, dk, dv, deu = torch.empty_like(Q), torch.empty_like(Kp), torch.empty_like(V), torch.empty_like(eu)
+    torch.cuda.synchronize()
+    tw0 = time.perf_counter()
+    n_e2e = max(1, min(K_steps, 3))
+    for _ in range(n_e2e):
+        dq.copy_(hq, non_blocking=True); dk.copy_(hk, non_blocking=True); dv.copy_(hv, non_blocking=True)
+        deu.copy_(heu, non_blocking=True)
+        ctx.masked_attention(dq, dk, dv, deu, layer_begin=0, out=out)
+        hout.copy_(out, non_blocking=True)
+    torch.cuda.synchronize()
+    ms_e2e = 1e3 * (time.perf_counter() - tw0) / n_e2e
+    if ctx.poll_status() != 0:
+        raise RuntimeError("device status")
+    ms, ms_e2e = max_over_ranks([ms, ms_e2e], dev, world)
+    if rank == 0:
+        inst = w.batch * w.heads
+        tokens = inst * S * world
+        causal = S * (S + 1) // 2
+        fl = {"masked_out": inst * causal * (4 * w.head_dim + 2 * w.rank), "rowstat": inst * causal * 2 * w.head_dim,
+              "psi": inst * S * 2 * (2 * w.head_dim * w.hidden + 2 * w.hidden * w.rank + w.rank * w.rank)}
+        kt = {k: (prof[k][0] / prof[k][1] if prof[k][1] else 0.0) for k in prof}
+        kt["psi"] *= 2                                   # psi and phi launches are booked under the same id
+        dominant = max(fl, key=lambda k: kt.get(k, 0.0))
+        pth = os.path.join(ROOT, "MEASURED_PEAKS.json")
+        peak, kind = (float(json.load(open(pth))["bf16_tflops_sustained"]), "of measured (sustained bf16 = fp16 rate)") \
+            if os.path.exists(pth) else (1400.0, "of fallback")
+        ach = fl[dominant] / (kt[dominant] * 1e-3) / 1e12 if kt.get(dominant) else 0.0
+        line = {"metric": "parallel-form head-tokens/s (one layer per step)", "value": tokens * K_steps / (ms * 1e-3),
+                "unit": "head-tokens/s", "n_gpus": world, "steps": K_steps, "warmup": W_steps, "ms_per_step": ms / K_steps,
+                "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+                "dtype": "f16 inputs, f32 accumulate", "data": "synthetic",
+                "config": {"workload": f"parallel form (B={w.batch}, {w.heads} heads, sequences of {S}, one layer per step, R={w.rank})",
+                           "instances_per_step": inst, "l2": "inputs, operands and output of a step exceed the 126 MB L2"
+                           if inst * S * 1300 > 126e6 else "a step's data fit the L2"},
+                "clocks": clocks,
+                "e2e": {"value": tokens / (ms_e2e * 1e-3), "unit": "head-tokens/s",
+                        "h2d_bytes_per_step": 3 * Q.numel() * 2 + eu.numel() * 4, "d2h_bytes_per_step": out.numel() * 4},
+                "gpu_launches": int(launches),
+                "roofline": {"bound": "tensor", "kernel": "masked_out_tc_kernel" if dominant == "masked_out" else dominant,
+                             "achieved": ach, "peak": peak, "unit": "TFLOP/s", "frac": ach / peak, "peak_kind": kind,
+                             "traffic": None, "algorithmic_flops_per_launch": fl[dominant],
+                             "kernel_ms": {k: v for k, v in kt.items() if v}}}
+        print(json.dumps(line))
+    ctx.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
 def main():
     args = parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.masked_form:
+        if args.steps == 1000:
+            args.steps = 20
+        run_masked(args)
     elif args.config == 5:
         if args.steps == 1000:
             args.steps = 5                # a step here is ~0.1 s of tensor-core work, not ~0.1 ms

@@ -198,3 +198,35 @@ def test_cfg2_grouped_query_heads_sampled_instances():
     print("cfg2 grouped decode", tf.worst)
     ctx.close()
     torch.cuda.empty_cache()
+
+
+def test_parallel_form_training_shape_sampled_instances():
+    """The parallel form at the shape `bench.py --masked-form` times (batch 2, 32 heads, sequences
+    of 4096, one layer per call): two whole instances against the oracle's S x S matrix."""
+    from oracle import less_oracle as lo
+    from paper_2402_09398_b200 import binding
+    import harness
+    S = 4096
+    w = wl.CONFIGS[2].with_(batch=2, prompt=S, heavy=204, recent=204)
+    W = wl.make_weights(w, DEV)
+    ctx = binding.from_workload(w, W, DEV, max_prefill_layers=1, flags=binding.LESS_WITH_PARALLEL_FORM)
+    layer = 7
+    Q, K, V = wl.make_prompt(w, layer, 1, DEV)
+    gen = torch.Generator(device=DEV).manual_seed(99)
+    pos = torch.arange(S, device=DEV).expand(w.batch, 1, w.heads, S)
+    eu = (pos + w.recent + torch.randint(0, 2 * w.slots, pos.shape, generator=gen, device=DEV)).to(torch.int32)
+    eu[:, :, :, ::97] = 2**31 - 1                         # some keys stay for good
+    eu = eu.contiguous()
+    out = ctx.masked_attention(Q, K, V, eu, layer_begin=layer)
+    torch.cuda.synchronize()
+    assert ctx.poll_status() == 0
+    for b, head in ((0, 3), (1, 31)):
+        wts = [W[n][layer, head].double().cpu().numpy() for n in ("w_phi1", "w_phi2", "w_psi1", "w_psi2", "w_psi3")]
+        phi_fn, psi_fn = lo.make_mlp_maps(*wts)
+        ref, _ = lo.masked_parallel_attention(*(t[b, 0, head].double().cpu().numpy() for t in (Q, K, V)),
+                                              eu[b, 0, head].cpu().numpy(), phi_fn, psi_fn)
+        err = float(np.max(np.abs(out[b, 0, head].double().cpu().numpy() - ref)))
+        print("parallel form 4096", b, head, err)
+        assert err <= harness.OUT_TOL
+    ctx.close()
+    torch.cuda.empty_cache()
