@@ -681,7 +681,7 @@ def run_masked(args):
         inst = w.batch * w.heads
         tokens = inst * S * world
         causal = S * (S + 1) // 2
-        fl = {"masked_out": inst * causal * (4 * w.head_dim + 2 * w.rank), "rowstat": inst * causal * 2 * w.head_dim,
+        fl = {"masked_out": inst * causal * (4 * w.head_dim + 2 * w.rank),
               "psi": inst * S * 2 * (2 * w.head_dim * w.hidden + 2 * w.hidden * w.rank + w.rank * w.rank)}
         kt = {k: (prof[k][0] / prof[k][1] if prof[k][1] else 0.0) for k in prof}
         kt["psi"] *= 2                                   # psi and phi launches are booked under the same id

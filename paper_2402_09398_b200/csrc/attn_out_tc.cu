@@ -8,7 +8,7 @@
 //
 // One CTA = one 128-row Q tile.  Per 128-key tile:
 //   S = Q K^T - b 1^T      tcgen05, fp32 in tensor memory (double-buffered)
-//   P = exp2(c S)           eight epilogue warps (lane = query row), causal test on the diagonal tile,
+//   P = exp2(c S)           sixteen epilogue warps (lane = query row), causal test on the diagonal tile,
 //                           rounded to fp16 and stored as the K-major A operand of
 //   O += P V                tcgen05, fp32 accumulator [128 x 128] in tensor memory
 // P is a probability (<= 1) rounded once to fp16 (relative 4.9e-4 per element, independent signs):
@@ -19,9 +19,9 @@
 
 namespace less {
 
-constexpr int AO_EPI_WARPS = 8;
+constexpr int AO_EPI_WARPS = 16;                    // four per lane quadrant: with two, the tensor-memory loads and the P hand-over were exposed
 constexpr int AO_EPI_THREADS = AO_EPI_WARPS * 32;
-constexpr int AO_THREADS = 64 + AO_EPI_THREADS + 32;   // warp 0 TMA (Q, K), warp 1 MMA, warps 2..9 epilogue, warp 10 TMA (V)
+constexpr int AO_THREADS = 64 + AO_EPI_THREADS + 32;   // warp 0 TMA (Q, K), warp 1 MMA, warps 2..17 epilogue, warp 18 TMA (V)
 constexpr int AO_TILE = 128;                        // query rows per CTA and keys per streamed tile
 constexpr int AO_TILE_BYTES = AO_TILE * kHeadDim * 2;
 constexpr int AO_STAGES = 2;
@@ -124,7 +124,7 @@ __global__ void __launch_bounds__(AO_THREADS) attn_out_tc_kernel(const __grid_co
         if (++s == AO_STAGES) { s = 0; ph ^= 1; }
       }
     }
-  } else if (warp == 10) {
+  } else if (warp == 2 + AO_EPI_WARPS) {
     // ---------------- TMA producer of the V tiles ----------------
     if (lane == 0) {
       uint32_t s = 0, ph = 0;
@@ -191,26 +191,27 @@ __global__ void __launch_bounds__(AO_THREADS) attn_out_tc_kernel(const __grid_co
       mma_commit(&sh->o_full);
     }
   } else {
-    // ---------------- epilogue warps: lane = query row, the two warps of a quadrant split the keys ----------------
-    const int quad = warp & 3, half = (warp - 2) >> 2;
+    // ---------------- epilogue warps: lane = query row, the four warps of a quadrant split the keys ----------------
+    const int quad = warp & 3, part = (warp - 2) >> 2;               // part: 32 of the tile's 128 keys
     const int r = quad * 32 + lane, i = i0 + r;
     const uint32_t lane_addr = tmem + ((uint32_t)(quad * 32) << 16);
-    unsigned char* prow = pbuf + half * (AO_TILE_BYTES / 2) + r * 128;   // this row's 64 keys of the half
+    // P: [2 key halves][128 rows][128 B]; this thread's 32 keys are 4 of the 8 chunks of its row in one half
+    unsigned char* prow = pbuf + (part >> 1) * (AO_TILE_BYTES / 2) + r * 128;
+    const int ch0 = (part & 1) * 4;
     uint32_t b = 0, bph = 0;
     for (int t = 0; t < ntile; ++t) {
       wait_or_give_up(&sh->s_full[b], bph, abortp, status, 105);
       tc_fence_after_sync();
-      uint32_t v[64];
-      tmem_ld32(lane_addr + b * AO_TILE + half * 64, v);
-      tmem_ld32(lane_addr + b * AO_TILE + half * 64 + 32, v + 32);
+      uint32_t v[32];
+      tmem_ld32(lane_addr + b * AO_TILE + part * 32, v);
       tmem_ld_wait();
       tc_fence_before_sync();
       mbar_arrive_warp(&sh->s_free[b]);
-      const int j0 = t * AO_TILE + half * 64;
-      uint32_t pk[32];
+      const int j0 = t * AO_TILE + part * 32;
+      uint32_t pk[16];
       if (t == ntile - 1) {                            // the tile that holds the diagonal
 #pragma unroll
-        for (int e = 0; e < 32; ++e) {
+        for (int e = 0; e < 16; ++e) {
           const float p0 = j0 + 2 * e <= i ? ao_ex2(__uint_as_float(v[2 * e]) * kAoExpScale) : 0.f;
           const float p1 = j0 + 2 * e + 1 <= i ? ao_ex2(__uint_as_float(v[2 * e + 1]) * kAoExpScale) : 0.f;
           const __half2 h = __floats2half2_rn(p0, p1);
@@ -218,7 +219,7 @@ __global__ void __launch_bounds__(AO_THREADS) attn_out_tc_kernel(const __grid_co
         }
       } else {
 #pragma unroll
-        for (int e = 0; e < 32; ++e) {
+        for (int e = 0; e < 16; ++e) {
           const __half2 h = __floats2half2_rn(ao_ex2(__uint_as_float(v[2 * e]) * kAoExpScale),
                                               ao_ex2(__uint_as_float(v[2 * e + 1]) * kAoExpScale));
           pk[e] = *reinterpret_cast<const uint32_t*>(&h);
@@ -226,26 +227,25 @@ __global__ void __launch_bounds__(AO_THREADS) attn_out_tc_kernel(const __grid_co
       }
       wait_or_give_up(&sh->p_free, (t & 1) ^ 1, abortp, status, 106);   // the previous tile's P V has read P
 #pragma unroll
-      for (int ch = 0; ch < 8; ++ch)                   // 16-byte chunk ch of the row, 128-byte swizzle
-        *reinterpret_cast<uint4*>(prow + ((ch ^ (r & 7)) << 4)) =
-            make_uint4(pk[ch * 4], pk[ch * 4 + 1], pk[ch * 4 + 2], pk[ch * 4 + 3]);
+      for (int c = 0; c < 4; ++c)                      // 16-byte chunk ch0 + c of the row, 128-byte swizzle
+        *reinterpret_cast<uint4*>(prow + (((ch0 + c) ^ (r & 7)) << 4)) =
+            make_uint4(pk[c * 4], pk[c * 4 + 1], pk[c * 4 + 2], pk[c * 4 + 3]);
       fence_proxy_async_smem();
       mbar_arrive_warp(&sh->p_full);
       if (b ^= 1, b == 0) bph ^= 1;
     }
-    // ---- the finished rows: O[row][64 columns of this warp] ----
+    // ---- the finished rows: O[row][32 columns of this warp] ----
     wait_or_give_up(&sh->o_full, 0, abortp, status, 107);
     tc_fence_after_sync();
-    float* orow = p.attn_out + (qm.q_row0 + i) * kHeadDim + half * 64;
-#pragma unroll 1
-    for (int cg = 0; cg < 2; ++cg) {
+    float* orow = p.attn_out + (qm.q_row0 + i) * kHeadDim + part * 32;
+    {
       uint32_t o[32];
-      tmem_ld32(lane_addr + ocol + half * 64 + cg * 32, o);
+      tmem_ld32(lane_addr + ocol + part * 32, o);
       tmem_ld_wait();
       if (i < p.S && !*abortp) {
 #pragma unroll
         for (int e = 0; e < 32; e += 4)
-          *reinterpret_cast<float4*>(orow + cg * 32 + e) =
+          *reinterpret_cast<float4*>(orow + e) =
               make_float4(__uint_as_float(o[e]), __uint_as_float(o[e + 1]), __uint_as_float(o[e + 2]),
                           __uint_as_float(o[e + 3]));
       }

@@ -100,7 +100,6 @@ size_t carve(const Dims& d, char* base, Arena* a) {
   t.ws_phiop = (unsigned char*)take(Iw * St * 8192);
   t.ws_psiop = (unsigned char*)take(Iw * St * 8192);
   t.ws_g = (float*)take(Iw * St * 128 * 4);
-  t.ws_nb = (float*)take(Iw * St * 128 * 4);
   t.ws_eu = (int32_t*)take(Iw * St * 128 * 4);
   if (a) *a = t;
   return off;

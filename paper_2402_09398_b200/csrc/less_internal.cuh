@@ -46,8 +46,7 @@ struct Arena {
   float* ws_phi;     // [Iw][Sp][R]  phi(q_i) of every row
   unsigned char* ws_phiop;  // [Iw][St][8 KB]  phi as fp16 hi / lo operand tiles
   unsigned char* ws_psiop;  // [Iw][St][8 KB]  psi likewise
-  float* ws_g;       // [Iw][St*128]  per row: factor of the low-rank entries
-  float* ws_nb;      // [Iw][St*128]  per row: exponent offset of the exact entries
+  float* ws_g;       // [Iw][St*128]  per row: log2 of (kernel value / value of the scaled operands)
   int32_t* ws_eu;    // [Iw][St*128]  exact_until, padded with zeros
   uint4* ws_bx;      // [Iw*G][Sbx]  per prompt row: -(m_i sqrt(D) - log2(1/l_i) / c) as three fp16 parts (column sums)
 };

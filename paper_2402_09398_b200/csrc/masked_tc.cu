@@ -6,25 +6,21 @@
 //            phi(q_i) psi(k_j)^T          otherwise                      (j <= i)
 //     out_i = sum_j A_ij v_j / sum_j A_ij
 //
-// Steps (launch_masked_form): the row statistics m_i, 1 / l_i of the plain causal softmax
-// (rowstat_tc_kernel) serve as each row's reference; psi(K) and phi(Q) come from the MLP kernel
-// (psi_tc.cu); masked_pack_kernel turns them into fp16 hi / lo operand tiles and computes the
-// per-row constants; masked_out_tc_kernel then works like the prompt-output kernel, with a second
-// accumulator:
+// Steps (launch_masked_form): psi(K) and phi(Q) come from the MLP kernel (psi_tc.cu);
+// masked_pack_kernel scales them by powers of two (phi per row, psi per instance), splits them into
+// fp16 hi + lo and writes them as operand tiles; masked_out_tc_kernel then works like the
+// prompt-output kernel, with a second accumulator:
 //   S = Q K^T                       tcgen05, fp32 in tensor memory (double-buffered)
 //   L = phi~ psi~^T                 tcgen05, hi hi + lo hi + hi lo of the scaled fp16 splits
-//   P_ij = i < exact_until[j] ? exp2(c S_ij + nb_i) : L_ij g_i       (epilogue warps, lane = row)
+//   P_ij = i < exact_until[j] ? exp2(c S_ij - E_i) : L_ij 2^(lscale_i - E_i)     (epilogue warps, lane = row)
 //   O += P V                        tcgen05;   r_i += sum_j P_ij (fp32, before rounding P to fp16)
 //   out_i = O_i / r_i
-// The key tiles stream past the Q tile twice.  The first sweep only adds up each row's entries in
-// fp32: a row whose dominant key has been discarded keeps a tiny share of the plain softmax's
-// mass, and its entries would sink into fp16's subnormals if P were formed against the plain
-// normaliser.  The second sweep divides by that sum first, so P holds the row's true
-// probabilities when it is rounded to fp16 for P V.
-// nb_i = -m_i log2(e) + log2(1 / l_i) + log2(w_i) makes the exact entries the plain softmax
-// probabilities times w_i, and g_i carries the same factors plus the operands' power-of-two scales.
-// w_i <= 1 is a power of two chosen from the bound  L_ij <= max(psi) sum_r phi_ir  so that no
-// entry of P exceeds 1 before it is rounded to fp16; it cancels in O_i / r_i.
+// The key tiles stream past the Q tile twice.  The first sweep only takes maxima: the row's largest
+// exact dot product and its largest kernel value give E_i = log2 of the row's largest entry.  The
+// second sweep forms P against it, so every entry is at most 1 and the largest is 1 when P is
+// rounded to fp16 for P V, whatever share of the plain softmax's mass the policy has left exact
+// (a row whose dominant key has been discarded keeps ~1e-6 of it: formed against the plain
+// normaliser its entries would sink into fp16's subnormals).
 // Every wait is bounded (pipeline.cuh).
 #include "prefill.cuh"
 #include "tc_common.cuh"
@@ -38,11 +34,10 @@ constexpr int MF_EU_BYTES = MF_TILE * 4;
 constexpr int MF_STAGES = 2;
 constexpr int MF_EU_SLOTS = 4;                      // exact_until tiles in flight: the epilogue frees them, later than the K stage
 constexpr int MF_STAGE_BYTES = 2 * MF_TILE_BYTES;   // K tile, then V tile
-constexpr int MF_EPI_WARPS = 8;
+constexpr int MF_EPI_WARPS = 16;                   // four per lane quadrant, 32 keys of a tile each
 constexpr int MF_EPI_THREADS = MF_EPI_WARPS * 32;
-constexpr int MF_THREADS = 64 + MF_EPI_THREADS + 32;   // warp 0 TMA (Q, K, operands), warp 1 MMA, warps 2..9 epilogue, warp 10 TMA (V)
+constexpr int MF_THREADS = 64 + MF_EPI_THREADS + 32;   // warp 0 TMA (Q, K, operands), warp 1 MMA, warps 2..17 epilogue, warp 18 TMA (V)
 constexpr float kMfExpScale = 0.12751743074602468f; // log2(e) / sqrt(128)
-constexpr float kLog2e = 1.4426950408889634f;
 
 struct MfParams {
   const int32_t* exact_until;   // [B, layer_count, Hd, S]
@@ -101,11 +96,10 @@ __global__ void __launch_bounds__(MF_TILE) masked_pack_kernel(PfParams p, MfPara
       ps[4 * e] = y.x; ps[4 * e + 1] = y.y; ps[4 * e + 2] = y.z; ps[4 * e + 3] = y.w;
     }
   }
-  float phmax = 0.f, phsum = 0.f;
+  float phmax = 0.f;
 #pragma unroll
   for (int e = 0; e < R; ++e) {
     phmax = fmaxf(phmax, ph[e]);
-    phsum += ph[e];
   }
   const float ephi = pow2_scale_exponent(phmax);
 
@@ -129,27 +123,10 @@ __global__ void __launch_bounds__(MF_TILE) masked_pack_kernel(PfParams p, MfPara
     so[0] = sh_[0]; so[CH] = sh_[R / 8 - 1]; so[2 * CH] = sl[0]; so[3 * CH] = sl[R / 8 - 1];
   }
 
-  // row constants
-  float nb = -60000.f, gi = 0.f;
-  int eu = 0;
-  if (valid) {
-    const float m = p.a.ws_m[(size_t)g * p.Sp + i];
-    const float il = p.a.ws_invl[(size_t)g * p.Sp + i];
-    const float base = fmaf(-m, kLog2e, log2f(il));      // log2 of e^{-m} / l
-    float lw = 0.f;                                      // log2 w_i
-    const float bound = pmax * phsum;                    // >= every phi(q_i) psi(k_j)^T of the row
-    if (bound > 0.f && bound < INFINITY) {
-      const float lb = log2f(bound) + base;
-      if (lb > 0.f) lw = -ceilf(lb);
-    }
-    nb = base + lw;
-    gi = exp2f(fminf(nb - ephi - epsi, 120.f));
-    eu = mf.exact_until[im.in_row0 + i];
-  }
+  // what turns a scaled kernel value back into phi(q_i) psi(k_j)^T, as a power of two; the key's mask
   const size_t row = (size_t)g * mf.St * MF_TILE + i;
-  p.a.ws_nb[row] = nb;
-  p.a.ws_g[row] = gi;
-  p.a.ws_eu[row] = eu;
+  p.a.ws_g[row] = -(ephi + epsi);
+  p.a.ws_eu[row] = valid ? mf.exact_until[im.in_row0 + i] : 0;
 }
 
 // ------------------------------------------------------------------------------------------- //
@@ -166,7 +143,8 @@ struct MfShared {
   uint64_t o_full;
   uint32_t tmem_base;
   int abort;
-  float rsum[2][MF_TILE];
+  float rsum[4][MF_TILE];
+  float rmax[4][MF_TILE];
 };
 
 __device__ __forceinline__ float mf_ex2(float x) {
@@ -259,7 +237,7 @@ __global__ void __launch_bounds__(MF_THREADS) masked_out_tc_kernel(const __grid_
         if (++s == MF_STAGES) { s = 0; ph ^= 1; }
       }
     }
-  } else if (warp == 10) {
+  } else if (warp == 2 + MF_EPI_WARPS) {
     // ---------------- producer of the V tiles ----------------
     if (lane == 0) {
       uint32_t s = 0, ph = 0;
@@ -338,52 +316,100 @@ __global__ void __launch_bounds__(MF_THREADS) masked_out_tc_kernel(const __grid_
       mma_commit(&sh->o_full);
     }
   } else {
-    // ---------------- epilogue warps: lane = query row, the two warps of a quadrant split the keys ----------------
-    const int quad = warp & 3, half = (warp - 2) >> 2;
+    // ---------------- epilogue warps: lane = query row, the four warps of a quadrant split the keys ----------------
+    const int quad = warp & 3, part = (warp - 2) >> 2;               // part: 32 of the tile's 128 keys
     const int r = quad * 32 + lane, i = i0 + r;
     const uint32_t lane_addr = tmem + ((uint32_t)(quad * 32) << 16);
-    unsigned char* prow = pbuf + half * (MF_TILE_BYTES / 2) + r * 128;   // this row's 64 keys of the half
-    float nb = p.a.ws_nb[rc0 + i], gi = p.a.ws_g[rc0 + i];
-    float rsum = 0.f;
+    // P: [2 key halves][128 rows][128 B]; this thread's 32 keys are 4 of the 8 chunks of its row in one half
+    unsigned char* prow = pbuf + (part >> 1) * (MF_TILE_BYTES / 2) + r * 128;
+    const int ch0 = (part & 1) * 4;
+    // sweep 1: the row's largest exact dot product and largest kernel value (scaled operands);
+    // sweep 2: P against the largest entry, so that every entry is <= 1 and the largest is 1
+    const float lscale = p.a.ws_g[rc0 + i];            // log2 of (true kernel value / scaled kernel value)
+    const bool live = i < p.S;
+    float mx = -INFINITY, ml = 0.f;
+    float nb = 0.f, gi = 0.f, rsum = 0.f, rsum2 = 0.f;
     uint32_t b = 0, bph = 0;
     for (int u = 0; u < 2 * ntile; ++u) {
       const bool second = u >= ntile;
       const int t = second ? u - ntile : u;
       if (u == ntile) {
-        // between the sweeps: the row's sum against the plain normaliser becomes its normaliser
-        sh->rsum[half][r] = rsum;
+        // between the sweeps: E = log2 of the row's largest entry; exact entries become
+        // exp2(c S - E), kernel entries L 2^(lscale - E)
+        sh->rsum[part][r] = mx;
+        sh->rmax[part][r] = ml;
         mf_epi_sync();
-        const float total = sh->rsum[0][r] + sh->rsum[1][r];
+        mx = fmaxf(fmaxf(sh->rsum[0][r], sh->rsum[1][r]), fmaxf(sh->rsum[2][r], sh->rsum[3][r]));
+        ml = fmaxf(fmaxf(sh->rmax[0][r], sh->rmax[1][r]), fmaxf(sh->rmax[2][r], sh->rmax[3][r]));
         mf_epi_sync();                                   // rsum is used again at the end
-        if (total > 0.f && total < INFINITY) {
-          nb -= log2f(total);
-          gi /= total;
+        const float ea = mx * kMfExpScale;               // -inf without exact entries
+        const float el = ml > 0.f ? log2f(ml) + lscale : -INFINITY;
+        const float E = fmaxf(ea, el);
+        if (live && E > -INFINITY && E < INFINITY) {
+          nb = -E;
+          gi = exp2f(fminf(lscale - E, 120.f));
+        } else {                                         // a row past the sequence, or one with nothing in it: all zeros
+          nb = -INFINITY;
+          gi = 0.f;
         }
-        rsum = 0.f;
       }
       wait_or_give_up(&sh->s_full[b], bph, abortp, status, 119);
       const int es = u % MF_EU_SLOTS;
       wait_or_give_up(&sh->eu_full[es], (u / MF_EU_SLOTS) & 1, abortp, status, 120);
       tc_fence_after_sync();
-      const int j0 = t * MF_TILE + half * 64;
-      const int2* eu2 = reinterpret_cast<const int2*>(euring + es * MF_EU_BYTES) + half * 32;
+      const int j0 = t * MF_TILE + part * 32;
+      const int4* eu4 = reinterpret_cast<const int4*>(euring + es * MF_EU_BYTES) + part * 8;
       const bool diag = t == ntile - 1;
-      uint32_t pk[32];
+      uint32_t pk[16];
+      uint32_t v[32], w[32];
+      tmem_ld32(lane_addr + b * MF_TILE + part * 32, v);
+      tmem_ld32(lane_addr + lcol + part * 32, w);
+      tmem_ld_wait();
+      tc_fence_before_sync();                            // both accumulators of this tile are in registers
+      mbar_arrive_warp(&sh->s_free[b]);
+      mbar_arrive_warp(&sh->l_free);
+      if (!second) {
+        // four independent chains per maximum
+        float a0 = -INFINITY, a1 = -INFINITY, a2 = -INFINITY, a3 = -INFINITY, l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
+        if (diag) {
 #pragma unroll
-      for (int hh = 0; hh < 2; ++hh) {
-        uint32_t v[32], w[32];
-        tmem_ld32(lane_addr + b * MF_TILE + half * 64 + hh * 32, v);
-        tmem_ld32(lane_addr + lcol + half * 64 + hh * 32, w);
-        tmem_ld_wait();
-        if (hh == 1) {                                   // both accumulators of this tile are in registers
-          tc_fence_before_sync();
-          mbar_arrive_warp(&sh->s_free[b]);
-          mbar_arrive_warp(&sh->l_free);
+          for (int e = 0; e < 8; ++e) {
+            const int4 eu = eu4[e];
+            const int j = j0 + 4 * e;
+            const bool x0 = i < eu.x, x1 = i < eu.y, x2 = i < eu.z, x3 = i < eu.w;
+            const bool c0 = j <= i, c1 = j + 1 <= i, c2 = j + 2 <= i, c3 = j + 3 <= i;     // causal
+            a0 = fmaxf(a0, (c0 && x0) ? __uint_as_float(v[4 * e]) : -INFINITY);
+            a1 = fmaxf(a1, (c1 && x1) ? __uint_as_float(v[4 * e + 1]) : -INFINITY);
+            a2 = fmaxf(a2, (c2 && x2) ? __uint_as_float(v[4 * e + 2]) : -INFINITY);
+            a3 = fmaxf(a3, (c3 && x3) ? __uint_as_float(v[4 * e + 3]) : -INFINITY);
+            l0 = fmaxf(l0, (c0 && !x0) ? __uint_as_float(w[4 * e]) : 0.f);
+            l1 = fmaxf(l1, (c1 && !x1) ? __uint_as_float(w[4 * e + 1]) : 0.f);
+            l2 = fmaxf(l2, (c2 && !x2) ? __uint_as_float(w[4 * e + 2]) : 0.f);
+            l3 = fmaxf(l3, (c3 && !x3) ? __uint_as_float(w[4 * e + 3]) : 0.f);
+          }
+        } else {
+#pragma unroll
+          for (int e = 0; e < 8; ++e) {
+            const int4 eu = eu4[e];
+            const bool x0 = i < eu.x, x1 = i < eu.y, x2 = i < eu.z, x3 = i < eu.w;
+            a0 = fmaxf(a0, x0 ? __uint_as_float(v[4 * e]) : -INFINITY);
+            a1 = fmaxf(a1, x1 ? __uint_as_float(v[4 * e + 1]) : -INFINITY);
+            a2 = fmaxf(a2, x2 ? __uint_as_float(v[4 * e + 2]) : -INFINITY);
+            a3 = fmaxf(a3, x3 ? __uint_as_float(v[4 * e + 3]) : -INFINITY);
+            l0 = fmaxf(l0, x0 ? 0.f : __uint_as_float(w[4 * e]));
+            l1 = fmaxf(l1, x1 ? 0.f : __uint_as_float(w[4 * e + 1]));
+            l2 = fmaxf(l2, x2 ? 0.f : __uint_as_float(w[4 * e + 2]));
+            l3 = fmaxf(l3, x3 ? 0.f : __uint_as_float(w[4 * e + 3]));
+          }
         }
+        mx = fmaxf(mx, fmaxf(fmaxf(a0, a1), fmaxf(a2, a3)));
+        ml = fmaxf(ml, fmaxf(fmaxf(l0, l1), fmaxf(l2, l3)));
+      } else {
+        const int2* eu2 = reinterpret_cast<const int2*>(eu4);
 #pragma unroll
         for (int e = 0; e < 16; ++e) {
-          const int2 eu = eu2[hh * 16 + e];
-          const int j = j0 + hh * 32 + 2 * e;
+          const int2 eu = eu2[e];
+          const int j = j0 + 2 * e;
           float p0 = i < eu.x ? mf_ex2(fmaf(__uint_as_float(v[2 * e]), kMfExpScale, nb)) : __uint_as_float(w[2 * e]) * gi;
           float p1 = i < eu.y ? mf_ex2(fmaf(__uint_as_float(v[2 * e + 1]), kMfExpScale, nb))
                               : __uint_as_float(w[2 * e + 1]) * gi;
@@ -391,41 +417,40 @@ __global__ void __launch_bounds__(MF_THREADS) masked_out_tc_kernel(const __grid_
             p0 = j <= i ? p0 : 0.f;
             p1 = j + 1 <= i ? p1 : 0.f;
           }
-          rsum += p0 + p1;
+          if (e & 1) rsum2 += p0 + p1; else rsum += p0 + p1;
           const __half2 h = __floats2half2_rn(p0, p1);
-          pk[hh * 16 + e] = *reinterpret_cast<const uint32_t*>(&h);
+          pk[e] = *reinterpret_cast<const uint32_t*>(&h);
         }
       }
       mbar_arrive_warp(&sh->eu_empty[es]);
       if (second) {
         wait_or_give_up(&sh->p_free, (t & 1) ^ 1, abortp, status, 121);   // the previous tile's P V has read P
 #pragma unroll
-        for (int ch = 0; ch < 8; ++ch)                 // 16-byte chunk ch of the row, 128-byte swizzle
-          *reinterpret_cast<uint4*>(prow + ((ch ^ (r & 7)) << 4)) =
-              make_uint4(pk[ch * 4], pk[ch * 4 + 1], pk[ch * 4 + 2], pk[ch * 4 + 3]);
+        for (int c = 0; c < 4; ++c)                    // 16-byte chunk ch0 + c of the row, 128-byte swizzle
+          *reinterpret_cast<uint4*>(prow + (((ch0 + c) ^ (r & 7)) << 4)) =
+              make_uint4(pk[c * 4], pk[c * 4 + 1], pk[c * 4 + 2], pk[c * 4 + 3]);
         fence_proxy_async_smem();
         mbar_arrive_warp(&sh->p_full);
       }
       if (b ^= 1, b == 0) bph ^= 1;
     }
-    // ---- the row's normaliser: both halves' sums ----
-    sh->rsum[half][r] = rsum;
+    // ---- the row's normaliser: the four parts' sums ----
+    sh->rsum[part][r] = rsum + rsum2;
     mf_epi_sync();
-    const float total = sh->rsum[0][r] + sh->rsum[1][r];
+    const float total = (sh->rsum[0][r] + sh->rsum[1][r]) + (sh->rsum[2][r] + sh->rsum[3][r]);
     const float inv = total > 0.f ? 1.0f / total : 0.f;
-    // ---- the finished rows: O[row][64 columns of this warp] / r_i ----
+    // ---- the finished rows: O[row][32 columns of this warp] / r_i ----
     wait_or_give_up(&sh->o_full, 0, abortp, status, 122);
     tc_fence_after_sync();
-    float* orow = mf.out + (im.in_row0 + i) * kHeadDim + half * 64;
-#pragma unroll 1
-    for (int cg = 0; cg < 2; ++cg) {
+    float* orow = mf.out + (im.in_row0 + i) * kHeadDim + part * 32;
+    {
       uint32_t o[32];
-      tmem_ld32(lane_addr + ocol + half * 64 + cg * 32, o);
+      tmem_ld32(lane_addr + ocol + part * 32, o);
       tmem_ld_wait();
       if (i < p.S && !*abortp) {
 #pragma unroll
         for (int e = 0; e < 32; e += 4)
-          *reinterpret_cast<float4*>(orow + cg * 32 + e) =
+          *reinterpret_cast<float4*>(orow + e) =
               make_float4(__uint_as_float(o[e]) * inv, __uint_as_float(o[e + 1]) * inv,
                           __uint_as_float(o[e + 2]) * inv, __uint_as_float(o[e + 3]) * inv);
       }
@@ -468,8 +493,7 @@ int launch_masked_form(less_ctx* c, int layer0, int nl, int lj0, int layer_count
   mf.out = (float*)out;
   mf.St = d.St;
 
-  int rc = launch_score_tc(c, p, G, s, false);           // m_i, 1 / l_i of the plain causal rows
-  if (rc != LESS_OK) return rc;
+  int rc;
   if (cudaMemsetAsync(c->a.ws_pmax, 0, (size_t)G * 4, s) != cudaSuccess) return fail_cuda("clearing the psi maxima");
   rc = launch_psi_tc(c, p, G, s);
   if (rc != LESS_OK) return rc;
