@@ -433,7 +433,7 @@ def run_b200(args):
                         + f"<{w.rank}" + (f", {1 if w.batch <= 1 else 2 if w.batch <= 2 else 4 if w.batch <= 4 else 8}>"
                                           if w.batch <= 8 else ">"),
                         "decode": (f"decode_kernel<{w.rank}, {1 if args.graph else 0}>" if w.group == 1 else
-                                   f"decode_group_kernel<{w.rank}, {w.group}, {1 if args.graph else 0}>")}
+                                   f"decode_group_mma_kernel<{w.rank}, {w.group}, {1 if args.graph else 0}>")}
         ach = kb[dominant] / (kt[dominant] * 1e-3) / 1e9 if kt[dominant] > 0 else 0.0
         step_bytes = kb["feature_map"] + kb["decode"]
         kv_state_bytes = w.instances * (n_live * (4 * w.head_dim + 8) + (0 if args.no_state else 2 * w.rank * w.head_dim * 4))

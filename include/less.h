@@ -27,9 +27,10 @@
  *     LESS_NO_OVERLAP (no programmatic dependent launch of the decode kernel),
  *     LESS_SCORE_KERNEL=plain (CUDA-core prompt scoring),
  *     LESS_FEATURE_STAGES=n (cap on the feature kernels' weight ring),
- *     LESS_GROUP_KERNEL=teams|rows (grouped query heads: force the decode kernel with
- *     one 128-thread team per query head, or the one with one 128-thread CTA per KV
- *     head; by default the number of KV heads per multiprocessor decides).
+ *     LESS_GROUP_KERNEL=teams|rows|mma (grouped query heads: force the decode kernel with
+ *     one 128-thread team per query head, the one with one 128-thread CTA per KV head on
+ *     CUDA cores, or that one with its two contractions as warp-level tensor-core
+ *     products; by default the number of KV heads per multiprocessor picks teams or mma).
  */
 #ifndef LESS_B200_H
 #define LESS_B200_H

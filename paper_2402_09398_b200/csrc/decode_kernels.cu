@@ -848,15 +848,347 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_group_rows_kernel(DecParam
   step_done<kCaptured>(p.a.tpos, p.t);
 }
 
+// The same step with the two contractions on the tensor cores.  With G query heads per KV head the
+// scores are a [slots x 128] x [128 x G] product and the numerators a [128 x slots] x [slots x G] one:
+// dense, but only G <= 8 wide and bound by the K / V stream, so the warp-level mma (m16n8k16, fp16
+// inputs used exactly, fp32 accumulation, N = 8 = the heads) fits: its fragments load straight from
+// global memory with no staging, four warps split the 16-slot tiles.  The probabilities enter the
+// second product rounded to fp16 (relative 4.9e-4, like the prompt-output kernel); the H2O scores
+// use the fp32 values.
+__device__ __forceinline__ void mma_m16n8k16(float* d, uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                             uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+      "{%0, %1, %2, %3};"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+__device__ __forceinline__ uint32_t word_of(const uint4& v, int w) {
+  return w == 0 ? v.x : w == 1 ? v.y : w == 2 ? v.z : v.w;
+}
+
+template <int R, int G, bool kCaptured>
+__global__ void __launch_bounds__(DEC_THREADS) decode_group_mma_kernel(DecParams p) {
+  extern __shared__ float dsm[];
+  const int Ns = p.Np + 4;
+  float* s_sc = dsm;                               // [G][Np + 4] scores, then e^{s - m_g}
+  float* s_red = s_sc + G * Ns;                    // [G][DEC_RG][128] partial numerators
+  __shared__ float s_small[DEC_THREADS / 32];
+  __shared__ unsigned long long s_key[DEC_THREADS / 32];
+  __shared__ int s_vic;
+  __shared__ float s_inv[G];
+
+  const int tid = threadIdx.x;
+  const size_t inst = blockIdx.x;
+  const int l16 = tid & 15, rg = tid >> 4;
+  const int N = p.N;
+  const int t_now = kCaptured ? __ldcg(p.a.tpos) : p.t;
+  int n = p.a.count[inst];
+  if (n < 0 || n > N) {
+    if (tid == 0) set_status(p.a.status, kStatusBounds, 1);
+    step_done<kCaptured>(p.a.tpos, p.t);
+    return;
+  }
+  const bool use_state = !(p.flags & LESS_NO_STATE);
+  const float scale = 0.08838834764831845f;        // 1 / sqrt(128)
+
+  const __half* Kb = p.a.kslots + inst * (size_t)N * kHeadDim;
+  const __half* Vb = p.a.vslots + inst * (size_t)N * kHeadDim;
+
+  const int warp = tid >> 5, lane = tid & 31;
+  const int fg = lane >> 2, ft = lane & 3;         // fragment coordinates of mma.m16n8k16: row group, thread in group
+  constexpr int Ng = G;
+  // ---- scores: S[16 slots x 8 heads] += K[16 slots x 16 dims] Q^T[16 dims x 8 heads], 8 k-steps per tile ----
+  // The contraction does not care which dims a k-slot stands for, as long as both operands agree:
+  // thread ft takes the 16-byte chunks ft, ft + 4, ft + 8, ft + 12 of a row, so every load is a
+  // whole chunk and a warp reads its 16 rows (4 KB) exactly once.
+  uint4 qfrag[4];                                  // B fragments: head fg, this thread's chunks
+#pragma unroll
+  for (int c = 0; c < 4; ++c)
+    qfrag[c] = fg < Ng ? *reinterpret_cast<const uint4*>(p.q + (inst * G + fg) * kHeadDim + (ft + 4 * c) * 8)
+                       : make_uint4(0, 0, 0, 0);
+  const int ntile16 = (n + 15) >> 4;
+  for (int tl = warp; tl < ntile16; tl += DEC_THREADS / 32) {
+    const int r0 = tl * 16 + fg, r1 = r0 + 8;
+    const int c0 = min(r0, n - 1), c1 = min(r1, n - 1);        // rows past the live slots repeat the last one; their scores are dropped
+    uint4 ka[4], kb[4];
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      ka[c] = ldg_stream(Kb + (size_t)c0 * kHeadDim + (ft + 4 * c) * 8);
+      kb[c] = ldg_stream(Kb + (size_t)c1 * kHeadDim + (ft + 4 * c) * 8);
+    }
+    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      mma_m16n8k16(acc, ka[c].x, kb[c].x, ka[c].y, kb[c].y, qfrag[c].x, qfrag[c].y);
+      mma_m16n8k16(acc, ka[c].z, kb[c].z, ka[c].w, kb[c].w, qfrag[c].z, qfrag[c].w);
+    }
+    // acc: (slot r0, head 2 ft), (r0, 2 ft + 1), (r1, 2 ft), (r1, 2 ft + 1)
+    if (2 * ft < Ng) {
+      if (r0 < n) s_sc[(2 * ft) * Ns + r0] = acc[0] * scale;
+      if (r1 < n) s_sc[(2 * ft) * Ns + r1] = acc[2] * scale;
+    }
+    if (2 * ft + 1 < Ng) {
+      if (r0 < n) s_sc[(2 * ft + 1) * Ns + r0] = acc[1] * scale;
+      if (r1 < n) s_sc[(2 * ft + 1) * Ns + r1] = acc[3] * scale;
+    }
+  }
+  const uint4 knew = *reinterpret_cast<const uint4*>(p.k + inst * kHeadDim + l16 * 8);
+  const uint4 vnew = *reinterpret_cast<const uint4*>(p.v + inst * kHeadDim + l16 * 8);
+  if (tid < 32) {
+    float kf[8];
+    half8_to_float(knew, kf);
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+      float qf[8];
+      half8_to_float(*reinterpret_cast<const uint4*>(p.q + (inst * G + g) * kHeadDim + l16 * 8), qf);
+      float dot = 0.f;
+#pragma unroll
+      for (int c = 0; c < 8; ++c) dot = fmaf(qf[c], kf[c], dot);
+#pragma unroll
+      for (int o = 8; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+      if (tid == 0) s_sc[g * Ns + n] = dot * scale;
+    }
+  }
+  __syncthreads();
+
+  // ---- per head: m_g, e_i = exp(s_i - m_g), l_g ----
+  float mg[G], lg[G];
+  if (G >= DEC_THREADS / 32) {                      // a warp takes whole heads: no block barrier per head
+    __shared__ float s_ml[2][G];
+    for (int g = warp; g < G; g += DEC_THREADS / 32) {
+      float* sc = s_sc + g * Ns;
+      float m = -INFINITY;
+      for (int i = lane; i <= n; i += 32) m = fmaxf(m, sc[i]);
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+      m = fmaxf(m, -80.f);
+      float lsum = 0.f;
+      for (int i = lane; i <= n; i += 32) {
+        const float e = __expf(sc[i] - m);
+        sc[i] = e;
+        lsum += e;
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) lsum += __shfl_xor_sync(0xffffffffu, lsum, o);   // fixed order
+      if (lane == 0) { s_ml[0][g] = m; s_ml[1][g] = lsum; }
+    }
+    __syncthreads();
+#pragma unroll
+    for (int g = 0; g < G; ++g) { mg[g] = s_ml[0][g]; lg[g] = s_ml[1][g]; }
+  } else {                                          // fewer heads than warps: the whole CTA works on each
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+      float* sc = s_sc + g * Ns;
+      float m = -INFINITY;
+      for (int i = tid; i <= n; i += DEC_THREADS) m = fmaxf(m, sc[i]);
+      m = block_max(m, s_small);
+      m = fmaxf(m, -80.f);
+      float lsum = 0.f;
+      for (int i = tid; i <= n; i += DEC_THREADS) {
+        const float e = __expf(sc[i] - m);
+        sc[i] = e;
+        lsum += e;
+      }
+      mg[g] = m;
+      lg[g] = block_sum(lsum, s_small);
+    }
+  }
+
+  // ---- O^T[16 dims x 8 heads] += V^T[16 dims x 16 slots] P^T[16 slots x 8 heads], 8 tiles of dims per 16 slots ----
+  // A fragment row fg of tile m stands for dim 8 fg + m, row fg + 8 for dim 8 (fg + 8) + m: a thread
+  // loads the chunks fg and fg + 8 of its four slots (k-slots 2 ft, 2 ft + 1, 2 ft + 8, 2 ft + 9)
+  // and pairs the halves of two slots with a byte permute; again every byte is loaded once.
+  float oacc[8][4];
+#pragma unroll
+  for (int m = 0; m < 8; ++m)
+#pragma unroll
+    for (int x = 0; x < 4; ++x) oacc[m][x] = 0.f;
+  for (int tl = warp; tl < ntile16; tl += DEC_THREADS / 32) {
+    const int base = tl * 16 + 2 * ft;
+    const int rr[4] = {base, base + 1, base + 8, base + 9};
+    uint4 va[4], vb[4];
+#pragma unroll
+    for (int x = 0; x < 4; ++x) {
+      const int row = min(rr[x], n - 1);
+      va[x] = ldg_stream(Vb + (size_t)row * kHeadDim + fg * 8);
+      vb[x] = ldg_stream(Vb + (size_t)row * kHeadDim + (fg + 8) * 8);
+    }
+    uint32_t b0 = 0u, b1 = 0u;                     // B fragment: head fg, this thread's four slots (zero past the live ones)
+    if (fg < Ng) {
+      const float* sc = s_sc + fg * Ns;
+      const __half2 h0 = __floats2half2_rn(rr[0] < n ? sc[rr[0]] : 0.f, rr[1] < n ? sc[rr[1]] : 0.f);
+      const __half2 h1 = __floats2half2_rn(rr[2] < n ? sc[rr[2]] : 0.f, rr[3] < n ? sc[rr[3]] : 0.f);
+      b0 = *reinterpret_cast<const uint32_t*>(&h0);
+      b1 = *reinterpret_cast<const uint32_t*>(&h1);
+    }
+#pragma unroll
+    for (int m = 0; m < 8; ++m) {
+      const int w = m >> 1;
+      const uint32_t sel = (m & 1) ? 0x7632u : 0x5410u;      // the high or the low halves of two words
+      mma_m16n8k16(oacc[m], __byte_perm(word_of(va[0], w), word_of(va[1], w), sel),
+                   __byte_perm(word_of(vb[0], w), word_of(vb[1], w), sel),
+                   __byte_perm(word_of(va[2], w), word_of(va[3], w), sel),
+                   __byte_perm(word_of(vb[2], w), word_of(vb[3], w), sel), b0, b1);
+    }
+  }
+  // oacc[m]: (dim 8 fg + m, head 2 ft), (same, 2 ft + 1), (dim 8 (fg + 8) + m, head 2 ft), (same, 2 ft + 1)
+  // partial numerators: rows 0..3 of s_red per head are the warps', row 4 the new pair's, the rest zero
+#pragma unroll
+  for (int m = 0; m < 8; ++m) {
+    const int d0 = 8 * fg + m, d1 = 8 * (fg + 8) + m;
+    if (2 * ft < Ng) {
+      s_red[((2 * ft) * DEC_RG + warp) * kHeadDim + d0] = oacc[m][0];
+      s_red[((2 * ft) * DEC_RG + warp) * kHeadDim + d1] = oacc[m][2];
+    }
+    if (2 * ft + 1 < Ng) {
+      s_red[((2 * ft + 1) * DEC_RG + warp) * kHeadDim + d0] = oacc[m][1];
+      s_red[((2 * ft + 1) * DEC_RG + warp) * kHeadDim + d1] = oacc[m][3];
+    }
+  }
+  {
+    const float vn = __half2float(p.v[inst * kHeadDim + tid]);
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+      s_red[(g * DEC_RG + 4) * kHeadDim + tid] = s_sc[g * Ns + n] * vn;
+#pragma unroll
+      for (int j = 5; j < DEC_RG; ++j) s_red[(g * DEC_RG + j) * kHeadDim + tid] = 0.f;
+    }
+  }
+  __syncthreads();
+
+  // ---- Eq. 3 per head over the shared H, z ----
+  const int d = tid;
+  float* Hb = p.a.H + inst * (size_t)R * kHeadDim;
+  float* zb = p.a.z + inst * R;
+  float hcol[R], zr[R];
+  if (use_state) {
+    pdl_wait_primary();
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+      hcol[r] = Hb[r * kHeadDim + d];
+      zr[r] = zb[r];
+    }
+  }
+#pragma unroll
+  for (int g = 0; g < G; ++g) {
+    float num = 0.f;
+#pragma unroll
+    for (int j = 0; j < DEC_RG; ++j) num += s_red[(g * DEC_RG + j) * kHeadDim + d];
+    float den = lg[g];
+    if (use_state) {
+      const float em = __expf(-mg[g]);
+      const float* ph = p.a.phi_q + (inst * G + g) * R;
+      float lr = 0.f, lz = 0.f;
+#pragma unroll
+      for (int r = 0; r < R; ++r) {
+        const float f = ph[r];
+        lr = fmaf(f, hcol[r], lr);
+        lz = fmaf(f, zr[r], lz);
+      }
+      num = fmaf(em, lr, num);
+      den = fmaf(em, lz, den);
+    }
+    p.out[(inst * G + g) * kHeadDim + d] = num / den;
+    if (tid == 0) s_inv[g] = 1.0f / ((p.flags & LESS_SCORE_NORM_SPARSE) ? lg[g] : den);
+  }
+  __syncthreads();
+  float inv[G];
+#pragma unroll
+  for (int g = 0; g < G; ++g) inv[g] = s_inv[g];
+
+  // ---- H2O over the group: acc_i += sum_g p_{g,i}; one victim for all heads ----
+  int32_t* posb = p.a.pos + inst * (size_t)p.Np;
+  float* accb = p.a.acc + inst * (size_t)p.Np;
+  const bool full = (n == N);
+  const bool lambda_policy = (p.flags & LESS_POLICY_LAMBDA) != 0;
+  unsigned long long best = ~0ull;
+  for (int i = tid; i < n; i += DEC_THREADS) {
+    float ps_sum = 0.f;
+#pragma unroll
+    for (int g = 0; g < G; ++g) ps_sum = fmaf(s_sc[g * Ns + i], inv[g], ps_sum);
+    const float a = accb[i] + ps_sum;
+    accb[i] = a;
+    if (full) {
+      const int ps = posb[i];
+      if (lambda_policy) {
+        if (ps >= p.heavy) best = (unsigned long long)(unsigned int)ps < best ? (unsigned int)ps : best;
+      } else if (ps <= t_now - p.recent) {
+        const unsigned long long key =
+            ((unsigned long long)__float_as_uint(a) << 32) | (unsigned int)ps;
+        best = key < best ? key : best;
+      }
+    }
+  }
+  float p_new = 0.f;
+#pragma unroll
+  for (int g = 0; g < G; ++g) p_new = fmaf(s_sc[g * Ns + n], inv[g], p_new);
+  int slot = n;
+  if (full) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const unsigned long long other = __shfl_xor_sync(0xffffffffu, best, o);
+      best = other < best ? other : best;
+    }
+    if ((tid & 31) == 0) s_key[tid >> 5] = best;
+    if (tid == 0) s_vic = -1;
+    __syncthreads();
+    best = s_key[0];
+#pragma unroll
+    for (int w = 1; w < DEC_THREADS / 32; ++w) best = s_key[w] < best ? s_key[w] : best;
+    const int vpos = (int)(unsigned int)(best & 0xffffffffull);
+    for (int i = tid; i < n; i += DEC_THREADS)
+      if (posb[i] == vpos && best != ~0ull) s_vic = i;
+    __syncthreads();
+    slot = s_vic;
+    if (slot < 0) {
+      if (tid == 0) {
+        set_status(p.a.status, kStatusBounds, 2);
+        if (p.evicted_pos) p.evicted_pos[inst] = -1;
+      }
+      step_done<kCaptured>(p.a.tpos, p.t);
+      return;
+    }
+    if (tid == 0 && p.evicted_pos) p.evicted_pos[inst] = vpos;
+    if (use_state) {                               // Eq. 4 / Eq. 5: psi acts on the key, the state is the KV head's
+      const float vv = __half2float(Vb[(size_t)slot * kHeadDim + d]);
+      const float* psv = p.a.psic + (inst * (size_t)N + slot) * R;
+#pragma unroll
+      for (int r = 0; r < R; ++r) Hb[r * kHeadDim + d] = fmaf(psv[r], vv, hcol[r]);
+      if (tid < R) zb[tid] += psv[tid];
+    }
+    __syncthreads();
+  } else {
+    if (tid == 0) {
+      p.a.count[inst] = n + 1;
+      if (p.evicted_pos) p.evicted_pos[inst] = -1;
+    }
+  }
+  __half* Kw = p.a.kslots + (inst * (size_t)N + slot) * kHeadDim;
+  __half* Vw = p.a.vslots + (inst * (size_t)N + slot) * kHeadDim;
+  if (rg == 0) *reinterpret_cast<uint4*>(Kw + l16 * 8) = knew;
+  if (rg == 1) *reinterpret_cast<uint4*>(Vw + l16 * 8) = vnew;
+  if (tid == 32) { posb[slot] = t_now; accb[slot] = p_new; }
+  if (tid >= 64 && tid < 64 + R)
+    p.a.psic[(inst * (size_t)N + slot) * R + (tid - 64)] =
+        use_state ? p.a.psi_k[inst * R + (tid - 64)] : 0.f;
+  step_done<kCaptured>(p.a.tpos, p.t);
+}
+
+
 size_t decode_smem_bytes(const Dims& d) {
   return (size_t)d.G * (d.Np + 4 + DEC_RG * kHeadDim) * 4;
 }
 
-// teams: one 128-thread team per query head (few KV heads, latency matters); else one 128-thread CTA per KV head
+// which: 1 a 128-thread team per query head (few KV heads, latency matters), 2 one 128-thread CTA per KV
+// head on CUDA cores, 3 the same with the contractions on the tensor cores
 template <int R, int G>
-static void* decode_group_entry(bool captured, bool teams) {
-  if (teams) return captured ? (void*)decode_group_kernel<R, G, true> : (void*)decode_group_kernel<R, G, false>;
-  return captured ? (void*)decode_group_rows_kernel<R, G, true> : (void*)decode_group_rows_kernel<R, G, false>;
+static void* decode_group_entry(bool captured, int which) {
+  if (which == 1) return captured ? (void*)decode_group_kernel<R, G, true> : (void*)decode_group_kernel<R, G, false>;
+  if (which == 2)
+    return captured ? (void*)decode_group_rows_kernel<R, G, true> : (void*)decode_group_rows_kernel<R, G, false>;
+  return captured ? (void*)decode_group_mma_kernel<R, G, true> : (void*)decode_group_mma_kernel<R, G, false>;
 }
 
 int launch_decode(less_ctx* c, const void* q, const void* k, const void* v, void* out,
@@ -879,10 +1211,12 @@ int launch_decode(less_ctx* c, const void* q, const void* k, const void* v, void
                         : (captured ? (void*)decode_kernel<16, true> : (void*)decode_kernel<16, false>);
   // grouped query heads: with fewer KV heads than two per SM a CTA's latency is the step's, and the
   // heads of a group run side by side (128 threads each); with more, throughput per SM counts
-  const bool teams = d.G > 1 && (c->group_path == 1 || (c->group_path == 0 && d.I < 2 * c->sms));
-  if (d.G == 2) kern = d.R == 8 ? decode_group_entry<8, 2>(captured, teams) : decode_group_entry<16, 2>(captured, teams);
-  if (d.G == 4) kern = d.R == 8 ? decode_group_entry<8, 4>(captured, teams) : decode_group_entry<16, 4>(captured, teams);
-  if (d.G == 8) kern = d.R == 8 ? decode_group_entry<8, 8>(captured, teams) : decode_group_entry<16, 8>(captured, teams);
+  int which = c->group_path;
+  if (which == 0) which = 3;
+  const bool teams = d.G > 1 && which == 1;
+  if (d.G == 2) kern = d.R == 8 ? decode_group_entry<8, 2>(captured, which) : decode_group_entry<16, 2>(captured, which);
+  if (d.G == 4) kern = d.R == 8 ? decode_group_entry<8, 4>(captured, which) : decode_group_entry<16, 4>(captured, which);
+  if (d.G == 8) kern = d.R == 8 ? decode_group_entry<8, 8>(captured, which) : decode_group_entry<16, 8>(captured, which);
   if (smem > 48 * 1024 &&
       cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
     return fail_cuda("shared memory opt-in of decode_kernel");

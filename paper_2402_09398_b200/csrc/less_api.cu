@@ -189,6 +189,7 @@ int less_create(const less_config* cfg, const less_weights* w, void* arena, size
   if (const char* e = getenv("LESS_GROUP_KERNEL")) {
     if (!strcmp(e, "teams")) c->group_path = 1;
     else if (!strcmp(e, "rows")) c->group_path = 2;
+    else if (!strcmp(e, "mma")) c->group_path = 3;
   }
   c->sms = 148;
   cudaDeviceGetAttribute(&c->sms, cudaDevAttrMultiProcessorCount, c->device);

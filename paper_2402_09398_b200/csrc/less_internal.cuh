@@ -80,7 +80,7 @@ struct less_ctx {
   int feature_stages;  // cap on the feature kernels' ring stages (LESS_FEATURE_STAGES), 0 = default
   int score_path;      // prompt scoring: 1 tensor cores, 0 CUDA cores (LESS_SCORE_KERNEL=plain)
   int feature_path;    // feature-map kernel: 2 tensor cores, 1 streaming GEMV, 0 plain (LESS_FEATURE_KERNEL)
-  int group_path;      // grouped decode kernel: 0 by instance count, 1 a team per query head, 2 one CTA per KV head (LESS_GROUP_KERNEL)
+  int group_path;      // grouped decode kernel: 0 by instance count, 1 a team per query head, 2 one CTA per KV head on CUDA cores, 3 with warp-level mma (LESS_GROUP_KERNEL)
   bool profile;                         // record an event pair around every launch
   std::vector<cudaEvent_t> prof_events; // start, stop, start, stop, ...
   std::vector<int> prof_kernel;         // kernel id of each pair

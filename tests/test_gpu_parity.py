@@ -423,7 +423,7 @@ def test_captured_step_replays_with_grouped_query_heads():
     test_captured_step_replays_like_direct_calls(3, group=4)
 
 
-@pytest.mark.parametrize("kernel", ["teams", "rows"])
+@pytest.mark.parametrize("kernel", ["teams", "rows", "mma"])
 @pytest.mark.parametrize("group,rank,flags", [(2, 8, 0), (4, 16, 0), (8, 8, 0), (4, 8, 4), (2, 16, 1), (4, 8, 2)])
 def test_grouped_query_heads_decode_from_empty(group, rank, flags, kernel, monkeypatch):
     """Section 3.2, multi-query attention: G query heads share one KV head's cache, scores and
@@ -485,9 +485,9 @@ def test_grouped_query_heads_rejected_configurations(monkeypatch):
         binding.from_workload(small(39, group=8, heavy=4000, recent=4000), W, DEV)   # scores of 8 heads x 8000 slots exceed shared memory
 
 
-def test_grouped_query_heads_many_kv_heads_pick_the_row_sharing_kernel():
-    """More than two KV heads per multiprocessor: the default choice is the decode kernel with one
-    128-thread CTA per KV head (K / V rows loaded once, G queries in registers)."""
+def test_grouped_query_heads_many_kv_heads_after_a_prompt():
+    """Several KV heads per multiprocessor, ragged slot tiles (24 slots = one and a half 16-slot
+    tiles of the default grouped decode kernel), on top of a prompt phase."""
     import harness
     w = small(38, batch=11, layers=3, heads=10, prompt=150, steps=4, heavy=12, recent=12, weight_std=0.1, group=4)
     assert w.instances > 2 * torch.cuda.get_device_properties(0).multi_processor_count
