@@ -868,12 +868,14 @@ __device__ __forceinline__ uint32_t word_of(const uint4& v, int w) {
   return w == 0 ? v.x : w == 1 ? v.y : w == 2 ? v.z : v.w;
 }
 
+constexpr int kMmaRed = DEC_THREADS / 32 + 1;   // partial numerators per head in the mma kernel
+
 template <int R, int G, bool kCaptured>
 __global__ void __launch_bounds__(DEC_THREADS) decode_group_mma_kernel(DecParams p) {
   extern __shared__ float dsm[];
   const int Ns = p.Np + 4;
   float* s_sc = dsm;                               // [G][Np + 4] scores, then e^{s - m_g}
-  float* s_red = s_sc + G * Ns;                    // [G][DEC_RG][128] partial numerators
+  float* s_red = s_sc + G * Ns;                    // [G][kMmaRed][128] partial numerators: one row per warp, one for the new pair
   __shared__ float s_small[DEC_THREADS / 32];
   __shared__ unsigned long long s_key[DEC_THREADS / 32];
   __shared__ int s_vic;
@@ -1034,26 +1036,24 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_group_mma_kernel(DecParams
     }
   }
   // oacc[m]: (dim 8 fg + m, head 2 ft), (same, 2 ft + 1), (dim 8 (fg + 8) + m, head 2 ft), (same, 2 ft + 1)
-  // partial numerators: rows 0..3 of s_red per head are the warps', row 4 the new pair's, the rest zero
+  // partial numerators: rows 0..3 of s_red per head are the warps', row 4 the new pair's
 #pragma unroll
   for (int m = 0; m < 8; ++m) {
     const int d0 = 8 * fg + m, d1 = 8 * (fg + 8) + m;
     if (2 * ft < Ng) {
-      s_red[((2 * ft) * DEC_RG + warp) * kHeadDim + d0] = oacc[m][0];
-      s_red[((2 * ft) * DEC_RG + warp) * kHeadDim + d1] = oacc[m][2];
+      s_red[((2 * ft) * kMmaRed + warp) * kHeadDim + d0] = oacc[m][0];
+      s_red[((2 * ft) * kMmaRed + warp) * kHeadDim + d1] = oacc[m][2];
     }
     if (2 * ft + 1 < Ng) {
-      s_red[((2 * ft + 1) * DEC_RG + warp) * kHeadDim + d0] = oacc[m][1];
-      s_red[((2 * ft + 1) * DEC_RG + warp) * kHeadDim + d1] = oacc[m][3];
+      s_red[((2 * ft + 1) * kMmaRed + warp) * kHeadDim + d0] = oacc[m][1];
+      s_red[((2 * ft + 1) * kMmaRed + warp) * kHeadDim + d1] = oacc[m][3];
     }
   }
   {
     const float vn = __half2float(p.v[inst * kHeadDim + tid]);
 #pragma unroll
     for (int g = 0; g < G; ++g) {
-      s_red[(g * DEC_RG + 4) * kHeadDim + tid] = s_sc[g * Ns + n] * vn;
-#pragma unroll
-      for (int j = 5; j < DEC_RG; ++j) s_red[(g * DEC_RG + j) * kHeadDim + tid] = 0.f;
+      s_red[(g * kMmaRed + 4) * kHeadDim + tid] = s_sc[g * Ns + n] * vn;
     }
   }
   __syncthreads();
@@ -1075,7 +1075,7 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_group_mma_kernel(DecParams
   for (int g = 0; g < G; ++g) {
     float num = 0.f;
 #pragma unroll
-    for (int j = 0; j < DEC_RG; ++j) num += s_red[(g * DEC_RG + j) * kHeadDim + d];
+    for (int j = 0; j < kMmaRed; ++j) num += s_red[(g * kMmaRed + j) * kHeadDim + d];
     float den = lg[g];
     if (use_state) {
       const float em = __expf(-mg[g]);
@@ -1205,7 +1205,7 @@ int launch_decode(less_ctx* c, const void* q, const void* k, const void* v, void
   cudaStreamIsCapturing(s, &capturing);
   const bool captured = capturing == cudaStreamCaptureStatusActive;   // then the position is read from, and advanced in, device memory
   p.flags = d.flags;
-  const size_t smem = decode_smem_bytes(d);
+  size_t smem = decode_smem_bytes(d);
   LaunchScope scope(c, LESS_KERNEL_DECODE, s);
   void* kern = d.R == 8 ? (captured ? (void*)decode_kernel<8, true> : (void*)decode_kernel<8, false>)
                         : (captured ? (void*)decode_kernel<16, true> : (void*)decode_kernel<16, false>);
@@ -1214,6 +1214,7 @@ int launch_decode(less_ctx* c, const void* q, const void* k, const void* v, void
   int which = c->group_path;
   if (which == 0) which = 3;
   const bool teams = d.G > 1 && which == 1;
+  if (d.G > 1 && which == 3) smem = (size_t)d.G * (d.Np + 4 + kMmaRed * kHeadDim) * 4;
   if (d.G == 2) kern = d.R == 8 ? decode_group_entry<8, 2>(captured, which) : decode_group_entry<16, 2>(captured, which);
   if (d.G == 4) kern = d.R == 8 ? decode_group_entry<8, 4>(captured, which) : decode_group_entry<16, 4>(captured, which);
   if (d.G == 8) kern = d.R == 8 ? decode_group_entry<8, 8>(captured, which) : decode_group_entry<16, 8>(captured, which);
