@@ -2,15 +2,21 @@
 // attention):   out_i = sum_{j <= i} P_ij v_j,   P_ij = exp(s_ij - m_i) / l_i.
 //
 // The row statistics are already known (rowstat_tc_kernel), so no running maximum and no
-// rescaling of the output are needed: as in the column-sum kernel the constants of a row are
-// folded into a ninth k-step,  P_ij = exp2( c (q_i . k_j - b_i) ),  this time with (-b_i) on the
-// resident (query) side and a column of ones on the streamed (key) side.
+// rescaling of the output are needed:  P_ij = exp2( c q_i . k_j + nb_i ),  c = log2(e) / sqrt(D),
+// nb_i = -m_i log2(e) + log2(1 / l_i); a tensor-memory lane is a query row here, so nb_i is a
+// per-thread constant and costs nothing (no ninth k-step as in the column-sum kernel).
 //
 // One CTA = one 128-row Q tile.  Per 128-key tile:
-//   S = Q K^T - b 1^T      tcgen05, fp32 in tensor memory (double-buffered)
-//   P = exp2(c S)           sixteen epilogue warps (lane = query row), causal test on the diagonal tile,
-//                           rounded to fp16 and stored as the K-major A operand of
-//   O += P V                tcgen05, fp32 accumulator [128 x 128] in tensor memory
+//   S = Q K^T              tcgen05, fp32 in tensor memory (double-buffered)
+//   P = exp2(c S + nb)      sixteen epilogue warps (lane = query row), causal test on the diagonal tile,
+//                           rounded to fp16 and written back over the warp's own S columns in tensor
+//                           memory (two keys per 32-bit column), where it is the A operand of
+//   O += P V                tcgen05 with A from tensor memory, fp32 accumulator [128 x 128] in tensor memory
+// P never touches shared memory (its stores and reads were a quarter of a tile's shared-memory traffic).
+// P inherits the double buffering of S: the scores of tile t + 2 overwrite the buffer once the P V of
+// tile t has completed (pv_done).
+// Two threads issue the MMAs, one per product: measured on this part, one thread gets an M = 128,
+// N = 128, K = 16 MMA out every ~84 cycles whatever the operands, two threads together one every ~65.
 // P is a probability (<= 1) rounded once to fp16 (relative 4.9e-4 per element, independent signs):
 // the output moves by ~1e-4 of its magnitude, well inside the 2e-3 the outputs are held to.
 // Every wait is bounded (pipeline.cuh).
@@ -21,13 +27,11 @@ namespace less {
 
 constexpr int AO_EPI_WARPS = 16;                    // four per lane quadrant: with two, the tensor-memory loads and the P hand-over were exposed
 constexpr int AO_EPI_THREADS = AO_EPI_WARPS * 32;
-constexpr int AO_THREADS = 64 + AO_EPI_THREADS + 32;   // warp 0 TMA (Q, K), warp 1 MMA, warps 2..17 epilogue, warp 18 TMA (V)
+constexpr int AO_THREADS = 64 + AO_EPI_THREADS + 64;   // warp 0 TMA (Q, K), warp 1 MMA (scores), warps 2..17 epilogue, warp 18 TMA (V), warp 19 MMA (P V)
 constexpr int AO_TILE = 128;                        // query rows per CTA and keys per streamed tile
 constexpr int AO_TILE_BYTES = AO_TILE * kHeadDim * 2;
 constexpr int AO_STAGES = 2;
 constexpr int AO_STAGE_BYTES = 2 * AO_TILE_BYTES;   // K tile, then V tile
-constexpr int AO_QX_BYTES = AO_TILE * 16;           // (-b_i): [16 row groups][8 rows][16 B], k = 0..7
-constexpr int AO_ONES_BYTES = AO_TILE * 32;         // ones: [16 row groups][2 k halves][8 rows][16 B]
 constexpr float kAoExpScale = 0.12751743074602468f; // log2(e) / sqrt(128)
 
 struct AoShared {
@@ -36,8 +40,8 @@ struct AoShared {
   // computed, a V stage only after P V, and the next scores must not wait for the latter
   uint64_t k_full[AO_STAGES], k_empty[AO_STAGES];
   uint64_t v_full[AO_STAGES], v_empty[AO_STAGES];
-  uint64_t s_full[2], s_free[2];
-  uint64_t p_full, p_free;
+  uint64_t s_full[2], pv_done[2];
+  uint64_t p_full;
   uint64_t o_full;
   uint32_t tmem_base;
   int abort;
@@ -55,10 +59,7 @@ __global__ void __launch_bounds__(AO_THREADS) attn_out_tc_kernel(const __grid_co
   extern __shared__ __align__(1024) unsigned char ao_smem[];
   unsigned char* qres = ao_smem;                                   // Q tile: [2 halves][128 rows][128 B]
   unsigned char* ring = qres + AO_TILE_BYTES;                      // [stages][K tile | V tile]
-  unsigned char* pbuf = ring + AO_STAGES * AO_STAGE_BYTES;         // P: [2 key halves][128 rows][128 B], swizzled
-  unsigned char* qx = pbuf + AO_TILE_BYTES;                        // (-b_i) of the rows, then 2 KB of zeros (k = 8..15)
-  unsigned char* ones = qx + 2 * AO_QX_BYTES;                      // ones columns of the key side
-  AoShared* sh = reinterpret_cast<AoShared*>(ones + AO_ONES_BYTES);
+  AoShared* sh = reinterpret_cast<AoShared*>(ring + AO_STAGES * AO_STAGE_BYTES);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int tiles = (p.S + AO_TILE - 1) / AO_TILE;
@@ -79,21 +80,12 @@ __global__ void __launch_bounds__(AO_THREADS) attn_out_tc_kernel(const __grid_co
     }
     for (int s = 0; s < 2; ++s) {
       mbar_init(&sh->s_full[s], 1);
-      mbar_init(&sh->s_free[s], AO_EPI_WARPS);
+      mbar_init(&sh->pv_done[s], 1);
     }
     mbar_init(&sh->p_full, AO_EPI_WARPS);
-    mbar_init(&sh->p_free, 1);
     mbar_init(&sh->o_full, 1);
     sh->abort = *reinterpret_cast<volatile int32_t*>(status) != 0;
     mbar_fence_init();
-  }
-  // constant parts of the ninth k-step: zeros for k = 8..15 of the query side; on the key side
-  // ones (1, 1, 1, 0 ...) for k = 0..7 and zeros for k = 8..15
-  for (int e = tid; e < (AO_QX_BYTES + AO_ONES_BYTES) / 16; e += AO_THREADS) {
-    uint4 v = make_uint4(0, 0, 0, 0);
-    const int unit = e - AO_QX_BYTES / 16;                         // 16-byte unit inside the ones block
-    if (unit >= 0 && ((unit >> 3) & 1) == 0) v = make_uint4(0x3c003c00u, 0x00003c00u, 0, 0);
-    *reinterpret_cast<uint4*>(qx + AO_QX_BYTES + e * 16) = v;
   }
   if (warp == 1) tmem_alloc(&sh->tmem_base, 512);
   fence_proxy_async_smem();
@@ -108,10 +100,9 @@ __global__ void __launch_bounds__(AO_THREADS) attn_out_tc_kernel(const __grid_co
     // ---------------- TMA producer ----------------
     if (lane == 0) {
       const int row0 = (int)(qm.q_row0 + i0);
-      mbar_expect_tx(&sh->res_full, AO_TILE_BYTES + AO_QX_BYTES);
+      mbar_expect_tx(&sh->res_full, AO_TILE_BYTES);
       tma_load_2d(qres, &tm_q, 0, row0, &sh->res_full);
       tma_load_2d(qres + AO_TILE_BYTES / 2, &tm_q, 64, row0, &sh->res_full);
-      bulk_g2s(qx, p.a.ws_bx + (size_t)g * p.Sbx + i0, AO_QX_BYTES, &sh->res_full);
       uint32_t s = 0, ph = 0;
       for (int t = 0; t < ntile; ++t) {
         wait_or_give_up(&sh->k_empty[s], ph ^ 1, abortp, status, 100);
@@ -140,52 +131,51 @@ __global__ void __launch_bounds__(AO_THREADS) attn_out_tc_kernel(const __grid_co
       }
     }
   } else if (warp == 1) {
-    // ---------------- MMA issuer ----------------
+    // ---------------- MMA issuer of the scores ----------------
+    // Two threads issue the MMAs, one per product: a single thread gets an M = 128, N = 128, K = 16 MMA
+    // out every ~84 cycles, two threads together one every ~65 (the tensor pipe's own rate).
     if (lane == 0) {
       constexpr uint32_t idesc_s = idesc_f16(AO_TILE, AO_TILE, 0, 0);   // A = Q (K-major), B = K (K-major)
-      constexpr uint32_t idesc_o = idesc_f16(AO_TILE, kHeadDim, 0, 1);  // A = P (K-major), B = V (N-major)
       const uint64_t ad_q = smem_desc(smem_u32(qres), 16, 1024, kLayoutSw128);
-      const uint64_t ad_qx = smem_desc(smem_u32(qx), AO_QX_BYTES, 128, kLayoutNone);   // k = 8..15: the zeros behind
-      const uint64_t bd_ones = smem_desc(smem_u32(ones), 128, 256, kLayoutNone);
-      const uint64_t ad_p = smem_desc(smem_u32(pbuf), 16, 1024, kLayoutSw128);
       const uint64_t bd_ring = smem_desc(smem_u32(ring), 16, 1024, kLayoutSw128);
-      const uint64_t bd_vring = smem_desc(smem_u32(ring) + AO_TILE_BYTES, AO_TILE_BYTES / 2, 1024, kLayoutSw128);
       wait_or_give_up(&sh->res_full, 0, abortp, status, 101);
-      uint32_t s1 = 0, ph1 = 0, b1 = 0, bph1 = 0;      // S stream: stage, S buffer and their phases
-      int issued = 0;
-      auto issue_s = [&]() {
+      uint32_t s1 = 0, ph1 = 0;
+      for (int t = 0; t < ntile; ++t) {
+        const int b1 = t & 1;
         wait_or_give_up(&sh->k_full[s1], ph1, abortp, status, 102);
-        wait_or_give_up(&sh->s_free[b1], bph1 ^ 1, abortp, status, 103);
-        if (*abortp) return;
+        // buffer b1 held S and then P of tile t - 2: free once that tile's P V has completed
+        if (t >= 2) wait_or_give_up(&sh->pv_done[b1], ((t >> 1) - 1) & 1, abortp, status, 103);
+        if (*abortp) break;
         tc_fence_after_sync();
         const uint64_t bd0 = bd_ring + (uint64_t)(s1 * (AO_STAGE_BYTES >> 4));
 #pragma unroll
         for (int ks = 0; ks < kHeadDim / 16; ++ks)
           mma_f16_ss(tmem + b1 * AO_TILE, ad_q + (uint64_t)((ks >> 2) * (AO_TILE_BYTES >> 5) + (ks & 3) * 2),
                      bd0 + (uint64_t)((ks >> 2) * (AO_TILE_BYTES >> 5) + (ks & 3) * 2), idesc_s, ks ? 1u : 0u);
-        mma_f16_ss(tmem + b1 * AO_TILE, ad_qx, bd_ones, idesc_s, 1u);
         mma_commit(&sh->k_empty[s1]);
         mma_commit(&sh->s_full[b1]);
         if (++s1 == AO_STAGES) { s1 = 0; ph1 ^= 1; }
-        if (b1 ^= 1, b1 == 0) bph1 ^= 1;
-        ++issued;
-      };
-      issue_s();
-      uint32_t s2 = 0, vph = 0, pph = 0;
-      for (int t = 0; t < ntile && !*abortp; ++t) {
-        if (issued < ntile) issue_s();                 // the next tile's scores run ahead of this tile's P V
+      }
+    }
+  } else if (warp == 3 + AO_EPI_WARPS) {
+    // ---------------- MMA issuer of P V ----------------
+    if (lane == 0) {
+      constexpr uint32_t idesc_o = idesc_f16(AO_TILE, kHeadDim, 0, 1);  // A = P (tensor memory), B = V (N-major)
+      const uint64_t bd_vring = smem_desc(smem_u32(ring) + AO_TILE_BYTES, AO_TILE_BYTES / 2, 1024, kLayoutSw128);
+      uint32_t s2 = 0, vph = 0;
+      for (int t = 0; t < ntile; ++t) {
         wait_or_give_up(&sh->v_full[s2], vph, abortp, status, 109);
-        wait_or_give_up(&sh->p_full, pph, abortp, status, 104);
+        wait_or_give_up(&sh->p_full, t & 1, abortp, status, 104);
         if (*abortp) break;
-        pph ^= 1;
         tc_fence_after_sync();
         const uint64_t bv0 = bd_vring + (uint64_t)(s2 * (AO_STAGE_BYTES >> 4));
 #pragma unroll
         for (int ks = 0; ks < AO_TILE / 16; ++ks)
-          mma_f16_ss(tmem + ocol, ad_p + (uint64_t)((ks >> 2) * (AO_TILE_BYTES >> 5) + (ks & 3) * 2),
+          // k-step ks = keys 16 ks .. 16 ks + 15 of the tile = 8 packed columns inside the 32 S columns of part ks / 2
+          mma_f16_ts(tmem + ocol, tmem + (t & 1) * AO_TILE + 32 * (ks >> 1) + 8 * (ks & 1),
                      bv0 + (uint64_t)(ks * (2048 >> 4)), idesc_o, (t | ks) ? 1u : 0u);
-        mma_commit(&sh->p_free);
         mma_commit(&sh->v_empty[s2]);
+        mma_commit(&sh->pv_done[t & 1]);
         if (++s2 == AO_STAGES) { s2 = 0; vph ^= 1; }
       }
       mma_commit(&sh->o_full);
@@ -195,9 +185,9 @@ __global__ void __launch_bounds__(AO_THREADS) attn_out_tc_kernel(const __grid_co
     const int quad = warp & 3, part = (warp - 2) >> 2;               // part: 32 of the tile's 128 keys
     const int r = quad * 32 + lane, i = i0 + r;
     const uint32_t lane_addr = tmem + ((uint32_t)(quad * 32) << 16);
-    // P: [2 key halves][128 rows][128 B]; this thread's 32 keys are 4 of the 8 chunks of its row in one half
-    unsigned char* prow = pbuf + (part >> 1) * (AO_TILE_BYTES / 2) + r * 128;
-    const int ch0 = (part & 1) * 4;
+    // the row's constant: exp2(c s + nb) = exp(s / sqrt(D) - m_i) / l_i; rows past the prompt give zeros
+    float nb = -INFINITY;
+    if (i < p.S) nb = fmaf(-p.a.ws_m[(size_t)g * p.Sp + i], 1.4426950408889634f, log2f(p.a.ws_invl[(size_t)g * p.Sp + i]));
     uint32_t b = 0, bph = 0;
     for (int t = 0; t < ntile; ++t) {
       wait_or_give_up(&sh->s_full[b], bph, abortp, status, 105);
@@ -205,32 +195,28 @@ __global__ void __launch_bounds__(AO_THREADS) attn_out_tc_kernel(const __grid_co
       uint32_t v[32];
       tmem_ld32(lane_addr + b * AO_TILE + part * 32, v);
       tmem_ld_wait();
-      tc_fence_before_sync();
-      mbar_arrive_warp(&sh->s_free[b]);
       const int j0 = t * AO_TILE + part * 32;
       uint32_t pk[16];
       if (t == ntile - 1) {                            // the tile that holds the diagonal
 #pragma unroll
         for (int e = 0; e < 16; ++e) {
-          const float p0 = j0 + 2 * e <= i ? ao_ex2(__uint_as_float(v[2 * e]) * kAoExpScale) : 0.f;
-          const float p1 = j0 + 2 * e + 1 <= i ? ao_ex2(__uint_as_float(v[2 * e + 1]) * kAoExpScale) : 0.f;
+          const float p0 = j0 + 2 * e <= i ? ao_ex2(fmaf(__uint_as_float(v[2 * e]), kAoExpScale, nb)) : 0.f;
+          const float p1 = j0 + 2 * e + 1 <= i ? ao_ex2(fmaf(__uint_as_float(v[2 * e + 1]), kAoExpScale, nb)) : 0.f;
           const __half2 h = __floats2half2_rn(p0, p1);
           pk[e] = *reinterpret_cast<const uint32_t*>(&h);
         }
       } else {
 #pragma unroll
         for (int e = 0; e < 16; ++e) {
-          const __half2 h = __floats2half2_rn(ao_ex2(__uint_as_float(v[2 * e]) * kAoExpScale),
-                                              ao_ex2(__uint_as_float(v[2 * e + 1]) * kAoExpScale));
+          const __half2 h = __floats2half2_rn(ao_ex2(fmaf(__uint_as_float(v[2 * e]), kAoExpScale, nb)),
+                                              ao_ex2(fmaf(__uint_as_float(v[2 * e + 1]), kAoExpScale, nb)));
           pk[e] = *reinterpret_cast<const uint32_t*>(&h);
         }
       }
-      wait_or_give_up(&sh->p_free, (t & 1) ^ 1, abortp, status, 106);   // the previous tile's P V has read P
-#pragma unroll
-      for (int c = 0; c < 4; ++c)                      // 16-byte chunk ch0 + c of the row, 128-byte swizzle
-        *reinterpret_cast<uint4*>(prow + (((ch0 + c) ^ (r & 7)) << 4)) =
-            make_uint4(pk[c * 4], pk[c * 4 + 1], pk[c * 4 + 2], pk[c * 4 + 3]);
-      fence_proxy_async_smem();
+      // P over the first 16 of this warp's own 32 S columns (they are in registers by now)
+      tmem_st16(lane_addr + b * AO_TILE + part * 32, pk);
+      tmem_st_wait();
+      tc_fence_before_sync();
       mbar_arrive_warp(&sh->p_full);
       if (b ^= 1, b == 0) bph ^= 1;
     }
@@ -265,7 +251,7 @@ int launch_attn_out_tc(less_ctx* c, const PfParams& p, int G, cudaStream_t s) {
       !make_tmap_f16_2d(&tk, p.K, rows, kHeadDim, kHeadDim * 2, AO_TILE) ||
       !make_tmap_f16_2d(&tv, p.V, rows, kHeadDim, kHeadDim * 2, AO_TILE))
     return fail_cuda("tensor maps of Q / K / V");
-  const size_t smem = (size_t)AO_TILE_BYTES * 2 + AO_STAGES * AO_STAGE_BYTES + 2 * AO_QX_BYTES + AO_ONES_BYTES +
+  const size_t smem = (size_t)AO_TILE_BYTES + AO_STAGES * AO_STAGE_BYTES +
                       sizeof(AoShared) + 1024;
   if (cudaFuncSetAttribute(attn_out_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
     return fail_cuda("shared memory opt-in of attn_out_tc_kernel");

@@ -13,7 +13,7 @@
 //   S = Q K^T                       tcgen05, fp32 in tensor memory (double-buffered)
 //   L = phi~ psi~^T                 tcgen05, hi hi + lo hi + hi lo of the scaled fp16 splits
 //   P_ij = i < exact_until[j] ? exp2(c S_ij - E_i) : L_ij 2^(lscale_i - E_i)     (epilogue warps, lane = row)
-//   O += P V                        tcgen05;   r_i += sum_j P_ij (fp32, before rounding P to fp16)
+//   O += P V                        tcgen05, P read from tensor memory;   r_i += sum_j P_ij (fp32, before rounding P to fp16)
 //   out_i = O_i / r_i
 // The key tiles stream past the Q tile twice.  The first sweep only takes maxima: the row's largest
 // exact dot product and its largest kernel value give E_i = log2 of the row's largest entry.  The
@@ -36,7 +36,7 @@ constexpr int MF_EU_SLOTS = 4;                      // exact_until tiles in flig
 constexpr int MF_STAGE_BYTES = 2 * MF_TILE_BYTES;   // K tile, then V tile
 constexpr int MF_EPI_WARPS = 16;                   // four per lane quadrant, 32 keys of a tile each
 constexpr int MF_EPI_THREADS = MF_EPI_WARPS * 32;
-constexpr int MF_THREADS = 64 + MF_EPI_THREADS + 32;   // warp 0 TMA (Q, K, operands), warp 1 MMA, warps 2..17 epilogue, warp 18 TMA (V)
+constexpr int MF_THREADS = 64 + MF_EPI_THREADS + 64;   // warp 0 TMA (Q, K, operands), warp 1 MMA (scores), warps 2..17 epilogue, warp 18 TMA (V), warp 19 MMA (P V)
 constexpr float kMfExpScale = 0.12751743074602468f; // log2(e) / sqrt(128)
 
 struct MfParams {
@@ -139,7 +139,8 @@ struct MfShared {
   uint64_t eu_full[MF_EU_SLOTS], eu_empty[MF_EU_SLOTS];   // exact_until of the key tile
   uint64_t s_full[2], s_free[2];                      // S buffer (and L) written / read
   uint64_t l_free;                                    // the single L buffer has been read
-  uint64_t p_full, p_free;
+  uint64_t p_full;
+  uint64_t pv_done[2];                                // the P V that read the S buffer's P has completed
   uint64_t o_full;
   uint32_t tmem_base;
   int abort;
@@ -163,8 +164,7 @@ __global__ void __launch_bounds__(MF_THREADS) masked_out_tc_kernel(const __grid_
   extern __shared__ __align__(1024) unsigned char mf_smem[];
   unsigned char* qres = mf_smem;                                   // Q tile: [2 halves][128 rows][128 B]
   unsigned char* ring = qres + MF_TILE_BYTES;                      // [stages][K tile, V tile]
-  unsigned char* pbuf = ring + MF_STAGES * MF_STAGE_BYTES;         // P: [2 key halves][128 rows][128 B], swizzled
-  unsigned char* phires = pbuf + MF_TILE_BYTES;                    // phi operand tile of the rows
+  unsigned char* phires = ring + MF_STAGES * MF_STAGE_BYTES;       // phi operand tile of the rows
   unsigned char* psiring = phires + MF_OP_BYTES;                   // [stages] psi operand tiles of the keys
   unsigned char* euring = psiring + MF_STAGES * MF_OP_BYTES;       // [slots] exact_until of the keys
   MfShared* sh = reinterpret_cast<MfShared*>(euring + MF_EU_SLOTS * MF_EU_BYTES);
@@ -195,10 +195,10 @@ __global__ void __launch_bounds__(MF_THREADS) masked_out_tc_kernel(const __grid_
     for (int s = 0; s < 2; ++s) {
       mbar_init(&sh->s_full[s], 1);
       mbar_init(&sh->s_free[s], MF_EPI_WARPS);
+      mbar_init(&sh->pv_done[s], 1);
     }
     mbar_init(&sh->l_free, MF_EPI_WARPS);
     mbar_init(&sh->p_full, MF_EPI_WARPS);
-    mbar_init(&sh->p_free, 1);
     mbar_init(&sh->o_full, 1);
     sh->abort = *reinterpret_cast<volatile int32_t*>(status) != 0;
     mbar_fence_init();
@@ -253,32 +253,38 @@ __global__ void __launch_bounds__(MF_THREADS) masked_out_tc_kernel(const __grid_
       }
     }
   } else if (warp == 1) {
-    // ---------------- MMA issuer ----------------
+    // ---------------- MMA issuer of the scores and kernel values (both sweeps) ----------------
+    // Two threads issue the MMAs, one per product: a single thread gets an M = 128, N = 128, K = 16 MMA
+    // out every ~84 cycles, two threads together one every ~65 (the tensor pipe's own rate).
     if (lane == 0) {
       constexpr uint32_t idesc_s = idesc_f16(MF_TILE, MF_TILE, 0, 0);   // A = Q (K-major), B = K (K-major); also phi x psi
-      constexpr uint32_t idesc_o = idesc_f16(MF_TILE, kHeadDim, 0, 1);  // A = P (K-major), B = V (N-major)
       const uint64_t ad_q = smem_desc(smem_u32(qres), 16, 1024, kLayoutSw128);
       // operand tiles without swizzle: chunks of 8 k are 2048 bytes apart, 8-row groups 128 bytes
       const uint64_t ad_phi = smem_desc(smem_u32(phires), 2048, 128, kLayoutNone);
       const uint64_t bd_psi = smem_desc(smem_u32(psiring), 2048, 128, kLayoutNone);
-      const uint64_t ad_p = smem_desc(smem_u32(pbuf), 16, 1024, kLayoutSw128);
       const uint64_t bd_ring = smem_desc(smem_u32(ring), 16, 1024, kLayoutSw128);
-      const uint64_t bd_vring = smem_desc(smem_u32(ring) + MF_TILE_BYTES, MF_TILE_BYTES / 2, 1024, kLayoutSw128);
       constexpr uint64_t kPair = 4096 >> 4;                             // two chunks = one 16-wide k-step further
       wait_or_give_up(&sh->res_full, 0, abortp, status, 113);
-      uint32_t s1 = 0, ph1 = 0, b1 = 0, bph1 = 0;
-      int issued = 0;
-      auto issue_s = [&]() {
+      uint32_t s1 = 0, ph1 = 0;
+      for (int u = 0; u < 2 * ntile; ++u) {
+        const int b1 = u & 1;
         wait_or_give_up(&sh->k_full[s1], ph1, abortp, status, 114);
-        wait_or_give_up(&sh->s_free[b1], bph1 ^ 1, abortp, status, 115);
-        wait_or_give_up(&sh->l_free, (issued & 1) ^ 1, abortp, status, 116);
-        if (*abortp) return;
+        // buffer b1 held tile u - 2: read by the epilogue (s_free) and, in the second sweep, rewritten
+        // with P and read by that tile's P V (pv_done); the single L buffer held tile u - 1 (l_free)
+        if (u >= 2) wait_or_give_up(&sh->s_free[b1], ((u >> 1) - 1) & 1, abortp, status, 115);
+        if (u - 2 >= ntile) wait_or_give_up(&sh->pv_done[b1], ((u - 2 - ntile) >> 1) & 1, abortp, status, 123);
+        if (*abortp) break;
         tc_fence_after_sync();
         const uint64_t bd0 = bd_ring + (uint64_t)(s1 * (MF_STAGE_BYTES >> 4));
 #pragma unroll
         for (int ks = 0; ks < kHeadDim / 16; ++ks)
           mma_f16_ss(tmem + b1 * MF_TILE, ad_q + (uint64_t)((ks >> 2) * (MF_TILE_BYTES >> 5) + (ks & 3) * 2),
                      bd0 + (uint64_t)((ks >> 2) * (MF_TILE_BYTES >> 5) + (ks & 3) * 2), idesc_s, ks ? 1u : 0u);
+        // the scores are under way before the single L buffer is waited for: the epilogue of tile u - 1
+        // reads it while these eight MMAs run
+        if (u >= 1) wait_or_give_up(&sh->l_free, (u - 1) & 1, abortp, status, 116);
+        if (*abortp) break;
+        tc_fence_after_sync();
         const uint64_t bp = bd_psi + (uint64_t)(s1 * (MF_OP_BYTES >> 4));
         if (R == 8) {
           mma_f16_ss(tmem + lcol, ad_phi, bp, idesc_s, 0u);                   // (hi, lo) x (hi, hi)
@@ -291,26 +297,28 @@ __global__ void __launch_bounds__(MF_THREADS) masked_out_tc_kernel(const __grid_
         mma_commit(&sh->k_empty[s1]);
         mma_commit(&sh->s_full[b1]);
         if (++s1 == MF_STAGES) { s1 = 0; ph1 ^= 1; }
-        if (b1 ^= 1, b1 == 0) bph1 ^= 1;
-        ++issued;
-      };
-      for (int u = 0; u < ntile && !*abortp; ++u) issue_s();   // first sweep: scores and kernel values only
-      issue_s();
-      uint32_t s2 = 0, vph = 0, pph = 0;
-      for (int t = 0; t < ntile && !*abortp; ++t) {
-        if (issued < 2 * ntile) issue_s();             // the next tile's scores run ahead of this tile's P V
+      }
+    }
+  } else if (warp == 3 + MF_EPI_WARPS) {
+    // ---------------- MMA issuer of P V (second sweep) ----------------
+    if (lane == 0) {
+      constexpr uint32_t idesc_o = idesc_f16(MF_TILE, kHeadDim, 0, 1);  // A = P (tensor memory), B = V (N-major)
+      const uint64_t bd_vring = smem_desc(smem_u32(ring) + MF_TILE_BYTES, MF_TILE_BYTES / 2, 1024, kLayoutSw128);
+      uint32_t s2 = 0, vph = 0;
+      for (int t = 0; t < ntile; ++t) {
+        const int bt = (ntile + t) & 1;                  // the S buffer this tile's P lives in
         wait_or_give_up(&sh->v_full[s2], vph, abortp, status, 117);
-        wait_or_give_up(&sh->p_full, pph, abortp, status, 118);
+        wait_or_give_up(&sh->p_full, t & 1, abortp, status, 118);
         if (*abortp) break;
-        pph ^= 1;
         tc_fence_after_sync();
         const uint64_t bv0 = bd_vring + (uint64_t)(s2 * (MF_STAGE_BYTES >> 4));
 #pragma unroll
         for (int ks = 0; ks < MF_TILE / 16; ++ks)
-          mma_f16_ss(tmem + ocol, ad_p + (uint64_t)((ks >> 2) * (MF_TILE_BYTES >> 5) + (ks & 3) * 2),
+          // A = P from tensor memory: k-step ks is 8 packed columns inside the S columns of part ks / 2
+          mma_f16_ts(tmem + ocol, tmem + bt * MF_TILE + 32 * (ks >> 1) + 8 * (ks & 1),
                      bv0 + (uint64_t)(ks * (2048 >> 4)), idesc_o, (t | ks) ? 1u : 0u);
-        mma_commit(&sh->p_free);
         mma_commit(&sh->v_empty[s2]);
+        mma_commit(&sh->pv_done[bt]);
         if (++s2 == MF_STAGES) { s2 = 0; vph ^= 1; }
       }
       mma_commit(&sh->o_full);
@@ -320,9 +328,6 @@ __global__ void __launch_bounds__(MF_THREADS) masked_out_tc_kernel(const __grid_
     const int quad = warp & 3, part = (warp - 2) >> 2;               // part: 32 of the tile's 128 keys
     const int r = quad * 32 + lane, i = i0 + r;
     const uint32_t lane_addr = tmem + ((uint32_t)(quad * 32) << 16);
-    // P: [2 key halves][128 rows][128 B]; this thread's 32 keys are 4 of the 8 chunks of its row in one half
-    unsigned char* prow = pbuf + (part >> 1) * (MF_TILE_BYTES / 2) + r * 128;
-    const int ch0 = (part & 1) * 4;
     // sweep 1: the row's largest exact dot product and largest kernel value (scaled operands);
     // sweep 2: P against the largest entry, so that every entry is <= 1 and the largest is 1
     const float lscale = p.a.ws_g[rc0 + i];            // log2 of (true kernel value / scaled kernel value)
@@ -424,12 +429,12 @@ __global__ void __launch_bounds__(MF_THREADS) masked_out_tc_kernel(const __grid_
       }
       mbar_arrive_warp(&sh->eu_empty[es]);
       if (second) {
-        wait_or_give_up(&sh->p_free, (t & 1) ^ 1, abortp, status, 121);   // the previous tile's P V has read P
-#pragma unroll
-        for (int c = 0; c < 4; ++c)                    // 16-byte chunk ch0 + c of the row, 128-byte swizzle
-          *reinterpret_cast<uint4*>(prow + (((ch0 + c) ^ (r & 7)) << 4)) =
-              make_uint4(pk[c * 4], pk[c * 4 + 1], pk[c * 4 + 2], pk[c * 4 + 3]);
-        fence_proxy_async_smem();
+        // P, rounded to fp16, over the first 16 of this warp's own 32 S columns (they are in registers):
+        // it inherits the double buffering of S, and the scores that overwrite the buffer are issued
+        // after the P V that reads it (the tensor pipe runs in issue order)
+        tmem_st16(lane_addr + b * MF_TILE + part * 32, pk);
+        tmem_st_wait();
+        tc_fence_before_sync();
         mbar_arrive_warp(&sh->p_full);
       }
       if (b ^= 1, b == 0) bph ^= 1;
@@ -511,7 +516,7 @@ int launch_masked_form(less_ctx* c, int layer0, int nl, int lj0, int layer_count
       !make_tmap_f16_2d(&tk, p.K, rows, kHeadDim, kHeadDim * 2, MF_TILE) ||
       !make_tmap_f16_2d(&tv, p.V, rows, kHeadDim, kHeadDim * 2, MF_TILE))
     return fail_cuda("tensor maps of Q / K / V");
-  const size_t smem = (size_t)MF_TILE_BYTES * 2 + MF_STAGES * MF_STAGE_BYTES + MF_OP_BYTES + MF_STAGES * MF_OP_BYTES +
+  const size_t smem = (size_t)MF_TILE_BYTES + MF_STAGES * MF_STAGE_BYTES + MF_OP_BYTES + MF_STAGES * MF_OP_BYTES +
                       MF_EU_SLOTS * MF_EU_BYTES + sizeof(MfShared) + 1024;
   LaunchScope scope(c, LESS_KERNEL_MASKED_OUT, s);
   if (d.R == 8) {
