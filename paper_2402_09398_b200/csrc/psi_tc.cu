@@ -11,18 +11,20 @@
 //   after 8 chunks: tcgen05.ld G2 -> c2 * gelu(c1 * .) -> W3 on CUDA cores -> abs -> psi[token][R]
 // The same kernel evaluates phi(q) = | gelu( gelu(q W1) W2 ) | (Eq. 1) over a sequence of queries for
 // the parallel form (PtMap::is_phi: no W3, no scalars, rows of Q).
-// Roles: warps 0-7 epilogue (lane quadrant = warp & 3, token row = tensor-memory lane; the two
-// warps of a quadrant split a chunk's 64 columns), warp 8 TMA producer, warp 9 MMA issuer.  Operands come in by TMA tiled loads with the 128-byte
-// swizzle (no multicast).  Every wait is bounded.
+// Roles: warps 0-15 epilogue (lane quadrant = warp & 3, token row = tensor-memory lane; the four
+// warps of a quadrant split a chunk's 64 columns), warp 16 TMA producer, warp 17 issues GEMM1, warp 18
+// GEMM2.  Operands come in by TMA tiled loads with the 128-byte swizzle (no multicast).  Every wait is bounded.
 #include "prefill.cuh"
 #include "tc_common.cuh"
 
 namespace less {
 
-constexpr int PT_WORKERS = 256;                    // 8 epilogue warps: two per tensor-memory lane quadrant
-constexpr int PT_THREADS = PT_WORKERS + 64;
+constexpr int PT_WORKERS = 512;                    // 16 epilogue warps: four per tensor-memory lane quadrant (GELU issue and latency bound the kernel)
+constexpr int PT_THREADS = PT_WORKERS + 96;         // + TMA producer, GEMM1 issuer, GEMM2 issuer
 constexpr int PT_TILE = 128;                       // tokens per tile
 constexpr int PT_CHUNK = 64;                       // hidden units per GEMM1 chunk
+constexpr int PT_PARTS = PT_WORKERS / 128;         // warps per lane quadrant
+constexpr int PT_COLS = PT_CHUNK / PT_PARTS;       // columns of a chunk per warp (16)
 constexpr int PT_KBYTES = PT_TILE * kHeadDim * 2;  // one K tile
 constexpr int PT_W2N = 16;                         // GEMM2 N (R padded to 16)
 
@@ -133,32 +135,42 @@ __global__ void __launch_bounds__(PT_THREADS) psi_tc_kernel(const __grid_constan
       }
     }
   } else if (warp == PT_WORKERS / 32 + 1) {
-    // ---------------- MMA issuer ----------------
+    // ---------------- MMA issuer of GEMM1 ----------------
+    // One issuing thread per GEMM: a single thread gets an MMA out every ~84 cycles, and 128 of them per
+    // token tile in one thread were on the critical path of every chunk; the two streams only meet at
+    // the barriers they already had (d1_free / d1_full, hid_full / hid_free, g2_free / g2_full).
     if (tid == PT_WORKERS + 32) {
       constexpr uint32_t idesc1 = idesc_f16(128, PT_CHUNK, 0, 1);   // A = K tile (K-major), B = W1 (N-major)
-      constexpr uint32_t idesc2 = idesc_f16(128, PT_W2N, 0, 1);     // A = hidden (K-major), B = W2 (N-major)
-      const uint32_t w1a = smem_u32(w1s), w2a = smem_u32(w2s), hida = smem_u32(hid);
+      const uint32_t w1a = smem_u32(w1s);
       pt_wait(&sh->w1_full, 0, abortp, status, 31);
       uint32_t q = 0;                                               // chunk counter over all tiles
-      auto issue_gemm1 = [&](uint32_t ka, int c, uint32_t qq) {
-        const int b = qq & 1;
-        pt_wait(&sh->d1_free[b], ((qq >> 1) & 1) ^ 1, abortp, status, 32);
-        tc_fence_after_sync();
-#pragma unroll
-        for (int ks = 0; ks < kHeadDim / 16; ++ks) {
-          const uint64_t ad = smem_desc(ka + (ks >> 2) * (PT_KBYTES / 2) + (ks & 3) * 32, 16, 1024, kLayoutSw128);
-          const uint64_t bd = smem_desc(w1a + c * 16384 + ks * 2048, 16384, 1024, kLayoutSw128);
-          mma_f16_ss(tmem + b * PT_CHUNK, ad, bd, idesc1, ks ? 1u : 0u);
-        }
-        mma_commit(&sh->d1_full[b]);
-      };
       for (int i = 0; i < ntiles && !*abortp; ++i) {
         pt_wait(&sh->k_full, i & 1, abortp, status, 33);
         const uint32_t ka = smem_u32(kbuf);
-        issue_gemm1(ka, 0, q);
+        for (int c = 0; c < nchunk && !*abortp; ++c, ++q) {
+          const int b = q & 1;
+          pt_wait(&sh->d1_free[b], ((q >> 1) & 1) ^ 1, abortp, status, 32);
+          if (*abortp) break;
+          tc_fence_after_sync();
+#pragma unroll
+          for (int ks = 0; ks < kHeadDim / 16; ++ks) {
+            const uint64_t ad = smem_desc(ka + (ks >> 2) * (PT_KBYTES / 2) + (ks & 3) * 32, 16, 1024, kLayoutSw128);
+            const uint64_t bd = smem_desc(w1a + c * 16384 + ks * 2048, 16384, 1024, kLayoutSw128);
+            mma_f16_ss(tmem + b * PT_CHUNK, ad, bd, idesc1, ks ? 1u : 0u);
+          }
+          mma_commit(&sh->d1_full[b]);
+        }
+        mma_commit(&sh->k_empty);                                   // all GEMM1s of this tile are issued
+      }
+    }
+  } else if (warp == PT_WORKERS / 32 + 2) {
+    // ---------------- MMA issuer of GEMM2 ----------------
+    if (tid == PT_WORKERS + 64) {
+      constexpr uint32_t idesc2 = idesc_f16(128, PT_W2N, 0, 1);     // A = hidden (K-major), B = W2 (N-major)
+      const uint32_t w2a = smem_u32(w2s), hida = smem_u32(hid);
+      uint32_t q = 0;
+      for (int i = 0; i < ntiles && !*abortp; ++i) {
         for (int c = 0; c < nchunk; ++c, ++q) {
-          if (c + 1 < nchunk) issue_gemm1(ka, c + 1, q + 1);
-          else mma_commit(&sh->k_empty);                            // all GEMM1s of this tile are issued
           if (c == 0) pt_wait(&sh->g2_free, (i & 1) ^ 1, abortp, status, 34);
           pt_wait(&sh->hid_full, q & 1, abortp, status, 35);
           if (*abortp) break;
@@ -173,13 +185,14 @@ __global__ void __launch_bounds__(PT_THREADS) psi_tc_kernel(const __grid_constan
           }
           mma_commit(&sh->hid_free);
         }
+        if (*abortp) break;
         mma_commit(&sh->g2_full);
       }
     }
   } else {
     // ---------------- epilogue workers ----------------
     const float c1 = sh->c1, c2 = sh->c2;
-    const int quad = warp & 3, half = warp >> 2;
+    const int quad = warp & 3, half = warp >> 2;       // half: which PT_COLS columns of a chunk
     const int row = quad * 32 + (tid & 31);                         // token row of the tile = tensor-memory lane
     const uint32_t lane_addr = tmem + ((uint32_t)(quad * 32) << 16);
     float* psi = mp.out + (size_t)g * p.Sp * R;
@@ -191,16 +204,15 @@ __global__ void __launch_bounds__(PT_THREADS) psi_tc_kernel(const __grid_constan
         const int b = q & 1;
         pt_wait(&sh->d1_full[b], (q >> 1) & 1, abortp, status, 36);
         tc_fence_after_sync();
-        uint32_t acc[PT_CHUNK / 2];                                  // this warp's 32 of the chunk's 64 columns
-#pragma unroll
-        for (int cc = 0; cc < PT_CHUNK / 32; ++cc)
-          tmem_ld16(lane_addr + b * PT_CHUNK + half * (PT_CHUNK / 2) + cc * 16, acc + cc * 16);
+        uint32_t acc[PT_COLS];                                       // this warp's 16 of the chunk's 64 columns
+        static_assert(PT_COLS == 16, "one 16-column tensor-memory load per warp and chunk");
+        tmem_ld16(lane_addr + b * PT_CHUNK + half * PT_COLS, acc);
         tmem_ld_wait();
         tc_fence_before_sync();
         mbar_arrive_warp(&sh->d1_free[b]);
-        uint32_t phi_[PT_CHUNK / 4], plo_[PT_CHUNK / 4];
+        uint32_t phi_[PT_COLS / 2], plo_[PT_COLS / 2];
 #pragma unroll
-        for (int e = 0; e < PT_CHUNK / 4; ++e) {
+        for (int e = 0; e < PT_COLS / 2; ++e) {
           // c1 multiplies the layer-2 sums instead (same value): the fp16 hi + lo operand then never
           // depends on how small the learnable scalar is (the paper initialises it to 1e-4)
           const float h0 = gelu_erf(__uint_as_float(acc[2 * e]));
@@ -213,8 +225,8 @@ __global__ void __launch_bounds__(PT_THREADS) psi_tc_kernel(const __grid_constan
         }
         pt_wait(&sh->hid_free, (q & 1) ^ 1, abortp, status, 37);
 #pragma unroll
-        for (int cq = 0; cq < 4; ++cq) {               // 16-byte chunk half * 4 + cq of this row, 128-byte swizzle
-          const int off = ((half * 4 + cq) ^ (row & 7)) << 4;
+        for (int cq = 0; cq < PT_COLS / 8; ++cq) {     // 16-byte chunk half * 2 + cq of this row, 128-byte swizzle
+          const int off = ((half * (PT_COLS / 8) + cq) ^ (row & 7)) << 4;
           *reinterpret_cast<uint4*>(hrow + off) =
               make_uint4(phi_[cq * 4], phi_[cq * 4 + 1], phi_[cq * 4 + 2], phi_[cq * 4 + 3]);
           *reinterpret_cast<uint4*>(hrow + 16384 + off) =
