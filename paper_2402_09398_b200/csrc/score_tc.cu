@@ -5,7 +5,7 @@
 //
 // Both stream 256-row tiles of the other operand past one resident 128-row tile and
 // compute 128 x 256 tiles of raw dot products with tcgen05 (kind::f16, fp16 inputs used
-// exactly, fp32 accumulators double-buffered in tensor memory); eight epilogue warps read
+// exactly, fp32 accumulators double-buffered in tensor memory); sixteen epilogue warps read
 // the tiles back (lane = row of the resident tile) and reduce them.
 //
 // Row statistics: resident Q tile, streamed K tiles up to the diagonal, online max / sum.
@@ -25,7 +25,11 @@
 
 namespace less {
 
-constexpr int SC_EPI_WARPS = 8;
+constexpr int SC_EPI_WARPS = 16;                   // four per lane quadrant: with two, the tensor-memory loads of a
+                                                  // tile's column groups were exposed and the XU idled a fifth of the time
+constexpr int SC_PARTS = SC_EPI_WARPS / 4;        // warps that split a tile's 256 columns
+constexpr int SC_PART_COLS = 256 / SC_PARTS;      // columns per warp (64)
+constexpr int SC_PART_GROUPS = SC_PART_COLS / 32; // 32-column loads per warp and tile
 constexpr int SC_EPI_THREADS = SC_EPI_WARPS * 32;
 constexpr int SC_TILE_M = 128;                    // rows of the resident tile
 constexpr int SC_TILE_N = 256;                    // rows of a streamed tile
@@ -41,7 +45,7 @@ struct ScShared {
   uint64_t d_full[2], d_free[2];
   uint32_t tmem_base;
   int abort;
-  float merge[SC_TILE_M][2];
+  float merge[SC_PARTS][SC_TILE_M][2];
 };
 
 __device__ __forceinline__ void sc_epi_sync() { asm volatile("bar.sync 1, %0;" ::"n"(SC_EPI_THREADS) : "memory"); }
@@ -153,19 +157,19 @@ __global__ void __launch_bounds__(RS_THREADS) rowstat_tc_kernel(const __grid_con
       }
     }
   } else {
-    // ---- epilogue: lane = row of the Q tile; the two warps of a lane quadrant split the columns ----
-    const int quad = warp & 3, half = (warp - 2) >> 2;
+    // ---- epilogue: lane = row of the Q tile; the four warps of a lane quadrant split the columns ----
+    const int quad = warp & 3, half = (warp - 2) >> 2;      // half: which SC_PART_COLS columns of a tile
     const int r = quad * 32 + lane, i = i0 + r;
-    const uint32_t lane_addr = tmem + ((uint32_t)(quad * 32) << 16) + half * (SC_TILE_N / 2);
+    const uint32_t lane_addr = tmem + ((uint32_t)(quad * 32) << 16) + half * SC_PART_COLS;
     float m = -INFINITY, l = 0.f;                      // m in raw dot-product units
     uint32_t b = 0, bph = 0;
     for (int t = 0; t < ntile; ++t) {
       wait_or_give_up(&sh->d_full[b], bph, abortp, status, 84);
       tc_fence_after_sync();
-      const int c0 = t * SC_TILE_N + half * (SC_TILE_N / 2);
+      const int c0 = t * SC_TILE_N + half * SC_PART_COLS;
       const bool edge = t == ntile - 1;                // only the last tile meets the diagonal or the prompt's end
 #pragma unroll 1
-      for (int cg = 0; cg < 4; ++cg) {
+      for (int cg = 0; cg < SC_PART_GROUPS; ++cg) {
         uint32_t v[32];
         tmem_ld32(lane_addr + b * SC_TILE_N + cg * 32, v);
         tmem_ld_wait();
@@ -198,15 +202,20 @@ __global__ void __launch_bounds__(RS_THREADS) rowstat_tc_kernel(const __grid_con
       mbar_arrive_warp(&sh->d_free[b]);
       if (b ^= 1, b == 0) bph ^= 1;
     }
-    // merge the two column halves of a row
-    if (half == 1) { sh->merge[r][0] = m; sh->merge[r][1] = l; }
+    // merge the column parts of a row
+    sh->merge[half][r][0] = m;
+    sh->merge[half][r][1] = l;
     sc_epi_sync();
     if (half == 0 && i < p.S && !*abortp) {
-      const float m2 = sh->merge[r][0], l2 = sh->merge[r][1];
-      const float mm = fmaxf(m, m2);
+      float mm = -INFINITY;
+#pragma unroll
+      for (int h = 0; h < SC_PARTS; ++h) mm = fmaxf(mm, sh->merge[h][r][0]);
       float lt = 0.f;
-      if (m > -INFINITY) lt += l * ex2_approx((m - mm) * kExpScale);
-      if (m2 > -INFINITY) lt += l2 * ex2_approx((m2 - mm) * kExpScale);
+#pragma unroll
+      for (int h = 0; h < SC_PARTS; ++h) {
+        const float mh = sh->merge[h][r][0];
+        if (mh > -INFINITY) lt += sh->merge[h][r][1] * ex2_approx((mh - mm) * kExpScale);
+      }
       const float il = 1.0f / lt;
       p.a.ws_m[(size_t)g * p.Sp + i] = mm * kRawScale;
       p.a.ws_invl[(size_t)g * p.Sp + i] = il;
@@ -330,18 +339,18 @@ __global__ void __launch_bounds__(CS_THREADS) colsum_tc_kernel(const __grid_cons
       }
     }
   } else {
-    // ---- epilogue: lane = key of the K tile; the two warps of a lane quadrant split the rows i ----
+    // ---- epilogue: lane = key of the K tile; the four warps of a lane quadrant split the rows i ----
     const int quad = warp & 3, half = (warp - 2) >> 2;
     const int r = quad * 32 + lane, j = j0 + r;
-    const uint32_t lane_addr = tmem + ((uint32_t)(quad * 32) << 16) + half * (SC_TILE_N / 2);
+    const uint32_t lane_addr = tmem + ((uint32_t)(quad * 32) << 16) + half * SC_PART_COLS;
     float acc = 0.f;
     uint32_t b = 0, bph = 0;
     for (int ts = 0, t = 0; ts < nstream; ++ts, t = (t + 1 == ntile ? 0 : t + 1)) {   // t: tile within the head
       wait_or_give_up(&sh->d_full[b], bph, abortp, status, 91);
       tc_fence_after_sync();
-      const int c0 = (t0 + t) * SC_TILE_N + half * (SC_TILE_N / 2);
+      const int c0 = (t0 + t) * SC_TILE_N + half * SC_PART_COLS;
 #pragma unroll 1
-      for (int cg = 0; cg < 4; ++cg) {
+      for (int cg = 0; cg < SC_PART_GROUPS; ++cg) {
         uint32_t v[32];
         tmem_ld32(lane_addr + b * SC_TILE_N + cg * 32, v);
         tmem_ld_wait();
@@ -363,9 +372,14 @@ __global__ void __launch_bounds__(CS_THREADS) colsum_tc_kernel(const __grid_cons
       mbar_arrive_warp(&sh->d_free[b]);
       if (b ^= 1, b == 0) bph ^= 1;
     }
-    if (half == 1) sh->merge[r][0] = acc;
+    sh->merge[half][r][0] = acc;
     sc_epi_sync();
-    if (half == 0 && j < p.S && !*abortp) p.a.ws_acc[(size_t)g * p.Sp + j] = acc + sh->merge[r][0];
+    if (half == 0 && j < p.S && !*abortp) {
+      float total = 0.f;
+#pragma unroll
+      for (int h = 0; h < SC_PARTS; ++h) total += sh->merge[h][r][0];      // fixed order
+      p.a.ws_acc[(size_t)g * p.Sp + j] = total;
+    }
   }
   drain_after_abort(abortp);
   tc_fence_before_sync();
