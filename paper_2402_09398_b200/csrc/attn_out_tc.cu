@@ -7,14 +7,14 @@
 // per-thread constant and costs nothing (no ninth k-step as in the column-sum kernel).
 //
 // One CTA = one 128-row Q tile.  Per 128-key tile:
-//   S = Q K^T              tcgen05, fp32 in tensor memory (double-buffered)
+//   S = Q K^T              tcgen05, fp32 in tensor memory (three buffers)
 //   P = exp2(c S + nb)      sixteen epilogue warps (lane = query row), causal test on the diagonal tile,
 //                           rounded to fp16 and written back over the warp's own S columns in tensor
 //                           memory (two keys per 32-bit column), where it is the A operand of
 //   O += P V                tcgen05 with A from tensor memory, fp32 accumulator [128 x 128] in tensor memory
 // P never touches shared memory (its stores and reads were a quarter of a tile's shared-memory traffic).
-// P inherits the double buffering of S: the scores of tile t + 2 overwrite the buffer once the P V of
-// tile t has completed (pv_done).
+// P inherits the buffering of S: the scores of tile t + 3 overwrite the buffer once the P V of tile t has
+// completed (pv_done); with three buffers the scores of a tile never wait for the P V two tiles back.
 // Two threads issue the MMAs, one per product: measured on this part, one thread gets an M = 128,
 // N = 128, K = 16 MMA out every ~84 cycles whatever the operands, two threads together one every ~65.
 // P is a probability (<= 1) rounded once to fp16 (relative 4.9e-4 per element, independent signs):
@@ -31,6 +31,7 @@ constexpr int AO_THREADS = 64 + AO_EPI_THREADS + 64;   // warp 0 TMA (Q, K), war
 constexpr int AO_TILE = 128;                        // query rows per CTA and keys per streamed tile
 constexpr int AO_TILE_BYTES = AO_TILE * kHeadDim * 2;
 constexpr int AO_STAGES = 2;
+constexpr int AO_SBUFS = 3;                         // S / P buffers in tensor memory (3 x 128 columns + 128 for O = 512)
 constexpr int AO_STAGE_BYTES = 2 * AO_TILE_BYTES;   // K tile, then V tile
 constexpr float kAoExpScale = 0.12751743074602468f; // log2(e) / sqrt(128)
 
@@ -40,7 +41,7 @@ struct AoShared {
   // computed, a V stage only after P V, and the next scores must not wait for the latter
   uint64_t k_full[AO_STAGES], k_empty[AO_STAGES];
   uint64_t v_full[AO_STAGES], v_empty[AO_STAGES];
-  uint64_t s_full[2], pv_done[2];
+  uint64_t s_full[AO_SBUFS], pv_done[AO_SBUFS];
   uint64_t p_full;
   uint64_t o_full;
   uint32_t tmem_base;
@@ -78,7 +79,7 @@ __global__ void __launch_bounds__(AO_THREADS) attn_out_tc_kernel(const __grid_co
       mbar_init(&sh->v_full[s], 1);
       mbar_init(&sh->v_empty[s], 1);
     }
-    for (int s = 0; s < 2; ++s) {
+    for (int s = 0; s < AO_SBUFS; ++s) {
       mbar_init(&sh->s_full[s], 1);
       mbar_init(&sh->pv_done[s], 1);
     }
@@ -93,7 +94,7 @@ __global__ void __launch_bounds__(AO_THREADS) attn_out_tc_kernel(const __grid_co
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem = sh->tmem_base;
-  const uint32_t ocol = 2 * AO_TILE;                               // O accumulator behind the two S buffers
+  const uint32_t ocol = AO_SBUFS * AO_TILE;                        // O accumulator behind the S buffers
   volatile int* abortp = &sh->abort;
 
   if (warp == 0) {
@@ -139,12 +140,11 @@ __global__ void __launch_bounds__(AO_THREADS) attn_out_tc_kernel(const __grid_co
       const uint64_t ad_q = smem_desc(smem_u32(qres), 16, 1024, kLayoutSw128);
       const uint64_t bd_ring = smem_desc(smem_u32(ring), 16, 1024, kLayoutSw128);
       wait_or_give_up(&sh->res_full, 0, abortp, status, 101);
-      uint32_t s1 = 0, ph1 = 0;
+      uint32_t s1 = 0, ph1 = 0, b1 = 0, bph1 = 0;     // bph1: parity of the buffer's current use
       for (int t = 0; t < ntile; ++t) {
-        const int b1 = t & 1;
         wait_or_give_up(&sh->k_full[s1], ph1, abortp, status, 102);
-        // buffer b1 held S and then P of tile t - 2: free once that tile's P V has completed
-        if (t >= 2) wait_or_give_up(&sh->pv_done[b1], ((t >> 1) - 1) & 1, abortp, status, 103);
+        // buffer b1 held S and then P of tile t - 3: free once that tile's P V has completed
+        if (t >= AO_SBUFS) wait_or_give_up(&sh->pv_done[b1], bph1 ^ 1, abortp, status, 103);
         if (*abortp) break;
         tc_fence_after_sync();
         const uint64_t bd0 = bd_ring + (uint64_t)(s1 * (AO_STAGE_BYTES >> 4));
@@ -155,6 +155,7 @@ __global__ void __launch_bounds__(AO_THREADS) attn_out_tc_kernel(const __grid_co
         mma_commit(&sh->k_empty[s1]);
         mma_commit(&sh->s_full[b1]);
         if (++s1 == AO_STAGES) { s1 = 0; ph1 ^= 1; }
+        if (++b1 == AO_SBUFS) { b1 = 0; bph1 ^= 1; }
       }
     }
   } else if (warp == 3 + AO_EPI_WARPS) {
@@ -162,7 +163,7 @@ __global__ void __launch_bounds__(AO_THREADS) attn_out_tc_kernel(const __grid_co
     if (lane == 0) {
       constexpr uint32_t idesc_o = idesc_f16(AO_TILE, kHeadDim, 0, 1);  // A = P (tensor memory), B = V (N-major)
       const uint64_t bd_vring = smem_desc(smem_u32(ring) + AO_TILE_BYTES, AO_TILE_BYTES / 2, 1024, kLayoutSw128);
-      uint32_t s2 = 0, vph = 0;
+      uint32_t s2 = 0, vph = 0, b2 = 0;
       for (int t = 0; t < ntile; ++t) {
         wait_or_give_up(&sh->v_full[s2], vph, abortp, status, 109);
         wait_or_give_up(&sh->p_full, t & 1, abortp, status, 104);
@@ -172,11 +173,12 @@ __global__ void __launch_bounds__(AO_THREADS) attn_out_tc_kernel(const __grid_co
 #pragma unroll
         for (int ks = 0; ks < AO_TILE / 16; ++ks)
           // k-step ks = keys 16 ks .. 16 ks + 15 of the tile = 8 packed columns inside the 32 S columns of part ks / 2
-          mma_f16_ts(tmem + ocol, tmem + (t & 1) * AO_TILE + 32 * (ks >> 1) + 8 * (ks & 1),
+          mma_f16_ts(tmem + ocol, tmem + b2 * AO_TILE + 32 * (ks >> 1) + 8 * (ks & 1),
                      bv0 + (uint64_t)(ks * (2048 >> 4)), idesc_o, (t | ks) ? 1u : 0u);
         mma_commit(&sh->v_empty[s2]);
-        mma_commit(&sh->pv_done[t & 1]);
+        mma_commit(&sh->pv_done[b2]);
         if (++s2 == AO_STAGES) { s2 = 0; vph ^= 1; }
+        if (++b2 == AO_SBUFS) b2 = 0;
       }
       mma_commit(&sh->o_full);
     }
@@ -218,7 +220,7 @@ __global__ void __launch_bounds__(AO_THREADS) attn_out_tc_kernel(const __grid_co
       tmem_st_wait();
       tc_fence_before_sync();
       mbar_arrive_warp(&sh->p_full);
-      if (b ^= 1, b == 0) bph ^= 1;
+      if (++b == AO_SBUFS) { b = 0; bph ^= 1; }
     }
     // ---- the finished rows: O[row][32 columns of this warp] ----
     wait_or_give_up(&sh->o_full, 0, abortp, status, 107);
