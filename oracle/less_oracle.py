@@ -402,7 +402,7 @@ def hellinger(p: np.ndarray, q: np.ndarray) -> float:
 NEVER = np.iinfo(np.int32).max
 
 
-def masked_parallel_attention(Q, K, V, exact_until, phi_fn, psi_fn):
+def masked_parallel_attention(Q, K, V, exact_until, phi_fn, psi_fn, rows=None):
     """The parallel form (Section 3.2, Inexpensive Training; Section 4.1): every row of the causal
     attention matrix at once.  Entry (i, j), j <= i, is exp(q_i . k_j / sqrt(D)) while key j is still
     in the sparse cache when query i attends, i.e. i < exact_until[j], and phi(q_i) psi(k_j)^T from
@@ -412,18 +412,20 @@ def masked_parallel_attention(Q, K, V, exact_until, phi_fn, psi_fn):
 
     The sparse policies here discard a pair once and for all, so one integer per key describes the
     mask: exact_until[j] = 1 + (the step at whose end j was evicted), NEVER if it stays.
-    Q, K, V: [S, D]; returns (out [S, D], A / row sums [S, S])."""
+    Q, K, V: [S, D]; returns (out [S, D], A / row sums [S, S]).  With `rows` (query positions) only
+    those rows are formed: out [len(rows), D], P [len(rows), S]; the rows do not depend on each other."""
     Q = np.asarray(Q, dtype=np.float64)
     K = np.asarray(K, dtype=np.float64)
     V = np.asarray(V, dtype=np.float64)
     eu = np.asarray(exact_until, dtype=np.int64)
     S, D = Q.shape
-    i = np.arange(S)[:, None]
+    qi = np.arange(S) if rows is None else np.asarray(rows, dtype=np.int64)
+    i = qi[:, None]
     j = np.arange(S)[None, :]
     causal = j <= i
     exact = causal & (i < eu[None, :])
-    A_exact = np.exp((Q @ K.T) / math.sqrt(D))
-    A_low = phi_fn(Q) @ psi_fn(K).T
+    A_exact = np.exp((Q[qi] @ K.T) / math.sqrt(D))
+    A_low = phi_fn(Q[qi]) @ psi_fn(K).T
     A = np.where(exact, A_exact, np.where(causal, A_low, 0.0))
     P = A / A.sum(axis=1, keepdims=True)
     return P @ V, P

@@ -230,3 +230,36 @@ def test_parallel_form_training_shape_sampled_instances():
         assert err <= harness.OUT_TOL
     ctx.close()
     torch.cuda.empty_cache()
+
+
+def test_parallel_form_long_sequences_sampled_rows():
+    """Sequences of 16 384 (128 key tiles per row block): sampled rows of two instances against the
+    oracle's rows, first and last rows and rows on both sides of tile boundaries included."""
+    from oracle import less_oracle as lo
+    from paper_2402_09398_b200 import binding
+    import harness
+    S = 16384
+    w = wl.CONFIGS[2].with_(batch=1, heads=4, prompt=S, heavy=819, recent=819)
+    W = wl.make_weights(w, DEV)
+    ctx = binding.from_workload(w, W, DEV, max_prefill_layers=1, flags=binding.LESS_WITH_PARALLEL_FORM)
+    layer = 30
+    Q, K, V = wl.make_prompt(w, layer, 1, DEV)
+    gen = torch.Generator(device=DEV).manual_seed(7)
+    pos = torch.arange(S, device=DEV).expand(w.batch, 1, w.heads, S)
+    eu = (pos + w.recent + torch.randint(0, 2 * w.slots, pos.shape, generator=gen, device=DEV)).to(torch.int32)
+    eu[:, :, :, ::61] = 2**31 - 1
+    eu = eu.contiguous()
+    out = ctx.masked_attention(Q, K, V, eu, layer_begin=layer)
+    torch.cuda.synchronize()
+    assert ctx.poll_status() == 0
+    rows = [0, 1, 127, 128, 129, 4095, 4096, 8191, 12345, S - 129, S - 128, S - 2, S - 1]
+    for head in (0, 3):
+        wts = [W[n][layer, head].double().cpu().numpy() for n in ("w_phi1", "w_phi2", "w_psi1", "w_psi2", "w_psi3")]
+        phi_fn, psi_fn = lo.make_mlp_maps(*wts)
+        ref, _ = lo.masked_parallel_attention(*(t[0, 0, head].double().cpu().numpy() for t in (Q, K, V)),
+                                              eu[0, 0, head].cpu().numpy(), phi_fn, psi_fn, rows=rows)
+        err = float(np.max(np.abs(out[0, 0, head][rows].double().cpu().numpy() - ref)))
+        print("parallel form 16384", head, err)
+        assert err <= harness.OUT_TOL
+    ctx.close()
+    torch.cuda.empty_cache()

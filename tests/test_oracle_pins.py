@@ -704,3 +704,13 @@ def test_parallel_form_mask_boundary_is_strict():
         if i >= 7:
             row[2] = low[i, 2]
         assert np.isclose(P[i, 2], want / row.sum(), rtol=1e-12)
+
+
+def test_parallel_form_row_subset_equals_the_full_matrix_rows():
+    w, Q, K, V, phi_fn, psi_fn = _sequence_case(114, S=30)
+    eu = np.arange(30) + 1 + (np.arange(30) * 7) % 11
+    out, P = lo.masked_parallel_attention(Q, K, V, eu, phi_fn, psi_fn)
+    rows = [0, 3, 17, 29]
+    out_r, P_r = lo.masked_parallel_attention(Q, K, V, eu, phi_fn, psi_fn, rows=rows)
+    assert np.array_equal(out_r, out[rows]) or np.allclose(out_r, out[rows], rtol=1e-13, atol=0)
+    assert np.allclose(P_r, P[rows], rtol=1e-13, atol=0)
