@@ -101,6 +101,9 @@ size_t carve(const Dims& d, char* base, Arena* a) {
   t.ws_psiop = (unsigned char*)take(Iw * St * 8192);
   t.ws_g = (float*)take(Iw * St * 128 * 4);
   t.ws_eu = (int32_t*)take(Iw * St * 128 * 4);
+  t.ws_ht = (float*)take(Iw * St * (R * D + R) * 4);
+  t.ws_hsum = (float*)take(Iw * St * (R * D + R) * 4);
+  t.ws_bucket = (int32_t*)take(Iw * St * 4);
   if (a) *a = t;
   return off;
 }

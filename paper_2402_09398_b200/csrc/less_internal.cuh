@@ -48,6 +48,9 @@ struct Arena {
   unsigned char* ws_psiop;  // [Iw][St][8 KB]  psi likewise
   float* ws_g;       // [Iw][St*128]  per row: log2 of (kernel value / value of the scaled operands)
   int32_t* ws_eu;    // [Iw][St*128]  exact_until, padded with zeros
+  float* ws_ht;      // [Iw][St][R*D + R]  H, z of every key tile
+  float* ws_hsum;    // [Iw][St][R*D + R]  per Q tile: H, z summed over the key tiles dead for it
+  int32_t* ws_bucket; // [Iw][St]  first Q tile a key tile is dead for
   uint4* ws_bx;      // [Iw*G][Sbx]  per prompt row: -(m_i sqrt(D) - log2(1/l_i) / c) as three fp16 parts (column sums)
 };
 

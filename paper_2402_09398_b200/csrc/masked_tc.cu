@@ -6,6 +6,8 @@
 //            phi(q_i) psi(k_j)^T          otherwise                      (j <= i)
 //     out_i = sum_j A_ij v_j / sum_j A_ij
 //
+// Key tiles whose keys have all been discarded before a Q tile's first row never stream past it: their
+// share of a row is phi(q_i) times the summed state of those tiles (see masked_tile_state_kernel).
 // Steps (launch_masked_form): psi(K) and phi(Q) come from the MLP kernel (psi_tc.cu);
 // masked_pack_kernel scales them by powers of two (phi per row, psi per instance), splits them into
 // fp16 hi + lo and writes them as operand tiles; masked_out_tc_kernel then works like the
@@ -43,6 +45,9 @@ struct MfParams {
   const int32_t* exact_until;   // [B, layer_count, Hd, S]
   float* out;                   // [B, layer_count, Hd, S, D]
   int St;                       // operand tiles per instance in the workspace
+  const float* phi;             // [Iw][Sp][R] phi(q_i), unscaled
+  const float* hsum;            // [Iw][St][R*D + R] per Q tile: H, z summed over the key tiles that are dead for it
+  const int32_t* bucket;        // [Iw][St] first Q tile for which a key tile is dead (all its keys discarded before it)
 };
 
 // ------------------------------------------------------------------------------------------- //
@@ -130,7 +135,82 @@ __global__ void __launch_bounds__(MF_TILE) masked_pack_kernel(PfParams p, MfPara
 }
 
 // ------------------------------------------------------------------------------------------- //
-// One CTA = one 128-row Q tile of one instance; key tiles 0 .. diagonal stream past it.
+// Dead key tiles.  A key tile T is dead for a Q tile q once every one of its keys has been discarded
+// before the Q tile's first row (max exact_until over the tile <= 128 q): then all its entries are kernel
+// values for all 128 rows, and its share of row i is phi(q_i) H_T and phi(q_i) z_T with
+// H_T = sum_j psi(k_j)^T v_j, z_T = sum_j psi(k_j) over the tile (Eq. 4, Eq. 5 for a block).  A tile that
+// is dead for q stays dead for every later Q tile, so Hsum_q = sum of H_T over the tiles dead for q is a
+// running sum over "buckets" (the first Q tile a key tile is dead for).  The attention kernel streams
+// only the tiles that are not dead; for an H2O-like schedule that is a band below the diagonal plus the
+// tiles that hold keys kept for good, instead of the whole triangle.
+// ------------------------------------------------------------------------------------------- //
+template <int R>
+__global__ void __launch_bounds__(MF_TILE) masked_tile_state_kernel(PfParams p, MfParams mf, float* ht, int32_t* bucket) {
+  const int T = blockIdx.x, g = blockIdx.y, d = threadIdx.x;
+  const InstMap im = map_instance(p, g);
+  const int j0 = T * MF_TILE, nj = min(MF_TILE, p.S - j0);
+  __shared__ float ps[MF_TILE][R];
+  __shared__ int s_death[MF_TILE / 32];
+  int death = 0;
+  if (d < nj) {
+#pragma unroll
+    for (int q = 0; q < R; ++q) ps[d][q] = p.a.ws_psi[((size_t)g * p.Sp + j0 + d) * R + q];
+    death = mf.exact_until[im.in_row0 + j0 + d];
+  }
+  death = __reduce_max_sync(0xffffffffu, death);
+  if ((d & 31) == 0) s_death[d >> 5] = death;
+  __syncthreads();
+  float h[R];
+#pragma unroll
+  for (int q = 0; q < R; ++q) h[q] = 0.f;
+  const __half* vcol = p.V + (im.in_row0 + j0) * kHeadDim + d;
+  for (int j = 0; j < nj; ++j) {
+    const float v = __half2float(vcol[(size_t)j * kHeadDim]);
+#pragma unroll
+    for (int q = 0; q < R; ++q) h[q] = fmaf(ps[j][q], v, h[q]);
+  }
+  float* dst = ht + ((size_t)g * mf.St + T) * (R * kHeadDim + R);
+#pragma unroll
+  for (int q = 0; q < R; ++q) dst[q * kHeadDim + d] = h[q];
+  if (d < R) {
+    float z = 0.f;
+    for (int j = 0; j < nj; ++j) z += ps[j][d];
+    dst[R * kHeadDim + d] = z;
+  }
+  if (d == 0) {
+    int dm = s_death[0];
+#pragma unroll
+    for (int w = 1; w < MF_TILE / 32; ++w) dm = max(dm, s_death[w]);
+    // first Q tile whose first row is >= every exact_until of the tile; never before the tile below the diagonal
+    const long long b = ((long long)dm + MF_TILE - 1) / MF_TILE;
+    bucket[(size_t)g * mf.St + T] = (int)min(max(b, (long long)T + 1), (long long)0x7fffffff);
+  }
+}
+
+// Hsum_q = sum of H_T, z_T over the key tiles with bucket <= q: one thread per element, key tiles in order
+// (a fixed order of additions), then a running sum over q.
+template <int R>
+__global__ void __launch_bounds__(256) masked_prefix_kernel(int tiles, int St, const float* ht, const int32_t* bucket, float* hsum) {
+  const int g = blockIdx.y, e = blockIdx.x * 256 + threadIdx.x;
+  constexpr int E = R * kHeadDim + R;
+  if (e >= E) return;
+  const float* src = ht + (size_t)g * St * E + e;
+  float* dst = hsum + (size_t)g * St * E + e;
+  const int32_t* bk = bucket + (size_t)g * St;
+  for (int q = 0; q < tiles; ++q) dst[(size_t)q * E] = 0.f;
+  for (int T = 0; T < tiles; ++T) {
+    const int b = bk[T];
+    if (b < tiles) dst[(size_t)b * E] += src[(size_t)T * E];
+  }
+  float run = 0.f;
+  for (int q = 0; q < tiles; ++q) {
+    run += dst[(size_t)q * E];
+    dst[(size_t)q * E] = run;
+  }
+}
+
+// ------------------------------------------------------------------------------------------- //
+// One CTA = one 128-row Q tile of one instance; the key tiles 0 .. diagonal that are not dead stream past it.
 // ------------------------------------------------------------------------------------------- //
 struct MfShared {
   uint64_t res_full;
@@ -146,6 +226,7 @@ struct MfShared {
   int abort;
   float rsum[4][MF_TILE];
   float rmax[4][MF_TILE];
+  int nlive;                                          // key tiles of this Q tile that are not dead
 };
 
 __device__ __forceinline__ float mf_ex2(float x) {
@@ -204,10 +285,22 @@ __global__ void __launch_bounds__(MF_THREADS) masked_out_tc_kernel(const __grid_
     mbar_fence_init();
   }
   if (warp == 1) tmem_alloc(&sh->tmem_base, 512);
+  // A key tile all of whose keys were discarded before this Q tile's first row is dead for it: its
+  // entries are phi(q_i) psi(k_j)^T for every row, so its whole contribution is phi(q_i) (sum psi^T v) and
+  // phi(q_i) (sum psi), which masked_prefix_kernel has added up per Q tile (Eq. 6 for a block of keys).
+  // Only the other tiles stream past the Q tile; every role skips the dead ones by the same test.
+  const int32_t* bucket = mf.bucket + (size_t)g * mf.St;
+  if (warp == 0) {
+    int c = 0;
+    for (int t = lane; t <= tile; t += 32) c += __ldg(bucket + t) > tile;
+    c = __reduce_add_sync(0xffffffffu, c);
+    if (lane == 0) sh->nlive = c;
+  }
   tc_fence_before_sync();
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem = sh->tmem_base;
+  const int nlive = sh->nlive;
   const uint32_t ocol = 2 * MF_TILE, lcol = 3 * MF_TILE;           // O and L behind the two S buffers
   volatile int* abortp = &sh->abort;
 
@@ -220,8 +313,10 @@ __global__ void __launch_bounds__(MF_THREADS) masked_out_tc_kernel(const __grid_
       tma_load_2d(qres + MF_TILE_BYTES / 2, &tm_q, 64, row0, &sh->res_full);
       bulk_g2s(phires, p.a.ws_phiop + op0 + (size_t)tile * MF_OP_BYTES, MF_OP_BYTES, &sh->res_full);
       uint32_t s = 0, ph = 0;
-      for (int u = 0; u < 2 * ntile; ++u) {              // two sweeps over the key tiles
-        const int t = u < ntile ? u : u - ntile;
+      int u = 0;                                         // live tiles issued so far, both sweeps
+      for (int sweep = 0; sweep < 2 && !*abortp; ++sweep)
+      for (int t = 0; t < ntile; ++t) {
+        if (__ldg(bucket + t) <= tile) continue;         // dead for this Q tile
         wait_or_give_up(&sh->k_empty[s], ph ^ 1, abortp, status, 110);
         const int es = u % MF_EU_SLOTS;
         wait_or_give_up(&sh->eu_empty[es], ((u / MF_EU_SLOTS) & 1) ^ 1, abortp, status, 111);
@@ -235,6 +330,7 @@ __global__ void __launch_bounds__(MF_THREADS) masked_out_tc_kernel(const __grid_
         mbar_expect_tx(&sh->eu_full[es], MF_EU_BYTES);
         bulk_g2s(euring + es * MF_EU_BYTES, p.a.ws_eu + rc0 + (size_t)t * MF_TILE, MF_EU_BYTES, &sh->eu_full[es]);
         if (++s == MF_STAGES) { s = 0; ph ^= 1; }
+        ++u;
       }
     }
   } else if (warp == 2 + MF_EPI_WARPS) {
@@ -242,6 +338,7 @@ __global__ void __launch_bounds__(MF_THREADS) masked_out_tc_kernel(const __grid_
     if (lane == 0) {
       uint32_t s = 0, ph = 0;
       for (int t = 0; t < ntile; ++t) {
+        if (__ldg(bucket + t) <= tile) continue;
         wait_or_give_up(&sh->v_empty[s], ph ^ 1, abortp, status, 112);
         if (*abortp) break;
         const int krow = (int)(im.in_row0 + (size_t)t * MF_TILE);
@@ -266,13 +363,13 @@ __global__ void __launch_bounds__(MF_THREADS) masked_out_tc_kernel(const __grid_
       constexpr uint64_t kPair = 4096 >> 4;                             // two chunks = one 16-wide k-step further
       wait_or_give_up(&sh->res_full, 0, abortp, status, 113);
       uint32_t s1 = 0, ph1 = 0;
-      for (int u = 0; u < 2 * ntile; ++u) {
+      for (int u = 0; u < 2 * nlive; ++u) {            // u counts live tiles; which tile it is does not matter here
         const int b1 = u & 1;
         wait_or_give_up(&sh->k_full[s1], ph1, abortp, status, 114);
         // buffer b1 held tile u - 2: read by the epilogue (s_free) and, in the second sweep, rewritten
         // with P and read by that tile's P V (pv_done); the single L buffer held tile u - 1 (l_free)
         if (u >= 2) wait_or_give_up(&sh->s_free[b1], ((u >> 1) - 1) & 1, abortp, status, 115);
-        if (u - 2 >= ntile) wait_or_give_up(&sh->pv_done[b1], ((u - 2 - ntile) >> 1) & 1, abortp, status, 123);
+        if (u - 2 >= nlive) wait_or_give_up(&sh->pv_done[b1], ((u - 2 - nlive) >> 1) & 1, abortp, status, 123);
         if (*abortp) break;
         tc_fence_after_sync();
         const uint64_t bd0 = bd_ring + (uint64_t)(s1 * (MF_STAGE_BYTES >> 4));
@@ -305,8 +402,8 @@ __global__ void __launch_bounds__(MF_THREADS) masked_out_tc_kernel(const __grid_
       constexpr uint32_t idesc_o = idesc_f16(MF_TILE, kHeadDim, 0, 1);  // A = P (tensor memory), B = V (N-major)
       const uint64_t bd_vring = smem_desc(smem_u32(ring) + MF_TILE_BYTES, MF_TILE_BYTES / 2, 1024, kLayoutSw128);
       uint32_t s2 = 0, vph = 0;
-      for (int t = 0; t < ntile; ++t) {
-        const int bt = (ntile + t) & 1;                  // the S buffer this tile's P lives in
+      for (int t = 0; t < nlive; ++t) {                // t counts the live tiles of the second sweep
+        const int bt = (nlive + t) & 1;                  // the S buffer this tile's P lives in
         wait_or_give_up(&sh->v_full[s2], vph, abortp, status, 117);
         wait_or_give_up(&sh->p_full, t & 1, abortp, status, 118);
         if (*abortp) break;
@@ -335,10 +432,11 @@ __global__ void __launch_bounds__(MF_THREADS) masked_out_tc_kernel(const __grid_
     float mx = -INFINITY, ml = 0.f;
     float nb = 0.f, gi = 0.f, rsum = 0.f, rsum2 = 0.f;
     uint32_t b = 0, bph = 0;
-    for (int u = 0; u < 2 * ntile; ++u) {
-      const bool second = u >= ntile;
-      const int t = second ? u - ntile : u;
-      if (u == ntile) {
+    int u = 0;                                           // live tiles done so far, both sweeps
+    for (int sweep = 0; sweep < 2; ++sweep)
+    for (int t = 0; t < ntile; ++t) {
+      const bool second = sweep == 1;
+      if (second && t == 0) {
         // between the sweeps: E = log2 of the row's largest entry; exact entries become
         // exp2(c S - E), kernel entries L 2^(lscale - E)
         sh->rsum[part][r] = mx;
@@ -350,14 +448,17 @@ __global__ void __launch_bounds__(MF_THREADS) masked_out_tc_kernel(const __grid_
         const float ea = mx * kMfExpScale;               // -inf without exact entries
         const float el = ml > 0.f ? log2f(ml) + lscale : -INFINITY;
         const float E = fmaxf(ea, el);
-        if (live && E > -INFINITY && E < INFINITY) {
-          nb = -E;
-          gi = exp2f(fminf(lscale - E, 120.f));
+        if (live && E < INFINITY) {
+          // a row with nothing in its live tiles (E = -inf) keeps scale 1 for the dead tiles' part
+          const float Es = E > -INFINITY ? E : 0.f;
+          nb = -Es;
+          gi = exp2f(fminf(lscale - Es, 120.f));
         } else {                                         // a row past the sequence, or one with nothing in it: all zeros
           nb = -INFINITY;
           gi = 0.f;
         }
       }
+      if (__ldg(bucket + t) <= tile) continue;           // dead for this Q tile
       wait_or_give_up(&sh->s_full[b], bph, abortp, status, 119);
       const int es = u % MF_EU_SLOTS;
       wait_or_give_up(&sh->eu_full[es], (u / MF_EU_SLOTS) & 1, abortp, status, 120);
@@ -438,11 +539,39 @@ __global__ void __launch_bounds__(MF_THREADS) masked_out_tc_kernel(const __grid_
         mbar_arrive_warp(&sh->p_full);
       }
       if (b ^= 1, b == 0) bph ^= 1;
+      ++u;
     }
     // ---- the row's normaliser: the four parts' sums ----
     sh->rsum[part][r] = rsum + rsum2;
     mf_epi_sync();
-    const float total = (sh->rsum[0][r] + sh->rsum[1][r]) + (sh->rsum[2][r] + sh->rsum[3][r]);
+    float total = (sh->rsum[0][r] + sh->rsum[1][r]) + (sh->rsum[2][r] + sh->rsum[3][r]);
+    // the dead key tiles: phi(q_i) Hsum and phi(q_i) zsum, in the scale of P (2^-E_i = 2^nb)
+    const float* hs = mf.hsum + ((size_t)g * mf.St + tile) * (R * kHeadDim + R);
+    float ph[R], dead[32];
+    const float f = live ? exp2f(fminf(nb, 120.f)) : 0.f;           // nb = -inf for an empty row: 0
+#pragma unroll
+    for (int e = 0; e < 32; ++e) dead[e] = 0.f;
+    if (live) {
+      float dz = 0.f;
+#pragma unroll
+      for (int q = 0; q < R; ++q) {
+        ph[q] = mf.phi[((size_t)g * p.Sp + i) * R + q] * f;
+        dz = fmaf(ph[q], __ldg(hs + R * kHeadDim + q), dz);
+      }
+      total += dz;
+#pragma unroll
+      for (int q = 0; q < R; ++q) {
+        const float4* hrow = reinterpret_cast<const float4*>(hs + q * kHeadDim + part * 32);
+#pragma unroll
+        for (int e4 = 0; e4 < 8; ++e4) {
+          const float4 h = __ldg(hrow + e4);
+          dead[e4 * 4] = fmaf(ph[q], h.x, dead[e4 * 4]);
+          dead[e4 * 4 + 1] = fmaf(ph[q], h.y, dead[e4 * 4 + 1]);
+          dead[e4 * 4 + 2] = fmaf(ph[q], h.z, dead[e4 * 4 + 2]);
+          dead[e4 * 4 + 3] = fmaf(ph[q], h.w, dead[e4 * 4 + 3]);
+        }
+      }
+    }
     const float inv = total > 0.f ? 1.0f / total : 0.f;
     // ---- the finished rows: O[row][32 columns of this warp] / r_i ----
     wait_or_give_up(&sh->o_full, 0, abortp, status, 122);
@@ -456,8 +585,8 @@ __global__ void __launch_bounds__(MF_THREADS) masked_out_tc_kernel(const __grid_
 #pragma unroll
         for (int e = 0; e < 32; e += 4)
           *reinterpret_cast<float4*>(orow + e) =
-              make_float4(__uint_as_float(o[e]) * inv, __uint_as_float(o[e + 1]) * inv,
-                          __uint_as_float(o[e + 2]) * inv, __uint_as_float(o[e + 3]) * inv);
+              make_float4((__uint_as_float(o[e]) + dead[e]) * inv, (__uint_as_float(o[e + 1]) + dead[e + 1]) * inv,
+                          (__uint_as_float(o[e + 2]) + dead[e + 2]) * inv, (__uint_as_float(o[e + 3]) + dead[e + 3]) * inv);
       }
     }
   }
@@ -509,6 +638,20 @@ int launch_masked_form(less_ctx* c, int layer0, int nl, int lj0, int layer_count
     LaunchScope scope(c, LESS_KERNEL_MASKED_PACK, s);
     if (d.R == 8) masked_pack_kernel<8><<<dim3(tiles, G), MF_TILE, 0, s>>>(p, mf);
     else masked_pack_kernel<16><<<dim3(tiles, G), MF_TILE, 0, s>>>(p, mf);
+  }
+  mf.phi = c->a.ws_phi;
+  mf.hsum = c->a.ws_hsum;
+  mf.bucket = c->a.ws_bucket;
+  {
+    LaunchScope scope(c, LESS_KERNEL_MASKED_PACK, s);
+    if (d.R == 8) masked_tile_state_kernel<8><<<dim3(tiles, G), MF_TILE, 0, s>>>(p, mf, c->a.ws_ht, c->a.ws_bucket);
+    else masked_tile_state_kernel<16><<<dim3(tiles, G), MF_TILE, 0, s>>>(p, mf, c->a.ws_ht, c->a.ws_bucket);
+  }
+  {
+    LaunchScope scope(c, LESS_KERNEL_MASKED_PACK, s);
+    const int E = d.R * kHeadDim + d.R;
+    if (d.R == 8) masked_prefix_kernel<8><<<dim3((E + 255) / 256, G), 256, 0, s>>>(tiles, d.St, c->a.ws_ht, c->a.ws_bucket, c->a.ws_hsum);
+    else masked_prefix_kernel<16><<<dim3((E + 255) / 256, G), 256, 0, s>>>(tiles, d.St, c->a.ws_ht, c->a.ws_bucket, c->a.ws_hsum);
   }
   CUtensorMap tq, tk, tv;
   const uint64_t rows = (uint64_t)d.B * layer_count * d.Hd * S;

@@ -215,7 +215,11 @@ def test_parallel_form_training_shape_sampled_instances():
     gen = torch.Generator(device=DEV).manual_seed(99)
     pos = torch.arange(S, device=DEV).expand(w.batch, 1, w.heads, S)
     eu = (pos + w.recent + torch.randint(0, 2 * w.slots, pos.shape, generator=gen, device=DEV)).to(torch.int32)
-    eu[:, :, :, ::97] = 2**31 - 1                         # some keys stay for good
+    # some keys stay for good: the first four (sinks) and a few in every eighth key tile, so that most
+    # key tiles are dead (wholly discarded) for the later row blocks and some never are
+    eu[:, :, :, :4] = 2**31 - 1
+    eu[:, :, :, 1024::1024] = 2**31 - 1
+    eu[:, :, :, 1500::1024] = 2**31 - 1
     eu = eu.contiguous()
     out = ctx.masked_attention(Q, K, V, eu, layer_begin=layer)
     torch.cuda.synchronize()
@@ -247,7 +251,9 @@ def test_parallel_form_long_sequences_sampled_rows():
     gen = torch.Generator(device=DEV).manual_seed(7)
     pos = torch.arange(S, device=DEV).expand(w.batch, 1, w.heads, S)
     eu = (pos + w.recent + torch.randint(0, 2 * w.slots, pos.shape, generator=gen, device=DEV)).to(torch.int32)
-    eu[:, :, :, ::61] = 2**31 - 1
+    eu[:, :, :, :4] = 2**31 - 1                          # sinks; every sixteenth key tile keeps two keys for good
+    eu[:, :, :, 2048::2048] = 2**31 - 1
+    eu[:, :, :, 2100::2048] = 2**31 - 1
     eu = eu.contiguous()
     out = ctx.masked_attention(Q, K, V, eu, layer_begin=layer)
     torch.cuda.synchronize()
