@@ -681,7 +681,16 @@ def run_masked(args):
         inst = w.batch * w.heads
         tokens = inst * S * world
         causal = S * (S + 1) // 2
-        fl = {"masked_out": inst * causal * (4 * w.head_dim + 2 * w.rank),
+        # flops of the entries the kernel has to form: 128 x 128 tiles that are not dead (a key tile all of
+        # whose keys were discarded before a Q tile's first row is handled through its summed state)
+        nt = (S + 127) // 128
+        eu_pad = torch.full((w.batch, 1, w.heads, nt * 128), 0, dtype=torch.int64, device=dev)
+        eu_pad[..., :S] = eu.long()
+        death = eu_pad.view(w.batch, 1, w.heads, nt, 128).amax(-1)
+        first_dead = torch.maximum((death + 127) // 128, torch.arange(nt, device=dev) + 1).clamp(max=nt)
+        live_pairs = int((first_dead - torch.arange(nt, device=dev)).sum().item())
+        live_frac = live_pairs / (inst * nt * (nt + 1) / 2)
+        fl = {"masked_out": live_pairs * 128 * 128 * (4 * w.head_dim + 2 * w.rank),
               "psi": inst * S * 2 * (2 * w.head_dim * w.hidden + 2 * w.hidden * w.rank + w.rank * w.rank)}
         kt = {k: (prof[k][0] / prof[k][1] if prof[k][1] else 0.0) for k in prof}
         kt["psi"] *= 2                                   # psi and phi launches are booked under the same id
@@ -695,7 +704,7 @@ def run_masked(args):
                 "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
                 "dtype": "f16 inputs, f32 accumulate", "data": "synthetic",
                 "config": {"workload": f"parallel form (B={w.batch}, {w.heads} heads, sequences of {S}, one layer per step, R={w.rank})",
-                           "instances_per_step": inst, "l2": "inputs, operands and output of a step exceed the 126 MB L2"
+                           "instances_per_step": inst, "live_tile_fraction": live_frac, "l2": "inputs, operands and output of a step exceed the 126 MB L2"
                            if inst * S * 1300 > 126e6 else "a step's data fit the L2"},
                 "clocks": clocks,
                 "e2e": {"value": tokens / (ms_e2e * 1e-3), "unit": "head-tokens/s",
