@@ -694,6 +694,7 @@ def run_masked(args):
               "psi": inst * S * 2 * (2 * w.head_dim * w.hidden + 2 * w.hidden * w.rank + w.rank * w.rank)}
         kt = {k: (prof[k][0] / prof[k][1] if prof[k][1] else 0.0) for k in prof}
         kt["psi"] *= 2                                   # psi and phi launches are booked under the same id
+        kt["masked_pack"] *= 3                           # operand pack, tile states, running sums
         dominant = max(fl, key=lambda k: kt.get(k, 0.0))
         pth = os.path.join(ROOT, "MEASURED_PEAKS.json")
         peak, kind = (float(json.load(open(pth))["bf16_tflops_sustained"]), "of measured (sustained bf16 = fp16 rate)") \
