@@ -1,6 +1,7 @@
 // Blackwell (sm_100a) tensor-core plumbing used by the prompt-phase kernels:
 // TMA tiled loads (no multicast anywhere), tcgen05 MMA with operands in shared
-// memory and accumulators in tensor memory, tensor-memory allocation and loads.
+// memory (or the A operand in tensor memory) and accumulators in tensor memory,
+// tensor-memory allocation, loads and stores.
 #pragma once
 
 #include <cuda.h>
