@@ -169,7 +169,7 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_kernel(DecParams p) {
   half8_to_float(*reinterpret_cast<const uint4*>(p.q + inst * kHeadDim + l16 * 8), qf);
 
   // ---- scores s_i = q . k_i / sqrt(D) over live slots, and the new pair ----
-#pragma unroll 4
+#pragma unroll 8
   for (int r0 = 0; r0 < n; r0 += DEC_RG) {         // r0 is block-uniform: shuffles stay converged
     const int r = r0 + rg;
     float dot = 0.f;
@@ -214,7 +214,7 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_kernel(DecParams p) {
   float u[8];
 #pragma unroll
   for (int c = 0; c < 8; ++c) u[c] = 0.f;
-#pragma unroll 4
+#pragma unroll 8
   for (int r = rg; r < n; r += DEC_RG) {
     float vf[8];
     half8_to_float(ldg_stream(Vb + (size_t)r * kHeadDim + l16 * 8), vf);
