@@ -32,11 +32,11 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures
 # summarised under profiles/ (None where no capture of that kernel and workload exists)
 NCU_TRAFFIC_BYTES = {
-    (2, "feature_map"): 285.91e6 + 5.83e6,   # profiles/decode_step_cfg2.md
-    (2, "decode"): 113.87e6 + 3.32e6,
+    (2, "feature_map"): 285.91e6 + 6.29e6,   # profiles/decode_step_cfg2.md
+    (2, "decode"): 113.88e6 + 3.77e6,
     # cfg3 captured at batch 16 (a quarter of the instances): the decode kernel's traffic is per
     # instance and scales by 4; the feature maps' weight traffic does not scale and is not listed
-    (3, "decode"): 4 * (1.824e9 + 50.9e6),
+    (3, "decode"): 4 * (1.824e9 + 56.1e6),
 }
 
 
