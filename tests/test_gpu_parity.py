@@ -514,6 +514,9 @@ def _schedule(w, kind, S, seed):
         return torch.full(shape, 2**31 - 1, dtype=torch.int32)
     if kind == "at_once":
         return (pos + 1).to(torch.int32)
+    if kind == "no_self":         # keys that are discarded before their own query attends (not what a policy
+        # produces, but the definition covers it): even the diagonal entry is a kernel value for most rows
+        return (pos - torch.randint(0, 50, shape, generator=g)).clamp(min=0).to(torch.int32)
     if kind == "banded":          # an H2O-like schedule: short lives, a few keys kept for good in two key tiles only
         eu = pos + 1 + torch.randint(0, 150, shape, generator=g)
         eu[..., :4] = 2**31 - 1
@@ -543,7 +546,8 @@ def _check_parallel_form(w, W, Q, K, V, eu, out, instances, psi_scale=None):
 
 @pytest.mark.parametrize("kind,rank,S,std", [("random", 8, 300, 0.1), ("random", 16, 513, 0.2), ("never", 8, 131, 0.1),
                                              ("at_once", 16, 257, 0.2), ("random", 8, 128, 0.3), ("random", 16, 40, 0.1),
-                                             ("banded", 8, 1500, 0.2), ("banded", 16, 1153, 0.3)])
+                                             ("banded", 8, 1500, 0.2), ("banded", 16, 1153, 0.3),
+                                             ("no_self", 8, 700, 0.3)])
 def test_parallel_form_against_the_oracle(kind, rank, S, std):
     from paper_2402_09398_b200 import binding
     w = small(30 + rank, prompt=S, rank=rank, weight_std=std)
