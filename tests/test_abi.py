@@ -89,3 +89,29 @@ def test_product_never_imports_the_oracle():
                 text = open(os.path.join(dirpath, f)).read()
                 assert not re.search(r"^\s*(from|import)\s+oracle\b", text, flags=re.M), f
                 assert "oracle/" not in text and "less_oracle" not in text, f
+
+
+def test_binding_structs_match_the_header(B, tmp_path):
+    """The ctypes mirrors of less_config and less_weights have the size and the field offsets a C
+    compiler gives the header's structs (a field added on one side only would shift every later one)."""
+    import shutil
+    import subprocess
+    gcc = shutil.which("gcc")
+    if gcc is None:
+        pytest.skip("no C compiler")
+    fields_c = [n for n, _ in B.less_config._fields_]
+    fields_w = [n for n, _ in B.less_weights._fields_]
+    src = tmp_path / "layout.c"
+    lines = ['#include <stdio.h>', '#include <stddef.h>', '#include "less.h"', 'int main(void) {',
+             '  printf("%zu %zu\\n", sizeof(less_config), sizeof(less_weights));']
+    lines += [f'  printf("%zu\\n", offsetof(less_config, {n}));' for n in fields_c]
+    lines += [f'  printf("%zu\\n", offsetof(less_weights, {n}));' for n in fields_w]
+    lines += ['  return 0;', '}']
+    src.write_text("\n".join(lines))
+    exe = tmp_path / "layout"
+    subprocess.run([gcc, "-I", os.path.join(ROOT, "include"), str(src), "-o", str(exe)], check=True)
+    out = subprocess.run([str(exe)], check=True, capture_output=True, text=True).stdout.split()
+    assert int(out[0]) == C.sizeof(B.less_config) and int(out[1]) == C.sizeof(B.less_weights)
+    offs = [int(x) for x in out[2:]]
+    want = [getattr(B.less_config, n).offset for n in fields_c] + [getattr(B.less_weights, n).offset for n in fields_w]
+    assert offs == want
