@@ -27,10 +27,9 @@
  *     LESS_NO_OVERLAP (no programmatic dependent launch of the decode kernel),
  *     LESS_SCORE_KERNEL=plain (CUDA-core prompt scoring),
  *     LESS_FEATURE_STAGES=n (cap on the feature kernels' weight ring),
- *     LESS_GROUP_KERNEL=teams|rows|mma (grouped query heads: force the decode kernel with
- *     one 128-thread team per query head, the one with one 128-thread CTA per KV head on
- *     CUDA cores, or that one with its two contractions as warp-level tensor-core
- *     products; by default the number of KV heads per multiprocessor picks teams or mma).
+ *     LESS_GROUP_KERNEL=rows (grouped query heads: the CUDA-core decode kernel instead of
+ *     the one with its two contractions as warp-level tensor-core products),
+ *     LESS_FEATURE_CTAS=n (cap on the persistent CTAs of the tensor-core feature kernels).
  */
 #ifndef LESS_B200_H
 #define LESS_B200_H
@@ -62,14 +61,14 @@ enum {
 /* flags */
 enum {
   /* H2O accumulates e^{s_i} / (sparse-only denominator) instead of Eq. 3's
-   * full denominator (the paper only says "accumulates attention
-   * probabilities", Section 2.1). */
+   * full denominator (Section 2.1 describes H2O as summing the attention
+   * probabilities a token receives and does not say under which normaliser). */
   LESS_SCORE_NORM_SPARSE = 1u,
   /* Sparse policy alone (the paper's Baseline / Baseline+, Section 4):
    * evicted pairs are dropped, H and z stay zero. */
   LESS_NO_STATE = 2u,
-  /* Lambda-masking as the sparse policy (Section 4: "the cache consists of the
-   * first 4 and most recent tokens") instead of H2O: `heavy` counts the first
+  /* Lambda-masking as the sparse policy (Section 4: a fixed handful of first
+   * positions plus the recent window are cached) instead of H2O: `heavy` counts the first
    * positions, which are never evicted, `recent` the sliding window; the prompt
    * keeps positions [0, heavy) and the last `recent`, a decode step evicts the
    * lowest position >= heavy.  Accumulated scores are not used (prompt scoring
@@ -85,7 +84,10 @@ enum {
    * LESS_POLICY_LAMBDA. */
   LESS_POLICY_TOVA = 8u,
   /* Reserve the workspace of less_masked_attention (the parallel form) in the arena. */
-  LESS_WITH_PARALLEL_FORM = 16u
+  LESS_WITH_PARALLEL_FORM = 16u,
+  /* less_decode_step / less_decode_step_host write the attention output as fp16 (rounded once
+   * from the fp32 result of Eq. 3) instead of fp32: half the output traffic of a step. */
+  LESS_OUT_F16 = 32u
 };
 
 #define LESS_MAX_SLOTS 32768
@@ -176,7 +178,7 @@ int less_masked_attention(less_ctx* ctx, int32_t layer_begin, int32_t layer_coun
  *   the new pair overwrites the victim's slot in place (Section 3.2), else
  *   it takes the next free slot.
  * q: device fp16 [B, L, H * group, D]; k, v: device fp16 [B, L, H, D]; out: device fp32
- * [B, L, H * group, D] (query head h * group + g belongs to KV head h).  With group > 1
+ * (fp16 with LESS_OUT_F16) [B, L, H * group, D] (query head h * group + g belongs to KV head h).  With group > 1
  * (Section 3.2: multi-query attention) every query head has its own phi and its own Eq. 3 over
  * the KV head's cache and state, and the H2O score of an entry grows by the sum of the query
  * heads' probabilities; policies: H2O and Lambda-masking.
@@ -192,10 +194,11 @@ int less_decode_step(less_ctx* ctx, const void* q, const void* k, const void* v,
 
 /* The same step for callers whose tensors live in host memory (Algorithm 1's
  * inputs and return value): q host fp16 [B, L, H * group, D], k, v host fp16
- * [B, L, H, D], out host fp32 [B, L, H * group, D].  q and k are copied to staging buffers inside the arena; v and
- * out are read / written in place by the decode kernel when they lie in pinned
- * (page-locked, device-mapped) memory, else they are staged and copied too.
- * Everything runs on the given stream, which is synchronised before returning. */
+ * [B, L, H, D], out host fp32 (fp16 with LESS_OUT_F16) [B, L, H * group, D].  q and k are copied
+ * to staging buffers inside the arena - in ONE copy when k_host starts exactly where q_host ends
+ * (one host block [q | k]), else in two; v and out are read / written in place by the decode
+ * kernel when they lie in pinned (page-locked, device-mapped) memory, else they are staged and
+ * copied too.  Everything runs on the given stream, which is synchronised before returning. */
 int less_decode_step_host(less_ctx* ctx, const void* q_host, const void* k_host, const void* v_host,
                           void* out_host, void* cuda_stream);
 
@@ -255,6 +258,22 @@ int less_poll_status(less_ctx* ctx, void* cuda_stream);
 /* Kernels of this library launched through this context so far. */
 int64_t less_launch_count(const less_ctx* ctx);
 
+/* Name of the kernel variant last launched under a LESS_KERNEL_* id (template arguments
+ * included), "" if none yet.  The string lives in the context. */
+const char* less_kernel_variant(const less_ctx* ctx, int kernel_id);
+
+/* The where-code that came with the status word at the last less_poll_status (which wait gave
+ * up, which check refused), 0 if the status was clean. */
+int less_last_status_where(const less_ctx* ctx);
+
+/* Self-test of the bounded device-side waits (no counterpart in the paper).  Launches one small
+ * CTA whose consumer waits, for at most `polls` polls (1 .. 2^20), on a barrier nothing ever
+ * arrives at, through the same helper every pipeline of the library waits with.  The wait runs
+ * out, the kernel returns, and the context's status word then reads LESS_ERR_DEVICE_TIMEOUT
+ * (less_poll_status; less_last_status_where gives 90).  The status word is sticky: use a context
+ * of its own for this call.  Asynchronous on the given stream. */
+int less_selftest_wait_timeout(less_ctx* ctx, uint32_t polls, void* cuda_stream);
+
 /* The paper has no counterpart for this entry point: it exists for callers
  * that may not allocate device memory (a process whose memory pool owns the
  * whole GPU, a plugin that is only handed buffers and a stream, code that must
@@ -275,7 +294,9 @@ int64_t less_launch_count(const less_ctx* ctx);
  *   - no part of the array needs clearing between calls (each call overwrites
  *     every row it reads);
  *   - the first call on each device looks up the array's device address: make
- *     that call with the device current and outside any stream capture.
+ *     that call with the device current and outside any stream capture; first
+ *     calls from several host threads at once are safe (the lookup is idempotent
+ *     and its result is published atomically).
  * Asynchronous on the given stream. */
 #define LESS_NOALLOC_MAX_ROWS 65536
 #define LESS_ERR_NOALLOC_TOO_LARGE (-12)

@@ -22,13 +22,15 @@ LESS_NO_STATE = 2
 LESS_POLICY_LAMBDA = 4
 LESS_POLICY_TOVA = 8
 LESS_WITH_PARALLEL_FORM = 16
+LESS_OUT_F16 = 32
 
 EXPORTED = [
     "less_arena_bytes", "less_create", "less_prefill", "less_decode_step", "less_position",
     "less_state_record_bytes", "less_export_state", "less_import_state",
     "less_read_feature_maps", "less_poll_status", "less_launch_count", "less_strerror",
     "less_destroy", "less_decode_step_host", "less_profile", "less_profile_read",
-    "less_prompt_scores_noalloc", "less_masked_attention",
+    "less_prompt_scores_noalloc", "less_masked_attention", "less_kernel_variant",
+    "less_last_status_where", "less_selftest_wait_timeout",
 ]
 LESS_NOALLOC_MAX_ROWS = 65536
 LESS_ERR_NOALLOC_TOO_LARGE = -12
@@ -106,6 +108,12 @@ def lib() -> C.CDLL:
     L.less_strerror.argtypes = [C.c_int]
     L.less_destroy.restype = C.c_int
     L.less_destroy.argtypes = [vp]
+    L.less_kernel_variant.restype = C.c_char_p
+    L.less_kernel_variant.argtypes = [vp, C.c_int]
+    L.less_last_status_where.restype = C.c_int
+    L.less_last_status_where.argtypes = [vp]
+    L.less_selftest_wait_timeout.restype = C.c_int
+    L.less_selftest_wait_timeout.argtypes = [vp, C.c_uint32, vp]
     _lib = L
     return L
 
@@ -192,6 +200,18 @@ def less_destroy(ctx) -> int:
     return lib().less_destroy(ctx)
 
 
+def less_kernel_variant(ctx, kernel_id: int) -> str:
+    return lib().less_kernel_variant(ctx, int(kernel_id)).decode()
+
+
+def less_last_status_where(ctx) -> int:
+    return int(lib().less_last_status_where(ctx))
+
+
+def less_selftest_wait_timeout(ctx, polls: int, stream) -> int:
+    return lib().less_selftest_wait_timeout(ctx, int(polls), stream)
+
+
 # --------------------------------------------------------------------------- #
 # convenience holder: owns the torch buffers the context borrows
 # --------------------------------------------------------------------------- #
@@ -237,6 +257,7 @@ class LessContext:
         self.group = max(1, group)
         self.N = heavy + recent
         self.record_bytes = less_state_record_bytes(self.cfg)
+        self.out_dtype = torch.float16 if flags & LESS_OUT_F16 else torch.float32
 
     # -- hot path ---------------------------------------------------------- #
     def prefill(self, Q, K, V, layer_begin=0, attn_out=None, stream=None):
@@ -265,7 +286,8 @@ class LessContext:
     def decode_step(self, q, k, v, out=None, evicted_pos=None, stream=None):
         assert q.dtype == k.dtype == v.dtype == torch.float16
         if out is None:
-            out = torch.empty(q.shape, dtype=torch.float32, device=q.device)
+            out = torch.empty(q.shape, dtype=self.out_dtype, device=q.device)
+        assert out.dtype == self.out_dtype
         _check(less_decode_step(self.ctx, _ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(evicted_pos),
                                 _stream_ptr(stream)), "less_decode_step")
         return out
@@ -348,6 +370,16 @@ class LessContext:
 
     def poll_status(self, stream=None) -> int:
         return less_poll_status(self.ctx, _stream_ptr(stream))
+
+    def kernel_variant(self, kernel: str) -> str:
+        """Name of the kernel variant last launched under a KERNEL_NAMES id."""
+        return less_kernel_variant(self.ctx, KERNEL_NAMES.index(kernel))
+
+    def status_where(self) -> int:
+        return less_last_status_where(self.ctx)
+
+    def selftest_wait_timeout(self, polls: int, stream=None) -> int:
+        return less_selftest_wait_timeout(self.ctx, polls, _stream_ptr(stream))
 
     def close(self):
         if getattr(self, "ctx", None) is not None:

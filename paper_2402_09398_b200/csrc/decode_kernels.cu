@@ -2,6 +2,9 @@
 //   feature_map_kernel  phi(q_t), psi(k_t)                         (Eq. 1, Eq. 2)
 //   decode_kernel       scores over the live slots, Eq. 3, H2O score update,
 //                       argmin eviction, Eq. 4 / Eq. 5, in-place slot overwrite
+//   decode_group_*      the same step for G query heads per KV head
+#include <stdio.h>
+
 #include "feature_gemv.cuh"
 #include "feature_mlp.cuh"
 
@@ -63,6 +66,8 @@ int launch_feature_maps(less_ctx* c, const void* q, const void* k, cudaStream_t 
   p.out[1] = c->a.psi_k;
   p.B = d.B; p.L = d.L; p.Hd = d.Hd; p.Rp = d.Rp;
   p.Hh[0] = d.Hd * d.G; p.Hh[1] = d.Hd;
+  p.feat_flag = nullptr; p.flag_stride = d.L * d.Hd * d.G;
+  c->flags_this_step = false;
   const int ndg = FM_THREADS / (d.Rp / 8);
   const size_t smem = (size_t)(FM_BR * kHeadDim + FM_BR * d.Rp + ndg * FM_BR * d.Rp) * 4;
   dim3 grid(d.L * d.Hd, (d.flags & LESS_NO_STATE) ? 1 : 2, (d.B + FM_BR - 1) / FM_BR);
@@ -70,7 +75,7 @@ int launch_feature_maps(less_ctx* c, const void* q, const void* k, cudaStream_t 
   if ((c->feature_path == 2 || d.G > 1) && feature_tc_supported(d)) return launch_feature_tc(c, p, s);
   if (d.G > 1) return LESS_ERR_INVALID_CONFIG;    // the CUDA-core kernels know one query head per KV head
   if (c->feature_path >= 1 && feature_gemv_supported(d)) return launch_feature_gemv(c, p, s);
-  LaunchScope scope(c, LESS_KERNEL_FEATURE_MAP, s);
+  LaunchScope scope(c, LESS_KERNEL_FEATURE_MAP, s, d.R == 8 ? "feature_map_kernel<8>" : "feature_map_kernel<16>");
   if (d.R == 8) {
     cudaFuncSetAttribute(feature_map_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     feature_map_kernel<8><<<grid, FM_THREADS, smem, s>>>(p);
@@ -89,12 +94,17 @@ constexpr int DEC_RG = DEC_THREADS / 16;   // row groups: 16 lanes x 16 B cover 
 
 struct DecParams {
   const __half* q; const __half* k; const __half* v;   // [I, D]
-  float* out;                                           // [I, D]
+  void* out;                                            // [I * G, D] fp32, or fp16 with LESS_OUT_F16
   int32_t* evicted_pos;                                 // [I] or null
   Arena a;
   int N, Np, heavy, recent;
   int t;             // position of this step's token (direct calls)
   uint32_t flags;
+  int B, LH;         // batch, layers x KV heads
+  const uint32_t* feat_flag;   // per-head counters of the feature-map kernel, or null: wait for its whole grid
+  int flag_stride;             // psi counters start here (= layers x query heads)
+  uint32_t flag_target[2];     // counter values that mean "this step's phi / psi of the head are written"
+  int head_major;              // CTAs numbered (layer-head, batch row) instead of by instance
 };
 
 __device__ __forceinline__ float block_max(float v, float* red) {
@@ -139,6 +149,216 @@ __device__ __forceinline__ void step_done(int32_t* tpos, int t) {
   }
 }
 
+// Where the feature maps of this step come from.  The feature-map kernel of the same step may still
+// be running (programmatic dependent launch): either the whole grid is awaited (griddepcontrol.wait),
+// or, when the feature kernel publishes a counter per (layer, head) and map, only this instance's
+// own phi(q_t) and psi(k_t) are: thread g < G polls the counter of query head g, thread G that of
+// psi, each with a bounded number of polls; a wait that runs out is recorded in the status word
+// and the step goes on (its result is then flagged, never hung).
+constexpr uint32_t kFlagPolls = 1u << 22;          // x 64 ns of back-off: a quarter of a second at most
+template <int G>
+__device__ __forceinline__ void wait_feature_maps(const DecParams& p, int lh) {
+  if (p.feat_flag == nullptr) {
+    pdl_wait_primary();
+    return;
+  }
+  const int tid = threadIdx.x;
+  if (tid <= G) {
+    const uint32_t* f = tid < G ? p.feat_flag + (size_t)lh * G + tid : p.feat_flag + p.flag_stride + lh;
+    const uint32_t want = tid < G ? p.flag_target[0] : p.flag_target[1];
+    uint32_t i = 0;
+    for (;;) {
+      uint32_t v;
+      asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(f) : "memory");
+      if ((int32_t)(v - want) >= 0) break;
+      if (++i >= kFlagPolls) {
+        set_status(p.a.status, kStatusTimeout, 3);
+        break;
+      }
+      __nanosleep(64);
+    }
+  }
+  __syncthreads();
+}
+
+__device__ __forceinline__ void store_out(const DecParams& p, size_t idx, float x) {
+  if (p.flags & LESS_OUT_F16) reinterpret_cast<__half*>(p.out)[idx] = __float2half_rn(x);
+  else reinterpret_cast<float*>(p.out)[idx] = x;
+}
+
+// The instance a CTA works on.  Behind a feature kernel that publishes per-head counters the CTAs
+// are numbered head-major (all batch rows of a head are neighbours), so that the first CTAs need
+// the first heads' feature maps; otherwise CTA = instance.
+__device__ __forceinline__ size_t decode_instance(const DecParams& p) {
+  if (!p.head_major) return blockIdx.x;
+  const int lh = blockIdx.x / p.B, b = blockIdx.x - lh * p.B;
+  return (size_t)b * p.LH + lh;
+}
+
+// The second half of a step, common to all decode kernels (one 128-thread CTA per KV head, thread
+// d owns column d of H): H2O score update with the probabilities of the G query heads, the choice
+// of the entry that leaves (policy), Eq. 4 / Eq. 5 for it, and the new pair's in-place write.
+//   s_sc  [G][Ns]  e^{s - m_g} of every live entry and, at index n, of the new pair
+//   inv   [G]      1 / normaliser of each head
+//   hcol  [R]      column d of H as read for Eq. 3
+template <int R, int G, bool kCaptured>
+__device__ __forceinline__ void decode_tail(const DecParams& p, size_t inst, int n, int t_now, const float* s_sc, int Ns,
+                                            const float (&inv)[G], const float (&hcol)[R], const uint4& knew,
+                                            const uint4& vnew, unsigned long long* s_key, int* s_vic) {
+  const int tid = threadIdx.x, d = tid, l16 = tid & 15, rg = tid >> 4;
+  const int N = p.N;
+  const bool use_state = !(p.flags & LESS_NO_STATE);
+  float* Hb = p.a.H + inst * (size_t)R * kHeadDim;
+  float* zb = p.a.z + inst * R;
+  const __half* Vb = p.a.vslots + inst * (size_t)N * kHeadDim;
+  int32_t* posb = p.a.pos + inst * (size_t)p.Np;
+  float* accb = p.a.acc + inst * (size_t)p.Np;
+  const bool full = (n == N);
+  const bool lambda_policy = (p.flags & LESS_POLICY_LAMBDA) != 0;
+  const bool tova_policy = G == 1 && (p.flags & LESS_POLICY_TOVA) != 0;
+  unsigned long long best = ~0ull;
+  for (int i = tid; i < n; i += DEC_THREADS) {
+    float ps_sum = 0.f;
+#pragma unroll
+    for (int g = 0; g < G; ++g) ps_sum = G == 1 ? s_sc[i] * inv[0] : fmaf(s_sc[g * Ns + i], inv[g], ps_sum);
+    // TOVA scores an entry by this query's probability alone; H2O accumulates
+    const float a = tova_policy ? ps_sum : accb[i] + ps_sum;
+    accb[i] = a;
+    if (full) {
+      const int ps = posb[i];
+      if (tova_policy) {                               // TOVA: every entry competes, nothing is protected
+        const unsigned long long key = ((unsigned long long)__float_as_uint(a) << 32) | (unsigned int)ps;
+        best = key < best ? key : best;
+      } else if (lambda_policy) {                      // Lambda-masking: the oldest position past the first tokens
+        if (ps >= p.heavy) best = (unsigned long long)(unsigned int)ps < best ? (unsigned int)ps : best;
+      } else if (ps <= t_now - p.recent) {             // H2O: lowest (accumulated score, position) outside the window
+        const unsigned long long key = ((unsigned long long)__float_as_uint(a) << 32) | (unsigned int)ps;
+        best = key < best ? key : best;
+      }
+    }
+  }
+  float p_new = 0.f;
+#pragma unroll
+  for (int g = 0; g < G; ++g) p_new = G == 1 ? s_sc[n] * inv[0] : fmaf(s_sc[g * Ns + n], inv[g], p_new);
+  int slot = n;                                        // next free slot
+  if (full) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const unsigned long long other = __shfl_xor_sync(0xffffffffu, best, o);
+      best = other < best ? other : best;
+    }
+    if ((tid & 31) == 0) s_key[tid >> 5] = best;
+    if (tid == 0) *s_vic = -1;
+    __syncthreads();
+    best = s_key[0];
+#pragma unroll
+    for (int w = 1; w < DEC_THREADS / 32; ++w) best = s_key[w] < best ? s_key[w] : best;
+    if (tova_policy) {
+      // the new pair competes too; if its own probability is the lowest it never enters the
+      // cache: it is absorbed into H, z at once and every slot stays as it is
+      const unsigned long long key_new = ((unsigned long long)__float_as_uint(p_new) << 32) | (unsigned int)t_now;
+      if (key_new < best) {                            // uniform over the CTA
+        if (tid == 0 && p.evicted_pos) p.evicted_pos[inst] = t_now;
+        if (use_state) {
+          const float vv = __half2float(p.v[inst * kHeadDim + d]);
+          const float* psn = p.a.psi_k + inst * R;
+#pragma unroll
+          for (int r = 0; r < R; ++r) Hb[r * kHeadDim + d] = fmaf(__ldcg(psn + r), vv, hcol[r]);
+          if (tid < R) zb[tid] += __ldcg(psn + tid);
+        }
+        step_done<kCaptured>(p.a.tpos, p.t);
+        return;
+      }
+    }
+    const int vpos = (int)(unsigned int)(best & 0xffffffffull);
+    for (int i = tid; i < n; i += DEC_THREADS)
+      if (posb[i] == vpos && best != ~0ull) *s_vic = i;   // positions are unique
+    __syncthreads();
+    slot = *s_vic;
+    if (slot < 0) {                                    // cannot happen with recent >= 1; refuse
+      if (tid == 0) {
+        set_status(p.a.status, kStatusBounds, 2);
+        if (p.evicted_pos) p.evicted_pos[inst] = -1;
+      }
+      step_done<kCaptured>(p.a.tpos, p.t);
+      return;
+    }
+    if (tid == 0 && p.evicted_pos) p.evicted_pos[inst] = vpos;
+    // ---- Eq. 4 / Eq. 5: absorb the victim (psi acts on the key: the state is the KV head's) ----
+    if (use_state) {
+      const float vv = __half2float(Vb[(size_t)slot * kHeadDim + d]);
+      const float* psv = p.a.psic + (inst * (size_t)N + slot) * R;
+#pragma unroll
+      for (int r = 0; r < R; ++r) Hb[r * kHeadDim + d] = fmaf(psv[r], vv, hcol[r]);
+      if (tid < R) zb[tid] += psv[tid];
+    }
+    __syncthreads();                                   // victim row fully read before overwrite
+  } else {
+    if (tid == 0) {
+      p.a.count[inst] = n + 1;
+      if (p.evicted_pos) p.evicted_pos[inst] = -1;
+    }
+  }
+  // ---- the new pair takes the slot in place ----
+  __half* Kw = p.a.kslots + (inst * (size_t)N + slot) * kHeadDim;
+  __half* Vw = p.a.vslots + (inst * (size_t)N + slot) * kHeadDim;
+  if (rg == 0) *reinterpret_cast<uint4*>(Kw + l16 * 8) = knew;
+  if (rg == 1) *reinterpret_cast<uint4*>(Vw + l16 * 8) = vnew;
+  if (tid == 32) { posb[slot] = t_now; accb[slot] = p_new; }
+  if (tid >= 64 && tid < 64 + R)
+    p.a.psic[(inst * (size_t)N + slot) * R + (tid - 64)] = use_state ? __ldcg(p.a.psi_k + inst * R + (tid - 64)) : 0.f;
+  step_done<kCaptured>(p.a.tpos, p.t);
+}
+
+// Eq. 3 of each of the G query heads over the KV head's shared H, z, from the heads' partial
+// numerators in shared memory (s_red [G][NRED][128]), then the common second half of the step.
+template <int R, int G, bool kCaptured, int NRED>
+__device__ __forceinline__ void group_eq3_and_tail(const DecParams& p, size_t inst, int n, int t_now, const float* s_sc,
+                                                   int Ns, const float* s_red, const float (&mg)[G], const float (&lg)[G],
+                                                   const uint4& knew, const uint4& vnew, float* s_inv,
+                                                   unsigned long long* s_key, int* s_vic) {
+  const int tid = threadIdx.x, d = tid;
+  const bool use_state = !(p.flags & LESS_NO_STATE);
+  const float* Hb = p.a.H + inst * (size_t)R * kHeadDim;
+  const float* zb = p.a.z + inst * R;
+  float hcol[R], zr[R];
+  if (use_state) {
+    wait_feature_maps<G>(p, p.head_major ? blockIdx.x / p.B : (int)(inst % p.LH));
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+      hcol[r] = Hb[r * kHeadDim + d];
+      zr[r] = zb[r];
+    }
+  }
+#pragma unroll
+  for (int g = 0; g < G; ++g) {
+    float num = 0.f;
+#pragma unroll
+    for (int j = 0; j < NRED; ++j) num += s_red[(g * NRED + j) * kHeadDim + d];
+    float den = lg[g];
+    if (use_state) {
+      const float em = __expf(-mg[g]);
+      const float* ph = p.a.phi_q + (inst * G + g) * R;
+      float lr = 0.f, lz = 0.f;
+#pragma unroll
+      for (int r = 0; r < R; ++r) {
+        const float f = __ldcg(ph + r);
+        lr = fmaf(f, hcol[r], lr);
+        lz = fmaf(f, zr[r], lz);
+      }
+      num = fmaf(em, lr, num);
+      den = fmaf(em, lz, den);
+    }
+    store_out(p, (inst * G + g) * kHeadDim + d, num / den);
+    if (tid == 0) s_inv[g] = 1.0f / ((p.flags & LESS_SCORE_NORM_SPARSE) ? lg[g] : den);
+  }
+  __syncthreads();
+  float inv[G];
+#pragma unroll
+  for (int g = 0; g < G; ++g) inv[g] = s_inv[g];
+  decode_tail<R, G, kCaptured>(p, inst, n, t_now, s_sc, Ns, inv, hcol, knew, vnew, s_key, s_vic);
+}
+
 template <int R, bool kCaptured>
 __global__ void __launch_bounds__(DEC_THREADS) decode_kernel(DecParams p) {
   extern __shared__ float dsm[];
@@ -149,7 +369,7 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_kernel(DecParams p) {
   __shared__ int s_vic;
 
   const int tid = threadIdx.x;
-  const size_t inst = blockIdx.x;
+  const size_t inst = decode_instance(p);
   const int l16 = tid & 15, rg = tid >> 4;
   const int N = p.N;
   const int t_now = kCaptured ? __ldcg(p.a.tpos) : p.t;   // tokens seen = this token's position
@@ -239,276 +459,16 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_kernel(DecParams p) {
 #pragma unroll
   for (int g = 0; g < DEC_RG; ++g) num += s_red[g * kHeadDim + d];
   float den = lsum;
-  float phi[R];
-  float* Hb = p.a.H + inst * (size_t)R * kHeadDim;
-  float* zb = p.a.z + inst * R;
+  const float* Hb = p.a.H + inst * (size_t)R * kHeadDim;
+  const float* zb = p.a.z + inst * R;
   float hcol[R];
   if (use_state) {
-    pdl_wait_primary();                            // phi(q_t), psi(k_t) of this step are complete from here on
+    wait_feature_maps<1>(p, p.head_major ? blockIdx.x / p.B : (int)(inst % p.LH));   // phi(q_t), psi(k_t) of this step are complete from here on
     const float em = __expf(-m);
     float lr = 0.f, lz = 0.f;
 #pragma unroll
     for (int r = 0; r < R; ++r) {
-      phi[r] = p.a.phi_q[inst * R + r];
-      hcol[r] = Hb[r * kHeadDim + d];
-      lr = fmaf(phi[r], hcol[r], lr);
-      lz = fmaf(phi[r], zb[r], lz);
-    }
-    num = fmaf(em, lr, num);
-    den = fmaf(em, lz, den);
-  }
-  p.out[inst * kHeadDim + d] = num / den;
-
-  // ---- H2O: acc_i += p_i; candidates pos <= t - recent; argmin (acc, pos) ----
-  const float inv = 1.0f / ((p.flags & LESS_SCORE_NORM_SPARSE) ? lsum : den);
-  int32_t* posb = p.a.pos + inst * (size_t)p.Np;
-  float* accb = p.a.acc + inst * (size_t)p.Np;
-  const bool full = (n == N);
-  const bool lambda_policy = (p.flags & LESS_POLICY_LAMBDA) != 0;
-  const bool tova_policy = (p.flags & LESS_POLICY_TOVA) != 0;
-  unsigned long long best = ~0ull;
-  for (int i = tid; i < n; i += DEC_THREADS) {
-    // TOVA scores an entry by this query's probability alone; H2O accumulates
-    const float a = tova_policy ? s_sc[i] * inv : accb[i] + s_sc[i] * inv;
-    accb[i] = a;
-    if (full) {
-      const int ps = posb[i];
-      if (tova_policy) {                             // TOVA: every entry competes, nothing is protected
-        const unsigned long long key =
-            ((unsigned long long)__float_as_uint(a) << 32) | (unsigned int)ps;
-        best = key < best ? key : best;
-      } else if (lambda_policy) {                           // Lambda-masking: the oldest position past the first tokens
-        if (ps >= p.heavy) best = (unsigned long long)(unsigned int)ps < best ? (unsigned int)ps : best;
-      } else if (ps <= t_now - p.recent) {             // H2O: lowest (accumulated score, position) outside the window
-        const unsigned long long key =
-            ((unsigned long long)__float_as_uint(a) << 32) | (unsigned int)ps;
-        best = key < best ? key : best;
-      }
-    }
-  }
-  const float p_new = s_sc[n] * inv;
-  int slot = n;                                    // next free slot
-  if (full) {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      const unsigned long long other = __shfl_xor_sync(0xffffffffu, best, o);
-      best = other < best ? other : best;
-    }
-    if ((tid & 31) == 0) s_key[tid >> 5] = best;
-    if (tid == 0) s_vic = -1;
-    __syncthreads();
-    best = s_key[0];
-#pragma unroll
-    for (int w = 1; w < DEC_THREADS / 32; ++w) best = s_key[w] < best ? s_key[w] : best;
-    if (tova_policy) {
-      // the new pair competes too; if its own probability is the lowest it never enters the
-      // cache: it is absorbed into H, z at once and every slot stays as it is
-      const unsigned long long key_new =
-          ((unsigned long long)__float_as_uint(p_new) << 32) | (unsigned int)t_now;
-      if (key_new < best) {                          // uniform over the CTA
-        if (tid == 0 && p.evicted_pos) p.evicted_pos[inst] = t_now;
-        if (use_state) {
-          const float vv = __half2float(p.v[inst * kHeadDim + d]);
-          const float* psn = p.a.psi_k + inst * R;
-#pragma unroll
-          for (int r = 0; r < R; ++r) Hb[r * kHeadDim + d] = fmaf(psn[r], vv, hcol[r]);
-          if (tid < R) zb[tid] += psn[tid];
-        }
-        step_done<kCaptured>(p.a.tpos, p.t);
-        return;
-      }
-    }
-    const int vpos = (int)(unsigned int)(best & 0xffffffffull);
-    for (int i = tid; i < n; i += DEC_THREADS)
-      if (posb[i] == vpos && best != ~0ull) s_vic = i;     // positions are unique
-    __syncthreads();
-    slot = s_vic;
-    if (slot < 0) {                                // cannot happen with recent >= 1; refuse
-      if (tid == 0) {
-        set_status(p.a.status, kStatusBounds, 2);
-        if (p.evicted_pos) p.evicted_pos[inst] = -1;
-      }
-      step_done<kCaptured>(p.a.tpos, p.t);
-      return;
-    }
-    if (tid == 0 && p.evicted_pos) p.evicted_pos[inst] = vpos;
-    // ---- Eq. 4 / Eq. 5: absorb the victim ----
-    if (use_state) {
-      const float vv = __half2float(Vb[(size_t)slot * kHeadDim + d]);
-      const float* psv = p.a.psic + (inst * (size_t)N + slot) * R;
-#pragma unroll
-      for (int r = 0; r < R; ++r) Hb[r * kHeadDim + d] = fmaf(psv[r], vv, hcol[r]);
-      if (tid < R) zb[tid] += psv[tid];
-    }
-    __syncthreads();                               // victim row fully read before overwrite
-  } else {
-    if (tid == 0) {
-      p.a.count[inst] = n + 1;
-      if (p.evicted_pos) p.evicted_pos[inst] = -1;
-    }
-  }
-  // ---- the new pair takes the slot in place ----
-  __half* Kw = p.a.kslots + (inst * (size_t)N + slot) * kHeadDim;
-  __half* Vw = p.a.vslots + (inst * (size_t)N + slot) * kHeadDim;
-  if (rg == 0) *reinterpret_cast<uint4*>(Kw + l16 * 8) = knew;
-  if (rg == 1) *reinterpret_cast<uint4*>(Vw + l16 * 8) = vnew;
-  if (tid == 32) { posb[slot] = t_now; accb[slot] = p_new; }
-  if (tid >= 64 && tid < 64 + R)
-    p.a.psic[(inst * (size_t)N + slot) * R + (tid - 64)] =
-        use_state ? p.a.psi_k[inst * R + (tid - 64)] : 0.f;
-  step_done<kCaptured>(p.a.tpos, p.t);
-}
-
-// --------------------------------------------------------------------------- //
-// Grouped query heads (Section 3.2, multi-query attention): G query heads share one KV head.
-// One CTA per KV head, 128 threads per query head: each 128-thread team runs Eq. 3 for its own
-// head (own phi, own normaliser) over the shared slots and the shared H, z, exactly as
-// decode_kernel does for a single head; the teams' reads of the same K / V rows meet in L1, so
-// the slots cross HBM once.  Then all threads add the G heads' probabilities into the entries'
-// H2O scores and pick the one entry that leaves for all heads.
-// --------------------------------------------------------------------------- //
-__device__ __forceinline__ void team_sync(int team) {
-  asm volatile("bar.sync %0, %1;" ::"r"(team + 1), "n"(DEC_THREADS) : "memory");
-}
-
-__device__ __forceinline__ float team_max(float v, float* red, int team) {
-  const int lane = threadIdx.x & 31, warp = (threadIdx.x >> 5) & 3;
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
-  if (lane == 0) red[warp] = v;
-  team_sync(team);
-  const float r = fmaxf(fmaxf(red[0], red[1]), fmaxf(red[2], red[3]));
-  team_sync(team);
-  return r;
-}
-
-__device__ __forceinline__ float team_sum(float v, float* red, int team) {
-  const int lane = threadIdx.x & 31, warp = (threadIdx.x >> 5) & 3;
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-  if (lane == 0) red[warp] = v;
-  team_sync(team);
-  const float r = ((red[0] + red[1]) + red[2]) + red[3];   // fixed order
-  team_sync(team);
-  return r;
-}
-
-template <int R, int G, bool kCaptured>
-__global__ void __launch_bounds__(DEC_THREADS * G) decode_group_kernel(DecParams p) {
-  extern __shared__ float dsm[];
-  const int Ns = p.Np + 4;
-  float* s_sc_all = dsm;                           // [G][Np + 4] scores, then e^{s - m_g}
-  float* s_red_all = s_sc_all + G * Ns;            // [G][DEC_RG][128] partial numerators
-  __shared__ float s_small[G][4];
-  __shared__ unsigned long long s_key[G * 4];
-  __shared__ int s_vic;
-  __shared__ float s_inv[G];
-
-  const int team = threadIdx.x / DEC_THREADS;      // query head of the group
-  const int tid = threadIdx.x % DEC_THREADS;       // thread within the team
-  const size_t inst = blockIdx.x;
-  const size_t qi = inst * G + team;               // query head among all query heads
-  const int l16 = tid & 15, rg = tid >> 4;
-  const int N = p.N;
-  const int t_now = kCaptured ? __ldcg(p.a.tpos) : p.t;
-  int n = p.a.count[inst];
-  if (n < 0 || n > N) {
-    if (threadIdx.x == 0) set_status(p.a.status, kStatusBounds, 1);
-    step_done<kCaptured>(p.a.tpos, p.t);
-    return;
-  }
-  const bool use_state = !(p.flags & LESS_NO_STATE);
-  const float scale = 0.08838834764831845f;        // 1 / sqrt(128)
-  float* s_sc = s_sc_all + team * Ns;
-  float* s_red = s_red_all + team * DEC_RG * kHeadDim;
-
-  const __half* Kb = p.a.kslots + inst * (size_t)N * kHeadDim;
-  const __half* Vb = p.a.vslots + inst * (size_t)N * kHeadDim;
-
-  float qf[8];
-  half8_to_float(*reinterpret_cast<const uint4*>(p.q + qi * kHeadDim + l16 * 8), qf);
-
-  // ---- this head's scores over the live slots and the new pair ----
-#pragma unroll 4
-  for (int r0 = 0; r0 < n; r0 += DEC_RG) {
-    const int r = r0 + rg;
-    float dot = 0.f;
-    if (r < n) {
-      float kf[8];
-      half8_to_float(*reinterpret_cast<const uint4*>(Kb + (size_t)r * kHeadDim + l16 * 8), kf);
-#pragma unroll
-      for (int c = 0; c < 8; ++c) dot = fmaf(qf[c], kf[c], dot);
-    }
-#pragma unroll
-    for (int o = 8; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
-    if (l16 == 0 && r < n) s_sc[r] = dot * scale;
-  }
-  const uint4 knew = *reinterpret_cast<const uint4*>(p.k + inst * kHeadDim + l16 * 8);
-  const uint4 vnew = *reinterpret_cast<const uint4*>(p.v + inst * kHeadDim + l16 * 8);
-  if (tid < 32) {
-    float kf[8];
-    half8_to_float(knew, kf);
-    float dot = 0.f;
-#pragma unroll
-    for (int c = 0; c < 8; ++c) dot = fmaf(qf[c], kf[c], dot);
-#pragma unroll
-    for (int o = 8; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
-    if (tid == 0) s_sc[n] = dot * scale;
-  }
-  team_sync(team);
-
-  float m = -INFINITY;
-  for (int i = tid; i <= n; i += DEC_THREADS) m = fmaxf(m, s_sc[i]);
-  m = team_max(m, s_small[team], team);
-  m = fmaxf(m, -80.f);
-  float lsum = 0.f;
-  for (int i = tid; i <= n; i += DEC_THREADS) {
-    const float e = __expf(s_sc[i] - m);
-    s_sc[i] = e;
-    lsum += e;
-  }
-  lsum = team_sum(lsum, s_small[team], team);
-
-  // ---- u = sum e_i v_i ----
-  float u[8];
-#pragma unroll
-  for (int c = 0; c < 8; ++c) u[c] = 0.f;
-#pragma unroll 4
-  for (int r = rg; r < n; r += DEC_RG) {
-    float vf[8];
-    half8_to_float(*reinterpret_cast<const uint4*>(Vb + (size_t)r * kHeadDim + l16 * 8), vf);
-    const float e = s_sc[r];
-#pragma unroll
-    for (int c = 0; c < 8; ++c) u[c] = fmaf(e, vf[c], u[c]);
-  }
-  if (rg == 0) {
-    float vf[8];
-    half8_to_float(vnew, vf);
-    const float e = s_sc[n];
-#pragma unroll
-    for (int c = 0; c < 8; ++c) u[c] = fmaf(e, vf[c], u[c]);
-  }
-#pragma unroll
-  for (int c = 0; c < 8; ++c) s_red[rg * kHeadDim + l16 * 8 + c] = u[c];
-  team_sync(team);
-
-  // ---- Eq. 3 of this head over the shared H, z ----
-  const int d = tid;
-  float num = 0.f;
-#pragma unroll
-  for (int j = 0; j < DEC_RG; ++j) num += s_red[j * kHeadDim + d];
-  float den = lsum;
-  float* Hb = p.a.H + inst * (size_t)R * kHeadDim;
-  float* zb = p.a.z + inst * R;
-  float hcol[R];
-  if (use_state) {
-    pdl_wait_primary();
-    const float em = __expf(-m);
-    const float* ph = p.a.phi_q + qi * R;
-    float lr = 0.f, lz = 0.f;
-#pragma unroll
-    for (int r = 0; r < R; ++r) {
-      const float f = ph[r];
+      const float f = __ldcg(p.a.phi_q + inst * R + r);
       hcol[r] = Hb[r * kHeadDim + d];
       lr = fmaf(f, hcol[r], lr);
       lz = fmaf(f, zb[r], lz);
@@ -516,96 +476,19 @@ __global__ void __launch_bounds__(DEC_THREADS * G) decode_group_kernel(DecParams
     num = fmaf(em, lr, num);
     den = fmaf(em, lz, den);
   }
-  p.out[qi * kHeadDim + d] = num / den;
-  if (tid == 0) s_inv[team] = 1.0f / ((p.flags & LESS_SCORE_NORM_SPARSE) ? lsum : den);
-  __syncthreads();                                 // every head's e_i and 1 / normaliser are in shared memory; H, z are read
-
-  // ---- H2O over the group: acc_i += sum_g p_{g,i}; one victim for all heads ----
-  float inv[G];
-#pragma unroll
-  for (int g = 0; g < G; ++g) inv[g] = s_inv[g];
-  int32_t* posb = p.a.pos + inst * (size_t)p.Np;
-  float* accb = p.a.acc + inst * (size_t)p.Np;
-  const bool full = (n == N);
-  const bool lambda_policy = (p.flags & LESS_POLICY_LAMBDA) != 0;
-  unsigned long long best = ~0ull;
-  for (int i = threadIdx.x; i < n; i += DEC_THREADS * G) {
-    float ps_sum = 0.f;
-#pragma unroll
-    for (int g = 0; g < G; ++g) ps_sum = fmaf(s_sc_all[g * Ns + i], inv[g], ps_sum);
-    const float a = accb[i] + ps_sum;
-    accb[i] = a;
-    if (full) {
-      const int ps = posb[i];
-      if (lambda_policy) {
-        if (ps >= p.heavy) best = (unsigned long long)(unsigned int)ps < best ? (unsigned int)ps : best;
-      } else if (ps <= t_now - p.recent) {
-        const unsigned long long key =
-            ((unsigned long long)__float_as_uint(a) << 32) | (unsigned int)ps;
-        best = key < best ? key : best;
-      }
-    }
-  }
-  float p_new = 0.f;
-#pragma unroll
-  for (int g = 0; g < G; ++g) p_new = fmaf(s_sc_all[g * Ns + n], inv[g], p_new);
-  int slot = n;
-  if (full) {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      const unsigned long long other = __shfl_xor_sync(0xffffffffu, best, o);
-      best = other < best ? other : best;
-    }
-    if ((threadIdx.x & 31) == 0) s_key[threadIdx.x >> 5] = best;
-    if (threadIdx.x == 0) s_vic = -1;
-    __syncthreads();
-    best = s_key[0];
-#pragma unroll
-    for (int w = 1; w < G * 4; ++w) best = s_key[w] < best ? s_key[w] : best;
-    const int vpos = (int)(unsigned int)(best & 0xffffffffull);
-    for (int i = threadIdx.x; i < n; i += DEC_THREADS * G)
-      if (posb[i] == vpos && best != ~0ull) s_vic = i;
-    __syncthreads();
-    slot = s_vic;
-    if (slot < 0) {
-      if (threadIdx.x == 0) {
-        set_status(p.a.status, kStatusBounds, 2);
-        if (p.evicted_pos) p.evicted_pos[inst] = -1;
-      }
-      step_done<kCaptured>(p.a.tpos, p.t);
-      return;
-    }
-    if (threadIdx.x == 0 && p.evicted_pos) p.evicted_pos[inst] = vpos;
-    if (use_state && team == 0) {                  // Eq. 4 / Eq. 5: psi acts on the key, the state is the KV head's
-      const float vv = __half2float(Vb[(size_t)slot * kHeadDim + d]);
-      const float* psv = p.a.psic + (inst * (size_t)N + slot) * R;
-#pragma unroll
-      for (int r = 0; r < R; ++r) Hb[r * kHeadDim + d] = fmaf(psv[r], vv, hcol[r]);
-      if (tid < R) zb[tid] += psv[tid];
-    }
-    __syncthreads();                               // victim row fully read before overwrite
-  } else {
-    if (threadIdx.x == 0) {
-      p.a.count[inst] = n + 1;
-      if (p.evicted_pos) p.evicted_pos[inst] = -1;
-    }
-  }
-  if (team == 0) {                                 // the new pair takes the slot in place
-    __half* Kw = p.a.kslots + (inst * (size_t)N + slot) * kHeadDim;
-    __half* Vw = p.a.vslots + (inst * (size_t)N + slot) * kHeadDim;
-    if (rg == 0) *reinterpret_cast<uint4*>(Kw + l16 * 8) = knew;
-    if (rg == 1) *reinterpret_cast<uint4*>(Vw + l16 * 8) = vnew;
-    if (tid == 32) { posb[slot] = t_now; accb[slot] = p_new; }
-    if (tid >= 64 && tid < 64 + R)
-      p.a.psic[(inst * (size_t)N + slot) * R + (tid - 64)] =
-          use_state ? p.a.psi_k[inst * R + (tid - 64)] : 0.f;
-  }
-  step_done<kCaptured>(p.a.tpos, p.t);
+  store_out(p, inst * kHeadDim + d, num / den);
+  const float inv[1] = {1.0f / ((p.flags & LESS_SCORE_NORM_SPARSE) ? lsum : den)};
+  decode_tail<R, 1, kCaptured>(p, inst, n, t_now, s_sc, p.Np + 4, inv, hcol, knew, vnew, s_key, &s_vic);
 }
 
-// The same step for many KV heads per SM (batched serving): 128 threads per KV head, so that
-// several CTAs share an SM; every K / V row is loaded and converted once and meets the G
-// queries in registers.
+// --------------------------------------------------------------------------- //
+// Grouped query heads (Section 3.2, multi-query attention): G query heads share one KV head.
+// One 128-thread CTA per KV head; every query head has its own phi and its own Eq. 3 (own
+// normaliser) over the shared slots and the shared H, z; then the G heads' probabilities are
+// added into the entries' H2O scores and one entry leaves for all heads.
+// CUDA-core version: every K / V row is loaded and converted once and meets the G queries in
+// registers.
+// --------------------------------------------------------------------------- //
 template <int R, int G, bool kCaptured>
 __global__ void __launch_bounds__(DEC_THREADS) decode_group_rows_kernel(DecParams p) {
   extern __shared__ float dsm[];
@@ -618,7 +501,7 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_group_rows_kernel(DecParam
   __shared__ float s_inv[G];
 
   const int tid = threadIdx.x;
-  const size_t inst = blockIdx.x;
+  const size_t inst = decode_instance(p);
   const int l16 = tid & 15, rg = tid >> 4;
   const int N = p.N;
   const int t_now = kCaptured ? __ldcg(p.a.tpos) : p.t;
@@ -730,122 +613,7 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_group_rows_kernel(DecParam
     for (int c = 0; c < 8; ++c) s_red[(g * DEC_RG + rg) * kHeadDim + l16 * 8 + c] = u[g][c];
   __syncthreads();
 
-  // ---- Eq. 3 per head over the shared H, z ----
-  const int d = tid;
-  float* Hb = p.a.H + inst * (size_t)R * kHeadDim;
-  float* zb = p.a.z + inst * R;
-  float hcol[R], zr[R];
-  if (use_state) {
-    pdl_wait_primary();
-#pragma unroll
-    for (int r = 0; r < R; ++r) {
-      hcol[r] = Hb[r * kHeadDim + d];
-      zr[r] = zb[r];
-    }
-  }
-#pragma unroll
-  for (int g = 0; g < G; ++g) {
-    float num = 0.f;
-#pragma unroll
-    for (int j = 0; j < DEC_RG; ++j) num += s_red[(g * DEC_RG + j) * kHeadDim + d];
-    float den = lg[g];
-    if (use_state) {
-      const float em = __expf(-mg[g]);
-      const float* ph = p.a.phi_q + (inst * G + g) * R;
-      float lr = 0.f, lz = 0.f;
-#pragma unroll
-      for (int r = 0; r < R; ++r) {
-        const float f = ph[r];
-        lr = fmaf(f, hcol[r], lr);
-        lz = fmaf(f, zr[r], lz);
-      }
-      num = fmaf(em, lr, num);
-      den = fmaf(em, lz, den);
-    }
-    p.out[(inst * G + g) * kHeadDim + d] = num / den;
-    if (tid == 0) s_inv[g] = 1.0f / ((p.flags & LESS_SCORE_NORM_SPARSE) ? lg[g] : den);
-  }
-  __syncthreads();
-  float inv[G];
-#pragma unroll
-  for (int g = 0; g < G; ++g) inv[g] = s_inv[g];
-
-  // ---- H2O over the group: acc_i += sum_g p_{g,i}; one victim for all heads ----
-  int32_t* posb = p.a.pos + inst * (size_t)p.Np;
-  float* accb = p.a.acc + inst * (size_t)p.Np;
-  const bool full = (n == N);
-  const bool lambda_policy = (p.flags & LESS_POLICY_LAMBDA) != 0;
-  unsigned long long best = ~0ull;
-  for (int i = tid; i < n; i += DEC_THREADS) {
-    float ps_sum = 0.f;
-#pragma unroll
-    for (int g = 0; g < G; ++g) ps_sum = fmaf(s_sc[g * Ns + i], inv[g], ps_sum);
-    const float a = accb[i] + ps_sum;
-    accb[i] = a;
-    if (full) {
-      const int ps = posb[i];
-      if (lambda_policy) {
-        if (ps >= p.heavy) best = (unsigned long long)(unsigned int)ps < best ? (unsigned int)ps : best;
-      } else if (ps <= t_now - p.recent) {
-        const unsigned long long key =
-            ((unsigned long long)__float_as_uint(a) << 32) | (unsigned int)ps;
-        best = key < best ? key : best;
-      }
-    }
-  }
-  float p_new = 0.f;
-#pragma unroll
-  for (int g = 0; g < G; ++g) p_new = fmaf(s_sc[g * Ns + n], inv[g], p_new);
-  int slot = n;
-  if (full) {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      const unsigned long long other = __shfl_xor_sync(0xffffffffu, best, o);
-      best = other < best ? other : best;
-    }
-    if ((tid & 31) == 0) s_key[tid >> 5] = best;
-    if (tid == 0) s_vic = -1;
-    __syncthreads();
-    best = s_key[0];
-#pragma unroll
-    for (int w = 1; w < DEC_THREADS / 32; ++w) best = s_key[w] < best ? s_key[w] : best;
-    const int vpos = (int)(unsigned int)(best & 0xffffffffull);
-    for (int i = tid; i < n; i += DEC_THREADS)
-      if (posb[i] == vpos && best != ~0ull) s_vic = i;
-    __syncthreads();
-    slot = s_vic;
-    if (slot < 0) {
-      if (tid == 0) {
-        set_status(p.a.status, kStatusBounds, 2);
-        if (p.evicted_pos) p.evicted_pos[inst] = -1;
-      }
-      step_done<kCaptured>(p.a.tpos, p.t);
-      return;
-    }
-    if (tid == 0 && p.evicted_pos) p.evicted_pos[inst] = vpos;
-    if (use_state) {                               // Eq. 4 / Eq. 5: psi acts on the key, the state is the KV head's
-      const float vv = __half2float(Vb[(size_t)slot * kHeadDim + d]);
-      const float* psv = p.a.psic + (inst * (size_t)N + slot) * R;
-#pragma unroll
-      for (int r = 0; r < R; ++r) Hb[r * kHeadDim + d] = fmaf(psv[r], vv, hcol[r]);
-      if (tid < R) zb[tid] += psv[tid];
-    }
-    __syncthreads();
-  } else {
-    if (tid == 0) {
-      p.a.count[inst] = n + 1;
-      if (p.evicted_pos) p.evicted_pos[inst] = -1;
-    }
-  }
-  __half* Kw = p.a.kslots + (inst * (size_t)N + slot) * kHeadDim;
-  __half* Vw = p.a.vslots + (inst * (size_t)N + slot) * kHeadDim;
-  if (rg == 0) *reinterpret_cast<uint4*>(Kw + l16 * 8) = knew;
-  if (rg == 1) *reinterpret_cast<uint4*>(Vw + l16 * 8) = vnew;
-  if (tid == 32) { posb[slot] = t_now; accb[slot] = p_new; }
-  if (tid >= 64 && tid < 64 + R)
-    p.a.psic[(inst * (size_t)N + slot) * R + (tid - 64)] =
-        use_state ? p.a.psi_k[inst * R + (tid - 64)] : 0.f;
-  step_done<kCaptured>(p.a.tpos, p.t);
+  group_eq3_and_tail<R, G, kCaptured, DEC_RG>(p, inst, n, t_now, s_sc, Ns, s_red, mg, lg, knew, vnew, s_inv, s_key, &s_vic);
 }
 
 // The same step with the two contractions on the tensor cores.  With G query heads per KV head the
@@ -882,7 +650,7 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_group_mma_kernel(DecParams
   __shared__ float s_inv[G];
 
   const int tid = threadIdx.x;
-  const size_t inst = blockIdx.x;
+  const size_t inst = decode_instance(p);
   const int l16 = tid & 15, rg = tid >> 4;
   const int N = p.N;
   const int t_now = kCaptured ? __ldcg(p.a.tpos) : p.t;
@@ -1058,134 +826,16 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_group_mma_kernel(DecParams
   }
   __syncthreads();
 
-  // ---- Eq. 3 per head over the shared H, z ----
-  const int d = tid;
-  float* Hb = p.a.H + inst * (size_t)R * kHeadDim;
-  float* zb = p.a.z + inst * R;
-  float hcol[R], zr[R];
-  if (use_state) {
-    pdl_wait_primary();
-#pragma unroll
-    for (int r = 0; r < R; ++r) {
-      hcol[r] = Hb[r * kHeadDim + d];
-      zr[r] = zb[r];
-    }
-  }
-#pragma unroll
-  for (int g = 0; g < G; ++g) {
-    float num = 0.f;
-#pragma unroll
-    for (int j = 0; j < kMmaRed; ++j) num += s_red[(g * kMmaRed + j) * kHeadDim + d];
-    float den = lg[g];
-    if (use_state) {
-      const float em = __expf(-mg[g]);
-      const float* ph = p.a.phi_q + (inst * G + g) * R;
-      float lr = 0.f, lz = 0.f;
-#pragma unroll
-      for (int r = 0; r < R; ++r) {
-        const float f = ph[r];
-        lr = fmaf(f, hcol[r], lr);
-        lz = fmaf(f, zr[r], lz);
-      }
-      num = fmaf(em, lr, num);
-      den = fmaf(em, lz, den);
-    }
-    p.out[(inst * G + g) * kHeadDim + d] = num / den;
-    if (tid == 0) s_inv[g] = 1.0f / ((p.flags & LESS_SCORE_NORM_SPARSE) ? lg[g] : den);
-  }
-  __syncthreads();
-  float inv[G];
-#pragma unroll
-  for (int g = 0; g < G; ++g) inv[g] = s_inv[g];
-
-  // ---- H2O over the group: acc_i += sum_g p_{g,i}; one victim for all heads ----
-  int32_t* posb = p.a.pos + inst * (size_t)p.Np;
-  float* accb = p.a.acc + inst * (size_t)p.Np;
-  const bool full = (n == N);
-  const bool lambda_policy = (p.flags & LESS_POLICY_LAMBDA) != 0;
-  unsigned long long best = ~0ull;
-  for (int i = tid; i < n; i += DEC_THREADS) {
-    float ps_sum = 0.f;
-#pragma unroll
-    for (int g = 0; g < G; ++g) ps_sum = fmaf(s_sc[g * Ns + i], inv[g], ps_sum);
-    const float a = accb[i] + ps_sum;
-    accb[i] = a;
-    if (full) {
-      const int ps = posb[i];
-      if (lambda_policy) {
-        if (ps >= p.heavy) best = (unsigned long long)(unsigned int)ps < best ? (unsigned int)ps : best;
-      } else if (ps <= t_now - p.recent) {
-        const unsigned long long key =
-            ((unsigned long long)__float_as_uint(a) << 32) | (unsigned int)ps;
-        best = key < best ? key : best;
-      }
-    }
-  }
-  float p_new = 0.f;
-#pragma unroll
-  for (int g = 0; g < G; ++g) p_new = fmaf(s_sc[g * Ns + n], inv[g], p_new);
-  int slot = n;
-  if (full) {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      const unsigned long long other = __shfl_xor_sync(0xffffffffu, best, o);
-      best = other < best ? other : best;
-    }
-    if ((tid & 31) == 0) s_key[tid >> 5] = best;
-    if (tid == 0) s_vic = -1;
-    __syncthreads();
-    best = s_key[0];
-#pragma unroll
-    for (int w = 1; w < DEC_THREADS / 32; ++w) best = s_key[w] < best ? s_key[w] : best;
-    const int vpos = (int)(unsigned int)(best & 0xffffffffull);
-    for (int i = tid; i < n; i += DEC_THREADS)
-      if (posb[i] == vpos && best != ~0ull) s_vic = i;
-    __syncthreads();
-    slot = s_vic;
-    if (slot < 0) {
-      if (tid == 0) {
-        set_status(p.a.status, kStatusBounds, 2);
-        if (p.evicted_pos) p.evicted_pos[inst] = -1;
-      }
-      step_done<kCaptured>(p.a.tpos, p.t);
-      return;
-    }
-    if (tid == 0 && p.evicted_pos) p.evicted_pos[inst] = vpos;
-    if (use_state) {                               // Eq. 4 / Eq. 5: psi acts on the key, the state is the KV head's
-      const float vv = __half2float(Vb[(size_t)slot * kHeadDim + d]);
-      const float* psv = p.a.psic + (inst * (size_t)N + slot) * R;
-#pragma unroll
-      for (int r = 0; r < R; ++r) Hb[r * kHeadDim + d] = fmaf(psv[r], vv, hcol[r]);
-      if (tid < R) zb[tid] += psv[tid];
-    }
-    __syncthreads();
-  } else {
-    if (tid == 0) {
-      p.a.count[inst] = n + 1;
-      if (p.evicted_pos) p.evicted_pos[inst] = -1;
-    }
-  }
-  __half* Kw = p.a.kslots + (inst * (size_t)N + slot) * kHeadDim;
-  __half* Vw = p.a.vslots + (inst * (size_t)N + slot) * kHeadDim;
-  if (rg == 0) *reinterpret_cast<uint4*>(Kw + l16 * 8) = knew;
-  if (rg == 1) *reinterpret_cast<uint4*>(Vw + l16 * 8) = vnew;
-  if (tid == 32) { posb[slot] = t_now; accb[slot] = p_new; }
-  if (tid >= 64 && tid < 64 + R)
-    p.a.psic[(inst * (size_t)N + slot) * R + (tid - 64)] =
-        use_state ? p.a.psi_k[inst * R + (tid - 64)] : 0.f;
-  step_done<kCaptured>(p.a.tpos, p.t);
+  group_eq3_and_tail<R, G, kCaptured, kMmaRed>(p, inst, n, t_now, s_sc, Ns, s_red, mg, lg, knew, vnew, s_inv, s_key, &s_vic);
 }
-
 
 size_t decode_smem_bytes(const Dims& d) {
   return (size_t)d.G * (d.Np + 4 + DEC_RG * kHeadDim) * 4;
 }
 
-// which: 1 a 128-thread team per query head (few KV heads, latency matters), 2 one 128-thread CTA per KV
-// head on CUDA cores, 3 the same with the contractions on the tensor cores
+// which: 2 the CUDA-core version, 3 (default) the one with the contractions on the tensor cores
 template <int R, int G>
 static void* decode_group_entry(bool captured, int which) {
-  if (which == 1) return captured ? (void*)decode_group_kernel<R, G, true> : (void*)decode_group_kernel<R, G, false>;
   if (which == 2)
     return captured ? (void*)decode_group_rows_kernel<R, G, true> : (void*)decode_group_rows_kernel<R, G, false>;
   return captured ? (void*)decode_group_mma_kernel<R, G, true> : (void*)decode_group_mma_kernel<R, G, false>;
@@ -1196,24 +846,30 @@ int launch_decode(less_ctx* c, const void* q, const void* k, const void* v, void
   const Dims& d = c->d;
   DecParams p;
   p.q = (const __half*)q; p.k = (const __half*)k; p.v = (const __half*)v;
-  p.out = (float*)out;
+  p.out = out;
   p.evicted_pos = evicted_pos;
   p.a = c->a;
   p.N = d.N; p.Np = d.Np; p.heavy = d.heavy; p.recent = d.recent;
   p.t = (int)c->t;
+  p.B = d.B; p.LH = d.L * d.Hd;
   cudaStreamCaptureStatus capturing = cudaStreamCaptureStatusNone;
   cudaStreamIsCapturing(s, &capturing);
   const bool captured = capturing == cudaStreamCaptureStatusActive;   // then the position is read from, and advanced in, device memory
   p.flags = d.flags;
+  // this step's feature-map launch published per-head counters: wait for the instance's own only
+  p.feat_flag = c->flags_this_step ? c->a.feat_flag : nullptr;
+  p.flag_stride = d.L * d.Hd * d.G;
+  p.flag_target[0] = c->flag_target[0];
+  p.flag_target[1] = c->flag_target[1];
+  p.head_major = p.feat_flag != nullptr && d.B > 1;
   size_t smem = decode_smem_bytes(d);
-  LaunchScope scope(c, LESS_KERNEL_DECODE, s);
+  int which = c->group_path == 2 ? 2 : 3;
+  char name[64];
+  if (d.G == 1) snprintf(name, sizeof name, "decode_kernel<%d, %d>", d.R, (int)captured);
+  else snprintf(name, sizeof name, "decode_group_%s_kernel<%d, %d, %d>", which == 2 ? "rows" : "mma", d.R, d.G, (int)captured);
+  LaunchScope scope(c, LESS_KERNEL_DECODE, s, name);
   void* kern = d.R == 8 ? (captured ? (void*)decode_kernel<8, true> : (void*)decode_kernel<8, false>)
                         : (captured ? (void*)decode_kernel<16, true> : (void*)decode_kernel<16, false>);
-  // grouped query heads: with fewer KV heads than two per SM a CTA's latency is the step's, and the
-  // heads of a group run side by side (128 threads each); with more, throughput per SM counts
-  int which = c->group_path;
-  if (which == 0) which = 3;
-  const bool teams = d.G > 1 && which == 1;
   if (d.G > 1 && which == 3) smem = (size_t)d.G * (d.Np + 4 + kMmaRed * kHeadDim) * 4;
   if (d.G == 2) kern = d.R == 8 ? decode_group_entry<8, 2>(captured, which) : decode_group_entry<16, 2>(captured, which);
   if (d.G == 4) kern = d.R == 8 ? decode_group_entry<8, 4>(captured, which) : decode_group_entry<16, 4>(captured, which);
@@ -1223,7 +879,7 @@ int launch_decode(less_ctx* c, const void* q, const void* k, const void* v, void
     return fail_cuda("shared memory opt-in of decode_kernel");
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(d.I);
-  cfg.blockDim = dim3(teams ? DEC_THREADS * d.G : DEC_THREADS);
+  cfg.blockDim = dim3(DEC_THREADS);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = s;
   cudaLaunchAttribute attr[1];

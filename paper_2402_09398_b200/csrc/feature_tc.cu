@@ -21,7 +21,7 @@
 // whose accumulator lives in tensor memory across the chunks.  After the last
 // chunk: c2 * gelu(c1 * .), W3 (psi only) and the absolute value on CUDA cores.
 // The hidden activations never leave the SM (the paper's "absorbed activation",
-// Section 3.2, taken to the whole MLP).  No multicast; every wait is bounded.
+// Section 3.2, taken to the whole MLP).  Plain TMA loads only; every wait is bounded.
 #include "feature_gemv.cuh"
 #include "tc_common.cuh"
 
@@ -55,22 +55,36 @@ struct FtGeom {
   int npad;        // tokens per tile (GEMM1 N): 16, 32 or 64
   int ntile;       // token tiles per (layer-head, map)
   int items;       // work items
-  int items_phi;   // of which phi items (L * query heads * ntile)
+  int per_head;    // items per KV head: (G + 1) * ntile
+  int G;           // query heads per KV head
   int nstage;      // ring stages
   uint32_t tmem_cols;
 };
 
 
-// Work item -> (token tile, map, layer-head of that map).  The phi items (one per query head)
-// come first, then the psi items (one per KV head).
+// Work item -> (token tile, map, layer-head of that map).  The items of one KV head are
+// neighbours - its G phi items (one per query head), then its psi item, each times the token
+// tiles - so that a head's feature maps are complete early and together: the decode kernel of the
+// same step, which may already be running, needs exactly those.
 struct FtItem { int tile, which, lh; };
 __device__ __forceinline__ FtItem ft_item(int it, const FtGeom& gm) {
   FtItem r;
-  r.which = it >= gm.items_phi;
-  const int rest = r.which ? it - gm.items_phi : it;
-  r.tile = rest % gm.ntile;
-  r.lh = rest / gm.ntile;
+  const int kv = it / gm.per_head, rest = it - kv * gm.per_head;
+  const int sub = rest / gm.ntile;
+  r.tile = rest - sub * gm.ntile;
+  r.which = sub == gm.G;
+  r.lh = r.which ? kv : kv * gm.G + sub;
   return r;
+}
+
+// A warp that has written its share of an item's phi / psi publishes it: every lane's stores are
+// fenced, the warp converges, one lane bumps the head's counter.  The decode kernel compares the
+// counter with the number of writer warps the head has had once this step is complete.
+__device__ __forceinline__ void publish_rows(const FmParams& p, int which, int lh) {
+  if (p.feat_flag == nullptr) return;
+  __threadfence();
+  __syncwarp();
+  if ((threadIdx.x & 31) == 0) atomicAdd(p.feat_flag + (which ? p.flag_stride : 0) + lh, 1u);
 }
 
 // The producer thread of both kernels: per item the input rows, W2 and W3 into the item's aux
@@ -335,6 +349,7 @@ __global__ void __launch_bounds__(FL_THREADS) feature_tc_kernel(
 #pragma unroll
         for (int r4 = 0; r4 < R / 4; ++r4) dst[r4] = make_float4(out[r4 * 4], out[r4 * 4 + 1], out[r4 * 4 + 2], out[r4 * 4 + 3]);
       }
+      if (mine) publish_rows(p, which, lh);              // ceil(nb / 32) writer warps per item
       // this warp is done with the item's W3
       __syncwarp();
       if (lane == 0) mbar_arrive(&sh->aux_empty[a]);
@@ -554,6 +569,7 @@ __global__ void __launch_bounds__(FT_THREADS) feature_tc_small_kernel(
         }
       }
       if (et < V && t < nb) p.out[which][((size_t)(b0 + t) * p.L * p.Hh[which] + lh) * R + r] = fabsf(gv);
+      if (ew * 32 < V) publish_rows(p, which, lh);         // ceil(V / 32) writer warps per item
       // this warp is done with the item's W2 and W3
       mbar_arrive_warp(&sh->aux_empty[a]);
     }
@@ -582,17 +598,24 @@ static size_t ft_fixed_smem(const Dims& d, int npad) {
   return (size_t)4 * npad * 256 + (size_t)(d.R == 16 ? 4 : 2) * d.Rp * d.R * 2 + sizeof(FtShared) + 1024;
 }
 
-int launch_feature_tc(less_ctx* c, const FmParams& p, cudaStream_t s) {
+int launch_feature_tc(less_ctx* c, const FmParams& p_in, cudaStream_t s) {
   const Dims& d = c->d;
+  FmParams p = p_in;
   FtGeom gm;
   // token tiles of at most 64: larger tiles leave too little shared memory for the weight ring
   gm.npad = d.B <= 16 ? 16 : d.B <= 32 ? 32 : 64;
   gm.ntile = (d.B + gm.npad - 1) / gm.npad;
-  gm.items_phi = d.L * p.Hh[0] * gm.ntile;
-  gm.items = gm.items_phi + d.L * p.Hh[1] * gm.ntile;
+  gm.G = d.G;
+  gm.per_head = (d.G + 1) * gm.ntile;
+  gm.items = d.L * d.Hd * gm.per_head;
   const size_t fixed = ft_fixed_smem(d, gm.npad);
   int ns = (int)((FT_SMEM_LIMIT - fixed) / FT_STAGE_BYTES);
   gm.nstage = ns > FT_MAX_STAGES ? FT_MAX_STAGES : ns;
+  // With the overlap on, the ring gives up stages so that decode CTAs of the same step fit beside
+  // this kernel's CTA on every SM (at these batch sizes the kernel is bound by its epilogue, not
+  // by the weight stream: three stages feed it).
+  const int cap_l = c->feature_stages >= 2 ? c->feature_stages : (c->pdl ? 3 : FT_MAX_STAGES);
+  if (gm.nstage > cap_l) gm.nstage = cap_l;
   if (gm.nstage < 2) return LESS_ERR_INVALID_CONFIG;
   const uint32_t need = 2u * gm.npad + 16u;
   gm.tmem_cols = need <= 64 ? 64 : need <= 128 ? 128 : need <= 256 ? 256 : 512;
@@ -607,12 +630,30 @@ int launch_feature_tc(less_ctx* c, const FmParams& p, cudaStream_t s) {
   if (!make_tmap_f16_2d(&tw1a, p.w1[0], lhq * kHeadDim, d.Rp, (uint64_t)d.Rp * 2, kHeadDim) ||
       !make_tmap_f16_2d(&tw1b, p.w1[1], lhk * kHeadDim, d.Rp, (uint64_t)d.Rp * 2, kHeadDim))
     return fail_cuda("tensor map of W1");
-  int sms = 148;
-  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, c->device);
+  int sms = c->sms;
+  if (c->feature_ctas > 0 && c->feature_ctas < sms) sms = c->feature_ctas;
   const int grid = gm.items < sms ? gm.items : sms;
-  LaunchScope scope(c, LESS_KERNEL_FEATURE_MAP, s);
+  const int nt = d.B <= 1 ? 1 : d.B <= 2 ? 2 : d.B <= 4 ? 4 : 8;
+  // Per-head counters: direct calls only (a captured step would replay a stale target), and only
+  // where the decode kernel can be a programmatic dependent.  Every flagged launch adds the same
+  // number of writer warps to every head's counter, so the target is one running total.
+  cudaStreamCaptureStatus capturing = cudaStreamCaptureStatusNone;
+  cudaStreamIsCapturing(s, &capturing);
+  if (capturing == cudaStreamCaptureStatusNone && c->pdl) {
+    uint32_t writers = 0;
+    if (d.B <= 8) writers = (uint32_t)(nt * d.R + 31) / 32;
+    else
+      for (int t = 0; t < gm.ntile; ++t) writers += (uint32_t)(((d.B - t * gm.npad < gm.npad ? d.B - t * gm.npad : gm.npad) + 31) / 32);
+    p.feat_flag = c->a.feat_flag;
+    c->flag_target[0] += writers;
+    c->flag_target[1] += writers;
+    c->flags_this_step = true;
+  }
+  char name[64];
+  if (d.B <= 8) snprintf(name, sizeof name, "feature_tc_small_kernel<%d, %d>", d.R, nt);
+  else snprintf(name, sizeof name, "feature_tc_kernel<%d>", d.R);
+  LaunchScope scope(c, LESS_KERNEL_FEATURE_MAP, s, name);
   if (d.B <= 8) {
-    const int nt = d.B <= 1 ? 1 : d.B <= 2 ? 2 : d.B <= 4 ? 4 : 8;
     const size_t shared_struct = sizeof(FsShared<1>) + (size_t)(2 * FT_EPI_WARPS + 2) * (nt * d.R - 1) * 4;
     const size_t fx = 8192 + (size_t)FS_AUX * d.Rp * d.R * 2 + shared_struct + 256;
     const int nsm = (int)((FT_SMEM_LIMIT - fx) / FT_STAGE_BYTES);
@@ -620,7 +661,7 @@ int launch_feature_tc(less_ctx* c, const FmParams& p, cudaStream_t s) {
     // With the overlap on, one stage of the ring is given up so that the decode kernel's CTAs of
     // the same step fit beside this kernel's CTA on every SM (measured on the Llama-2-7B shape at
     // batch 1: 83.5 us per step with 6 stages and no room, 74.5 us with 5, 74.2 us with 4).
-    const int cap = c->feature_stages >= 2 ? c->feature_stages : (c->pdl && c->d.I <= 8 * c->sms ? 5 : FT_MAX_STAGES);
+    const int cap = c->feature_stages >= 2 ? c->feature_stages : (c->pdl ? 5 : FT_MAX_STAGES);
     if (gm.nstage > cap) gm.nstage = cap;
     if (gm.nstage < 2) return LESS_ERR_INVALID_CONFIG;
     const size_t sm = fx + (size_t)gm.nstage * FT_STAGE_BYTES;

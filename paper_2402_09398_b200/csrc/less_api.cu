@@ -25,7 +25,7 @@ bool valid_config(const less_config* c) {
   if (c->max_prefill_layers < 1 || c->max_prefill_layers > c->layers) return false;
   if ((int64_t)c->batch * c->heads * c->max_prefill_layers * (c->group > 1 ? c->group : 1) > 65535)
     return false;                                                                   // grid.y of the prompt kernels
-  if (c->flags & ~(uint32_t)(LESS_SCORE_NORM_SPARSE | LESS_NO_STATE | LESS_POLICY_LAMBDA | LESS_POLICY_TOVA | LESS_WITH_PARALLEL_FORM)) return false;
+  if (c->flags & ~(uint32_t)(LESS_SCORE_NORM_SPARSE | LESS_NO_STATE | LESS_POLICY_LAMBDA | LESS_POLICY_TOVA | LESS_WITH_PARALLEL_FORM | LESS_OUT_F16)) return false;
   if ((c->flags & LESS_POLICY_LAMBDA) && (c->flags & LESS_POLICY_TOVA)) return false;
   if (c->group < 0 || c->group > 8 || (c->group & (c->group - 1))) return false;          // 0, 1, 2, 4, 8
   if (c->group > 1 && (c->flags & LESS_POLICY_TOVA)) return false;                         // TOVA stays per head
@@ -83,6 +83,7 @@ size_t carve(const Dims& d, char* base, Arena* a) {
   t.psi_k = (float*)take(I * R * 4);
   t.status = (int32_t*)take(4 * 4);
   t.tpos = (int32_t*)take(4 * 4);
+  t.feat_flag = (uint32_t*)take((size_t)d.L * d.Hd * (G + 1) * 4);
   t.stage_q = (__half*)take(I * G * D * 2);
   t.stage_k = (__half*)take(I * D * 2);
   t.stage_v = (__half*)take(I * D * 2);
@@ -175,6 +176,12 @@ int less_create(const less_config* cfg, const less_weights* w, void* arena, size
   c->arena_bytes = need;
   c->t = 0;
   c->launches = 0;
+  c->flags_this_step = false;
+  c->flag_target[0] = c->flag_target[1] = 0;
+  c->status_where = 0;
+  memset(c->variant, 0, sizeof c->variant);
+  c->feature_ctas = 0;
+  if (const char* e = getenv("LESS_FEATURE_CTAS")) c->feature_ctas = atoi(e);
   c->profile = false;
   c->feature_path = 2;
   c->pdl = getenv("LESS_NO_OVERLAP") == nullptr;
@@ -188,12 +195,9 @@ int less_create(const less_config* cfg, const less_weights* w, void* arena, size
     else if (!strcmp(e, "plain")) c->feature_path = 0;
   }
   if (cudaGetDevice(&c->device) != cudaSuccess) { delete c; return LESS_ERR_CUDA; }
-  c->group_path = 0;
-  if (const char* e = getenv("LESS_GROUP_KERNEL")) {
-    if (!strcmp(e, "teams")) c->group_path = 1;
-    else if (!strcmp(e, "rows")) c->group_path = 2;
-    else if (!strcmp(e, "mma")) c->group_path = 3;
-  }
+  c->group_path = 3;
+  if (const char* e = getenv("LESS_GROUP_KERNEL"))
+    if (!strcmp(e, "rows")) c->group_path = 2;
   c->sms = 148;
   cudaDeviceGetAttribute(&c->sms, cudaDevAttrMultiProcessorCount, c->device);
   // H_0 = 0, z_0 = 0, no live slots, clean status
@@ -202,6 +206,7 @@ int less_create(const less_config* cfg, const less_weights* w, void* arena, size
   if (e == cudaSuccess) e = cudaMemset(c->a.count, 0, (size_t)d.I * 4);
   if (e == cudaSuccess) e = cudaMemset(c->a.status, 0, 16);
   if (e == cudaSuccess) e = cudaMemset(c->a.tpos, 0, 16);
+  if (e == cudaSuccess) e = cudaMemset(c->a.feat_flag, 0, (size_t)d.L * d.Hd * (d.G + 1) * 4);
   if (e == cudaSuccess) e = cudaMemset(c->a.phi_q, 0, (size_t)d.I * d.G * d.R * 4);
   if (e == cudaSuccess) e = cudaMemset(c->a.psi_k, 0, (size_t)d.I * d.R * 4);
   if (e == cudaSuccess) e = cudaDeviceSynchronize();
@@ -219,6 +224,11 @@ int less_destroy(less_ctx* ctx) {
 }
 
 int64_t less_position(const less_ctx* ctx) { return ctx ? ctx->t : -1; }
+const char* less_kernel_variant(const less_ctx* ctx, int kernel_id) {
+  if (!ctx || kernel_id < 0 || kernel_id >= LESS_KERNEL_COUNT) return "";
+  return ctx->variant[kernel_id];
+}
+int less_last_status_where(const less_ctx* ctx) { return ctx ? ctx->status_where : 0; }
 int64_t less_launch_count(const less_ctx* ctx) { return ctx ? ctx->launches : -1; }
 
 int less_prefill(less_ctx* c, int32_t layer_begin, int32_t layer_count, int32_t prompt_len,
@@ -299,15 +309,18 @@ int less_decode_step_host(less_ctx* c, const void* qh, const void* kh, const voi
                           void* stream) {
   if (!c || !qh || !kh || !vh || !outh) return LESS_ERR_NULL_POINTER;
   cudaStream_t s = (cudaStream_t)stream;
-  const size_t nin = (size_t)c->d.I * c->d.D * 2, nq = nin * c->d.G, nout = (size_t)c->d.I * c->d.G * c->d.D * 4;
-  // q and k feed the feature-map kernel's TMA loads and are staged in the arena.  v and the output
-  // are touched once per instance by the decode kernel: from pinned host memory it reads / writes
-  // them in place, which saves two copy launches per step.
+  const size_t osz = (c->d.flags & LESS_OUT_F16) ? 2 : 4;
+  const size_t nin = (size_t)c->d.I * c->d.D * 2, nq = nin * c->d.G, nout = (size_t)c->d.I * c->d.G * c->d.D * osz;
+  // q and k feed the feature-map kernel's TMA loads and are staged in the arena (the two staging
+  // buffers are neighbours, so a caller that keeps k directly behind q pays one copy, not two).
+  // v and the output are touched once per instance by the decode kernel: from pinned host memory
+  // it reads / writes them in place, which saves two more copies per step.
   const void* v_dev = device_alias(vh);
   void* out_dev = device_alias(outh);
   if (((uintptr_t)v_dev & 15) || ((uintptr_t)out_dev & 15)) { v_dev = nullptr; out_dev = nullptr; }
-  cudaError_t e = cudaMemcpyAsync(c->a.stage_q, qh, nq, cudaMemcpyHostToDevice, s);
-  if (e == cudaSuccess) e = cudaMemcpyAsync(c->a.stage_k, kh, nin, cudaMemcpyHostToDevice, s);
+  const bool one_block = (const char*)kh == (const char*)qh + nq && (char*)c->a.stage_k == (char*)c->a.stage_q + nq;
+  cudaError_t e = cudaMemcpyAsync(c->a.stage_q, qh, one_block ? nq + nin : nq, cudaMemcpyHostToDevice, s);
+  if (e == cudaSuccess && !one_block) e = cudaMemcpyAsync(c->a.stage_k, kh, nin, cudaMemcpyHostToDevice, s);
   if (e == cudaSuccess && !v_dev) e = cudaMemcpyAsync(c->a.stage_v, vh, nin, cudaMemcpyHostToDevice, s);
   if (e != cudaSuccess) return LESS_ERR_CUDA;
   int rc = less_decode_step(c, c->a.stage_q, c->a.stage_k, v_dev ? v_dev : c->a.stage_v,
@@ -434,6 +447,7 @@ int less_poll_status(less_ctx* c, void* stream) {
   if (e == cudaSuccess) e = cudaStreamSynchronize(s);
   if (e != cudaSuccess) return LESS_ERR_CUDA;
   c->t = tdev;                                   // replays of a captured step advance only the device's count
+  c->status_where = st[1];
   if (st[0] == kStatusTimeout) return LESS_ERR_DEVICE_TIMEOUT;
   if (st[0] == kStatusBounds) return LESS_ERR_DEVICE_BOUNDS;
   return LESS_OK;

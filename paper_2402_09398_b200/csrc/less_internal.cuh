@@ -5,6 +5,7 @@
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
+#include <stdio.h>
 
 #include <vector>
 
@@ -30,6 +31,8 @@ struct Arena {
   float* psi_k;      // [I][R]      psi(k_t) of the current step
   int32_t* status;   // [4]         device status word(s)
   int32_t* tpos;     // [4]         [0] tokens seen = position of the next decode token, [1] decode CTAs finished this step
+  uint32_t* feat_flag; // [L*Hd*G + L*Hd]  per (layer, head): writer warps of the feature-map kernel that have published
+                     //             phi(q_t) (first L*Hd*G entries, per query head) / psi(k_t) so far, over all steps
   __half* stage_q;   // [I*G][D]    staging of host inputs (less_decode_step_host)
   __half* stage_k;   // [I][D]
   __half* stage_v;   // [I][D]
@@ -83,7 +86,12 @@ struct less_ctx {
   int feature_stages;  // cap on the feature kernels' ring stages (LESS_FEATURE_STAGES), 0 = default
   int score_path;      // prompt scoring: 1 tensor cores, 0 CUDA cores (LESS_SCORE_KERNEL=plain)
   int feature_path;    // feature-map kernel: 2 tensor cores, 1 streaming GEMV, 0 plain (LESS_FEATURE_KERNEL)
-  int group_path;      // grouped decode kernel: 0 by instance count, 1 a team per query head, 2 one CTA per KV head on CUDA cores, 3 with warp-level mma (LESS_GROUP_KERNEL)
+  int group_path;      // grouped decode kernel: 2 on CUDA cores (LESS_GROUP_KERNEL=rows), else with warp-level mma
+  int feature_ctas;    // cap on the feature kernels' persistent CTAs (LESS_FEATURE_CTAS), 0 = one per multiprocessor
+  bool flags_this_step;     // the step's feature-map launch publishes per-head counters (set by its launcher)
+  uint32_t flag_target[2];  // counter value of a head once this step's phi / psi are written
+  int status_where;         // where-code of the last status word read by less_poll_status
+  char variant[LESS_KERNEL_COUNT][64];   // name of the kernel variant last launched under each kernel id
   bool profile;                         // record an event pair around every launch
   std::vector<cudaEvent_t> prof_events; // start, stop, start, stop, ...
   std::vector<int> prof_kernel;         // kernel id of each pair
@@ -154,8 +162,10 @@ struct LaunchScope {
   less_ctx* c;
   cudaStream_t s;
   bool on;
-  LaunchScope(less_ctx* ctx, int kernel_id, cudaStream_t stream) : c(ctx), s(stream), on(ctx->profile) {
+  LaunchScope(less_ctx* ctx, int kernel_id, cudaStream_t stream, const char* variant = nullptr)
+      : c(ctx), s(stream), on(ctx->profile) {
     c->launches += 1;
+    if (variant) snprintf(c->variant[kernel_id], sizeof c->variant[kernel_id], "%s", variant);
     if (!on) return;
     cudaEvent_t a = take(), b = take();
     c->prof_events.push_back(a);
@@ -188,11 +198,13 @@ inline int check_launch(const char* kernel) {
 }
 
 // Whether the decode kernel is launched as a programmatic dependent of the feature-map kernel.
-// It pays only while every decode CTA can be resident beside the feature-map CTAs: with more
-// instances than that, the early CTAs sit on their SMs waiting for the feature maps and only take
-// bandwidth and room from the weight stream (measured: 64 x 1024 instances 1.54 -> 1.71 ms per step).
+// When it waits for the feature kernel's whole grid this pays only while every decode CTA can be
+// resident beside the feature-map CTAs: with more instances than that, the early CTAs sit on
+// their SMs waiting and only take bandwidth and room from the weight stream (measured: 64 x 1024
+// instances 1.54 -> 1.71 ms per step).  With per-head counters a decode CTA waits for its own
+// head's feature maps only, and any number of instances can follow the feature kernel.
 inline bool overlap_decode(const less_ctx* c) {
-  return c->pdl && !c->profile && !(c->d.flags & LESS_NO_STATE) && c->d.I <= 8 * c->sms;
+  return c->pdl && !c->profile && !(c->d.flags & LESS_NO_STATE) && (c->flags_this_step || c->d.I <= 8 * c->sms);
 }
 
 // launchers (host), defined in the kernel translation units

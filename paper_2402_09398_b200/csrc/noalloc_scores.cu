@@ -19,6 +19,7 @@
 //     it later reads;
 //   * the first call on each device looks up the array's device address; make
 //     that first call outside any stream capture.
+#include <atomic>
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -36,8 +37,9 @@ constexpr int kMaxDevices = 64;
 // [0, MAX_ROWS): row maxima; [MAX_ROWS, 2*MAX_ROWS): reciprocal row sums
 static __device__ __align__(256) float g_noalloc_scratch[2 * LESS_NOALLOC_MAX_ROWS];
 
-// In host code the name above is only a handle; kernels need the address below.
-float* g_scratch_addr[kMaxDevices] = {nullptr};
+// In host code the name above is only a handle; kernels need the address below.  Atomic, so that
+// first calls from several host threads may race on the look-up: both find the same address.
+std::atomic<float*> g_scratch_addr[kMaxDevices];
 
 __device__ __forceinline__ void row_to_float(float* x, const __half* row) {
 #pragma unroll
@@ -159,13 +161,12 @@ extern "C" int less_prompt_scores_noalloc(const void* Q, const void* K, int32_t 
   if (n_inst == 0 || prompt_len == 0) return LESS_OK;
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return LESS_ERR_CUDA;
-  if (!g_scratch_addr[dev]) {
+  float* sm = g_scratch_addr[dev].load(std::memory_order_relaxed);
+  if (!sm) {
     // once per device, with that device current: the device address of the array
-    float* p = nullptr;
-    if (cudaGetSymbolAddress((void**)&p, g_noalloc_scratch) != cudaSuccess || !p) return LESS_ERR_CUDA;
-    g_scratch_addr[dev] = p;
+    if (cudaGetSymbolAddress((void**)&sm, g_noalloc_scratch) != cudaSuccess || !sm) return LESS_ERR_CUDA;
+    g_scratch_addr[dev].store(sm, std::memory_order_relaxed);
   }
-  float* sm = g_scratch_addr[dev];
   float* sl = sm + LESS_NOALLOC_MAX_ROWS;
   cudaStream_t s = (cudaStream_t)cuda_stream;
   const dim3 grid((prompt_len + kTile - 1) / kTile, n_inst);

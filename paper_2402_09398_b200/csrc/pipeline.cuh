@@ -53,9 +53,9 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
   return ok != 0;
 }
 
-// Bounded wait for the phase with the given parity to complete.  false = gave up.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
-  for (uint32_t i = 0; i < kSpinLimit; ++i)
+// Bounded wait for the phase with the given parity to complete.  false = gave up after `limit` polls.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, uint32_t limit = kSpinLimit) {
+  for (uint32_t i = 0; i < limit; ++i)
     if (mbar_try_wait(bar, parity)) return true;
   return false;
 }
@@ -64,10 +64,10 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
 // waiter leaves at once if its CTA has given up; a wait that runs out makes the CTA give up and
 // records where in the device status word (first writer wins), so that nothing can hang.
 __device__ __forceinline__ void wait_or_give_up(uint64_t* bar, uint32_t parity, volatile int* abort, int32_t* status,
-                                                int where) {
+                                                int where, uint32_t limit = kSpinLimit) {
   if (mbar_try_wait(bar, parity)) return;
   if (*abort) return;
-  if (!mbar_wait(bar, parity)) {
+  if (!mbar_wait(bar, parity, limit)) {
     *abort = 1;
     if (atomicCAS(status, 0, 1 /* timeout */) == 0) status[1] = where;
   }

@@ -2,7 +2,7 @@
 (batch, layer, head) instances and compares the library's results with them.
 
 Tolerances (fp16 inputs, fp32 accumulation on the GPU, fp64 in the oracle):
-  outputs            max-abs <= 2e-3
+  outputs            max-abs <= 2e-3 (fp16 outputs: plus half an fp16 ulp of the value, 2^-11 |x|)
   H, z, dH, dz       norm-wise relative <= 1e-3
   phi, psi           norm-wise relative <= 1e-3
   accumulated score  relative <= 2e-5 (+1e-7 absolute)
@@ -118,6 +118,7 @@ class TeacherForced:
                       "lr_num": 0.0, "lr_den": 0.0}
         dev = ctx.device
         self.evicted = torch.empty(ctx.instances, dtype=torch.int32, device=dev)
+        self.f16_out = bool(flags & 32)
 
     def step(self, q, k, v):
         ctx, w = self.ctx, self.w
@@ -136,7 +137,8 @@ class TeacherForced:
             r = orc.decode(qh[inst], kh[inst], vh[inst])
             err = float(np.max(np.abs(out_h[inst] - r["out"])))
             self.worst["out"] = max(self.worst["out"], err)
-            assert err <= OUT_TOL, f"inst {inst} t={a['t']}: out max-abs {err}"
+            tol = OUT_TOL + (2.0 ** -11 * np.abs(r["out"]) if self.f16_out else 0.0)
+            assert np.all(np.abs(out_h[inst] - r["out"]) <= tol), f"inst {inst} t={a['t']}: out max-abs {err}"
             if use_state:
                 e1 = rel_err(phi_g[inst], orc.phi_fn(qh[inst][None])[0])
                 e2 = rel_err(psi_g[inst], orc.psi_fn(kh[inst][None])[0])
@@ -278,6 +280,7 @@ class GroupTeacherForced:
         self.evictions = 0
         self.worst = {"out": 0.0, "dH": 0.0, "dz": 0.0, "acc": 0.0, "phi": 0.0, "psi": 0.0}
         self.evicted = torch.empty(ctx.instances, dtype=torch.int32, device=ctx.device)
+        self.f16_out = bool(flags & 32)
 
     def step(self, q, k, v):
         ctx, w, G, D = self.ctx, self.w, self.w.group, self.w.head_dim
@@ -297,7 +300,8 @@ class GroupTeacherForced:
             r = orc.decode(qh[inst], kh[inst], vh[inst])
             err = float(np.max(np.abs(out_h[inst] - r["out"])))
             self.worst["out"] = max(self.worst["out"], err)
-            assert err <= OUT_TOL, f"inst {inst} t={a['t']}: out max-abs {err}"
+            tol = OUT_TOL + (2.0 ** -11 * np.abs(r["out"]) if self.f16_out else 0.0)
+            assert np.all(np.abs(out_h[inst] - r["out"]) <= tol), f"inst {inst} t={a['t']}: out max-abs {err}"
             if use_state:
                 for g in range(G):
                     e1 = rel_err(phi_g[inst, g], orc.phi_fns[g](qh[inst, g][None])[0])

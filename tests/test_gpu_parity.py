@@ -328,6 +328,106 @@ def test_decode_many_instances_and_ragged_slots(overlap, monkeypatch):
     ctx.close()
 
 
+@pytest.mark.parametrize("batch,layers,heads,rank,ctas", [(4, 4, 80, 8, 0), (20, 2, 32, 16, 0), (70, 1, 19, 8, 0),
+                                                          (20, 2, 32, 8, 16)])
+def test_decode_follows_the_feature_kernel_head_by_head(batch, layers, heads, rank, ctas, monkeypatch):
+    """More instances than can wait on the GPU at once (> 8 per SM): the decode kernel starts as a
+    programmatic dependent of the feature-map kernel and every CTA waits only for the counters of
+    its own head's phi and psi; CTAs are numbered head-major.  Small-batch and large-batch feature
+    kernels, several token tiles (batch 70), a feature grid cut to 16 CTAs.  Teacher-forced parity,
+    then free-running steps back to back must equal, bit for bit, a context without the overlap."""
+    import harness
+    if ctas:
+        monkeypatch.setenv("LESS_FEATURE_CTAS", str(ctas))
+    w = small(130 + batch, batch=batch, layers=layers, heads=heads, prompt=40, steps=3, heavy=9, recent=9,
+              rank=rank, weight_std=0.1)
+    assert w.instances > 8 * 148
+    ctx, W = _setup(w)
+    assert "tc" in ctx.kernel_variant("feature_map") or ctx.kernel_variant("feature_map") == ""
+    _prefill_all(ctx, w, with_out=False)
+    tf = harness.TeacherForced(ctx, w, W, list(range(0, w.instances, 97)) + [w.instances - 1])
+    for s in range(w.steps):
+        tf.step(*wl.make_decode_inputs(w, s, DEV))
+    assert ctx.poll_status() == 0
+    assert ctx.kernel_variant("feature_map").startswith("feature_tc")
+    monkeypatch.setenv("LESS_NO_OVERLAP", "1")
+    ref, _ = _setup(w)
+    monkeypatch.delenv("LESS_NO_OVERLAP")
+    inst = list(range(0, w.instances, 53))
+    ref.import_state(inst, ctx.export_state(inst))
+    sub = torch.tensor(inst, device=DEV)
+    ins = [wl.make_decode_inputs(w, 3 + s, DEV) for s in range(6)]
+    outs_a = [ctx.decode_step(*x).clone() for x in ins]          # no synchronisation between the steps
+    outs_b = [ref.decode_step(*x).clone() for x in ins]
+    for a, b in zip(outs_a, outs_b):
+        assert torch.equal(a.reshape(-1, w.head_dim)[sub], b.reshape(-1, w.head_dim)[sub])
+    for a, b in zip(ctx.export_state(inst), ref.export_state(inst)):
+        for key in ("pos", "acc", "K", "V", "psi", "H", "z"):
+            assert np.array_equal(a[key], b[key]), key
+    assert ctx.poll_status() == 0 and ref.poll_status() == 0
+    ctx.close(); ref.close()
+
+
+@pytest.mark.parametrize("group", [1, 4])
+def test_fp16_output_flag(group):
+    """LESS_OUT_F16: the attention output is the fp32 result rounded once to fp16 (tolerance: the
+    2e-3 of fp32 outputs plus half an fp16 ulp of the value); cache and state do not depend on it."""
+    import harness
+    w = small(140 + group, steps=5, weight_std=0.1, group=group)
+    ctx16, W = _setup(w, flags=32)
+    ctx32, _ = _setup(w)
+    for c in (ctx16, ctx32):
+        _prefill_all(c, w, with_out=False)
+    inst = list(range(w.instances))
+    tf = (harness.GroupTeacherForced if group > 1 else harness.TeacherForced)(ctx16, w, W, inst, flags=32)
+    for s in range(w.steps):
+        q, k, v = wl.make_decode_inputs(w, s, DEV)
+        o16 = tf.step(q, k, v)
+        o32 = ctx32.decode_step(q, k, v)
+        assert o16.dtype == torch.float16 and torch.equal(o16, o32.to(torch.float16))
+    for a, b in zip(ctx16.export_state(inst), ctx32.export_state(inst)):
+        for key in ("pos", "acc", "K", "V", "psi", "H", "z"):
+            assert np.array_equal(a[key], b[key]), key
+    # host entry: fp16 output written in place into pinned memory; q and k as one host block
+    q, k, v = wl.make_decode_inputs(w, w.steps, DEV)
+    ref = ctx32.decode_step(q, k, v).to(torch.float16).cpu()
+    qk = torch.empty(q.numel() + k.numel(), dtype=torch.float16).pin_memory()
+    hq, hk = qk[:q.numel()].view(q.shape), qk[q.numel():].view(k.shape)
+    hq.copy_(q); hk.copy_(k)
+    hv = v.cpu().pin_memory()
+    hout = torch.zeros(ref.shape, dtype=torch.float16).pin_memory()
+    ctx16.decode_step_host(hq, hk, hv, hout)
+    assert torch.equal(hout, ref)
+    assert ctx16.poll_status() == 0
+    ctx16.close(); ctx32.close()
+
+
+def test_bounded_wait_runs_out_and_the_context_reports_it():
+    """A wait that nothing ever satisfies (a barrier without a producer, a limit of a few thousand
+    polls) ends by itself: the kernel returns, the status word says which wait gave up, and a fresh
+    context on the same GPU works normally afterwards.  Nothing here faults or waits without limit."""
+    import harness
+    from paper_2402_09398_b200 import binding
+    w = small(150, batch=1, layers=1, heads=2, prompt=32, steps=2, heavy=6, recent=6)
+    ctx, W = _setup(w)
+    assert ctx.poll_status() == 0 and ctx.status_where() == 0
+    assert ctx.selftest_wait_timeout(0) == -1 and ctx.selftest_wait_timeout(1 << 21) == -1
+    assert ctx.selftest_wait_timeout(3000) == 0
+    assert ctx.poll_status() == -7                       # LESS_ERR_DEVICE_TIMEOUT
+    assert ctx.status_where() == 90
+    assert "wait" in binding.less_strerror(-7)
+    assert ctx.selftest_wait_timeout(3000) == 0          # a context that has given up skips the wait
+    assert ctx.poll_status() == -7
+    ctx.close()
+    ctx, W = _setup(w)                                   # the GPU and the library are unaffected
+    _prefill_all(ctx, w, with_out=False)
+    tf = harness.TeacherForced(ctx, w, W, list(range(w.instances)))
+    for s in range(w.steps):
+        tf.step(*wl.make_decode_inputs(w, s, DEV))
+    assert ctx.poll_status() == 0
+    ctx.close()
+
+
 @pytest.mark.parametrize("pinned,group", [(True, 1), (False, 1), (True, 4), (False, 2)])
 def test_host_buffer_entry_matches_device_entry(pinned, group):
     """less_decode_step_host with pinned (read / written in place by the kernel) and pageable
@@ -423,7 +523,7 @@ def test_captured_step_replays_with_grouped_query_heads():
     test_captured_step_replays_like_direct_calls(3, group=4)
 
 
-@pytest.mark.parametrize("kernel", ["teams", "rows", "mma"])
+@pytest.mark.parametrize("kernel", ["rows", "mma"])
 @pytest.mark.parametrize("group,rank,flags", [(2, 8, 0), (4, 16, 0), (8, 8, 0), (4, 8, 4), (2, 16, 1), (4, 8, 2)])
 def test_grouped_query_heads_decode_from_empty(group, rank, flags, kernel, monkeypatch):
     """Section 3.2, multi-query attention: G query heads share one KV head's cache, scores and

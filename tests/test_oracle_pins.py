@@ -560,50 +560,69 @@ def test_tova_can_evict_the_new_token_itself():
 # --------------------------------------------------------------------------- #
 # Grouped query heads (Section 3.2: H2O scores aggregated across the query heads of a KV head)
 # --------------------------------------------------------------------------- #
-def _group_case(G, cfg_id=100, S=28, T=12, heavy=3, recent=4, D=16, R=4, policy="h2o", use_state=True):
+def _group_case(G, cfg_id=100, S=28, T=12, heavy=3, recent=4, D=16, R=4, policy="h2o", use_state=True,
+                score_norm="less"):
     w = tiny(cfg_id=cfg_id, S=S, T=T, heavy=heavy, recent=recent, D=D, R=R, heads=G + 1)
     W = wl.make_weights(w)
     Q, K, V = wl.make_prompt(w, 0, 1)
     phis = [lo.make_mlp_maps(*head_weights(W, 0, g))[0] for g in range(G)]      # phi of query head g
     psi_w = head_weights(W, 0, G)                                               # psi of the KV head
     psi_fn = lo.make_mlp_maps(*psi_w)[1]
-    grp = lo.LessGroup(D, R, heavy, recent, phis, psi_fn, use_state=use_state, policy=policy)
+    grp = lo.LessGroup(D, R, heavy, recent, phis, psi_fn, score_norm=score_norm, use_state=use_state, policy=policy)
     Qg = np.stack([Q[0, 0, g].double().numpy() for g in range(G)])
     Kk, Vv = K[0, 0, G].double().numpy(), V[0, 0, G].double().numpy()
     return w, W, grp, Qg, Kk, Vv, psi_w
 
 
-def test_group_of_one_is_the_single_head_instance():
-    w, W, grp, Qg, Kk, Vv, psi_w = _group_case(1)
-    one = lo.LessInstance(16, 4, 3, 4, grp.phi_fns[0], grp.psi_fn)
+GROUP_MODES = [(policy, norm, state) for policy in ("h2o", "lambda") for norm in ("less", "sparse")
+               for state in (True, False)]
+
+
+@pytest.mark.parametrize("policy,norm,state", GROUP_MODES)
+def test_group_of_one_is_the_single_head_instance(policy, norm, state):
+    """G = 1 reduces the grouped recursion to LessInstance in every mode the grouped CUDA kernels
+    are compared against: both policies, both normalisers of the H2O scores, state on and off."""
+    w, W, grp, Qg, Kk, Vv, psi_w = _group_case(1, policy=policy, use_state=state, score_norm=norm)
+    one = lo.LessInstance(16, 4, 3, 4, grp.phi_fns[0], grp.psi_fn, score_norm=norm, use_state=state, policy=policy)
     assert np.array_equal(grp.prefill(Qg, Kk, Vv)[0], one.prefill(Qg[0], Kk, Vv))
+    assert list(grp.pos) == list(one.pos) and np.array_equal(grp.acc, one.acc)
     for s in range(w.steps):
         q, k, v = (a[0, 0].double().numpy() for a in wl.make_decode_inputs(w, s))
         a, b = grp.decode(q[:1], k[1], v[1]), one.decode(q[0], k[1], v[1])
         assert np.array_equal(a["out"][0], b["out"]) and a["evicted_pos"] == b["evicted_pos"]
-    assert np.array_equal(grp.H, one.H) and list(grp.pos) == list(one.pos)
+        assert np.array_equal(grp.acc, one.acc)
+    assert np.array_equal(grp.H, one.H) and np.array_equal(grp.z, one.z) and list(grp.pos) == list(one.pos)
+    if not state:
+        assert not grp.H.any() and not grp.z.any()
 
 
+@pytest.mark.parametrize("policy,norm,state", GROUP_MODES)
 @pytest.mark.parametrize("G", [2, 4])
-def test_group_scores_are_summed_over_heads_and_state_is_shared(G):
-    """Independent check with torch: every head's output is Eq. 3 over the shared kept set and the
-    shared Eq. 6 sums; the victim is the minimum of the head-summed accumulated probabilities, kept
-    here in a dict by position and rebuilt from scratch every step."""
-    w, W, grp, Qg, Kk, Vv, psi_w = _group_case(G, cfg_id=101)
+def test_group_scores_are_summed_over_heads_and_state_is_shared(G, policy, norm, state):
+    """Independent replay with torch, in every mode: each head's output is Eq. 3 over the shared
+    kept set and the shared Eq. 6 sums (zero with the state off); H2O's victim is the minimum of
+    the head-summed accumulated probabilities - each head's probability under its own normaliser,
+    Eq. 3's or the sparse-only one - kept here in a dict by position and rebuilt every step;
+    Lambda-masking's kept set is its closed form, the first `heavy` positions plus the window."""
+    w, W, grp, Qg, Kk, Vv, psi_w = _group_case(G, cfg_id=101, policy=policy, use_state=state, score_norm=norm)
     heavy, recent, N = 3, 4, 7
     grp.prefill(Qg, Kk, Vv)
     Kt, Vt = [torch.tensor(Kk)], [torch.tensor(Vv)]
     S = w.prompt
-    # prompt scores: sum over heads of the causal softmax column sums
-    score = np.zeros(S)
-    for g in range(G):
-        s = torch.tensor(Qg[g]) @ Kt[0].T / math.sqrt(16)
-        s = s.masked_fill(torch.triu(torch.ones_like(s), 1).bool(), float("-inf"))
-        score += torch.softmax(s, dim=-1).sum(0).numpy()
-    cand = sorted(range(S - recent), key=lambda j: (score[j], j))
-    kept = set(range(S)) - set(cand[: S - N])
+    if policy == "h2o":
+        # prompt scores: sum over heads of the causal softmax column sums
+        score = np.zeros(S)
+        for g in range(G):
+            s = torch.tensor(Qg[g]) @ Kt[0].T / math.sqrt(16)
+            s = s.masked_fill(torch.triu(torch.ones_like(s), 1).bool(), float("-inf"))
+            score += torch.softmax(s, dim=-1).sum(0).numpy()
+        cand = sorted(range(S - recent), key=lambda j: (score[j], j))
+        gone = set(cand[: S - N])
+    else:
+        score = np.zeros(S)
+        gone = set(range(heavy, S - recent))
+    kept = set(range(S)) - gone
     hist = {j: score[j] for j in kept}
-    gone = set(cand[: S - N])
     assert sorted(kept) == list(grp.pos)
     phi_w = [head_weights(W, 0, g)[:2] for g in range(G)]
     for i in range(w.steps):
@@ -614,23 +633,58 @@ def test_group_scores_are_summed_over_heads_and_state_is_shared(G):
         r = grp.decode(q[:G], k[G], v[G])
         idx = sorted(kept) + [t]
         g_idx = sorted(gone)
-        psi = torch_psi(Kall[g_idx].numpy(), *psi_w[2:])
-        Hs, zs = psi.T @ Vall[g_idx], psi.sum(0)
+        if state:
+            psi = torch_psi(Kall[g_idx].numpy(), *psi_w[2:])
+            Hs, zs = psi.T @ Vall[g_idx], psi.sum(0)
+            assert np.allclose(r["lr_num"][0], (torch_phi(q[0][None], *phi_w[0])[0] @ Hs).numpy(), rtol=1e-9, atol=1e-13)
+        else:
+            Hs, zs = torch.zeros(4, 16, dtype=torch.float64), torch.zeros(4, dtype=torch.float64)
+            assert not grp.H.any() and not grp.z.any()
         psum = np.zeros(len(idx))
         for g in range(G):
             e = torch.exp(Kall[idx] @ torch.tensor(q[g]) / math.sqrt(16))
             phi = torch_phi(q[g][None], *phi_w[g])[0]
             den = phi @ zs + e.sum()
             assert np.allclose(r["out"][g], ((phi @ Hs + e @ Vall[idx]) / den).numpy(), rtol=1e-10, atol=1e-13)
-            psum += (e / den).numpy()
-        for j, pj in zip(idx, psum):
-            hist[j] = hist.get(j, 0.0) + pj
-        victim = min((hist[j], j) for j in idx if j <= t - recent)[1]
+            psum += (e / (den if norm == "less" else e.sum())).numpy()
+        assert np.allclose(r["p"], psum, rtol=1e-10, atol=1e-14)
+        if policy == "h2o":
+            for j, pj in zip(idx, psum):
+                hist[j] = hist.get(j, 0.0) + pj
+            victim = min((hist[j], j) for j in idx if j <= t - recent)[1]
+            del hist[victim]
+        else:
+            victim = min(j for j in idx if j >= heavy)
+            assert victim == t - recent                # closed form: the window slides by one
         assert r["evicted_pos"] == victim
         kept = (kept | {t}) - {victim}
         gone.add(victim)
-        del hist[victim]
+        if policy == "lambda":
+            assert kept == set(range(heavy)) | set(range(t - recent + 1, t + 1))
     assert sorted(kept) == list(grp.pos)
+    if policy == "h2o":
+        assert np.allclose(grp.acc, [hist[j] for j in sorted(kept)], rtol=1e-10, atol=1e-14)
+
+
+def test_group_sparse_normaliser_differs_only_through_the_low_rank_mass():
+    """A planted slip - the sparse normaliser applied where Eq. 3's belongs - changes the
+    accumulated scores exactly when z != 0: with the state off the two modes agree bit for bit,
+    with it on they must differ."""
+    runs = {}
+    for norm in ("less", "sparse"):
+        for state in (True, False):
+            w, W, grp, Qg, Kk, Vv, _ = _group_case(2, cfg_id=102, use_state=state, score_norm=norm)
+            grp.prefill(Qg, Kk, Vv)
+            for i in range(w.steps):
+                q, k, v = (a[0, 0].double().numpy() for a in wl.make_decode_inputs(w, i))
+                grp.decode(q[:2], k[2], v[2])
+            runs[norm, state] = (list(grp.pos), grp.acc.copy())
+    assert runs["less", False][0] == runs["sparse", False][0]
+    assert np.array_equal(runs["less", False][1], runs["sparse", False][1])
+    common = sorted(set(runs["less", True][0]) & set(runs["sparse", True][0]))
+    a = np.array([runs["less", True][1][runs["less", True][0].index(j)] for j in common])
+    b = np.array([runs["sparse", True][1][runs["sparse", True][0].index(j)] for j in common])
+    assert np.all(b >= a) and np.any(b > a)            # the sparse normaliser is the smaller one
 
 
 # --------------------------------------------------------------------------- #

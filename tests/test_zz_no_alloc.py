@@ -6,8 +6,10 @@ buffers and a stream and nothing more.  For them the library carries its
 scratch in a fixed array of its own.  This test calls that entry point through
 the C ABI twice in a row (the second call with a different prompt length, so it
 runs over whatever the first one left in the shared array) and checks each
-result against the accumulated scores that less_prefill produces for the same
-inputs, within the tolerance the prefill parity tests use for those scores.
+result against the CPU oracle's prompt scores of the same inputs and against
+the accumulated scores that less_prefill produces, within the tolerance the
+prefill parity tests use for those scores; a third call fills the scratch
+array to its last row.
 
 The file sorts last on purpose: a run that stops at the first failure has then
 already run every other test.
@@ -38,6 +40,19 @@ def _scores_from_prefill(w, Q, K, V):
     return out
 
 
+def _scores_oracle(w, Q, K, V):
+    """prompt_acc of every head from the fp64 oracle (nothing evicted: slots >= tokens)."""
+    from oracle import less_oracle as lo
+    out = np.zeros((w.instances, w.prompt))
+    ident = lambda x: np.abs(x[:, :w.rank])             # the scores do not depend on the feature maps
+    for inst in range(w.instances):
+        b, layer, head = wl.instance_coords(w, inst)
+        o = lo.LessInstance(w.head_dim, w.rank, w.heavy, w.recent, ident, ident)
+        o.prefill(*(t[b, layer, head].double().cpu().numpy() for t in (Q, K, V)))
+        out[inst] = o.prompt_acc
+    return out
+
+
 def _scores_noalloc(w, Q, K):
     from paper_2402_09398_b200 import binding as B
     # [B, L, H, S, D] contiguous is [n_inst, S, D] in the instance order of the library
@@ -57,10 +72,22 @@ def test_noalloc_scores_match_prefill_twice_in_a_row():
         Q, K, V = wl.make_prompt(w, 0, w.layers, DEV)
         got = _scores_noalloc(w, Q, K)
         want = _scores_from_prefill(w, Q, K, V)
+        ref = _scores_oracle(w, Q, K, V)
         assert np.isfinite(got).all()
+        assert np.allclose(got, ref, rtol=ACC_RTOL, atol=ACC_ATOL), np.max(np.abs(got - ref))
         assert np.allclose(got, want, rtol=ACC_RTOL, atol=ACC_ATOL), np.max(np.abs(got - want))
         # every causal softmax row sums to one, so the scores of a head sum to the prompt length
         assert np.allclose(got.sum(axis=1), w.prompt, rtol=1e-4)
+    # exactly as many rows as the scratch array holds: the last row is used, nothing beyond it
+    w = wl.Workload(63, 64, 1, 4, 128, B.LESS_NOALLOC_MAX_ROWS // 256, 0, 300, 300, 8, heavy_rule="none")
+    assert w.instances * w.prompt == B.LESS_NOALLOC_MAX_ROWS
+    Q, K, V = wl.make_prompt(w, 0, w.layers, DEV)
+    got = _scores_noalloc(w, Q, K)
+    last = w.instances - 1                             # the head whose rows end the scratch array
+    ref = _scores_oracle(w.with_(batch=1, heads=1), *(t.reshape(-1, 1, 1, w.prompt, 128)[last:last + 1]
+                                                       for t in (Q, K, V)))
+    assert np.allclose(got[-1], ref[0], rtol=ACC_RTOL, atol=ACC_ATOL)
+    assert np.allclose(got.sum(axis=1), w.prompt, rtol=1e-4)
     # sizes beyond the built-in scratch are refused before anything is launched
     big = B.LESS_NOALLOC_MAX_ROWS // 64 + 1
     dummy = torch.zeros(16, dtype=torch.float16, device=DEV)
