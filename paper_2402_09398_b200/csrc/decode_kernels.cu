@@ -175,6 +175,8 @@ __device__ __forceinline__ void wait_feature_maps(const DecParams& p, int lh) {
         set_status(p.a.status, kStatusTimeout, 3);
         break;
       }
+      // once any wait of this context has given up, the others do not sit theirs out
+      if ((i & 255u) == 0 && *reinterpret_cast<volatile int32_t*>(p.a.status) != 0) break;
       __nanosleep(64);
     }
   }

@@ -614,7 +614,7 @@ int launch_feature_tc(less_ctx* c, const FmParams& p_in, cudaStream_t s) {
   // With the overlap on, the ring gives up stages so that decode CTAs of the same step fit beside
   // this kernel's CTA on every SM (at these batch sizes the kernel is bound by its epilogue, not
   // by the weight stream: three stages feed it).
-  const int cap_l = c->feature_stages >= 2 ? c->feature_stages : (c->pdl ? 3 : FT_MAX_STAGES);
+  const int cap_l = c->feature_stages >= 2 ? c->feature_stages : (c->pdl ? 3 : FT_MAX_STAGES);   // d.I is not known to be small here either way: three stages feed this kernel
   if (gm.nstage > cap_l) gm.nstage = cap_l;
   if (gm.nstage < 2) return LESS_ERR_INVALID_CONFIG;
   const uint32_t need = 2u * gm.npad + 16u;
@@ -634,12 +634,18 @@ int launch_feature_tc(less_ctx* c, const FmParams& p_in, cudaStream_t s) {
   if (c->feature_ctas > 0 && c->feature_ctas < sms) sms = c->feature_ctas;
   const int grid = gm.items < sms ? gm.items : sms;
   const int nt = d.B <= 1 ? 1 : d.B <= 2 ? 2 : d.B <= 4 ? 4 : 8;
-  // Per-head counters: direct calls only (a captured step would replay a stale target), and only
-  // where the decode kernel can be a programmatic dependent.  Every flagged launch adds the same
-  // number of writer warps to every head's counter, so the target is one running total.
+  // Per-head counters, so that any number of decode CTAs can follow this kernel as programmatic
+  // dependents.  Direct calls only (a captured step would replay a stale target).  Not needed
+  // while every decode CTA fits on the GPU at once, and not used behind the small-batch kernel with
+  // more instances than that: that kernel is bound by its weight stream, and successive waves of
+  // decode CTAs take so much of the bandwidth from it that the feature maps they wait for arrive
+  // later than without the overlap (measured, 4 x 1600 heads x 654 slots: 533 us per step against 486).
+  // Every flagged launch adds the same number of writer warps to every head's counter, so the target
+  // is one running total.
   cudaStreamCaptureStatus capturing = cudaStreamCaptureStatusNone;
   cudaStreamIsCapturing(s, &capturing);
-  if (capturing == cudaStreamCaptureStatusNone && c->pdl) {
+  const bool many = d.I > 8 * c->sms;
+  if (capturing == cudaStreamCaptureStatusNone && c->pdl && many && d.B > 8) {
     uint32_t writers = 0;
     if (d.B <= 8) writers = (uint32_t)(nt * d.R + 31) / 32;
     else
@@ -661,7 +667,7 @@ int launch_feature_tc(less_ctx* c, const FmParams& p_in, cudaStream_t s) {
     // With the overlap on, one stage of the ring is given up so that the decode kernel's CTAs of
     // the same step fit beside this kernel's CTA on every SM (measured on the Llama-2-7B shape at
     // batch 1: 83.5 us per step with 6 stages and no room, 74.5 us with 5, 74.2 us with 4).
-    const int cap = c->feature_stages >= 2 ? c->feature_stages : (c->pdl ? 5 : FT_MAX_STAGES);
+    const int cap = c->feature_stages >= 2 ? c->feature_stages : (c->pdl && !many ? 5 : FT_MAX_STAGES);
     if (gm.nstage > cap) gm.nstage = cap;
     if (gm.nstage < 2) return LESS_ERR_INVALID_CONFIG;
     const size_t sm = fx + (size_t)gm.nstage * FT_STAGE_BYTES;

@@ -2,9 +2,10 @@
 coefficients together with the error of the fp32 evaluation.
 
     gelu(x) = x * Phi(x),   Phi(-u) = E(u) / 2,   Phi(u) = 1 - E(u) / 2   (u = |x|)
+            = max(x, 0) - u * E(u) / 2        (both signs in one expression, no select)
     E(u) = erfc(u / sqrt(2)) = 2^(-u * g(u))
 
-g is smooth on [0, 8] (g(0) = sqrt(2 / pi) / ln 2), so a degree-7 polynomial in u reproduces it
+g is smooth on [0, 8] (g(0) = sqrt(2 / pi) / ln 2), so a degree-5 polynomial in u reproduces it
 well enough that the fp32 result is limited by rounding, not by the fit; both tails come out of
 the exponential directly, without the cancellation of 1 - erf.  Run:  python gelu_fit.py
 """
@@ -13,7 +14,7 @@ from numpy.polynomial import chebyshev as C
 from scipy.special import erfc
 
 U = 8.0      # u is clamped here: E(8) = 1.2e-15, below fp32 resolution of every use
-DEG = 7
+DEG = 5
 
 
 def fit():
@@ -34,8 +35,9 @@ def gelu_f32(xs, co):
     for a in co[-2::-1]:
         q = (q * u + a).astype(np.float32)
     E = np.exp2((-q * u).astype(np.float32)).astype(np.float32)
-    phi = np.where(xs < 0, np.float32(0.5) * E, np.float32(1) - np.float32(0.5) * E).astype(np.float32)
-    return (xs * phi).astype(np.float32)
+    t = (u * E).astype(np.float32)
+    # fma(-0.5, t, max(x, 0)): one rounding
+    return (np.maximum(xs, np.float32(0)).astype(np.float64) - 0.5 * t.astype(np.float64)).astype(np.float32)
 
 
 if __name__ == "__main__":

@@ -318,9 +318,18 @@ int less_decode_step_host(less_ctx* c, const void* qh, const void* kh, const voi
   const void* v_dev = device_alias(vh);
   void* out_dev = device_alias(outh);
   if (((uintptr_t)v_dev & 15) || ((uintptr_t)out_dev & 15)) { v_dev = nullptr; out_dev = nullptr; }
-  const bool one_block = (const char*)kh == (const char*)qh + nq && (char*)c->a.stage_k == (char*)c->a.stage_q + nq;
-  cudaError_t e = cudaMemcpyAsync(c->a.stage_q, qh, one_block ? nq + nin : nq, cudaMemcpyHostToDevice, s);
-  if (e == cudaSuccess && !one_block) e = cudaMemcpyAsync(c->a.stage_k, kh, nin, cudaMemcpyHostToDevice, s);
+  cudaError_t e = cudaSuccess;
+  bool copied = false;
+  if ((const char*)kh == (const char*)qh + nq && (char*)c->a.stage_k == (char*)c->a.stage_q + nq) {
+    // k directly behind q.  If the two are separate host allocations that merely touch, the runtime
+    // refuses the copy that spans them (nothing is enqueued): then they go one by one.
+    copied = cudaMemcpyAsync(c->a.stage_q, qh, nq + nin, cudaMemcpyHostToDevice, s) == cudaSuccess;
+    if (!copied) cudaGetLastError();
+  }
+  if (!copied) {
+    e = cudaMemcpyAsync(c->a.stage_q, qh, nq, cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(c->a.stage_k, kh, nin, cudaMemcpyHostToDevice, s);
+  }
   if (e == cudaSuccess && !v_dev) e = cudaMemcpyAsync(c->a.stage_v, vh, nin, cudaMemcpyHostToDevice, s);
   if (e != cudaSuccess) return LESS_ERR_CUDA;
   int rc = less_decode_step(c, c->a.stage_q, c->a.stage_k, v_dev ? v_dev : c->a.stage_v,

@@ -64,6 +64,7 @@ int launch_attn_out_tc(less_ctx* c, const PfParams& p, int G, cudaStream_t s);
 int launch_state_tc(less_ctx* c, const PfParams& p, int G, cudaStream_t s);
 bool psi_tc_supported(const Dims& d);
 int launch_psi_tc(less_ctx* c, const PfParams& p, int G, cudaStream_t s);
+int launch_psi_state_tc(less_ctx* c, const PfParams& p, int G, cudaStream_t s);   // psi fused with the state build
 int launch_phi_tc(less_ctx* c, const PfParams& p, int G, cudaStream_t s, float* out);
 
 }  // namespace less

@@ -496,8 +496,9 @@ int launch_prefill_group(less_ctx* c, int layer0, int nl, int lj0, int layer_cou
   }
   const size_t smem = (size_t)(FM_BR * kHeadDim + mlp_smem_floats(d.Rp)) * 4;
   const bool use_state = !(d.flags & LESS_NO_STATE);
-  if (nsplit > 0 && use_state && psi_tc_supported(d)) {
-    const int rc = launch_psi_tc(c, p, G, s);
+  const bool fused = nsplit > 0 && use_state && psi_tc_supported(d);   // psi and the state build in one kernel
+  if (fused) {
+    const int rc = launch_psi_state_tc(c, p, G, s);
     if (rc != LESS_OK) return rc;
   } else if (nsplit > 0 && use_state) {
     LaunchScope scope(c, LESS_KERNEL_PSI, s);
@@ -515,7 +516,7 @@ int launch_prefill_group(less_ctx* c, int layer0, int nl, int lj0, int layer_cou
     if (d.R == 8) gather_kernel<8><<<dim3(gx, G), GA_THREADS, 0, s>>>(p);
     else gather_kernel<16><<<dim3(gx, G), GA_THREADS, 0, s>>>(p);
   }
-  if (nsplit > 0 && use_state) {
+  if (nsplit > 0 && use_state && !fused) {
     const int rc = launch_state_tc(c, p, G, s);
     if (rc != LESS_OK) return rc;
   }
