@@ -740,7 +740,7 @@ def measure_prefill(args, ranks, cpu_seconds, steps=None):
 
         def part(keys):
             ms = sum(kt.get(k, 0.0) for k in keys)
-            f = sum(fl[k] for k in keys if k in fl)
+            f = sum(fl[k] for k in keys if k in fl and kt.get(k, 0.0) > 0)
             tf = f / (ms * 1e-3) / 1e12 if ms else 0.0
             return {"ms": ms, "algorithmic_flops": f, "TFLOPs": tf, "frac": tf / peak}
         rec = {"metric": PROMPT_METRIC,

@@ -291,8 +291,9 @@ __global__ void __launch_bounds__(FL_THREADS) feature_tc_kernel(
               // columns past the last token hold products with zero-filled rows: no GELU spent on them
               // (c1 multiplies the layer-2 sums instead: the fp16 operand must not depend on how
               // small that learnable scalar is)
-              const float h0 = blk * 8 + 2 * e < nb ? gelu_erf(__uint_as_float(acc[i][2 * e])) : 0.f;
-              const float h1 = blk * 8 + 2 * e + 1 < nb ? gelu_erf(__uint_as_float(acc[i][2 * e + 1])) : 0.f;
+              float h0 = 0.f, h1 = 0.f;
+              if (blk * 8 + 2 * e + 1 < nb) gelu_erf2(__uint_as_float(acc[i][2 * e]), __uint_as_float(acc[i][2 * e + 1]), h0, h1);
+              else if (blk * 8 + 2 * e < nb) h0 = gelu_erf(__uint_as_float(acc[i][2 * e]));
               const __half2 hh = __floats2half2_rn(h0, h1);
               const float2 hf2 = __half22float2(hh);
               const __half2 ll = __floats2half2_rn(h0 - hf2.x, h1 - hf2.y);

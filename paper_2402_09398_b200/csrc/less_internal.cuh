@@ -135,6 +135,43 @@ __device__ __forceinline__ float gelu_erf(float x) {
   return fmaf(-0.5f, u * e, fmaxf(x, 0.f));
 }
 
+// The same function for two values at once with Blackwell's packed fp32 arithmetic (fma / mul
+// .f32x2: two results per issued instruction; bit-identical to gelu_erf, one rounding per
+// operation either way).  The MLP epilogues are bound by instruction issue, not by the FMA lanes.
+__device__ __forceinline__ uint64_t f32x2_pack(float a, float b) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
+  return r;
+}
+__device__ __forceinline__ void f32x2_unpack(uint64_t v, float& a, float& b) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v));
+}
+__device__ __forceinline__ uint64_t f32x2_fma(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t r;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+  return r;
+}
+__device__ __forceinline__ uint64_t f32x2_mul(uint64_t a, uint64_t b) {
+  uint64_t r;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+__device__ __forceinline__ void gelu_erf2(float x0, float x1, float& r0, float& r1) {
+  const uint64_t u = f32x2_pack(fminf(fabsf(x0), 8.0f), fminf(fabsf(x1), 8.0f));
+  uint64_t g = f32x2_pack(-3.155045488e-05f, -3.155045488e-05f);
+  g = f32x2_fma(g, u, f32x2_pack(7.533458411e-04f, 7.533458411e-04f));
+  g = f32x2_fma(g, u, f32x2_pack(-8.018460125e-03f, -8.018460125e-03f));
+  g = f32x2_fma(g, u, f32x2_pack(5.329473317e-02f, 5.329473317e-02f));
+  g = f32x2_fma(g, u, f32x2_pack(4.588809609e-01f, 4.588809609e-01f));
+  g = f32x2_fma(g, u, f32x2_pack(1.151154518e+00f, 1.151154518e+00f));
+  float t0, t1, e0, e1;
+  f32x2_unpack(f32x2_mul(g, u), t0, t1);
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e0) : "f"(-t0));
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e1) : "f"(-t1));
+  f32x2_unpack(f32x2_fma(f32x2_pack(-0.5f, -0.5f), f32x2_mul(u, f32x2_pack(e0, e1)),
+                         f32x2_pack(fmaxf(x0, 0.f), fmaxf(x1, 0.f))), r0, r1);
+}
+
 __device__ __forceinline__ void half8_to_float(const uint4& u, float* f) {
   const __half2* h = reinterpret_cast<const __half2*>(&u);
 #pragma unroll

@@ -448,12 +448,13 @@ int launch_prefill_group(less_ctx* c, int layer0, int nl, int lj0, int layer_cou
   p.grp = d.G;
   // grouped query heads run on the tensor-core scoring kernels only
   if (d.G > 1 && S > 0 && !(c->score_path == 1 && score_tc_supported())) return LESS_ERR_INVALID_CONFIG;
-  // Token splits of the state build: whole 128-token tiles, long enough that the head's W1
-  // (128 KB, reloaded per split) is amortised, short enough that the grid fills the GPU.
+  // Token splits of the state build: whole 128-token tiles, as long as they can be (the head's W1,
+  // 128 KB, and the CTA's set-up are paid per split) while the grid still is several waves deep,
+  // so that the last wave's imbalance stays small.
   const int G = d.B * nl * d.Hd;
-  int nsplit = 0, split_tokens = 1024;
+  int nsplit = 0, split_tokens = 8192;
   if (S > 0) {
-    while (split_tokens > 128 && (long long)G * ((S + split_tokens - 1) / split_tokens) < 148) split_tokens >>= 1;
+    while (split_tokens > 128 && (long long)G * ((S + split_tokens - 1) / split_tokens) < 8 * c->sms) split_tokens >>= 1;
     if ((S + split_tokens - 1) / split_tokens > kMaxSplit)
       split_tokens = ((S + kMaxSplit - 1) / kMaxSplit + 127) / 128 * 128;
     nsplit = (S + split_tokens - 1) / split_tokens;

@@ -33,23 +33,28 @@
 namespace less {
 
 constexpr int PT_WORKERS = 512;                    // 16 epilogue warps: four per tensor-memory lane quadrant
-constexpr int PT_THREADS = PT_WORKERS + 128;       // + TMA producer, GEMM1, GEMM2 and state-product issuers
+constexpr int PT_THREADS = PT_WORKERS + 128;       // + TMA producer, GEMM1, GEMM2 and state-product issuers: a warp each (two
+                                                   // issuers in one warp would block each other in their waits)
 constexpr int PT_TILE = 128;                       // tokens per tile
 constexpr int PT_CHUNK = 128;                      // hidden units per GEMM1 chunk (64 when the hidden width is 64)
 constexpr int PT_KBYTES = PT_TILE * kHeadDim * 2;  // one K (or V) tile
 constexpr int PT_W2N = 16;                         // GEMM2 N (R padded to 16)
-// tensor-memory columns: D1 buffers at 0 and 128, G2 at 256, per-tile state accumulators behind
-constexpr uint32_t PT_G2COL = 256, PT_HCOL = 288, PT_HSTRIDE = 64, PT_TMEM = 512;
+// tensor-memory columns: three D1 buffers of 128, G2 at 384, the per-tile state accumulators (H^T, then
+// z 32 columns on) behind.  Three D1 buffers, not two: the chain "GEMM2 reads the hidden layer of chunk
+// q - 1, GEMM1 refills that buffer" takes about as long as the epilogue of one chunk (a thread gets
+// an MMA out every ~84 cycles), so with two buffers the epilogue warps waited for it at every chunk.
+constexpr int PT_D1BUFS = 3;
+constexpr uint32_t PT_G2COL = 384, PT_HCOL = 416, PT_TMEM = 512;
 
 struct PtShared {
   uint64_t w1_full;
   uint64_t k_full, k_empty;
   uint64_t v_full, v_empty;
-  uint64_t d1_full[2], d1_free[2];
-  uint64_t hid_full[2];   // per D1 buffer: a warp cannot arrive for the buffer's next use before this one is consumed
+  uint64_t d1_full[PT_D1BUFS], d1_free[PT_D1BUFS];
+  uint64_t hid_full[PT_D1BUFS];   // per D1 buffer: a warp cannot arrive for the buffer's next use before this one is consumed
   uint64_t g2_full, g2_free;
   uint64_t b_full, b_free;
-  uint64_t h_full[2], h_free[2];
+  uint64_t h_full, h_free;
   uint64_t mx_bar;        // the four finishing warps meet here twice per tile
   uint32_t tmem_base;
   int abort;
@@ -57,6 +62,7 @@ struct PtShared {
   float c1, c2;
   float wmax[4];          // per quadrant: largest psi of the tile that enters the state
   float inv_scale[2];     // per state accumulator buffer: 1 / the tile's scale
+  float zacc[16];         // the split's z (one thread adds a tile's z at a time)
 };
 
 __device__ __forceinline__ void pt_wait(uint64_t* bar, uint32_t parity, volatile int* abort, int32_t* status,
@@ -82,8 +88,8 @@ struct PtMap {
 __device__ __forceinline__ void gelu_split(uint32_t a0, uint32_t a1, uint32_t& hi, uint32_t& lo) {
   // c1 multiplies the layer-2 sums instead (same value): the fp16 hi + lo operand then never
   // depends on how small the learnable scalar is (the paper initialises it to 1e-4)
-  const float h0 = gelu_erf(__uint_as_float(a0));
-  const float h1 = gelu_erf(__uint_as_float(a1));
+  float h0, h1;
+  gelu_erf2(__uint_as_float(a0), __uint_as_float(a1), h0, h1);
   const __half2 hh = __floats2half2_rn(h0, h1);
   const float2 hf = __half22float2(hh);
   const __half2 ll = __floats2half2_rn(h0 - hf.x, h1 - hf.y);
@@ -128,13 +134,13 @@ __global__ void __launch_bounds__(PT_THREADS) psi_tc_kernel(const __grid_constan
     mbar_init(&sh->k_empty, 1);
     mbar_init(&sh->v_full, 1);
     mbar_init(&sh->v_empty, 1);
-    for (int s = 0; s < 2; ++s) {
+    for (int s = 0; s < PT_D1BUFS; ++s) {
       mbar_init(&sh->d1_full[s], 1);
       mbar_init(&sh->d1_free[s], 1);
       mbar_init(&sh->hid_full[s], PT_WORKERS / 32);
-      mbar_init(&sh->h_full[s], 1);
-      mbar_init(&sh->h_free[s], 4);
     }
+    mbar_init(&sh->h_full, 1);
+    mbar_init(&sh->h_free, 4);
     mbar_init(&sh->g2_full, 1);
     mbar_init(&sh->g2_free, 4);
     mbar_init(&sh->b_full, 4);
@@ -202,13 +208,12 @@ __global__ void __launch_bounds__(PT_THREADS) psi_tc_kernel(const __grid_constan
       const uint32_t idesc1 = idesc_f16(128, chunk, 0, 1);          // A = K tile (K-major), B = W1 (N-major)
       const uint32_t w1a = smem_u32(w1s);
       pt_wait(&sh->w1_full, 0, abortp, status, 31);
-      uint32_t q = 0;                                               // chunk counter over all tiles
+      uint32_t b = 0, bph = 0;                                      // D1 buffer of the chunk and its phase: counted
       for (int i = 0; i < ntiles && !*abortp; ++i) {
         pt_wait(&sh->k_full, i & 1, abortp, status, 33);
         const uint32_t ka = smem_u32(kbuf);
-        for (int c = 0; c < nchunk && !*abortp; ++c, ++q) {
-          const int b = q & 1;
-          pt_wait(&sh->d1_free[b], ((q >> 1) & 1) ^ 1, abortp, status, 32);   // GEMM2 has read the hidden layer of chunk q - 2
+        for (int c = 0; c < nchunk && !*abortp; ++c, (++b == PT_D1BUFS ? (b = 0, bph ^= 1) : 0u)) {
+          pt_wait(&sh->d1_free[b], bph ^ 1, abortp, status, 32);   // GEMM2 has read the hidden layer this buffer held before
           if (*abortp) break;
           tc_fence_after_sync();
 #pragma unroll
@@ -228,12 +233,11 @@ __global__ void __launch_bounds__(PT_THREADS) psi_tc_kernel(const __grid_constan
     if (tid == PT_WORKERS + 64) {
       constexpr uint32_t idesc2 = idesc_f16(128, PT_W2N, 0, 1);     // A = hidden (tensor memory), B = W2 (N-major)
       const uint32_t w2a = smem_u32(w2s);
-      uint32_t q = 0;
+      uint32_t b = 0, bph = 0;
       for (int i = 0; i < ntiles && !*abortp; ++i) {
-        for (int c = 0; c < nchunk; ++c, ++q) {
-          const int b = q & 1;
+        for (int c = 0; c < nchunk; ++c, (++b == PT_D1BUFS ? (b = 0, bph ^= 1) : 0u)) {
           if (c == 0) pt_wait(&sh->g2_free, (i & 1) ^ 1, abortp, status, 34);
-          pt_wait(&sh->hid_full[b], (q >> 1) & 1, abortp, status, 35);
+          pt_wait(&sh->hid_full[b], bph, abortp, status, 35);
           if (*abortp) break;
           tc_fence_after_sync();
           // part w of the chunk: hidden units 32 w .. 32 w + 31 sit in D1 columns 32 w .. 32 w + 31 as
@@ -260,13 +264,12 @@ __global__ void __launch_bounds__(PT_THREADS) psi_tc_kernel(const __grid_constan
       constexpr uint32_t idesc_z = idesc_f16(128, NB, 0, 1);   // A = ones (K-major)
       const uint32_t ones_addr = smem_u32(ones), va = smem_u32(vbuf), ba = smem_u32(bbuf);
       for (int i = 0; i < ntiles; ++i) {
-        const int b = i & 1;
         pt_wait(&sh->v_full, i & 1, abortp, status, 21);
         pt_wait(&sh->b_full, i & 1, abortp, status, 22);
-        pt_wait(&sh->h_free[b], ((i >> 1) & 1) ^ 1, abortp, status, 23);
+        pt_wait(&sh->h_free, (i & 1) ^ 1, abortp, status, 23);      // the tile before has been collected
         if (*abortp) break;
         tc_fence_after_sync();
-        const uint32_t hcol = tmem + PT_HCOL + b * PT_HSTRIDE;
+        const uint32_t hcol = tmem + PT_HCOL;
 #pragma unroll
         for (int ks = 0; ks < PT_TILE / 16; ++ks) {
           const uint64_t bd = smem_desc(ba + ks * 2 * B_LBO, B_LBO, B_SBO, kLayoutNone);
@@ -277,7 +280,7 @@ __global__ void __launch_bounds__(PT_THREADS) psi_tc_kernel(const __grid_constan
         }
         mma_commit(&sh->v_empty);
         mma_commit(&sh->b_free);
-        mma_commit(&sh->h_full[b]);
+        mma_commit(&sh->h_full);
       }
     }
   } else {
@@ -289,41 +292,44 @@ __global__ void __launch_bounds__(PT_THREADS) psi_tc_kernel(const __grid_constan
     const uint32_t lane_addr = tmem + ((uint32_t)(quad * 32) << 16);
     float* psi = mp.out + (size_t)g * p.Sp * R;
     const int32_t* slot_of = p.a.ws_slot + (size_t)g * p.Sp;
-    uint32_t q = 0;
     float pmax = 0.f;                                  // largest psi this thread has produced
-    float hacc[kState ? R : 1], zacc[kState ? R : 1]; // part 1: column `row` of the split's H^T, and z
+    float hacc[kState ? R : 1];                        // part 1: column `row` of the split's H^T
 #pragma unroll
-    for (int r = 0; r < (kState ? R : 1); ++r) hacc[r] = zacc[r] = 0.f;
+    for (int r = 0; r < (kState ? R : 1); ++r) hacc[r] = 0.f;
+    if (kState && part == 1 && row < R) sh->zacc[row] = 0.f;   // lanes of one warp (quadrant 0, part 1), which alone touches it afterwards
+    __syncwarp();
     // the tile whose state products part 1 still has to collect
     auto collect = [&](int i) {
-      const int b = i & 1;
-      pt_wait(&sh->h_full[b], (i >> 1) & 1, abortp, status, 24);
+      pt_wait(&sh->h_full, i & 1, abortp, status, 24);
       tc_fence_after_sync();
-      uint32_t hv[NB], zv[NB];
-      const uint32_t hcol = lane_addr + PT_HCOL + b * PT_HSTRIDE;
-      if (NB == 32) { tmem_ld32(hcol, hv); tmem_ld32(hcol + 32, zv); }
-      else { tmem_ld16(hcol, hv); tmem_ld16(hcol + 32, zv); }
+      uint32_t hv[NB];
+      const uint32_t hcol = lane_addr + PT_HCOL;
+      const float inv = sh->inv_scale[i & 1];          // exact: a power of two
+      if (NB == 32) tmem_ld32(hcol, hv); else tmem_ld16(hcol, hv);
       tmem_ld_wait();
-      const float inv = sh->inv_scale[b];              // exact: a power of two
-      tc_fence_before_sync();
-      mbar_arrive_warp(&sh->h_free[b]);
 #pragma unroll
-      for (int r = 0; r < R; ++r) {
-        hacc[r] = fmaf(__uint_as_float(hv[r]) + __uint_as_float(hv[R + r]), inv, hacc[r]);
-        zacc[r] = fmaf(__uint_as_float(zv[r]) + __uint_as_float(zv[R + r]), inv, zacc[r]);
+      for (int r = 0; r < R; ++r) hacc[r] = fmaf(__uint_as_float(hv[r]) + __uint_as_float(hv[R + r]), inv, hacc[r]);
+      if (quad == 0) {                                 // every row of the z accumulator holds the tile's z: lane 0 keeps the sum
+        if (NB == 32) tmem_ld32(hcol + 32, hv); else tmem_ld16(hcol + 32, hv);
+        tmem_ld_wait();
+        if (lane == 0) {
+#pragma unroll
+          for (int r = 0; r < R; ++r) sh->zacc[r] = fmaf(__uint_as_float(hv[r]) + __uint_as_float(hv[R + r]), inv, sh->zacc[r]);
+        }
       }
+      tc_fence_before_sync();
+      mbar_arrive_warp(&sh->h_free);
     };
+    uint32_t b = 0, bph = 0;                           // D1 buffer of the chunk and its phase: counted
     for (int i = 0; i < ntiles && !*abortp; ++i) {
-      for (int c = 0; c < nchunk && !*abortp; ++c, ++q) {
-        const int b = q & 1;
+      for (int c = 0; c < nchunk && !*abortp; ++c, (++b == PT_D1BUFS ? (b = 0, bph ^= 1) : 0u)) {
         if (part < cparts) {
-          pt_wait(&sh->d1_full[b], (q >> 1) & 1, abortp, status, 36);
+          pt_wait(&sh->d1_full[b], bph, abortp, status, 36);
           tc_fence_after_sync();
-          uint32_t acc[32];                              // this warp's 32 of the chunk's columns
+          uint32_t acc[32], hi[16], lo[16];              // this warp's 32 of the chunk's columns
           const uint32_t col = lane_addr + b * 128 + part * 32;
           tmem_ld32(col, acc);
           tmem_ld_wait();
-          uint32_t hi[16], lo[16];
 #pragma unroll
           for (int e = 0; e < 16; ++e) gelu_split(acc[2 * e], acc[2 * e + 1], hi[e], lo[e]);
           tmem_st16(col, hi);
@@ -417,9 +423,9 @@ __global__ void __launch_bounds__(PT_THREADS) psi_tc_kernel(const __grid_constan
       float* hp = p.a.ws_hpart + ((size_t)g * kMaxSplit + split) * (R * kHeadDim + R);
 #pragma unroll
       for (int r = 0; r < R; ++r) hp[r * kHeadDim + row] = hacc[r];
-      if (row == 0) {                                    // every row of the z accumulator holds z
+      if (row == 0) {
 #pragma unroll
-        for (int r = 0; r < R; ++r) hp[R * kHeadDim + r] = zacc[r];
+        for (int r = 0; r < R; ++r) hp[R * kHeadDim + r] = sh->zacc[r];
       }
     }
     if (!kState) {
