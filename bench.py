@@ -575,7 +575,12 @@ def measure_decode(args, ranks, cfg_id, cpu_seconds):
     variants = {k: ctx.kernel_variant(k) for k in ("feature_map", "decode")}
 
     # ---- end to end through the host-buffer entry point ----
-    hq, hk, hv = (torch.empty(base[0][i].shape, dtype=torch.float16).pin_memory() for i in range(3))
+    # q and k in one pinned block (k directly behind q: one host-to-device copy), v and the output in
+    # pinned memory too (read / written in place by the decode kernel)
+    nq_el, nk_el = base[0][0].numel(), base[0][1].numel()
+    hqk = torch.empty(nq_el + nk_el, dtype=torch.float16).pin_memory()
+    hq, hk = hqk[:nq_el].view(base[0][0].shape), hqk[nq_el:].view(base[0][1].shape)
+    hv = torch.empty(base[0][2].shape, dtype=torch.float16).pin_memory()
     hq.copy_(base[0][0]); hk.copy_(base[0][1]); hv.copy_(base[0][2])
     hout = torch.empty(out.shape, dtype=out_dtype).pin_memory()
     for _ in range(3):
