@@ -622,15 +622,26 @@ int launch_feature_tc(less_ctx* c, const FmParams& p_in, cudaStream_t s) {
   gm.tmem_cols = need <= 64 ? 64 : need <= 128 ? 128 : need <= 256 ? 256 : 512;
   const size_t smem = fixed + (size_t)gm.nstage * FT_STAGE_BYTES;
 
-  CUtensorMap tq, tk, tw1a, tw1b;
+  static_assert(sizeof(CUtensorMap) <= 128, "tensor map cache slot");
+  CUtensorMap* tmc = reinterpret_cast<CUtensorMap*>(c->tm_cache);
+  CUtensorMap &tq = tmc[0], &tk = tmc[1], &tw1a = tmc[2], &tw1b = tmc[3];
   const uint64_t lhq = (uint64_t)d.L * p.Hh[0], lhk = (uint64_t)d.L * p.Hh[1];   // layer-heads of phi / psi
-  // q, k: [B rows][L*Hd*128 columns]; a box is npad batch rows x 64 columns of one head
-  if (!make_tmap_f16_2d(&tq, p.x[0], d.B, lhq * kHeadDim, lhq * kHeadDim * 2, gm.npad) ||
-      !make_tmap_f16_2d(&tk, p.x[1], d.B, lhk * kHeadDim, lhk * kHeadDim * 2, gm.npad))
-    return fail_cuda("tensor map of q / k");
-  if (!make_tmap_f16_2d(&tw1a, p.w1[0], lhq * kHeadDim, d.Rp, (uint64_t)d.Rp * 2, kHeadDim) ||
-      !make_tmap_f16_2d(&tw1b, p.w1[1], lhk * kHeadDim, d.Rp, (uint64_t)d.Rp * 2, kHeadDim))
-    return fail_cuda("tensor map of W1");
+  // q, k: [B rows][L*Hd*128 columns]; a box is `box` batch rows x 64 columns of one head (the small
+  // kernel loads 8 input rows per half tile).  The maps are kept in the context between steps.
+  const int box = d.B <= 8 ? FS_XROWS : gm.npad;
+  if (c->tm_box != box || c->tm_q != p.x[0] || c->tm_k != p.x[1]) {
+    c->tm_box = 0;
+    if (!make_tmap_f16_2d(&tq, p.x[0], d.B, lhq * kHeadDim, lhq * kHeadDim * 2, box) ||
+        !make_tmap_f16_2d(&tk, p.x[1], d.B, lhk * kHeadDim, lhk * kHeadDim * 2, box))
+      return fail_cuda("tensor map of q / k");
+    c->tm_q = p.x[0]; c->tm_k = p.x[1]; c->tm_box = box;
+  }
+  if (!c->tm_w_ok) {
+    if (!make_tmap_f16_2d(&tw1a, p.w1[0], lhq * kHeadDim, d.Rp, (uint64_t)d.Rp * 2, kHeadDim) ||
+        !make_tmap_f16_2d(&tw1b, p.w1[1], lhk * kHeadDim, d.Rp, (uint64_t)d.Rp * 2, kHeadDim))
+      return fail_cuda("tensor map of W1");
+    c->tm_w_ok = true;
+  }
   int sms = c->sms;
   if (c->feature_ctas > 0 && c->feature_ctas < sms) sms = c->feature_ctas;
   const int grid = gm.items < sms ? gm.items : sms;
@@ -672,10 +683,6 @@ int launch_feature_tc(less_ctx* c, const FmParams& p_in, cudaStream_t s) {
     if (gm.nstage > cap) gm.nstage = cap;
     if (gm.nstage < 2) return LESS_ERR_INVALID_CONFIG;
     const size_t sm = fx + (size_t)gm.nstage * FT_STAGE_BYTES;
-    // the small kernel loads 8 input rows per half tile
-    if (!make_tmap_f16_2d(&tq, p.x[0], d.B, lhq * kHeadDim, lhq * kHeadDim * 2, FS_XROWS) ||
-        !make_tmap_f16_2d(&tk, p.x[1], d.B, lhk * kHeadDim, lhk * kHeadDim * 2, FS_XROWS))
-      return fail_cuda("tensor map of q / k");
     if (d.R == 8) {
       if (nt == 1) return launch_small<8, 1>(c, p, gm, tq, tk, tw1a, tw1b, sm, grid, s);
       if (nt == 2) return launch_small<8, 2>(c, p, gm, tq, tk, tw1a, tw1b, sm, grid, s);

@@ -179,6 +179,9 @@ int less_create(const less_config* cfg, const less_weights* w, void* arena, size
   c->flags_this_step = false;
   c->flag_target[0] = c->flag_target[1] = 0;
   c->status_where = 0;
+  c->tm_q = c->tm_k = nullptr;
+  c->tm_box = 0;
+  c->tm_w_ok = false;
   memset(c->variant, 0, sizeof c->variant);
   c->feature_ctas = 0;
   if (const char* e = getenv("LESS_FEATURE_CTAS")) c->feature_ctas = atoi(e);

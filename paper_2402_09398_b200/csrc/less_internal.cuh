@@ -92,6 +92,13 @@ struct less_ctx {
   uint32_t flag_target[2];  // counter value of a head once this step's phi / psi are written
   int status_where;         // where-code of the last status word read by less_poll_status
   char variant[LESS_KERNEL_COUNT][64];   // name of the kernel variant last launched under each kernel id
+  // tensor maps of the feature-map kernels, kept between steps (encoding four of them costs more host
+  // time than a small step's launches): W1 of phi / psi (fixed), q / k rows (re-encoded when the
+  // caller's pointers change)
+  alignas(64) unsigned char tm_cache[4][128];
+  const void* tm_q; const void* tm_k;
+  int tm_box;          // rows per box of the cached q / k maps, 0 = none cached
+  bool tm_w_ok;
   bool profile;                         // record an event pair around every launch
   std::vector<cudaEvent_t> prof_events; // start, stop, start, stop, ...
   std::vector<int> prof_kernel;         // kernel id of each pair
