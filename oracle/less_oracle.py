@@ -63,8 +63,8 @@ def psi_map(k: np.ndarray, w1: np.ndarray, w2: np.ndarray, w3: np.ndarray,
             scale: Optional[np.ndarray] = None) -> np.ndarray:
     """Eq. 2: psi(k) = | gelu( gelu(k W1) W2 ) W3 |, W3 [R,R].
 
-    `scale` = the two learnable scalars of Section 3.2 ("between layers in
-    psi"), read as one multiplier after each GELU; None means both are 1.
+    `scale` = the two learnable scalars Section 3.2 places inside psi, read as
+    one multiplier after each GELU; None means both are 1.
     """
     k = np.asarray(k, dtype=np.float64)
     c1, c2 = (1.0, 1.0) if scale is None else (float(scale[0]), float(scale[1]))
@@ -103,8 +103,8 @@ class LessInstance:
             raise ValueError("need recent >= 1 and heavy >= 0")
         if policy not in ("h2o", "lambda", "tova"):
             raise ValueError("policy is 'h2o', 'lambda' or 'tova'")
-        # 'lambda' = Lambda-masking (Section 4: "the cache consists of the first 4 and most recent
-        # tokens"): `heavy` counts the first tokens that are always kept, `recent` the window;
+        # 'lambda' = Lambda-masking (Section 4: a handful of first positions plus the recent window
+        # are cached): `heavy` counts the first tokens that are always kept, `recent` the window;
         # accumulated scores play no role in it.
         # 'tova' = the third policy Section 4 names.  The paper gives no definition of it; this is
         # the published rule of the work it cites, per head: whenever the cache overflows, the
@@ -266,8 +266,8 @@ class LessInstance:
 class LessGroup:
     """One KV head shared by G query heads (multi-query / grouped-query attention).
 
-    Section 3.2: "For multi-query attention, we extend H2O to aggregate attention scores across
-    all query attention heads to determine KV pairs to evict."  Reading taken here: the cache
+    Section 3.2 extends H2O to multi-query attention by summing the attention scores of all query
+    heads before it decides which pair to evict.  Reading taken here: the cache
     (kept K, V), the accumulated scores and the low-rank state H, z belong to the KV head (psi
     acts on keys, so H = sum psi(k)^T v does not depend on the query head); every query head g has
     its own phi_g and its own Eq. 3 over the shared cache and state; the H2O score of an entry
@@ -406,7 +406,8 @@ def masked_parallel_attention(Q, K, V, exact_until, phi_fn, psi_fn, rows=None):
     """The parallel form (Section 3.2, Inexpensive Training; Section 4.1): every row of the causal
     attention matrix at once.  Entry (i, j), j <= i, is exp(q_i . k_j / sqrt(D)) while key j is still
     in the sparse cache when query i attends, i.e. i < exact_until[j], and phi(q_i) psi(k_j)^T from
-    then on (the entry "found by the kernel functions"); each row is normalised once, as in Eq. 3:
+    then on (Section 3.2: the kernel functions supply what the sparse cache no longer holds); each
+    row is normalised once, as in Eq. 3:
 
         out_i = sum_j A_ij v_j / sum_j A_ij.
 

@@ -58,6 +58,7 @@ __global__ void __launch_bounds__(AO_THREADS) attn_out_tc_kernel(const __grid_co
                                                                  const __grid_constant__ CUtensorMap tm_k,
                                                                  const __grid_constant__ CUtensorMap tm_v, PfParams p) {
   extern __shared__ __align__(1024) unsigned char ao_smem[];
+  if (smem_misaligned(ao_smem, p.a.status, 100)) return;
   unsigned char* qres = ao_smem;                                   // Q tile: [2 halves][128 rows][128 B]
   unsigned char* ring = qres + AO_TILE_BYTES;                      // [stages][K tile | V tile]
   AoShared* sh = reinterpret_cast<AoShared*>(ring + AO_STAGES * AO_STAGE_BYTES);

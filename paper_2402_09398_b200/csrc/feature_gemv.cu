@@ -5,7 +5,7 @@
 // warp streams the item's weights (W1 in 16-KB row chunks, then W2) into a
 // shared-memory ring with bulk asynchronous copies, eight consumer warps do
 // the arithmetic.  The hidden activations never leave shared memory (the
-// paper's "absorbed activation", Section 3.2, taken to the whole MLP).
+// paper folds the activation into the preceding linear kernel, Section 3.2, taken to the whole MLP).
 #include "feature_gemv.cuh"
 #include "pipeline.cuh"
 

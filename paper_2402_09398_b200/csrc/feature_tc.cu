@@ -20,7 +20,7 @@
 //     D2[tokens x 16] += H[tokens x 128 hidden] * W2[chunk rows, :]       (GEMM2)
 // whose accumulator lives in tensor memory across the chunks.  After the last
 // chunk: c2 * gelu(c1 * .), W3 (psi only) and the absolute value on CUDA cores.
-// The hidden activations never leave the SM (the paper's "absorbed activation",
+// The hidden activations never leave the SM (the paper folds the activation into the preceding linear kernel,
 // Section 3.2, taken to the whole MLP).  Plain TMA loads only; every wait is bounded.
 #include "feature_gemv.cuh"
 #include "tc_common.cuh"
@@ -130,6 +130,7 @@ __global__ void __launch_bounds__(FL_THREADS) feature_tc_kernel(
     const __grid_constant__ CUtensorMap tm_w1phi, const __grid_constant__ CUtensorMap tm_w1psi, FmParams p,
     FtGeom gm, int32_t* status) {
   extern __shared__ __align__(1024) unsigned char ft_smem[];
+  if (smem_misaligned(ft_smem, status, 60)) return;
   const int Rp = p.Rp, nchunk = Rp / FT_CHUNK, npad = gm.npad, nstage = gm.nstage;
   const uint32_t hbytes = (uint32_t)npad * 256;      // hi (or lo): npad/8 token blocks x 2 KB
   const uint32_t xbytes = (uint32_t)npad * 256;      // two 64-column halves of npad rows x 128 B
@@ -427,6 +428,7 @@ __global__ void __launch_bounds__(FT_THREADS) feature_tc_small_kernel(
     const __grid_constant__ CUtensorMap tm_w1phi, const __grid_constant__ CUtensorMap tm_w1psi, FmParams p,
     FtGeom gm, int32_t* status) {
   extern __shared__ __align__(1024) unsigned char ft_smem[];
+  if (smem_misaligned(ft_smem, status, 60)) return;
   constexpr int V = NT * R;
   const int Rp = p.Rp, nchunk = Rp / FT_CHUNK, nstage = gm.nstage;
   const uint32_t w2bytes = (uint32_t)Rp * R * 2;

@@ -243,6 +243,7 @@ __global__ void __launch_bounds__(MF_THREADS) masked_out_tc_kernel(const __grid_
                                                                    const __grid_constant__ CUtensorMap tm_v,
                                                                    PfParams p, MfParams mf) {
   extern __shared__ __align__(1024) unsigned char mf_smem[];
+  if (smem_misaligned(mf_smem, p.a.status, 120)) return;
   unsigned char* qres = mf_smem;                                   // Q tile: [2 halves][128 rows][128 B]
   unsigned char* ring = qres + MF_TILE_BYTES;                      // [stages][K tile, V tile]
   unsigned char* phires = ring + MF_STAGES * MF_STAGE_BYTES;       // phi operand tile of the rows

@@ -106,6 +106,7 @@ __global__ void __launch_bounds__(PT_THREADS) psi_tc_kernel(const __grid_constan
   constexpr uint32_t B_SBO = 128;                    // between 8-column blocks
   constexpr uint32_t B_LBO = (NB / 8) * 128;         // between 8-token groups
   extern __shared__ __align__(1024) unsigned char pt_smem[];
+  if (smem_misaligned(pt_smem, p.a.status, 29)) return;
   const int Rp = p.Rp;
   const int chunk = Rp < PT_CHUNK ? Rp : PT_CHUNK;   // hidden units per chunk
   const int nchunk = Rp / chunk;
@@ -117,10 +118,6 @@ __global__ void __launch_bounds__(PT_THREADS) psi_tc_kernel(const __grid_constan
   unsigned char* bbuf = vbuf + (kState ? PT_KBYTES : 0);         // kState: psi hi | lo as B operand
   __half* ones = reinterpret_cast<__half*>(bbuf + (kState ? PT_TILE * NB * 2 : 0));   // kState: 4 KB of 1.0
   PtShared* sh = reinterpret_cast<PtShared*>(reinterpret_cast<unsigned char*>(ones) + (kState ? 4096 : 0));
-  if (smem_u32(pt_smem) & 1023) {                    // the swizzled tiles need their 1024-byte alignment
-    if (threadIdx.x == 0) set_status(p.a.status, kStatusBounds, 29);
-    return;
-  }
 
   const int tid = threadIdx.x, warp = tid >> 5;
   const int split = blockIdx.x, g = blockIdx.y;

@@ -81,6 +81,7 @@ constexpr int RS_THREADS = 64 + SC_EPI_THREADS;
 __global__ void __launch_bounds__(RS_THREADS) rowstat_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
                                                                 const __grid_constant__ CUtensorMap tm_k, PfParams p) {
   extern __shared__ __align__(1024) unsigned char sc_smem[];
+  if (smem_misaligned(sc_smem, p.a.status, 80)) return;
   unsigned char* qres = sc_smem;                                 // [2 halves][128 rows][128 B]
   unsigned char* ring = qres + SC_RES_BYTES;                     // [stages][2 halves][256 rows][128 B]
   ScShared* sh = reinterpret_cast<ScShared*>(ring + SC_STAGES * SC_STAGE_BYTES);
@@ -243,6 +244,7 @@ constexpr int SC_ONES_BYTES = SC_TILE_M * 32;      // [16 row groups][2 k halves
 __global__ void __launch_bounds__(CS_THREADS) colsum_tc_kernel(const __grid_constant__ CUtensorMap tm_q,
                                                                const __grid_constant__ CUtensorMap tm_k, PfParams p) {
   extern __shared__ __align__(1024) unsigned char sc_smem[];
+  if (smem_misaligned(sc_smem, p.a.status, 80)) return;
   unsigned char* kres = sc_smem;                                 // resident K tile
   unsigned char* ring = kres + SC_RES_BYTES;                     // streamed Q tiles
   unsigned char* bx = ring + SC_STAGES * SC_STAGE_BYTES;         // [stages] (-b_i) columns of the Q tiles, then zeros

@@ -49,6 +49,7 @@ __global__ void __launch_bounds__(ST_THREADS) state_tc_kernel(const __grid_const
   constexpr uint32_t B_SBO = 128;                   // between 8-column blocks
   constexpr uint32_t B_LBO = (NB / 8) * 128;        // between 8-token groups
   extern __shared__ __align__(1024) unsigned char st_smem[];
+  if (smem_misaligned(st_smem, p.a.status, 19)) return;
   unsigned char* vbuf = st_smem;                                        // [stages][2 dblocks][128][128 B]
   unsigned char* bbuf = vbuf + ST_STAGES * ST_VBYTES;                   // [stages][BBYTES]
   __half* ones = reinterpret_cast<__half*>(bbuf + ST_STAGES * BBYTES);  // 4 KB of 1.0

@@ -56,6 +56,19 @@ inline bool make_tmap_f16_2d(CUtensorMap* m, const void* base, uint64_t rows, ui
 }
 
 // ---------------------------------------------------------------------------
+// device: the dynamic shared memory of a kernel with 128-byte-swizzled tiles must start on a
+// 1024-byte boundary (the swizzle pattern is a function of the address).  The declaration asks for
+// it; should a toolchain or a later static __shared__ variable ever break it, the operands would be
+// mis-swizzled silently, so every such kernel checks on entry, records the refusal in the status word
+// (code 2 = a device-side check failed) and returns before it touches a barrier or tensor memory.
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ bool smem_misaligned(const void* dyn_smem, int32_t* status, int where) {
+  if ((smem_u32(dyn_smem) & 1023u) == 0) return false;
+  if (threadIdx.x == 0 && atomicCAS(status, 0, 2) == 0) status[1] = where;
+  return true;
+}
+
+// ---------------------------------------------------------------------------
 // device: TMA
 // ---------------------------------------------------------------------------
 // x = innermost (column) coordinate in elements: must be a multiple of 8 (16 bytes).
