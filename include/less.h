@@ -22,6 +22,7 @@
  *     their inputs must stay valid until the stream reaches the call.
  *   - A context is not thread-safe.
  *   - 16-bit inputs are IEEE fp16; accumulation, scores, H, z and outputs fp32.
+ *   - D below is less_config.head_dim.
  *   - Environment, read by less_create: LESS_LOG (explain host-side failures on
  *     stderr), LESS_FEATURE_KERNEL=gemv|plain (CUDA-core feature-map kernels),
  *     LESS_NO_OVERLAP (no programmatic dependent launch of the decode kernel),
@@ -94,7 +95,7 @@ enum {
 
 typedef struct less_config {
   int32_t batch, layers, heads; /* heads = KV heads: one cache, one H, z and one eviction per (batch, layer, head) */
-  int32_t head_dim;           /* D, must be 128 */
+  int32_t head_dim;           /* D: 128, or 64 (general shapes, see `group`) */
   int32_t rank;               /* R: 8 or 16 (Section 4: R = 8 by default) */
   int32_t hidden;             /* R' = 512 (Section 3.2) */
   int32_t heavy, recent;      /* slots per instance: heavy >= 0, recent >= 1, heavy + recent <= LESS_MAX_SLOTS */
@@ -102,11 +103,16 @@ typedef struct less_config {
   int32_t max_prefill_layers; /* layers scored together in less_prefill (>= 1): sizes the workspace */
   uint32_t flags;
   int32_t group;              /* query heads per KV head (Section 3.2, multi-query attention): 0 or 1 = one;
-                               * 2, 4 or 8 need hidden in {128, 256, 512}, a policy other than
+                               * 2, 4 or 8 with head_dim 128 need hidden in {128, 256, 512}, a policy other than
                                * LESS_POLICY_TOVA, the tensor-core prompt scoring, and
                                * group * (heavy + recent + 1028) * 4 bytes <= 227 KB (the decode kernel
-                               * keeps one score per slot and query head in shared memory);
-                               * anything else is LESS_ERR_INVALID_CONFIG */
+                               * keeps one score per slot and query head in shared memory).
+                               * General shapes - head_dim 64, or any other group up to 128 (Section 4's
+                               * multi-query model has 71 query heads over one KV head of dimension 64) -
+                               * decode on CUDA cores from an empty cache: less_prefill accepts only
+                               * prompt_len == 0 (reset) and less_masked_attention is not available for them;
+                               * 9 * (heavy + recent + 1028) * 4 bytes <= 227 KB, no LESS_POLICY_TOVA with
+                               * group > 1.  Anything else is LESS_ERR_INVALID_CONFIG */
 } less_config;
 
 /* Per-head feature-map weights (Eq. 1, Eq. 2), device, fp16, row-major, no biases:

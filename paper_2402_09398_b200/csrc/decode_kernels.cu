@@ -16,23 +16,25 @@ namespace less {
 // The hidden activations never leave shared memory.
 // --------------------------------------------------------------------------- //
 template <int R>
-__global__ void __launch_bounds__(FM_THREADS) feature_map_kernel(FmParams p) {
+__global__ void __launch_bounds__(FM_THREADS) feature_map_kernel(FmParams p, int which0) {
   extern __shared__ float fm_smem[];
-  float* xs = fm_smem;                         // [FM_BR][128]
-  float* hs = xs + FM_BR * kHeadDim;           // [FM_BR][Rp]
+  const int D = p.D;
+  float* xs = fm_smem;                         // [FM_BR][D]
+  float* hs = xs + FM_BR * D;                  // [FM_BR][Rp]
   float* part = hs + FM_BR * p.Rp;             // [ndg][FM_BR][Rp]
   pdl_launch_dependents();
-  const int lh = blockIdx.x;                   // layer * Hd + head
-  const int which = blockIdx.y;                // 0 phi(q), 1 psi(k)
+  const int which = which0 + blockIdx.y;       // 0 phi(q), 1 psi(k)
+  const int Hh = p.Hh[which];                  // heads of this map per layer
+  const int lh = blockIdx.x;                   // layer * Hh + head
   const int b0 = blockIdx.z * FM_BR;
   const int nb = min(FM_BR, p.B - b0);
   const int tid = threadIdx.x;
-  const int layer = lh / p.Hd, head = lh % p.Hd;
-  for (int e = tid; e < FM_BR * kHeadDim; e += FM_THREADS) {
-    const int b = e / kHeadDim, d = e % kHeadDim;
+  const int layer = lh / Hh, head = lh % Hh;
+  for (int e = tid; e < FM_BR * D; e += FM_THREADS) {
+    const int b = e / D, d = e % D;
     float v = 0.f;
     if (b < nb)
-      v = __half2float(p.x[which][(((size_t)(b0 + b) * p.L + layer) * p.Hd + head) * kHeadDim + d]);
+      v = __half2float(p.x[which][(((size_t)(b0 + b) * p.L + layer) * Hh + head) * D + d]);
     xs[e] = v;
   }
   __syncthreads();
@@ -41,14 +43,23 @@ __global__ void __launch_bounds__(FM_THREADS) feature_map_kernel(FmParams p) {
     c1 = p.psi_scale[lh * 2];
     c2 = p.psi_scale[lh * 2 + 1];
   }
-  const float r = mlp_rows<R>(xs, part, hs, nb, p.w1[which] + (size_t)lh * kHeadDim * p.Rp,
+  const float r = mlp_rows<R>(xs, part, hs, nb, p.w1[which] + (size_t)lh * D * p.Rp,
                               p.w2[which] + (size_t)lh * p.Rp * R, p.w3 + (size_t)lh * R * R, c1,
-                              c2, p.Rp, which == 1);
+                              c2, p.Rp, which == 1, D);
   const int warp = tid >> 5, lane = tid & 31;
   if (warp < nb && lane < R) {
-    const size_t inst = ((size_t)(b0 + warp) * p.L + layer) * p.Hd + head;
+    const size_t inst = ((size_t)(b0 + warp) * p.L + layer) * Hh + head;
     p.out[which][inst * R + lane] = r;
   }
+}
+
+template <int R>
+static int launch_plain_feature_maps(less_ctx* c, const FmParams& p, dim3 grid, int which0, size_t smem, cudaStream_t s) {
+  LaunchScope scope(c, LESS_KERNEL_FEATURE_MAP, s, R == 8 ? "feature_map_kernel<8>" : "feature_map_kernel<16>");
+  if (cudaFuncSetAttribute(feature_map_kernel<R>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+    return fail_cuda("shared memory opt-in of feature_map_kernel");
+  feature_map_kernel<R><<<grid, FM_THREADS, smem, s>>>(p, which0);
+  return check_launch("feature_map_kernel");
 }
 
 int launch_feature_maps(less_ctx* c, const void* q, const void* k, cudaStream_t s) {
@@ -64,26 +75,29 @@ int launch_feature_maps(less_ctx* c, const void* q, const void* k, cudaStream_t 
   p.psi_scale = c->w.psi_scale;
   p.out[0] = c->a.phi_q;
   p.out[1] = c->a.psi_k;
-  p.B = d.B; p.L = d.L; p.Hd = d.Hd; p.Rp = d.Rp;
+  p.B = d.B; p.L = d.L; p.Hd = d.Hd; p.Rp = d.Rp; p.D = d.D;
   p.Hh[0] = d.Hd * d.G; p.Hh[1] = d.Hd;
   p.feat_flag = nullptr; p.flag_stride = d.L * d.Hd * d.G;
   c->flags_this_step = false;
   const int ndg = FM_THREADS / (d.Rp / 8);
-  const size_t smem = (size_t)(FM_BR * kHeadDim + FM_BR * d.Rp + ndg * FM_BR * d.Rp) * 4;
-  dim3 grid(d.L * d.Hd, (d.flags & LESS_NO_STATE) ? 1 : 2, (d.B + FM_BR - 1) / FM_BR);
+  const size_t smem = (size_t)(FM_BR * d.D + FM_BR * d.Rp + ndg * FM_BR * d.Rp) * 4;
   if (d.flags & LESS_NO_STATE) return LESS_OK;   // neither phi nor psi is used
-  if ((c->feature_path == 2 || d.G > 1) && feature_tc_supported(d)) return launch_feature_tc(c, p, s);
-  if (d.G > 1) return LESS_ERR_INVALID_CONFIG;    // the CUDA-core kernels know one query head per KV head
-  if (c->feature_path >= 1 && feature_gemv_supported(d)) return launch_feature_gemv(c, p, s);
-  LaunchScope scope(c, LESS_KERNEL_FEATURE_MAP, s, d.R == 8 ? "feature_map_kernel<8>" : "feature_map_kernel<16>");
-  if (d.R == 8) {
-    cudaFuncSetAttribute(feature_map_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    feature_map_kernel<8><<<grid, FM_THREADS, smem, s>>>(p);
-  } else {
-    cudaFuncSetAttribute(feature_map_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    feature_map_kernel<16><<<grid, FM_THREADS, smem, s>>>(p);
+  const int nbz = (d.B + FM_BR - 1) / FM_BR;
+  if (!d.general) {
+    if ((c->feature_path == 2 || d.G > 1) && feature_tc_supported(d)) return launch_feature_tc(c, p, s);
+    if (d.G > 1) return LESS_ERR_INVALID_CONFIG;    // the streaming kernels below know one query head per KV head
+    if (c->feature_path >= 1 && feature_gemv_supported(d)) return launch_feature_gemv(c, p, s);
+    const dim3 grid(d.L * d.Hd, 2, nbz);
+    return d.R == 8 ? launch_plain_feature_maps<8>(c, p, grid, 0, smem, s) : launch_plain_feature_maps<16>(c, p, grid, 0, smem, s);
   }
-  return check_launch("feature_map_kernel");
+  // general shapes: phi over the query heads, then psi over the KV heads
+  for (int which = 0; which < 2; ++which) {
+    const dim3 grid(d.L * p.Hh[which], 1, nbz);
+    const int rc = d.R == 8 ? launch_plain_feature_maps<8>(c, p, grid, which, smem, s)
+                            : launch_plain_feature_maps<16>(c, p, grid, which, smem, s);
+    if (rc != LESS_OK) return rc;
+  }
+  return LESS_OK;
 }
 
 // --------------------------------------------------------------------------- //
@@ -203,16 +217,19 @@ __device__ __forceinline__ size_t decode_instance(const DecParams& p) {
 //   s_sc  [G][Ns]  e^{s - m_g} of every live entry and, at index n, of the new pair
 //   inv   [G]      1 / normaliser of each head
 //   hcol  [R]      column d of H as read for Eq. 3
-template <int R, int G, bool kCaptured>
+//   D     head dimension: a slot row is D / 8 chunks of 16 bytes; threads d < D own a column of H
+template <int R, int G, bool kCaptured, int D = kHeadDim>
 __device__ __forceinline__ void decode_tail(const DecParams& p, size_t inst, int n, int t_now, const float* s_sc, int Ns,
                                             const float (&inv)[G], const float (&hcol)[R], const uint4& knew,
                                             const uint4& vnew, unsigned long long* s_key, int* s_vic) {
-  const int tid = threadIdx.x, d = tid, l16 = tid & 15, rg = tid >> 4;
+  constexpr int LPR = D / 8;                           // lanes per slot row
+  const int tid = threadIdx.x, d = tid, l16 = tid % LPR, rg = tid / LPR;
+  const bool own = D == DEC_THREADS || d < D;
   const int N = p.N;
   const bool use_state = !(p.flags & LESS_NO_STATE);
-  float* Hb = p.a.H + inst * (size_t)R * kHeadDim;
+  float* Hb = p.a.H + inst * (size_t)R * D;
   float* zb = p.a.z + inst * R;
-  const __half* Vb = p.a.vslots + inst * (size_t)N * kHeadDim;
+  const __half* Vb = p.a.vslots + inst * (size_t)N * D;
   int32_t* posb = p.a.pos + inst * (size_t)p.Np;
   float* accb = p.a.acc + inst * (size_t)p.Np;
   const bool full = (n == N);
@@ -262,10 +279,12 @@ __device__ __forceinline__ void decode_tail(const DecParams& p, size_t inst, int
       if (key_new < best) {                            // uniform over the CTA
         if (tid == 0 && p.evicted_pos) p.evicted_pos[inst] = t_now;
         if (use_state) {
-          const float vv = __half2float(p.v[inst * kHeadDim + d]);
           const float* psn = p.a.psi_k + inst * R;
+          if (own) {
+            const float vv = __half2float(p.v[inst * D + d]);
 #pragma unroll
-          for (int r = 0; r < R; ++r) Hb[r * kHeadDim + d] = fmaf(__ldcg(psn + r), vv, hcol[r]);
+            for (int r = 0; r < R; ++r) Hb[r * D + d] = fmaf(__ldcg(psn + r), vv, hcol[r]);
+          }
           if (tid < R) zb[tid] += __ldcg(psn + tid);
         }
         step_done<kCaptured>(p.a.tpos, p.t);
@@ -288,10 +307,12 @@ __device__ __forceinline__ void decode_tail(const DecParams& p, size_t inst, int
     if (tid == 0 && p.evicted_pos) p.evicted_pos[inst] = vpos;
     // ---- Eq. 4 / Eq. 5: absorb the victim (psi acts on the key: the state is the KV head's) ----
     if (use_state) {
-      const float vv = __half2float(Vb[(size_t)slot * kHeadDim + d]);
       const float* psv = p.a.psic + (inst * (size_t)N + slot) * R;
+      if (own) {
+        const float vv = __half2float(Vb[(size_t)slot * D + d]);
 #pragma unroll
-      for (int r = 0; r < R; ++r) Hb[r * kHeadDim + d] = fmaf(psv[r], vv, hcol[r]);
+        for (int r = 0; r < R; ++r) Hb[r * D + d] = fmaf(psv[r], vv, hcol[r]);
+      }
       if (tid < R) zb[tid] += psv[tid];
     }
     __syncthreads();                                   // victim row fully read before overwrite
@@ -302,8 +323,8 @@ __device__ __forceinline__ void decode_tail(const DecParams& p, size_t inst, int
     }
   }
   // ---- the new pair takes the slot in place ----
-  __half* Kw = p.a.kslots + (inst * (size_t)N + slot) * kHeadDim;
-  __half* Vw = p.a.vslots + (inst * (size_t)N + slot) * kHeadDim;
+  __half* Kw = p.a.kslots + (inst * (size_t)N + slot) * D;
+  __half* Vw = p.a.vslots + (inst * (size_t)N + slot) * D;
   if (rg == 0) *reinterpret_cast<uint4*>(Kw + l16 * 8) = knew;
   if (rg == 1) *reinterpret_cast<uint4*>(Vw + l16 * 8) = vnew;
   if (tid == 32) { posb[slot] = t_now; accb[slot] = p_new; }
@@ -831,6 +852,184 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_group_mma_kernel(DecParams
   group_eq3_and_tail<R, G, kCaptured, kMmaRed>(p, inst, n, t_now, s_sc, Ns, s_red, mg, lg, knew, vnew, s_inv, s_key, &s_vic);
 }
 
+// --------------------------------------------------------------------------- //
+// The same step for shapes the kernels above do not take: head dimension 64 or 128 and any number
+// of query heads per KV head (the multi-query model the paper evaluates has 71 query heads over
+// one KV head of dimension 64).  CUDA cores; one 128-thread CTA per KV head.  The query heads are
+// taken eight at a time: every pass scores its heads against all live slots (the K and V rows of the
+// later passes come from L1 / L2), runs their softmaxes (a warp per head) and their Eq. 3, and
+// adds its heads' probabilities into one sum per entry; the tail then works on that sum as if it were
+// a single head's probability.
+// --------------------------------------------------------------------------- //
+constexpr int kLoopHeads = 8;     // query heads per pass
+
+template <int R, int D, bool kCaptured>
+__global__ void __launch_bounds__(DEC_THREADS) decode_group_loop_kernel(DecParams p, int G) {
+  constexpr int LPR = D / 8;                       // lanes per slot row
+  constexpr int RGN = DEC_THREADS / LPR;           // row groups
+  constexpr int GC = kLoopHeads;
+  extern __shared__ float dsm[];
+  const int Ns = p.Np + 4;
+  float* s_e = dsm;                                // [GC][Ns] scores of this pass's heads, then e^{s - m_g}
+  float* s_ps = s_e + GC * Ns;                     // [Ns] sum over all heads of their probabilities
+  float* s_red = s_ps + Ns;                        // [GC][RGN][D] partial numerators
+  __shared__ float s_ml[2][GC];
+  __shared__ float s_inv[GC];
+  __shared__ unsigned long long s_key[DEC_THREADS / 32];
+  __shared__ int s_vic;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int lp = tid % LPR, rg = tid / LPR, d = tid;
+  const bool own = D == DEC_THREADS || d < D;
+  const size_t inst = decode_instance(p);
+  const int N = p.N;
+  const int t_now = kCaptured ? __ldcg(p.a.tpos) : p.t;
+  int n = p.a.count[inst];
+  if (n < 0 || n > N) {
+    if (tid == 0) set_status(p.a.status, kStatusBounds, 1);
+    step_done<kCaptured>(p.a.tpos, p.t);
+    return;
+  }
+  const bool use_state = !(p.flags & LESS_NO_STATE);
+  const float scale = D == 64 ? 0.125f : 0.08838834764831845f;   // 1 / sqrt(D)
+  const __half* Kb = p.a.kslots + inst * (size_t)N * D;
+  const __half* Vb = p.a.vslots + inst * (size_t)N * D;
+  const uint4 knew = *reinterpret_cast<const uint4*>(p.k + inst * D + lp * 8);
+  const uint4 vnew = *reinterpret_cast<const uint4*>(p.v + inst * D + lp * 8);
+  for (int i = tid; i <= n; i += DEC_THREADS) s_ps[i] = 0.f;
+  float hcol[R], zr[R];
+#pragma unroll
+  for (int r = 0; r < R; ++r) hcol[r] = zr[r] = 0.f;
+
+  for (int g0 = 0; g0 < G; g0 += GC) {
+    const int gc = min(GC, G - g0);
+    float qf[GC][8];
+#pragma unroll
+    for (int g = 0; g < GC; ++g) {
+      if (g < gc) half8_to_float(*reinterpret_cast<const uint4*>(p.q + (inst * G + g0 + g) * D + lp * 8), qf[g]);
+      else
+#pragma unroll
+        for (int c = 0; c < 8; ++c) qf[g][c] = 0.f;
+    }
+    // ---- scores of this pass's heads against every live slot and the new pair ----
+    for (int r0 = 0; r0 <= n; r0 += RGN) {          // r0 is block-uniform: shuffles stay converged; row n = the new pair
+      const int r = r0 + rg;
+      float dot[GC];
+#pragma unroll
+      for (int g = 0; g < GC; ++g) dot[g] = 0.f;
+      if (r <= n) {
+        float kf[8];
+        half8_to_float(r < n ? *reinterpret_cast<const uint4*>(Kb + (size_t)r * D + lp * 8) : knew, kf);
+#pragma unroll
+        for (int g = 0; g < GC; ++g)
+#pragma unroll
+          for (int c = 0; c < 8; ++c) dot[g] = fmaf(qf[g][c], kf[c], dot[g]);
+      }
+#pragma unroll
+      for (int g = 0; g < GC; ++g) {
+#pragma unroll
+        for (int o = LPR / 2; o > 0; o >>= 1) dot[g] += __shfl_xor_sync(0xffffffffu, dot[g], o);
+        if (lp == 0 && r <= n) s_e[g * Ns + r] = dot[g] * scale;
+      }
+    }
+    __syncthreads();
+    // ---- per head: m_g, e_i = exp(s_i - m_g), l_g (a warp takes whole heads) ----
+    for (int g = warp; g < gc; g += DEC_THREADS / 32) {
+      float* sc = s_e + g * Ns;
+      float m = -INFINITY;
+      for (int i = lane; i <= n; i += 32) m = fmaxf(m, sc[i]);
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+      m = fmaxf(m, -80.f);
+      float lsum = 0.f;
+      for (int i = lane; i <= n; i += 32) {
+        const float e = __expf(sc[i] - m);
+        sc[i] = e;
+        lsum += e;
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) lsum += __shfl_xor_sync(0xffffffffu, lsum, o);   // fixed order
+      if (lane == 0) { s_ml[0][g] = m; s_ml[1][g] = lsum; }
+    }
+    __syncthreads();
+    // ---- u_g = sum e_{g,i} v_i over the live slots and the new pair ----
+    float u[GC][8];
+#pragma unroll
+    for (int g = 0; g < GC; ++g)
+#pragma unroll
+      for (int c = 0; c < 8; ++c) u[g][c] = 0.f;
+    for (int r = rg; r <= n; r += RGN) {
+      float vf[8];
+      half8_to_float(r < n ? *reinterpret_cast<const uint4*>(Vb + (size_t)r * D + lp * 8) : vnew, vf);
+#pragma unroll
+      for (int g = 0; g < GC; ++g) {
+        const float e = g < gc ? s_e[g * Ns + r] : 0.f;
+#pragma unroll
+        for (int c = 0; c < 8; ++c) u[g][c] = fmaf(e, vf[c], u[g][c]);
+      }
+    }
+#pragma unroll
+    for (int g = 0; g < GC; ++g)
+#pragma unroll
+      for (int c = 0; c < 8; ++c) s_red[(g * RGN + rg) * D + lp * 8 + c] = u[g][c];
+    __syncthreads();
+    // ---- Eq. 3 of each head over the KV head's shared H, z ----
+    if (g0 == 0 && use_state) {
+      wait_feature_maps<1>(p, 0);                    // general shapes never run with per-head counters: waits for the whole feature-map grid
+      if (own) {
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+          hcol[r] = p.a.H[(inst * R + r) * D + d];
+          zr[r] = p.a.z[inst * R + r];
+        }
+      }
+    }
+    if (own) {
+      for (int g = 0; g < gc; ++g) {
+        float num = 0.f;
+#pragma unroll
+        for (int j = 0; j < RGN; ++j) num += s_red[(g * RGN + j) * D + d];
+        const float lg = s_ml[1][g];
+        float den = lg;
+        if (use_state) {
+          const float em = __expf(-s_ml[0][g]);
+          const float* ph = p.a.phi_q + (inst * G + g0 + g) * R;
+          float lr = 0.f, lz = 0.f;
+#pragma unroll
+          for (int r = 0; r < R; ++r) {
+            const float f = __ldcg(ph + r);
+            lr = fmaf(f, hcol[r], lr);
+            lz = fmaf(f, zr[r], lz);
+          }
+          num = fmaf(em, lr, num);
+          den = fmaf(em, lz, den);
+        }
+        store_out(p, (inst * G + g0 + g) * D + d, num / den);
+        if (d == 0) s_inv[g] = 1.0f / ((p.flags & LESS_SCORE_NORM_SPARSE) ? lg : den);
+      }
+    }
+    __syncthreads();
+    // ---- this pass's share of the aggregated probabilities ----
+    for (int i = tid; i <= n; i += DEC_THREADS) {
+      float ps = s_ps[i];
+      for (int g = 0; g < gc; ++g) ps = fmaf(s_e[g * Ns + i], s_inv[g], ps);
+      s_ps[i] = ps;
+    }
+    __syncthreads();                                 // before the next pass rewrites s_e, s_ml, s_inv
+  }
+  const float one[1] = {1.0f};
+  decode_tail<R, 1, kCaptured, D>(p, inst, n, t_now, s_ps, Ns, one, hcol, knew, vnew, s_key, &s_vic);
+}
+
+template <int R, int D>
+static void* decode_loop_entry(bool captured) {
+  return captured ? (void*)decode_group_loop_kernel<R, D, true> : (void*)decode_group_loop_kernel<R, D, false>;
+}
+
+size_t decode_loop_smem_bytes(int Np, int D) {
+  return ((size_t)(kLoopHeads + 1) * (Np + 4) + (size_t)kLoopHeads * (DEC_THREADS / (D / 8)) * D) * 4;
+}
+
 size_t decode_smem_bytes(const Dims& d) {
   return (size_t)d.G * (d.Np + 4 + DEC_RG * kHeadDim) * 4;
 }
@@ -873,9 +1072,16 @@ int launch_decode(less_ctx* c, const void* q, const void* k, const void* v, void
   void* kern = d.R == 8 ? (captured ? (void*)decode_kernel<8, true> : (void*)decode_kernel<8, false>)
                         : (captured ? (void*)decode_kernel<16, true> : (void*)decode_kernel<16, false>);
   if (d.G > 1 && which == 3) smem = (size_t)d.G * (d.Np + 4 + kMmaRed * kHeadDim) * 4;
-  if (d.G == 2) kern = d.R == 8 ? decode_group_entry<8, 2>(captured, which) : decode_group_entry<16, 2>(captured, which);
-  if (d.G == 4) kern = d.R == 8 ? decode_group_entry<8, 4>(captured, which) : decode_group_entry<16, 4>(captured, which);
-  if (d.G == 8) kern = d.R == 8 ? decode_group_entry<8, 8>(captured, which) : decode_group_entry<16, 8>(captured, which);
+  int G_arg = d.G;
+  if (d.general) {
+    smem = decode_loop_smem_bytes(d.Np, d.D);
+    kern = d.D == 64 ? (d.R == 8 ? decode_loop_entry<8, 64>(captured) : decode_loop_entry<16, 64>(captured))
+                     : (d.R == 8 ? decode_loop_entry<8, 128>(captured) : decode_loop_entry<16, 128>(captured));
+    snprintf(c->variant[LESS_KERNEL_DECODE], sizeof c->variant[0], "decode_group_loop_kernel<%d, %d, %d>", d.R, d.D, (int)captured);
+  }
+  if (!d.general && d.G == 2) kern = d.R == 8 ? decode_group_entry<8, 2>(captured, which) : decode_group_entry<16, 2>(captured, which);
+  if (!d.general && d.G == 4) kern = d.R == 8 ? decode_group_entry<8, 4>(captured, which) : decode_group_entry<16, 4>(captured, which);
+  if (!d.general && d.G == 8) kern = d.R == 8 ? decode_group_entry<8, 8>(captured, which) : decode_group_entry<16, 8>(captured, which);
   if (smem > 48 * 1024 &&
       cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
     return fail_cuda("shared memory opt-in of decode_kernel");
@@ -893,7 +1099,7 @@ int launch_decode(less_ctx* c, const void* q, const void* k, const void* v, void
   const bool overlap = overlap_decode(c);
   cfg.attrs = attr;
   cfg.numAttrs = overlap ? 1 : 0;
-  void* args[] = {&p};
+  void* args[] = {&p, &G_arg};                         // the second argument is the general kernel's only
   if (cudaLaunchKernelExC(&cfg, kern, args) != cudaSuccess) return fail_cuda("launch of decode_kernel");
   return check_launch("decode_kernel");
 }

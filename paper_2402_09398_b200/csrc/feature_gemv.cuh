@@ -13,6 +13,7 @@ struct FmParams {
   const float* psi_scale; // [L, Hd, 2] or null
   float* out[2];          // phi_q [B, L, Hh[0], R], psi_k [B, L, Hh[1], R]
   int B, L, Hd, Rp;
+  int D;                  // head dimension (128; 64 on the general path)
   int Hh[2];              // heads of each map per layer: query heads for phi (Hd * group), KV heads for psi
   uint32_t* feat_flag;    // per-head counters to publish phi / psi through (psi's start at flag_stride), or null
   int flag_stride;

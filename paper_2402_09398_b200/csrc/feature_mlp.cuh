@@ -9,7 +9,8 @@ namespace less {
 constexpr int FM_THREADS = 256;
 constexpr int FM_BR = 4;
 
-// One MLP evaluation for `nb` rows already staged in xs (fp32 [FM_BR][128]).
+// One MLP evaluation for `nb` rows already staged in xs (fp32 [FM_BR][D], D = head dimension, a
+// multiple of FM_THREADS / (Rp / 8)).
 // part: [FM_THREADS / (Rp/8)][FM_BR][Rp] floats, hs: [FM_BR][Rp] floats.
 // Result: lanes < R of warp b (b < nb) return feature r = lane of row b; other threads 0.
 template <int R>
@@ -17,12 +18,12 @@ __device__ __forceinline__ float mlp_rows(const float* xs, float* part, float* h
                                           const __half* __restrict__ w1,
                                           const __half* __restrict__ w2,
                                           const __half* __restrict__ w3, float c1, float c2,
-                                          int Rp, bool is_psi) {
+                                          int Rp, bool is_psi, int D = kHeadDim) {
   const int tid = threadIdx.x;
   const int ncg = Rp >> 3;               // column groups of 8 hidden units
   const int ndg = FM_THREADS / ncg;      // groups along d
   const int cg = tid % ncg, dg = tid / ncg;
-  const int dper = kHeadDim / ndg;
+  const int dper = D / ndg;
   float acc[FM_BR][8];
 #pragma unroll
   for (int b = 0; b < FM_BR; ++b)
@@ -36,7 +37,7 @@ __device__ __forceinline__ float mlp_rows(const float* xs, float* part, float* h
     const int d = dg * dper + dd;
 #pragma unroll
     for (int b = 0; b < FM_BR; ++b) {
-      const float xv = xs[b * kHeadDim + d];
+      const float xv = xs[b * D + d];
 #pragma unroll
       for (int c = 0; c < 8; ++c) acc[b][c] = fmaf(xv, wf[c], acc[b][c]);
     }

@@ -13,10 +13,16 @@ namespace {
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+// head dimension 64, or a number of query heads per KV head other than 1, 2, 4, 8: the general path
+bool general_shape(const less_config* c) {
+  const int g = c->group > 1 ? c->group : 1;
+  return c->head_dim != kHeadDim || !(g == 1 || g == 2 || g == 4 || g == 8);
+}
+
 bool valid_config(const less_config* c) {
   if (!c) return false;
   if (c->batch < 1 || c->layers < 1 || c->heads < 1) return false;
-  if (c->head_dim != kHeadDim) return false;
+  if (c->head_dim != kHeadDim && c->head_dim != 64) return false;
   if (c->rank != 8 && c->rank != 16) return false;
   if (c->hidden < 64 || c->hidden > 1024 || (c->hidden & (c->hidden - 1))) return false;
   if (c->heavy < 0 || c->recent < 1) return false;
@@ -27,12 +33,18 @@ bool valid_config(const less_config* c) {
     return false;                                                                   // grid.y of the prompt kernels
   if (c->flags & ~(uint32_t)(LESS_SCORE_NORM_SPARSE | LESS_NO_STATE | LESS_POLICY_LAMBDA | LESS_POLICY_TOVA | LESS_WITH_PARALLEL_FORM | LESS_OUT_F16)) return false;
   if ((c->flags & LESS_POLICY_LAMBDA) && (c->flags & LESS_POLICY_TOVA)) return false;
-  if (c->group < 0 || c->group > 8 || (c->group & (c->group - 1))) return false;          // 0, 1, 2, 4, 8
+  if (c->group < 0 || c->group > 128) return false;
   if (c->group > 1 && (c->flags & LESS_POLICY_TOVA)) return false;                         // TOVA stays per head
-  // the decode kernel keeps one score per slot and query head in shared memory (227 KB per CTA)
-  if (c->group > 1 && (int64_t)c->group * ((((int64_t)c->heavy + c->recent + 3) & ~3) + 4 + 1024) * 4 > 227 * 1024)
-    return false;
-  if (c->group > 1 && c->hidden != 128 && c->hidden != 256 && c->hidden != 512) return false;   // tensor-core feature maps only
+  if (general_shape(c)) {
+    // decode only, on CUDA cores: eight heads' scores plus the aggregated ones per slot in shared memory
+    if (c->flags & LESS_WITH_PARALLEL_FORM) return false;
+    if ((int64_t)9 * ((((int64_t)c->heavy + c->recent + 3) & ~3) + 4 + 1024) * 4 > 227 * 1024) return false;
+  } else {
+    // the decode kernel keeps one score per slot and query head in shared memory (227 KB per CTA)
+    if (c->group > 1 && (int64_t)c->group * ((((int64_t)c->heavy + c->recent + 3) & ~3) + 4 + 1024) * 4 > 227 * 1024)
+      return false;
+    if (c->group > 1 && c->hidden != 128 && c->hidden != 256 && c->hidden != 512) return false;   // tensor-core feature maps only
+  }
   int64_t inst = (int64_t)c->batch * c->layers * c->heads;
   if (inst > (1 << 24)) return false;
   return true;
@@ -52,6 +64,7 @@ Dims make_dims(const less_config* c) {
   d.Np = (d.N + 3) & ~3;
   d.I = c->batch * c->layers * c->heads;
   d.G = c->group > 1 ? c->group : 1;
+  d.general = general_shape(c) ? 1 : 0;
   d.Sp = (c->max_prompt + 3) & ~3;
   d.Sbx = ((c->max_prompt + 255) & ~255) + 256;
   d.St = (c->max_prompt + 127) / 128;
@@ -249,6 +262,22 @@ int less_prefill(less_ctx* c, int32_t layer_begin, int32_t layer_count, int32_t 
       return LESS_ERR_MISALIGNED;
   }
   cudaStream_t s = (cudaStream_t)stream;
+  if (c->d.general) {
+    // general shapes decode from an empty cache: the prompt kernels are built for head dimension 128
+    // and 1, 2, 4 or 8 query heads per KV head.  prompt_len == 0 resets the layers (H_0 = 0, z_0 = 0).
+    if (prompt_len > 0) return LESS_ERR_INVALID_CONFIG;
+    const Dims& d = c->d;
+    for (int b = 0; b < d.B; ++b) {
+      const size_t i0 = ((size_t)b * d.L + layer_begin) * d.Hd, ni = (size_t)layer_count * d.Hd;
+      if (cudaMemsetAsync(c->a.H + i0 * d.R * d.D, 0, ni * d.R * d.D * 4, s) != cudaSuccess ||
+          cudaMemsetAsync(c->a.z + i0 * d.R, 0, ni * d.R * 4, s) != cudaSuccess ||
+          cudaMemsetAsync(c->a.count + i0, 0, ni * 4, s) != cudaSuccess)
+        return fail_cuda("reset of the layers");
+    }
+    if (cudaMemsetAsync(c->a.tpos, 0, 8, s) != cudaSuccess) return fail_cuda("reset of the position");
+    c->t = 0;
+    return LESS_OK;
+  }
   for (int lj0 = 0; lj0 < layer_count; lj0 += c->d.Lw) {
     int nl = layer_count - lj0 < c->d.Lw ? layer_count - lj0 : c->d.Lw;
     int rc = launch_prefill_group(c, layer_begin + lj0, nl, lj0, layer_count, prompt_len, Q, K, V,
@@ -263,7 +292,7 @@ int less_masked_attention(less_ctx* c, int32_t layer_begin, int32_t layer_count,
                           const void* Q, const void* K, const void* V, const int32_t* exact_until,
                           void* out, void* stream) {
   if (!c) return LESS_ERR_NULL_POINTER;
-  if (!(c->d.flags & LESS_WITH_PARALLEL_FORM) || c->d.G > 1) return LESS_ERR_INVALID_CONFIG;
+  if (!(c->d.flags & LESS_WITH_PARALLEL_FORM) || c->d.G > 1 || c->d.general) return LESS_ERR_INVALID_CONFIG;
   if (layer_begin < 0 || layer_count < 1 || layer_begin + layer_count > c->d.L)
     return LESS_ERR_BAD_LAYER_RANGE;
   if (seq_len < 0) return LESS_ERR_INVALID_CONFIG;

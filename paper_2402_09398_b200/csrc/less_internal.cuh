@@ -62,6 +62,7 @@ struct Dims {
   int32_t heavy, recent, N, Np; // slots; Np = N rounded up to a multiple of 4
   int32_t I;                    // instances (one per KV head)
   int32_t G;                    // query heads per KV head
+  int32_t general;              // head_dim 64 or a group size other than 1, 2, 4, 8: the general CUDA-core decode path
   int32_t Sp;                   // max_prompt rounded up to a multiple of 4
   int32_t Sbx;                  // max_prompt rounded up to a multiple of 256 (+256)
   int32_t St;                   // 128-row tiles of max_prompt

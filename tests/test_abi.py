@@ -42,11 +42,16 @@ def test_config_validation(B):
     good = B.less_arena_bytes(cfg())
     assert good > 0 and good % 256 == 0
     assert B.less_state_record_bytes(cfg()) == 16 + 16 * 8 + 2 * 16 * 128 * 2 + 16 * 8 * 4 + 8 * 128 * 4 + 8 * 4
-    for bad in (dict(head_dim=64), dict(rank=4), dict(recent=0), dict(heavy=-1), dict(hidden=500),
+    for bad in (dict(head_dim=32), dict(head_dim=64, flags=16), dict(group=129), dict(group=3, flags=8), dict(rank=4), dict(recent=0), dict(heavy=-1), dict(hidden=500),
                 dict(batch=0), dict(max_prefill_layers=3), dict(flags=64), dict(max_prompt=-1),
                 dict(heavy=32000, recent=769)):        # more than LESS_MAX_SLOTS = 32768
         assert B.less_arena_bytes(cfg(**bad)) == 0, bad
     assert B.less_arena_bytes(cfg(heavy=32000, recent=768)) > good
+    # general shapes: head dimension 64, any number of query heads per KV head up to 128
+    assert 0 < B.less_arena_bytes(cfg(head_dim=64)) < good
+    assert B.less_arena_bytes(cfg(head_dim=64, group=71)) > B.less_arena_bytes(cfg(head_dim=64))
+    assert B.less_arena_bytes(cfg(group=3)) > good
+    assert B.less_state_record_bytes(cfg(head_dim=64)) == 16 + 16 * 8 + 2 * 16 * 64 * 2 + 16 * 8 * 4 + 8 * 64 * 4 + 8 * 4
     # arena grows with slots and with the prefill workspace
     assert B.less_arena_bytes(cfg(heavy=80)) > good
     assert B.less_arena_bytes(cfg(max_prompt=4096)) > good

@@ -547,6 +547,37 @@ def test_grouped_query_heads_decode_from_empty(group, rank, flags, kernel, monke
     ctx.close()
 
 
+@pytest.mark.parametrize("head_dim,group,rank,batch,flags", [(64, 71, 8, 1, 0), (64, 71, 16, 2, 0), (64, 1, 8, 3, 0),
+                                                            (128, 3, 8, 2, 0), (64, 12, 16, 2, 4), (64, 5, 8, 2, 1),
+                                                            (64, 6, 8, 2, 2), (64, 1, 8, 2, 8), (128, 71, 8, 1, 0)])
+def test_general_shapes_decode_from_empty(head_dim, group, rank, batch, flags):
+    """Head dimension 64 and any number of query heads per KV head, up to the multi-query shape the
+    paper evaluates (Section 4: 71 query heads over one KV head of dimension 64): the general decode
+    kernel, teacher-forced against the grouped oracle from an empty cache through filling, the first
+    evictions and on; both policies, both normalisers, state off, TOVA with one head."""
+    import harness
+    from paper_2402_09398_b200 import binding
+    w = small(160 + group, batch=batch, layers=2, heads=2, head_dim=head_dim, prompt=0, steps=26, heavy=5, recent=6,
+              rank=rank, weight_std=0.1, group=group)
+    ctx, W = _setup(w, flags=flags, max_prompt=64)
+    ctx.reset()
+    inst = list(range(w.instances))
+    tf = (harness.GroupTeacherForced if group > 1 else harness.TeacherForced)(ctx, w, W, inst, flags=flags)
+    for s in range(w.steps):
+        tf.step(*wl.make_decode_inputs(w, s, DEV, prompt=0))
+    assert tf.evictions > 0 and ctx.poll_status() == 0
+    assert ctx.kernel_variant("decode").startswith("decode_group_loop_kernel")
+    # the prompt kernels are not built for these shapes: refused with an error code, nothing launched
+    Q, K, V = wl.make_prompt(w, 0, w.layers, DEV, prompt=16)
+    with pytest.raises(binding.LessError) as e:
+        ctx.prefill(Q, K, V, 0)
+    assert e.value.code == -1
+    ctx.reset()                                          # prompt_len == 0 still resets
+    rec = ctx.export_state(inst)
+    assert all(r["count"] == 0 and not r["H"].any() and not r["z"].any() for r in rec) and ctx.position == 0
+    ctx.close()
+
+
 @pytest.mark.parametrize("group,rank,prompt,flags", [(2, 8, 300, 0), (4, 16, 513, 0), (8, 8, 131, 0),
                                                      (4, 8, 300, 4), (2, 8, 700, 1), (2, 16, 260, 2)])
 def test_grouped_query_heads_prompt_and_decode(group, rank, prompt, flags):
@@ -575,10 +606,10 @@ def test_grouped_query_heads_prompt_and_decode(group, rank, prompt, flags):
 
 def test_grouped_query_heads_rejected_configurations(monkeypatch):
     from paper_2402_09398_b200 import binding
-    w = small(39, group=3)
+    w = small(39, group=129)
     W = wl.make_weights(w.with_(group=4), DEV)
     with pytest.raises(binding.LessError):
-        binding.from_workload(w, W, DEV)                       # not a power of two
+        binding.from_workload(w, W, DEV)                       # more query heads per KV head than the library takes
     with pytest.raises(binding.LessError):
         binding.from_workload(small(39, group=2), W, DEV, flags=8)   # TOVA stays per head
     with pytest.raises(binding.LessError):
