@@ -51,7 +51,8 @@ def parse_args(argv=None):
     ap.add_argument("--steps", type=int, default=20, help="steps per timed block")
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--config", type=int, default=0,
-                    help="workload id (1-4 decode; 5 = prompt compression, one layer per step); "
+                    help="workload id (1-4 decode; 5 = prompt compression, one layer per step; 6 = the multi-query "
+                         "shape of Section 4, context run); "
                          "0 = cfg3 as the headline plus sub-records for the other four")
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--cpu-seconds", type=float, default=12.0, help="budget of the CPU-baseline leg")
@@ -433,6 +434,7 @@ WORKLOAD_NAMES = {
     3: "cfg3 batched serving (B=64, 32 layers x 32 heads, prompt 1024, 102+102 slots, R=8)",
     4: "cfg4 long context (B=4, 40 layers x 40 heads, prompt 16384, 327+327 slots, R=16)",
     5: "cfg5 prefill compression (B=8, 32 heads, one layer per step, prompt 32768, 1638+1638 slots, R=16)",
+    6: "multi-query shape (B=64, 32 layers x 1 KV head x 71 query heads, D=64, 102+102 slots filled by decoding, R=8)",
 }
 PROMPT_METRIC = "prompt head-tokens/s (prompt scoring, selection, state build; one layer per step)"
 
@@ -479,6 +481,8 @@ def measure_decode(args, ranks, cfg_id, cpu_seconds):
     w = wl.CONFIGS[cfg_id]
     if args.batch:
         w = w.with_(batch=args.batch)
+    if w.cfg_id == 6:
+        cpu_seconds = 0
     if args.group > 1:
         if args.tova or w.heads % args.group:
             raise SystemExit("--group needs a head count it divides and is not defined for --tova")
@@ -507,14 +511,21 @@ def measure_decode(args, ranks, cfg_id, cpu_seconds):
 
     # replicas: every rank runs the whole workload on its own GPU, no collective in the path
     Wt = wl.make_weights(w, dev)
-    layers_per_call = max(1, min(w.layers, (1 << 30) // max(1, w.batch * w.heads * w.group * w.prompt * w.head_dim * 2)))
+    layers_per_call = max(1, min(w.layers, (1 << 30) // max(1, w.batch * w.heads * w.group * w.prompt * w.head_dim * 2))) \
+        if w.prompt else 1
     ctx = binding.from_workload(w_run, Wt, dev, max_prefill_layers=layers_per_call, flags=flags)
     t_pre0 = time.perf_counter()
-    for l0 in range(0, w.layers, layers_per_call):
+    for l0 in range(0, w.layers if w.prompt else 0, layers_per_call):
         n = min(layers_per_call, w.layers - l0)
         Q, Kp, V = wl.make_prompt(w, l0, n, dev)
         ctx.prefill(Q, Kp, V, l0)
         del Q, Kp, V
+    if not w.prompt:                       # no prompt phase for this shape: the cache fills by decoding
+        ctx.reset()
+        fill = [wl.make_decode_inputs(w, s, dev) for s in range(4)]
+        for s in range(w_run.slots + 4):
+            ctx.decode_step(*fill[s % 4])
+        del fill
     torch.cuda.synchronize()
     t_prefill = time.perf_counter() - t_pre0
 
@@ -596,7 +607,7 @@ def measure_decode(args, ranks, cfg_id, cpu_seconds):
     st_e2e = block_stats(e2e_times, K_steps)
     status = ctx.poll_status()
     if status != 0:
-        raise RuntimeError(f"device status {status}")
+        raise RuntimeError(f"device status {status} (where-code {ctx.status_where()})")
 
     rec = None
     if ranks.rank == 0:
@@ -605,7 +616,7 @@ def measure_decode(args, ranks, cfg_id, cpu_seconds):
         value = units * world / (ms_step * 1e-3)
         e2e_value = units * world / (st_e2e["ms_per_step"] * 1e-3)
         peak, _, peak_kind = peaks()
-        n_live = min(w_run.slots, w.prompt + W_steps)
+        n_live = min(w_run.slots, w.prompt + W_steps) if w.prompt else w_run.slots
         evicting = not args.full_cache
         kb = {"feature_map": feature_map_bytes(w, args.no_state),
               "decode": decode_bytes(w, n_live, evicting, args.no_state, out_bytes)}
@@ -713,7 +724,7 @@ def measure_prefill(args, ranks, cpu_seconds, steps=None):
     torch.cuda.synchronize()
     prof = ctx.profile_read()
     ctx.profile(False)
-    variants = {k: ctx.kernel_variant(k) for k in ("rowstat", "colsum", "psi", "build", "attn_out")}
+    variants = {k: ctx.kernel_variant(k) for k in ("rowstat", "colsum", "attn_out", "select", "psi", "gather", "build", "finalize")}
     # end to end: the layer's Q, K, V come from pinned host memory, the kept positions go back
     hq, hk, hv = (torch.empty(t.shape, dtype=torch.float16).pin_memory() for t in (Q, Kp, V))
     hq.copy_(Q); hk.copy_(Kp); hv.copy_(V)
@@ -729,8 +740,9 @@ def measure_prefill(args, ranks, cpu_seconds, steps=None):
         ctx.export_state(inst0[:1])                    # device -> host read of one instance's kept set
     torch.cuda.synchronize()
     ms_e2e = 1e3 * (time.perf_counter() - tw0) / n_e2e
-    if ctx.poll_status() != 0:
-        raise RuntimeError("device status")
+    status = ctx.poll_status()
+    if status != 0:
+        raise RuntimeError(f"device status {status} (where-code {ctx.status_where()})")
     ms_e2e = ranks.reduce_max([ms_e2e])[0]
     rec = None
     if ranks.rank == 0:
@@ -842,8 +854,9 @@ def measure_masked(args, ranks):
         hout.copy_(out, non_blocking=True)
     torch.cuda.synchronize()
     ms_e2e = 1e3 * (time.perf_counter() - tw0) / n_e2e
-    if ctx.poll_status() != 0:
-        raise RuntimeError("device status")
+    status = ctx.poll_status()
+    if status != 0:
+        raise RuntimeError(f"device status {status} (where-code {ctx.status_where()})")
     ms_e2e = ranks.reduce_max([ms_e2e])[0]
     rec = None
     if ranks.rank == 0:

@@ -30,7 +30,10 @@
  *     LESS_FEATURE_STAGES=n (cap on the feature kernels' weight ring),
  *     LESS_GROUP_KERNEL=rows (grouped query heads: the CUDA-core decode kernel instead of
  *     the one with its two contractions as warp-level tensor-core products),
- *     LESS_FEATURE_CTAS=n (cap on the persistent CTAs of the tensor-core feature kernels).
+ *     LESS_FEATURE_CTAS=n (cap on the persistent CTAs of the tensor-core feature kernels),
+ *     LESS_HEAD_COUNTERS=1 (with more instances than fit the GPU at once and more than 8 batch rows:
+ *     the decode kernel starts behind the feature-map kernel and each of its CTAs waits for its own
+ *     head's feature maps through a per-head counter; measured neutral, off by default).
  */
 #ifndef LESS_B200_H
 #define LESS_B200_H

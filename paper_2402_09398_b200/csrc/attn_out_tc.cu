@@ -259,7 +259,7 @@ int launch_attn_out_tc(less_ctx* c, const PfParams& p, int G, cudaStream_t s) {
   if (cudaFuncSetAttribute(attn_out_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
     return fail_cuda("shared memory opt-in of attn_out_tc_kernel");
   const int tiles = (p.S + AO_TILE - 1) / AO_TILE;
-  LaunchScope scope(c, LESS_KERNEL_ATTN_OUT, s);
+  LaunchScope scope(c, LESS_KERNEL_ATTN_OUT, s, "attn_out_tc_kernel");
   attn_out_tc_kernel<<<dim3(tiles, G * p.grp), AO_THREADS, smem, s>>>(tq, tk, tv, p);
   return check_launch("attn_out_tc_kernel");
 }

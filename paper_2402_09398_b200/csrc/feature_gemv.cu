@@ -252,7 +252,7 @@ static int launch_one(less_ctx* c, const FmParams& p, cudaStream_t s) {
   cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, GV_THREADS, smem);
   if (per_sm < 1) per_sm = 1;
   const int grid = items < sms * per_sm ? items : sms * per_sm;
-  LaunchScope scope(c, LESS_KERNEL_FEATURE_MAP, s);
+  LaunchScope scope(c, LESS_KERNEL_FEATURE_MAP, s, "feature_gemv_kernel");
   kern<<<grid, GV_THREADS, smem, s>>>(p, nchunk_b, items, c->a.status);
   return check_launch("feature_gemv_kernel");
 }

@@ -617,7 +617,7 @@ int launch_feature_tc(less_ctx* c, const FmParams& p_in, cudaStream_t s) {
   // With the overlap on, the ring gives up stages so that decode CTAs of the same step fit beside
   // this kernel's CTA on every SM (at these batch sizes the kernel is bound by its epilogue, not
   // by the weight stream: three stages feed it).
-  const int cap_l = c->feature_stages >= 2 ? c->feature_stages : (c->pdl ? 3 : FT_MAX_STAGES);   // d.I is not known to be small here either way: three stages feed this kernel
+  const int cap_l = c->feature_stages >= 2 ? c->feature_stages : (c->pdl && (c->head_counters || d.I <= 8 * c->sms) ? 3 : FT_MAX_STAGES);
   if (gm.nstage > cap_l) gm.nstage = cap_l;
   if (gm.nstage < 2) return LESS_ERR_INVALID_CONFIG;
   const uint32_t need = 2u * gm.npad + 16u;
@@ -649,17 +649,22 @@ int launch_feature_tc(less_ctx* c, const FmParams& p_in, cudaStream_t s) {
   const int grid = gm.items < sms ? gm.items : sms;
   const int nt = d.B <= 1 ? 1 : d.B <= 2 ? 2 : d.B <= 4 ? 4 : 8;
   // Per-head counters, so that any number of decode CTAs can follow this kernel as programmatic
-  // dependents.  Direct calls only (a captured step would replay a stale target).  Not needed
-  // while every decode CTA fits on the GPU at once, and not used behind the small-batch kernel with
-  // more instances than that: that kernel is bound by its weight stream, and successive waves of
-  // decode CTAs take so much of the bandwidth from it that the feature maps they wait for arrive
-  // later than without the overlap (measured, 4 x 1600 heads x 654 slots: 533 us per step against 486).
+  // dependents, each waiting for its own head's feature maps only.  Off unless LESS_HEAD_COUNTERS is
+  // set: measured on 64 x 1024 heads x 204 slots the overlap gains nothing (1.337 ms per step with it,
+  // 1.325 ms without; feature grids of 24 to 148 CTAs all within 1 %) - at that size the decode kernel
+  // is bound by what the SMs can keep in flight, not by HBM, so every SM-microsecond the feature
+  // kernel takes is lost to it wherever it is scheduled - and with grouped query heads it costs
+  // (8192 KV heads x 2 query heads: 1.02 ms against 0.86 ms).  Direct calls only (a captured step
+  // would replay a stale target).  Never behind the small-batch kernel with more instances than fit
+  // the GPU at once: that kernel is bound by its weight stream, and successive waves of decode CTAs
+  // take so much of the bandwidth from it that the feature maps they wait for arrive later than
+  // without the overlap (measured, 4 x 1600 heads x 654 slots: 533 us per step against 486).
   // Every flagged launch adds the same number of writer warps to every head's counter, so the target
   // is one running total.
   cudaStreamCaptureStatus capturing = cudaStreamCaptureStatusNone;
   cudaStreamIsCapturing(s, &capturing);
   const bool many = d.I > 8 * c->sms;
-  if (capturing == cudaStreamCaptureStatusNone && c->pdl && many && d.B > 8) {
+  if (capturing == cudaStreamCaptureStatusNone && c->pdl && c->head_counters && many && d.B > 8) {
     uint32_t writers = 0;
     if (d.B <= 8) writers = (uint32_t)(nt * d.R + 31) / 32;
     else

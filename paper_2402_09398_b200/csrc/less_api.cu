@@ -197,6 +197,7 @@ int less_create(const less_config* cfg, const less_weights* w, void* arena, size
   c->tm_w_ok = false;
   memset(c->variant, 0, sizeof c->variant);
   c->feature_ctas = 0;
+  c->head_counters = getenv("LESS_HEAD_COUNTERS") != nullptr;
   if (const char* e = getenv("LESS_FEATURE_CTAS")) c->feature_ctas = atoi(e);
   c->profile = false;
   c->feature_path = 2;

@@ -88,6 +88,7 @@ struct less_ctx {
   int score_path;      // prompt scoring: 1 tensor cores, 0 CUDA cores (LESS_SCORE_KERNEL=plain)
   int feature_path;    // feature-map kernel: 2 tensor cores, 1 streaming GEMV, 0 plain (LESS_FEATURE_KERNEL)
   int group_path;      // grouped decode kernel: 2 on CUDA cores (LESS_GROUP_KERNEL=rows), else with warp-level mma
+  bool head_counters;  // decode CTAs follow the large-batch feature kernel head by head (LESS_HEAD_COUNTERS=1; off by default)
   int feature_ctas;    // cap on the feature kernels' persistent CTAs (LESS_FEATURE_CTAS), 0 = one per multiprocessor
   bool flags_this_step;     // the step's feature-map launch publishes per-head counters (set by its launcher)
   uint32_t flag_target[2];  // counter value of a head once this step's phi / psi are written

@@ -662,7 +662,7 @@ int launch_masked_form(less_ctx* c, int layer0, int nl, int lj0, int layer_count
     return fail_cuda("tensor maps of Q / K / V");
   const size_t smem = (size_t)MF_TILE_BYTES + MF_STAGES * MF_STAGE_BYTES + MF_OP_BYTES + MF_STAGES * MF_OP_BYTES +
                       MF_EU_SLOTS * MF_EU_BYTES + sizeof(MfShared) + 1024;
-  LaunchScope scope(c, LESS_KERNEL_MASKED_OUT, s);
+  LaunchScope scope(c, LESS_KERNEL_MASKED_OUT, s, "masked_out_tc_kernel");
   if (d.R == 8) {
     if (cudaFuncSetAttribute(masked_out_tc_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
       return fail_cuda("shared memory opt-in of masked_out_tc_kernel");

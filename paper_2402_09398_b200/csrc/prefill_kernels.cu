@@ -471,11 +471,11 @@ int launch_prefill_group(less_ctx* c, int layer0, int nl, int lj0, int layer_cou
       if (rc != LESS_OK) return rc;
     } else {
       {
-        LaunchScope scope(c, LESS_KERNEL_ROWSTAT, s);
+        LaunchScope scope(c, LESS_KERNEL_ROWSTAT, s, "rowstat_kernel");
         rowstat_kernel<<<dim3(tiles, G), PF_TILE, 0, s>>>(p);
       }
       if (h2o) {
-        LaunchScope scope(c, LESS_KERNEL_COLSUM, s);
+        LaunchScope scope(c, LESS_KERNEL_COLSUM, s, "colsum_kernel");
         colsum_kernel<<<dim3(tiles, G), PF_TILE, 0, s>>>(p);
       }
     }
@@ -483,16 +483,16 @@ int launch_prefill_group(less_ctx* c, int layer0, int nl, int lj0, int layer_cou
       const int rc = launch_attn_out_tc(c, p, G, s);
       if (rc != LESS_OK) return rc;
     } else if (attn_out) {
-      LaunchScope scope(c, LESS_KERNEL_ATTN_OUT, s);
+      LaunchScope scope(c, LESS_KERNEL_ATTN_OUT, s, "attn_out_kernel");
       attn_out_kernel<<<dim3((S + AO_ROWS - 1) / AO_ROWS, G), PF_TILE, 0, s>>>(p);
     }
   }
   if (S > 0 && (d.flags & LESS_POLICY_TOVA)) {
-    LaunchScope scope(c, LESS_KERNEL_COLSUM, s);
+    LaunchScope scope(c, LESS_KERNEL_COLSUM, s, "lastrow_kernel");
     lastrow_kernel<<<G, LR_THREADS, 0, s>>>(p);
   }
   {
-    LaunchScope scope(c, LESS_KERNEL_SELECT, s);
+    LaunchScope scope(c, LESS_KERNEL_SELECT, s, "select_kernel");
     select_kernel<<<G, SEL_THREADS, 0, s>>>(p);
   }
   const size_t smem = (size_t)(FM_BR * kHeadDim + mlp_smem_floats(d.Rp)) * 4;
@@ -502,7 +502,7 @@ int launch_prefill_group(less_ctx* c, int layer0, int nl, int lj0, int layer_cou
     const int rc = launch_psi_state_tc(c, p, G, s);
     if (rc != LESS_OK) return rc;
   } else if (nsplit > 0 && use_state) {
-    LaunchScope scope(c, LESS_KERNEL_PSI, s);
+    LaunchScope scope(c, LESS_KERNEL_PSI, s, "psi_kernel");
     if (d.R == 8) {
       cudaFuncSetAttribute(psi_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
       psi_kernel<8><<<dim3(nsplit, G), FM_THREADS, smem, s>>>(p);
@@ -512,7 +512,7 @@ int launch_prefill_group(less_ctx* c, int layer0, int nl, int lj0, int layer_cou
     }
   }
   if (S > 0) {
-    LaunchScope scope(c, LESS_KERNEL_GATHER, s);
+    LaunchScope scope(c, LESS_KERNEL_GATHER, s, "gather_kernel");
     const int gx = (min(S, d.N) + 63) / 64 > 0 ? (min(S, d.N) + 63) / 64 : 1;
     if (d.R == 8) gather_kernel<8><<<dim3(gx, G), GA_THREADS, 0, s>>>(p);
     else gather_kernel<16><<<dim3(gx, G), GA_THREADS, 0, s>>>(p);
@@ -522,7 +522,7 @@ int launch_prefill_group(less_ctx* c, int layer0, int nl, int lj0, int layer_cou
     if (rc != LESS_OK) return rc;
   }
   {
-    LaunchScope scope(c, LESS_KERNEL_FINALIZE, s);
+    LaunchScope scope(c, LESS_KERNEL_FINALIZE, s, "finalize_kernel");
     if (d.R == 8) finalize_kernel<8><<<G, kHeadDim, 0, s>>>(p);
     else finalize_kernel<16><<<G, kHeadDim, 0, s>>>(p);
   }

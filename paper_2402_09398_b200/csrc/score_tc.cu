@@ -409,11 +409,11 @@ int launch_score_tc(less_ctx* c, const PfParams& p, int G, cudaStream_t s, bool 
       cudaFuncSetAttribute(colsum_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem2) != cudaSuccess)
     return fail_cuda("shared memory opt-in of the scoring kernels");
   {
-    LaunchScope scope(c, LESS_KERNEL_ROWSTAT, s);
+    LaunchScope scope(c, LESS_KERNEL_ROWSTAT, s, "rowstat_tc_kernel");
     rowstat_tc_kernel<<<dim3(tiles, G * p.grp), RS_THREADS, smem1, s>>>(tq_res, tk, p);   // one row of CTAs per query head
   }
   if (with_column_sums) {
-    LaunchScope scope(c, LESS_KERNEL_COLSUM, s);
+    LaunchScope scope(c, LESS_KERNEL_COLSUM, s, "colsum_tc_kernel");
     colsum_tc_kernel<<<dim3(tiles, G), CS_THREADS, smem2, s>>>(tq, tk_res, p);
   }
   return check_launch("scoring kernels");

@@ -200,7 +200,7 @@ int launch_state_tc(less_ctx* c, const PfParams& p, int G, cudaStream_t s) {
   if (!make_tmap_f16_2d(&tmap_v, p.V, rows, kHeadDim, kHeadDim * 2, ST_TILE)) return fail_cuda("tensor map of V");
   const int NB = 2 * d.R;
   const size_t smem = (size_t)ST_STAGES * (ST_VBYTES + ST_TILE * NB * 2) + 4096 + sizeof(StShared) + 1024;
-  LaunchScope scope(c, LESS_KERNEL_BUILD, s);
+  LaunchScope scope(c, LESS_KERNEL_BUILD, s, "state_tc_kernel");
   if (d.R == 8) {
     cudaFuncSetAttribute(state_tc_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     state_tc_kernel<8><<<dim3(p.nsplit, G), ST_THREADS, smem, s>>>(tmap_v, p);

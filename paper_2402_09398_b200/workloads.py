@@ -65,6 +65,10 @@ CONFIGS: Dict[int, Workload] = {
                 heavy_rule="bernoulli", heavy_param=0.005, sink_prefix=4),
     5: Workload(5, 8, 32, 32, 128, 32768, 0, _half_budget(0.05, 32768), _half_budget(0.05, 32768), 16,
                 heavy_rule="none"),
+    # context shape, not one of the five benchmark configurations: the multi-query model the paper
+    # evaluates (Section 4: 32 layers, 71 query heads over one KV head of dimension 64, context 2048
+    # -> 102 + 102 slots at 10 %), batch 64, decoding from an empty cache
+    6: Workload(6, 64, 32, 1, 64, 0, 128, 102, 102, 8, heavy_rule="bernoulli", heavy_param=0.01, group=71),
 }
 
 

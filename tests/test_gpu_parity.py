@@ -331,12 +331,14 @@ def test_decode_many_instances_and_ragged_slots(overlap, monkeypatch):
 @pytest.mark.parametrize("batch,layers,heads,rank,ctas", [(4, 4, 80, 8, 0), (20, 2, 32, 16, 0), (70, 1, 19, 8, 0),
                                                           (20, 2, 32, 8, 16)])
 def test_decode_follows_the_feature_kernel_head_by_head(batch, layers, heads, rank, ctas, monkeypatch):
-    """More instances than can wait on the GPU at once (> 8 per SM): the decode kernel starts as a
-    programmatic dependent of the feature-map kernel and every CTA waits only for the counters of
-    its own head's phi and psi; CTAs are numbered head-major.  Small-batch and large-batch feature
-    kernels, several token tiles (batch 70), a feature grid cut to 16 CTAs.  Teacher-forced parity,
-    then free-running steps back to back must equal, bit for bit, a context without the overlap."""
+    """More instances than can wait on the GPU at once (> 8 per SM), per-head counters switched on:
+    behind the large-batch feature kernel the decode kernel starts as a programmatic dependent and
+    every CTA waits only for the counters of its own head's phi and psi, CTAs numbered head-major
+    (batches 20 and 70: one and two token tiles; a feature grid cut to 16 CTAs); behind the small-batch
+    kernel (batch 4) the step stays serial.  Teacher-forced parity, then free-running steps back to
+    back must equal, bit for bit, a context without the overlap."""
     import harness
+    monkeypatch.setenv("LESS_HEAD_COUNTERS", "1")
     if ctas:
         monkeypatch.setenv("LESS_FEATURE_CTAS", str(ctas))
     w = small(130 + batch, batch=batch, layers=layers, heads=heads, prompt=40, steps=3, heavy=9, recent=9,
