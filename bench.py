@@ -325,47 +325,91 @@ class ClockSampler:
 # --------------------------------------------------------------------------- #
 # CPU oracle timing (cpu_baseline leg and --impl reference)
 # --------------------------------------------------------------------------- #
-def oracle_rate(w, seconds, records=None, instances=None, W=None, max_instances=16):
-    """Times oracle decode steps on a bounded sample of instances.  With
-    `records` (states exported from the GPU) the oracle starts from them, else it
-    runs its own prompt phase first (untimed).  Returns (head-tokens/s, cores, text, steps, s)."""
+def _oracle_worker(job):
+    """One worker process of the CPU baseline (no torch, no CUDA in here): builds its share of the
+    sampled instances from their records and times oracle decode steps, one numpy thread."""
     from threadpoolctl import threadpool_limits
+    from oracle import less_oracle as lo
+    D, R, heavy, recent, weights, records, q, k, v, seconds = job
+    with threadpool_limits(limits=1):
+        orcs = []
+        for wts, r in zip(weights, records):
+            o = lo.LessInstance(D, R, heavy, recent, *lo.make_mlp_maps(*wts))
+            o.import_state(r["pos"], r["K"], r["V"], r["acc"], r["H"], r["z"], r["t"])
+            orcs.append(o)
+        units, steps, t0 = 0, 0, time.perf_counter()
+        while True:                                   # the step inputs are used round-robin until the time is up
+            s = steps % q.shape[0]
+            for i, o in enumerate(orcs):
+                o.decode(q[s, i], k[s, i], v[s, i])
+            units += len(orcs)
+            steps += 1
+            if time.perf_counter() - t0 > seconds or steps >= 100000:
+                break
+        return units, time.perf_counter() - t0, steps
+
+
+def oracle_rate(w, seconds, records=None, instances=None, W=None, max_instances=16, max_steps=64):
+    """Times oracle decode steps on a bounded sample of instances (`seconds` of CPU work in total), the
+    instances spread over worker processes on the host's cores (the oracle itself is untouched: one numpy
+    thread per instance; the sampled steps' inputs are reused round-robin until the time is up).  With
+    `records` (states exported from the GPU) the oracle starts from them, else it runs its own prompt
+    phase first (untimed).  Returns (head-tokens/s, cores, text, steps, s)."""
+    import multiprocessing as mp
+    from concurrent.futures import ProcessPoolExecutor
+    import numpy as np
     from oracle import less_oracle as lo
     from paper_2402_09398_b200 import workloads as wl
     if W is None:
         W = wl.make_weights(w, "cpu")
-    with threadpool_limits(limits=1):
-        if instances is None:
-            instances = list(range(0, w.instances, max(1, w.instances // max_instances)))[:max_instances]
-        orcs = []
-        prompt_cache = {}
-        for n, inst in enumerate(instances):
-            b, layer, head = wl.instance_coords(w, inst)
-            wts = [W[k][layer, head].double().cpu().numpy() for k in
-                   ("w_phi1", "w_phi2", "w_psi1", "w_psi2", "w_psi3")]
+    if instances is None:
+        instances = list(range(0, w.instances, max(1, w.instances // max_instances)))[:max_instances]
+    weights, prompt_cache = [], {}
+    built = records is None
+    if built:
+        records = []
+    for n, inst in enumerate(instances):
+        b, layer, head = wl.instance_coords(w, inst)
+        wts = [W[k][layer, head].double().cpu().numpy() for k in ("w_phi1", "w_phi2", "w_psi1", "w_psi2", "w_psi3")]
+        weights.append(wts)
+        if built:
+            if layer not in prompt_cache:
+                prompt_cache = {layer: wl.make_prompt(w, layer, 1, "cpu")}
+            Q, K, V = prompt_cache[layer]
             o = lo.LessInstance(w.head_dim, w.rank, w.heavy, w.recent, *lo.make_mlp_maps(*wts))
-            if records is not None:
-                r = records[n]
-                o.import_state(r["pos"], r["K"], r["V"], r["acc"], r["H"], r["z"], r["t"])
-            else:
-                if layer not in prompt_cache:
-                    prompt_cache = {layer: wl.make_prompt(w, layer, 1, "cpu")}
-                Q, K, V = prompt_cache[layer]
-                o.prefill(*(t[b, 0, head].double().numpy() for t in (Q, K, V)))
-            orcs.append(o)
-        units, t_used, step = 0, 0.0, 0
-        while t_used < seconds and step < max(w.steps, 1):
-            q, k, v = wl.make_decode_inputs(w, step, "cpu")
-            q, k, v = (t.reshape(-1, w.head_dim).double().numpy() for t in (q, k, v))
-            t0 = time.perf_counter()
-            for inst, o in zip(instances, orcs):
-                o.decode(q[inst], k[inst], v[inst])
-            t_used += time.perf_counter() - t0
-            units += len(instances)
-            step += 1
-    sample = (f"{len(instances)} of {w.instances} instances x {step} decode steps "
-              f"({'GPU-exported' if records is not None else 'oracle-prefilled'} state), fp64 numpy, 1 thread")
-    return units / t_used, 1, sample, step, t_used
+            o.prefill(*(t[b, 0, head].double().numpy() for t in (Q, K, V)))
+            records.append({"pos": o.pos, "K": o.K, "V": o.V, "acc": o.acc, "H": o.H, "z": o.z, "t": o.t})
+    # decode inputs of the sampled instances only (the generators draw whole steps)
+    nsteps = max(1, min(max_steps, w.steps if w.steps else max_steps))
+    idx = np.asarray(instances)
+    qs, ks, vs = [], [], []
+    for s in range(nsteps):
+        q, k, v = wl.make_decode_inputs(w, s, "cpu")
+        qs.append(q.reshape(-1, w.head_dim)[idx].double().numpy())
+        ks.append(k.reshape(-1, w.head_dim)[idx].double().numpy())
+        vs.append(v.reshape(-1, w.head_dim)[idx].double().numpy())
+    q, k, v = np.stack(qs), np.stack(ks), np.stack(vs)               # [steps, instances, D]
+    try:
+        avail = len(os.sched_getaffinity(0))
+    except AttributeError:
+        avail = os.cpu_count() or 1
+    cores = max(1, min(avail, len(instances), 16))
+    shares = [list(range(c, len(instances), cores)) for c in range(cores)]
+    # `seconds` = CPU work in total: every worker runs for its share of it
+    jobs = [(w.head_dim, w.rank, w.heavy, w.recent, [weights[i] for i in sh], [records[i] for i in sh],
+             q[:, sh], k[:, sh], v[:, sh], seconds / cores) for sh in shares]
+    if cores == 1:
+        results = [_oracle_worker(jobs[0])]
+    else:
+        with ProcessPoolExecutor(max_workers=cores, mp_context=mp.get_context("spawn")) as pool:
+            results = list(pool.map(_oracle_worker, jobs))
+    units = sum(r[0] for r in results)
+    t_used = max(r[1] for r in results)
+    steps = max(r[2] for r in results)
+    sample = (f"{len(instances)} of {w.instances} instances x {steps} decode steps "
+              f"({'oracle-prefilled' if built else 'GPU-exported'} state), fp64 numpy, one thread per instance, "
+              f"{cores} worker process(es) on {avail} available core(s)")
+    return units / t_used, cores, sample, steps, t_used
 
 
 def oracle_prompt_rate(w, prompt, seconds):
@@ -414,7 +458,7 @@ def run_reference(args):
     # batch rows: the per-instance work does not depend on the batch)
     n_inst = 8
     w_run = w.with_(batch=min(w.batch, 2), steps=args.steps + args.warmup)
-    rate, cores, sample, steps_done, t_used = oracle_rate(w_run, seconds=90.0, max_instances=n_inst)
+    rate, cores, sample, steps_done, t_used = oracle_rate(w_run, seconds=60.0, max_instances=n_inst)
     sample = sample.replace(f"of {w_run.instances} instances", f"of {w.instances} instances")
     line = {
         "impl": "reference", "metric": METRIC, "value": rate, "unit": UNIT, "n_gpus": 0,
@@ -661,7 +705,7 @@ def measure_decode(args, ranks, cfg_id, cpu_seconds):
             instances = list(range(0, w.instances, max(1, w.instances // 16)))[:16]
             recs = ctx.export_state(instances)
             Wc = {k: v.cpu() for k, v in Wt.items()}
-            rate, cores, sample, _, _ = oracle_rate(w.with_(steps=max(w.steps, 64)), cpu_seconds, recs, instances, Wc)
+            rate, cores, sample, _, _ = oracle_rate(w, cpu_seconds, recs, instances, Wc)
             rec["cpu_baseline"] = {"value": rate, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample}
     ctx.close()
     del ctx, base, out, Wt
@@ -931,8 +975,25 @@ def run_b200(args):
                     raise
             if ranks.rank == 0:
                 subs[f"cfg{cfg}"] = {k: r[k] for k in SUB_RECORD_KEYS if k in r} if "error" not in r else r
+        # context: the same decode kernel over a full cache (nothing evicted) and with the sparse policy
+        # alone (Baseline+), on the batch-1 Llama-2-7B shape
+        import copy
+        context = {}
+        for name, kw in (("cfg2_full_cache", {"full_cache": True}), ("cfg2_baseline_plus", {"no_state": True})):
+            a = copy.copy(args)
+            for k, v in kw.items():
+                setattr(a, k, v)
+            try:
+                r = measure_decode(a, ranks, 2, 0)
+            except Exception as e:                    # noqa: BLE001 - reported in the line
+                r = {"error": repr(e)}
+                if ranks.world > 1:
+                    raise
+            if ranks.rank == 0:
+                context[name] = {k: r[k] for k in SUB_RECORD_KEYS if k in r} if "error" not in r else r
         if ranks.rank == 0:
             line["configs"] = subs
+            line["context"] = context
     if ranks.rank == 0:
         print(json.dumps(line))
     ranks.close()

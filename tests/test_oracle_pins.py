@@ -89,8 +89,9 @@ def test_budget_fraction_of_prompt():
     assert 2 * lo.budget_from_fraction(0.05, 2048) == lo.h2o_token_count(10, 2048)
     assert lo.budget_from_fraction(0.02, 16384) == 327
     assert lo.budget_from_fraction(0.05, 32768) == 1638
+    assert wl.CONFIGS[6].slots == lo.h2o_token_count(10, 2048)   # Table 1: Falcon at 10 % of its 2048 context
     for cid, w in wl.CONFIGS.items():      # the product's host logic agrees
-        frac = {1: None, 2: 0.05, 3: 0.10, 4: 0.02, 5: 0.05}[cid]
+        frac = {2: 0.05, 3: 0.10, 4: 0.02, 5: 0.05}.get(cid)      # 1: fixed slots; 6: the multi-query context shape
         if frac is not None:
             assert w.heavy == w.recent == lo.budget_from_fraction(frac, w.prompt)
 
