@@ -42,7 +42,11 @@ struct AoShared {
   uint64_t k_full[AO_STAGES], k_empty[AO_STAGES];
   uint64_t v_full[AO_STAGES], v_empty[AO_STAGES];
   uint64_t s_full[AO_SBUFS], pv_done[AO_SBUFS];
-  uint64_t p_full;
+  // One hand-over barrier per S / P buffer.  A single barrier with one phase per tile is not enough: the
+  // epilogue warps may run up to three tiles ahead of the P V issuer, and two phases completing unseen
+  // make a parity wait mistake the current phase for the one it wants (it then waits for a tile that
+  // never comes); per buffer, a warp cannot arrive for the buffer's next use before this use is consumed.
+  uint64_t p_full[AO_SBUFS];
   uint64_t o_full;
   uint32_t tmem_base;
   int abort;
@@ -83,8 +87,8 @@ __global__ void __launch_bounds__(AO_THREADS) attn_out_tc_kernel(const __grid_co
     for (int s = 0; s < AO_SBUFS; ++s) {
       mbar_init(&sh->s_full[s], 1);
       mbar_init(&sh->pv_done[s], 1);
+      mbar_init(&sh->p_full[s], AO_EPI_WARPS);
     }
-    mbar_init(&sh->p_full, AO_EPI_WARPS);
     mbar_init(&sh->o_full, 1);
     sh->abort = *reinterpret_cast<volatile int32_t*>(status) != 0;
     mbar_fence_init();
@@ -164,10 +168,10 @@ __global__ void __launch_bounds__(AO_THREADS) attn_out_tc_kernel(const __grid_co
     if (lane == 0) {
       constexpr uint32_t idesc_o = idesc_f16(AO_TILE, kHeadDim, 0, 1);  // A = P (tensor memory), B = V (N-major)
       const uint64_t bd_vring = smem_desc(smem_u32(ring) + AO_TILE_BYTES, AO_TILE_BYTES / 2, 1024, kLayoutSw128);
-      uint32_t s2 = 0, vph = 0, b2 = 0;
+      uint32_t s2 = 0, vph = 0, b2 = 0, b2ph = 0;
       for (int t = 0; t < ntile; ++t) {
         wait_or_give_up(&sh->v_full[s2], vph, abortp, status, 109);
-        wait_or_give_up(&sh->p_full, t & 1, abortp, status, 104);
+        wait_or_give_up(&sh->p_full[b2], b2ph, abortp, status, 104);
         if (*abortp) break;
         tc_fence_after_sync();
         const uint64_t bv0 = bd_vring + (uint64_t)(s2 * (AO_STAGE_BYTES >> 4));
@@ -179,7 +183,7 @@ __global__ void __launch_bounds__(AO_THREADS) attn_out_tc_kernel(const __grid_co
         mma_commit(&sh->v_empty[s2]);
         mma_commit(&sh->pv_done[b2]);
         if (++s2 == AO_STAGES) { s2 = 0; vph ^= 1; }
-        if (++b2 == AO_SBUFS) b2 = 0;
+        if (++b2 == AO_SBUFS) { b2 = 0; b2ph ^= 1; }
       }
       mma_commit(&sh->o_full);
     }
@@ -220,7 +224,7 @@ __global__ void __launch_bounds__(AO_THREADS) attn_out_tc_kernel(const __grid_co
       tmem_st16(lane_addr + b * AO_TILE + part * 32, pk);
       tmem_st_wait();
       tc_fence_before_sync();
-      mbar_arrive_warp(&sh->p_full);
+      mbar_arrive_warp(&sh->p_full[b]);
       if (++b == AO_SBUFS) { b = 0; bph ^= 1; }
     }
     // ---- the finished rows: O[row][32 columns of this warp] ----

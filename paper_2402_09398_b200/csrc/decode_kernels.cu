@@ -337,7 +337,7 @@ __device__ __forceinline__ void decode_tail(const DecParams& p, size_t inst, int
 // numerators in shared memory (s_red [G][NRED][128]), then the common second half of the step.
 template <int R, int G, bool kCaptured, int NRED>
 __device__ __forceinline__ void group_eq3_and_tail(const DecParams& p, size_t inst, int n, int t_now, const float* s_sc,
-                                                   int Ns, const float* s_red, const float (&mg)[G], const float (&lg)[G],
+                                                   int Ns, const float* s_red, const float* s_m, const float* s_l,
                                                    const uint4& knew, const uint4& vnew, float* s_inv,
                                                    unsigned long long* s_key, int* s_vic) {
   const int tid = threadIdx.x, d = tid;
@@ -358,9 +358,10 @@ __device__ __forceinline__ void group_eq3_and_tail(const DecParams& p, size_t in
     float num = 0.f;
 #pragma unroll
     for (int j = 0; j < NRED; ++j) num += s_red[(g * NRED + j) * kHeadDim + d];
-    float den = lg[g];
+    const float lg = s_l[g];                         // the heads' maxima and sums stay in shared memory: registers
+    float den = lg;                                  // decide how many of these CTAs an SM holds
     if (use_state) {
-      const float em = __expf(-mg[g]);
+      const float em = __expf(-s_m[g]);
       const float* ph = p.a.phi_q + (inst * G + g) * R;
       float lr = 0.f, lz = 0.f;
 #pragma unroll
@@ -373,7 +374,7 @@ __device__ __forceinline__ void group_eq3_and_tail(const DecParams& p, size_t in
       den = fmaf(em, lz, den);
     }
     store_out(p, (inst * G + g) * kHeadDim + d, num / den);
-    if (tid == 0) s_inv[g] = 1.0f / ((p.flags & LESS_SCORE_NORM_SPARSE) ? lg[g] : den);
+    if (tid == 0) s_inv[g] = 1.0f / ((p.flags & LESS_SCORE_NORM_SPARSE) ? lg : den);
   }
   __syncthreads();
   float inv[G];
@@ -585,7 +586,7 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_group_rows_kernel(DecParam
   __syncthreads();
 
   // ---- per head: m_g, e_i = exp(s_i - m_g), l_g ----
-  float mg[G], lg[G];
+  __shared__ float s_ml[2][G];
 #pragma unroll
   for (int g = 0; g < G; ++g) {
     float* sc = s_sc + g * Ns;
@@ -599,8 +600,8 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_group_rows_kernel(DecParam
       sc[i] = e;
       lsum += e;
     }
-    mg[g] = m;
-    lg[g] = block_sum(lsum, s_small);
+    lsum = block_sum(lsum, s_small);
+    if (tid == 0) { s_ml[0][g] = m; s_ml[1][g] = lsum; }
   }
 
   // ---- u_g = sum e_{g,i} v_i (each V row is read once) ----
@@ -636,7 +637,7 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_group_rows_kernel(DecParam
     for (int c = 0; c < 8; ++c) s_red[(g * DEC_RG + rg) * kHeadDim + l16 * 8 + c] = u[g][c];
   __syncthreads();
 
-  group_eq3_and_tail<R, G, kCaptured, DEC_RG>(p, inst, n, t_now, s_sc, Ns, s_red, mg, lg, knew, vnew, s_inv, s_key, &s_vic);
+  group_eq3_and_tail<R, G, kCaptured, DEC_RG>(p, inst, n, t_now, s_sc, Ns, s_red, s_ml[0], s_ml[1], knew, vnew, s_inv, s_key, &s_vic);
 }
 
 // The same step with the two contractions on the tensor cores.  With G query heads per KV head the
@@ -747,9 +748,8 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_group_mma_kernel(DecParams
   __syncthreads();
 
   // ---- per head: m_g, e_i = exp(s_i - m_g), l_g ----
-  float mg[G], lg[G];
+  __shared__ float s_ml[2][G];
   if (G >= DEC_THREADS / 32) {                      // a warp takes whole heads: no block barrier per head
-    __shared__ float s_ml[2][G];
     for (int g = warp; g < G; g += DEC_THREADS / 32) {
       float* sc = s_sc + g * Ns;
       float m = -INFINITY;
@@ -768,8 +768,6 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_group_mma_kernel(DecParams
       if (lane == 0) { s_ml[0][g] = m; s_ml[1][g] = lsum; }
     }
     __syncthreads();
-#pragma unroll
-    for (int g = 0; g < G; ++g) { mg[g] = s_ml[0][g]; lg[g] = s_ml[1][g]; }
   } else {                                          // fewer heads than warps: the whole CTA works on each
 #pragma unroll
     for (int g = 0; g < G; ++g) {
@@ -784,8 +782,8 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_group_mma_kernel(DecParams
         sc[i] = e;
         lsum += e;
       }
-      mg[g] = m;
-      lg[g] = block_sum(lsum, s_small);
+      lsum = block_sum(lsum, s_small);
+      if (tid == 0) { s_ml[0][g] = m; s_ml[1][g] = lsum; }
     }
   }
 
@@ -849,7 +847,7 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_group_mma_kernel(DecParams
   }
   __syncthreads();
 
-  group_eq3_and_tail<R, G, kCaptured, kMmaRed>(p, inst, n, t_now, s_sc, Ns, s_red, mg, lg, knew, vnew, s_inv, s_key, &s_vic);
+  group_eq3_and_tail<R, G, kCaptured, kMmaRed>(p, inst, n, t_now, s_sc, Ns, s_red, s_ml[0], s_ml[1], knew, vnew, s_inv, s_key, &s_vic);
 }
 
 // --------------------------------------------------------------------------- //

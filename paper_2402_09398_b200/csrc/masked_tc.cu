@@ -219,7 +219,7 @@ struct MfShared {
   uint64_t eu_full[MF_EU_SLOTS], eu_empty[MF_EU_SLOTS];   // exact_until of the key tile
   uint64_t s_full[2], s_free[2];                      // S buffer (and L) written / read
   uint64_t l_free;                                    // the single L buffer has been read
-  uint64_t p_full;
+  uint64_t p_full[2];                                 // per S / P buffer: one barrier for both would let two phases pass unseen
   uint64_t pv_done[2];                                // the P V that read the S buffer's P has completed
   uint64_t o_full;
   uint32_t tmem_base;
@@ -280,7 +280,8 @@ __global__ void __launch_bounds__(MF_THREADS) masked_out_tc_kernel(const __grid_
       mbar_init(&sh->pv_done[s], 1);
     }
     mbar_init(&sh->l_free, MF_EPI_WARPS);
-    mbar_init(&sh->p_full, MF_EPI_WARPS);
+    mbar_init(&sh->p_full[0], MF_EPI_WARPS);
+    mbar_init(&sh->p_full[1], MF_EPI_WARPS);
     mbar_init(&sh->o_full, 1);
     sh->abort = *reinterpret_cast<volatile int32_t*>(status) != 0;
     mbar_fence_init();
@@ -406,7 +407,7 @@ __global__ void __launch_bounds__(MF_THREADS) masked_out_tc_kernel(const __grid_
       for (int t = 0; t < nlive; ++t) {                // t counts the live tiles of the second sweep
         const int bt = (nlive + t) & 1;                  // the S buffer this tile's P lives in
         wait_or_give_up(&sh->v_full[s2], vph, abortp, status, 117);
-        wait_or_give_up(&sh->p_full, t & 1, abortp, status, 118);
+        wait_or_give_up(&sh->p_full[bt], (t >> 1) & 1, abortp, status, 118);   // the buffer's (t / 2)-th P
         if (*abortp) break;
         tc_fence_after_sync();
         const uint64_t bv0 = bd_vring + (uint64_t)(s2 * (MF_STAGE_BYTES >> 4));
@@ -537,7 +538,7 @@ __global__ void __launch_bounds__(MF_THREADS) masked_out_tc_kernel(const __grid_
         tmem_st16(lane_addr + b * MF_TILE + part * 32, pk);
         tmem_st_wait();
         tc_fence_before_sync();
-        mbar_arrive_warp(&sh->p_full);
+        mbar_arrive_warp(&sh->p_full[b]);
       }
       if (b ^= 1, b == 0) bph ^= 1;
       ++u;
