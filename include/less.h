@@ -112,10 +112,9 @@ typedef struct less_config {
                                * keeps one score per slot and query head in shared memory).
                                * General shapes - head_dim 64, or any other group up to 128 (Section 4's
                                * multi-query model has 71 query heads over one KV head of dimension 64) -
-                               * decode on CUDA cores from an empty cache: less_prefill accepts only
-                               * prompt_len == 0 (reset) and less_masked_attention is not available for them;
-                               * 9 * (heavy + recent + 1028) * 4 bytes <= 227 KB, no LESS_POLICY_TOVA with
-                               * group > 1.  Anything else is LESS_ERR_INVALID_CONFIG */
+                               * run on CUDA-core kernels (prompt phase and decode); less_masked_attention
+                               * is not available for them; 9 * (heavy + recent + 1028) * 4 bytes <= 227 KB,
+                               * no LESS_POLICY_TOVA with group > 1.  Anything else is LESS_ERR_INVALID_CONFIG */
 } less_config;
 
 /* Per-head feature-map weights (Eq. 1, Eq. 2), device, fp16, row-major, no biases:

@@ -263,22 +263,6 @@ int less_prefill(less_ctx* c, int32_t layer_begin, int32_t layer_count, int32_t 
       return LESS_ERR_MISALIGNED;
   }
   cudaStream_t s = (cudaStream_t)stream;
-  if (c->d.general) {
-    // general shapes decode from an empty cache: the prompt kernels are built for head dimension 128
-    // and 1, 2, 4 or 8 query heads per KV head.  prompt_len == 0 resets the layers (H_0 = 0, z_0 = 0).
-    if (prompt_len > 0) return LESS_ERR_INVALID_CONFIG;
-    const Dims& d = c->d;
-    for (int b = 0; b < d.B; ++b) {
-      const size_t i0 = ((size_t)b * d.L + layer_begin) * d.Hd, ni = (size_t)layer_count * d.Hd;
-      if (cudaMemsetAsync(c->a.H + i0 * d.R * d.D, 0, ni * d.R * d.D * 4, s) != cudaSuccess ||
-          cudaMemsetAsync(c->a.z + i0 * d.R, 0, ni * d.R * 4, s) != cudaSuccess ||
-          cudaMemsetAsync(c->a.count + i0, 0, ni * 4, s) != cudaSuccess)
-        return fail_cuda("reset of the layers");
-    }
-    if (cudaMemsetAsync(c->a.tpos, 0, 8, s) != cudaSuccess) return fail_cuda("reset of the position");
-    c->t = 0;
-    return LESS_OK;
-  }
   for (int lj0 = 0; lj0 < layer_count; lj0 += c->d.Lw) {
     int nl = layer_count - lj0 < c->d.Lw ? layer_count - lj0 : c->d.Lw;
     int rc = launch_prefill_group(c, layer_begin + lj0, nl, lj0, layer_count, prompt_len, Q, K, V,

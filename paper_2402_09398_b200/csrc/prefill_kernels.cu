@@ -14,12 +14,16 @@ namespace less {
 
 constexpr int PF_TILE = 128;   // rows (or columns) per CTA, one per thread
 constexpr int PF_KT = 32;      // rows of the other operand staged per iteration
-constexpr float kScale = 0.08838834764831845f;   // 1 / sqrt(128)
+// The CUDA-core kernels take the head dimension D as a template argument (128, or 64 on the general
+// path) and any number of query heads per KV head (PfParams::grp).
+template <int D>
+__device__ __forceinline__ float inv_sqrt_d() { return D == 64 ? 0.125f : 0.08838834764831845f; }
 
-__device__ __forceinline__ float dot128(const float* x, const __half* row) {
+template <int D>
+__device__ __forceinline__ float dot_row(const float* x, const __half* row) {
   float s = 0.f;
 #pragma unroll
-  for (int c8 = 0; c8 < 16; ++c8) {
+  for (int c8 = 0; c8 < D / 8; ++c8) {
     float f[8];
     half8_to_float(*reinterpret_cast<const uint4*>(row + c8 * 8), f);
 #pragma unroll
@@ -28,39 +32,42 @@ __device__ __forceinline__ float dot128(const float* x, const __half* row) {
   return s;
 }
 
-__device__ __forceinline__ void load_row128(float* x, const __half* row) {
+template <int D>
+__device__ __forceinline__ void load_row(float* x, const __half* row) {
 #pragma unroll
-  for (int c8 = 0; c8 < 16; ++c8)
+  for (int c8 = 0; c8 < D / 8; ++c8)
     half8_to_float(__ldg(reinterpret_cast<const uint4*>(row + c8 * 8)), x + c8 * 8);
 }
 
-// ---- P1: row statistics -------------------------------------------------- //
+// ---- P1: row statistics (one grid row per query head) --------------------- //
+template <int D>
 __global__ void __launch_bounds__(PF_TILE) rowstat_kernel(PfParams p) {
-  __shared__ __align__(16) __half ks[PF_KT][kHeadDim];
-  const int g = blockIdx.y, i0 = blockIdx.x * PF_TILE, tid = threadIdx.x;
-  const InstMap im = map_instance(p, g);
+  constexpr int CH = D / 8;
+  __shared__ __align__(16) __half ks[PF_KT][D];
+  const int gq = blockIdx.y, i0 = blockIdx.x * PF_TILE, tid = threadIdx.x;
+  const QueryMap qm = map_query(p, gq);
   const int i = i0 + tid;
   const bool live = i < p.S;
-  float q[kHeadDim];
-  if (live) load_row128(q, p.Q + (im.in_row0 + i) * kHeadDim);
+  float q[D];
+  if (live) load_row<D>(q, p.Q + (qm.q_row0 + i) * D);
   else {
 #pragma unroll
-    for (int c = 0; c < kHeadDim; ++c) q[c] = 0.f;
+    for (int c = 0; c < D; ++c) q[c] = 0.f;
   }
   float m = -INFINITY, l = 0.f;
   const int jend = min(p.S, i0 + PF_TILE);
   for (int j0 = 0; j0 < jend; j0 += PF_KT) {
-    for (int e = tid; e < PF_KT * 16; e += PF_TILE) {
-      const int r = e >> 4, c = e & 15;
+    for (int e = tid; e < PF_KT * CH; e += PF_TILE) {
+      const int r = e / CH, c = e % CH;
       uint4 v = make_uint4(0, 0, 0, 0);
-      if (j0 + r < p.S) v = __ldg(reinterpret_cast<const uint4*>(p.K + (im.in_row0 + j0 + r) * kHeadDim) + c);
+      if (j0 + r < p.S) v = __ldg(reinterpret_cast<const uint4*>(p.K + (qm.kv_row0 + j0 + r) * D) + c);
       reinterpret_cast<uint4*>(&ks[r][0])[c] = v;
     }
     __syncthreads();
     if (live) {
       const int jmax = min(PF_KT, i - j0 + 1);
       for (int jj = 0; jj < jmax; ++jj) {
-        const float s = dot128(q, &ks[jj][0]) * kScale;
+        const float s = dot_row<D>(q, &ks[jj][0]) * inv_sqrt_d<D>();
         if (s > m) { l = l * __expf(m - s) + 1.f; m = s; }
         else l += __expf(s - m);
       }
@@ -68,63 +75,71 @@ __global__ void __launch_bounds__(PF_TILE) rowstat_kernel(PfParams p) {
     __syncthreads();
   }
   if (live) {
-    p.a.ws_m[(size_t)g * p.Sp + i] = m;
-    p.a.ws_invl[(size_t)g * p.Sp + i] = 1.0f / l;
+    p.a.ws_m[(size_t)gq * p.Sp + i] = m;
+    p.a.ws_invl[(size_t)gq * p.Sp + i] = 1.0f / l;
   }
 }
 
-// ---- P2: column sums ------------------------------------------------------ //
+// ---- P2: column sums, over the rows of all query heads of the KV head ------- //
+template <int D>
 __global__ void __launch_bounds__(PF_TILE) colsum_kernel(PfParams p) {
-  __shared__ __align__(16) __half qs[PF_KT][kHeadDim];
+  constexpr int CH = D / 8;
+  __shared__ __align__(16) __half qs[PF_KT][D];
   __shared__ float ms[PF_KT], ls[PF_KT];
   const int g = blockIdx.y, j0 = blockIdx.x * PF_TILE, tid = threadIdx.x;
   const InstMap im = map_instance(p, g);
   const int j = j0 + tid;
   const bool live = j < p.S;
-  float k[kHeadDim];
-  if (live) load_row128(k, p.K + (im.in_row0 + j) * kHeadDim);
+  float k[D];
+  if (live) load_row<D>(k, p.K + (im.in_row0 + j) * D);
   else {
 #pragma unroll
-    for (int c = 0; c < kHeadDim; ++c) k[c] = 0.f;
+    for (int c = 0; c < D; ++c) k[c] = 0.f;
   }
   float acc = 0.f;
-  for (int i0 = j0; i0 < p.S; i0 += PF_KT) {       // j0 is a multiple of PF_KT
-    for (int e = tid; e < PF_KT * 16; e += PF_TILE) {
-      const int r = e >> 4, c = e & 15;
-      uint4 v = make_uint4(0, 0, 0, 0);
-      if (i0 + r < p.S) v = __ldg(reinterpret_cast<const uint4*>(p.Q + (im.in_row0 + i0 + r) * kHeadDim) + c);
-      reinterpret_cast<uint4*>(&qs[r][0])[c] = v;
-    }
-    if (tid < PF_KT) {
-      const bool ok = i0 + tid < p.S;
-      ms[tid] = ok ? p.a.ws_m[(size_t)g * p.Sp + i0 + tid] : 0.f;
-      ls[tid] = ok ? p.a.ws_invl[(size_t)g * p.Sp + i0 + tid] : 0.f;
-    }
-    __syncthreads();
-    if (live) {
-      const int iimax = min(PF_KT, p.S - i0);
-      for (int ii = max(0, j - i0); ii < iimax; ++ii) {
-        const float s = dot128(k, &qs[ii][0]) * kScale;
-        acc += __expf(s - ms[ii]) * ls[ii];
+  for (int qg = 0; qg < p.grp; ++qg) {
+    const int gq = g * p.grp + qg;
+    const size_t q_row0 = map_query(p, gq).q_row0;
+    for (int i0 = j0; i0 < p.S; i0 += PF_KT) {       // j0 is a multiple of PF_KT
+      for (int e = tid; e < PF_KT * CH; e += PF_TILE) {
+        const int r = e / CH, c = e % CH;
+        uint4 v = make_uint4(0, 0, 0, 0);
+        if (i0 + r < p.S) v = __ldg(reinterpret_cast<const uint4*>(p.Q + (q_row0 + i0 + r) * D) + c);
+        reinterpret_cast<uint4*>(&qs[r][0])[c] = v;
       }
+      if (tid < PF_KT) {
+        const bool ok = i0 + tid < p.S;
+        ms[tid] = ok ? p.a.ws_m[(size_t)gq * p.Sp + i0 + tid] : 0.f;
+        ls[tid] = ok ? p.a.ws_invl[(size_t)gq * p.Sp + i0 + tid] : 0.f;
+      }
+      __syncthreads();
+      if (live) {
+        const int iimax = min(PF_KT, p.S - i0);
+        for (int ii = max(0, j - i0); ii < iimax; ++ii) {
+          const float s = dot_row<D>(k, &qs[ii][0]) * inv_sqrt_d<D>();
+          acc += __expf(s - ms[ii]) * ls[ii];
+        }
+      }
+      __syncthreads();
     }
-    __syncthreads();
   }
   if (live) p.a.ws_acc[(size_t)g * p.Sp + j] = acc;
 }
 
-// ---- optional prompt attention output ------------------------------------- //
+// ---- optional prompt attention output (one grid row per query head) -------- //
 constexpr int AO_ROWS = 8;
+template <int D>
 __global__ void __launch_bounds__(PF_TILE) attn_out_kernel(PfParams p) {
-  __shared__ float qs[AO_ROWS][kHeadDim];
-  __shared__ __align__(16) __half ks[PF_KT][kHeadDim];
-  __shared__ __align__(16) __half vs[PF_KT][kHeadDim];
+  constexpr int CH = D / 8;
+  __shared__ float qs[AO_ROWS][D];
+  __shared__ __align__(16) __half ks[PF_KT][D];
+  __shared__ __align__(16) __half vs[PF_KT][D];
   __shared__ float ps[AO_ROWS][PF_KT];
-  const int g = blockIdx.y, i0 = blockIdx.x * AO_ROWS, tid = threadIdx.x;
-  const InstMap im = map_instance(p, g);
-  for (int e = tid; e < AO_ROWS * kHeadDim; e += PF_TILE) {
-    const int r = e / kHeadDim, c = e % kHeadDim;
-    qs[r][c] = (i0 + r < p.S) ? __half2float(p.Q[(im.in_row0 + i0 + r) * kHeadDim + c]) : 0.f;
+  const int gq = blockIdx.y, i0 = blockIdx.x * AO_ROWS, tid = threadIdx.x;
+  const QueryMap qm = map_query(p, gq);
+  for (int e = tid; e < AO_ROWS * D; e += PF_TILE) {
+    const int r = e / D, c = e % D;
+    qs[r][c] = (i0 + r < p.S) ? __half2float(p.Q[(qm.q_row0 + i0 + r) * D + c]) : 0.f;
   }
   float o[AO_ROWS];
 #pragma unroll
@@ -132,12 +147,12 @@ __global__ void __launch_bounds__(PF_TILE) attn_out_kernel(PfParams p) {
   const int jend = min(p.S, i0 + AO_ROWS);
   for (int j0 = 0; j0 < jend; j0 += PF_KT) {
     __syncthreads();
-    for (int e = tid; e < PF_KT * 16; e += PF_TILE) {
-      const int r = e >> 4, c = e & 15;
+    for (int e = tid; e < PF_KT * CH; e += PF_TILE) {
+      const int r = e / CH, c = e % CH;
       uint4 kv = make_uint4(0, 0, 0, 0), vv = kv;
       if (j0 + r < p.S) {
-        kv = __ldg(reinterpret_cast<const uint4*>(p.K + (im.in_row0 + j0 + r) * kHeadDim) + c);
-        vv = __ldg(reinterpret_cast<const uint4*>(p.V + (im.in_row0 + j0 + r) * kHeadDim) + c);
+        kv = __ldg(reinterpret_cast<const uint4*>(p.K + (qm.kv_row0 + j0 + r) * D) + c);
+        vv = __ldg(reinterpret_cast<const uint4*>(p.V + (qm.kv_row0 + j0 + r) * D) + c);
       }
       reinterpret_cast<uint4*>(&ks[r][0])[c] = kv;
       reinterpret_cast<uint4*>(&vs[r][0])[c] = vv;
@@ -148,38 +163,43 @@ __global__ void __launch_bounds__(PF_TILE) attn_out_kernel(PfParams p) {
       const int i = i0 + r, j = j0 + jj;
       float pr = 0.f;
       if (i < p.S && j <= i) {
-        const float s = dot128(&qs[r][0], &ks[jj][0]) * kScale;
-        pr = __expf(s - p.a.ws_m[(size_t)g * p.Sp + i]) * p.a.ws_invl[(size_t)g * p.Sp + i];
+        const float s = dot_row<D>(&qs[r][0], &ks[jj][0]) * inv_sqrt_d<D>();
+        pr = __expf(s - p.a.ws_m[(size_t)gq * p.Sp + i]) * p.a.ws_invl[(size_t)gq * p.Sp + i];
       }
       ps[r][jj] = pr;
     }
     __syncthreads();
-    for (int jj = 0; jj < PF_KT; ++jj) {
-      const float vv = __half2float(vs[jj][tid]);
+    if (tid < D) {
+      for (int jj = 0; jj < PF_KT; ++jj) {
+        const float vv = __half2float(vs[jj][tid]);
 #pragma unroll
-      for (int r = 0; r < AO_ROWS; ++r) o[r] = fmaf(ps[r][jj], vv, o[r]);
+        for (int r = 0; r < AO_ROWS; ++r) o[r] = fmaf(ps[r][jj], vv, o[r]);
+      }
     }
   }
+  if (tid < D) {
 #pragma unroll
-  for (int r = 0; r < AO_ROWS; ++r)
-    if (i0 + r < p.S) p.attn_out[(im.in_row0 + i0 + r) * kHeadDim + tid] = o[r];
+    for (int r = 0; r < AO_ROWS; ++r)
+      if (i0 + r < p.S) p.attn_out[(qm.q_row0 + i0 + r) * D + tid] = o[r];
+  }
 }
 
 // ---- TOVA: the last prompt query's attention probabilities ------------------- //
 // p_j = softmax_j( q_{S-1} . k_j / sqrt(D) ) over the whole prompt, into ws_acc.  One CTA per
 // instance: scores, block maximum, exponentials and their block sum, normalisation in place.
 constexpr int LR_THREADS = 1024;
+template <int D>
 __global__ void __launch_bounds__(LR_THREADS) lastrow_kernel(PfParams p) {
-  __shared__ float qs[kHeadDim];
+  __shared__ float qs[D];
   __shared__ float red[LR_THREADS / 32];
   const int g = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const InstMap im = map_instance(p, g);
   float* pr = p.a.ws_acc + (size_t)g * p.Sp;
-  if (tid < kHeadDim) qs[tid] = __half2float(p.Q[(im.in_row0 + p.S - 1) * kHeadDim + tid]);
+  if (tid < D) qs[tid] = __half2float(p.Q[(im.in_row0 + p.S - 1) * D + tid]);
   __syncthreads();
   float m = -INFINITY;
   for (int j = tid; j < p.S; j += LR_THREADS) {
-    const float s = dot128(qs, p.K + (im.in_row0 + j) * kHeadDim) * kScale;
+    const float s = dot_row<D>(qs, p.K + (im.in_row0 + j) * D) * inv_sqrt_d<D>();
     pr[j] = s;
     m = fmaxf(m, s);
   }
@@ -340,30 +360,30 @@ __global__ void __launch_bounds__(SEL_THREADS) select_kernel(PfParams p) {
 }
 
 // ---- P5: psi(k_j) of every prompt token (CUDA-core MLP) -------------------- //
-template <int R>
+template <int R, int D>
 __global__ void __launch_bounds__(FM_THREADS) psi_kernel(PfParams p) {
   extern __shared__ float bsm[];
-  float* xs = bsm;                              // [FM_BR][128]
-  float* hs = xs + FM_BR * kHeadDim;
+  float* xs = bsm;                              // [FM_BR][D]
+  float* hs = xs + FM_BR * D;
   float* part = hs + FM_BR * p.Rp;
   const int split = blockIdx.x, g = blockIdx.y, tid = threadIdx.x;
   const InstMap im = map_instance(p, g);
   const int jbeg = split * p.split_tokens, jend = min(p.S, jbeg + p.split_tokens);
   float c1 = 1.f, c2 = 1.f;
   if (p.psi_scale) { c1 = p.psi_scale[im.lh * 2]; c2 = p.psi_scale[im.lh * 2 + 1]; }
-  const __half* w1 = p.w_psi1 + (size_t)im.lh * kHeadDim * p.Rp;
+  const __half* w1 = p.w_psi1 + (size_t)im.lh * D * p.Rp;
   const __half* w2 = p.w_psi2 + (size_t)im.lh * p.Rp * R;
   const __half* w3 = p.w_psi3 + (size_t)im.lh * R * R;
   float* psi = p.a.ws_psi + (size_t)g * p.Sp * R;
   float pmax = 0.f;
   for (int j0 = jbeg; j0 < jend; j0 += FM_BR) {
     const int nb = min(FM_BR, jend - j0);
-    for (int e = tid; e < FM_BR * kHeadDim; e += FM_THREADS) {
-      const int b = e / kHeadDim, d = e % kHeadDim;
-      xs[e] = b < nb ? __half2float(p.K[(im.in_row0 + j0 + b) * kHeadDim + d]) : 0.f;
+    for (int e = tid; e < FM_BR * D; e += FM_THREADS) {
+      const int b = e / D, d = e % D;
+      xs[e] = b < nb ? __half2float(p.K[(im.in_row0 + j0 + b) * D + d]) : 0.f;
     }
     __syncthreads();
-    const float r = mlp_rows<R>(xs, part, hs, nb, w1, w2, w3, c1, c2, p.Rp, true);
+    const float r = mlp_rows<R>(xs, part, hs, nb, w1, w2, w3, c1, c2, p.Rp, true, D);
     const int warp = tid >> 5, lane = tid & 31;
     if (warp < nb && lane < R) {
       psi[(size_t)(j0 + warp) * R + lane] = r;
@@ -376,15 +396,16 @@ __global__ void __launch_bounds__(FM_THREADS) psi_kernel(PfParams p) {
 
 // ---- P4: kept rows go to their slots (K, V, position, score, psi) ----------- //
 constexpr int GA_THREADS = 256;
-template <int R>
+template <int R, int D>
 __global__ void __launch_bounds__(GA_THREADS) gather_kernel(PfParams p) {
+  constexpr int CH = D / 8;                          // 16-byte chunks per row
   const int g = blockIdx.y, tid = threadIdx.x;
   const InstMap im = map_instance(p, g);
   const bool use_state = !(p.flags & LESS_NO_STATE);
   const int32_t* slot_of = p.a.ws_slot + (size_t)g * p.Sp;
   const float* acc = p.a.ws_acc + (size_t)g * p.Sp;
   const float* psi = p.a.ws_psi + (size_t)g * p.Sp * R;
-  // 32 threads per token: 16 move the K row, 16 the V row
+  // 32 threads per token: CH move the K row, CH the V row
   const int sub = tid & 31;
   for (int j = blockIdx.x * (GA_THREADS / 32) + (tid >> 5); j < p.S; j += gridDim.x * (GA_THREADS / 32)) {
     const int sl = slot_of[j];
@@ -393,11 +414,11 @@ __global__ void __launch_bounds__(GA_THREADS) gather_kernel(PfParams p) {
       if (sub == 0) set_status(p.a.status, kStatusBounds, 4);
       continue;
     }
-    const size_t dst = (im.inst * (size_t)p.N + sl) * kHeadDim;
-    const size_t src = (im.in_row0 + j) * kHeadDim;
-    if (sub < 16)
+    const size_t dst = (im.inst * (size_t)p.N + sl) * D;
+    const size_t src = (im.in_row0 + j) * D;
+    if (sub < CH)
       reinterpret_cast<uint4*>(p.a.kslots + dst)[sub] = __ldg(reinterpret_cast<const uint4*>(p.K + src) + sub);
-    else
+    else if (sub >= 16 && sub < 16 + CH)
       reinterpret_cast<uint4*>(p.a.vslots + dst)[sub - 16] =
           __ldg(reinterpret_cast<const uint4*>(p.V + src) + (sub - 16));
     if (sub == 0) {
@@ -408,23 +429,90 @@ __global__ void __launch_bounds__(GA_THREADS) gather_kernel(PfParams p) {
   }
 }
 
-template <int R>
-__global__ void __launch_bounds__(kHeadDim) finalize_kernel(PfParams p) {
+template <int R, int D>
+__global__ void __launch_bounds__(D) finalize_kernel(PfParams p) {
   const int g = blockIdx.x, tid = threadIdx.x;
   const InstMap im = map_instance(p, g);
   const bool use_state = !(p.flags & LESS_NO_STATE);
-  const float* hp = p.a.ws_hpart + (size_t)g * kMaxSplit * (R * kHeadDim + R);
+  const float* hp = p.a.ws_hpart + (size_t)g * kMaxSplit * (R * D + R);
   const int ns = use_state ? p.nsplit : 0;
 #pragma unroll
   for (int r = 0; r < R; ++r) {
     float s = 0.f;
-    for (int sp = 0; sp < ns; ++sp) s += hp[(size_t)sp * (R * kHeadDim + R) + r * kHeadDim + tid];
-    p.a.H[(im.inst * R + r) * kHeadDim + tid] = s;
+    for (int sp = 0; sp < ns; ++sp) s += hp[(size_t)sp * (R * D + R) + r * D + tid];
+    p.a.H[(im.inst * R + r) * D + tid] = s;
   }
   if (tid < R) {
     float s = 0.f;
-    for (int sp = 0; sp < ns; ++sp) s += hp[(size_t)sp * (R * kHeadDim + R) + R * kHeadDim + tid];
+    for (int sp = 0; sp < ns; ++sp) s += hp[(size_t)sp * (R * D + R) + R * D + tid];
     p.a.z[im.inst * R + tid] = s;
+  }
+}
+
+// ---- P6 on CUDA cores (general shapes): the split's share of Eq. 4 / Eq. 5 over D_1 ---------- //
+// One CTA per (token split, instance), thread d = one column of H: H[r][d] += psi_j[r] v_j[d] over
+// the split's discarded tokens in ascending position (fixed order), z[r] likewise.
+template <int R, int D>
+__global__ void __launch_bounds__(D) state_kernel(PfParams p) {
+  const int split = blockIdx.x, g = blockIdx.y, tid = threadIdx.x;
+  const InstMap im = map_instance(p, g);
+  const int jbeg = split * p.split_tokens, jend = min(p.S, jbeg + p.split_tokens);
+  const float* psi = p.a.ws_psi + (size_t)g * p.Sp * R;
+  const int32_t* slot_of = p.a.ws_slot + (size_t)g * p.Sp;
+  float h[R], z = 0.f;
+#pragma unroll
+  for (int r = 0; r < R; ++r) h[r] = 0.f;
+  for (int j = jbeg; j < jend; ++j) {
+    if (slot_of[j] >= 0) continue;                    // kept: stays in the cache
+    const float v = __half2float(p.V[(im.in_row0 + j) * D + tid]);
+#pragma unroll
+    for (int r = 0; r < R; ++r) h[r] = fmaf(__ldg(psi + (size_t)j * R + r), v, h[r]);
+    if (tid < R) z += __ldg(psi + (size_t)j * R + tid);
+  }
+  float* hp = p.a.ws_hpart + ((size_t)g * kMaxSplit + split) * (R * D + R);
+#pragma unroll
+  for (int r = 0; r < R; ++r) hp[r * D + tid] = h[r];
+  if (tid < R) hp[R * D + tid] = z;
+}
+
+// The CUDA-core prompt phase for one head dimension: every step of launch_prefill_group below that
+// has no tensor-core kernel for the shape at hand.
+template <int R, int D>
+static void launch_cuda_core_tail(less_ctx* c, const PfParams& p, int G, int S, bool use_state, bool with_psi,
+                                  bool with_state, cudaStream_t s) {
+  const Dims& d = c->d;
+  if (with_psi) {
+    const size_t smem = (size_t)(FM_BR * D + mlp_smem_floats(d.Rp)) * 4;
+    LaunchScope scope(c, LESS_KERNEL_PSI, s, "psi_kernel");
+    cudaFuncSetAttribute(psi_kernel<R, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    psi_kernel<R, D><<<dim3(p.nsplit, G), FM_THREADS, smem, s>>>(p);
+  }
+  if (S > 0) {
+    LaunchScope scope(c, LESS_KERNEL_GATHER, s, "gather_kernel");
+    const int gx = (min(S, d.N) + 63) / 64 > 0 ? (min(S, d.N) + 63) / 64 : 1;
+    gather_kernel<R, D><<<dim3(gx, G), GA_THREADS, 0, s>>>(p);
+  }
+  if (with_state) {
+    LaunchScope scope(c, LESS_KERNEL_BUILD, s, "state_kernel");
+    state_kernel<R, D><<<dim3(p.nsplit, G), D, 0, s>>>(p);
+  }
+  (void)use_state;
+}
+
+template <int D>
+static void launch_cuda_core_scoring(less_ctx* c, const PfParams& p, int G, int S, bool h2o, bool with_out, cudaStream_t s) {
+  const int tiles = (S + PF_TILE - 1) / PF_TILE;
+  {
+    LaunchScope scope(c, LESS_KERNEL_ROWSTAT, s, "rowstat_kernel");
+    rowstat_kernel<D><<<dim3(tiles, G * p.grp), PF_TILE, 0, s>>>(p);
+  }
+  if (h2o) {
+    LaunchScope scope(c, LESS_KERNEL_COLSUM, s, "colsum_kernel");
+    colsum_kernel<D><<<dim3(tiles, G), PF_TILE, 0, s>>>(p);
+  }
+  if (with_out) {
+    LaunchScope scope(c, LESS_KERNEL_ATTN_OUT, s, "attn_out_kernel");
+    attn_out_kernel<D><<<dim3((S + AO_ROWS - 1) / AO_ROWS, G * p.grp), PF_TILE, 0, s>>>(p);
   }
 }
 
@@ -446,8 +534,6 @@ int launch_prefill_group(less_ctx* c, int layer0, int nl, int lj0, int layer_cou
   p.heavy = d.heavy; p.recent = d.recent; p.Rp = d.Rp;
   p.flags = d.flags;
   p.grp = d.G;
-  // grouped query heads run on the tensor-core scoring kernels only
-  if (d.G > 1 && S > 0 && !(c->score_path == 1 && score_tc_supported())) return LESS_ERR_INVALID_CONFIG;
   // Token splits of the state build: whole 128-token tiles, as long as they can be (the head's W1,
   // 128 KB, and the CTA's set-up are paid per split) while the grid still is several waves deep,
   // so that the last wave's imbalance stays small.
@@ -464,67 +550,59 @@ int launch_prefill_group(less_ctx* c, int layer0, int nl, int lj0, int layer_cou
   // needed for the prompt's attention output
   const bool h2o = !(d.flags & (LESS_POLICY_LAMBDA | LESS_POLICY_TOVA));
   const bool need_scores = h2o || attn_out != nullptr;
+  // tensor-core kernels: head dimension 128 and 1, 2, 4 or 8 query heads per KV head; everything else
+  // (and LESS_SCORE_KERNEL=plain) runs the CUDA-core kernels, which take any of the shapes
+  const bool tc_scoring = !d.general && c->score_path == 1 && score_tc_supported();
   if (S > 0 && need_scores) {
-    const int tiles = (S + PF_TILE - 1) / PF_TILE;
-    if (c->score_path == 1 && score_tc_supported()) {
-      const int rc = launch_score_tc(c, p, G, s, h2o);   // column sums only where H2O ranks by them
+    if (tc_scoring) {
+      int rc = launch_score_tc(c, p, G, s, h2o);   // column sums only where H2O ranks by them
+      if (rc == LESS_OK && attn_out) rc = launch_attn_out_tc(c, p, G, s);
       if (rc != LESS_OK) return rc;
+    } else if (d.D == 64) {
+      launch_cuda_core_scoring<64>(c, p, G, S, h2o, attn_out != nullptr, s);
     } else {
-      {
-        LaunchScope scope(c, LESS_KERNEL_ROWSTAT, s, "rowstat_kernel");
-        rowstat_kernel<<<dim3(tiles, G), PF_TILE, 0, s>>>(p);
-      }
-      if (h2o) {
-        LaunchScope scope(c, LESS_KERNEL_COLSUM, s, "colsum_kernel");
-        colsum_kernel<<<dim3(tiles, G), PF_TILE, 0, s>>>(p);
-      }
-    }
-    if (attn_out && c->score_path == 1 && score_tc_supported()) {
-      const int rc = launch_attn_out_tc(c, p, G, s);
-      if (rc != LESS_OK) return rc;
-    } else if (attn_out) {
-      LaunchScope scope(c, LESS_KERNEL_ATTN_OUT, s, "attn_out_kernel");
-      attn_out_kernel<<<dim3((S + AO_ROWS - 1) / AO_ROWS, G), PF_TILE, 0, s>>>(p);
+      launch_cuda_core_scoring<kHeadDim>(c, p, G, S, h2o, attn_out != nullptr, s);
     }
   }
   if (S > 0 && (d.flags & LESS_POLICY_TOVA)) {
     LaunchScope scope(c, LESS_KERNEL_COLSUM, s, "lastrow_kernel");
-    lastrow_kernel<<<G, LR_THREADS, 0, s>>>(p);
+    if (d.D == 64) lastrow_kernel<64><<<G, LR_THREADS, 0, s>>>(p);
+    else lastrow_kernel<kHeadDim><<<G, LR_THREADS, 0, s>>>(p);
   }
   {
     LaunchScope scope(c, LESS_KERNEL_SELECT, s, "select_kernel");
     select_kernel<<<G, SEL_THREADS, 0, s>>>(p);
   }
-  const size_t smem = (size_t)(FM_BR * kHeadDim + mlp_smem_floats(d.Rp)) * 4;
   const bool use_state = !(d.flags & LESS_NO_STATE);
-  const bool fused = nsplit > 0 && use_state && psi_tc_supported(d);   // psi and the state build in one kernel
+  const bool with_state = nsplit > 0 && use_state;
+  const bool fused = with_state && !d.general && psi_tc_supported(d);   // psi and the state build in one kernel
   if (fused) {
     const int rc = launch_psi_state_tc(c, p, G, s);
     if (rc != LESS_OK) return rc;
-  } else if (nsplit > 0 && use_state) {
-    LaunchScope scope(c, LESS_KERNEL_PSI, s, "psi_kernel");
-    if (d.R == 8) {
-      cudaFuncSetAttribute(psi_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-      psi_kernel<8><<<dim3(nsplit, G), FM_THREADS, smem, s>>>(p);
-    } else {
-      cudaFuncSetAttribute(psi_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-      psi_kernel<16><<<dim3(nsplit, G), FM_THREADS, smem, s>>>(p);
-    }
   }
-  if (S > 0) {
-    LaunchScope scope(c, LESS_KERNEL_GATHER, s, "gather_kernel");
-    const int gx = (min(S, d.N) + 63) / 64 > 0 ? (min(S, d.N) + 63) / 64 : 1;
-    if (d.R == 8) gather_kernel<8><<<dim3(gx, G), GA_THREADS, 0, s>>>(p);
-    else gather_kernel<16><<<dim3(gx, G), GA_THREADS, 0, s>>>(p);
+  // psi on CUDA cores where the fused kernel does not apply; the kept rows to their slots; the state
+  // build of the general shapes
+  const bool cc_state = with_state && d.general;
+  if (d.D == 64) {
+    if (d.R == 8) launch_cuda_core_tail<8, 64>(c, p, G, S, use_state, with_state && !fused, cc_state, s);
+    else launch_cuda_core_tail<16, 64>(c, p, G, S, use_state, with_state && !fused, cc_state, s);
+  } else {
+    if (d.R == 8) launch_cuda_core_tail<8, kHeadDim>(c, p, G, S, use_state, with_state && !fused, cc_state, s);
+    else launch_cuda_core_tail<16, kHeadDim>(c, p, G, S, use_state, with_state && !fused, cc_state, s);
   }
-  if (nsplit > 0 && use_state && !fused) {
+  if (with_state && !fused && !cc_state) {
     const int rc = launch_state_tc(c, p, G, s);
     if (rc != LESS_OK) return rc;
   }
   {
     LaunchScope scope(c, LESS_KERNEL_FINALIZE, s, "finalize_kernel");
-    if (d.R == 8) finalize_kernel<8><<<G, kHeadDim, 0, s>>>(p);
-    else finalize_kernel<16><<<G, kHeadDim, 0, s>>>(p);
+    if (d.D == 64) {
+      if (d.R == 8) finalize_kernel<8, 64><<<G, 64, 0, s>>>(p);
+      else finalize_kernel<16, 64><<<G, 64, 0, s>>>(p);
+    } else {
+      if (d.R == 8) finalize_kernel<8, kHeadDim><<<G, kHeadDim, 0, s>>>(p);
+      else finalize_kernel<16, kHeadDim><<<G, kHeadDim, 0, s>>>(p);
+    }
   }
   return check_launch("the prompt-phase kernels");
 }

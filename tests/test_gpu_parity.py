@@ -558,7 +558,6 @@ def test_general_shapes_decode_from_empty(head_dim, group, rank, batch, flags):
     kernel, teacher-forced against the grouped oracle from an empty cache through filling, the first
     evictions and on; both policies, both normalisers, state off, TOVA with one head."""
     import harness
-    from paper_2402_09398_b200 import binding
     w = small(160 + group, batch=batch, layers=2, heads=2, head_dim=head_dim, prompt=0, steps=26, heavy=5, recent=6,
               rank=rank, weight_std=0.1, group=group)
     ctx, W = _setup(w, flags=flags, max_prompt=64)
@@ -569,14 +568,39 @@ def test_general_shapes_decode_from_empty(head_dim, group, rank, batch, flags):
         tf.step(*wl.make_decode_inputs(w, s, DEV, prompt=0))
     assert tf.evictions > 0 and ctx.poll_status() == 0
     assert ctx.kernel_variant("decode").startswith("decode_group_loop_kernel")
-    # the prompt kernels are not built for these shapes: refused with an error code, nothing launched
-    Q, K, V = wl.make_prompt(w, 0, w.layers, DEV, prompt=16)
-    with pytest.raises(binding.LessError) as e:
-        ctx.prefill(Q, K, V, 0)
-    assert e.value.code == -1
-    ctx.reset()                                          # prompt_len == 0 still resets
+    ctx.reset()                                          # prompt_len == 0 resets the layers
     rec = ctx.export_state(inst)
     assert all(r["count"] == 0 and not r["H"].any() and not r["z"].any() for r in rec) and ctx.position == 0
+    ctx.close()
+
+
+@pytest.mark.parametrize("head_dim,group,rank,prompt,flags", [(64, 71, 8, 150, 0), (64, 5, 16, 300, 0), (64, 1, 8, 131, 0),
+                                                             (128, 3, 8, 257, 0), (64, 4, 8, 200, 4), (64, 1, 8, 140, 8),
+                                                             (64, 6, 8, 200, 2), (64, 3, 16, 180, 1)])
+def test_general_shapes_prompt_and_decode(head_dim, group, rank, prompt, flags):
+    """The prompt phase of the general shapes (head dimension 64, any number of query heads per KV
+    head) on the CUDA-core kernels: per-query-head attention output, column sums over the group's
+    heads, selection, cached psi, H and z against the oracle; then teacher-forced decode steps on top."""
+    import harness
+    w = small(170 + group, batch=1, layers=2, heads=2, head_dim=head_dim, prompt=prompt, steps=6, heavy=20, recent=20,
+              rank=rank, weight_std=0.1, group=group)
+    if flags & 4:
+        w = w.with_(heavy=4, recent=36)
+    ctx, W = _setup(w, flags=flags)
+    Q, K, V, out = _prefill_all(ctx, w)
+    assert Q.shape[2] == w.heads * group and Q.shape[-1] == head_dim and ctx.poll_status() == 0
+    assert ctx.kernel_variant("rowstat") in ("rowstat_kernel", "") and ctx.kernel_variant("psi") in ("psi_kernel", "")
+    inst = list(range(w.instances))
+    if group > 1:
+        r = harness.check_prefill_group(ctx, w, W, Q, K, V, inst, out, flags)
+        tf = harness.GroupTeacherForced(ctx, w, W, inst, flags)
+    else:
+        r = harness.check_prefill(ctx, w, W, Q, K, V, inst, out, flags)
+        tf = harness.TeacherForced(ctx, w, W, inst, flags)
+    assert r["exempt"] <= 2
+    for s in range(w.steps):
+        tf.step(*wl.make_decode_inputs(w, s, DEV))
+    assert tf.evictions == w.steps * w.instances and ctx.poll_status() == 0
     ctx.close()
 
 
