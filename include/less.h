@@ -202,11 +202,13 @@ int less_decode_step(less_ctx* ctx, const void* q, const void* k, const void* v,
 
 /* The same step for callers whose tensors live in host memory (Algorithm 1's
  * inputs and return value): q host fp16 [B, L, H * group, D], k, v host fp16
- * [B, L, H, D], out host fp32 (fp16 with LESS_OUT_F16) [B, L, H * group, D].  q and k are copied
- * to staging buffers inside the arena - in ONE copy when k_host starts exactly where q_host ends
- * (one host block [q | k]), else in two; v and out are read / written in place by the decode
- * kernel when they lie in pinned (page-locked, device-mapped) memory, else they are staged and
- * copied too.  Everything runs on the given stream, which is synchronised before returning. */
+ * [B, L, H, D], out host fp32 (fp16 with LESS_OUT_F16) [B, L, H * group, D].  From pinned
+ * (page-locked, device-mapped) memory v and out are read / written in place by the decode kernel,
+ * and with at most 8 batch rows q and k are read in place too (the feature-map kernel then fetches
+ * its rows with plain loads while the weights stream: no copy in front of the step).  Otherwise q
+ * and k are copied to staging buffers inside the arena - in ONE copy when k_host starts exactly
+ * where q_host ends (one host block [q | k]), else in two - and pageable v / out are staged and
+ * copied as well.  Everything runs on the given stream, which is synchronised before returning. */
 int less_decode_step_host(less_ctx* ctx, const void* q_host, const void* k_host, const void* v_host,
                           void* out_host, void* cuda_stream);
 

@@ -78,6 +78,7 @@ int launch_feature_maps(less_ctx* c, const void* q, const void* k, cudaStream_t 
   p.B = d.B; p.L = d.L; p.Hd = d.Hd; p.Rp = d.Rp; p.D = d.D;
   p.Hh[0] = d.Hd * d.G; p.Hh[1] = d.Hd;
   p.feat_flag = nullptr; p.flag_stride = d.L * d.Hd * d.G;
+  p.x_plain = c->x_plain ? 1 : 0;
   c->flags_this_step = false;
   const int ndg = FM_THREADS / (d.Rp / 8);
   const size_t smem = (size_t)(FM_BR * d.D + FM_BR * d.Rp + ndg * FM_BR * d.Rp) * 4;

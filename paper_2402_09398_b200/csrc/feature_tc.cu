@@ -29,7 +29,7 @@ namespace less {
 
 constexpr int FT_EPI_WARPS = 8;
 constexpr int FT_EPI_THREADS = FT_EPI_WARPS * 32;
-constexpr int FT_THREADS = 64 + FT_EPI_THREADS;   // small-batch kernel: warp 0 TMA, warp 1 MMA, warps 2..9 epilogue
+constexpr int FT_THREADS = 96 + FT_EPI_THREADS;   // small-batch kernel: warp 0 TMA, warp 1 MMA, warps 2..9 epilogue, warp 10 input rows by plain loads
 // The larger-batch kernel runs four epilogue warps per lane quadrant: its GELU chains are long and
 // dependent, and with two warps per scheduler the issue slots sat idle (4700 cycles per chunk
 // measured for 32 GELUs per thread).
@@ -105,10 +105,12 @@ __device__ __forceinline__ void ft_produce(const CUtensorMap* tm_q, const CUtens
     if (*abortp) return;                                 // issue nothing more once the CTA has given up
     const CUtensorMap* tx = im.which ? tm_k : tm_q;
     const CUtensorMap* tw1 = im.which ? tm_w1psi : tm_w1phi;
-    mbar_expect_tx(&aux_full[a], xbytes + w2bytes + (im.which ? R * R * 2 : 0));
+    mbar_expect_tx(&aux_full[a], (p.x_plain ? 0u : xbytes) + w2bytes + (im.which ? R * R * 2 : 0));
     unsigned char* xa = xbuf + a * xbytes;
-    tma_load_2d(xa, tx, im.lh * kHeadDim, im.tile * gm.npad, &aux_full[a]);
-    tma_load_2d(xa + xbytes / 2, tx, im.lh * kHeadDim + 64, im.tile * gm.npad, &aux_full[a]);
+    if (!p.x_plain) {
+      tma_load_2d(xa, tx, im.lh * kHeadDim, im.tile * gm.npad, &aux_full[a]);
+      tma_load_2d(xa + xbytes / 2, tx, im.lh * kHeadDim + 64, im.tile * gm.npad, &aux_full[a]);
+    }
     // W2 comes as one contiguous copy (a tiled load of 16-byte rows is far slower)
     bulk_g2s(w2dst + a * w2bytes, p.w2[im.which] + (size_t)im.lh * p.Rp * R, w2bytes, &aux_full[a]);
     if (im.which) bulk_g2s(w3buf + a * 256, p.w3 + (size_t)im.lh * R * R, R * R * 2, &aux_full[a]);
@@ -447,7 +449,7 @@ __global__ void __launch_bounds__(FT_THREADS) feature_tc_small_kernel(
       mbar_init(&sh->empty[s], 1);
     }
     for (int s = 0; s < FS_AUX; ++s) {
-      mbar_init(&sh->aux_full[s], 1);
+      mbar_init(&sh->aux_full[s], p.x_plain ? 2 : 1);    // the producer's copies, and the row loader's arrival
       mbar_init(&sh->aux_empty[s], 1 + FT_EPI_WARPS);
     }
     for (int s = 0; s < FS_BUFS; ++s) {
@@ -471,6 +473,34 @@ __global__ void __launch_bounds__(FT_THREADS) feature_tc_small_kernel(
     if (lane == 0)
       ft_produce<R>(&tm_q, &tm_k, &tm_w1phi, &tm_w1psi, p, gm, my_items, nchunk, xbuf, FS_XBYTES, w2raw, w2bytes,
                     &sh->w3[0][0], ring, sh->full, sh->empty, sh->aux_full, sh->aux_empty, FS_AUX, abortp, status);
+  } else if (warp == 2 + FT_EPI_WARPS) {
+    // ---------------- input rows by plain loads ----------------
+    // Used when q and k lie in pinned host memory (the host entry point): the rows come over PCIe
+    // while the weights stream, no staging copy in front of the step.  The warp writes what the
+    // tiled load would have written: per half of 64 columns, 8 rows of 128 bytes, the 16-byte chunk c
+    // of row r at chunk position c ^ r (128-byte swizzle); rows past the batch are zeros.
+    if (p.x_plain) {
+      uint32_t a = 0, aph = 0;
+      for (int n = 0; n < my_items; ++n, (++a == FS_AUX ? (a = 0, aph ^= 1) : 0u)) {
+        const FtItem im = ft_item(blockIdx.x + n * gridDim.x, gm);
+        wait_or_give_up(&sh->aux_empty[a], aph ^ 1, abortp, status, 67);
+        if (*abortp) break;
+        unsigned char* xa = xbuf + a * FS_XBYTES;
+        const __half* src = p.x[im.which] + (size_t)im.lh * kHeadDim;
+        const size_t row_stride = (size_t)p.L * p.Hh[im.which] * kHeadDim;
+        const int b0 = im.tile * FS_NPAD;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const int e = lane + 32 * i;                 // 128 chunks: (half, row, chunk)
+          const int h = e >> 6, r = (e >> 3) & 7, c = e & 7;
+          uint4 v = make_uint4(0, 0, 0, 0);
+          if (b0 + r < p.B) v = *reinterpret_cast<const uint4*>(src + (size_t)(b0 + r) * row_stride + h * 64 + c * 8);
+          *reinterpret_cast<uint4*>(xa + h * (FS_XBYTES / 2) + r * 128 + ((c ^ r) << 4)) = v;
+        }
+        fence_proxy_async_smem();
+        mbar_arrive_warp(&sh->aux_full[a]);
+      }
+    }
   } else if (warp == 1) {
     // ---------------- MMA issuer: GEMM1 only ----------------
     if (lane == 0) {
@@ -591,6 +621,13 @@ static int launch_small(less_ctx* c, const FmParams& p, const FtGeom& gm, const 
     return fail_cuda("shared memory opt-in of feature_tc_small_kernel");
   kern<<<grid, FT_THREADS, smem, s>>>(tq, tk, tw1a, tw1b, p, gm, c->a.status);
   return check_launch("feature_tc_small_kernel");
+}
+
+// whether a decode step of this context runs the small-batch tensor-core kernel (the one that can fetch
+// the step's q, k rows with plain loads)
+bool feature_small_tc_path(const less_ctx* c) {
+  const Dims& d = c->d;
+  return !d.general && !(d.flags & LESS_NO_STATE) && (c->feature_path == 2 || d.G > 1) && feature_tc_supported(d) && d.B <= 8;
 }
 
 bool feature_tc_supported(const Dims& d) {

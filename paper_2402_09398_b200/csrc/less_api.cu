@@ -198,6 +198,7 @@ int less_create(const less_config* cfg, const less_weights* w, void* arena, size
   memset(c->variant, 0, sizeof c->variant);
   c->feature_ctas = 0;
   c->head_counters = getenv("LESS_HEAD_COUNTERS") != nullptr;
+  c->x_plain = false;
   if (const char* e = getenv("LESS_FEATURE_CTAS")) c->feature_ctas = atoi(e);
   c->profile = false;
   c->feature_path = 2;
@@ -328,29 +329,40 @@ int less_decode_step_host(less_ctx* c, const void* qh, const void* kh, const voi
   cudaStream_t s = (cudaStream_t)stream;
   const size_t osz = (c->d.flags & LESS_OUT_F16) ? 2 : 4;
   const size_t nin = (size_t)c->d.I * c->d.D * 2, nq = nin * c->d.G, nout = (size_t)c->d.I * c->d.G * c->d.D * osz;
-  // q and k feed the feature-map kernel's TMA loads and are staged in the arena (the two staging
-  // buffers are neighbours, so a caller that keeps k directly behind q pays one copy, not two).
   // v and the output are touched once per instance by the decode kernel: from pinned host memory
-  // it reads / writes them in place, which saves two more copies per step.
+  // it reads / writes them in place.  q and k feed the feature-map kernel: with more than 8 batch rows
+  // its TMA loads want them in device memory and they are staged in the arena (the two staging
+  // buffers are neighbours, so a caller that keeps k directly behind q pays one copy, not two).
   const void* v_dev = device_alias(vh);
   void* out_dev = device_alias(outh);
   if (((uintptr_t)v_dev & 15) || ((uintptr_t)out_dev & 15)) { v_dev = nullptr; out_dev = nullptr; }
   cudaError_t e = cudaSuccess;
-  bool copied = false;
-  if ((const char*)kh == (const char*)qh + nq && (char*)c->a.stage_k == (char*)c->a.stage_q + nq) {
-    // k directly behind q.  If the two are separate host allocations that merely touch, the runtime
-    // refuses the copy that spans them (nothing is enqueued): then they go one by one.
-    copied = cudaMemcpyAsync(c->a.stage_q, qh, nq + nin, cudaMemcpyHostToDevice, s) == cudaSuccess;
-    if (!copied) cudaGetLastError();
-  }
-  if (!copied) {
-    e = cudaMemcpyAsync(c->a.stage_q, qh, nq, cudaMemcpyHostToDevice, s);
-    if (e == cudaSuccess) e = cudaMemcpyAsync(c->a.stage_k, kh, nin, cudaMemcpyHostToDevice, s);
+  // With a small batch the feature-map kernel can fetch its q, k rows with plain loads: from pinned
+  // host memory they are then read in place too (by both kernels), and the step has no copy in front
+  // of it - the rows cross PCIe while the weights stream.
+  const void* q_dev = device_alias(qh);
+  const void* k_dev = device_alias(kh);
+  const bool qk_in_place = q_dev && k_dev && !((uintptr_t)q_dev & 15) && !((uintptr_t)k_dev & 15) &&
+                           (feature_small_tc_path(c) || (c->d.flags & LESS_NO_STATE));
+  if (!qk_in_place) {
+    bool copied = false;
+    if ((const char*)kh == (const char*)qh + nq && (char*)c->a.stage_k == (char*)c->a.stage_q + nq) {
+      // k directly behind q.  If the two are separate host allocations that merely touch, the runtime
+      // refuses the copy that spans them (nothing is enqueued): then they go one by one.
+      copied = cudaMemcpyAsync(c->a.stage_q, qh, nq + nin, cudaMemcpyHostToDevice, s) == cudaSuccess;
+      if (!copied) cudaGetLastError();
+    }
+    if (!copied) {
+      e = cudaMemcpyAsync(c->a.stage_q, qh, nq, cudaMemcpyHostToDevice, s);
+      if (e == cudaSuccess) e = cudaMemcpyAsync(c->a.stage_k, kh, nin, cudaMemcpyHostToDevice, s);
+    }
   }
   if (e == cudaSuccess && !v_dev) e = cudaMemcpyAsync(c->a.stage_v, vh, nin, cudaMemcpyHostToDevice, s);
   if (e != cudaSuccess) return LESS_ERR_CUDA;
-  int rc = less_decode_step(c, c->a.stage_q, c->a.stage_k, v_dev ? v_dev : c->a.stage_v,
-                            out_dev ? out_dev : c->a.stage_out, nullptr, s);
+  c->x_plain = qk_in_place;
+  int rc = less_decode_step(c, qk_in_place ? q_dev : c->a.stage_q, qk_in_place ? k_dev : c->a.stage_k,
+                            v_dev ? v_dev : c->a.stage_v, out_dev ? out_dev : c->a.stage_out, nullptr, s);
+  c->x_plain = false;
   if (rc != LESS_OK) return rc;
   if (!out_dev) e = cudaMemcpyAsync(outh, c->a.stage_out, nout, cudaMemcpyDeviceToHost, s);
   if (e == cudaSuccess) e = cudaStreamSynchronize(s);

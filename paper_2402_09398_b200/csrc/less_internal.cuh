@@ -88,6 +88,7 @@ struct less_ctx {
   int score_path;      // prompt scoring: 1 tensor cores, 0 CUDA cores (LESS_SCORE_KERNEL=plain)
   int feature_path;    // feature-map kernel: 2 tensor cores, 1 streaming GEMV, 0 plain (LESS_FEATURE_KERNEL)
   int group_path;      // grouped decode kernel: 2 on CUDA cores (LESS_GROUP_KERNEL=rows), else with warp-level mma
+  bool x_plain;        // set by the host entry around a step whose q, k are read in place from pinned host memory
   bool head_counters;  // decode CTAs follow the large-batch feature kernel head by head (LESS_HEAD_COUNTERS=1; off by default)
   int feature_ctas;    // cap on the feature kernels' persistent CTAs (LESS_FEATURE_CTAS), 0 = one per multiprocessor
   bool flags_this_step;     // the step's feature-map launch publishes per-head counters (set by its launcher)
@@ -253,6 +254,8 @@ inline bool overlap_decode(const less_ctx* c) {
 
 // launchers (host), defined in the kernel translation units
 int launch_feature_maps(less_ctx* c, const void* q, const void* k, cudaStream_t s);
+// whether a decode step of this context runs the small-batch tensor-core feature kernel (feature_tc.cu)
+bool feature_small_tc_path(const less_ctx* c);
 int launch_decode(less_ctx* c, const void* q, const void* k, const void* v, void* out,
                   int32_t* evicted_pos, cudaStream_t s);
 int launch_prefill_group(less_ctx* c, int layer0, int nlayers, int lj0, int layer_count, int S,
