@@ -478,8 +478,8 @@ __global__ void __launch_bounds__(D) state_kernel(PfParams p) {
 // The CUDA-core prompt phase for one head dimension: every step of launch_prefill_group below that
 // has no tensor-core kernel for the shape at hand.
 template <int R, int D>
-static void launch_cuda_core_tail(less_ctx* c, const PfParams& p, int G, int S, bool use_state, bool with_psi,
-                                  bool with_state, cudaStream_t s) {
+static void launch_cuda_core_tail(less_ctx* c, const PfParams& p, int G, int S, bool with_psi, bool with_state,
+                                  cudaStream_t s) {
   const Dims& d = c->d;
   if (with_psi) {
     const size_t smem = (size_t)(FM_BR * D + mlp_smem_floats(d.Rp)) * 4;
@@ -496,7 +496,6 @@ static void launch_cuda_core_tail(less_ctx* c, const PfParams& p, int G, int S, 
     LaunchScope scope(c, LESS_KERNEL_BUILD, s, "state_kernel");
     state_kernel<R, D><<<dim3(p.nsplit, G), D, 0, s>>>(p);
   }
-  (void)use_state;
 }
 
 template <int D>
@@ -584,11 +583,11 @@ int launch_prefill_group(less_ctx* c, int layer0, int nl, int lj0, int layer_cou
   // build of the general shapes
   const bool cc_state = with_state && d.general;
   if (d.D == 64) {
-    if (d.R == 8) launch_cuda_core_tail<8, 64>(c, p, G, S, use_state, with_state && !fused, cc_state, s);
-    else launch_cuda_core_tail<16, 64>(c, p, G, S, use_state, with_state && !fused, cc_state, s);
+    if (d.R == 8) launch_cuda_core_tail<8, 64>(c, p, G, S, with_state && !fused, cc_state, s);
+    else launch_cuda_core_tail<16, 64>(c, p, G, S, with_state && !fused, cc_state, s);
   } else {
-    if (d.R == 8) launch_cuda_core_tail<8, kHeadDim>(c, p, G, S, use_state, with_state && !fused, cc_state, s);
-    else launch_cuda_core_tail<16, kHeadDim>(c, p, G, S, use_state, with_state && !fused, cc_state, s);
+    if (d.R == 8) launch_cuda_core_tail<8, kHeadDim>(c, p, G, S, with_state && !fused, cc_state, s);
+    else launch_cuda_core_tail<16, kHeadDim>(c, p, G, S, with_state && !fused, cc_state, s);
   }
   if (with_state && !fused && !cc_state) {
     const int rc = launch_state_tc(c, p, G, s);
