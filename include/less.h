@@ -206,9 +206,11 @@ int less_decode_step(less_ctx* ctx, const void* q, const void* k, const void* v,
  * (page-locked, device-mapped) memory v and out are read / written in place by the decode kernel,
  * and with at most 8 batch rows q and k are read in place too (the feature-map kernel then fetches
  * its rows with plain loads while the weights stream: no copy in front of the step).  Otherwise q
- * and k are copied to staging buffers inside the arena - in ONE copy when k_host starts exactly
- * where q_host ends (one host block [q | k]), else in two - and pageable v / out are staged and
- * copied as well.  Everything runs on the given stream, which is synchronised before returning. */
+ * and k are copied to staging buffers inside the arena: a large step goes in four layer segments
+ * whose copies (on a stream the context creates at the first such call) run under the kernels of
+ * the segment before; a small one in ONE copy when k_host starts exactly where q_host ends (one
+ * host block [q | k]), else in two.  Pageable v / out are staged and copied as well.  Everything is
+ * ordered behind the given stream, which is synchronised before returning. */
 int less_decode_step_host(less_ctx* ctx, const void* q_host, const void* k_host, const void* v_host,
                           void* out_host, void* cuda_stream);
 

@@ -79,6 +79,7 @@ int launch_feature_maps(less_ctx* c, const void* q, const void* k, cudaStream_t 
   p.Hh[0] = d.Hd * d.G; p.Hh[1] = d.Hd;
   p.feat_flag = nullptr; p.flag_stride = d.L * d.Hd * d.G;
   p.x_plain = c->x_plain ? 1 : 0;
+  p.lh0 = c->seg_l0 * d.Hd; p.nlh = c->seg_nl * d.Hd;
   c->flags_this_step = false;
   const int ndg = FM_THREADS / (d.Rp / 8);
   const size_t smem = (size_t)(FM_BR * d.D + FM_BR * d.Rp + ndg * FM_BR * d.Rp) * 4;
@@ -86,6 +87,7 @@ int launch_feature_maps(less_ctx* c, const void* q, const void* k, cudaStream_t 
   const int nbz = (d.B + FM_BR - 1) / FM_BR;
   if (!d.general) {
     if ((c->feature_path == 2 || d.G > 1) && feature_tc_supported(d)) return launch_feature_tc(c, p, s);
+    if (c->seg_nl != d.L) return LESS_ERR_INVALID_CONFIG;   // only the tensor-core kernels take a layer range
     if (d.G > 1) return LESS_ERR_INVALID_CONFIG;    // the streaming kernels below know one query head per KV head
     if (c->feature_path >= 1 && feature_gemv_supported(d)) return launch_feature_gemv(c, p, s);
     const dim3 grid(d.L * d.Hd, 2, nbz);
@@ -120,6 +122,7 @@ struct DecParams {
   int flag_stride;             // psi counters start here (= layers x query heads)
   uint32_t flag_target[2];     // counter values that mean "this step's phi / psi of the head are written"
   int head_major;              // CTAs numbered (layer-head, batch row) instead of by instance
+  int lh0;                     // first (layer, KV head) of this launch (head-major numbering only)
 };
 
 __device__ __forceinline__ float block_max(float v, float* red) {
@@ -208,8 +211,8 @@ __device__ __forceinline__ void store_out(const DecParams& p, size_t idx, float 
 // the first heads' feature maps; otherwise CTA = instance.
 __device__ __forceinline__ size_t decode_instance(const DecParams& p) {
   if (!p.head_major) return blockIdx.x;
-  const int lh = blockIdx.x / p.B, b = blockIdx.x - lh * p.B;
-  return (size_t)b * p.LH + lh;
+  const int lhi = blockIdx.x / p.B, b = blockIdx.x - lhi * p.B;
+  return (size_t)b * p.LH + p.lh0 + lhi;
 }
 
 // The second half of a step, common to all decode kernels (one 128-thread CTA per KV head, thread
@@ -347,7 +350,7 @@ __device__ __forceinline__ void group_eq3_and_tail(const DecParams& p, size_t in
   const float* zb = p.a.z + inst * R;
   float hcol[R], zr[R];
   if (use_state) {
-    wait_feature_maps<G>(p, p.head_major ? blockIdx.x / p.B : (int)(inst % p.LH));
+    wait_feature_maps<G>(p, (int)(inst % p.LH));
 #pragma unroll
     for (int r = 0; r < R; ++r) {
       hcol[r] = Hb[r * kHeadDim + d];
@@ -488,7 +491,7 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_kernel(DecParams p) {
   const float* zb = p.a.z + inst * R;
   float hcol[R];
   if (use_state) {
-    wait_feature_maps<1>(p, p.head_major ? blockIdx.x / p.B : (int)(inst % p.LH));   // phi(q_t), psi(k_t) of this step are complete from here on
+    wait_feature_maps<1>(p, (int)(inst % p.LH));   // phi(q_t), psi(k_t) of this step are complete from here on
     const float em = __expf(-m);
     float lr = 0.f, lz = 0.f;
 #pragma unroll
@@ -1061,7 +1064,9 @@ int launch_decode(less_ctx* c, const void* q, const void* k, const void* v, void
   p.flag_stride = d.L * d.Hd * d.G;
   p.flag_target[0] = c->flag_target[0];
   p.flag_target[1] = c->flag_target[1];
-  p.head_major = p.feat_flag != nullptr && d.B > 1;
+  const bool segment = c->seg_nl != d.L;            // a layer range: CTAs are numbered inside it, head-major
+  p.lh0 = c->seg_l0 * d.Hd;
+  p.head_major = (p.feat_flag != nullptr && d.B > 1) || segment;
   size_t smem = decode_smem_bytes(d);
   int which = c->group_path == 2 ? 2 : 3;
   char name[64];
@@ -1085,7 +1090,7 @@ int launch_decode(less_ctx* c, const void* q, const void* k, const void* v, void
       cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
     return fail_cuda("shared memory opt-in of decode_kernel");
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(d.I);
+  cfg.gridDim = dim3(segment ? d.B * c->seg_nl * d.Hd : d.I);
   cfg.blockDim = dim3(DEC_THREADS);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = s;

@@ -15,6 +15,7 @@ struct FmParams {
   int B, L, Hd, Rp;
   int D;                  // head dimension (128; 64 on the general path)
   int Hh[2];              // heads of each map per layer: query heads for phi (Hd * group), KV heads for psi
+  int lh0, nlh;           // (layer, KV head) range of this launch: [lh0, lh0 + nlh) of L * Hd (tensor-core kernels)
   int x_plain;            // small-batch tensor-core kernel: a warp fetches the q / k rows with plain loads (they may
                           // lie in pinned host memory) instead of TMA
   uint32_t* feat_flag;    // per-head counters to publish phi / psi through (psi's start at flag_stride), or null

@@ -57,6 +57,7 @@ struct FtGeom {
   int items;       // work items
   int per_head;    // items per KV head: (G + 1) * ntile
   int G;           // query heads per KV head
+  int kv0;         // first (layer, KV head) of this launch
   int nstage;      // ring stages
   uint32_t tmem_cols;
 };
@@ -69,7 +70,7 @@ struct FtGeom {
 struct FtItem { int tile, which, lh; };
 __device__ __forceinline__ FtItem ft_item(int it, const FtGeom& gm) {
   FtItem r;
-  const int kv = it / gm.per_head, rest = it - kv * gm.per_head;
+  const int kvi = it / gm.per_head, rest = it - kvi * gm.per_head, kv = gm.kv0 + kvi;
   const int sub = rest / gm.ntile;
   r.tile = rest - sub * gm.ntile;
   r.which = sub == gm.G;
@@ -623,12 +624,13 @@ static int launch_small(less_ctx* c, const FmParams& p, const FtGeom& gm, const 
   return check_launch("feature_tc_small_kernel");
 }
 
-// whether a decode step of this context runs the small-batch tensor-core kernel (the one that can fetch
-// the step's q, k rows with plain loads)
-bool feature_small_tc_path(const less_ctx* c) {
+// whether a decode step of this context runs a tensor-core feature kernel (they take a layer range), and
+// whether it is the small-batch one (which can fetch the step's q, k rows with plain loads)
+bool feature_tc_path(const less_ctx* c) {
   const Dims& d = c->d;
-  return !d.general && !(d.flags & LESS_NO_STATE) && (c->feature_path == 2 || d.G > 1) && feature_tc_supported(d) && d.B <= 8;
+  return !d.general && !(d.flags & LESS_NO_STATE) && (c->feature_path == 2 || d.G > 1) && feature_tc_supported(d);
 }
+bool feature_small_tc_path(const less_ctx* c) { return feature_tc_path(c) && c->d.B <= 8; }
 
 bool feature_tc_supported(const Dims& d) {
   return (d.Rp == 128 || d.Rp == 256 || d.Rp == 512) && encode_tiled_fn() != nullptr;
@@ -647,7 +649,8 @@ int launch_feature_tc(less_ctx* c, const FmParams& p_in, cudaStream_t s) {
   gm.ntile = (d.B + gm.npad - 1) / gm.npad;
   gm.G = d.G;
   gm.per_head = (d.G + 1) * gm.ntile;
-  gm.items = d.L * d.Hd * gm.per_head;
+  gm.kv0 = p.lh0;
+  gm.items = p.nlh * gm.per_head;
   const size_t fixed = ft_fixed_smem(d, gm.npad);
   int ns = (int)((FT_SMEM_LIMIT - fixed) / FT_STAGE_BYTES);
   gm.nstage = ns > FT_MAX_STAGES ? FT_MAX_STAGES : ns;

@@ -199,6 +199,9 @@ int less_create(const less_config* cfg, const less_weights* w, void* arena, size
   c->feature_ctas = 0;
   c->head_counters = getenv("LESS_HEAD_COUNTERS") != nullptr;
   c->x_plain = false;
+  c->seg_l0 = 0; c->seg_nl = d.L;
+  c->copy_stream = nullptr;
+  for (cudaEvent_t& ev : c->seg_event) ev = nullptr;
   if (const char* e = getenv("LESS_FEATURE_CTAS")) c->feature_ctas = atoi(e);
   c->profile = false;
   c->feature_path = 2;
@@ -237,6 +240,8 @@ int less_destroy(less_ctx* ctx) {
   if (!ctx) return LESS_ERR_NULL_POINTER;
   for (cudaEvent_t e : ctx->prof_events) cudaEventDestroy(e);
   for (cudaEvent_t e : ctx->prof_pool) cudaEventDestroy(e);
+  for (cudaEvent_t e : ctx->seg_event) if (e) cudaEventDestroy(e);
+  if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
   delete ctx;
   return LESS_OK;
 }
@@ -312,6 +317,49 @@ int less_decode_step(less_ctx* c, const void* q, const void* k, const void* v, v
   return LESS_OK;
 }
 
+// The host entry's large steps: the layers in kSegments ranges, each range's q, k copied on a stream
+// of its own and its two kernels launched behind the copy, so that all copies but the first run
+// under the kernels of the range before.
+static constexpr int kSegments = 4;
+
+static int staged_step_in_segments(less_ctx* c, const void* qh, const void* kh, const void* v_dev, void* out_dev,
+                                   cudaStream_t s) {
+  const Dims& d = c->d;
+  if (!c->copy_stream) {
+    if (cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking) != cudaSuccess) return fail_cuda("copy stream");
+    for (int i = 0; i < 2 * kSegments; ++i)
+      if (cudaEventCreateWithFlags(&c->seg_event[i], cudaEventDisableTiming) != cudaSuccess) return fail_cuda("segment events");
+  }
+  // the copies may start once the caller's stream has reached this call
+  if (cudaEventRecord(c->seg_event[kSegments], s) != cudaSuccess ||
+      cudaStreamWaitEvent(c->copy_stream, c->seg_event[kSegments], 0) != cudaSuccess)
+    return fail_cuda("segment ordering");
+  const size_t rowq = (size_t)d.Hd * d.G * d.D * 2, rowk = (size_t)d.Hd * d.D * 2;   // bytes of one layer of one batch row
+  int l0[kSegments + 1];
+  for (int i = 0; i <= kSegments; ++i) l0[i] = (int)((long long)d.L * i / kSegments);
+  for (int i = 0; i < kSegments; ++i) {
+    const int nl = l0[i + 1] - l0[i];
+    if (cudaMemcpy2DAsync((char*)c->a.stage_q + l0[i] * rowq, d.L * rowq, (const char*)qh + l0[i] * rowq, d.L * rowq,
+                          nl * rowq, d.B, cudaMemcpyHostToDevice, c->copy_stream) != cudaSuccess ||
+        cudaMemcpy2DAsync((char*)c->a.stage_k + l0[i] * rowk, d.L * rowk, (const char*)kh + l0[i] * rowk, d.L * rowk,
+                          nl * rowk, d.B, cudaMemcpyHostToDevice, c->copy_stream) != cudaSuccess ||
+        cudaEventRecord(c->seg_event[i], c->copy_stream) != cudaSuccess)
+      return fail_cuda("segment copy");
+  }
+  int rc = LESS_OK;
+  for (int i = 0; i < kSegments && rc == LESS_OK; ++i) {
+    if (cudaStreamWaitEvent(s, c->seg_event[i], 0) != cudaSuccess) return fail_cuda("segment wait");
+    c->seg_l0 = l0[i];
+    c->seg_nl = l0[i + 1] - l0[i];
+    rc = launch_feature_maps(c, c->a.stage_q, c->a.stage_k, s);
+    if (rc == LESS_OK) rc = launch_decode(c, c->a.stage_q, c->a.stage_k, v_dev, out_dev, nullptr, s);
+  }
+  c->seg_l0 = 0;
+  c->seg_nl = d.L;
+  if (rc == LESS_OK) c->t += 1;
+  return rc;
+}
+
 // Device-visible alias of a host buffer: pinned (page-locked, mapped) memory can be read and
 // written by kernels directly over PCIe; pageable memory cannot (nullptr).
 static void* device_alias(const void* host) {
@@ -344,6 +392,13 @@ int less_decode_step_host(less_ctx* c, const void* qh, const void* kh, const voi
   const void* k_dev = device_alias(kh);
   const bool qk_in_place = q_dev && k_dev && !((uintptr_t)q_dev & 15) && !((uintptr_t)k_dev & 15) &&
                            (feature_small_tc_path(c) || (c->d.flags & LESS_NO_STATE));
+  // a large staged step: its layers in segments, the copies under the kernels
+  if (!qk_in_place && v_dev && out_dev && feature_tc_path(c) && !c->head_counters && c->d.L >= kSegments &&
+      nq + nin >= ((size_t)4 << 20) && c->t < 0x7fffff00) {
+    const int rc = staged_step_in_segments(c, qh, kh, v_dev, out_dev, s);
+    if (rc != LESS_OK) return rc;
+    return cudaStreamSynchronize(s) == cudaSuccess ? LESS_OK : LESS_ERR_CUDA;
+  }
   if (!qk_in_place) {
     bool copied = false;
     if ((const char*)kh == (const char*)qh + nq && (char*)c->a.stage_k == (char*)c->a.stage_q + nq) {

@@ -88,6 +88,10 @@ struct less_ctx {
   int score_path;      // prompt scoring: 1 tensor cores, 0 CUDA cores (LESS_SCORE_KERNEL=plain)
   int feature_path;    // feature-map kernel: 2 tensor cores, 1 streaming GEMV, 0 plain (LESS_FEATURE_KERNEL)
   int group_path;      // grouped decode kernel: 2 on CUDA cores (LESS_GROUP_KERNEL=rows), else with warp-level mma
+  int seg_l0, seg_nl;  // layers [seg_l0, seg_l0 + seg_nl) of the step being launched (the host entry launches a
+                       // large step in layer segments so that its input copies overlap the kernels); default all
+  cudaStream_t copy_stream;            // host entry: input copies of the later segments (created on first use)
+  cudaEvent_t seg_event[8];            // host entry: "segment's inputs are in device memory"
   bool x_plain;        // set by the host entry around a step whose q, k are read in place from pinned host memory
   bool head_counters;  // decode CTAs follow the large-batch feature kernel head by head (LESS_HEAD_COUNTERS=1; off by default)
   int feature_ctas;    // cap on the feature kernels' persistent CTAs (LESS_FEATURE_CTAS), 0 = one per multiprocessor
@@ -254,7 +258,8 @@ inline bool overlap_decode(const less_ctx* c) {
 
 // launchers (host), defined in the kernel translation units
 int launch_feature_maps(less_ctx* c, const void* q, const void* k, cudaStream_t s);
-// whether a decode step of this context runs the small-batch tensor-core feature kernel (feature_tc.cu)
+// whether a decode step of this context runs a tensor-core feature kernel, and the small-batch one (feature_tc.cu)
+bool feature_tc_path(const less_ctx* c);
 bool feature_small_tc_path(const less_ctx* c);
 int launch_decode(less_ctx* c, const void* q, const void* k, const void* v, void* out,
                   int32_t* evicted_pos, cudaStream_t s);

@@ -456,6 +456,32 @@ def test_host_buffer_entry_matches_device_entry(pinned, group):
     ctx_d.close(); ctx_h.close()
 
 
+def test_host_entry_in_layer_segments_matches_the_device_entry():
+    """A step large enough that the host entry launches it in layer segments (q, k of a segment copied
+    on a stream of its own while the segment before computes): outputs and state bit-identical to the
+    device entry's single launch, over several steps."""
+    w = small(57, batch=16, layers=8, heads=64, prompt=24, steps=4, heavy=6, recent=6, weight_std=0.1)
+    assert w.instances * w.head_dim * 2 * 2 >= 4 << 20
+    ctx_d, W = _setup(w)
+    ctx_h, _ = _setup(w)
+    for ctx in (ctx_d, ctx_h):
+        _prefill_all(ctx, w, with_out=False)
+    for s in range(w.steps):
+        q, k, v = wl.make_decode_inputs(w, s, DEV)
+        ref = ctx_d.decode_step(q, k, v).cpu()
+        hq, hk, hv = (t.cpu().pin_memory() for t in (q, k, v))
+        hout = torch.full(ref.shape, float("nan"), dtype=torch.float32).pin_memory()
+        ctx_h.decode_step_host(hq, hk, hv, hout)
+        assert torch.equal(hout, ref)
+    assert ctx_h.position == ctx_d.position
+    inst = list(range(0, w.instances, 61))
+    for a, b in zip(ctx_d.export_state(inst), ctx_h.export_state(inst)):
+        for key in ("pos", "acc", "K", "V", "psi", "H", "z"):
+            assert np.array_equal(a[key], b[key]), key
+    assert ctx_h.poll_status() == 0
+    ctx_d.close(); ctx_h.close()
+
+
 def test_tova_new_token_can_evict_itself():
     """TOVA: a new key the query points away from has the lowest probability of its own step;
     it is absorbed into H, z at once and no slot changes (imported state)."""
