@@ -1,5 +1,6 @@
 // Host side of the C ABI: config validation, arena carving, state export /
 // import, status polling.  No device memory is allocated here.
+#include <algorithm>
 #include <new>
 #include <stdio.h>
 #include <stdlib.h>
@@ -461,19 +462,39 @@ static int copy_state(less_ctx* c, const int32_t* inst, int32_t n, void* host, s
     e = to_host ? cudaMemcpyAsync(hostp, devp, nbytes, kind, s)
                 : cudaMemcpyAsync(devp, hostp, nbytes, kind, s);
   };
-  for (int i = 0; i < n; ++i) {
-    int32_t ii = inst[i];
-    if (ii < 0 || ii >= d.I) return LESS_ERR_INVALID_CONFIG;
-    char* rec = (char*)host + r.total * (size_t)i;
-    size_t I = ii;
-    cp(rec, c->a.count + I, 4);
-    cp(rec + r.pos, c->a.pos + I * d.Np, (size_t)d.N * 4);
-    cp(rec + r.acc, c->a.acc + I * d.Np, (size_t)d.N * 4);
-    cp(rec + r.K, c->a.kslots + I * d.N * d.D, (size_t)d.N * d.D * 2);
-    cp(rec + r.V, c->a.vslots + I * d.N * d.D, (size_t)d.N * d.D * 2);
-    cp(rec + r.psi, c->a.psic + I * d.N * d.R, (size_t)d.N * d.R * 4);
-    cp(rec + r.H, c->a.H + I * d.R * d.D, (size_t)d.R * d.D * 4);
-    cp(rec + r.z, c->a.z + I * d.R, (size_t)d.R * 4);
+  for (int i = 0; i < n; ++i)
+    if (inst[i] < 0 || inst[i] >= d.I) return LESS_ERR_INVALID_CONFIG;
+  // Records are packed / unpacked on the device, a batch at a time, in the host entry's staging
+  // buffers (free between calls): the instance list in stage_q, the records in stage_out; the host
+  // then sees one copy per batch.  Contexts whose staging buffer is smaller than one record (a handful
+  // of instances with many slots) copy field by field.
+  const size_t stage_bytes = (size_t)d.I * d.G * d.D * 4, list_cap = (size_t)d.I * d.G * d.D * 2 / 4;
+  const size_t per_batch = std::min(stage_bytes / r.total, list_cap);
+  if (per_batch >= 1 && r.total % 4 == 0) {
+    for (size_t i0 = 0; i0 < (size_t)n && e == cudaSuccess; i0 += per_batch) {
+      const int nb = (int)std::min(per_batch, (size_t)n - i0);
+      char* rec = (char*)host + r.total * i0;
+      e = cudaMemcpyAsync(c->a.stage_q, inst + i0, (size_t)nb * 4, cudaMemcpyHostToDevice, s);
+      if (e == cudaSuccess && !to_host) e = cudaMemcpyAsync(c->a.stage_out, rec, r.total * nb, cudaMemcpyHostToDevice, s);
+      if (e == cudaSuccess && launch_state_io(c, (const int32_t*)c->a.stage_q, nb, c->a.stage_out, r.total, to_host, s) != LESS_OK)
+        return LESS_ERR_CUDA;
+      if (e == cudaSuccess && to_host) e = cudaMemcpyAsync(rec, c->a.stage_out, r.total * nb, cudaMemcpyDeviceToHost, s);
+      // the staging buffers are reused by the next batch
+      if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    }
+  } else {
+    for (int i = 0; i < n; ++i) {
+      char* rec = (char*)host + r.total * (size_t)i;
+      size_t I = inst[i];
+      cp(rec, c->a.count + I, 4);
+      cp(rec + r.pos, c->a.pos + I * d.Np, (size_t)d.N * 4);
+      cp(rec + r.acc, c->a.acc + I * d.Np, (size_t)d.N * 4);
+      cp(rec + r.K, c->a.kslots + I * d.N * d.D, (size_t)d.N * d.D * 2);
+      cp(rec + r.V, c->a.vslots + I * d.N * d.D, (size_t)d.N * d.D * 2);
+      cp(rec + r.psi, c->a.psic + I * d.N * d.R, (size_t)d.N * d.R * 4);
+      cp(rec + r.H, c->a.H + I * d.R * d.D, (size_t)d.R * d.D * 4);
+      cp(rec + r.z, c->a.z + I * d.R, (size_t)d.R * 4);
+    }
   }
   // the position lives on the device (a captured step advances it without the host); the host
   // keeps a copy for less_position

@@ -266,6 +266,9 @@ int launch_decode(less_ctx* c, const void* q, const void* k, const void* v, void
 int launch_prefill_group(less_ctx* c, int layer0, int nlayers, int lj0, int layer_count, int S,
                          const void* Q, const void* K, const void* V, void* attn_out,
                          cudaStream_t s);
+// n state records between the arena and a device staging buffer (state_io.cu)
+int launch_state_io(less_ctx* c, const int32_t* inst_dev, int n, void* records_dev, size_t rec_bytes, bool to_records,
+                    cudaStream_t s);
 // the parallel form of one layer group (masked_tc.cu)
 int launch_masked_form(less_ctx* c, int layer0, int nlayers, int lj0, int layer_count, int S, const void* Q,
                        const void* K, const void* V, const int32_t* exact_until, void* out, cudaStream_t s);
