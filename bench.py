@@ -845,6 +845,8 @@ def measure_masked(args, ranks):
     dev, world = ranks.dev, ranks.world
     S = args.seq
     w = wl.CONFIGS[2].with_(batch=args.batch or 2, prompt=S, heavy=int(0.05 * S), recent=int(0.05 * S))
+    if args.group > 1:                                   # the same query heads over fewer KV heads
+        w = w.with_(heads=w.heads // args.group, group=args.group)
     K_steps, W_steps = args.steps, max(args.warmup, 3)
     Wt = wl.make_weights(w, dev)
     ctx = binding.from_workload(w, Wt, dev, max_prefill_layers=1, flags=binding.LESS_WITH_PARALLEL_FORM)
@@ -905,7 +907,7 @@ def measure_masked(args, ranks):
     rec = None
     if ranks.rank == 0:
         ms_step = st["ms_per_step"]
-        inst = w.batch * w.heads
+        inst = w.batch * w.heads * w.group               # sequences of query rows
         tokens = inst * S * world
         # flops of the entries the kernel has to form: 128 x 128 tiles that are not dead (a key tile all of
         # whose keys were discarded before a Q tile's first row is handled through its summed state)
@@ -914,10 +916,10 @@ def measure_masked(args, ranks):
         eu_pad[..., :S] = eu.long()
         death = eu_pad.view(w.batch, 1, w.heads, nt, 128).amax(-1)
         first_dead = torch.maximum((death + 127) // 128, torch.arange(nt, device=dev) + 1).clamp(max=nt)
-        live_pairs = int((first_dead - torch.arange(nt, device=dev)).sum().item())
+        live_pairs = int((first_dead - torch.arange(nt, device=dev)).sum().item()) * w.group
         live_frac = live_pairs / (inst * nt * (nt + 1) / 2)
         fl = {"masked_out": live_pairs * 128 * 128 * (4 * w.head_dim + 2 * w.rank),
-              "psi": inst * S * 2 * (2 * w.head_dim * w.hidden + 2 * w.hidden * w.rank + w.rank * w.rank)}
+              "psi": (inst + w.batch * w.heads) * S * (2 * w.head_dim * w.hidden + 2 * w.hidden * w.rank + w.rank * w.rank)}
         kt = {k: (prof[k][0] / prof[k][1] if prof[k][1] else 0.0) for k in prof}
         kt["psi"] *= 2                                   # psi and phi launches are booked under the same id
         kt["masked_pack"] *= 3                           # operand pack, tile states, running sums
@@ -930,7 +932,9 @@ def measure_masked(args, ranks):
                "ms_per_step_min": st["ms_per_step_min"], "blocks": st["blocks"],
                "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
                "dtype": "f16 inputs, f32 accumulate", "data": "synthetic",
-               "config": {"workload": f"parallel form (B={w.batch}, {w.heads} heads, sequences of {S}, one layer per step, R={w.rank})",
+               "config": {"workload": f"parallel form (B={w.batch}, {w.heads * w.group} query heads"
+                                      + (f" over {w.heads} KV heads" if w.group > 1 else "")
+                                      + f", sequences of {S}, one layer per step, R={w.rank})",
                           "instances_per_step": inst, "live_tile_fraction": live_frac, "l2": "inputs, operands and output of a step exceed the 126 MB L2"
                           if inst * S * 1300 > 126e6 else "a step's data fit the L2"},
                "clocks": clocks,

@@ -169,10 +169,12 @@ int less_prefill(less_ctx* ctx, int32_t layer_begin, int32_t layer_count, int32_
  * policy discarded key j (so exact_until[j] > j when a token attends to itself), INT32_MAX
  * for a key that is never discarded; the caller obtains it from the policy (e.g. the
  * evicted_pos record of less_decode_step).
- * Q, K, V as in less_prefill (seq_len <= max_prompt); out: device fp32 [B, layer_count, H,
- * seq_len, D].  Reads the context's weights, touches no cache or state; needs
- * LESS_WITH_PARALLEL_FORM at creation, group <= 1 and the tensor-core kernels
- * (hidden in {64, 128, 256, 512}), else LESS_ERR_INVALID_CONFIG. */
+ * Q, K, V as in less_prefill (seq_len <= max_prompt); out: device fp32, Q's shape
+ * [B, layer_count, H * group, seq_len, D].  With group > 1 the query heads of a group read
+ * the same K, V, psi(K) and exact_until (the cache belongs to the KV head); each has its own
+ * phi and its own normalisation.  Reads the context's weights, touches no cache or state;
+ * needs LESS_WITH_PARALLEL_FORM at creation, head_dim 128 with group in {1, 2, 4, 8} and the
+ * tensor-core kernels (hidden in {64, 128, 256, 512}), else LESS_ERR_INVALID_CONFIG. */
 int less_masked_attention(less_ctx* ctx, int32_t layer_begin, int32_t layer_count, int32_t seq_len,
                           const void* Q, const void* K, const void* V, const int32_t* exact_until,
                           void* out, void* cuda_stream);

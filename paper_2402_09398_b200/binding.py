@@ -268,8 +268,9 @@ class LessContext:
                             _stream_ptr(stream)), "less_prefill")
 
     def masked_attention(self, Q, K, V, exact_until, layer_begin=0, out=None, stream=None):
-        """The parallel form: Q, K, V fp16 [B, Lc, H, S, D], exact_until int32 [B, Lc, H, S]."""
-        B, Lc, H, S, D = Q.shape
+        """The parallel form: Q fp16 [B, Lc, H * group, S, D], K, V fp16 [B, Lc, H, S, D], exact_until int32
+        [B, Lc, H, S]; the result has Q's shape."""
+        B, Lc, _, S, D = Q.shape
         assert Q.dtype == K.dtype == V.dtype == torch.float16 and exact_until.dtype == torch.int32
         assert Q.is_contiguous() and K.is_contiguous() and V.is_contiguous() and exact_until.is_contiguous()
         if out is None:

@@ -111,10 +111,10 @@ size_t carve(const Dims& d, char* base, Arena* a) {
   t.ws_bx = (uint4*)take(Iw * G * (size_t)d.Sbx * 16);
   t.ws_pmax = (int32_t*)take(Iw * 4);
   const size_t St = (d.flags & LESS_WITH_PARALLEL_FORM) ? d.St : 0;
-  t.ws_phi = (float*)take(St ? Iw * Sp * R * 4 : 0);
-  t.ws_phiop = (unsigned char*)take(Iw * St * 8192);
+  t.ws_phi = (float*)take(St ? Iw * G * Sp * R * 4 : 0);      // the query side of the parallel form: per query head
+  t.ws_phiop = (unsigned char*)take(Iw * G * St * 8192);
   t.ws_psiop = (unsigned char*)take(Iw * St * 8192);
-  t.ws_g = (float*)take(Iw * St * 128 * 4);
+  t.ws_g = (float*)take(Iw * G * St * 128 * 4);
   t.ws_eu = (int32_t*)take(Iw * St * 128 * 4);
   t.ws_ht = (float*)take(Iw * St * (R * D + R) * 4);
   t.ws_hsum = (float*)take(Iw * St * (R * D + R) * 4);
@@ -284,13 +284,13 @@ int less_masked_attention(less_ctx* c, int32_t layer_begin, int32_t layer_count,
                           const void* Q, const void* K, const void* V, const int32_t* exact_until,
                           void* out, void* stream) {
   if (!c) return LESS_ERR_NULL_POINTER;
-  if (!(c->d.flags & LESS_WITH_PARALLEL_FORM) || c->d.G > 1 || c->d.general) return LESS_ERR_INVALID_CONFIG;
+  if (!(c->d.flags & LESS_WITH_PARALLEL_FORM) || c->d.general) return LESS_ERR_INVALID_CONFIG;
   if (layer_begin < 0 || layer_count < 1 || layer_begin + layer_count > c->d.L)
     return LESS_ERR_BAD_LAYER_RANGE;
   if (seq_len < 0) return LESS_ERR_INVALID_CONFIG;
   if (seq_len > c->cfg.max_prompt) return LESS_ERR_PROMPT_TOO_LONG;
   if (seq_len == 0) return LESS_OK;
-  if ((int64_t)c->d.B * layer_count * c->d.Hd * seq_len > 0x7fffffffLL) return LESS_ERR_PROMPT_TOO_LONG;
+  if ((int64_t)c->d.B * layer_count * c->d.Hd * c->d.G * seq_len > 0x7fffffffLL) return LESS_ERR_PROMPT_TOO_LONG;
   if (!Q || !K || !V || !exact_until || !out) return LESS_ERR_NULL_POINTER;
   if (misaligned(Q) || misaligned(K) || misaligned(V) || misaligned(out) || ((uintptr_t)exact_until & 3))
     return LESS_ERR_MISALIGNED;

@@ -46,10 +46,10 @@ struct Arena {
   float* ws_psi;     // [Iw][Sp][R]  psi(k_j) of every prompt token
   int32_t* ws_pmax;  // [Iw]        bit pattern of max psi over the instance's prompt tokens (scales the state build's fp16 operand)
   // parallel form only (LESS_WITH_PARALLEL_FORM); St = 128-row tiles of max_prompt
-  float* ws_phi;     // [Iw][Sp][R]  phi(q_i) of every row
-  unsigned char* ws_phiop;  // [Iw][St][8 KB]  phi as fp16 hi / lo operand tiles
+  float* ws_phi;     // [Iw * G][Sp][R]  phi(q_i) of every row of every query head
+  unsigned char* ws_phiop;  // [Iw * G][St][8 KB]  phi as fp16 hi / lo operand tiles
   unsigned char* ws_psiop;  // [Iw][St][8 KB]  psi likewise
-  float* ws_g;       // [Iw][St*128]  per row: log2 of (kernel value / value of the scaled operands)
+  float* ws_g;       // [Iw * G][St*128]  per row: log2 of (kernel value / value of the scaled operands)
   int32_t* ws_eu;    // [Iw][St*128]  exact_until, padded with zeros
   float* ws_ht;      // [Iw][St][R*D + R]  H, z of every key tile
   float* ws_hsum;    // [Iw][St][R*D + R]  per Q tile: H, z summed over the key tiles dead for it

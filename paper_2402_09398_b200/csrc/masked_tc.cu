@@ -23,6 +23,8 @@
 // rounded to fp16 for P V, whatever share of the plain softmax's mass the policy has left exact
 // (a row whose dominant key has been discarded keeps ~1e-6 of it: formed against the plain
 // normaliser its entries would sink into fp16's subnormals).
+// With grouped query heads (Section 3.2, multi-query attention) the query heads of a group share the
+// key side (K, V, psi, exact_until, the dead-tile sums); each has its own Q rows, phi and output.
 // Every wait is bounded (pipeline.cuh).
 #include "prefill.cuh"
 #include "tc_common.cuh"
@@ -43,15 +45,16 @@ constexpr float kMfExpScale = 0.12751743074602468f; // log2(e) / sqrt(128)
 
 struct MfParams {
   const int32_t* exact_until;   // [B, layer_count, Hd, S]
-  float* out;                   // [B, layer_count, Hd, S, D]
+  float* out;                   // [B, layer_count, Hd * grp, S, D]
   int St;                       // operand tiles per instance in the workspace
-  const float* phi;             // [Iw][Sp][R] phi(q_i), unscaled
+  const float* phi;             // [Iw * grp][Sp][R] phi(q_i), unscaled
   const float* hsum;            // [Iw][St][R*D + R] per Q tile: H, z summed over the key tiles that are dead for it
   const int32_t* bucket;        // [Iw][St] first Q tile for which a key tile is dead (all its keys discarded before it)
 };
 
 // ------------------------------------------------------------------------------------------- //
-// Operand tiles and row constants.  One CTA = one 128-row tile of one instance, one thread per row.
+// Operand tiles and row constants.  One CTA = one 128-row tile of one query head, one thread per row;
+// the group's first query head also writes the key side (psi operand, exact_until).
 // ------------------------------------------------------------------------------------------- //
 __device__ __forceinline__ float pow2_scale_exponent(float vmax) {
   // exponent e with vmax * 2^e in [8192, 16384): hi parts far from fp16's overflow, lo parts far from its underflow
@@ -81,7 +84,9 @@ __device__ __forceinline__ void split_row(const float* x, float scale, uint4* hi
 
 template <int R>
 __global__ void __launch_bounds__(MF_TILE) masked_pack_kernel(PfParams p, MfParams mf) {
-  const int T = blockIdx.x, g = blockIdx.y, r = threadIdx.x;
+  const int T = blockIdx.x, gq = blockIdx.y, r = threadIdx.x;
+  const int g = gq / p.grp;                              // the KV instance of this query head
+  const bool first = gq == g * p.grp;
   const int i = T * MF_TILE + r;
   const bool valid = i < p.S;
   const InstMap im = map_instance(p, g);
@@ -92,7 +97,7 @@ __global__ void __launch_bounds__(MF_TILE) masked_pack_kernel(PfParams p, MfPara
 #pragma unroll
   for (int e = 0; e < R; ++e) ph[e] = ps[e] = 0.f;
   if (valid) {
-    const float4* a = reinterpret_cast<const float4*>(p.a.ws_phi + ((size_t)g * p.Sp + i) * R);
+    const float4* a = reinterpret_cast<const float4*>(p.a.ws_phi + ((size_t)gq * p.Sp + i) * R);
     const float4* b = reinterpret_cast<const float4*>(p.a.ws_psi + ((size_t)g * p.Sp + i) * R);
 #pragma unroll
     for (int e = 0; e < R / 4; ++e) {
@@ -114,24 +119,22 @@ __global__ void __launch_bounds__(MF_TILE) masked_pack_kernel(PfParams p, MfPara
   uint4 fh[R / 8], fl[R / 8], sh_[R / 8], sl[R / 8];
   split_row<R>(ph, exp2f(ephi), fh, fl);
   split_row<R>(ps, exp2f(epsi), sh_, sl);
-  const size_t tile = ((size_t)g * mf.St + T) * MF_OP_BYTES;
   const int off = (r >> 3) * 128 + (r & 7) * 16;
-  uint4* fo = reinterpret_cast<uint4*>(p.a.ws_phiop + tile + off);
-  uint4* so = reinterpret_cast<uint4*>(p.a.ws_psiop + tile + off);
+  uint4* fo = reinterpret_cast<uint4*>(p.a.ws_phiop + ((size_t)gq * mf.St + T) * MF_OP_BYTES + off);
+  uint4* so = reinterpret_cast<uint4*>(p.a.ws_psiop + ((size_t)g * mf.St + T) * MF_OP_BYTES + off);
   const uint4 zero = make_uint4(0, 0, 0, 0);
   constexpr int CH = 2048 / 16;                        // chunk stride in uint4
   if (R == 8) {
     fo[0] = fh[0]; fo[CH] = fl[0]; fo[2 * CH] = fh[0]; fo[3 * CH] = zero;
-    so[0] = sh_[0]; so[CH] = sh_[0]; so[2 * CH] = sl[0]; so[3 * CH] = zero;
+    if (first) { so[0] = sh_[0]; so[CH] = sh_[0]; so[2 * CH] = sl[0]; so[3 * CH] = zero; }
   } else {
     fo[0] = fh[0]; fo[CH] = fh[R / 8 - 1]; fo[2 * CH] = fl[0]; fo[3 * CH] = fl[R / 8 - 1];
-    so[0] = sh_[0]; so[CH] = sh_[R / 8 - 1]; so[2 * CH] = sl[0]; so[3 * CH] = sl[R / 8 - 1];
+    if (first) { so[0] = sh_[0]; so[CH] = sh_[R / 8 - 1]; so[2 * CH] = sl[0]; so[3 * CH] = sl[R / 8 - 1]; }
   }
 
   // what turns a scaled kernel value back into phi(q_i) psi(k_j)^T, as a power of two; the key's mask
-  const size_t row = (size_t)g * mf.St * MF_TILE + i;
-  p.a.ws_g[row] = -(ephi + epsi);
-  p.a.ws_eu[row] = valid ? mf.exact_until[im.in_row0 + i] : 0;
+  p.a.ws_g[(size_t)gq * mf.St * MF_TILE + i] = -(ephi + epsi);
+  if (first) p.a.ws_eu[(size_t)g * mf.St * MF_TILE + i] = valid ? mf.exact_until[im.in_row0 + i] : 0;
 }
 
 // ------------------------------------------------------------------------------------------- //
@@ -210,7 +213,7 @@ __global__ void __launch_bounds__(256) masked_prefix_kernel(int tiles, int St, c
 }
 
 // ------------------------------------------------------------------------------------------- //
-// One CTA = one 128-row Q tile of one instance; the key tiles 0 .. diagonal that are not dead stream past it.
+// One CTA = one 128-row Q tile of one query head; the key tiles 0 .. diagonal that are not dead stream past it.
 // ------------------------------------------------------------------------------------------- //
 struct MfShared {
   uint64_t res_full;
@@ -254,13 +257,16 @@ __global__ void __launch_bounds__(MF_THREADS) masked_out_tc_kernel(const __grid_
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int tiles = (p.S + MF_TILE - 1) / MF_TILE;
   const int tile = tiles - 1 - (int)blockIdx.x;                    // long rows first
-  const int g = blockIdx.y;
+  const int gq = blockIdx.y, g = gq / p.grp;                      // query head, its KV instance
   const InstMap im = map_instance(p, g);
+  const QueryMap qm = map_query(p, gq);
   const int i0 = tile * MF_TILE;
   const int ntile = tile + 1;                                      // key tiles 0 .. tile (the last holds the diagonal)
   int32_t* status = p.a.status;
-  const size_t op0 = (size_t)g * mf.St * MF_OP_BYTES;              // this instance's operand tiles
-  const size_t rc0 = (size_t)g * mf.St * MF_TILE;                  // ... and row constants
+  const size_t op0 = (size_t)g * mf.St * MF_OP_BYTES;              // the KV instance's operand tiles (psi)
+  const size_t rc0 = (size_t)g * mf.St * MF_TILE;                  // ... and exact_until
+  const size_t op0q = (size_t)gq * mf.St * MF_OP_BYTES;            // the query head's operand tiles (phi)
+  const size_t rc0q = (size_t)gq * mf.St * MF_TILE;                // ... and row constants
 
   if (tid == 0) {
     mbar_init(&sh->res_full, 1);
@@ -309,11 +315,11 @@ __global__ void __launch_bounds__(MF_THREADS) masked_out_tc_kernel(const __grid_
   if (warp == 0) {
     // ---------------- producer: Q and its phi operand, then K + psi operand + exact_until per key tile ----------------
     if (lane == 0) {
-      const int row0 = (int)(im.in_row0 + i0);
+      const int row0 = (int)(qm.q_row0 + i0);
       mbar_expect_tx(&sh->res_full, MF_TILE_BYTES + MF_OP_BYTES);
       tma_load_2d(qres, &tm_q, 0, row0, &sh->res_full);
       tma_load_2d(qres + MF_TILE_BYTES / 2, &tm_q, 64, row0, &sh->res_full);
-      bulk_g2s(phires, p.a.ws_phiop + op0 + (size_t)tile * MF_OP_BYTES, MF_OP_BYTES, &sh->res_full);
+      bulk_g2s(phires, p.a.ws_phiop + op0q + (size_t)tile * MF_OP_BYTES, MF_OP_BYTES, &sh->res_full);
       uint32_t s = 0, ph = 0;
       int u = 0;                                         // live tiles issued so far, both sweeps
       for (int sweep = 0; sweep < 2 && !*abortp; ++sweep)
@@ -429,7 +435,7 @@ __global__ void __launch_bounds__(MF_THREADS) masked_out_tc_kernel(const __grid_
     const uint32_t lane_addr = tmem + ((uint32_t)(quad * 32) << 16);
     // sweep 1: the row's largest exact dot product and largest kernel value (scaled operands);
     // sweep 2: P against the largest entry, so that every entry is <= 1 and the largest is 1
-    const float lscale = p.a.ws_g[rc0 + i];            // log2 of (true kernel value / scaled kernel value)
+    const float lscale = p.a.ws_g[rc0q + i];            // log2 of (true kernel value / scaled kernel value)
     const bool live = i < p.S;
     float mx = -INFINITY, ml = 0.f;
     float nb = 0.f, gi = 0.f, rsum = 0.f, rsum2 = 0.f;
@@ -557,7 +563,7 @@ __global__ void __launch_bounds__(MF_THREADS) masked_out_tc_kernel(const __grid_
       float dz = 0.f;
 #pragma unroll
       for (int q = 0; q < R; ++q) {
-        ph[q] = mf.phi[((size_t)g * p.Sp + i) * R + q] * f;
+        ph[q] = mf.phi[((size_t)gq * p.Sp + i) * R + q] * f;
         dz = fmaf(ph[q], __ldg(hs + R * kHeadDim + q), dz);
       }
       total += dz;
@@ -578,7 +584,7 @@ __global__ void __launch_bounds__(MF_THREADS) masked_out_tc_kernel(const __grid_
     // ---- the finished rows: O[row][32 columns of this warp] / r_i ----
     wait_or_give_up(&sh->o_full, 0, abortp, status, 122);
     tc_fence_after_sync();
-    float* orow = mf.out + (im.in_row0 + i) * kHeadDim + part * 32;
+    float* orow = mf.out + (qm.q_row0 + i) * kHeadDim + part * 32;
     {
       uint32_t o[32];
       tmem_ld32(lane_addr + ocol + part * 32, o);
@@ -615,8 +621,8 @@ int launch_masked_form(less_ctx* c, int layer0, int nl, int lj0, int layer_count
   p.B = d.B; p.L = d.L; p.Hd = d.Hd; p.N = d.N; p.Np = d.Np;
   p.heavy = d.heavy; p.recent = d.recent; p.Rp = d.Rp;
   p.flags = d.flags;
-  p.grp = 1;
-  const int G = d.B * nl * d.Hd;
+  p.grp = d.G;
+  const int G = d.B * nl * d.Hd, Gq = G * d.G;       // KV instances, query heads
   // token splits of the MLP kernel, as in the prompt phase
   int split_tokens = 1024;
   while (split_tokens > 128 && (long long)G * ((S + split_tokens - 1) / split_tokens) < 148) split_tokens >>= 1;
@@ -633,13 +639,13 @@ int launch_masked_form(less_ctx* c, int layer0, int nl, int lj0, int layer_count
   if (cudaMemsetAsync(c->a.ws_pmax, 0, (size_t)G * 4, s) != cudaSuccess) return fail_cuda("clearing the psi maxima");
   rc = launch_psi_tc(c, p, G, s);
   if (rc != LESS_OK) return rc;
-  rc = launch_phi_tc(c, p, G, s, c->a.ws_phi);
+  rc = launch_phi_tc(c, p, Gq, s, c->a.ws_phi);
   if (rc != LESS_OK) return rc;
   const int tiles = (S + MF_TILE - 1) / MF_TILE;
   {
     LaunchScope scope(c, LESS_KERNEL_MASKED_PACK, s);
-    if (d.R == 8) masked_pack_kernel<8><<<dim3(tiles, G), MF_TILE, 0, s>>>(p, mf);
-    else masked_pack_kernel<16><<<dim3(tiles, G), MF_TILE, 0, s>>>(p, mf);
+    if (d.R == 8) masked_pack_kernel<8><<<dim3(tiles, Gq), MF_TILE, 0, s>>>(p, mf);
+    else masked_pack_kernel<16><<<dim3(tiles, Gq), MF_TILE, 0, s>>>(p, mf);
   }
   mf.phi = c->a.ws_phi;
   mf.hsum = c->a.ws_hsum;
@@ -657,7 +663,7 @@ int launch_masked_form(less_ctx* c, int layer0, int nl, int lj0, int layer_count
   }
   CUtensorMap tq, tk, tv;
   const uint64_t rows = (uint64_t)d.B * layer_count * d.Hd * S;
-  if (!make_tmap_f16_2d(&tq, p.Q, rows, kHeadDim, kHeadDim * 2, MF_TILE) ||
+  if (!make_tmap_f16_2d(&tq, p.Q, rows * d.G, kHeadDim, kHeadDim * 2, MF_TILE) ||
       !make_tmap_f16_2d(&tk, p.K, rows, kHeadDim, kHeadDim * 2, MF_TILE) ||
       !make_tmap_f16_2d(&tv, p.V, rows, kHeadDim, kHeadDim * 2, MF_TILE))
     return fail_cuda("tensor maps of Q / K / V");
@@ -667,11 +673,11 @@ int launch_masked_form(less_ctx* c, int layer0, int nl, int lj0, int layer_count
   if (d.R == 8) {
     if (cudaFuncSetAttribute(masked_out_tc_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
       return fail_cuda("shared memory opt-in of masked_out_tc_kernel");
-    masked_out_tc_kernel<8><<<dim3(tiles, G), MF_THREADS, smem, s>>>(tq, tk, tv, p, mf);
+    masked_out_tc_kernel<8><<<dim3(tiles, Gq), MF_THREADS, smem, s>>>(tq, tk, tv, p, mf);
   } else {
     if (cudaFuncSetAttribute(masked_out_tc_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
       return fail_cuda("shared memory opt-in of masked_out_tc_kernel");
-    masked_out_tc_kernel<16><<<dim3(tiles, G), MF_THREADS, smem, s>>>(tq, tk, tv, p, mf);
+    masked_out_tc_kernel<16><<<dim3(tiles, Gq), MF_THREADS, smem, s>>>(tq, tk, tv, p, mf);
   }
   return check_launch("the parallel-form kernels");
 }

@@ -121,7 +121,13 @@ __global__ void __launch_bounds__(PT_THREADS) psi_tc_kernel(const __grid_constan
 
   const int tid = threadIdx.x, warp = tid >> 5;
   const int split = blockIdx.x, g = blockIdx.y;
-  const InstMap im = map_instance(p, g);
+  // phi belongs to the query head: g then counts query heads (grp per KV instance), each with its own
+  // rows of Q and its own weights
+  InstMap im = map_instance(p, mp.is_phi ? g / p.grp : g);
+  if (mp.is_phi) {
+    im.in_row0 = map_query(p, g).q_row0;
+    im.lh = im.lh * p.grp + g % p.grp;
+  }
   const int jbeg = split * p.split_tokens, jend = min(p.S, jbeg + p.split_tokens);
   const int ntiles = (jend - jbeg + PT_TILE - 1) / PT_TILE;
 
@@ -451,17 +457,18 @@ static int launch_variant(const CUtensorMap& tk, const CUtensorMap& tv, const CU
   return check_launch("psi_tc_kernel");
 }
 
-// x: the rows the map is applied to ([B, layer_count, Hd, S, D]); with_state: psi fused with the
+// x: the rows the map is applied to ([B, layer_count, Hd, S, D]; for phi, Q with Hd * group heads); with_state: psi fused with the
 // prompt state build (needs the kept / discarded map of select_kernel and V)
 static int launch_map_tc(less_ctx* c, const PfParams& p, int G, cudaStream_t s, const __half* x, const void* w1,
                          const PtMap& mp, bool with_state) {
   const Dims& d = c->d;
   CUtensorMap tmap_k, tmap_v, tmap_w1;
+  const uint64_t hg = mp.is_phi ? (uint64_t)p.grp : 1;            // query heads per KV head where the map is phi
   const uint64_t rows = (uint64_t)d.B * p.layer_count * d.Hd * p.S;
-  if (!make_tmap_f16_2d(&tmap_k, x, rows, kHeadDim, kHeadDim * 2, PT_TILE)) return fail_cuda("tensor map of K");
-  if (!make_tmap_f16_2d(&tmap_v, with_state ? p.V : x, rows, kHeadDim, kHeadDim * 2, PT_TILE))
+  if (!make_tmap_f16_2d(&tmap_k, x, rows * hg, kHeadDim, kHeadDim * 2, PT_TILE)) return fail_cuda("tensor map of K");
+  if (!make_tmap_f16_2d(&tmap_v, with_state ? p.V : x, with_state ? rows : rows * hg, kHeadDim, kHeadDim * 2, PT_TILE))
     return fail_cuda("tensor map of V");
-  if (!make_tmap_f16_2d(&tmap_w1, w1, (uint64_t)d.L * d.Hd * kHeadDim, d.Rp, (uint64_t)d.Rp * 2, kHeadDim))
+  if (!make_tmap_f16_2d(&tmap_w1, w1, (uint64_t)d.L * d.Hd * hg * kHeadDim, d.Rp, (uint64_t)d.Rp * 2, kHeadDim))
     return fail_cuda("tensor map of W1");
   const size_t smem = (size_t)(d.Rp / 64) * 16384 + PT_KBYTES + (size_t)d.Rp * PT_W2N * 2 +
                       (with_state ? PT_KBYTES + (size_t)PT_TILE * 2 * d.R * 2 + 4096 : 0) + sizeof(PtShared) + 64;
@@ -490,7 +497,7 @@ int launch_psi_state_tc(less_ctx* c, const PfParams& p, int G, cudaStream_t s) {
   return launch_map_tc(c, p, G, s, p.K, p.w_psi1, mp, true);
 }
 
-// phi(q_i) of every row of Q into `out` [Iw][Sp][R] (one query head per KV head)
+// phi(q_i) of every row of Q into `out` [G][Sp][R]; G counts query heads (p.grp per KV instance)
 int launch_phi_tc(less_ctx* c, const PfParams& p, int G, cudaStream_t s, float* out) {
   PtMap mp;
   mp.w2 = (const __half*)c->w.w_phi2; mp.w3 = nullptr; mp.out = out; mp.pmax = nullptr; mp.is_phi = 1;

@@ -774,6 +774,70 @@ def test_parallel_form_rows_equal_the_decode_steps():
     ctx.close()
 
 
+@pytest.mark.parametrize("group,rank,S,kind", [(2, 8, 300, "random"), (4, 16, 257, "random"), (8, 8, 131, "banded"),
+                                               (4, 8, 1153, "banded"), (2, 16, 128, "at_once")])
+def test_parallel_form_with_grouped_query_heads(group, rank, S, kind):
+    """Every query head of a group against the oracle's single-head parallel form on the KV head's
+    K, V and schedule, with the query head's own Q rows and phi (Section 3.2, multi-query attention)."""
+    from paper_2402_09398_b200 import binding
+    from oracle import less_oracle as lo
+    import harness
+    w = small(60 + group + rank, prompt=S, rank=rank, weight_std=0.2, group=group, heads=2)
+    ctx, W = _setup(w, flags=binding.LESS_WITH_PARALLEL_FORM)
+    Q, K, V = wl.make_prompt(w, 0, w.layers, DEV)
+    assert Q.shape[2] == w.heads * group
+    eu = _schedule(w, kind, S, seed=S + group)
+    out = ctx.masked_attention(Q, K, V, eu.to(DEV))
+    torch.cuda.synchronize()
+    assert ctx.poll_status() == 0 and out.shape == Q.shape
+    worst = 0.0
+    for inst in range(w.instances):
+        b, layer, head = wl.instance_coords(w, inst)
+        psi_w = [W[n][layer, head].double().numpy() for n in ("w_psi1", "w_psi2", "w_psi3")]
+        Kh, Vh = (t[b, layer, head].double().cpu().numpy() for t in (K, V))
+        for g in range(group):
+            hq = head * group + g
+            phi_fn, psi_fn = lo.make_mlp_maps(W["w_phi1"][layer, hq].double().numpy(),
+                                              W["w_phi2"][layer, hq].double().numpy(), *psi_w)
+            ref, _ = lo.masked_parallel_attention(Q[b, layer, hq].double().cpu().numpy(), Kh, Vh,
+                                                  eu[b, layer, head].numpy(), phi_fn, psi_fn)
+            err = float(np.max(np.abs(out[b, layer, hq].double().cpu().numpy() - ref)))
+            worst = max(worst, err)
+            assert err <= harness.OUT_TOL, f"inst {inst} query head {g}: parallel form max-abs {err}"
+    print("grouped parallel form", group, rank, S, kind, worst)
+    ctx.close()
+
+
+def test_grouped_parallel_form_rows_equal_the_decode_steps():
+    """The identity of the single-head test with four query heads per KV head: the schedule comes
+    from the grouped decode steps' own evictions."""
+    from paper_2402_09398_b200 import binding
+    S, G = 140, 4
+    w = small(27, prompt=0, steps=S, heavy=12, recent=12, weight_std=0.2, group=G)
+    ctx, W = _setup(w, flags=binding.LESS_WITH_PARALLEL_FORM, max_prompt=S)
+    qs, ks, vs, outs = [], [], [], []
+    eu = torch.full((w.batch, w.layers, w.heads, S), 2**31 - 1, dtype=torch.int32)
+    ev = torch.empty(w.instances, dtype=torch.int32, device=DEV)
+    for t in range(S):
+        q, k, v = wl.make_decode_inputs(w, t, DEV)
+        outs.append(ctx.decode_step(q, k, v, evicted_pos=ev).clone())
+        e = ev.cpu().reshape(w.batch, w.layers, w.heads)
+        idx = torch.nonzero(e >= 0, as_tuple=True)
+        eu[idx[0], idx[1], idx[2], e[idx].long()] = t + 1
+        qs.append(q); ks.append(k); vs.append(v)
+    Q, K, V = (torch.stack(x, dim=3).contiguous() for x in (qs, ks, vs))
+    assert Q.shape == (w.batch, w.layers, w.heads * G, S, w.head_dim)
+    seq = torch.stack(outs, dim=3)
+    par = ctx.masked_attention(Q, K, V, eu.to(DEV))
+    torch.cuda.synchronize()
+    assert ctx.poll_status() == 0
+    assert (eu != 2**31 - 1).sum() == (S - w.slots) * w.instances
+    err = float((par - seq).abs().max())
+    print("grouped parallel vs sequential", err)
+    assert err <= 2e-3
+    ctx.close()
+
+
 def test_parallel_form_needs_its_flag_and_scaled_maps():
     from paper_2402_09398_b200 import binding
     w = small(28, prompt=200, weight_std=0.2)
