@@ -939,7 +939,8 @@ def measure_masked(args, ranks):
                           if inst * S * 1300 > 126e6 else "a step's data fit the L2"},
                "clocks": clocks,
                "e2e": {"value": tokens / (ms_e2e * 1e-3), "unit": "head-tokens/s",
-                       "h2d_bytes_per_step": 3 * Q.numel() * 2 + eu.numel() * 4, "d2h_bytes_per_step": out.numel() * 4},
+                       "h2d_bytes_per_step": (Q.numel() + 2 * Kp.numel()) * 2 + eu.numel() * 4,
+                       "d2h_bytes_per_step": out.numel() * 4},
                "gpu_launches": int(launches),
                "roofline": {"bound": "tensor", "kernel": "masked_out_tc_kernel" if dominant == "masked_out" else dominant,
                             "achieved": ach, "peak": peak, "unit": "TFLOP/s", "frac": ach / peak, "peak_kind": kind,
