@@ -33,7 +33,11 @@
  *     LESS_FEATURE_CTAS=n (cap on the persistent CTAs of the tensor-core feature kernels),
  *     LESS_HEAD_COUNTERS=1 (with more instances than fit the GPU at once and more than 8 batch rows:
  *     the decode kernel starts behind the feature-map kernel and each of its CTAs waits for its own
- *     head's feature maps through a per-head counter; measured neutral, off by default).
+ *     head's feature maps through a per-head counter; measured neutral, off by default),
+ *     LESS_SMALL_STEP=0|1 (a decode step as ONE launch - a thread-block cluster per head splits the
+ *     two MLPs and runs the step of each batch row - never / whenever the shape allows: head_dim 128,
+ *     group 1, at most 4 batch rows, hidden in {128, 256, 512}, the state in use; by default when
+ *     layers x heads x (batch + 4) CTAs fit the GPU's multiprocessors at once).
  */
 #ifndef LESS_B200_H
 #define LESS_B200_H

@@ -3,6 +3,8 @@
 //   decode_kernel       scores over the live slots, Eq. 3, H2O score update,
 //                       argmin eviction, Eq. 4 / Eq. 5, in-place slot overwrite
 //   decode_group_*      the same step for G query heads per KV head
+//   small_step_kernel   both in one launch for workloads of a few heads: a cluster of CTAs per head
+//                       splits the two MLPs, then one CTA per batch row runs the decode step
 #include <stdio.h>
 
 #include "feature_gemv.cuh"
@@ -123,6 +125,7 @@ struct DecParams {
   uint32_t flag_target[2];     // counter values that mean "this step's phi / psi of the head are written"
   int head_major;              // CTAs numbered (layer-head, batch row) instead of by instance
   int lh0;                     // first (layer, KV head) of this launch (head-major numbering only)
+  int done_ctas;               // CTAs of this launch that run a decode step (captured steps count themselves out)
 };
 
 __device__ __forceinline__ float block_max(float v, float* red) {
@@ -157,11 +160,12 @@ __device__ __forceinline__ float block_sum(float v, float* red) {
 // last one advances it for the next replay (one contended atomic per CTA: the price of replaying
 // without the host, paid only by captured steps).
 template <bool kCaptured>
-__device__ __forceinline__ void step_done(int32_t* tpos, int t) {
+__device__ __forceinline__ void step_done(const DecParams& p) {
+  int32_t* tpos = p.a.tpos;
   if (threadIdx.x != 0) return;
   if (!kCaptured) {
-    if (blockIdx.x == 0) tpos[0] = t + 1;
-  } else if (atomicAdd(tpos + 1, 1) == (int)gridDim.x - 1) {   // every thread read the position barriers ago
+    if (blockIdx.x == 0) tpos[0] = p.t + 1;
+  } else if (atomicAdd(tpos + 1, 1) == p.done_ctas - 1) {      // every thread read the position barriers ago
     tpos[1] = 0;
     atomicAdd(tpos, 1);
   }
@@ -291,7 +295,7 @@ __device__ __forceinline__ void decode_tail(const DecParams& p, size_t inst, int
           }
           if (tid < R) zb[tid] += __ldcg(psn + tid);
         }
-        step_done<kCaptured>(p.a.tpos, p.t);
+        step_done<kCaptured>(p);
         return;
       }
     }
@@ -305,7 +309,7 @@ __device__ __forceinline__ void decode_tail(const DecParams& p, size_t inst, int
         set_status(p.a.status, kStatusBounds, 2);
         if (p.evicted_pos) p.evicted_pos[inst] = -1;
       }
-      step_done<kCaptured>(p.a.tpos, p.t);
+      step_done<kCaptured>(p);
       return;
     }
     if (tid == 0 && p.evicted_pos) p.evicted_pos[inst] = vpos;
@@ -334,7 +338,7 @@ __device__ __forceinline__ void decode_tail(const DecParams& p, size_t inst, int
   if (tid == 32) { posb[slot] = t_now; accb[slot] = p_new; }
   if (tid >= 64 && tid < 64 + R)
     p.a.psic[(inst * (size_t)N + slot) * R + (tid - 64)] = use_state ? __ldcg(p.a.psi_k + inst * R + (tid - 64)) : 0.f;
-  step_done<kCaptured>(p.a.tpos, p.t);
+  step_done<kCaptured>(p);
 }
 
 // Eq. 3 of each of the G query heads over the KV head's shared H, z, from the heads' partial
@@ -404,7 +408,7 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_kernel(DecParams p) {
   int n = p.a.count[inst];
   if (n < 0 || n > N) {                            // refuse a corrupt count, touch nothing
     if (tid == 0) set_status(p.a.status, kStatusBounds, 1);
-    step_done<kCaptured>(p.a.tpos, p.t);
+    step_done<kCaptured>(p);
     return;
   }
   const bool use_state = !(p.flags & LESS_NO_STATE);
@@ -510,6 +514,389 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_kernel(DecParams p) {
 }
 
 // --------------------------------------------------------------------------- //
+// A whole step in one launch, for workloads of a few heads (Algorithm 1 from phi(q_t), psi(k_t) to
+// the slot overwrite).  With so little to move, a step is bound by launches and by the chain
+// "weights -> hidden layer -> layer 2 -> Eq. 3" rather than by bandwidth.  One cluster per
+// (layer, head): one CTA per batch row runs the decode step of its instance, and SS_FEAT more CTAs
+// each take 1 / SS_FEAT of the hidden units of both MLPs for all batch rows of the head (Eq. 1,
+// Eq. 2: the sums over hidden units split exactly) while the decode CTAs are busy with the scores and
+// the softmax.  The feature CTAs write their partial layer-2 sums of batch row b into the shared
+// memory of the decode CTA of that row (plain st.shared::cluster over distributed shared memory) and
+// arrive at the cluster barrier; behind it the decode CTA adds the SS_FEAT partials in rank order,
+// finishes the maps (second GELU, W3 of psi, absolute value) and goes on with Eq. 3.  The barrier
+// is the hardware's (barrier.cluster): every thread that has not left reaches it on every path.
+// --------------------------------------------------------------------------- //
+constexpr int SS_THREADS = 512;       // threads per CTA of the small-step kernel (a decode CTA runs its step on the first 128)
+constexpr int SS_FEAT = 4;           // feature-map CTAs per head
+constexpr int SS_MAXB = 4;           // batch rows (decode CTAs) per head: SS_FEAT + SS_MAXB = the portable cluster size
+constexpr int SS_MAXJ = 128;         // hidden units per feature CTA at the widest hidden layer (512)
+
+struct SsMaps {
+  const __half* w1[2];    // W_phi1, W_psi1 [L, Hd, D, Rp]
+  const __half* w2[2];    // W_phi2, W_psi2 [L, Hd, Rp, R]
+  const __half* w3;       // W_psi3         [L, Hd, R, R]
+  const float* psi_scale; // [L, Hd, 2] or null
+  int Rp;
+};
+
+__device__ __forceinline__ uint32_t cluster_rank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
+// writes v at `local` (an address in this CTA's shared memory) in the shared memory of CTA `rank` of the cluster
+__device__ __forceinline__ void cluster_peer_store_f32(float* local, uint32_t rank, float v) {
+  const uint32_t a = (uint32_t)__cvta_generic_to_shared(local);
+  uint32_t ra;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ra) : "r"(a), "r"(rank));
+  asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(ra), "f"(v) : "memory");
+}
+
+// D += A B for one 16 x 8 x 16 tile on the tensor cores (warp-level mma: fp16 operands, fp32 accumulation)
+__device__ __forceinline__ void mma_m16n8k16(float* d, uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                             uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+      "{%0, %1, %2, %3};"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+// four 8 x 8 fp16 matrices from shared memory, transposed on the way (lane l gives the address of row l & 7 of matrix l >> 3)
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3, const void* row) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+               : "r"((uint32_t)__cvta_generic_to_shared(row)));
+}
+
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gmem_src)
+               : "memory");
+}
+__device__ __forceinline__ void cp_async8(void* smem_dst, const void* gmem_src) {
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gmem_src)
+               : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+
+// max / sum over the SS_THREADS threads of a CTA (warp tree, then the warps in order: fixed)
+__device__ __forceinline__ float wide_max(float v, float* red) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  if (lane == 0) red[warp] = v;
+  __syncthreads();
+  float r = red[0];
+#pragma unroll
+  for (int w = 1; w < SS_THREADS / 32; ++w) r = fmaxf(r, red[w]);
+  return r;                                        // `red` is not reused: no second barrier
+}
+__device__ __forceinline__ float wide_sum(float v, float* red) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  if (lane == 0) red[warp] = v;
+  __syncthreads();
+  float r = red[0];
+#pragma unroll
+  for (int w = 1; w < SS_THREADS / 32; ++w) r += red[w];
+  return r;
+}
+
+// What the decode CTA of the small-step kernel knows about its cluster.
+struct SsDecoder {
+  const float* part;      // [SS_FEAT][2][R] the feature CTAs' partial layer-2 sums of this batch row (written by them)
+  float* own;             // this CTA's: gsum [2 R], phi [R], c1, c2, (pad), then W3 [R R] as halves
+};
+
+// The decode step of one instance in the small-step kernel.  The same arithmetic as decode_kernel, laid
+// out for latency instead of bandwidth: with one small CTA per multiprocessor every phase is a chain of
+// dependent latencies that only more warps can shorten, so the scores, the softmax and the weighted
+// sum of the V rows run on all sixteen warps (32 slot rows per pass); the twelve extra warps then
+// leave, and the first four meet the feature CTAs, finish phi(q_t), psi(k_t), and run Eq. 3 and the
+// common second half of the step (decode_tail).
+template <int R, bool kCaptured>
+__device__ __forceinline__ void small_step_decode(const DecParams& p, const size_t inst, float* dsm, const SsDecoder& cl) {
+  constexpr int RG = SS_THREADS / 16;              // slot rows per pass
+  float* s_sc = dsm;                               // [Np + 4] scores, then e^{s - m}
+  float* s_red = s_sc + p.Np + 4;                  // [RG][128] partial numerators
+  __shared__ float s_w[2][SS_THREADS / 32];        // one row per reduction
+  __shared__ unsigned long long s_key[DEC_THREADS / 32];
+  __shared__ int s_vic;
+
+  const int tid = threadIdx.x;
+  const int l16 = tid & 15, rg = tid >> 4;
+  const int N = p.N;
+  const int t_now = kCaptured ? __ldcg(p.a.tpos) : p.t;
+  const int n = p.a.count[inst];
+  if (n < 0 || n > N) {                            // refuse a corrupt count, touch nothing; the cluster is still met
+    if (tid >= DEC_THREADS) return;
+    cp_async_wait_all();
+    cluster_wait();                                // the start-up phase, then the one the feature CTAs arrive at
+    cluster_arrive();
+    cluster_wait();
+    if (tid == 0) set_status(p.a.status, kStatusBounds, 1);
+    step_done<kCaptured>(p);
+    return;
+  }
+  const float scale = 0.08838834764831845f;        // 1 / sqrt(128)
+  const __half* Kb = p.a.kslots + inst * (size_t)N * kHeadDim;
+  const __half* Vb = p.a.vslots + inst * (size_t)N * kHeadDim;
+  // the state is last step's: its loads are under way long before the maps arrive
+  const int d = tid & (kHeadDim - 1);
+  float hcol[R], zr[R];
+  if (tid < DEC_THREADS) {
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+      hcol[r] = p.a.H[inst * (size_t)R * kHeadDim + r * kHeadDim + d];
+      zr[r] = p.a.z[inst * R + r];
+    }
+  }
+
+  float qf[8];
+  half8_to_float(*reinterpret_cast<const uint4*>(p.q + inst * kHeadDim + l16 * 8), qf);
+  const uint4 knew = *reinterpret_cast<const uint4*>(p.k + inst * kHeadDim + l16 * 8);
+  const uint4 vnew = *reinterpret_cast<const uint4*>(p.v + inst * kHeadDim + l16 * 8);
+  // ---- scores s_i = q . k_i / sqrt(D) over live slots, and the new pair ----
+#pragma unroll 2
+  for (int r0 = 0; r0 < n; r0 += RG) {             // r0 is block-uniform: shuffles stay converged
+    const int r = r0 + rg;
+    float dot = 0.f;
+    if (r < n) {
+      float kf[8];
+      half8_to_float(*reinterpret_cast<const uint4*>(Kb + (size_t)r * kHeadDim + l16 * 8), kf);
+#pragma unroll
+      for (int c = 0; c < 8; ++c) dot = fmaf(qf[c], kf[c], dot);
+    }
+#pragma unroll
+    for (int o = 8; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+    if (l16 == 0 && r < n) s_sc[r] = dot * scale;
+  }
+  if (tid < 32) {                                  // whole warp 0 (both halves compute the same)
+    float kf[8];
+    half8_to_float(knew, kf);
+    float dot = 0.f;
+#pragma unroll
+    for (int c = 0; c < 8; ++c) dot = fmaf(qf[c], kf[c], dot);
+#pragma unroll
+    for (int o = 8; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+    if (tid == 0) s_sc[n] = dot * scale;
+  }
+  __syncthreads();
+
+  // ---- m = max, e_i = exp(s_i - m), l = sum e_i  (entries 0..n, n = new pair) ----
+  float m = -INFINITY;
+  for (int i = tid; i <= n; i += SS_THREADS) m = fmaxf(m, s_sc[i]);
+  m = wide_max(m, s_w[0]);
+  m = fmaxf(m, -80.f);                             // keeps e^{-m} finite for the low-rank terms
+  float lsum = 0.f;
+  for (int i = tid; i <= n; i += SS_THREADS) {
+    const float e = __expf(s_sc[i] - m);
+    s_sc[i] = e;
+    lsum += e;
+  }
+  lsum = wide_sum(lsum, s_w[1]);                   // also orders the s_sc writes
+
+  // ---- u = sum e_i v_i ----
+  float u[8];
+#pragma unroll
+  for (int c = 0; c < 8; ++c) u[c] = 0.f;
+#pragma unroll 2
+  for (int r = rg; r < n; r += RG) {
+    float vf[8];
+    half8_to_float(*reinterpret_cast<const uint4*>(Vb + (size_t)r * kHeadDim + l16 * 8), vf);
+    const float e = s_sc[r];
+#pragma unroll
+    for (int c = 0; c < 8; ++c) u[c] = fmaf(e, vf[c], u[c]);
+  }
+  if (rg == 0) {
+    float vf[8];
+    half8_to_float(vnew, vf);
+    const float e = s_sc[n];
+#pragma unroll
+    for (int c = 0; c < 8; ++c) u[c] = fmaf(e, vf[c], u[c]);
+  }
+#pragma unroll
+  for (int c = 0; c < 8; c += 4)
+    *reinterpret_cast<float4*>(s_red + rg * kHeadDim + l16 * 8 + c) = make_float4(u[c], u[c + 1], u[c + 2], u[c + 3]);
+  __syncthreads();
+  if (tid >= DEC_THREADS) return;                  // the rest of the step runs on four warps; barriers count those left
+
+  float num = 0.f;
+#pragma unroll 8
+  for (int g = 0; g < RG; ++g) num += s_red[g * kHeadDim + d];   // fixed order
+
+  // ---- phi(q_t), psi(k_t): the feature CTAs' partial layer-2 sums, in rank order (Eq. 1, Eq. 2) ----
+  float* gsum = cl.own;
+  float* phis = cl.own + 2 * R;
+  cp_async_wait_all();                             // W3 and the scalars, asked for when the kernel started
+  cluster_wait();                                  // the start-up phase (complete long ago)
+  cluster_arrive();                                // behind this barrier the feature CTAs' partial sums are here
+  cluster_wait();
+  if (tid < 2 * R) {
+    const int mm = tid / R, r = tid % R;
+    float g = 0.f;
+#pragma unroll
+    for (int c = 0; c < SS_FEAT; ++c) g += cl.part[(c * 2 + mm) * R + r];   // rank order
+    const float c1 = mm ? cl.own[3 * R] : 1.f, c2 = mm ? cl.own[3 * R + 1] : 1.f;
+    g = c2 * gelu_erf(c1 * g);
+    gsum[tid] = g;
+    if (mm == 0) {
+      phis[r] = fabsf(g);
+      p.a.phi_q[inst * R + r] = fabsf(g);
+    }
+  }
+  __syncthreads();
+  if (tid < R) {                                   // the third layer of psi
+    const __half* w3 = reinterpret_cast<const __half*>(cl.own + 3 * R + 4);
+    float sacc = 0.f;
+#pragma unroll
+    for (int rr = 0; rr < R; ++rr) sacc = fmaf(gsum[R + rr], __half2float(w3[rr * R + tid]), sacc);
+    p.a.psi_k[inst * R + tid] = fabsf(sacc);       // decode_tail reads it from memory (behind its barriers)
+  }
+
+  // ---- low-rank correction and the single normalisation (Eq. 3) ----
+  float den = lsum;
+  {
+    const float em = __expf(-m);
+    float lr = 0.f, lz = 0.f;
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+      const float f = phis[r];
+      lr = fmaf(f, hcol[r], lr);
+      lz = fmaf(f, zr[r], lz);
+    }
+    num = fmaf(em, lr, num);
+    den = fmaf(em, lz, den);
+  }
+  store_out(p, inst * kHeadDim + d, num / den);
+  const float inv[1] = {1.0f / ((p.flags & LESS_SCORE_NORM_SPARSE) ? lsum : den)};
+  decode_tail<R, 1, kCaptured>(p, inst, n, t_now, s_sc, p.Np + 4, inv, hcol, knew, vnew, s_key, &s_vic);
+}
+
+template <int R, bool kCaptured>
+__global__ void __launch_bounds__(SS_THREADS) small_step_kernel(DecParams p, SsMaps mp) {
+  extern __shared__ float dsm[];
+  float* part = dsm;                                     // [SS_FEAT][2][R]  a decode CTA's inbox for the partial layer-2 sums
+  float* role = part + SS_FEAT * 2 * R;                  // the rest belongs to the CTA's role
+  const int tid = threadIdx.x;
+  const int nb = p.B;                                    // <= SS_MAXB
+  const int cs = nb + SS_FEAT;                           // CTAs per cluster
+  const int rank = (int)cluster_rank();
+  const int lh = blockIdx.x / cs;                        // layer * Hd + head
+  // "this CTA runs": distributed shared memory may only be touched once its owner has started.  Everyone
+  // arrives here at once; whoever needs the fact waits for it much later, when it has long been true.
+  cluster_arrive();
+
+  if (rank < nb) {
+    // ---------------- decode CTA of batch row `rank` ----------------
+    const size_t inst = (size_t)rank * p.LH + lh;
+    SsDecoder cl;
+    cl.part = part;
+    cl.own = role + p.Np + 4 + (SS_THREADS / 16) * kHeadDim;   // behind the step's scores and partial sums
+    if (tid == 0) {
+      if (mp.psi_scale) {
+        cp_async8(cl.own + 3 * R, mp.psi_scale + lh * 2);
+      } else {
+        cl.own[3 * R] = 1.f;
+        cl.own[3 * R + 1] = 1.f;
+      }
+    }
+    if (tid < R * R / 8)
+      cp_async16(reinterpret_cast<__half*>(cl.own + 3 * R + 4) + tid * 8, mp.w3 + (size_t)lh * R * R + tid * 8);
+    small_step_decode<R, kCaptured>(p, inst, role, cl);  // the barriers inside order these writes before their use
+    return;
+  }
+
+  // ---------------- feature CTA: 1 / SS_FEAT of the hidden units of both maps ----------------
+  // Short rolled loops over operands staged in shared memory; 16 warps, because every phase is a
+  // chain of dependent latencies that only other warps can fill.
+  const int fr = rank - nb;
+  const int Rp = mp.Rp, J = Rp / SS_FEAT;                // hidden units of this CTA: 128, 64 or 32
+  const int lj = 31 - __clz(J);                          // J = 1 << lj
+  const int lpr = J / 8, llpr = lj - 3;                  // 16-byte chunks per weight row of this CTA: 16, 8 or 4
+  const int ws = J + 8;                                  // padded row of the staged W1: the transposing loads below then
+                                                         // find their eight rows in eight different bank groups
+  __half* w1s = reinterpret_cast<__half*>(role);         // [2][128 rows][J + 8]
+  __half* xh = w1s + 2 * kHeadDim * (SS_MAXJ + 8);       // [2][SS_MAXB][128] q rows, then k rows
+  __half* w2h = xh + 2 * SS_MAXB * kHeadDim;             // [2][J][R] this CTA's rows of W2
+  float* hs = reinterpret_cast<float*>(w2h + 2 * SS_MAXJ * R);   // [2][SS_MAXB][SS_MAXJ] gelu(hidden)
+  // ---- stage everything with asynchronous copies: all loads in flight at once, no registers held ----
+  for (int e = tid; e < 2 * kHeadDim * lpr; e += SS_THREADS) {
+    const int m = e >> (7 + llpr), d = (e >> llpr) & (kHeadDim - 1), ch = e & (lpr - 1);
+    cp_async16(w1s + (size_t)(m * kHeadDim + d) * ws + ch * 8,
+               mp.w1[m] + ((size_t)lh * kHeadDim + d) * Rp + (size_t)fr * J + ch * 8);
+  }
+  if (tid < 2 * nb * 16) {
+    const int m = tid / (nb * 16), b = (tid >> 4) % nb, ch = tid & 15;
+    cp_async16(xh + (m * SS_MAXB + b) * kHeadDim + ch * 8,
+               (m == 0 ? p.q : p.k) + ((size_t)b * p.LH + lh) * kHeadDim + ch * 8);
+  }
+  const int w2chunks = J * R / 8;                        // 16-byte chunks of this CTA's rows of W2, per map (contiguous)
+  if (tid < 2 * w2chunks) {
+    const int m = tid >= w2chunks, ch = tid - m * w2chunks;
+    cp_async16(w2h + (m * J * R) + ch * 8, mp.w2[m] + ((size_t)lh * Rp + (size_t)fr * J) * R + ch * 8);
+  }
+  cp_async_wait_all();
+  __syncthreads();
+
+  // ---- layer 1 as warp-level MMAs (fp16 operands, used exactly; fp32 sums): the head's batch rows are the
+  //      first rows of the 16-row A operand (the rest zero), a tile of eight hidden units the B operand, read
+  //      from the staged [d][j] rows with transposing loads.  One warp per tile; gelu on the way out. ----
+  {
+    const int lane = tid & 31, warp = tid >> 5;
+    const int row = lane >> 2;                           // batch row of this lane's A and accumulator elements
+    const bool live = row < nb;
+    const int tiles = J >> 3;                            // per map
+    for (int tile = warp; tile < 2 * tiles; tile += SS_THREADS / 32) {
+      const int m = tile >= tiles, n0 = (tile - m * tiles) * 8;
+      const __half* xrow = xh + (m * SS_MAXB + row) * kHeadDim + 2 * (lane & 3);
+      const __half* wrow = w1s + (size_t)(m * kHeadDim + (lane >> 3) * 8 + (lane & 7)) * ws + n0;
+      float c[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+      for (int kk = 0; kk < kHeadDim / 32; ++kk) {       // two k-steps of 16 input dimensions per pass
+        uint32_t b0, b1, b2, b3;
+        ldmatrix_x4_trans(b0, b1, b2, b3, wrow + (size_t)kk * 32 * ws);
+        uint32_t a[4] = {0u, 0u, 0u, 0u};
+        if (live) {
+#pragma unroll
+          for (int q4 = 0; q4 < 4; ++q4) a[q4] = *reinterpret_cast<const uint32_t*>(xrow + kk * 32 + q4 * 8);
+        }
+        mma_m16n8k16(c, a[0], 0u, a[1], 0u, b0, b1);
+        mma_m16n8k16(c, a[2], 0u, a[3], 0u, b2, b3);
+      }
+      if (live) {
+        float* h = hs + (m * SS_MAXB + row) * SS_MAXJ + n0 + 2 * (lane & 3);
+        h[0] = gelu_erf(c[0]);
+        h[1] = gelu_erf(c[1]);
+      }
+    }
+  }
+  __syncthreads();
+  cluster_wait();                                        // the start-up phase: every decode CTA of the cluster runs
+  // ---- layer 2, this CTA's share: sum_j gelu(h_j) W2[j][r] into the inbox of the decode CTA of batch row b;
+  //      eight lanes per output, each over every eighth hidden unit, then a fixed shuffle tree ----
+#pragma unroll 1
+  for (int e0 = 0; e0 < 2 * nb * R; e0 += SS_THREADS / 8) {   // uniform over the CTA: the shuffles stay converged
+    const int e = e0 + (tid >> 3), jp = tid & 7;
+    const bool on = e < 2 * nb * R;
+    const int m = e >= nb * R, rem = e - m * nb * R, b = rem / R, r = rem % R;
+    float a = 0.f;
+    if (on) {
+      const float* h = hs + (m * SS_MAXB + b) * SS_MAXJ;
+      const __half* w = w2h + m * J * R + r;
+#pragma unroll 4
+      for (int j = jp; j < J; j += 8) a = fmaf(h[j], __half2float(w[j * R]), a);
+    }
+#pragma unroll
+    for (int o = 4; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
+    if (on && jp == 0) cluster_peer_store_f32(part + (fr * 2 + m) * R + r, (uint32_t)b, a);
+  }
+  cluster_arrive();                                      // releases the stores above to the decode CTAs; nothing to wait for
+}
+
+// --------------------------------------------------------------------------- //
 // Grouped query heads (Section 3.2, multi-query attention): G query heads share one KV head.
 // One 128-thread CTA per KV head; every query head has its own phi and its own Eq. 3 (own
 // normaliser) over the shared slots and the shared H, z; then the G heads' probabilities are
@@ -536,7 +923,7 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_group_rows_kernel(DecParam
   int n = p.a.count[inst];
   if (n < 0 || n > N) {
     if (tid == 0) set_status(p.a.status, kStatusBounds, 1);
-    step_done<kCaptured>(p.a.tpos, p.t);
+    step_done<kCaptured>(p);
     return;
   }
   const bool use_state = !(p.flags & LESS_NO_STATE);
@@ -644,21 +1031,6 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_group_rows_kernel(DecParam
   group_eq3_and_tail<R, G, kCaptured, DEC_RG>(p, inst, n, t_now, s_sc, Ns, s_red, s_ml[0], s_ml[1], knew, vnew, s_inv, s_key, &s_vic);
 }
 
-// The same step with the two contractions on the tensor cores.  With G query heads per KV head the
-// scores are a [slots x 128] x [128 x G] product and the numerators a [128 x slots] x [slots x G] one:
-// dense, but only G <= 8 wide and bound by the K / V stream, so the warp-level mma (m16n8k16, fp16
-// inputs used exactly, fp32 accumulation, N = 8 = the heads) fits: its fragments load straight from
-// global memory with no staging, four warps split the 16-slot tiles.  The probabilities enter the
-// second product rounded to fp16 (relative 4.9e-4, like the prompt-output kernel); the H2O scores
-// use the fp32 values.
-__device__ __forceinline__ void mma_m16n8k16(float* d, uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
-                                             uint32_t b0, uint32_t b1) {
-  asm volatile(
-      "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
-      "{%0, %1, %2, %3};"
-      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-}
 
 __device__ __forceinline__ uint32_t word_of(const uint4& v, int w) {
   return w == 0 ? v.x : w == 1 ? v.y : w == 2 ? v.z : v.w;
@@ -666,6 +1038,13 @@ __device__ __forceinline__ uint32_t word_of(const uint4& v, int w) {
 
 constexpr int kMmaRed = DEC_THREADS / 32 + 1;   // partial numerators per head in the mma kernel
 
+// The same step with the two contractions on the tensor cores.  With G query heads per KV head the
+// scores are a [slots x 128] x [128 x G] product and the numerators a [128 x slots] x [slots x G] one:
+// dense, but only G <= 8 wide and bound by the K / V stream, so the warp-level mma (m16n8k16, fp16
+// inputs used exactly, fp32 accumulation, N = 8 = the heads) fits: its fragments load straight from
+// global memory with no staging, four warps split the 16-slot tiles.  The probabilities enter the
+// second product rounded to fp16 (relative 4.9e-4, like the prompt-output kernel); the H2O scores
+// use the fp32 values.
 template <int R, int G, bool kCaptured>
 __global__ void __launch_bounds__(DEC_THREADS) decode_group_mma_kernel(DecParams p) {
   extern __shared__ float dsm[];
@@ -685,7 +1064,7 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_group_mma_kernel(DecParams
   int n = p.a.count[inst];
   if (n < 0 || n > N) {
     if (tid == 0) set_status(p.a.status, kStatusBounds, 1);
-    step_done<kCaptured>(p.a.tpos, p.t);
+    step_done<kCaptured>(p);
     return;
   }
   const bool use_state = !(p.flags & LESS_NO_STATE);
@@ -889,7 +1268,7 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_group_loop_kernel(DecParam
   int n = p.a.count[inst];
   if (n < 0 || n > N) {
     if (tid == 0) set_status(p.a.status, kStatusBounds, 1);
-    step_done<kCaptured>(p.a.tpos, p.t);
+    step_done<kCaptured>(p);
     return;
   }
   const bool use_state = !(p.flags & LESS_NO_STATE);
@@ -1091,6 +1470,7 @@ int launch_decode(less_ctx* c, const void* q, const void* k, const void* v, void
     return fail_cuda("shared memory opt-in of decode_kernel");
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(segment ? d.B * c->seg_nl * d.Hd : d.I);
+  p.done_ctas = (int)cfg.gridDim.x;
   cfg.blockDim = dim3(DEC_THREADS);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = s;
@@ -1106,6 +1486,80 @@ int launch_decode(less_ctx* c, const void* q, const void* k, const void* v, void
   void* args[] = {&p, &G_arg};                         // the second argument is the general kernel's only
   if (cudaLaunchKernelExC(&cfg, kern, args) != cudaSuccess) return fail_cuda("launch of decode_kernel");
   return check_launch("decode_kernel");
+}
+
+// Whether a step of this context runs as the single small_step_kernel launch: the shapes the kernel
+// takes, and (unless forced) few enough heads that all its CTAs find a multiprocessor of their own -
+// up to there a step is bound by launches and latency (measured: 8 heads 8.3 against 8.7 us per step
+// replayed from a graph, 10.3 against 11.4 us by direct calls), past it by the weight stream, which
+// the tensor-core feature kernel moves faster.
+bool small_step_path(const less_ctx* c) {
+  const Dims& d = c->d;
+  if (c->small_step == 0 || d.general || d.G != 1 || d.D != kHeadDim || (d.flags & LESS_NO_STATE)) return false;
+  if (d.B > SS_MAXB || (d.Rp != 128 && d.Rp != 256 && d.Rp != 512) || c->seg_nl != d.L) return false;
+  if (c->feature_path != 2) return false;             // a feature-map kernel was asked for by name
+  return c->small_step == 1 || d.L * d.Hd * (d.B + SS_FEAT) <= c->sms;
+}
+
+int launch_small_step(less_ctx* c, const void* q, const void* k, const void* v, void* out, int32_t* evicted_pos,
+                      cudaStream_t s) {
+  const Dims& d = c->d;
+  DecParams p;
+  p.q = (const __half*)q; p.k = (const __half*)k; p.v = (const __half*)v;
+  p.out = out;
+  p.evicted_pos = evicted_pos;
+  p.a = c->a;
+  p.N = d.N; p.Np = d.Np; p.heavy = d.heavy; p.recent = d.recent;
+  p.t = (int)c->t;
+  p.B = d.B; p.LH = d.L * d.Hd;
+  p.flags = d.flags;
+  p.feat_flag = nullptr; p.flag_stride = 0; p.flag_target[0] = p.flag_target[1] = 0;
+  p.head_major = 0; p.lh0 = 0;
+  p.done_ctas = d.I;
+  SsMaps mp;
+  mp.w1[0] = (const __half*)c->w.w_phi1; mp.w1[1] = (const __half*)c->w.w_psi1;
+  mp.w2[0] = (const __half*)c->w.w_phi2; mp.w2[1] = (const __half*)c->w.w_psi2;
+  mp.w3 = (const __half*)c->w.w_psi3;
+  mp.psi_scale = c->w.psi_scale;
+  mp.Rp = d.Rp;
+  cudaStreamCaptureStatus capturing = cudaStreamCaptureStatusNone;
+  cudaStreamIsCapturing(s, &capturing);
+  const bool captured = capturing == cudaStreamCaptureStatusActive;
+  // the partial sums, then the larger of the two roles' shared memory
+  const size_t dec_bytes = (size_t)(d.Np + 4 + (SS_THREADS / 16) * kHeadDim) * 4 + (size_t)(3 * d.R + 4) * 4 + (size_t)d.R * d.R * 2;
+  const size_t feat_bytes = (size_t)2 * kHeadDim * (SS_MAXJ + 8) * 2 + (size_t)2 * SS_MAXB * kHeadDim * 2 +
+                            (size_t)2 * SS_MAXJ * d.R * 2 + (size_t)2 * SS_MAXB * SS_MAXJ * 4;
+  const size_t smem = (size_t)SS_FEAT * 2 * d.R * 4 + (dec_bytes > feat_bytes ? dec_bytes : feat_bytes);
+  // a step this small is bound by the host's work per launch as well: names and attributes are set once
+  LaunchScope scope(c, LESS_KERNEL_DECODE, s);
+  void* kern = d.R == 8 ? (captured ? (void*)small_step_kernel<8, true> : (void*)small_step_kernel<8, false>)
+                        : (captured ? (void*)small_step_kernel<16, true> : (void*)small_step_kernel<16, false>);
+  if (!c->small_step_ready[captured]) {
+    if (smem > 48 * 1024 &&
+        cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+      return fail_cuda("shared memory opt-in of small_step_kernel");
+    c->small_step_ready[captured] = true;
+  }
+  if (c->small_step_named != (int)captured) {
+    snprintf(c->variant[LESS_KERNEL_DECODE], sizeof c->variant[0], "small_step_kernel<%d, %d>", d.R, (int)captured);
+    c->variant[LESS_KERNEL_FEATURE_MAP][0] = 0;         // no feature-map kernel of its own
+    c->small_step_named = (int)captured;
+  }
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(d.L * d.Hd * (d.B + SS_FEAT));
+  cfg.blockDim = dim3(SS_THREADS);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = d.B + SS_FEAT;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  void* args[] = {&p, &mp};
+  if (cudaLaunchKernelExC(&cfg, kern, args) != cudaSuccess) return fail_cuda("launch of small_step_kernel");
+  return check_launch("small_step_kernel");
 }
 
 }  // namespace less

@@ -217,6 +217,10 @@ int less_create(const less_config* cfg, const less_weights* w, void* arena, size
     else if (!strcmp(e, "plain")) c->feature_path = 0;
   }
   if (cudaGetDevice(&c->device) != cudaSuccess) { delete c; return LESS_ERR_CUDA; }
+  c->small_step = -1;
+  c->small_step_ready[0] = c->small_step_ready[1] = false;
+  c->small_step_named = -1;
+  if (const char* e = getenv("LESS_SMALL_STEP")) c->small_step = !strcmp(e, "0") ? 0 : (!strcmp(e, "1") ? 1 : -1);
   c->group_path = 3;
   if (const char* e = getenv("LESS_GROUP_KERNEL"))
     if (!strcmp(e, "rows")) c->group_path = 2;
@@ -310,6 +314,11 @@ int less_decode_step(less_ctx* c, const void* q, const void* k, const void* v, v
     return LESS_ERR_MISALIGNED;
   if (c->t >= 0x7fffff00) return LESS_ERR_BAD_STATE;
   cudaStream_t s = (cudaStream_t)stream;
+  if (small_step_path(c)) {
+    const int rc1 = launch_small_step(c, q, k, v, out, evicted_pos, s);
+    if (rc1 == LESS_OK) c->t += 1;
+    return rc1;
+  }
   int rc = launch_feature_maps(c, q, k, s);
   if (rc != LESS_OK) return rc;
   rc = launch_decode(c, q, k, v, out, evicted_pos, s);
@@ -392,7 +401,7 @@ int less_decode_step_host(less_ctx* c, const void* qh, const void* kh, const voi
   const void* q_dev = device_alias(qh);
   const void* k_dev = device_alias(kh);
   const bool qk_in_place = q_dev && k_dev && !((uintptr_t)q_dev & 15) && !((uintptr_t)k_dev & 15) &&
-                           (feature_small_tc_path(c) || (c->d.flags & LESS_NO_STATE));
+                           (feature_small_tc_path(c) || small_step_path(c) || (c->d.flags & LESS_NO_STATE));
   // a large staged step: its layers in segments, the copies under the kernels
   if (!qk_in_place && v_dev && out_dev && feature_tc_path(c) && !c->head_counters && c->d.L >= kSegments &&
       nq + nin >= ((size_t)4 << 20) && c->t < 0x7fffff00) {

@@ -87,6 +87,10 @@ struct less_ctx {
   int feature_stages;  // cap on the feature kernels' ring stages (LESS_FEATURE_STAGES), 0 = default
   int score_path;      // prompt scoring: 1 tensor cores, 0 CUDA cores (LESS_SCORE_KERNEL=plain)
   int feature_path;    // feature-map kernel: 2 tensor cores, 1 streaming GEMV, 0 plain (LESS_FEATURE_KERNEL)
+  int small_step;      // the single-launch step for workloads of a few heads: -1 by size (default), 0 never, 1 whenever
+                       // the shape allows (LESS_SMALL_STEP)
+  bool small_step_ready[2];   // shared-memory opt-in of the small-step kernel done (direct / captured variant)
+  int small_step_named;       // which variant's name is in `variant`, -1 = neither
   int group_path;      // grouped decode kernel: 2 on CUDA cores (LESS_GROUP_KERNEL=rows), else with warp-level mma
   int seg_l0, seg_nl;  // layers [seg_l0, seg_l0 + seg_nl) of the step being launched (the host entry launches a
                        // large step in layer segments so that its input copies overlap the kernels); default all
@@ -263,6 +267,10 @@ bool feature_tc_path(const less_ctx* c);
 bool feature_small_tc_path(const less_ctx* c);
 int launch_decode(less_ctx* c, const void* q, const void* k, const void* v, void* out,
                   int32_t* evicted_pos, cudaStream_t s);
+// feature maps and decode step of a workload of a few heads in one launch (decode_kernels.cu)
+bool small_step_path(const less_ctx* c);
+int launch_small_step(less_ctx* c, const void* q, const void* k, const void* v, void* out, int32_t* evicted_pos,
+                      cudaStream_t s);
 int launch_prefill_group(less_ctx* c, int layer0, int nlayers, int lj0, int layer_count, int S,
                          const void* Q, const void* K, const void* V, void* attn_out,
                          cudaStream_t s);

@@ -73,8 +73,11 @@ def _decode_steps(ctx, w, W, instances, steps):
     return tf
 
 
-def test_cfg1_smallest_every_instance_every_step():
+@pytest.mark.parametrize("path", ["single_launch", "two_kernels"])
+def test_cfg1_smallest_every_instance_every_step(path, monkeypatch):
     w = wl.CONFIGS[1]
+    if path == "single_launch":             # what a workload of eight heads runs by default
+        monkeypatch.delenv("LESS_SMALL_STEP", raising=False)
     ctx, W = _ctx(w, w.layers)
     Q, K, V = wl.make_prompt(w, 0, w.layers, DEV)
     ctx.prefill(Q, K, V, 0)
@@ -82,7 +85,8 @@ def test_cfg1_smallest_every_instance_every_step():
     print("cfg1 prompt", _check_prompt(ctx, w, W, inst))
     tf = _decode_steps(ctx, w, W, inst, w.steps)
     assert tf.evictions == w.steps * w.instances
-    print("cfg1 decode", tf.worst, "exempt", tf.exempt)
+    assert ctx.kernel_variant("decode").startswith("small_step_kernel") == (path == "single_launch")
+    print("cfg1 decode", path, tf.worst, "exempt", tf.exempt)
     ctx.close()
 
 

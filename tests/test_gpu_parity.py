@@ -101,6 +101,73 @@ def test_prefill_and_teacher_forced_decode(variant, monkeypatch):
     ctx.close()
 
 
+@pytest.mark.parametrize("variant", ["one_row_eight_heads", "rank16_two_rows", "four_rows_hidden256",
+                                     "hidden128_scaled", "sparse_norm", "lambda_masking", "tova", "from_empty",
+                                     "by_size"])
+def test_small_step_single_launch(variant, monkeypatch):
+    """The single-launch step for workloads of a few heads (a cluster of CTAs per head computes phi(q_t)
+    and psi(k_t), then one CTA per batch row runs Algorithm 1): every step against the oracle, started
+    from the library's own pre-step state, with the feature maps compared too."""
+    import harness
+    monkeypatch.setenv("LESS_SMALL_STEP", "1")
+    flags, psi_scale = 0, None
+    w = small(40, batch=1, layers=1, heads=8, weight_std=0.1)
+    if variant == "rank16_two_rows":
+        w = small(41, rank=16, prompt=257, weight_std=0.2)
+    elif variant == "four_rows_hidden256":
+        w = small(42, batch=4, layers=1, heads=2, hidden=256, weight_std=0.1, prompt=131, heavy=7, recent=9)
+    elif variant == "hidden128_scaled":
+        w = small(43, batch=3, hidden=128, weight_std=0.2)
+        g = torch.Generator().manual_seed(6)
+        psi_scale = 0.5 + 2.0 * torch.rand(w.layers, w.heads, 2, generator=g)
+    elif variant == "sparse_norm":
+        w, flags = small(44, weight_std=0.2), 1
+    elif variant == "lambda_masking":
+        w, flags = small(45, heavy=4, recent=36, weight_std=0.1), 4
+    elif variant == "tova":
+        w, flags = small(46, weight_std=0.1, steps=16), 8
+    elif variant == "from_empty":
+        w = small(47, prompt=0, steps=30, heavy=5, recent=6, weight_std=0.2)
+    elif variant == "by_size":              # no switch: few heads go this way by themselves
+        monkeypatch.delenv("LESS_SMALL_STEP")
+    ctx, W = _setup(w, flags, psi_scale, max_prompt=max(w.prompt, 16))
+    inst = list(range(w.instances))
+    if w.prompt:
+        Q, K, V, out = _prefill_all(ctx, w)
+        harness.check_prefill(ctx, w, W, Q, K, V, inst, out, flags, psi_scale)
+    tf = harness.TeacherForced(ctx, w, W, inst, flags, psi_scale)
+    for s in range(w.steps):
+        tf.step(*wl.make_decode_inputs(w, s, DEV))
+    assert ctx.kernel_variant("decode").startswith("small_step_kernel")
+    assert ctx.poll_status() == 0
+    assert tf.evictions == (w.steps * w.instances if w.prompt else (w.steps - w.slots) * w.instances)
+    assert tf.exempt <= 0.02 * tf.evictions + 1
+    n0 = ctx.launches
+    ctx.decode_step(*wl.make_decode_inputs(w, w.steps, DEV))
+    assert ctx.launches - n0 == 1 and ctx.poll_status() == 0  # one kernel per step
+    print("small step", variant, tf.worst, "exempt", tf.exempt)
+    ctx.close()
+
+
+def test_small_step_shapes_it_does_not_take_use_the_two_kernels(monkeypatch):
+    monkeypatch.setenv("LESS_SMALL_STEP", "1")
+    import harness
+    for kw, flags in ((dict(batch=5), 0), (dict(group=2), 0), (dict(), 2)):
+        w = small(48, steps=3, weight_std=0.1, **kw)
+        ctx, W = _setup(w, flags)
+        _prefill_all(ctx, w, with_out=False)
+        tf = (harness.GroupTeacherForced if w.group > 1 else harness.TeacherForced)(ctx, w, W, [0, w.instances - 1], flags)
+        for s in range(w.steps):
+            tf.step(*wl.make_decode_inputs(w, s, DEV))
+        assert not ctx.kernel_variant("decode").startswith("small_step_kernel") and ctx.poll_status() == 0
+        ctx.close()
+
+
+def test_small_step_captured_replays_like_direct_calls(monkeypatch):
+    monkeypatch.setenv("LESS_SMALL_STEP", "1")
+    test_captured_step_replays_like_direct_calls(3)
+
+
 def test_short_prompt_fills_without_eviction_then_evicts():
     """prompt_len <= slots: everything is kept; decode appends until full."""
     import harness
