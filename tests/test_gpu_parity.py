@@ -1,5 +1,7 @@
 """GPU parity: the CUDA path, called through the C ABI, against the fp64 oracle
 on the same seeded inputs."""
+import os
+
 import numpy as np
 import pytest
 import torch
@@ -161,6 +163,14 @@ def test_small_step_shapes_it_does_not_take_use_the_two_kernels(monkeypatch):
             tf.step(*wl.make_decode_inputs(w, s, DEV))
         assert not ctx.kernel_variant("decode").startswith("small_step_kernel") and ctx.poll_status() == 0
         ctx.close()
+
+
+@pytest.mark.parametrize("pinned", [True, False])
+def test_small_step_host_entry_matches_the_device_entry(pinned, monkeypatch):
+    """The single-launch step through less_decode_step_host: pinned q, k, v and the output are read /
+    written in place by the kernel (asynchronous copies and plain loads over PCIe), pageable ones staged."""
+    monkeypatch.setenv("LESS_SMALL_STEP", "1")
+    test_host_buffer_entry_matches_device_entry(pinned, 1)
 
 
 def test_small_step_captured_replays_like_direct_calls(monkeypatch):
@@ -520,6 +530,7 @@ def test_host_buffer_entry_matches_device_entry(pinned, group):
         for key in ("pos", "acc", "K", "V", "psi", "H", "z"):
             assert np.array_equal(a[key], b[key]), key
     assert ctx_h.poll_status() == 0
+    assert ctx_h.kernel_variant("decode").startswith("small_step") == (os.environ.get("LESS_SMALL_STEP") == "1")
     ctx_d.close(); ctx_h.close()
 
 
