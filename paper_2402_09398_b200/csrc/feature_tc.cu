@@ -30,11 +30,18 @@ namespace less {
 constexpr int FT_EPI_WARPS = 8;
 constexpr int FT_EPI_THREADS = FT_EPI_WARPS * 32;
 constexpr int FT_THREADS = 96 + FT_EPI_THREADS;   // small-batch kernel: warp 0 TMA, warp 1 MMA, warps 2..9 epilogue, warp 10 input rows by plain loads
-// The larger-batch kernel runs four epilogue warps per lane quadrant: its GELU chains are long and
-// dependent, and with two warps per scheduler the issue slots sat idle (4700 cycles per chunk
-// measured for 32 GELUs per thread).
-constexpr int FL_EPI_WARPS = 16;
-constexpr int FL_THREADS = 64 + FL_EPI_WARPS * 32;
+// The larger-batch kernel runs sixteen GELU warps (four per scheduler: with two the issue slots sat
+// idle) in two groups of eight that take the 128-unit chunks in turn, each with its own accumulator
+// buffer and its own hidden-layer operand: while one group is saturating the schedulers with GELUs,
+// the other sits in the phases that issue little (waiting for GEMM1, loading the accumulator, storing
+// the operand, the proxy fence).  In lockstep the sixteen warps spent 1 350 of a chunk's 3 200 cycles
+// in the GELU phase and the rest with the schedulers mostly idle.  Four more warps, one per lane
+// quadrant, finish the items (second layer's GELU, W3, output), so that the GELU warps never wait for it.
+constexpr int FL_GROUPS = 2;
+constexpr int FL_GROUP_WARPS = 8;
+constexpr int FL_EPI_WARPS = FL_GROUPS * FL_GROUP_WARPS;
+constexpr int FL_FIN_WARPS = 4;
+constexpr int FL_THREADS = 64 + (FL_EPI_WARPS + FL_FIN_WARPS) * 32;
 constexpr int FT_CHUNK = 128;                     // hidden units per GEMM1
 constexpr int FT_STAGE_BYTES = FT_CHUNK * kHeadDim * 2;
 constexpr int FT_MAX_STAGES = 6;
@@ -44,7 +51,7 @@ struct FtShared {
   uint64_t full[FT_MAX_STAGES], empty[FT_MAX_STAGES];
   uint64_t aux_full[2], aux_empty[2];
   uint64_t d1_full[2], d1_free[2];
-  uint64_t hid_full, hid_free;
+  uint64_t hid_full[FL_GROUPS], hid_free[FL_GROUPS];   // per epilogue group
   uint64_t d2_full, d2_free;
   uint32_t tmem_base;
   int abort;
@@ -128,7 +135,7 @@ __device__ __forceinline__ void ft_produce(const CUtensorMap* tm_q, const CUtens
 }
 
 template <int R>
-__global__ void __launch_bounds__(FL_THREADS) feature_tc_kernel(
+__global__ void __launch_bounds__(FL_THREADS, 1) feature_tc_kernel(
     const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
     const __grid_constant__ CUtensorMap tm_w1phi, const __grid_constant__ CUtensorMap tm_w1psi, FmParams p,
     FtGeom gm, int32_t* status) {
@@ -138,8 +145,8 @@ __global__ void __launch_bounds__(FL_THREADS) feature_tc_kernel(
   const uint32_t hbytes = (uint32_t)npad * 256;      // hi (or lo): npad/8 token blocks x 2 KB
   const uint32_t xbytes = (uint32_t)npad * 256;      // two 64-column halves of npad rows x 128 B
   const uint32_t w2bytes = (uint32_t)Rp * R * 2;
-  unsigned char* hbuf = ft_smem;                     // hi, then lo
-  unsigned char* xbuf = hbuf + 2 * hbytes;           // [2][xbytes]
+  unsigned char* hbuf = ft_smem;                     // per group: hi, then lo
+  unsigned char* xbuf = hbuf + FL_GROUPS * 2 * hbytes;   // [2][xbytes]
   unsigned char* ring = xbuf + 2 * xbytes;           // [nstage][32 KB]
   unsigned char* w2buf = ring + (size_t)nstage * FT_STAGE_BYTES;   // [2][R/8 column blocks][Rp rows][16 B]
   unsigned char* w2raw = w2buf + 2 * w2bytes;        // R = 16 only: [2][Rp rows][32 B] as it lies in HBM
@@ -153,14 +160,14 @@ __global__ void __launch_bounds__(FL_THREADS) feature_tc_kernel(
     }
     for (int s = 0; s < 2; ++s) {
       mbar_init(&sh->aux_full[s], 1);
-      mbar_init(&sh->aux_empty[s], 1 + FL_EPI_WARPS);
+      mbar_init(&sh->aux_empty[s], 1 + FL_FIN_WARPS);
       mbar_init(&sh->d1_full[s], 1);
-      mbar_init(&sh->d1_free[s], FL_EPI_WARPS);
+      mbar_init(&sh->d1_free[s], FL_GROUP_WARPS);
+      mbar_init(&sh->hid_full[s], FL_GROUP_WARPS);
+      mbar_init(&sh->hid_free[s], 1);
     }
-    mbar_init(&sh->hid_full, FL_EPI_WARPS);
-    mbar_init(&sh->hid_free, 1);
     mbar_init(&sh->d2_full, 1);
-    mbar_init(&sh->d2_free, FL_EPI_WARPS);
+    mbar_init(&sh->d2_free, FL_FIN_WARPS);
     // a CTA that starts after another one has given up skips every wait: the grid drains at once
     sh->abort = *reinterpret_cast<volatile int32_t*>(status) != 0;
     mbar_fence_init();
@@ -174,6 +181,7 @@ __global__ void __launch_bounds__(FL_THREADS) feature_tc_kernel(
   const uint32_t d2col = 2u * (uint32_t)npad;
   volatile int* abortp = &sh->abort;
   const int my_items = blockIdx.x < gm.items ? (gm.items - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
+  const uint32_t total = (uint32_t)my_items * nchunk;   // chunks of this CTA, counted across its items
 
   if (warp == 0) {
     // ---------------- TMA producer ----------------
@@ -194,16 +202,15 @@ __global__ void __launch_bounds__(FL_THREADS) feature_tc_kernel(
       // R = 8 fills one 8-column block; the second block of the N = 16 tile then only has to
       // lie inside this CTA's shared memory (its columns of D2 are never read)
       const uint64_t bd_w2 = smem_desc(smem_u32(w2buf), 128, R == 16 ? (uint32_t)Rp * 16 : 128u, kLayoutNone);
-      const uint64_t ad_hi = smem_desc(smem_u32(hbuf), 128, 2048, kLayoutNone);
-      const uint64_t ad_lo = ad_hi + (uint64_t)(hbytes >> 4);
-      const uint32_t total = (uint32_t)my_items * nchunk;
-      // GEMM1 runs one chunk ahead of GEMM2
-      uint32_t s = 0, sph = 0, b1 = 0, b1ph = 0, c1 = 0, n1 = 0, issued = 0;
+      const uint64_t ad_hid = smem_desc(smem_u32(hbuf), 128, 2048, kLayoutNone);
+      // GEMM1 runs two chunks ahead of GEMM2: one chunk per epilogue group is in work at any time.
+      // Chunk qq (counted over the CTA's items) lives in accumulator buffer qq & 1 and belongs to group qq & 1.
+      uint32_t s = 0, sph = 0, c1 = 0, n1 = 0, issued = 0;
       auto issue_gemm1 = [&]() {
-        const uint32_t a = n1 & 1;
+        const uint32_t a = n1 & 1, b1 = issued & 1;
         if (c1 == 0) wait_or_give_up(&sh->aux_full[a], (n1 >> 1) & 1, abortp, status, 42);
         wait_or_give_up(&sh->full[s], sph, abortp, status, 43);
-        wait_or_give_up(&sh->d1_free[b1], b1ph ^ 1, abortp, status, 44);
+        wait_or_give_up(&sh->d1_free[b1], ((issued >> 1) & 1) ^ 1, abortp, status, 44);   // the group has loaded the buffer's last chunk
         if (*abortp) return;
         tc_fence_after_sync();
         const uint64_t ad0 = ad_ring + (uint64_t)(s * (FT_STAGE_BYTES >> 4));
@@ -216,78 +223,86 @@ __global__ void __launch_bounds__(FL_THREADS) feature_tc_kernel(
         mma_commit(&sh->empty[s]);
         mma_commit(&sh->d1_full[b1]);
         if (++s == (uint32_t)nstage) { s = 0; sph ^= 1; }
-        if (b1 ^= 1, b1 == 0) b1ph ^= 1;
         if (++c1 == (uint32_t)nchunk) { c1 = 0; ++n1; }
         ++issued;
       };
       issue_gemm1();
-      uint32_t hph = 0;
+      if (issued < total && !*abortp) issue_gemm1();
+      uint32_t qq = 0;
       for (uint32_t n = 0; n < (uint32_t)my_items && !*abortp; ++n) {
         const uint32_t a = n & 1;
-        for (uint32_t c = 0; c < (uint32_t)nchunk; ++c) {
+        for (uint32_t c = 0; c < (uint32_t)nchunk; ++c, ++qq) {
+          const uint32_t g = qq & 1;
+          // the chunk two ahead first: its accumulator buffer is free as soon as group g has loaded chunk qq
           if (issued < total) issue_gemm1();
           if (c == 0) wait_or_give_up(&sh->d2_free, (n & 1) ^ 1, abortp, status, 45);
-          wait_or_give_up(&sh->hid_full, hph, abortp, status, 46);
+          wait_or_give_up(&sh->hid_full[g], (qq >> 1) & 1, abortp, status, 46);
           if (*abortp) break;
-          hph ^= 1;
           tc_fence_after_sync();
           const uint64_t bd0 = bd_w2 + (uint64_t)(a * (w2bytes >> 4) + c * (FT_CHUNK * 16 >> 4));
+          const uint64_t ad_hi = ad_hid + (uint64_t)(g * (2 * hbytes >> 4));
+          const uint64_t ad_lo = ad_hi + (uint64_t)(hbytes >> 4);
 #pragma unroll
           for (int ks = 0; ks < FT_CHUNK / 16; ++ks) {
             mma_f16_ss(tmem + d2col, ad_hi + (uint64_t)(ks * 16), bd0 + (uint64_t)(ks * 16), idesc2, (c | ks) ? 1u : 0u);
             mma_f16_ss(tmem + d2col, ad_lo + (uint64_t)(ks * 16), bd0 + (uint64_t)(ks * 16), idesc2, 1u);
           }
-          mma_commit(&sh->hid_free);
+          mma_commit(&sh->hid_free[g]);
         }
         if (*abortp) break;
         mma_commit(&sh->d2_full);
         mma_commit(&sh->aux_empty[a]);
       }
     }
-  } else {
-    // ---------------- epilogue warps ----------------
+  } else if (warp < 2 + FL_EPI_WARPS) {
+    // ---------------- GELU warps: group g takes the chunks qq = g, g + 2, ... ----------------
     const int ew = warp - 2;                   // 0..15
+    const int g = ew >> 3;                     // group = accumulator buffer = hidden operand buffer
     const int quad = warp & 3;                 // tensor-memory lane quadrant this warp may read
-    const int hf = ew >> 2;                    // which quarter of the token blocks (0..3)
+    const int hf = (ew & 7) >> 2;              // which half of the token blocks (blocks hf, hf + 2, hf + 4, hf + 6)
     const int j = quad * 32 + lane;            // hidden unit inside the chunk = accumulator lane
     const uint32_t lane_addr = tmem + ((uint32_t)(quad * 32) << 16);
-    unsigned char* hrow = hbuf + (j >> 3) * 128 + (j & 7) * 16;
-    uint32_t q = 0;
-    for (int n = 0; n < my_items && !*abortp; ++n) {
-      const int it = blockIdx.x + n * gridDim.x;
-      const FtItem im = ft_item(it, gm);
-      const int tile = im.tile, which = im.which, lh = im.lh;
-      const int a = n & 1;
-      const int b0 = tile * npad, nb = min(npad, p.B - b0), nblk = (nb + 7) >> 3;
-      float c1 = 1.f, c2 = 1.f;
-      if (which && p.psi_scale) { c1 = __ldg(p.psi_scale + lh * 2); c2 = __ldg(p.psi_scale + lh * 2 + 1); }
-      wait_or_give_up(&sh->aux_full[a], (n >> 1) & 1, abortp, status, 50);
-      if (R == 16) {
-        // 32-byte rows -> two blocks of 16-byte rows; the GEMM2s that read this buffer two items
-        // ago are complete (their D2 was read), and the first hid_full arrival below publishes it
+    unsigned char* hrow = hbuf + (size_t)g * 2 * hbytes + (j >> 3) * 128 + (j & 7) * 16;
+    int n_cur = -1, nb = 0, nblk = 0, a = 0;
+    int n = g / nchunk, c = g % nchunk;        // item and chunk of qq, advanced by counting
+    for (uint32_t qq = g, u = 0; qq < total && !*abortp; qq += FL_GROUPS, ++u) {
+      if (n != n_cur) {
+        n_cur = n;
+        const FtItem im = ft_item(blockIdx.x + n * gridDim.x, gm);
+        nb = min(npad, p.B - im.tile * npad);
+        nblk = (nb + 7) >> 3;
+        a = n & 1;
+      }
+      if (R == 16 && c == 0) {
+        // the item's W2: 32-byte rows -> two blocks of 16-byte rows, by the group that has the item's first
+        // chunk; the GEMM2s that read this buffer two items ago are complete (the producer waited for them
+        // before refilling the raw copy), and this group's hid_full arrival below publishes it
+        wait_or_give_up(&sh->aux_full[a], (n >> 1) & 1, abortp, status, 50);
         const uint4* src = reinterpret_cast<const uint4*>(w2raw + a * w2bytes);
         unsigned char* dst = w2buf + a * w2bytes;
-        for (int u = tid - 64; u < Rp * 2; u += FL_EPI_WARPS * 32)
-          *reinterpret_cast<uint4*>(dst + ((size_t)(u & 1) * Rp + (u >> 1)) * 16) = src[u];
+        for (int x = (ew & 7) * 32 + lane; x < Rp * 2; x += FL_GROUP_WARPS * 32)
+          *reinterpret_cast<uint4*>(dst + ((size_t)(x & 1) * Rp + (x >> 1)) * 16) = src[x];
       }
-      for (int c = 0; c < nchunk && !*abortp; ++c, ++q) {
-        const int b = q & 1;
-        wait_or_give_up(&sh->d1_full[b], (q >> 1) & 1, abortp, status, 47);
-        tc_fence_after_sync();
-        // this warp's token blocks: hf, hf + 4  (a tile has at most 8 blocks of 8 tokens)
-        uint32_t acc[2][8];
+      wait_or_give_up(&sh->d1_full[g], u & 1, abortp, status, 47);
+      // the GEMM2 of this group's chunk before has read the hidden operand (two chunks ago: long done)
+      wait_or_give_up(&sh->hid_free[g], (u & 1) ^ 1, abortp, status, 48);
+      if (*abortp) break;
+      tc_fence_after_sync();
+      // this warp's four token blocks (a tile has at most 8 blocks of 8 tokens), all in registers at once:
+      // sixteen independent GELU chains per thread keep a scheduler with two such warps issuing
+      {
+        uint32_t acc[4][8];
 #pragma unroll
-        for (int i = 0; i < 2; ++i) {
-          const int blk = hf + 4 * i;
-          if (blk < nblk) tmem_ld8(lane_addr + b * npad + blk * 8, acc[i]);
+        for (int i = 0; i < 4; ++i) {
+          const int blk = hf + 2 * i;
+          if (blk < nblk) tmem_ld8(lane_addr + g * npad + blk * 8, acc[i]);
         }
         tmem_ld_wait();
-        tc_fence_before_sync();
-        mbar_arrive_warp(&sh->d1_free[b]);
-        uint4 hi[2], lo[2];
+        tc_fence_before_sync();                // the accumulator buffer is in registers: GEMM1 may refill it
+        mbar_arrive_warp(&sh->d1_free[g]);
 #pragma unroll
-        for (int i = 0; i < 2; ++i) {
-          const int blk = hf + 4 * i;
+        for (int i = 0; i < 4; ++i) {
+          const int blk = hf + 2 * i;
           if (blk < nblk) {
             uint32_t ph[4], pl[4];
 #pragma unroll
@@ -304,27 +319,33 @@ __global__ void __launch_bounds__(FL_THREADS) feature_tc_kernel(
               ph[e] = *reinterpret_cast<const uint32_t*>(&hh);
               pl[e] = *reinterpret_cast<const uint32_t*>(&ll);
             }
-            hi[i] = make_uint4(ph[0], ph[1], ph[2], ph[3]);
-            lo[i] = make_uint4(pl[0], pl[1], pl[2], pl[3]);
+            *reinterpret_cast<uint4*>(hrow + blk * 2048) = make_uint4(ph[0], ph[1], ph[2], ph[3]);
+            *reinterpret_cast<uint4*>(hrow + hbytes + blk * 2048) = make_uint4(pl[0], pl[1], pl[2], pl[3]);
           }
         }
-        wait_or_give_up(&sh->hid_free, (q & 1) ^ 1, abortp, status, 48);
-#pragma unroll
-        for (int i = 0; i < 2; ++i) {
-          const int blk = hf + 4 * i;
-          if (blk < nblk) {
-            *reinterpret_cast<uint4*>(hrow + blk * 2048) = hi[i];
-            *reinterpret_cast<uint4*>(hrow + hbytes + blk * 2048) = lo[i];
-          }
-        }
-        fence_proxy_async_smem();
-        mbar_arrive_warp(&sh->hid_full);
       }
-      if (*abortp) break;
-      // ---- layer 2 result: token = accumulator lane ----
+      fence_proxy_async_smem();
+      mbar_arrive_warp(&sh->hid_full[g]);
+      c += FL_GROUPS;
+      while (c >= nchunk) { c -= nchunk; ++n; }
+    }
+  } else {
+    // ---------------- finishing warps, one per lane quadrant: layer 2's result, token = accumulator lane ----------------
+    const int quad = warp & 3;
+    const int j = quad * 32 + lane;
+    const uint32_t lane_addr = tmem + ((uint32_t)(quad * 32) << 16);
+    for (int n = 0; n < my_items && !*abortp; ++n) {
+      const FtItem im = ft_item(blockIdx.x + n * gridDim.x, gm);
+      const int which = im.which, lh = im.lh;
+      const int a = n & 1;
+      const int b0 = im.tile * npad, nb = min(npad, p.B - b0);
+      float c1 = 1.f, c2 = 1.f;
+      if (which && p.psi_scale) { c1 = __ldg(p.psi_scale + lh * 2); c2 = __ldg(p.psi_scale + lh * 2 + 1); }
+      wait_or_give_up(&sh->aux_full[a], (n >> 1) & 1, abortp, status, 51);   // the item's W3
       wait_or_give_up(&sh->d2_full, n & 1, abortp, status, 49);
+      if (*abortp) break;
       tc_fence_after_sync();
-      const bool mine = hf == 0 && quad * 32 < nb;         // warp-uniform
+      const bool mine = quad * 32 < nb;                    // warp-uniform
       uint32_t g2[16];
       if (mine) {
 #pragma unroll
@@ -341,10 +362,10 @@ __global__ void __launch_bounds__(FL_THREADS) feature_tc_kernel(
           const __half* w3 = &sh->w3[a][0];
 #pragma unroll
           for (int r = 0; r < R; ++r) {
-            float s = 0.f;
+            float sacc = 0.f;
 #pragma unroll
-            for (int rr = 0; rr < R; ++rr) s = fmaf(gv[rr], __half2float(w3[rr * R + r]), s);
-            out[r] = fabsf(s);
+            for (int rr = 0; rr < R; ++rr) sacc = fmaf(gv[rr], __half2float(w3[rr * R + r]), sacc);
+            out[r] = fabsf(sacc);
           }
         } else {
 #pragma unroll
@@ -637,7 +658,7 @@ bool feature_tc_supported(const Dims& d) {
 }
 
 static size_t ft_fixed_smem(const Dims& d, int npad) {
-  return (size_t)4 * npad * 256 + (size_t)(d.R == 16 ? 4 : 2) * d.Rp * d.R * 2 + sizeof(FtShared) + 1024;
+  return (size_t)(2 * FL_GROUPS + 2) * npad * 256 + (size_t)(d.R == 16 ? 4 : 2) * d.Rp * d.R * 2 + sizeof(FtShared) + 1024;
 }
 
 int launch_feature_tc(less_ctx* c, const FmParams& p_in, cudaStream_t s) {

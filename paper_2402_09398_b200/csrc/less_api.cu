@@ -226,6 +226,9 @@ int less_create(const less_config* cfg, const less_weights* w, void* arena, size
     if (!strcmp(e, "rows")) c->group_path = 2;
   c->sms = 148;
   cudaDeviceGetAttribute(&c->sms, cudaDevAttrMultiProcessorCount, c->device);
+  int cluster_launch = 0;                               // e.g. off under some partitioning modes: then the step stays two kernels
+  if (cudaDeviceGetAttribute(&cluster_launch, cudaDevAttrClusterLaunch, c->device) != cudaSuccess || !cluster_launch)
+    c->small_step = 0;
   // H_0 = 0, z_0 = 0, no live slots, clean status
   cudaError_t e = cudaMemset(c->a.H, 0, (size_t)d.I * d.R * d.D * 4);
   if (e == cudaSuccess) e = cudaMemset(c->a.z, 0, (size_t)d.I * d.R * 4);
