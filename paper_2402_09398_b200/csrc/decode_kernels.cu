@@ -9,6 +9,7 @@
 
 #include "feature_gemv.cuh"
 #include "feature_mlp.cuh"
+#include "pipeline.cuh"
 
 namespace less {
 
@@ -226,10 +227,19 @@ __device__ __forceinline__ size_t decode_instance(const DecParams& p) {
 //   inv   [G]      1 / normaliser of each head
 //   hcol  [R]      column d of H as read for Eq. 3
 //   D     head dimension: a slot row is D / 8 chunks of 16 bytes; threads d < D own a column of H
+//   stg   copies of the instance's V rows, scores, positions and cached psi the caller holds in shared
+//         memory (the one-launch step of small workloads), or all null: read them from the arena
+struct TailStage {
+  const __half* V = nullptr;        // [N][D]
+  const float* acc = nullptr;       // [Np]
+  const int32_t* pos = nullptr;     // [Np]
+  const float* psic = nullptr;      // [N][R]
+};
 template <int R, int G, bool kCaptured, int D = kHeadDim>
 __device__ __forceinline__ void decode_tail(const DecParams& p, size_t inst, int n, int t_now, const float* s_sc, int Ns,
                                             const float (&inv)[G], const float (&hcol)[R], const uint4& knew,
-                                            const uint4& vnew, unsigned long long* s_key, int* s_vic) {
+                                            const uint4& vnew, unsigned long long* s_key, int* s_vic,
+                                            const TailStage stg = TailStage()) {
   constexpr int LPR = D / 8;                           // lanes per slot row
   const int tid = threadIdx.x, d = tid, l16 = tid % LPR, rg = tid / LPR;
   const bool own = D == DEC_THREADS || d < D;
@@ -237,9 +247,11 @@ __device__ __forceinline__ void decode_tail(const DecParams& p, size_t inst, int
   const bool use_state = !(p.flags & LESS_NO_STATE);
   float* Hb = p.a.H + inst * (size_t)R * D;
   float* zb = p.a.z + inst * R;
-  const __half* Vb = p.a.vslots + inst * (size_t)N * D;
+  const __half* Vb = stg.V ? stg.V : p.a.vslots + inst * (size_t)N * D;
   int32_t* posb = p.a.pos + inst * (size_t)p.Np;
   float* accb = p.a.acc + inst * (size_t)p.Np;
+  const int32_t* pos_r = stg.V ? stg.pos : posb;        // where the step reads them (never both copies of a slot
+  const float* acc_r = stg.V ? stg.acc : accb;         // after its write below: reads come first)
   const bool full = (n == N);
   const bool lambda_policy = (p.flags & LESS_POLICY_LAMBDA) != 0;
   const bool tova_policy = G == 1 && (p.flags & LESS_POLICY_TOVA) != 0;
@@ -249,10 +261,10 @@ __device__ __forceinline__ void decode_tail(const DecParams& p, size_t inst, int
 #pragma unroll
     for (int g = 0; g < G; ++g) ps_sum = G == 1 ? s_sc[i] * inv[0] : fmaf(s_sc[g * Ns + i], inv[g], ps_sum);
     // TOVA scores an entry by this query's probability alone; H2O accumulates
-    const float a = tova_policy ? ps_sum : accb[i] + ps_sum;
+    const float a = tova_policy ? ps_sum : acc_r[i] + ps_sum;
     accb[i] = a;
     if (full) {
-      const int ps = posb[i];
+      const int ps = pos_r[i];
       if (tova_policy) {                               // TOVA: every entry competes, nothing is protected
         const unsigned long long key = ((unsigned long long)__float_as_uint(a) << 32) | (unsigned int)ps;
         best = key < best ? key : best;
@@ -301,7 +313,7 @@ __device__ __forceinline__ void decode_tail(const DecParams& p, size_t inst, int
     }
     const int vpos = (int)(unsigned int)(best & 0xffffffffull);
     for (int i = tid; i < n; i += DEC_THREADS)
-      if (posb[i] == vpos && best != ~0ull) *s_vic = i;   // positions are unique
+      if (pos_r[i] == vpos && best != ~0ull) *s_vic = i;   // positions are unique
     __syncthreads();
     slot = *s_vic;
     if (slot < 0) {                                    // cannot happen with recent >= 1; refuse
@@ -315,7 +327,7 @@ __device__ __forceinline__ void decode_tail(const DecParams& p, size_t inst, int
     if (tid == 0 && p.evicted_pos) p.evicted_pos[inst] = vpos;
     // ---- Eq. 4 / Eq. 5: absorb the victim (psi acts on the key: the state is the KV head's) ----
     if (use_state) {
-      const float* psv = p.a.psic + (inst * (size_t)N + slot) * R;
+      const float* psv = stg.V ? stg.psic + (size_t)slot * R : p.a.psic + (inst * (size_t)N + slot) * R;
       if (own) {
         const float vv = __half2float(Vb[(size_t)slot * D + d]);
 #pragma unroll
@@ -530,6 +542,7 @@ constexpr int SS_THREADS = 512;       // threads per CTA of the small-step kerne
 constexpr int SS_FEAT = 4;           // feature-map CTAs per head
 constexpr int SS_MAXB = 4;           // batch rows (decode CTAs) per head: SS_FEAT + SS_MAXB = the portable cluster size
 constexpr int SS_MAXJ = 128;         // hidden units per feature CTA at the widest hidden layer (512)
+constexpr int SS_STAGE_SLOTS = 128;  // up to this many slots a decode CTA keeps its instance's rows in shared memory
 
 struct SsMaps {
   const __half* w1[2];    // W_phi1, W_psi1 [L, Hd, D, Rp]
@@ -545,6 +558,8 @@ __device__ __forceinline__ uint32_t cluster_rank() {
   return r;
 }
 __device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
+// an arrival that publishes nothing
+__device__ __forceinline__ void cluster_arrive_relaxed() { asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory"); }
 __device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
 // writes v at `local` (an address in this CTA's shared memory) in the shared memory of CTA `rank` of the cluster
 __device__ __forceinline__ void cluster_peer_store_f32(float* local, uint32_t rank, float v) {
@@ -572,10 +587,6 @@ __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t& r0, uint32_t& r1, ui
 
 __device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gmem_src)
-               : "memory");
-}
-__device__ __forceinline__ void cp_async8(void* smem_dst, const void* gmem_src) {
-  asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gmem_src)
                : "memory");
 }
 __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
@@ -608,6 +619,10 @@ __device__ __forceinline__ float wide_sum(float v, float* red) {
 struct SsDecoder {
   const float* part;      // [SS_FEAT][2][R] the feature CTAs' partial layer-2 sums of this batch row (written by them)
   float* own;             // this CTA's: gsum [2 R], phi [R], c1, c2, (pad), then W3 [R R] as halves
+  const __half* K;        // the instance's K rows in shared memory, or null: not staged (too many slots)
+  TailStage tail;         // ... and what the second half of the step reads
+  uint64_t* bar;          // the bulk copies of all that (and of W3) complete here
+  int* abort;
 };
 
 // The decode step of one instance in the small-step kernel.  The same arithmetic as decode_kernel, laid
@@ -617,7 +632,7 @@ struct SsDecoder {
 // leave, and the first four meet the feature CTAs, finish phi(q_t), psi(k_t), and run Eq. 3 and the
 // common second half of the step (decode_tail).
 template <int R, bool kCaptured>
-__device__ __forceinline__ void small_step_decode(const DecParams& p, const size_t inst, float* dsm, const SsDecoder& cl) {
+__device__ __forceinline__ void small_step_decode(const DecParams& p, const size_t inst, float* dsm, const SsDecoder cl) {
   constexpr int RG = SS_THREADS / 16;              // slot rows per pass
   float* s_sc = dsm;                               // [Np + 4] scores, then e^{s - m}
   float* s_red = s_sc + p.Np + 4;                  // [RG][128] partial numerators
@@ -631,8 +646,9 @@ __device__ __forceinline__ void small_step_decode(const DecParams& p, const size
   const int t_now = kCaptured ? __ldcg(p.a.tpos) : p.t;
   const int n = p.a.count[inst];
   if (n < 0 || n > N) {                            // refuse a corrupt count, touch nothing; the cluster is still met
+    __syncthreads();                               // the barrier's initialisation is visible
+    wait_or_give_up(cl.bar, 0, cl.abort, p.a.status, 130);   // leave with no copy into this CTA's shared memory in flight
     if (tid >= DEC_THREADS) return;
-    cp_async_wait_all();
     cluster_wait();                                // the start-up phase, then the one the feature CTAs arrive at
     cluster_arrive();
     cluster_wait();
@@ -641,8 +657,9 @@ __device__ __forceinline__ void small_step_decode(const DecParams& p, const size
     return;
   }
   const float scale = 0.08838834764831845f;        // 1 / sqrt(128)
-  const __half* Kb = p.a.kslots + inst * (size_t)N * kHeadDim;
-  const __half* Vb = p.a.vslots + inst * (size_t)N * kHeadDim;
+  const bool staged = cl.K != nullptr;
+  const __half* Kb = staged ? cl.K : p.a.kslots + inst * (size_t)N * kHeadDim;
+  const __half* Vb = staged ? cl.tail.V : p.a.vslots + inst * (size_t)N * kHeadDim;
   // the state is last step's: its loads are under way long before the maps arrive
   const int d = tid & (kHeadDim - 1);
   float hcol[R], zr[R];
@@ -658,6 +675,8 @@ __device__ __forceinline__ void small_step_decode(const DecParams& p, const size
   half8_to_float(*reinterpret_cast<const uint4*>(p.q + inst * kHeadDim + l16 * 8), qf);
   const uint4 knew = *reinterpret_cast<const uint4*>(p.k + inst * kHeadDim + l16 * 8);
   const uint4 vnew = *reinterpret_cast<const uint4*>(p.v + inst * kHeadDim + l16 * 8);
+  __syncthreads();                                 // the barrier's initialisation is visible
+  wait_or_give_up(cl.bar, 0, cl.abort, p.a.status, 131);   // the bulk copies of the instance's rows (and W3) have landed
   // ---- scores s_i = q . k_i / sqrt(D) over live slots, and the new pair ----
 #pragma unroll 2
   for (int r0 = 0; r0 < n; r0 += RG) {             // r0 is block-uniform: shuffles stay converged
@@ -730,7 +749,6 @@ __device__ __forceinline__ void small_step_decode(const DecParams& p, const size
   // ---- phi(q_t), psi(k_t): the feature CTAs' partial layer-2 sums, in rank order (Eq. 1, Eq. 2) ----
   float* gsum = cl.own;
   float* phis = cl.own + 2 * R;
-  cp_async_wait_all();                             // W3 and the scalars, asked for when the kernel started
   cluster_wait();                                  // the start-up phase (complete long ago)
   cluster_arrive();                                // behind this barrier the feature CTAs' partial sums are here
   cluster_wait();
@@ -772,7 +790,7 @@ __device__ __forceinline__ void small_step_decode(const DecParams& p, const size
   }
   store_out(p, inst * kHeadDim + d, num / den);
   const float inv[1] = {1.0f / ((p.flags & LESS_SCORE_NORM_SPARSE) ? lsum : den)};
-  decode_tail<R, 1, kCaptured>(p, inst, n, t_now, s_sc, p.Np + 4, inv, hcol, knew, vnew, s_key, &s_vic);
+  decode_tail<R, 1, kCaptured>(p, inst, n, t_now, s_sc, p.Np + 4, inv, hcol, knew, vnew, s_key, &s_vic, cl.tail);
 }
 
 template <int R, bool kCaptured>
@@ -787,7 +805,16 @@ __global__ void __launch_bounds__(SS_THREADS) small_step_kernel(DecParams p, SsM
   const int lh = blockIdx.x / cs;                        // layer * Hd + head
   // "this CTA runs": distributed shared memory may only be touched once its owner has started.  Everyone
   // arrives here at once; whoever needs the fact waits for it much later, when it has long been true.
-  cluster_arrive();
+  cluster_arrive_relaxed();
+  // Operands come as bulk copies that complete on this barrier: a copy per contiguous piece issued by a
+  // few threads, where sixteen warps of 16-byte copies took thousands of cycles just to issue.
+  __shared__ uint64_t s_stage_bar;
+  __shared__ int s_abort;
+  if (tid == 0) {
+    mbar_init(&s_stage_bar, 1);
+    s_abort = 0;
+    mbar_fence_init();
+  }
 
   if (rank < nb) {
     // ---------------- decode CTA of batch row `rank` ----------------
@@ -795,16 +822,39 @@ __global__ void __launch_bounds__(SS_THREADS) small_step_kernel(DecParams p, SsM
     SsDecoder cl;
     cl.part = part;
     cl.own = role + p.Np + 4 + (SS_THREADS / 16) * kHeadDim;   // behind the step's scores and partial sums
+    // Everything the step reads of its instance, asked for at once: the step is otherwise a chain of dependent
+    // round trips to L2 (slot count -> K rows -> V rows -> scores and positions -> the victim's psi and V row).
+    // While the slots fit; with more of them the rows stream from the arena as in the large kernels.
+    cl.K = nullptr;
+    cl.tail = TailStage();
+    cl.bar = &s_stage_bar; cl.abort = &s_abort;
+    __half* w3s = reinterpret_cast<__half*>(cl.own + 3 * R + 4);
+    const bool stage = p.N <= SS_STAGE_SLOTS;
+    const size_t N = p.N;
+    unsigned char* st = reinterpret_cast<unsigned char*>(w3s) + R * R * 2;   // behind W3; 16-byte aligned
+    __half* Ks = reinterpret_cast<__half*>(st);
+    __half* Vs = Ks + N * kHeadDim;
+    float* accs = reinterpret_cast<float*>(Vs + N * kHeadDim);
+    int32_t* poss = reinterpret_cast<int32_t*>(accs + p.Np);
+    float* psics = reinterpret_cast<float*>(poss + p.Np);
     if (tid == 0) {
-      if (mp.psi_scale) {
-        cp_async8(cl.own + 3 * R, mp.psi_scale + lh * 2);
-      } else {
-        cl.own[3 * R] = 1.f;
-        cl.own[3 * R + 1] = 1.f;
+      const uint32_t kv = (uint32_t)(N * kHeadDim * 2), ap = (uint32_t)p.Np * 4, ps = (uint32_t)(N * R * 4);
+      mbar_expect_tx(&s_stage_bar, (uint32_t)(R * R * 2) + (stage ? 2 * kv + 2 * ap + ps : 0u));
+      bulk_g2s(w3s, mp.w3 + (size_t)lh * R * R, R * R * 2, &s_stage_bar);
+      if (stage) {
+        bulk_g2s(Ks, p.a.kslots + inst * N * kHeadDim, kv, &s_stage_bar);
+        bulk_g2s(Vs, p.a.vslots + inst * N * kHeadDim, kv, &s_stage_bar);
+        bulk_g2s(accs, p.a.acc + inst * (size_t)p.Np, ap, &s_stage_bar);
+        bulk_g2s(poss, p.a.pos + inst * (size_t)p.Np, ap, &s_stage_bar);
+        bulk_g2s(psics, p.a.psic + inst * N * R, ps, &s_stage_bar);
       }
     }
-    if (tid < R * R / 8)
-      cp_async16(reinterpret_cast<__half*>(cl.own + 3 * R + 4) + tid * 8, mp.w3 + (size_t)lh * R * R + tid * 8);
+    if (tid >= SS_THREADS - 2)                           // psi's learnable scalars, by threads of a warp that has time to wait for them
+      cl.own[3 * R + (tid & 1)] = mp.psi_scale ? mp.psi_scale[lh * 2 + (tid & 1)] : 1.f;
+    if (stage) {
+      cl.K = Ks;
+      cl.tail.V = Vs; cl.tail.acc = accs; cl.tail.pos = poss; cl.tail.psic = psics;
+    }
     small_step_decode<R, kCaptured>(p, inst, role, cl);  // the barriers inside order these writes before their use
     return;
   }
@@ -1526,7 +1576,8 @@ int launch_small_step(less_ctx* c, const void* q, const void* k, const void* v, 
   cudaStreamIsCapturing(s, &capturing);
   const bool captured = capturing == cudaStreamCaptureStatusActive;
   // the partial sums, then the larger of the two roles' shared memory
-  const size_t dec_bytes = (size_t)(d.Np + 4 + (SS_THREADS / 16) * kHeadDim) * 4 + (size_t)(3 * d.R + 4) * 4 + (size_t)d.R * d.R * 2;
+  size_t dec_bytes = (size_t)(d.Np + 4 + (SS_THREADS / 16) * kHeadDim) * 4 + (size_t)(3 * d.R + 4) * 4 + (size_t)d.R * d.R * 2;
+  if (d.N <= SS_STAGE_SLOTS) dec_bytes += (size_t)2 * d.N * kHeadDim * 2 + (size_t)2 * d.Np * 4 + (size_t)d.N * d.R * 4;
   const size_t feat_bytes = (size_t)2 * kHeadDim * (SS_MAXJ + 8) * 2 + (size_t)2 * SS_MAXB * kHeadDim * 2 +
                             (size_t)2 * SS_MAXJ * d.R * 2 + (size_t)2 * SS_MAXB * SS_MAXJ * 4;
   const size_t smem = (size_t)SS_FEAT * 2 * d.R * 4 + (dec_bytes > feat_bytes ? dec_bytes : feat_bytes);
