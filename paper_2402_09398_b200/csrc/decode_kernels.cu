@@ -9,7 +9,7 @@
 
 #include "feature_gemv.cuh"
 #include "feature_mlp.cuh"
-#include "pipeline.cuh"
+#include "tc_common.cuh"
 
 namespace less {
 
@@ -794,10 +794,13 @@ __device__ __forceinline__ void small_step_decode(const DecParams& p, const size
 }
 
 template <int R, bool kCaptured>
-__global__ void __launch_bounds__(SS_THREADS) small_step_kernel(DecParams p, SsMaps mp) {
-  extern __shared__ float dsm[];
+__global__ void __launch_bounds__(SS_THREADS) small_step_kernel(const __grid_constant__ CUtensorMap tm_w1phi,
+                                                                const __grid_constant__ CUtensorMap tm_w1psi, DecParams p,
+                                                                SsMaps mp) {
+  extern __shared__ __align__(1024) float dsm[];
   float* part = dsm;                                     // [SS_FEAT][2][R]  a decode CTA's inbox for the partial layer-2 sums
-  float* role = part + SS_FEAT * 2 * R;                  // the rest belongs to the CTA's role
+  float* role = dsm + 256;                               // the rest belongs to the CTA's role (on a 1024-byte boundary:
+                                                         // the feature CTAs' weight tiles are 128-byte-swizzled)
   const int tid = threadIdx.x;
   const int nb = p.B;                                    // <= SS_MAXB
   const int cs = nb + SS_FEAT;                           // CTAs per cluster
@@ -865,19 +868,35 @@ __global__ void __launch_bounds__(SS_THREADS) small_step_kernel(DecParams p, SsM
   const int fr = rank - nb;
   const int Rp = mp.Rp, J = Rp / SS_FEAT;                // hidden units of this CTA: 128, 64 or 32
   const int lj = 31 - __clz(J);                          // J = 1 << lj
-  const int lpr = J / 8, llpr = lj - 3;                  // 16-byte chunks per weight row of this CTA: 16, 8 or 4
-  const int ws = J + 8;                                  // padded row of the staged W1: the transposing loads below then
-                                                         // find their eight rows in eight different bank groups
-  __half* w1s = reinterpret_cast<__half*>(role);         // [2][128 rows][J + 8]
+  // W1 slice of this CTA: with 64 or 128 hidden units per CTA it comes as tiled TMA loads of 128 rows x 64
+  // columns (two or four per CTA; the same tensor maps the tensor-core feature kernels use), 128-byte-swizzled,
+  // which the transposing loads below undo; with 32 units (hidden width 128) as 16-byte asynchronous copies into
+  // rows padded by 16 bytes.  Either way the eight rows of a transposing load lie in eight different bank groups.
+  const bool tiled = J >= 64;
+  const int ws = tiled ? 64 : J + 8;                     // halves per staged row
+  __half* w1s = reinterpret_cast<__half*>(role);         // tiled: [2 maps][J / 64 halves][128 rows][64]; else [2][128 rows][J + 8]
   __half* xh = w1s + 2 * kHeadDim * (SS_MAXJ + 8);       // [2][SS_MAXB][128] q rows, then k rows
   __half* w2h = xh + 2 * SS_MAXB * kHeadDim;             // [2][J][R] this CTA's rows of W2
   float* hs = reinterpret_cast<float*>(w2h + 2 * SS_MAXJ * R);   // [2][SS_MAXB][SS_MAXJ] gelu(hidden)
-  // ---- stage everything with asynchronous copies: all loads in flight at once, no registers held ----
-  for (int e = tid; e < 2 * kHeadDim * lpr; e += SS_THREADS) {
-    const int m = e >> (7 + llpr), d = (e >> llpr) & (kHeadDim - 1), ch = e & (lpr - 1);
-    cp_async16(w1s + (size_t)(m * kHeadDim + d) * ws + ch * 8,
-               mp.w1[m] + ((size_t)lh * kHeadDim + d) * Rp + (size_t)fr * J + ch * 8);
+  if (tiled) {
+    if (smem_misaligned(dsm, p.a.status, 133)) return;   // (a CTA that leaves is no longer waited for by its cluster)
+    if (tid == 0) {
+      const int halves = J >> 6;
+      mbar_expect_tx(&s_stage_bar, (uint32_t)(2 * halves * kHeadDim * 128));
+      for (int m = 0; m < 2; ++m)
+        for (int i = 0; i < halves; ++i)
+          tma_load_2d(w1s + (size_t)(m * halves + i) * kHeadDim * 64, m ? &tm_w1psi : &tm_w1phi, fr * J + i * 64,
+                      lh * kHeadDim, &s_stage_bar);
+    }
+  } else {
+    const int lpr = J / 8, llpr = lj - 3;                // 16-byte chunks per weight row of this CTA
+    for (int e = tid; e < 2 * kHeadDim * lpr; e += SS_THREADS) {
+      const int m = e >> (7 + llpr), d = (e >> llpr) & (kHeadDim - 1), ch = e & (lpr - 1);
+      cp_async16(w1s + (size_t)(m * kHeadDim + d) * ws + ch * 8,
+                 mp.w1[m] + ((size_t)lh * kHeadDim + d) * Rp + (size_t)fr * J + ch * 8);
+    }
   }
+  // the few q / k rows and this CTA's rows of W2 with 16-byte asynchronous copies (q, k may lie in pinned host memory)
   if (tid < 2 * nb * 16) {
     const int m = tid / (nb * 16), b = (tid >> 4) % nb, ch = tid & 15;
     cp_async16(xh + (m * SS_MAXB + b) * kHeadDim + ch * 8,
@@ -889,7 +908,8 @@ __global__ void __launch_bounds__(SS_THREADS) small_step_kernel(DecParams p, SsM
     cp_async16(w2h + (m * J * R) + ch * 8, mp.w2[m] + ((size_t)lh * Rp + (size_t)fr * J) * R + ch * 8);
   }
   cp_async_wait_all();
-  __syncthreads();
+  __syncthreads();                                       // ... which also makes the barrier's initialisation visible
+  if (tiled) wait_or_give_up(&s_stage_bar, 0, &s_abort, p.a.status, 132);
 
   // ---- layer 1 as warp-level MMAs (fp16 operands, used exactly; fp32 sums): the head's batch rows are the
   //      first rows of the 16-row A operand (the rest zero), a tile of eight hidden units the B operand, read
@@ -902,7 +922,12 @@ __global__ void __launch_bounds__(SS_THREADS) small_step_kernel(DecParams p, SsM
     for (int tile = warp; tile < 2 * tiles; tile += SS_THREADS / 32) {
       const int m = tile >= tiles, n0 = (tile - m * tiles) * 8;
       const __half* xrow = xh + (m * SS_MAXB + row) * kHeadDim + 2 * (lane & 3);
-      const __half* wrow = w1s + (size_t)(m * kHeadDim + (lane >> 3) * 8 + (lane & 7)) * ws + n0;
+      // row k = 32 kk + 8 (lane >> 3) + (lane & 7) of the tile's eight columns: in a swizzled tile the 16-byte
+      // chunk c of row k lies at chunk c ^ (k & 7) of its 128-byte row
+      const int krow = (lane >> 3) * 8 + (lane & 7);
+      const __half* wrow = tiled ? w1s + (size_t)(m * (J >> 6) + (n0 >> 6)) * kHeadDim * 64 + (size_t)krow * 64 +
+                                       ((((n0 & 63) >> 3) ^ (lane & 7)) << 3)
+                                 : w1s + (size_t)(m * kHeadDim + krow) * ws + n0;
       float c[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
       for (int kk = 0; kk < kHeadDim / 32; ++kk) {       // two k-steps of 16 input dimensions per pass
@@ -1580,7 +1605,7 @@ int launch_small_step(less_ctx* c, const void* q, const void* k, const void* v, 
   if (d.N <= SS_STAGE_SLOTS) dec_bytes += (size_t)2 * d.N * kHeadDim * 2 + (size_t)2 * d.Np * 4 + (size_t)d.N * d.R * 4;
   const size_t feat_bytes = (size_t)2 * kHeadDim * (SS_MAXJ + 8) * 2 + (size_t)2 * SS_MAXB * kHeadDim * 2 +
                             (size_t)2 * SS_MAXJ * d.R * 2 + (size_t)2 * SS_MAXB * SS_MAXJ * 4;
-  const size_t smem = (size_t)SS_FEAT * 2 * d.R * 4 + (dec_bytes > feat_bytes ? dec_bytes : feat_bytes);
+  const size_t smem = 1024 + (dec_bytes > feat_bytes ? dec_bytes : feat_bytes);
   // a step this small is bound by the host's work per launch as well: names and attributes are set once
   LaunchScope scope(c, LESS_KERNEL_DECODE, s);
   void* kern = d.R == 8 ? (captured ? (void*)small_step_kernel<8, true> : (void*)small_step_kernel<8, false>)
@@ -1608,7 +1633,18 @@ int launch_small_step(less_ctx* c, const void* q, const void* k, const void* v, 
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  void* args[] = {&p, &mp};
+  // W1 of phi / psi as tensor maps (boxes of 128 rows x 64 columns, 128-byte-swizzled), kept in the context
+  // like the feature kernels' (the same two maps)
+  static_assert(sizeof(CUtensorMap) <= 128, "tensor map cache slot");
+  CUtensorMap* tmc = reinterpret_cast<CUtensorMap*>(c->tm_cache);
+  if (!c->tm_w_ok) {
+    const uint64_t lh = (uint64_t)d.L * d.Hd;
+    if (!make_tmap_f16_2d(&tmc[2], c->w.w_phi1, lh * kHeadDim, d.Rp, (uint64_t)d.Rp * 2, kHeadDim) ||
+        !make_tmap_f16_2d(&tmc[3], c->w.w_psi1, lh * kHeadDim, d.Rp, (uint64_t)d.Rp * 2, kHeadDim))
+      return fail_cuda("tensor map of W1");
+    c->tm_w_ok = true;
+  }
+  void* args[] = {&tmc[2], &tmc[3], &p, &mp};
   if (cudaLaunchKernelExC(&cfg, kern, args) != cudaSuccess) return fail_cuda("launch of small_step_kernel");
   return check_launch("small_step_kernel");
 }
