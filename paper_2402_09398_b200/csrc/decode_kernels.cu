@@ -1565,8 +1565,8 @@ int launch_decode(less_ctx* c, const void* q, const void* k, const void* v, void
 
 // Whether a step of this context runs as the single small_step_kernel launch: the shapes the kernel
 // takes, and (unless forced) few enough heads that all its CTAs find a multiprocessor of their own -
-// up to there a step is bound by launches and latency (measured: 8 heads 8.3 against 8.7 us per step
-// replayed from a graph, 10.3 against 11.4 us by direct calls), past it by the weight stream, which
+// up to there a step is bound by launches and latency (measured: 8 heads 7.2 against 8.7 us per step
+// replayed from a graph, 8.2 against 11.5 us by direct calls), past it by the weight stream, which
 // the tensor-core feature kernel moves faster.
 bool small_step_path(const less_ctx* c) {
   const Dims& d = c->d;
