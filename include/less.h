@@ -37,7 +37,7 @@
  *     LESS_SMALL_STEP=0|1 (a decode step as ONE launch - a thread-block cluster per head splits the
  *     two MLPs and runs the step of each batch row - never / whenever the shape allows: head_dim 128,
  *     group 1, at most 4 batch rows, hidden in {128, 256, 512}, the state in use; by default when
- *     layers x heads x (batch + 4) CTAs fit the GPU's multiprocessors at once).
+ *     layers x heads x (batch + 4) CTAs are at most two per multiprocessor).
  */
 #ifndef LESS_B200_H
 #define LESS_B200_H

@@ -809,6 +809,11 @@ __global__ void __launch_bounds__(SS_THREADS) small_step_kernel(const __grid_con
   // "this CTA runs": distributed shared memory may only be touched once its owner has started.  Everyone
   // arrives here at once; whoever needs the fact waits for it much later, when it has long been true.
   cluster_arrive_relaxed();
+  // Programmatic dependent launch, both ways: the next kernel in the stream (the next step, typically) may
+  // start while this one runs, and this one may have started while its predecessor still ran.  Whatever an
+  // earlier kernel may have written - the step's q, k, v, the arena - is read only behind pdl_wait_primary();
+  // the feature-map weights never change and are fetched before it.
+  pdl_launch_dependents();
   // Operands come as bulk copies that complete on this barrier: a copy per contiguous piece issued by a
   // few threads, where sixteen warps of 16-byte copies took thousands of cycles just to issue.
   __shared__ uint64_t s_stage_bar;
@@ -840,6 +845,7 @@ __global__ void __launch_bounds__(SS_THREADS) small_step_kernel(const __grid_con
     float* accs = reinterpret_cast<float*>(Vs + N * kHeadDim);
     int32_t* poss = reinterpret_cast<int32_t*>(accs + p.Np);
     float* psics = reinterpret_cast<float*>(poss + p.Np);
+    pdl_wait_primary();
     if (tid == 0) {
       const uint32_t kv = (uint32_t)(N * kHeadDim * 2), ap = (uint32_t)p.Np * 4, ps = (uint32_t)(N * R * 4);
       mbar_expect_tx(&s_stage_bar, (uint32_t)(R * R * 2) + (stage ? 2 * kv + 2 * ap + ps : 0u));
@@ -896,16 +902,18 @@ __global__ void __launch_bounds__(SS_THREADS) small_step_kernel(const __grid_con
                  mp.w1[m] + ((size_t)lh * kHeadDim + d) * Rp + (size_t)fr * J + ch * 8);
     }
   }
-  // the few q / k rows and this CTA's rows of W2 with 16-byte asynchronous copies (q, k may lie in pinned host memory)
-  if (tid < 2 * nb * 16) {
-    const int m = tid / (nb * 16), b = (tid >> 4) % nb, ch = tid & 15;
-    cp_async16(xh + (m * SS_MAXB + b) * kHeadDim + ch * 8,
-               (m == 0 ? p.q : p.k) + ((size_t)b * p.LH + lh) * kHeadDim + ch * 8);
-  }
+  // this CTA's rows of W2 and, once the kernels before this one are done, the few q / k rows with 16-byte
+  // asynchronous copies (q, k may lie in pinned host memory)
   const int w2chunks = J * R / 8;                        // 16-byte chunks of this CTA's rows of W2, per map (contiguous)
   if (tid < 2 * w2chunks) {
     const int m = tid >= w2chunks, ch = tid - m * w2chunks;
     cp_async16(w2h + (m * J * R) + ch * 8, mp.w2[m] + ((size_t)lh * Rp + (size_t)fr * J) * R + ch * 8);
+  }
+  pdl_wait_primary();
+  if (tid < 2 * nb * 16) {
+    const int m = tid / (nb * 16), b = (tid >> 4) % nb, ch = tid & 15;
+    cp_async16(xh + (m * SS_MAXB + b) * kHeadDim + ch * 8,
+               (m == 0 ? p.q : p.k) + ((size_t)b * p.LH + lh) * kHeadDim + ch * 8);
   }
   cp_async_wait_all();
   __syncthreads();                                       // ... which also makes the barrier's initialisation visible
@@ -1564,16 +1572,16 @@ int launch_decode(less_ctx* c, const void* q, const void* k, const void* v, void
 }
 
 // Whether a step of this context runs as the single small_step_kernel launch: the shapes the kernel
-// takes, and (unless forced) few enough heads that all its CTAs find a multiprocessor of their own -
-// up to there a step is bound by launches and latency (measured: 8 heads 7.2 against 8.7 us per step
-// replayed from a graph, 8.2 against 11.5 us by direct calls), past it by the weight stream, which
-// the tensor-core feature kernel moves faster.
+// takes, and (unless forced) no more CTAs than two per multiprocessor - up to there a step is bound by
+// launches and latency (measured, batch 1: 8 heads 6.7 against 8.7 us per step replayed from a graph, 7.7
+// against 11.3 us by direct calls; 32 heads 7.6 against 9.0 and 7.7 against 11.2; 64 heads 11.8 against
+// 9.5 and 11.6 against 11.8), past it by the weight stream, which the tensor-core feature kernel moves faster.
 bool small_step_path(const less_ctx* c) {
   const Dims& d = c->d;
   if (c->small_step == 0 || d.general || d.G != 1 || d.D != kHeadDim || (d.flags & LESS_NO_STATE)) return false;
   if (d.B > SS_MAXB || (d.Rp != 128 && d.Rp != 256 && d.Rp != 512) || c->seg_nl != d.L) return false;
   if (c->feature_path != 2) return false;             // a feature-map kernel was asked for by name
-  return c->small_step == 1 || d.L * d.Hd * (d.B + SS_FEAT) <= c->sms;
+  return c->small_step == 1 || d.L * d.Hd * (d.B + SS_FEAT) <= 2 * c->sms;
 }
 
 int launch_small_step(less_ctx* c, const void* q, const void* k, const void* v, void* out, int32_t* evicted_pos,
@@ -1626,13 +1634,15 @@ int launch_small_step(less_ctx* c, const void* q, const void* k, const void* v, 
   cfg.blockDim = dim3(SS_THREADS);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = s;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = d.B + SS_FEAT;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = (c->pdl && !c->profile) ? 2 : 1;       // with per-kernel timing on, an ordinary launch
   // W1 of phi / psi as tensor maps (boxes of 128 rows x 64 columns, 128-byte-swizzled), kept in the context
   // like the feature kernels' (the same two maps)
   static_assert(sizeof(CUtensorMap) <= 128, "tensor map cache slot");
