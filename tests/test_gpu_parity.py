@@ -105,7 +105,7 @@ def test_prefill_and_teacher_forced_decode(variant, monkeypatch):
 
 @pytest.mark.parametrize("variant", ["one_row_eight_heads", "rank16_two_rows", "four_rows_hidden256",
                                      "hidden128_scaled", "sparse_norm", "lambda_masking", "tova", "from_empty",
-                                     "by_size"])
+                                     "by_size", "odd_slots", "more_slots_than_staged"])
 def test_small_step_single_launch(variant, monkeypatch):
     """The single-launch step for workloads of a few heads (a cluster of CTAs per head computes phi(q_t)
     and psi(k_t), then one CTA per batch row runs Algorithm 1): every step against the oracle, started
@@ -132,6 +132,10 @@ def test_small_step_single_launch(variant, monkeypatch):
         w = small(47, prompt=0, steps=30, heavy=5, recent=6, weight_std=0.2)
     elif variant == "by_size":              # no switch: few heads go this way by themselves
         monkeypatch.delenv("LESS_SMALL_STEP")
+    elif variant == "odd_slots":            # 21 slots: the staged copies' sizes and offsets off the round numbers
+        w = small(35, heavy=10, recent=11, weight_std=0.2)
+    elif variant == "more_slots_than_staged":   # 170 slots: the K / V rows stream from the arena instead
+        w = small(36, heavy=90, recent=80, prompt=400, steps=6, weight_std=0.2)
     ctx, W = _setup(w, flags, psi_scale, max_prompt=max(w.prompt, 16))
     inst = list(range(w.instances))
     if w.prompt:
