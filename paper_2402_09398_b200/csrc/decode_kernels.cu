@@ -406,6 +406,7 @@ __device__ __forceinline__ void group_eq3_and_tail(const DecParams& p, size_t in
 template <int R, bool kCaptured>
 __global__ void __launch_bounds__(DEC_THREADS) decode_kernel(DecParams p) {
   extern __shared__ float dsm[];
+  pdl_launch_dependents();                         // the next step's feature-map kernel may come up while this one runs
   float* s_sc = dsm;                               // [Np + 4] scores, then e^{s - m}
   float* s_red = s_sc + p.Np + 4;                  // [DEC_RG][128] partial numerators
   __shared__ float s_small[DEC_THREADS / 32];

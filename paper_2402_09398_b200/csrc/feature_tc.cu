@@ -67,6 +67,8 @@ struct FtGeom {
   int kv0;         // first (layer, KV head) of this launch
   int nstage;      // ring stages
   uint32_t tmem_cols;
+  int late_inputs; // the kernel may have started before the kernel before it in the stream was done (programmatic
+                   // dependent launch): weights are fetched at once, the step's q, k only behind the wait for it
 };
 
 
@@ -107,6 +109,9 @@ __device__ __forceinline__ void ft_produce(const CUtensorMap* tm_q, const CUtens
                                            int naux, volatile int* abortp, int32_t* status) {
   uint32_t s = 0, sph = 0, a = 0, aph = 0;
   const uint64_t stream_policy = l2_evict_first_policy();
+  // The first item of a kernel that may have started early: its weights (W2, W3 and as many W1 chunks as the
+  // ring takes) are asked for at once, its input rows only once the kernels before this one are done.
+  bool inputs_later = gm.late_inputs != 0;
   for (int n = 0; n < my_items; ++n, (++a == (uint32_t)naux ? (a = 0, aph ^= 1) : 0u)) {
     const FtItem im = ft_item(blockIdx.x + n * gridDim.x, gm);
     wait_or_give_up(&aux_empty[a], aph ^ 1, abortp, status, 40);
@@ -115,14 +120,23 @@ __device__ __forceinline__ void ft_produce(const CUtensorMap* tm_q, const CUtens
     const CUtensorMap* tw1 = im.which ? tm_w1psi : tm_w1phi;
     mbar_expect_tx(&aux_full[a], (p.x_plain ? 0u : xbytes) + w2bytes + (im.which ? R * R * 2 : 0));
     unsigned char* xa = xbuf + a * xbytes;
-    if (!p.x_plain) {
+    auto load_inputs = [&]() {
+      if (p.x_plain) return;
       tma_load_2d(xa, tx, im.lh * kHeadDim, im.tile * gm.npad, &aux_full[a]);
       tma_load_2d(xa + xbytes / 2, tx, im.lh * kHeadDim + 64, im.tile * gm.npad, &aux_full[a]);
-    }
+    };
+    if (!inputs_later) load_inputs();
     // W2 comes as one contiguous copy (a tiled load of 16-byte rows is far slower)
     bulk_g2s(w2dst + a * w2bytes, p.w2[im.which] + (size_t)im.lh * p.Rp * R, w2bytes, &aux_full[a]);
     if (im.which) bulk_g2s(w3buf + a * 256, p.w3 + (size_t)im.lh * R * R, R * R * 2, &aux_full[a]);
+    const int ahead = nchunk < gm.nstage ? nchunk : gm.nstage;   // chunks whose ring stages are free without the consumer
     for (int c = 0; c < nchunk; ++c) {
+      if (inputs_later && c == ahead) {
+        pdl_wait_primary();
+        pdl_launch_dependents();                         // only now: the step's decode kernel reads the arena before it waits
+        load_inputs();
+        inputs_later = false;
+      }
       wait_or_give_up(&empty[s], sph ^ 1, abortp, status, 41);
       if (*abortp) return;
       mbar_expect_tx(&full[s], FT_STAGE_BYTES);
@@ -130,6 +144,12 @@ __device__ __forceinline__ void ft_produce(const CUtensorMap* tm_q, const CUtens
       tma_load_2d_hint(st, tw1, c * FT_CHUNK, im.lh * kHeadDim, &full[s], stream_policy);
       tma_load_2d_hint(st + FT_STAGE_BYTES / 2, tw1, c * FT_CHUNK + 64, im.lh * kHeadDim, &full[s], stream_policy);
       if (++s == (uint32_t)gm.nstage) { s = 0; sph ^= 1; }
+    }
+    if (inputs_later) {                                  // every chunk of the first item fitted the ring
+      pdl_wait_primary();
+      pdl_launch_dependents();
+      load_inputs();
+      inputs_later = false;
     }
   }
 }
@@ -485,7 +505,10 @@ __global__ void __launch_bounds__(FT_THREADS) feature_tc_small_kernel(
   tc_fence_before_sync();
   __syncthreads();
   tc_fence_after_sync();
-  pdl_launch_dependents();
+  // The decode kernel of this step may start now - unless this kernel itself started early (late_inputs):
+  // the decode kernel reads the arena before it waits for anything, so it is let go only once the
+  // kernels before this one are known to be done (the producer thread does that, behind its own wait).
+  if (!gm.late_inputs) pdl_launch_dependents();
   const uint32_t tmem = sh->tmem_base;
   volatile int* abortp = &sh->abort;
   const int my_items = blockIdx.x < gm.items ? (gm.items - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
@@ -502,6 +525,7 @@ __global__ void __launch_bounds__(FT_THREADS) feature_tc_small_kernel(
     // tiled load would have written: per half of 64 columns, 8 rows of 128 bytes, the 16-byte chunk c
     // of row r at chunk position c ^ r (128-byte swizzle); rows past the batch are zeros.
     if (p.x_plain) {
+      if (gm.late_inputs) pdl_wait_primary();           // the rows may be written by the kernel before this one
       uint32_t a = 0, aph = 0;
       for (int n = 0; n < my_items; ++n, (++a == FS_AUX ? (a = 0, aph ^= 1) : 0u)) {
         const FtItem im = ft_item(blockIdx.x + n * gridDim.x, gm);
@@ -641,7 +665,25 @@ static int launch_small(less_ctx* c, const FmParams& p, const FtGeom& gm, const 
   auto kern = feature_tc_small_kernel<R, NT>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
     return fail_cuda("shared memory opt-in of feature_tc_small_kernel");
-  kern<<<grid, FT_THREADS, smem, s>>>(tq, tk, tw1a, tw1b, p, gm, c->a.status);
+  if (!gm.late_inputs) {
+    kern<<<grid, FT_THREADS, smem, s>>>(tq, tk, tw1a, tw1b, p, gm, c->a.status);
+    return check_launch("feature_tc_small_kernel");
+  }
+  // as a programmatic dependent of the kernel before it in the stream (the decode kernel of the step before,
+  // typically): its CTAs come up and fetch their first weights while that kernel finishes
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(FT_THREADS);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  int32_t* status = c->a.status;
+  if (cudaLaunchKernelEx(&cfg, kern, tq, tk, tw1a, tw1b, p, gm, status) != cudaSuccess)
+    return fail_cuda("launch of feature_tc_small_kernel");
   return check_launch("feature_tc_small_kernel");
 }
 
@@ -672,6 +714,10 @@ int launch_feature_tc(less_ctx* c, const FmParams& p_in, cudaStream_t s) {
   gm.per_head = (d.G + 1) * gm.ntile;
   gm.kv0 = p.lh0;
   gm.items = p.nlh * gm.per_head;
+  // Every decode CTA of a step resident at once (the regime of the small-batch kernel's overlap): the next
+  // step's feature kernel may then start while this step's decode kernel finishes.  With more instances its
+  // waiting CTAs would only take multiprocessors from the decode kernel's later waves.
+  gm.late_inputs = (d.B <= 8 && c->pdl && !c->profile && d.I <= 8 * c->sms && !c->head_counters) ? 1 : 0;
   const size_t fixed = ft_fixed_smem(d, gm.npad);
   int ns = (int)((FT_SMEM_LIMIT - fixed) / FT_STAGE_BYTES);
   gm.nstage = ns > FT_MAX_STAGES ? FT_MAX_STAGES : ns;
