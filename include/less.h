@@ -25,7 +25,8 @@
  *   - D below is less_config.head_dim.
  *   - Environment, read by less_create: LESS_LOG (explain host-side failures on
  *     stderr), LESS_FEATURE_KERNEL=gemv|plain (CUDA-core feature-map kernels),
- *     LESS_NO_OVERLAP (no programmatic dependent launch of the decode kernel),
+ *     LESS_NO_OVERLAP (no programmatic dependent launches: neither the decode kernel behind its step's
+ *     feature-map kernel nor a step's first kernel behind the kernel before it in the stream),
  *     LESS_SCORE_KERNEL=plain (CUDA-core prompt scoring),
  *     LESS_FEATURE_STAGES=n (cap on the feature kernels' weight ring),
  *     LESS_GROUP_KERNEL=rows (grouped query heads: the CUDA-core decode kernel instead of
