@@ -629,6 +629,40 @@ def test_captured_step_replays_like_direct_calls(batch, group=1):
     ctx_d.close(); ctx_g.close()
 
 
+@pytest.mark.parametrize("small_step", ["0", "1"])
+def test_back_to_back_steps_equal_serialised_ones(small_step, monkeypatch):
+    """Steps launched back to back, with nothing between them: each step's first kernel may start while the
+    step before still runs (programmatic dependent launch).  Outputs of every step and the final state must be
+    bit-identical to a context that launches every kernel the ordinary way (LESS_NO_OVERLAP)."""
+    monkeypatch.setenv("LESS_SMALL_STEP", small_step)
+    w = small(33, batch=2, layers=4, heads=12, steps=24, heavy=12, recent=12, weight_std=0.2)
+    ctx_o, _ = _setup(w)
+    monkeypatch.setenv("LESS_NO_OVERLAP", "1")
+    ctx_s, _ = _setup(w)
+    monkeypatch.delenv("LESS_NO_OVERLAP")
+    for ctx in (ctx_o, ctx_s):
+        _prefill_all(ctx, w, with_out=False)
+    inputs = [wl.make_decode_inputs(w, s, DEV) for s in range(w.steps)]
+    torch.cuda.synchronize()
+    outs = {}
+    for name, ctx in (("overlapped", ctx_o), ("serial", ctx_s)):
+        bufs = [torch.empty(inputs[0][0].shape, dtype=torch.float32, device=DEV) for _ in range(w.steps)]
+        for s in range(w.steps):
+            ctx.decode_step(*inputs[s], out=bufs[s])
+        torch.cuda.synchronize()
+        outs[name] = bufs
+        assert ctx.poll_status() == 0
+    assert ctx_o.kernel_variant("decode").startswith("small_step") == (small_step == "1")
+    for s in range(w.steps):
+        assert torch.equal(outs["overlapped"][s], outs["serial"][s]), s
+    inst = list(range(w.instances))
+    for a, b in zip(ctx_o.export_state(inst), ctx_s.export_state(inst)):
+        assert a["t"] == b["t"]
+        for key in ("pos", "acc", "K", "V", "psi", "H", "z"):
+            assert np.array_equal(a[key], b[key]), key
+    ctx_o.close(); ctx_s.close()
+
+
 def test_captured_step_replays_with_grouped_query_heads():
     test_captured_step_replays_like_direct_calls(3, group=4)
 
