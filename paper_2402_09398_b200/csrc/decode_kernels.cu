@@ -991,6 +991,7 @@ __global__ void __launch_bounds__(SS_THREADS) small_step_kernel(const __grid_con
 template <int R, int G, bool kCaptured>
 __global__ void __launch_bounds__(DEC_THREADS) decode_group_rows_kernel(DecParams p) {
   extern __shared__ float dsm[];
+  pdl_launch_dependents();                         // the next step's feature-map kernel may come up while this one runs
   const int Ns = p.Np + 4;
   float* s_sc = dsm;                               // [G][Np + 4] scores, then e^{s - m_g}
   float* s_red = s_sc + G * Ns;                    // [G][DEC_RG][128] partial numerators
@@ -1132,6 +1133,7 @@ constexpr int kMmaRed = DEC_THREADS / 32 + 1;   // partial numerators per head i
 template <int R, int G, bool kCaptured>
 __global__ void __launch_bounds__(DEC_THREADS) decode_group_mma_kernel(DecParams p) {
   extern __shared__ float dsm[];
+  pdl_launch_dependents();                         // the next step's feature-map kernel may come up while this one runs
   const int Ns = p.Np + 4;
   float* s_sc = dsm;                               // [G][Np + 4] scores, then e^{s - m_g}
   float* s_red = s_sc + G * Ns;                    // [G][kMmaRed][128] partial numerators: one row per warp, one for the new pair
@@ -1334,6 +1336,7 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_group_loop_kernel(DecParam
   constexpr int RGN = DEC_THREADS / LPR;           // row groups
   constexpr int GC = kLoopHeads;
   extern __shared__ float dsm[];
+  pdl_launch_dependents();
   const int Ns = p.Np + 4;
   float* s_e = dsm;                                // [GC][Ns] scores of this pass's heads, then e^{s - m_g}
   float* s_ps = s_e + GC * Ns;                     // [Ns] sum over all heads of their probabilities

@@ -196,7 +196,7 @@ __global__ void __launch_bounds__(FL_THREADS, 1) feature_tc_kernel(
   tc_fence_before_sync();
   __syncthreads();
   tc_fence_after_sync();
-  pdl_launch_dependents();
+  if (!gm.late_inputs) pdl_launch_dependents();   // else by the producer thread, behind its wait for the kernels before
   const uint32_t tmem = sh->tmem_base;
   const uint32_t d2col = 2u * (uint32_t)npad;
   volatile int* abortp = &sh->abort;
@@ -714,10 +714,11 @@ int launch_feature_tc(less_ctx* c, const FmParams& p_in, cudaStream_t s) {
   gm.per_head = (d.G + 1) * gm.ntile;
   gm.kv0 = p.lh0;
   gm.items = p.nlh * gm.per_head;
-  // Every decode CTA of a step resident at once (the regime of the small-batch kernel's overlap): the next
-  // step's feature kernel may then start while this step's decode kernel finishes.  With more instances its
-  // waiting CTAs would only take multiprocessors from the decode kernel's later waves.
-  gm.late_inputs = (d.B <= 8 && c->pdl && !c->profile && d.I <= 8 * c->sms && !c->head_counters) ? 1 : 0;
+  // The kernel is launched as a programmatic dependent of the kernel before it in the stream - the decode
+  // kernel of the step before, typically, which lets its dependents go when it starts: the CTAs come up on
+  // multiprocessors as that kernel drains from them (they need most of a multiprocessor's shared memory, so
+  // they never displace its CTAs) and fetch their first weights meanwhile.
+  gm.late_inputs = (c->pdl && !c->profile && !c->head_counters) ? 1 : 0;
   const size_t fixed = ft_fixed_smem(d, gm.npad);
   int ns = (int)((FT_SMEM_LIMIT - fixed) / FT_STAGE_BYTES);
   gm.nstage = ns > FT_MAX_STAGES ? FT_MAX_STAGES : ns;
@@ -808,15 +809,22 @@ int launch_feature_tc(less_ctx* c, const FmParams& p_in, cudaStream_t s) {
     if (nt == 4) return launch_small<16, 4>(c, p, gm, tq, tk, tw1a, tw1b, sm, grid, s);
     return launch_small<16, 8>(c, p, gm, tq, tk, tw1a, tw1b, sm, grid, s);
   }
-  if (d.R == 8) {
-    if (cudaFuncSetAttribute(feature_tc_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-      return fail_cuda("shared memory opt-in of feature_tc_kernel");
-    feature_tc_kernel<8><<<grid, FL_THREADS, smem, s>>>(tq, tk, tw1a, tw1b, p, gm, c->a.status);
-  } else {
-    if (cudaFuncSetAttribute(feature_tc_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-      return fail_cuda("shared memory opt-in of feature_tc_kernel");
-    feature_tc_kernel<16><<<grid, FL_THREADS, smem, s>>>(tq, tk, tw1a, tw1b, p, gm, c->a.status);
-  }
+  auto kern = d.R == 8 ? feature_tc_kernel<8> : feature_tc_kernel<16>;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+    return fail_cuda("shared memory opt-in of feature_tc_kernel");
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(FL_THREADS);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = gm.late_inputs ? 1 : 0;
+  int32_t* status = c->a.status;
+  if (cudaLaunchKernelEx(&cfg, kern, tq, tk, tw1a, tw1b, p, gm, status) != cudaSuccess)
+    return fail_cuda("launch of feature_tc_kernel");
   return check_launch("feature_tc_kernel");
 }
 
