@@ -18,6 +18,9 @@
  *   - The library allocates no device memory: the caller provides one arena
  *     (less_arena_bytes) that the context carves up and owns until destroy.
  *   - Weight buffers and the arena are BORROWED for the context's lifetime.
+ *     The weights must not change while the context exists: a decode step may fetch them before the work
+ *     enqueued ahead of it on its stream has finished (its kernels are programmatic dependent launches; everything
+ *     else a step reads - its inputs, the arena - it reads only once that work is complete).
  *   - less_prefill / less_decode_step are asynchronous on the given stream;
  *     their inputs must stay valid until the stream reaches the call.
  *   - A context is not thread-safe.
