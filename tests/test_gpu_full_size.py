@@ -273,3 +273,42 @@ def test_parallel_form_long_sequences_sampled_rows():
         assert err <= harness.OUT_TOL
     ctx.close()
     torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("cfg,kw", [(2, {}), (4, {}), (3, dict(batch=16)), (3, dict(batch=16, heads=4, group=8))])
+def test_back_to_back_steps_at_full_size_equal_serialised_ones(cfg, kw, monkeypatch):
+    """24 steps with nothing between them, where a step's feature-map kernel comes up while the step before is
+    still finishing, against a context that launches every kernel the ordinary way: every output and the
+    sampled final state bit for bit."""
+    monkeypatch.setenv("LESS_SMALL_STEP", "0")
+    w = wl.CONFIGS[cfg].with_(**kw) if kw else wl.CONFIGS[cfg]
+    from paper_2402_09398_b200 import binding
+    W = wl.make_weights(w, DEV)
+    ctx_o = binding.from_workload(w, W, DEV, max_prefill_layers=4)
+    monkeypatch.setenv("LESS_NO_OVERLAP", "1")
+    ctx_s = binding.from_workload(w, W, DEV, max_prefill_layers=4)
+    monkeypatch.delenv("LESS_NO_OVERLAP")
+    for l0 in range(0, w.layers, 4):
+        Q, K, V = wl.make_prompt(w, l0, 4, DEV)
+        ctx_o.prefill(Q, K, V, l0)
+        ctx_s.prefill(Q, K, V, l0)
+    del Q, K, V
+    steps = 24
+    inputs = [wl.make_decode_inputs(w, s, DEV) for s in range(steps)]
+    torch.cuda.synchronize()
+    outs = []
+    for ctx in (ctx_o, ctx_s):
+        bufs = [torch.empty(inputs[0][0].shape, dtype=torch.float32, device=DEV) for _ in range(steps)]
+        for s in range(steps):
+            ctx.decode_step(*inputs[s], out=bufs[s])
+        torch.cuda.synchronize()
+        assert ctx.poll_status() == 0
+        outs.append(bufs)
+    for s in range(steps):
+        assert torch.equal(outs[0][s], outs[1][s]), s
+    inst = list(range(0, w.instances, max(1, w.instances // 64)))
+    for a, b in zip(ctx_o.export_state(inst), ctx_s.export_state(inst)):
+        for key in ("pos", "acc", "K", "V", "psi", "H", "z"):
+            assert np.array_equal(a[key], b[key]), key
+    ctx_o.close(); ctx_s.close()
+
